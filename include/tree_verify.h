@@ -1,0 +1,163 @@
+/*
+ * tree_verify.h -- C ABI of the tree-verification library for recurrent
+ * linear-attention layers (gated linear attention and the gated delta rule).
+ *
+ * What it computes.  A hybrid model keeps, per request, layer and state head,
+ * one committed state S_pre.  A drafter proposes a token tree of T nodes with
+ * parent map pi (nodes indexed parent before child; pi(i) = -1 marks a child
+ * of the virtual root whose state is S_pre).  Every node i carries
+ * q_i, k_i (dk), v_i (dv), a decay gate alpha_i > 0 (the paper's gamma_i) and,
+ * for the delta rule, a write gate beta_i.  Sequential execution along a
+ * root-to-node path applies (Section II-B Eq. 1; Section IV-A Table II,
+ * "Sequential rule")
+ *
+ *     S~_i = alpha_i S_pi(i),   u_i = beta_i (v_i - S~_i^T k_i)   [delta]
+ *                               u_i = v_i                         [gated]
+ *     S_i  = S~_i + k_i u_i^T,  o_i = S_i^T q_i.
+ *
+ * tv_tree_verify returns o_i (and optionally u_i) for ALL nodes in one pass
+ * from the single immutable S_pre, without forming any per-node state
+ * (Section IV-A Theorem 1, Eq. 2, with Lemmas 1-3).  tv_commit_path then
+ * writes the one state that must persist, the state at the end of the accepted
+ * root-to-node path (Section IV-D Eq. 10).
+ *
+ * Memory layout (all tensors dense, row-major, innermost index last):
+ *     S_pre, S_new : float  [L][B][H][dv][dk]   (the serving cache layout
+ *                    "[H, dv, dk]" of Section IV-D, i.e. the transpose of the
+ *                    paper's S in R^{dk x dv})
+ *     q, k         : float or bf16 [L][B][H][T][dk]
+ *     v            : float or bf16 [L][B][H][T][dv]
+ *     alpha, beta  : float  [L][B][H][T]
+ *     O, U         : float  [L][B][H][T][dv]
+ * L = number of recurrent layers handled by one call (independent problems
+ * that share the trees and the accepted nodes).  Pointers marked "dev" are
+ * device pointers on the current CUDA device, 16-byte aligned; "host" are
+ * ordinary host pointers.  The caller owns every tensor and the stream; the
+ * library owns tv_tree objects only.
+ *
+ * Every function returns TV_OK (0) or a negative tv_status.  Nothing throws,
+ * aborts or prints.  Arguments are validated on the host before any launch.
+ * Preconditions that cannot be checked on the host: all inputs finite,
+ * alpha > 0.
+ */
+#ifndef TREE_VERIFY_H_
+#define TREE_VERIFY_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define TV_MAX_NODES 128   /* T <= 128: ancestor sets are 128-bit masks   */
+#define TV_MAX_DIM   128   /* dk, dv <= 128, multiples of 4               */
+
+typedef enum tv_status {
+  TV_OK = 0,
+  TV_ERR_BAD_ARG = -1,        /* null / misaligned pointer, size out of range   */
+  TV_ERR_INVALID_TREE = -2,   /* parent[i] >= i or parent[i] < -1               */
+  TV_ERR_UNSUPPORTED = -3,    /* shape outside what the kernels cover           */
+  TV_ERR_CUDA = -4,           /* a CUDA runtime call failed (tv_last_cuda_error)*/
+  TV_ERR_NOT_UPLOADED = -5,   /* tree metadata not on the device yet            */
+  TV_ERR_DEVICE_TIMEOUT = -6, /* a bounded device-side wait ran out             */
+  TV_ERR_NOMEM = -7
+} tv_status;
+
+enum { TV_GATED = 0, TV_GATED_DELTA = 1 };  /* update rule                      */
+enum { TV_F32 = 0, TV_BF16 = 1 };           /* dtype of q, k, v                 */
+enum { TV_IMPL_AUTO = 0, TV_IMPL_SIMT = 1, TV_IMPL_TC = 2 }; /* kernel choice   */
+
+typedef struct tv_tree tv_tree;             /* opaque, library-owned            */
+
+typedef struct tv_dims {
+  int32_t L, B, H, T, dk, dv;
+  int32_t rule;        /* TV_GATED / TV_GATED_DELTA                             */
+  int32_t qkv_dtype;   /* TV_F32 / TV_BF16                                      */
+  int32_t impl;        /* TV_IMPL_AUTO picks the tensor-core kernel when the
+                          shape allows it (bf16, dk = dv = 128) and the SIMT
+                          fp32 kernel otherwise                                 */
+} tv_dims;
+
+const char* tv_strerror(int status);
+int tv_version(void);
+/* cudaError_t value of the last failed CUDA call on this thread (0 if none). */
+int tv_last_cuda_error(void);
+
+/* ---- tree metadata (Section IV-A Table II: Anc(i), d, M^-; Section IV-C
+ * "Round-level topology preprocessing": built once per request and round,
+ * reused by every layer and head, in fixed buffers) -------------------------
+ *
+ * tv_tree_build: host only, no CUDA call.  parent is host int32
+ * [n_trees][n], -1 <= parent[t][i] < i, 1 <= n <= TV_MAX_NODES.  Produces, per
+ * node, the strict-ancestor set as a 128-bit mask (bit j&63 of word j>>6 set
+ * iff j in Anc(i): row i of M^-), depth[i] = |Anc(i)| (0 for a root child) and
+ * per tree max_depth = d.  *out is owned by the library until tv_tree_free.
+ * Returns TV_ERR_INVALID_TREE (and leaves *out NULL) for a malformed parent
+ * array.                                                                      */
+int tv_tree_build(const int32_t* parent /*host*/, int32_t n_trees, int32_t n,
+                  tv_tree** out);
+/* Same sizes, new topology, no allocation (fixed buffers across rounds).      */
+int tv_tree_rebuild(tv_tree* tree, const int32_t* parent /*host*/);
+/* Copy metadata out (host): anc [n_trees][n][2], depth [n_trees][n],
+ * max_depth [n_trees].  Any output pointer may be NULL.                       */
+int tv_tree_meta(const tv_tree* tree, uint64_t* anc, int32_t* depth,
+                 int32_t* max_depth);
+/* n_trees, n and the maximum depth over all trees.                            */
+int tv_tree_info(const tv_tree* tree, int32_t* n_trees, int32_t* n,
+                 int32_t* max_depth_all);
+/* Accepted-path indices (Section IV-D: P(a) = Anc(a) + {a}, topological
+ * order).  accepted is host int32 [n_req]; request r uses tree r (tree 0 when
+ * n_trees == 1); accepted[r] = -1 means no draft token accepted (len 0).
+ * path is host int32 [n_req][path_stride], path_stride >= max_depth_all + 1,
+ * unused entries set to -1; len is host int32 [n_req].                        */
+int tv_tree_path(const tv_tree* tree, const int32_t* accepted, int32_t n_req,
+                 int32_t* path, int32_t path_stride, int32_t* len);
+/* Copy the metadata to the current device on `stream` (a cudaStream_t).  The
+ * first call allocates the device mirror and a pinned staging block; later
+ * calls (after tv_tree_rebuild) only copy.  The copy is asynchronous; kernels
+ * launched later on the same stream see it.                                   */
+int tv_tree_upload(tv_tree* tree, void* stream);
+int tv_tree_free(tv_tree* tree);
+
+/* ---- verification (Section IV-A Theorem 1, Eq. 2; Eq. 4; Lemma 2 Eq. 5) ----
+ *
+ * For every layer, request, head and node i:
+ *     O[i] = P_i S_pre^T q_i + sum_{j in Anc(i)+{i}} (P_i/P_j)(q_i.k_j) u_j,
+ * P_i = prod of alpha over Anc(i)+{i}; u_j = v_j (TV_GATED) or the solution of
+ * the ancestor-masked system (I+G)U = R of Lemma 2 (TV_GATED_DELTA).
+ * tree must hold 1 tree (shared by the batch) or B trees, with n == T, and be
+ * uploaded.  S_pre is read only.  beta may be NULL for TV_GATED.  U may be
+ * NULL; when given it receives the correction rows u_i (for TV_GATED a copy of
+ * v widened to float).  One asynchronous launch sequence on `stream`; no
+ * allocation, no host synchronisation.                                        */
+int tv_tree_verify(const tv_tree* tree, const tv_dims* dims,
+                   const float* S_pre /*dev*/,
+                   const void* q /*dev*/, const void* k /*dev*/, const void* v /*dev*/,
+                   const float* alpha /*dev*/, const float* beta /*dev or NULL*/,
+                   float* O /*dev*/, float* U /*dev or NULL*/,
+                   void* stream);
+
+/* ---- accepted-path commit (Section IV-D Eq. 10; Lemma 1 Eq. 3) -------------
+ *
+ *     S_new = P_a S_pre + sum_{j in P(a)} (P_a/P_j) k_j u_j^T   (stored [dv][dk])
+ * for the accepted terminal node a = accepted[b] of each request, all L layers
+ * and all heads in one launch.  accepted is a DEVICE int32 [B] (it comes from
+ * the sampler), each value in [-1, T); -1 leaves the slot unchanged (nothing
+ * is read or written when S_new == S_pre, S_pre is copied otherwise).  Values
+ * outside [-1, T) are treated as -1.  U: the corrections written by
+ * tv_tree_verify, or NULL -- then TV_GATED uses u_j = v_j and TV_GATED_DELTA
+ * re-derives u_j along the accepted path from S_pre (needs dk in {64,128}).
+ * S_new may alias S_pre exactly (in place) or not overlap it at all.          */
+int tv_commit_path(const tv_tree* tree, const tv_dims* dims,
+                   const int32_t* accepted /*dev [B]*/,
+                   const float* S_pre /*dev*/,
+                   const void* k /*dev*/, const void* v /*dev*/,
+                   const float* alpha /*dev*/, const float* beta /*dev or NULL*/,
+                   const float* U /*dev or NULL*/,
+                   float* S_new /*dev*/,
+                   void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TREE_VERIFY_H_ */

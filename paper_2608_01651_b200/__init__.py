@@ -1,0 +1,231 @@
+"""Python binding of libtreeverify (argument marshalling only).
+
+Every function here has the name of the C entry point it forwards to
+(``include/tree_verify.h``) minus the ``tv_`` prefix; all arithmetic runs in
+the CUDA kernels of the shared library.  PyTorch supplies device memory and
+the current stream, nothing else.  If the shared library has not been built
+the first call raises: there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+
+GATED, DELTA = 0, 1
+F32, BF16 = 0, 1
+IMPL_AUTO, IMPL_SIMT, IMPL_TC = 0, 1, 2
+MAX_NODES = 128
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libtreeverify.so")
+_lib = None
+
+
+class TreeVerifyError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = lib().tv_strerror(status).decode()
+        if status == -4:
+            msg += f" [cudaError {lib().tv_last_cuda_error()}]"
+        super().__init__(f"{where}: {msg} ({status})")
+
+
+class _Dims(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in
+                ("L", "B", "H", "T", "dk", "dv", "rule", "qkv_dtype", "impl")]
+
+
+def lib() -> ctypes.CDLL:
+    """Load libtreeverify.so; raises if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2608_01651_b200.build` "
+            "(there is no non-CUDA fallback)")
+    L = ctypes.CDLL(LIB_PATH)
+    vp, i32, p = ctypes.c_void_p, ctypes.c_int32, ctypes.POINTER
+    L.tv_strerror.restype = ctypes.c_char_p
+    L.tv_strerror.argtypes = [ctypes.c_int]
+    L.tv_version.restype = ctypes.c_int
+    L.tv_last_cuda_error.restype = ctypes.c_int
+    L.tv_tree_build.argtypes = [vp, i32, i32, p(vp)]
+    L.tv_tree_rebuild.argtypes = [vp, vp]
+    L.tv_tree_meta.argtypes = [vp, vp, vp, vp]
+    L.tv_tree_info.argtypes = [vp, p(i32), p(i32), p(i32)]
+    L.tv_tree_path.argtypes = [vp, vp, i32, vp, i32, vp]
+    L.tv_tree_upload.argtypes = [vp, vp]
+    L.tv_tree_free.argtypes = [vp]
+    L.tv_tree_verify.argtypes = [vp, p(_Dims)] + [vp] * 9
+    L.tv_commit_path.argtypes = [vp, p(_Dims)] + [vp] * 9
+    for name in ("tv_tree_build", "tv_tree_rebuild", "tv_tree_meta", "tv_tree_info", "tv_tree_path",
+                 "tv_tree_upload", "tv_tree_free", "tv_tree_verify", "tv_commit_path"):
+        getattr(L, name).restype = ctypes.c_int
+    _lib = L
+    return L
+
+
+def _check(st: int, where: str):
+    if st != 0:
+        raise TreeVerifyError(st, where)
+
+
+def _np_i32(a) -> np.ndarray:
+    return np.ascontiguousarray(np.asarray(a), dtype=np.int32)
+
+
+class Tree:
+    """Handle of a library-owned ``tv_tree`` (metadata of 1 or B proposal trees)."""
+
+    def __init__(self, handle, n_trees, n):
+        self._h = handle
+        self.n_trees = n_trees
+        self.n = n
+
+    def rebuild(self, parent):
+        par = _np_i32(parent).reshape(self.n_trees, self.n)
+        _check(lib().tv_tree_rebuild(self._h, par.ctypes.data), "tv_tree_rebuild")
+        return self
+
+    def meta(self):
+        """(anc uint64 [n_trees,n,2], depth int32 [n_trees,n], max_depth int32 [n_trees])."""
+        anc = np.zeros((self.n_trees, self.n, 2), dtype=np.uint64)
+        depth = np.zeros((self.n_trees, self.n), dtype=np.int32)
+        md = np.zeros(self.n_trees, dtype=np.int32)
+        _check(lib().tv_tree_meta(self._h, anc.ctypes.data, depth.ctypes.data, md.ctypes.data),
+               "tv_tree_meta")
+        return anc, depth, md
+
+    @property
+    def max_depth(self) -> int:
+        md = ctypes.c_int32()
+        _check(lib().tv_tree_info(self._h, None, None, ctypes.byref(md)), "tv_tree_info")
+        return md.value
+
+    def path(self, accepted):
+        """(path int32 [n_req, max_depth+1] padded with -1, len int32 [n_req])."""
+        acc = _np_i32(accepted).reshape(-1)
+        stride = self.max_depth + 1
+        path = np.zeros((len(acc), stride), dtype=np.int32)
+        ln = np.zeros(len(acc), dtype=np.int32)
+        _check(lib().tv_tree_path(self._h, acc.ctypes.data, len(acc), path.ctypes.data, stride,
+                                  ln.ctypes.data), "tv_tree_path")
+        return path, ln
+
+    def upload(self, stream=None):
+        _check(lib().tv_tree_upload(self._h, _stream_ptr(stream)), "tv_tree_upload")
+        return self
+
+    def free(self):
+        if self._h:
+            lib().tv_tree_free(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.free()
+        except Exception:
+            pass
+
+
+def tree_build(parent) -> Tree:
+    """``tv_tree_build``: parent int32 [n] or [n_trees, n], -1 <= parent[i] < i."""
+    par = _np_i32(parent)
+    if par.ndim == 1:
+        par = par[None]
+    n_trees, n = par.shape
+    h = ctypes.c_void_p()
+    _check(lib().tv_tree_build(par.ctypes.data, n_trees, n, ctypes.byref(h)), "tv_tree_build")
+    return Tree(h, n_trees, n)
+
+
+def _stream_ptr(stream):
+    if stream is None:
+        import torch
+        if torch.cuda.is_available():
+            return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+        return ctypes.c_void_p(0)
+    if hasattr(stream, "cuda_stream"):
+        return ctypes.c_void_p(stream.cuda_stream)
+    return ctypes.c_void_p(int(stream))
+
+
+def _ptr(t):
+    return ctypes.c_void_p(0 if t is None else t.data_ptr())
+
+
+def _dims(S_pre, k, v, rule, impl) -> _Dims:
+    import torch
+    if S_pre.dim() == 4:
+        L = 1
+        B, H, dv, dk = S_pre.shape
+    elif S_pre.dim() == 5:
+        L, B, H, dv, dk = S_pre.shape
+    else:
+        raise ValueError("S_pre must be [B,H,dv,dk] or [L,B,H,dv,dk]")
+    T = k.shape[-2]
+    if k.dtype == torch.bfloat16:
+        dt = BF16
+    elif k.dtype == torch.float32:
+        dt = F32
+    else:
+        raise ValueError("q/k/v must be float32 or bfloat16")
+    return _Dims(L, B, H, T, dk, dv, rule, dt, impl)
+
+
+def _require(t, name, dtype=None):
+    if t is None:
+        return
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError(f"{name} must be a contiguous CUDA tensor")
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError(f"{name} must be {dtype}")
+
+
+def tree_verify(tree: Tree, S_pre, q, k, v, alpha, beta=None, *, rule=GATED, O=None, U=None,
+                want_U=False, impl=IMPL_AUTO, stream=None):
+    """``tv_tree_verify``: per-node outputs O (and corrections U) for all nodes.
+
+    Tensors are CUDA, contiguous, in the layout of ``tree_verify.h``.  Returns
+    ``O`` or ``(O, U)``.
+    """
+    import torch
+    for t, n in ((S_pre, "S_pre"), (alpha, "alpha"), (beta, "beta")):
+        _require(t, n, torch.float32)
+    for t, n in ((q, "q"), (k, "k"), (v, "v")):
+        _require(t, n, k.dtype)
+    d = _dims(S_pre, k, v, rule, impl)
+    if O is None:
+        O = torch.empty(*v.shape[:-1], d.dv, device=v.device, dtype=torch.float32)
+    if U is None and want_U:
+        U = torch.empty_like(O)
+    _require(O, "O", torch.float32)
+    _require(U, "U", torch.float32)
+    _check(lib().tv_tree_verify(tree._h, ctypes.byref(d), _ptr(S_pre), _ptr(q), _ptr(k), _ptr(v),
+                                _ptr(alpha), _ptr(beta), _ptr(O), _ptr(U), _stream_ptr(stream)),
+           "tv_tree_verify")
+    return (O, U) if U is not None else O
+
+
+def commit_path(tree: Tree, accepted, S_pre, k, v, alpha, beta=None, *, rule=GATED, U=None,
+                S_new=None, stream=None):
+    """``tv_commit_path``: write the state at the end of the accepted path.
+
+    ``accepted`` is a CUDA int32 tensor [B].  ``S_new=None`` commits in place
+    and returns ``S_pre``.
+    """
+    import torch
+    _require(accepted, "accepted", torch.int32)
+    for t, n in ((S_pre, "S_pre"), (alpha, "alpha"), (beta, "beta"), (U, "U"), (S_new, "S_new")):
+        _require(t, n, torch.float32)
+    for t, n in ((k, "k"), (v, "v")):
+        _require(t, n, k.dtype)
+    d = _dims(S_pre, k, v, rule, IMPL_AUTO)
+    out = S_pre if S_new is None else S_new
+    _check(lib().tv_commit_path(tree._h, ctypes.byref(d), _ptr(accepted), _ptr(S_pre), _ptr(k),
+                                _ptr(v), _ptr(alpha), _ptr(beta), _ptr(U), _ptr(out),
+                                _stream_ptr(stream)), "tv_commit_path")
+    return out

@@ -1,0 +1,269 @@
+// C ABI of libtreeverify: host-side tree metadata, argument validation, dispatch.
+#include <cstring>
+#include <new>
+
+#include "tv_internal.h"
+
+static thread_local int g_last_cuda_error = 0;
+void tv_set_cuda_error(cudaError_t e) { g_last_cuda_error = (int)e; }
+
+#define TV_API __attribute__((visibility("default")))
+
+extern "C" {
+
+TV_API const char* tv_strerror(int s) {
+  switch (s) {
+    case TV_OK: return "ok";
+    case TV_ERR_BAD_ARG: return "bad argument (null or misaligned pointer, or size out of range)";
+    case TV_ERR_INVALID_TREE: return "invalid tree (need -1 <= parent[i] < i)";
+    case TV_ERR_UNSUPPORTED: return "unsupported shape, dtype or rule";
+    case TV_ERR_CUDA: return "CUDA runtime error (see tv_last_cuda_error)";
+    case TV_ERR_NOT_UPLOADED: return "tree metadata not uploaded to the device";
+    case TV_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait ran out";
+    case TV_ERR_NOMEM: return "out of memory";
+    default: return "unknown status";
+  }
+}
+
+TV_API int tv_version(void) { return 100; }
+TV_API int tv_last_cuda_error(void) { return g_last_cuda_error; }
+
+// ---------------------------------------------------------------------------
+// Tree metadata.  Nodes are indexed parent before child, so one forward sweep
+// gives every strict-ancestor set: anc(i) = anc(parent(i)) + {parent(i)}.
+// ---------------------------------------------------------------------------
+static int fill_tree(tv_tree* t, const int32_t* parent) {
+  const int n = t->n;
+  int md_all = 0;
+  for (int tr = 0; tr < t->n_trees; ++tr) {
+    const int32_t* par = parent + (size_t)tr * n;
+    for (int i = 0; i < n; ++i)
+      if (par[i] < -1 || par[i] >= i) return TV_ERR_INVALID_TREE;
+  }
+  for (int tr = 0; tr < t->n_trees; ++tr) {
+    const int32_t* par = parent + (size_t)tr * n;
+    uint64_t* anc = t->anc.data() + (size_t)tr * n * 2;
+    int32_t* dep = t->depth.data() + (size_t)tr * n;
+    int md = 0;
+    for (int i = 0; i < n; ++i) {
+      const int p = par[i];
+      uint64_t w0 = 0, w1 = 0;
+      int d = 0;
+      if (p >= 0) {
+        w0 = anc[2 * p];
+        w1 = anc[2 * p + 1];
+        if (p < 64) w0 |= (uint64_t)1 << p; else w1 |= (uint64_t)1 << (p - 64);
+        d = dep[p] + 1;
+      }
+      anc[2 * i] = w0;
+      anc[2 * i + 1] = w1;
+      dep[i] = d;
+      if (d > md) md = d;
+    }
+    t->max_depth[tr] = md;
+    if (md > md_all) md_all = md;
+  }
+  std::memcpy(t->parent.data(), parent, sizeof(int32_t) * (size_t)t->n_trees * n);
+  t->max_depth_all = md_all;
+  t->uploaded = false;
+  return TV_OK;
+}
+
+TV_API int tv_tree_build(const int32_t* parent, int32_t n_trees, int32_t n, tv_tree** out) {
+  if (!out) return TV_ERR_BAD_ARG;
+  *out = nullptr;
+  if (!parent || n_trees < 1 || n < 1) return TV_ERR_BAD_ARG;
+  if (n > TV_MAX_NODES) return TV_ERR_UNSUPPORTED;
+  tv_tree* t = new (std::nothrow) tv_tree();
+  if (!t) return TV_ERR_NOMEM;
+  t->n_trees = n_trees;
+  t->n = n;
+  try {
+    t->parent.resize((size_t)n_trees * n);
+    t->depth.resize((size_t)n_trees * n);
+    t->max_depth.resize(n_trees);
+    t->anc.resize((size_t)n_trees * n * 2);
+  } catch (...) {
+    delete t;
+    return TV_ERR_NOMEM;
+  }
+  int st = fill_tree(t, parent);
+  if (st != TV_OK) {
+    delete t;
+    return st;
+  }
+  *out = t;
+  return TV_OK;
+}
+
+TV_API int tv_tree_rebuild(tv_tree* t, const int32_t* parent) {
+  if (!t || !parent) return TV_ERR_BAD_ARG;
+  return fill_tree(t, parent);
+}
+
+TV_API int tv_tree_meta(const tv_tree* t, uint64_t* anc, int32_t* depth, int32_t* max_depth) {
+  if (!t) return TV_ERR_BAD_ARG;
+  if (anc) std::memcpy(anc, t->anc.data(), t->anc.size() * sizeof(uint64_t));
+  if (depth) std::memcpy(depth, t->depth.data(), t->depth.size() * sizeof(int32_t));
+  if (max_depth) std::memcpy(max_depth, t->max_depth.data(), t->max_depth.size() * sizeof(int32_t));
+  return TV_OK;
+}
+
+TV_API int tv_tree_info(const tv_tree* t, int32_t* n_trees, int32_t* n, int32_t* max_depth_all) {
+  if (!t) return TV_ERR_BAD_ARG;
+  if (n_trees) *n_trees = t->n_trees;
+  if (n) *n = t->n;
+  if (max_depth_all) *max_depth_all = t->max_depth_all;
+  return TV_OK;
+}
+
+TV_API int tv_tree_path(const tv_tree* t, const int32_t* accepted, int32_t n_req, int32_t* path,
+                 int32_t path_stride, int32_t* len) {
+  if (!t || !accepted || !path || !len || n_req < 0) return TV_ERR_BAD_ARG;
+  if (path_stride < t->max_depth_all + 1) return TV_ERR_BAD_ARG;
+  if (t->n_trees != 1 && n_req > t->n_trees) return TV_ERR_BAD_ARG;
+  for (int r = 0; r < n_req; ++r)
+    if (accepted[r] < -1 || accepted[r] >= t->n) return TV_ERR_BAD_ARG;
+  for (int r = 0; r < n_req; ++r) {
+    const int tr = t->n_trees == 1 ? 0 : r;
+    int32_t* row = path + (size_t)r * path_stride;
+    for (int s = 0; s < path_stride; ++s) row[s] = -1;
+    const int a = accepted[r];
+    if (a < 0) {
+      len[r] = 0;
+      continue;
+    }
+    // Indices grow along a root-to-node path, so the set bits of the ancestor
+    // mask in increasing order are the path in topological order.
+    const uint64_t* m = t->anc.data() + ((size_t)tr * t->n + a) * 2;
+    int c = 0;
+    for (int j = 0; j < t->n; ++j)
+      if ((m[j >> 6] >> (j & 63)) & 1) row[c++] = j;
+    row[c++] = a;
+    len[r] = c;
+  }
+  return TV_OK;
+}
+
+TV_API int tv_tree_upload(tv_tree* t, void* stream) {
+  if (!t) return TV_ERR_BAD_ARG;
+  const size_t nn = (size_t)t->n_trees * t->n;
+  const size_t anc_b = nn * 2 * sizeof(uint64_t), i32_b = nn * sizeof(int32_t);
+  const size_t total = anc_b + 2 * i32_b;
+  int dev = 0;
+  TV_CUDA_TRY(cudaGetDevice(&dev));
+  if (t->d_blob && (t->device != dev || t->blob_bytes != total)) return TV_ERR_BAD_ARG;
+  if (!t->d_blob) {
+    TV_CUDA_TRY(cudaMalloc(&t->d_blob, total));
+    cudaError_t e = cudaMallocHost(&t->h_stage, total);
+    if (e != cudaSuccess) {
+      cudaFree(t->d_blob);
+      t->d_blob = nullptr;
+      tv_set_cuda_error(e);
+      return TV_ERR_CUDA;
+    }
+    t->blob_bytes = total;
+    t->device = dev;
+    char* base = (char*)t->d_blob;
+    t->d_anc = (const uint64_t*)base;
+    t->d_depth = (const int32_t*)(base + anc_b);
+    t->d_parent = (const int32_t*)(base + anc_b + i32_b);
+  }
+  cudaStream_t s = (cudaStream_t)stream;
+  // The staging block may still be in flight from an earlier upload.
+  TV_CUDA_TRY(cudaStreamSynchronize(s));
+  char* hs = (char*)t->h_stage;
+  std::memcpy(hs, t->anc.data(), anc_b);
+  std::memcpy(hs + anc_b, t->depth.data(), i32_b);
+  std::memcpy(hs + anc_b + i32_b, t->parent.data(), i32_b);
+  TV_CUDA_TRY(cudaMemcpyAsync(t->d_blob, t->h_stage, total, cudaMemcpyHostToDevice, s));
+  t->uploaded = true;
+  return TV_OK;
+}
+
+TV_API int tv_tree_free(tv_tree* t) {
+  if (!t) return TV_OK;
+  if (t->d_blob) cudaFree(t->d_blob);
+  if (t->h_stage) cudaFreeHost(t->h_stage);
+  delete t;
+  return TV_OK;
+}
+
+// ---------------------------------------------------------------------------
+// Validation shared by verify and commit.
+// ---------------------------------------------------------------------------
+static bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
+
+static int check_common(const tv_tree* t, const tv_dims* d) {
+  if (!t || !d) return TV_ERR_BAD_ARG;
+  if (d->L < 1 || d->B < 1 || d->H < 1 || d->T < 1 || d->dk < 1 || d->dv < 1) return TV_ERR_BAD_ARG;
+  if (d->rule != TV_GATED && d->rule != TV_GATED_DELTA) return TV_ERR_BAD_ARG;
+  if (d->qkv_dtype != TV_F32 && d->qkv_dtype != TV_BF16) return TV_ERR_BAD_ARG;
+  if (d->T > TV_MAX_NODES || d->dk > TV_MAX_DIM || d->dv > TV_MAX_DIM) return TV_ERR_UNSUPPORTED;
+  if ((d->dk & 3) || (d->dv & 3)) return TV_ERR_UNSUPPORTED;
+  if (d->qkv_dtype == TV_BF16 && ((d->dk & 7) || (d->dv & 7))) return TV_ERR_UNSUPPORTED;
+  if (t->n != d->T) return TV_ERR_BAD_ARG;
+  if (t->n_trees != 1 && t->n_trees != d->B) return TV_ERR_BAD_ARG;
+  if ((int64_t)d->L * d->B * d->H > 0x7fffffffLL) return TV_ERR_UNSUPPORTED;
+  if (!t->uploaded) return TV_ERR_NOT_UPLOADED;
+  return TV_OK;
+}
+
+static TreeDev tree_dev(const tv_tree* t) {
+  TreeDev td;
+  td.anc = t->d_anc;
+  td.depth = t->d_depth;
+  td.parent = t->d_parent;
+  td.n_trees = t->n_trees;
+  td.max_depth_all = t->max_depth_all;
+  return td;
+}
+
+TV_API int tv_tree_verify(const tv_tree* tree, const tv_dims* d, const float* S_pre, const void* q,
+                   const void* k, const void* v, const float* alpha, const float* beta, float* O,
+                   float* U, void* stream) {
+  int st = check_common(tree, d);
+  if (st != TV_OK) return st;
+  if (!S_pre || !q || !k || !v || !alpha || !O) return TV_ERR_BAD_ARG;
+  if (d->rule == TV_GATED_DELTA && !beta) return TV_ERR_BAD_ARG;
+  if (!aligned16(S_pre) || !aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(O) ||
+      !aligned16(U) || ((uintptr_t)alpha & 3) || ((uintptr_t)beta & 3))
+    return TV_ERR_BAD_ARG;
+  if (d->impl != TV_IMPL_AUTO && d->impl != TV_IMPL_SIMT && d->impl != TV_IMPL_TC) return TV_ERR_BAD_ARG;
+  VerifyArgs a;
+  a.tree = tree_dev(tree);
+  a.L = d->L; a.B = d->B; a.H = d->H; a.T = d->T; a.dk = d->dk; a.dv = d->dv;
+  a.rule = d->rule; a.bf16 = d->qkv_dtype == TV_BF16;
+  a.S_pre = S_pre; a.q = q; a.k = k; a.v = v; a.alpha = alpha; a.beta = beta; a.O = O; a.U = U;
+  if (d->impl == TV_IMPL_TC) return TV_ERR_UNSUPPORTED;
+  return tv_launch_verify_simt(a, (cudaStream_t)stream);
+}
+
+TV_API int tv_commit_path(const tv_tree* tree, const tv_dims* d, const int32_t* accepted,
+                   const float* S_pre, const void* k, const void* v, const float* alpha,
+                   const float* beta, const float* U, float* S_new, void* stream) {
+  int st = check_common(tree, d);
+  if (st != TV_OK) return st;
+  if (!accepted || !S_pre || !k || !alpha || !S_new) return TV_ERR_BAD_ARG;
+  if (!U && !v) return TV_ERR_BAD_ARG;
+  if (d->rule == TV_GATED_DELTA && !U && !beta) return TV_ERR_BAD_ARG;
+  if (!aligned16(S_pre) || !aligned16(S_new) || !aligned16(k) || !aligned16(v) || !aligned16(U) ||
+      ((uintptr_t)alpha & 3) || ((uintptr_t)beta & 3) || ((uintptr_t)accepted & 3))
+    return TV_ERR_BAD_ARG;
+  if (S_new != S_pre) {
+    const size_t bytes = sizeof(float) * (size_t)d->L * d->B * d->H * d->dv * d->dk;
+    const char* a0 = (const char*)S_pre;
+    const char* b0 = (const char*)S_new;
+    if (a0 < b0 + bytes && b0 < a0 + bytes) return TV_ERR_BAD_ARG;  // partial overlap
+  }
+  if (d->rule == TV_GATED_DELTA && !U && d->dk != 64 && d->dk != 128) return TV_ERR_UNSUPPORTED;
+  CommitArgs a;
+  a.tree = tree_dev(tree);
+  a.L = d->L; a.B = d->B; a.H = d->H; a.T = d->T; a.dk = d->dk; a.dv = d->dv;
+  a.rule = d->rule; a.bf16 = d->qkv_dtype == TV_BF16;
+  a.accepted = accepted; a.S_pre = S_pre; a.k = k; a.v = v; a.alpha = alpha; a.beta = beta;
+  a.U = U; a.S_new = S_new;
+  return tv_launch_commit(a, (cudaStream_t)stream);
+}
+
+}  // extern "C"

@@ -1,0 +1,269 @@
+// Accepted-path commit (Section IV-D Eq. 10; Lemma 1 Eq. 3).
+//
+//   S_new[v][k] = P_a S_pre[v][k] + sum_{j in P(a)} (P_a/P_j) u_j[v] k_j[k]
+//
+// One CTA streams one (layer, request, head) state of dv x dk floats through
+// registers exactly once: 16-byte loads issued back to back, the rank-len
+// update applied from shared memory, 16-byte stores.  HBM-bound: 8 dk dv bytes
+// per state against (1 + len) FMAs per element.
+//
+// The accepted path needs no parent walk: node indices grow along a
+// root-to-node path, so the set bits of the 128-bit ancestor mask of a, plus a
+// itself, are the path in topological order.
+#include <cuda_bf16.h>
+
+#include "tv_internal.h"
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kPathChunk = 16;  // path rows staged in shared memory at a time
+constexpr int kMaxVec = 16;     // float4 per thread: dk*dv <= 16384
+
+template <bool BF16>
+__device__ __forceinline__ float load_elem(const void* base, size_t idx) {
+  if (BF16) return __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(base)[idx]);
+  return reinterpret_cast<const float*>(base)[idx];
+}
+
+struct PathInfo {
+  int len;
+};
+
+// Fills path_s[0..len) (topological order), w_s[p] = P_a / P_path[p] and *Pa_s.
+__device__ __forceinline__ int build_path(const TreeDev& tree, int tb, int T, int acc,
+                                          const float* alpha_row, int* path_s, float* w_s,
+                                          float* Pa_s) {
+  const uint64_t* m = tree.anc + ((size_t)tb * T + acc) * 2;
+  uint64_t m0 = m[0], m1 = m[1];
+  if (acc < 64) m0 |= 1ull << acc; else m1 |= 1ull << (acc - 64);
+  const int len = __popcll(m0) + __popcll(m1);
+  const int t = threadIdx.x;
+  if (t < 128) {
+    const uint64_t w = t < 64 ? m0 : m1;
+    const int bit = t & 63;
+    if ((w >> bit) & 1) {
+      int pos = __popcll(w & ((1ull << bit) - 1));
+      if (t >= 64) pos += __popcll(m0);
+      path_s[pos] = t;
+    }
+  }
+  __syncthreads();
+  if (t == 0) {
+    float w = 1.f;
+    for (int p = len - 1; p >= 0; --p) {
+      w_s[p] = w;
+      w *= alpha_row[path_s[p]];
+    }
+    *Pa_s = w;
+  }
+  __syncthreads();
+  return len;
+}
+
+// Commit from given correction rows u_j: U (float) when a.U != NULL, else v.
+template <bool BF16>
+__global__ void __launch_bounds__(kThreads) commit_factored_kernel(CommitArgs a) {
+  __shared__ int path_s[TV_MAX_NODES];
+  __shared__ float w_s[TV_MAX_NODES];
+  __shared__ float Pa_s;
+  __shared__ __align__(16) float k_s[kPathChunk][TV_MAX_DIM];
+  __shared__ float cu_s[kPathChunk][TV_MAX_DIM];
+
+  const int item = blockIdx.x;
+  const int b = (item / a.H) % a.B;
+  const int tid = threadIdx.x;
+  const int dk = a.dk, dv = a.dv, T = a.T;
+  const int n4 = dv * dk / 4;
+  const size_t sbase = (size_t)item * dv * dk;
+  const float4* src = reinterpret_cast<const float4*>(a.S_pre + sbase);
+  float4* dst = reinterpret_cast<float4*>(a.S_new + sbase);
+
+  int acc = a.accepted[b];
+  if (acc >= T) acc = -1;
+  if (acc < 0) {
+    if (a.S_new != a.S_pre)
+      for (int i = tid; i < n4; i += kThreads) dst[i] = src[i];
+    return;
+  }
+  const int tb = a.tree.n_trees == 1 ? 0 : b;
+  const size_t node0 = (size_t)item * T;  // first node row of this (l, b, h)
+  const int len = build_path(a.tree, tb, T, acc, a.alpha + node0, path_s, w_s, &Pa_s);
+  const float Pa = Pa_s;
+
+  float4 s[kMaxVec];
+#pragma unroll
+  for (int e = 0; e < kMaxVec; ++e) {
+    const int i = tid + e * kThreads;
+    if (i < n4) s[e] = src[i];
+  }
+#pragma unroll
+  for (int e = 0; e < kMaxVec; ++e) {
+    s[e].x *= Pa; s[e].y *= Pa; s[e].z *= Pa; s[e].w *= Pa;
+  }
+  const int dk4 = dk >> 2;
+  for (int c0 = 0; c0 < len; c0 += kPathChunk) {
+    const int nc = min(kPathChunk, len - c0);
+    __syncthreads();
+    for (int i = tid; i < nc * dk; i += kThreads) {
+      const int p = i / dk, kk = i - p * dk;
+      k_s[p][kk] = load_elem<BF16>(a.k, (node0 + path_s[c0 + p]) * dk + kk);
+    }
+    for (int i = tid; i < nc * dv; i += kThreads) {
+      const int p = i / dv, vv = i - p * dv;
+      const size_t idx = (node0 + path_s[c0 + p]) * dv + vv;
+      const float u = a.U ? a.U[idx] : load_elem<BF16>(a.v, idx);
+      cu_s[p][vv] = w_s[c0 + p] * u;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int e = 0; e < kMaxVec; ++e) {
+      const int i = tid + e * kThreads;
+      if (i < n4) {
+        const int row = i / dk4, c4 = i - row * dk4;
+        for (int p = 0; p < nc; ++p) {
+          const float cu = cu_s[p][row];
+          const float4 kv = *reinterpret_cast<const float4*>(&k_s[p][c4 * 4]);
+          s[e].x = fmaf(cu, kv.x, s[e].x);
+          s[e].y = fmaf(cu, kv.y, s[e].y);
+          s[e].z = fmaf(cu, kv.z, s[e].z);
+          s[e].w = fmaf(cu, kv.w, s[e].w);
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int e = 0; e < kMaxVec; ++e) {
+    const int i = tid + e * kThreads;
+    if (i < n4) dst[i] = s[e];
+  }
+}
+
+// Delta rule without stored corrections: every row v of the [dv][dk] state
+// evolves independently along the accepted path,
+//   s <- alpha_j s;  u = beta_j (v_j[v] - s . k_j);  s <- s + u k_j,
+// which is the sequential rule restricted to one value channel.  A warp owns a
+// row at a time (NPL consecutive floats per lane, dk = 32 NPL); the dot
+// product is a shuffle reduction.
+template <bool BF16, int NPL>
+__global__ void __launch_bounds__(kThreads) commit_delta_rows_kernel(CommitArgs a) {
+  constexpr int DK = 32 * NPL;
+  constexpr int kRowsPerWarp = TV_MAX_DIM / (kThreads / 32);  // 16
+  __shared__ int path_s[TV_MAX_NODES];
+  __shared__ float w_s[TV_MAX_NODES];
+  __shared__ float Pa_s;
+  __shared__ __align__(16) float k_s[kPathChunk][DK];
+  __shared__ float v_s[kPathChunk][TV_MAX_DIM];
+  __shared__ float al_s[kPathChunk], be_s[kPathChunk];
+
+  const int item = blockIdx.x;
+  const int b = (item / a.H) % a.B;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int dv = a.dv, T = a.T;
+  const size_t sbase = (size_t)item * dv * DK;
+  const int n4 = dv * DK / 4;
+
+  int acc = a.accepted[b];
+  if (acc >= T) acc = -1;
+  if (acc < 0) {
+    if (a.S_new != a.S_pre) {
+      const float4* src = reinterpret_cast<const float4*>(a.S_pre + sbase);
+      float4* dst = reinterpret_cast<float4*>(a.S_new + sbase);
+      for (int i = tid; i < n4; i += kThreads) dst[i] = src[i];
+    }
+    return;
+  }
+  const int tb = a.tree.n_trees == 1 ? 0 : b;
+  const size_t node0 = (size_t)item * T;
+  const int len = build_path(a.tree, tb, T, acc, a.alpha + node0, path_s, w_s, &Pa_s);
+
+  float s[kRowsPerWarp][NPL];
+#pragma unroll
+  for (int r = 0; r < kRowsPerWarp; ++r) {
+    const int row = warp + r * (kThreads / 32);
+    if (row < dv) {
+      const float* p = a.S_pre + sbase + (size_t)row * DK + lane * NPL;
+      if (NPL == 4) {
+        const float4 t = *reinterpret_cast<const float4*>(p);
+        s[r][0] = t.x; s[r][1] = t.y; s[r][2 % NPL] = t.z; s[r][3 % NPL] = t.w;
+      } else {
+        const float2 t = *reinterpret_cast<const float2*>(p);
+        s[r][0] = t.x; s[r][1] = t.y;
+      }
+    }
+  }
+  for (int c0 = 0; c0 < len; c0 += kPathChunk) {
+    const int nc = min(kPathChunk, len - c0);
+    __syncthreads();
+    for (int i = tid; i < nc * DK; i += kThreads) {
+      const int p = i / DK, kk = i - p * DK;
+      k_s[p][kk] = load_elem<BF16>(a.k, (node0 + path_s[c0 + p]) * DK + kk);
+    }
+    for (int i = tid; i < nc * dv; i += kThreads) {
+      const int p = i / dv, vv = i - p * dv;
+      v_s[p][vv] = load_elem<BF16>(a.v, (node0 + path_s[c0 + p]) * dv + vv);
+    }
+    if (tid < nc) {
+      al_s[tid] = a.alpha[node0 + path_s[c0 + tid]];
+      be_s[tid] = a.beta[node0 + path_s[c0 + tid]];
+    }
+    __syncthreads();
+    for (int p = 0; p < nc; ++p) {
+      float kr[NPL];
+#pragma unroll
+      for (int x = 0; x < NPL; ++x) kr[x] = k_s[p][lane * NPL + x];
+      const float al = al_s[p], be = be_s[p];
+#pragma unroll
+      for (int r = 0; r < kRowsPerWarp; ++r) {
+        const int row = warp + r * (kThreads / 32);
+        if (row < dv) {
+          float dot = 0.f;
+#pragma unroll
+          for (int x = 0; x < NPL; ++x) {
+            s[r][x] *= al;
+            dot = fmaf(s[r][x], kr[x], dot);
+          }
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+          const float u = be * (v_s[p][row] - dot);
+#pragma unroll
+          for (int x = 0; x < NPL; ++x) s[r][x] = fmaf(u, kr[x], s[r][x]);
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < kRowsPerWarp; ++r) {
+    const int row = warp + r * (kThreads / 32);
+    if (row < dv) {
+      float* p = a.S_new + sbase + (size_t)row * DK + lane * NPL;
+      if (NPL == 4) {
+        *reinterpret_cast<float4*>(p) = make_float4(s[r][0], s[r][1], s[r][2 % NPL], s[r][3 % NPL]);
+      } else {
+        *reinterpret_cast<float2*>(p) = make_float2(s[r][0], s[r][1]);
+      }
+    }
+  }
+}
+
+}  // namespace
+
+int tv_launch_commit(const CommitArgs& a, cudaStream_t stream) {
+  const int items = a.L * a.B * a.H;
+  if ((size_t)a.dk * a.dv > (size_t)kMaxVec * kThreads * 4) return TV_ERR_UNSUPPORTED;
+  const bool recompute = a.rule == TV_GATED_DELTA && a.U == nullptr;
+  if (!recompute) {
+    if (a.bf16) commit_factored_kernel<true><<<items, kThreads, 0, stream>>>(a);
+    else commit_factored_kernel<false><<<items, kThreads, 0, stream>>>(a);
+  } else if (a.dk == 128) {
+    if (a.bf16) commit_delta_rows_kernel<true, 4><<<items, kThreads, 0, stream>>>(a);
+    else commit_delta_rows_kernel<false, 4><<<items, kThreads, 0, stream>>>(a);
+  } else if (a.dk == 64) {
+    if (a.bf16) commit_delta_rows_kernel<true, 2><<<items, kThreads, 0, stream>>>(a);
+    else commit_delta_rows_kernel<false, 2><<<items, kThreads, 0, stream>>>(a);
+  } else {
+    return TV_ERR_UNSUPPORTED;
+  }
+  TV_CUDA_TRY(cudaGetLastError());
+  return TV_OK;
+}

@@ -1,0 +1,138 @@
+"""Parity of the CUDA path against the fp64 oracle, through the C ABI.
+
+Bar: tree metadata bit-exact (test_tree_host.py); outputs, corrections and
+committed states within the workload's tolerance -- max over nodes of the
+relative L2 error of each output vector, max over (request, head) of the
+relative Frobenius error of each state: 1e-5 for all-fp32 operands, 2e-3 for
+bf16 q/k/v with fp32 state and accumulation.
+"""
+import numpy as np
+import pytest
+import torch
+
+import paper_2608_01651_b200 as tv
+from paper_2608_01651_b200 import inputs
+from tests import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+IMPLS = [tv.IMPL_SIMT]
+
+
+def _run(wl, parents, accepted, tens, tol, items=None, **kw):
+    O, U, Sn, tree = pu.gpu_round(wl, parents, accepted, tens, **kw)
+    ver, com = pu.oracle_round(wl, parents, accepted, tens, items=items)
+    eO, eU, eS = pu.compare(wl, O, U, Sn, ver, com)
+    assert np.isfinite(O).all() and np.isfinite(Sn).all()
+    assert eO <= tol, f"O rel-L2 {eO:.3e} > {tol}"
+    assert eU <= tol, f"U rel-L2 {eU:.3e} > {tol}"
+    assert eS <= tol, f"S_new rel-Fro {eS:.3e} > {tol}"
+    return eO, eU, eS
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("name", ["c1", "c2", "c3", "c4"])
+def test_workload_full(name, impl):
+    wl = inputs.workload(name)
+    parents, accepted = inputs.make_trees(wl)
+    tens = inputs.make_tensors(wl)
+    _run(wl, parents, accepted, tens, wl.tol, impl=impl)
+    if wl.rule == inputs.DELTA:
+        _run(wl, parents, accepted, tens, wl.tol, impl=impl, commit_with_U=True, in_place=True)
+    else:
+        _run(wl, parents, accepted, tens, wl.tol, impl=impl, in_place=True)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_c5_full_size_sampled(impl):
+    """Full batch and tree size of the throughput workload, 2 layers in one
+    call; the oracle checks a seeded sample of (layer, request, head) items."""
+    wl = inputs.workload("c5", L=2)
+    parents, accepted = inputs.make_trees(wl)
+    tens = [inputs.make_tensors(wl, layer=l) for l in range(wl.L)]
+    stacked = {k: (None if tens[0][k] is None else torch.stack([t[k] for t in tens]))
+               for k in tens[0]}
+    O, U, Sn, tree = pu.gpu_round(wl, parents, accepted, stacked, impl=impl, want_U=False)
+    rng = np.random.default_rng(5)
+    for layer in range(wl.L):
+        items = [(int(rng.integers(wl.B)), int(rng.integers(wl.H))) for _ in range(12)]
+        items += [(0, 0), (wl.B - 1, wl.H - 1)]
+        ver, com = pu.oracle_round(wl, parents, accepted, stacked, items=items, layer=layer)
+        eO, _, eS = pu.compare(wl, O, None, Sn, ver, com, layer=layer)
+        assert eO <= wl.tol and eS <= wl.tol, (eO, eS)
+
+
+EDGE = [
+    # T, dk, dv, B, H, tree, shared tree
+    (1, 64, 64, 2, 2, "chain", False),
+    (2, 128, 128, 1, 3, "chain", False),
+    (15, 128, 128, 2, 2, "binary", True),
+    (63, 128, 128, 2, 2, "frontier", False),
+    (65, 128, 128, 1, 2, "frontier", False),
+    (127, 128, 128, 1, 2, "spine", False),
+    (128, 128, 128, 1, 2, "chain", False),     # maximum depth 127
+    (128, 128, 128, 2, 1, "star", False),      # depth 0 everywhere
+    (40, 64, 128, 2, 2, "frontier", False),    # dk != dv
+    (40, 128, 64, 2, 2, "frontier", False),
+    (33, 32, 96, 1, 2, "frontier", True),
+]
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("rule", [inputs.GATED, inputs.DELTA])
+@pytest.mark.parametrize("dtype", [inputs.BF16, inputs.F32])
+@pytest.mark.parametrize("case", EDGE)
+def test_edge_shapes(case, dtype, rule, impl):
+    T, dk, dv, B, H, kind, shared = case
+    wl = inputs.workload("c2", T=T, dk=dk, dv=dv, B=B, H=H, rule=rule, qkv_dtype=dtype,
+                         tree="frontier" if kind == "star" else kind, seed=100 + T)
+    parents, accepted = inputs.make_trees(wl, per_request=not shared)
+    if kind == "star":
+        parents[:] = -1
+        accepted[:] = T - 1
+    accepted[0] = -1 if T % 2 else accepted[0]          # some requests accept nothing
+    tens = inputs.make_tensors(wl)
+    tol = 1e-5 if dtype == inputs.F32 else 2e-3
+    if kind == "chain" and T == 128:
+        tol = 5e-5 if dtype == inputs.F32 else 2e-3     # 128 sequential fp32 steps
+    recompute_ok = rule == inputs.GATED or dk in (64, 128)
+    if recompute_ok:
+        _run(wl, parents, accepted, tens, tol, impl=impl)
+    _run(wl, parents, accepted, tens, tol, impl=impl, commit_with_U=True, in_place=True)
+
+
+def test_all_rejected_leaves_state_untouched():
+    wl = inputs.workload("c2", B=2, H=2, T=20)
+    parents, accepted = inputs.make_trees(wl)
+    accepted[:] = -1
+    tens = inputs.make_tensors(wl)
+    O, U, Sn, _ = pu.gpu_round(wl, parents, accepted, tens, in_place=True)
+    assert np.array_equal(Sn, tens["S_pre"].double().numpy())
+    O, U, Sn, _ = pu.gpu_round(wl, parents, accepted, tens, in_place=False)
+    assert np.array_equal(Sn, tens["S_pre"].double().numpy())
+
+
+def test_argument_errors_on_device():
+    wl = inputs.workload("c2", B=1, H=1, T=8)
+    parents, accepted = inputs.make_trees(wl)
+    tens = {k: (None if v is None else v.cuda()) for k, v in inputs.make_tensors(wl).items()}
+    tree = tv.tree_build(parents)
+    with pytest.raises(tv.TreeVerifyError) as e:
+        tv.tree_verify(tree, tens["S_pre"], tens["q"], tens["k"], tens["v"], tens["alpha"])
+    assert e.value.status == -5                      # not uploaded
+    tree.upload()
+    with pytest.raises(tv.TreeVerifyError) as e:     # delta rule without beta
+        tv.tree_verify(tree, tens["S_pre"], tens["q"], tens["k"], tens["v"], tens["alpha"], rule=tv.DELTA)
+    assert e.value.status == -1
+    mis = torch.empty(8 * 128 + 1, device="cuda", dtype=torch.float32)[1:].view(1, 1, 8, 128)
+    with pytest.raises(tv.TreeVerifyError) as e:     # misaligned output
+        tv.tree_verify(tree, tens["S_pre"], tens["q"], tens["k"], tens["v"], tens["alpha"], O=mis)
+    assert e.value.status == -1
+    S = tens["S_pre"]
+    flat = torch.empty(S.numel() + 64, device="cuda", dtype=torch.float32)
+    acc = torch.zeros(1, device="cuda", dtype=torch.int32)
+    with pytest.raises(tv.TreeVerifyError) as e:     # partial overlap of S_pre and S_new
+        tv.commit_path(tree, acc, flat[:S.numel()].view_as(S), tens["k"], tens["v"], tens["alpha"],
+                       S_new=flat[64:].view_as(S))
+    assert e.value.status == -1
+    torch.cuda.synchronize()
