@@ -157,6 +157,26 @@ int tv_commit_path(const tv_tree* tree, const tv_dims* dims,
                    float* S_new /*dev*/,
                    void* stream);
 
+/* ---- host-buffer round ------------------------------------------------------
+ * The whole hot path (tv_tree_build -> tv_tree_verify -> tv_commit_path, i.e.
+ * Section IV-C topology step, Theorem 1 and Eq. 10 in sequence) for callers
+ * whose tensors live in HOST memory (pinned memory makes the copies
+ * asynchronous).  A session owns device copies sized for `dims` (allocated
+ * once by tv_session_create on the current device; n_trees is 1 or B).
+ * tv_session_round copies parent/accepted/S_pre/q/k/v/alpha/beta to the device
+ * on `stream`, verifies, commits in place on the device copy (the delta rule
+ * commits from the corrections U that verify wrote), copies O and S_new back
+ * and synchronises the stream before returning.  All pointers are host
+ * pointers in the layouts above; beta may be NULL for TV_GATED.               */
+typedef struct tv_session tv_session;
+int tv_session_create(const tv_dims* dims, int32_t n_trees, tv_session** out);
+int tv_session_round(tv_session* s, const int32_t* parent /*[n_trees][T]*/,
+                     const int32_t* accepted /*[B]*/, const float* S_pre,
+                     const void* q, const void* k, const void* v,
+                     const float* alpha, const float* beta,
+                     float* O, float* S_new, void* stream);
+int tv_session_free(tv_session* s);
+
 #ifdef __cplusplus
 }
 #endif

@@ -61,6 +61,11 @@ def lib() -> ctypes.CDLL:
     L.tv_tree_free.argtypes = [vp]
     L.tv_tree_verify.argtypes = [vp, p(_Dims)] + [vp] * 9
     L.tv_commit_path.argtypes = [vp, p(_Dims)] + [vp] * 9
+    L.tv_session_create.argtypes = [p(_Dims), i32, p(vp)]
+    L.tv_session_round.argtypes = [vp] + [vp] * 11
+    L.tv_session_free.argtypes = [vp]
+    for name in ("tv_session_create", "tv_session_round", "tv_session_free"):
+        getattr(L, name).restype = ctypes.c_int
     for name in ("tv_tree_build", "tv_tree_rebuild", "tv_tree_meta", "tv_tree_info", "tv_tree_path",
                  "tv_tree_upload", "tv_tree_free", "tv_tree_verify", "tv_commit_path"):
         getattr(L, name).restype = ctypes.c_int
@@ -229,3 +234,39 @@ def commit_path(tree: Tree, accepted, S_pre, k, v, alpha, beta=None, *, rule=GAT
                                 _ptr(v), _ptr(alpha), _ptr(beta), _ptr(U), _ptr(out),
                                 _stream_ptr(stream)), "tv_commit_path")
     return out
+
+
+class Session:
+    """Handle of a ``tv_session``: device copies for host-buffer rounds."""
+
+    def __init__(self, L, B, H, T, dk, dv, *, rule=GATED, qkv_dtype=BF16, n_trees=None,
+                 impl=IMPL_AUTO):
+        self.dims = _Dims(L, B, H, T, dk, dv, rule, qkv_dtype, impl)
+        self._h = ctypes.c_void_p()
+        _check(lib().tv_session_create(ctypes.byref(self.dims), B if n_trees is None else n_trees,
+                                       ctypes.byref(self._h)), "tv_session_create")
+
+    def round(self, parent, accepted, S_pre, q, k, v, alpha, beta, O, S_new, stream=None):
+        """``tv_session_round``: all arguments are HOST tensors/arrays (torch CPU
+        tensors, ideally pinned; parent/accepted int32 numpy arrays)."""
+        par = _np_i32(parent)
+        acc = _np_i32(accepted)
+        _check(lib().tv_session_round(self._h, par.ctypes.data, acc.ctypes.data, _ptr(S_pre), _ptr(q),
+                                      _ptr(k), _ptr(v), _ptr(alpha), _ptr(beta), _ptr(O), _ptr(S_new),
+                                      _stream_ptr(stream)), "tv_session_round")
+        return O, S_new
+
+    def free(self):
+        if self._h:
+            lib().tv_session_free(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.free()
+        except Exception:
+            pass
+
+
+def session_create(*args, **kw) -> Session:
+    return Session(*args, **kw)
