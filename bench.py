@@ -1,0 +1,434 @@
+#!/usr/bin/env python
+"""Benchmark of the tree-verification hot path on B200.
+
+A step is one pass of the whole path over one batch of synthetic trees:
+tree_build (host metadata + upload) -> tree_verify for every layer ->
+commit_path over all layers, through the C ABI of libtreeverify.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c3]
+    python bench.py --impl reference ...      # the fp64 CPU oracle, timed
+
+Prints ONE JSON line on rank 0.  ``value`` = verified tree nodes per second
+per recurrent layer (B*T*L nodes per step over the step time, all ranks
+summed), inputs resident in HBM; ``e2e`` = the same with HOST buffers through
+tv_session_round (copies inside the timed region); ``roofline`` = achieved
+algorithmic HBM GB/s of the verify kernel against the measured copy peak;
+``cpu_baseline`` = the oracle on a bounded sample on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2608_01651_b200 import inputs  # noqa: E402
+
+FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 8000.0
+L2_BYTES = 126 * 2 ** 20
+
+DESCR = {
+    "c1": "c1: B1 H4 T15 dk=dv=64 gated, f32 q/k/v, f32 state",
+    "c2": "c2: B1 H16 T63 dk=dv=128 gated, bf16 q/k/v, f32 state",
+    "c3": "c3: B32 H32 T64 dk=dv=128 gated, bf16 q/k/v, f32 state, draft-style level trees",
+    "c4": "c4: B16 H32 T64 dk=dv=128 gated delta rule, bf16 q/k/v, f32 state",
+    "c5": "c5: B128 H32 T128 dk=dv=128 gated, bf16 q/k/v, f32 state, 48 layers",
+}
+
+
+# --------------------------------------------------------------------------
+# Algorithmic bytes (what the method must move; the design doc states the formulae)
+# --------------------------------------------------------------------------
+def verify_bytes_per_layer(wl, with_U: bool) -> int:
+    eb = 2 if wl.qkv_dtype == inputs.BF16 else 4
+    per = 4 * wl.dk * wl.dv + eb * wl.T * (2 * wl.dk + wl.dv) + 4 * wl.T + 4 * wl.T * wl.dv
+    if wl.rule == inputs.DELTA:
+        per += 4 * wl.T
+    if with_U:
+        per += 4 * wl.T * wl.dv
+    return per * wl.B * wl.H
+
+
+def commit_bytes_per_layer(wl, acc_len: np.ndarray, with_U: bool) -> int:
+    """In-place commit: requests that accept nothing move no bytes."""
+    eb = 2 if wl.qkv_dtype == inputs.BF16 else 4
+    tot = 0
+    for ln in acc_len:
+        if ln > 0:
+            tot += wl.H * (8 * wl.dk * wl.dv + ln * (eb * wl.dk + (4 if with_U else eb) * wl.dv))
+    return tot
+
+
+def accepted_lengths(parents, accepted):
+    out = []
+    for b, a in enumerate(accepted):
+        d = inputs.node_depths(parents[b if parents.shape[0] > 1 else 0])
+        out.append(0 if a < 0 else int(d[a]) + 1)
+    return np.array(out)
+
+
+def _jsonable(o):
+    return o.item() if hasattr(o, "item") else str(o)
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+# --------------------------------------------------------------------------
+# Clock sampling during the timed region
+# --------------------------------------------------------------------------
+class ClockSampler:
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        try:
+            self.p = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-i", str(index), "-lms", "100"], stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self) -> dict:
+        if self.p is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx = [], []
+        reasons = set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.f.read().splitlines():
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        self.f.close()
+        os.unlink(self.f.name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None,
+                "sm_max_mhz": float(max(mx)) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# --------------------------------------------------------------------------
+# CPU baseline: the oracle, as it stands, on a bounded sample
+# --------------------------------------------------------------------------
+def oracle_sample(wl, parents, accepted, tens_cpu, budget_s: float, max_items: int):
+    """Time the oracle (verify + commit) on (b,h) items until the budget is spent.
+    Returns (nodes/s per layer, items, seconds, threads)."""
+    from oracle import tree_oracle as orc
+    try:
+        from threadpoolctl import threadpool_limits
+        ctx = threadpool_limits(limits=1)
+        threads = 1
+    except Exception:
+        import contextlib
+        ctx = contextlib.nullcontext()
+        threads = os.cpu_count() or 1
+    f = {k: inputs.to_f64(v) for k, v in tens_cpu.items()}
+    done = 0
+    t0 = time.perf_counter()
+    with ctx:
+        for b in range(wl.B):
+            for h in range(wl.H):
+                orc.verify_batch(f["S_pre"], f["q"], f["k"], f["v"], f["alpha"], f["beta"], parents,
+                                 wl.rule_name, memo=True, items=[(b, h)])
+                orc.commit_batch(f["S_pre"], f["k"], f["v"], f["alpha"], f["beta"], parents, accepted,
+                                 wl.rule_name, items=[(b, h)])
+                done += 1
+                if time.perf_counter() - t0 > budget_s or done >= max_items:
+                    break
+            else:
+                continue
+            break
+    dt = time.perf_counter() - t0
+    # one "node" of the metric is a tree node through all H heads of a layer
+    return done * wl.T / wl.H / dt, done, dt, threads
+
+
+def slice_request(wl, tens, nb):
+    return {k: (None if v is None else v[:nb].contiguous()) for k, v in tens.items()}
+
+
+def run_reference(args, wl, rank, world):
+    """--impl reference: the CPU oracle timed on bounded samples."""
+    if rank != 0:
+        return
+    parents, accepted = inputs.make_trees(wl)
+    nb = min(wl.B, 2)
+    small = inputs.workload(wl.name, B=nb, L=1)
+    tens = inputs.make_tensors(small)
+    items_per_step = max(1, min(nb * wl.H, args.ref_items))
+    vals = []
+    threads = 1
+    for s in range(args.warmup + args.steps):
+        v, done, dt, threads = oracle_sample(small, parents[:nb] if parents.shape[0] > 1 else parents,
+                                             accepted[:nb], tens, 1e9, items_per_step)
+        if s >= args.warmup:
+            vals.append((v, dt))
+    value = float(np.mean([v for v, _ in vals]))
+    ms = float(np.mean([dt for _, dt in vals]) * 1e3)
+    sample = (f"{items_per_step} (request, head) items of {DESCR[wl.name]} per step: memoised fp64 walk of "
+              f"all {wl.T} nodes plus commit")
+    line = {
+        "impl": "reference", "metric": "verified_tree_nodes_per_s_per_layer", "value": value,
+        "unit": "nodes/s", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": DESCR[wl.name], "sample": sample},
+        "cpu_baseline": {"value": value, "unit": "nodes/s", "cores": threads, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": "nodes/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line, default=_jsonable), flush=True)
+
+
+# --------------------------------------------------------------------------
+# The CUDA path
+# --------------------------------------------------------------------------
+def run_ours(args, wl, rank, world, local_rank):
+    import paper_2608_01651_b200 as tv
+    import torch.distributed as dist
+
+    tv.lib()  # fail loudly if the library is missing
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    wl = inputs.workload(wl.name, seed=wl.seed + 101 * rank, L=args.layers or wl.L)
+    parents, accepted = inputs.make_trees(wl)
+    acc_len = accepted_lengths(parents, accepted)
+    delta = wl.rule == inputs.DELTA
+    impl = {"auto": tv.IMPL_AUTO, "simt": tv.IMPL_SIMT, "tc": tv.IMPL_TC}[args.kernel]
+
+    # Input sets rotated between steps so that consecutive steps never find
+    # their inputs in L2: every set is larger than L2, or there are several.
+    eb = 2 if wl.qkv_dtype == inputs.BF16 else 4
+    set_bytes = wl.L * wl.B * wl.H * (4 * wl.dk * wl.dv + eb * wl.T * (2 * wl.dk + wl.dv) + 4 * wl.T * wl.dv)
+    n_sets = args.sets or max(2, min(8, int(np.ceil(4 * L2_BYTES / set_bytes))))
+    if set_bytes > 4 * L2_BYTES:
+        n_sets = args.sets or 1
+    sets = []
+    for s in range(n_sets):
+        layers = [inputs.make_tensors(wl, layer=s * wl.L + l, device=dev) for l in range(wl.L)]
+        st = {k: (None if layers[0][k] is None else torch.stack([x[k] for x in layers]))
+              for k in layers[0]}
+        del layers
+        st["O"] = torch.empty(wl.L, wl.B, wl.H, wl.T, wl.dv, device=dev, dtype=torch.float32)
+        st["U"] = torch.empty_like(st["O"]) if delta else None
+        sets.append(st)
+    acc_dev = torch.from_numpy(accepted).to(dev)
+    tree = tv.tree_build(parents)
+    stream = torch.cuda.current_stream()
+
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    kernel_events = []
+
+    def step(i, record):
+        st = sets[i % n_sets]
+        tree.rebuild(parents)
+        tree.upload(stream)
+        e0, e1, e2 = (ev(), ev(), ev()) if record else (None, None, None)
+        if record:
+            e0.record(stream)
+        for l in range(wl.L):
+            tv.tree_verify(tree, st["S_pre"][l], st["q"][l], st["k"][l], st["v"][l], st["alpha"][l],
+                           None if st["beta"] is None else st["beta"][l], rule=wl.rule,
+                           O=st["O"][l], U=None if st["U"] is None else st["U"][l], impl=impl,
+                           stream=stream)
+        if record:
+            e1.record(stream)
+        tv.commit_path(tree, acc_dev, st["S_pre"], st["k"], st["v"], st["alpha"], st["beta"],
+                       rule=wl.rule, U=st["U"], stream=stream)
+        if record:
+            e2.record(stream)
+            kernel_events.append((e0, e1, e2))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    for i in range(args.warmup):
+        step(i, False)
+    torch.cuda.synchronize()
+    barrier()
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    t_start, t_end = ev(), ev()
+    torch.cuda.synchronize()
+    t_start.record(stream)
+    for i in range(args.steps):
+        step(args.warmup + i, True)
+    t_end.record(stream)
+    torch.cuda.synchronize()
+    barrier()
+    clocks = sampler.stop() if sampler else None
+    total_ms = t_start.elapsed_time(t_end)
+    v_ms = float(np.mean([a.elapsed_time(b) for a, b, _ in kernel_events])) / wl.L
+    c_ms = float(np.mean([b.elapsed_time(c) for _, b, c in kernel_events]))
+
+    # ---- end to end with host buffers through tv_session_round -------------
+    e2e = None
+    e2e_L = 1 if wl.L > 4 else wl.L
+    if not args.no_e2e:
+        wl_e = inputs.workload(wl.name, seed=wl.seed, L=e2e_L)
+        host = [inputs.make_tensors(wl_e, layer=l) for l in range(e2e_L)]
+        hs = {k: (None if host[0][k] is None else torch.stack([x[k] for x in host]).pin_memory())
+              for k in host[0]}
+        hO = torch.empty(e2e_L, wl.B, wl.H, wl.T, wl.dv, dtype=torch.float32).pin_memory()
+        hS = torch.empty_like(hs["S_pre"]).pin_memory()
+        sess = tv.Session(e2e_L, wl.B, wl.H, wl.T, wl.dk, wl.dv, rule=wl.rule, qkv_dtype=wl.qkv_dtype,
+                          impl=impl)
+        n_e2e = max(3, min(args.steps, 10))
+        for _ in range(2):
+            sess.round(parents, accepted, hs["S_pre"], hs["q"], hs["k"], hs["v"], hs["alpha"], hs["beta"],
+                       hO, hS, stream)
+        torch.cuda.synchronize()
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(n_e2e):
+            sess.round(parents, accepted, hs["S_pre"], hs["q"], hs["k"], hs["v"], hs["alpha"], hs["beta"],
+                       hO, hS, stream)
+        torch.cuda.synchronize()
+        dt_e = (time.perf_counter() - t0) / n_e2e
+        h2d = sum(t.numel() * t.element_size() for k, t in hs.items() if t is not None) \
+            + parents.size * 24 + accepted.nbytes   # metadata blob: 16 B mask + depth + parent
+        d2h = hO.numel() * 4 + hS.numel() * 4
+        e2e = [dt_e, h2d, d2h, n_e2e]
+        sess.free()
+        del hs, hO, hS
+
+    # ---- max over ranks -----------------------------------------------------
+    if world > 1:
+        t = torch.tensor([total_ms, v_ms, c_ms, e2e[0] if e2e else 0.0], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, v_ms, c_ms, e2e_dt = [float(x) for x in t.tolist()]
+        if e2e:
+            e2e[0] = e2e_dt
+    if rank != 0:
+        return
+
+    ms_per_step = total_ms / args.steps
+    nodes_step = wl.B * wl.T * wl.L * world
+    value = nodes_step / (ms_per_step * 1e-3)
+    peak, peak_kind = measured_peak()
+    vbytes = verify_bytes_per_layer(wl, with_U=delta)
+    cbytes = commit_bytes_per_layer(wl, acc_len, with_U=delta) * wl.L
+    v_gbs = vbytes / (v_ms * 1e-3) / 1e9
+    c_gbs = cbytes / (c_ms * 1e-3) / 1e9 if c_ms > 0 else 0.0
+
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        nb = min(wl.B, 8)
+        small = inputs.workload(wl.name, B=nb, L=1, seed=wl.seed)
+        tens = inputs.make_tensors(small)
+        v, done, dt, threads = oracle_sample(small, parents[:nb] if parents.shape[0] > 1 else parents,
+                                             accepted[:nb], tens, args.cpu_budget, nb * wl.H)
+        cpu = {"value": v, "unit": "nodes/s", "cores": threads, "kind": "oracle",
+               "sample": f"{done} (request, head) items of the workload (memoised fp64 walk of all "
+                         f"{wl.T} nodes + commit), {dt:.1f} s"}
+
+    line = {
+        "metric": "verified_tree_nodes_per_s_per_layer",
+        "value": value, "unit": "nodes/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {
+            "workload": DESCR[wl.name], "layers_per_step": wl.L, "kernel": args.kernel,
+            "step": "tree_build(host)+upload, tree_verify per layer, commit_path over all layers (in place)",
+            "l2": f"{n_sets} rotating input set(s) of {set_bytes / 2**20:.0f} MiB each (L2 is 126 MiB)",
+            "trees": inputs.tree_stats(parents, accepted),
+        },
+        "verify": {"ms_per_layer": v_ms, "nodes_per_s_per_layer": wl.B * wl.T / (v_ms * 1e-3),
+                   "algorithmic_GBps": v_gbs, "frac_of_measured_copy": v_gbs / peak,
+                   "frac_of_nominal_8TBps": v_gbs / NOMINAL_HBM_GBS},
+        "commit": {"ms": c_ms, "algorithmic_GBps": c_gbs, "bytes": cbytes,
+                   "frac_of_measured_copy": c_gbs / peak, "frac_of_nominal_8TBps": c_gbs / NOMINAL_HBM_GBS},
+        "roofline": {"kernel": "tree_verify", "bound": "hbm", "achieved": v_gbs, "peak": peak,
+                     "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": v_gbs / peak,
+                     "traffic": args.traffic},
+        "cpu_baseline": cpu,
+        "e2e": None if e2e is None else {
+            "value": wl.B * wl.T * e2e_L * world / e2e[0], "unit": "nodes/s",
+            "h2d_bytes_per_step": int(e2e[1]), "d2h_bytes_per_step": int(e2e[2]),
+            "steps": e2e[3], "layers": e2e_L,
+            "call": "tv_session_round (pinned host buffers in, O and S_new out)"},
+        "gpu_launches": args.steps * (wl.L + 1),
+        "clocks": clocks,
+    }
+    print(json.dumps(line, default=_jsonable), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="c3", choices=sorted(DESCR))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--kernel", default="auto", choices=["auto", "simt", "tc"])
+    ap.add_argument("--layers", type=int, default=0, help="override layers per step")
+    ap.add_argument("--sets", type=int, default=0, help="override number of rotating input sets")
+    ap.add_argument("--cpu-budget", type=float, default=15.0)
+    ap.add_argument("--ref-items", type=int, default=8)
+    ap.add_argument("--traffic", type=float, default=None,
+                    help="ncu dram bytes per verify launch to echo into roofline.traffic")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    wl = inputs.workload(args.workload)
+
+    if args.impl == "reference":
+        run_reference(args, wl, rank, world)
+        return
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl")
+    try:
+        run_ours(args, wl, rank, world, local_rank)
+    finally:
+        if world > 1:
+            import torch.distributed as dist
+            dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -117,6 +117,11 @@ int tv_tree_path(const tv_tree* tree, const int32_t* accepted, int32_t n_req,
  * calls (after tv_tree_rebuild) only copy.  The copy is asynchronous; kernels
  * launched later on the same stream see it.                                   */
 int tv_tree_upload(tv_tree* tree, void* stream);
+/* Synchronises `stream` and reports whether any kernel launched with this tree
+ * since its last upload gave up on a bounded device-side wait (a TMA or tensor-
+ * core completion that never came): TV_OK or TV_ERR_DEVICE_TIMEOUT.  After a
+ * timeout the outputs of that launch are undefined; the context stays usable. */
+int tv_tree_device_status(tv_tree* tree, void* stream);
 int tv_tree_free(tv_tree* tree);
 
 /* ---- verification (Section IV-A Theorem 1, Eq. 2; Eq. 4; Lemma 2 Eq. 5) ----

@@ -59,6 +59,8 @@ def lib() -> ctypes.CDLL:
     L.tv_tree_path.argtypes = [vp, vp, i32, vp, i32, vp]
     L.tv_tree_upload.argtypes = [vp, vp]
     L.tv_tree_free.argtypes = [vp]
+    L.tv_tree_device_status.argtypes = [vp, vp]
+    L.tv_tree_device_status.restype = ctypes.c_int
     L.tv_tree_verify.argtypes = [vp, p(_Dims)] + [vp] * 9
     L.tv_commit_path.argtypes = [vp, p(_Dims)] + [vp] * 9
     L.tv_session_create.argtypes = [p(_Dims), i32, p(vp)]
@@ -123,6 +125,10 @@ class Tree:
     def upload(self, stream=None):
         _check(lib().tv_tree_upload(self._h, _stream_ptr(stream)), "tv_tree_upload")
         return self
+
+    def device_status(self, stream=None):
+        """``tv_tree_device_status``: synchronise and raise if a device wait timed out."""
+        _check(lib().tv_tree_device_status(self._h, _stream_ptr(stream)), "tv_tree_device_status")
 
     def free(self):
         if self._h:

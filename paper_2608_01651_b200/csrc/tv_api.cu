@@ -149,7 +149,8 @@ TV_API int tv_tree_upload(tv_tree* t, void* stream) {
   if (!t) return TV_ERR_BAD_ARG;
   const size_t nn = (size_t)t->n_trees * t->n;
   const size_t anc_b = nn * 2 * sizeof(uint64_t), i32_b = nn * sizeof(int32_t);
-  const size_t total = anc_b + 2 * i32_b;
+  const size_t meta_b = anc_b + 2 * i32_b;
+  const size_t total = ((meta_b + 15) & ~(size_t)15) + 16;  // + status word
   int dev = 0;
   TV_CUDA_TRY(cudaGetDevice(&dev));
   if (t->d_blob && (t->device != dev || t->blob_bytes != total)) return TV_ERR_BAD_ARG;
@@ -168,23 +169,38 @@ TV_API int tv_tree_upload(tv_tree* t, void* stream) {
     t->d_anc = (const uint64_t*)base;
     t->d_depth = (const int32_t*)(base + anc_b);
     t->d_parent = (const int32_t*)(base + anc_b + i32_b);
+    t->d_status = (int32_t*)(base + total - 16);
   }
   cudaStream_t s = (cudaStream_t)stream;
-  // The staging block may still be in flight from an earlier upload.
-  TV_CUDA_TRY(cudaStreamSynchronize(s));
+  // The staging block may still be in flight from an earlier upload: wait for
+  // that copy only, not for the stream.
+  if (t->staged) TV_CUDA_TRY(cudaEventSynchronize(t->staged));
+  else TV_CUDA_TRY(cudaEventCreateWithFlags(&t->staged, cudaEventDisableTiming));
   char* hs = (char*)t->h_stage;
   std::memcpy(hs, t->anc.data(), anc_b);
   std::memcpy(hs + anc_b, t->depth.data(), i32_b);
   std::memcpy(hs + anc_b + i32_b, t->parent.data(), i32_b);
+  std::memset(hs + total - 16, 0, 16);
   TV_CUDA_TRY(cudaMemcpyAsync(t->d_blob, t->h_stage, total, cudaMemcpyHostToDevice, s));
+  TV_CUDA_TRY(cudaEventRecord(t->staged, s));
   t->uploaded = true;
   return TV_OK;
+}
+
+TV_API int tv_tree_device_status(tv_tree* t, void* stream) {
+  if (!t) return TV_ERR_BAD_ARG;
+  if (!t->d_status) return TV_ERR_NOT_UPLOADED;
+  int32_t st = 0;
+  TV_CUDA_TRY(cudaMemcpyAsync(&st, t->d_status, sizeof(st), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+  TV_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+  return st == 0 ? TV_OK : TV_ERR_DEVICE_TIMEOUT;
 }
 
 TV_API int tv_tree_free(tv_tree* t) {
   if (!t) return TV_OK;
   if (t->d_blob) cudaFree(t->d_blob);
   if (t->h_stage) cudaFreeHost(t->h_stage);
+  if (t->staged) cudaEventDestroy(t->staged);
   delete t;
   return TV_OK;
 }
@@ -235,7 +251,9 @@ TV_API int tv_tree_verify(const tv_tree* tree, const tv_dims* d, const float* S_
   a.L = d->L; a.B = d->B; a.H = d->H; a.T = d->T; a.dk = d->dk; a.dv = d->dv;
   a.rule = d->rule; a.bf16 = d->qkv_dtype == TV_BF16;
   a.S_pre = S_pre; a.q = q; a.k = k; a.v = v; a.alpha = alpha; a.beta = beta; a.O = O; a.U = U;
-  if (d->impl == TV_IMPL_TC) return TV_ERR_UNSUPPORTED;
+  const bool tc_ok = tv_verify_tc_supports(a);
+  if (d->impl == TV_IMPL_TC && !tc_ok) return TV_ERR_UNSUPPORTED;
+  if (tc_ok && d->impl != TV_IMPL_SIMT) return tv_launch_verify_tc(a, tree->d_status, (cudaStream_t)stream);
   return tv_launch_verify_simt(a, (cudaStream_t)stream);
 }
 

@@ -31,14 +31,17 @@ struct PathInfo {
 };
 
 // Fills path_s[0..len) (topological order), w_s[p] = P_a / P_path[p] and *Pa_s.
+// al_s is scratch for the T decay gates (loaded by T threads in parallel so that
+// the serial suffix product below never waits on global memory).
 __device__ __forceinline__ int build_path(const TreeDev& tree, int tb, int T, int acc,
                                           const float* alpha_row, int* path_s, float* w_s,
-                                          float* Pa_s) {
+                                          float* al_s, float* Pa_s) {
   const uint64_t* m = tree.anc + ((size_t)tb * T + acc) * 2;
+  const int t = threadIdx.x;
+  if (t < T) al_s[t] = alpha_row[t];
   uint64_t m0 = m[0], m1 = m[1];
   if (acc < 64) m0 |= 1ull << acc; else m1 |= 1ull << (acc - 64);
   const int len = __popcll(m0) + __popcll(m1);
-  const int t = threadIdx.x;
   if (t < 128) {
     const uint64_t w = t < 64 ? m0 : m1;
     const int bit = t & 63;
@@ -53,12 +56,24 @@ __device__ __forceinline__ int build_path(const TreeDev& tree, int tb, int T, in
     float w = 1.f;
     for (int p = len - 1; p >= 0; --p) {
       w_s[p] = w;
-      w *= alpha_row[path_s[p]];
+      w *= al_s[path_s[p]];
     }
     *Pa_s = w;
   }
   __syncthreads();
   return len;
+}
+
+// Streaming 16-byte load / store: the state is touched exactly once.
+__device__ __forceinline__ float4 ld_stream(const float4* p) {
+  float4 v;
+  asm volatile("ld.global.L1::no_allocate.v4.f32 {%0,%1,%2,%3}, [%4];"
+               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
+  return v;
+}
+__device__ __forceinline__ void st_stream(float4* p, const float4& v) {
+  asm volatile("st.global.L1::no_allocate.v4.f32 [%0], {%1,%2,%3,%4};"
+               :: "l"(p), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
 }
 
 // Commit from given correction rows u_j: U (float) when a.U != NULL, else v.
@@ -67,6 +82,7 @@ __global__ void __launch_bounds__(kThreads) commit_factored_kernel(CommitArgs a)
   __shared__ int path_s[TV_MAX_NODES];
   __shared__ float w_s[TV_MAX_NODES];
   __shared__ float Pa_s;
+  __shared__ float al_s[TV_MAX_NODES];
   __shared__ __align__(16) float k_s[kPathChunk][TV_MAX_DIM];
   __shared__ float cu_s[kPathChunk][TV_MAX_DIM];
 
@@ -83,20 +99,20 @@ __global__ void __launch_bounds__(kThreads) commit_factored_kernel(CommitArgs a)
   if (acc >= T) acc = -1;
   if (acc < 0) {
     if (a.S_new != a.S_pre)
-      for (int i = tid; i < n4; i += kThreads) dst[i] = src[i];
+      for (int i = tid; i < n4; i += kThreads) st_stream(dst + i, ld_stream(src + i));
     return;
   }
-  const int tb = a.tree.n_trees == 1 ? 0 : b;
-  const size_t node0 = (size_t)item * T;  // first node row of this (l, b, h)
-  const int len = build_path(a.tree, tb, T, acc, a.alpha + node0, path_s, w_s, &Pa_s);
-  const float Pa = Pa_s;
-
+  // The whole state goes in flight first; the path is worked out under its latency.
   float4 s[kMaxVec];
 #pragma unroll
   for (int e = 0; e < kMaxVec; ++e) {
     const int i = tid + e * kThreads;
-    if (i < n4) s[e] = src[i];
+    if (i < n4) s[e] = ld_stream(src + i);
   }
+  const int tb = a.tree.n_trees == 1 ? 0 : b;
+  const size_t node0 = (size_t)item * T;  // first node row of this (l, b, h)
+  const int len = build_path(a.tree, tb, T, acc, a.alpha + node0, path_s, w_s, al_s, &Pa_s);
+  const float Pa = Pa_s;
 #pragma unroll
   for (int e = 0; e < kMaxVec; ++e) {
     s[e].x *= Pa; s[e].y *= Pa; s[e].z *= Pa; s[e].w *= Pa;
@@ -135,7 +151,7 @@ __global__ void __launch_bounds__(kThreads) commit_factored_kernel(CommitArgs a)
 #pragma unroll
   for (int e = 0; e < kMaxVec; ++e) {
     const int i = tid + e * kThreads;
-    if (i < n4) dst[i] = s[e];
+    if (i < n4) st_stream(dst + i, s[e]);
   }
 }
 
@@ -154,7 +170,8 @@ __global__ void __launch_bounds__(kThreads) commit_delta_rows_kernel(CommitArgs 
   __shared__ float Pa_s;
   __shared__ __align__(16) float k_s[kPathChunk][DK];
   __shared__ float v_s[kPathChunk][TV_MAX_DIM];
-  __shared__ float al_s[kPathChunk], be_s[kPathChunk];
+  __shared__ float alc_s[kPathChunk], be_s[kPathChunk];
+  __shared__ float al_s[TV_MAX_NODES];
 
   const int item = blockIdx.x;
   const int b = (item / a.H) % a.B;
@@ -175,7 +192,7 @@ __global__ void __launch_bounds__(kThreads) commit_delta_rows_kernel(CommitArgs 
   }
   const int tb = a.tree.n_trees == 1 ? 0 : b;
   const size_t node0 = (size_t)item * T;
-  const int len = build_path(a.tree, tb, T, acc, a.alpha + node0, path_s, w_s, &Pa_s);
+  const int len = build_path(a.tree, tb, T, acc, a.alpha + node0, path_s, w_s, al_s, &Pa_s);
 
   float s[kRowsPerWarp][NPL];
 #pragma unroll
@@ -204,7 +221,7 @@ __global__ void __launch_bounds__(kThreads) commit_delta_rows_kernel(CommitArgs 
       v_s[p][vv] = load_elem<BF16>(a.v, (node0 + path_s[c0 + p]) * dv + vv);
     }
     if (tid < nc) {
-      al_s[tid] = a.alpha[node0 + path_s[c0 + tid]];
+      alc_s[tid] = al_s[path_s[c0 + tid]];
       be_s[tid] = a.beta[node0 + path_s[c0 + tid]];
     }
     __syncthreads();
@@ -212,7 +229,7 @@ __global__ void __launch_bounds__(kThreads) commit_delta_rows_kernel(CommitArgs 
       float kr[NPL];
 #pragma unroll
       for (int x = 0; x < NPL; ++x) kr[x] = k_s[p][lane * NPL + x];
-      const float al = al_s[p], be = be_s[p];
+      const float al = alc_s[p], be = be_s[p];
 #pragma unroll
       for (int r = 0; r < kRowsPerWarp; ++r) {
         const int row = warp + r * (kThreads / 32);

@@ -20,7 +20,9 @@ struct tv_tree {
   const uint64_t* d_anc = nullptr;
   const int32_t* d_depth = nullptr;
   const int32_t* d_parent = nullptr;
+  int32_t* d_status = nullptr;  // device status word (0 = ok), cleared by every upload
   bool uploaded = false;
+  cudaEvent_t staged = nullptr;  // completion of the last staging copy
 };
 
 // Kernel-side view of the tree metadata.
@@ -63,6 +65,8 @@ void tv_set_cuda_error(cudaError_t e);
 // Launchers (each returns a tv_status; all work is asynchronous on `stream`).
 int tv_launch_verify_simt(const VerifyArgs& a, cudaStream_t stream);
 int tv_launch_commit(const CommitArgs& a, cudaStream_t stream);
+bool tv_verify_tc_supports(const VerifyArgs& a);
+int tv_launch_verify_tc(const VerifyArgs& a, int32_t* status, cudaStream_t stream);
 
 #define TV_CUDA_TRY(expr)                 \
   do {                                    \

@@ -102,7 +102,7 @@ __device__ __forceinline__ void dense_pass(const VerifyArgs& a, const Smem& sm, 
       sm.A_s[i * kALD + kk] = x;
     }
     __syncthreads();
-    const int kmax = min(kKC, dk - k0);
+    const int kmax = ty * 8 < T ? min(kKC, dk - k0) : 0;  // skip row tiles past the tree
     for (int kk = 0; kk < kmax; ++kk) {
       float av[8];
 #pragma unroll

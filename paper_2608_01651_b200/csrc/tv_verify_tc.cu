@@ -1,0 +1,560 @@
+// Tree verification on the 5th-generation tensor cores (tcgen05 + TMEM + TMA).
+//
+// Shapes: bf16 q/k/v, fp32 state, dk = dv = 128, T <= 128, gated rule.
+// One persistent CTA per SM walks (layer, request, head) items.  Per item
+// (Theorem 1 / Eq. 4 with U = V):
+//
+//   scores  Sc = Q K^T                 bf16 x bf16 -> fp32 in TMEM (exact products)
+//   prefix  A1 = Q S_pre^T             tf32: Q widened bf16 -> fp32 into TMEM as
+//                                      the A operand (exact), S_pre consumed as
+//                                      raw fp32 straight from the TMA buffer
+//   C_ij    = 1[j in Anc(i)+{i}] exp2(g_i - g_j) Sc_ij,  g = sum log2(alpha)
+//             over the path (decay ratio only ever taken on ancestor pairs),
+//             split into bf16 hi + lo so that C V keeps ~16 mantissa bits
+//   readout A2 = C_hi V + C_lo V       bf16 x bf16 -> fp32 in TMEM
+//   O_i     = P_i A1_i + A2_i          fp32 epilogue, P_i = exp2(g_i)
+//
+// S_pre (the HBM-dominant stream) goes TMA -> shared memory -> tensor core and
+// is never touched by a thread.  Nothing but O is written.
+//
+// Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer (owns TMEM), warps
+// 2..9 = 8 compute warps; compute warp w reads TMEM lanes 32 (w % 4) .. +31
+// (the hardware's lane window of that warp) and half of the columns.
+// Every wait is an mbarrier wait with a time limit; on expiry the CTA sets the
+// status word, drains its own copies and leaves (TMEM is freed on every path).
+#include <cuda.h>
+#include <cudaTypedefs.h>
+#include <cuda_bf16.h>
+
+#include "tv_internal.h"
+
+namespace {
+
+constexpr int kThreads = 320;
+constexpr int kComputeWarps = 8;
+constexpr uint32_t kTile = 16384;  // one 128-row x 128-byte operand tile
+
+// shared memory map (byte offsets from the 1024-aligned base)
+constexpr uint32_t kOffQ = 0;                     // 2 tiles: k halves of Q  [128][64] bf16
+constexpr uint32_t kOffK = kOffQ + 2 * kTile;     // 2 tiles: k halves of K
+constexpr uint32_t kOffV = kOffK + 2 * kTile;     // 2 tiles: dv halves of V [128 j][64] bf16
+constexpr uint32_t kOffS = kOffV + 2 * kTile;     // 4 tiles: k chunks of S_pre [128 v][32] f32
+constexpr uint32_t kOffChi = kOffS + 4 * kTile;   // 2 tiles: j halves of C_hi [128 i][64] bf16
+constexpr uint32_t kOffClo = kOffChi + 2 * kTile; // 2 tiles: j halves of C_lo
+constexpr uint32_t kOffG = kOffClo + 2 * kTile;   // float g[128]
+constexpr uint32_t kOffAl = kOffG + 512;          // float log2(alpha)[128]
+constexpr uint32_t kOffBar = kOffAl + 512;        // mbarriers
+constexpr uint32_t kOffMisc = kOffBar + 8 * 16;   // tmem base, abort flag
+constexpr uint32_t kSmemBytes = kOffMisc + 16 + 1024;  // + alignment slack
+
+enum Bar {
+  QK_FULL = 0, QK_FREE, S_FULL, S_FREE, V_FULL, V_FREE,
+  SC_DONE, SC_FREE, QF_READY, C_READY, ACC_DONE, ACC_FREE, SETUP
+};
+
+// TMEM columns
+constexpr uint32_t kColQf = 0, kColSc = 128, kColA1 = 256, kColA2 = 384;
+
+constexpr uint32_t kIdescBf16KK = (1u << 4) | (1u << 7) | (1u << 10) | (16u << 17) | (8u << 24);
+constexpr uint32_t kIdescBf16KMn = kIdescBf16KK | (1u << 16);
+constexpr uint32_t kIdescTf32 = (1u << 4) | (2u << 7) | (2u << 10) | (16u << 17) | (8u << 24);
+
+constexpr long long kWaitLimitCycles = 1ll << 31;  // ~1 s
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+
+// ---- mbarrier ---------------------------------------------------------------
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false when the limit ran out or another role gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (uint32_t spin = 1;; ++spin) {
+    if (mbar_try(bar, parity)) return true;
+    if ((spin & 1023u) == 0) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > kWaitLimitCycles) {
+        *abort_flag = 1;
+        return false;
+      }
+    }
+  }
+}
+
+// Same for a whole warp: every lane gets the same answer, so that the warp never
+// splits around the warp-collective tcgen05 instructions that follow.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  const bool ok = mbar_wait(bar, parity, abort_flag);
+  return __all_sync(0xffffffffu, ok);
+}
+
+// ---- TMA --------------------------------------------------------------------
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar,
+                                            int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+
+// ---- tcgen05 ----------------------------------------------------------------
+__device__ __forceinline__ void tc_fence_before() {
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after() {
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+               ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mma_bf16_ss(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc,
+                                            uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d), "l"(a), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void mma_tf32_ts(uint32_t d, uint32_t a_tmem, uint64_t b, uint32_t idesc,
+                                            uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d), "r"(a_tmem), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
+        "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),
+        "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]),
+        "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+        "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]),
+        "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]),
+        "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]),
+        "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]),
+        "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+// Shared-memory matrix descriptors, 128-byte swizzle, 1024-byte swizzle atoms.
+// K-major: rows of 128 bytes, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t desc_kmajor(uint32_t saddr) {
+  return (uint64_t)((saddr & 0x3ffffu) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) |
+         (1ull << 46) | (2ull << 61);
+}
+// MN-major (V as the B operand, dv contiguous): 64-column blocks `lbo` bytes
+// apart, 8-row k groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t desc_mnmajor(uint32_t saddr, uint32_t lbo) {
+  return (uint64_t)((saddr & 0x3ffffu) >> 4) | ((uint64_t)(lbo >> 4) << 16) |
+         ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&t);
+}
+
+struct TcParams {
+  TreeDev tree;
+  int32_t n_items, B, H, T;
+  const float* alpha;
+  float* O;
+  int32_t* status;
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                       const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmS,
+                       const TcParams p) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* sm = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  const uint32_t sbase = smem_u32(sm);
+  float* g_s = reinterpret_cast<float*>(sm + kOffG);
+  float* la_s = reinterpret_cast<float*>(sm + kOffAl);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + kOffMisc);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + kOffMisc + 4);
+  auto bar = [&](int i) { return sbase + kOffBar + 8u * i; };
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int T = p.T;
+  const int n_jh = T > 64 ? 2 : 1;  // 64-wide j halves that hold real nodes
+
+  if (tid == 0) {
+    abort_flag[0] = 0;
+    abort_flag[1] = 0;
+    mbar_init(bar(QK_FULL), 1);  mbar_init(bar(QK_FREE), 1 + kComputeWarps);
+    mbar_init(bar(S_FULL), 1);   mbar_init(bar(S_FREE), 1);
+    mbar_init(bar(V_FULL), 1);   mbar_init(bar(V_FREE), 1);
+    mbar_init(bar(SC_DONE), 1);  mbar_init(bar(SC_FREE), kComputeWarps);
+    mbar_init(bar(QF_READY), kComputeWarps);
+    mbar_init(bar(C_READY), kComputeWarps);
+    mbar_init(bar(ACC_DONE), 1); mbar_init(bar(ACC_FREE), kComputeWarps);
+    mbar_init(bar(SETUP), kComputeWarps);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(tmem_slot)), "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  if (warp == 0) {
+    // ===================== TMA producer =====================
+    if (lane == 0) {
+      int pend_qk = 0, pend_s = 0, pend_v = 0;
+      uint32_t it = 0;
+      for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++it) {
+        const uint32_t ph = it & 1;
+        if (!mbar_wait(bar(QK_FREE), ph ^ 1, abort_flag)) break;
+        mbar_expect_tx(bar(QK_FULL), 4 * kTile);
+        tma_load_3d(sbase + kOffQ, &tmQ, bar(QK_FULL), 0, 0, item);
+        tma_load_3d(sbase + kOffQ + kTile, &tmQ, bar(QK_FULL), 64, 0, item);
+        tma_load_3d(sbase + kOffK, &tmK, bar(QK_FULL), 0, 0, item);
+        tma_load_3d(sbase + kOffK + kTile, &tmK, bar(QK_FULL), 64, 0, item);
+        pend_qk = 1 + (int)ph;
+        if (!mbar_wait(bar(S_FREE), ph ^ 1, abort_flag)) break;
+        mbar_expect_tx(bar(S_FULL), 4 * kTile);
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+          tma_load_3d(sbase + kOffS + c * kTile, &tmS, bar(S_FULL), 32 * c, 0, item);
+        pend_s = 1 + (int)ph;
+        if (!mbar_wait(bar(V_FREE), ph ^ 1, abort_flag)) break;
+        mbar_expect_tx(bar(V_FULL), 2 * kTile);
+        tma_load_3d(sbase + kOffV, &tmV, bar(V_FULL), 0, 0, item);
+        tma_load_3d(sbase + kOffV + kTile, &tmV, bar(V_FULL), 64, 0, item);
+        pend_v = 1 + (int)ph;
+      }
+      if (*abort_flag) {
+        // Leave no copy of ours in flight: wait (bounded) for the last loads issued.
+        if (pend_qk) mbar_wait(bar(QK_FULL), pend_qk - 1, abort_flag + 1);
+        if (pend_s) mbar_wait(bar(S_FULL), pend_s - 1, abort_flag + 1);
+        if (pend_v) mbar_wait(bar(V_FULL), pend_v - 1, abort_flag + 1);
+      }
+    }
+  } else if (warp == 1) {
+    // ===================== MMA issuer =====================
+    if (lane == 0) {
+      uint32_t it = 0;
+      for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++it) {
+        const uint32_t ph = it & 1;
+        // scores = Q K^T
+        if (!mbar_wait(bar(QK_FULL), ph, abort_flag)) break;
+        if (!mbar_wait(bar(SC_FREE), ph ^ 1, abort_flag)) break;
+        tc_fence_after();
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+#pragma unroll
+          for (int s = 0; s < 4; ++s)
+            mma_bf16_ss(tmem + kColSc, desc_kmajor(sbase + kOffQ + h * kTile + s * 32),
+                        desc_kmajor(sbase + kOffK + h * kTile + s * 32), kIdescBf16KK, (h | s) != 0);
+        tc_commit(bar(SC_DONE));
+        tc_commit(bar(QK_FREE));
+        // prefix = Q S_pre^T  (A = Q as fp32 in TMEM, B = S_pre chunks)
+        if (!mbar_wait(bar(S_FULL), ph, abort_flag)) break;
+        if (!mbar_wait(bar(QF_READY), ph, abort_flag)) break;
+        if (!mbar_wait(bar(ACC_FREE), ph ^ 1, abort_flag)) break;
+        tc_fence_after();
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+#pragma unroll
+          for (int s = 0; s < 4; ++s)
+            mma_tf32_ts(tmem + kColA1, tmem + kColQf + c * 32 + s * 8,
+                        desc_kmajor(sbase + kOffS + c * kTile + s * 32), kIdescTf32, (c | s) != 0);
+        tc_commit(bar(S_FREE));
+        // readout = C_hi V + C_lo V
+        if (!mbar_wait(bar(C_READY), ph, abort_flag)) break;
+        if (!mbar_wait(bar(V_FULL), ph, abort_flag)) break;
+        tc_fence_after();
+        for (int jh = 0; jh < n_jh; ++jh)
+#pragma unroll
+          for (int s = 0; s < 4; ++s) {
+            const uint64_t bdesc = desc_mnmajor(sbase + kOffV + (jh * 4 + s) * 2048, kTile);
+            mma_bf16_ss(tmem + kColA2, desc_kmajor(sbase + kOffChi + jh * kTile + s * 32), bdesc,
+                        kIdescBf16KMn, (jh | s) != 0);
+            mma_bf16_ss(tmem + kColA2, desc_kmajor(sbase + kOffClo + jh * kTile + s * 32), bdesc,
+                        kIdescBf16KMn, 1);
+          }
+        tc_commit(bar(V_FREE));
+        tc_commit(bar(ACC_DONE));
+      }
+    }
+  } else {
+    // ===================== compute warps =====================
+    const int cw = warp - 2;
+    const int quad = warp & 3;          // TMEM lane window of this warp
+    const int hc = cw >> 2;             // column half handled by this warp
+    const int row = quad * 32 + lane;   // node i
+    const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+    const uint32_t swz = (uint32_t)(row & 7);
+    uint32_t it = 0;
+    for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++it) {
+      const uint32_t ph = it & 1;
+      const int b = (item / p.H) % p.B;
+      const int tb = p.tree.n_trees == 1 ? 0 : b;
+      const size_t node0 = (size_t)item * T;
+      // ---- path decay: g_i = sum of log2(alpha) over Anc(i) + {i} ----
+      uint64_t m0 = 0, m1 = 0;
+      if (row < T) {
+        const uint64_t* m = p.tree.anc + ((size_t)tb * T + row) * 2;
+        m0 = m[0];
+        m1 = m[1];
+        if (hc == 0) la_s[row] = log2f(p.alpha[node0 + row]);
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(SETUP));
+      if (!mbar_wait_warp(bar(SETUP), 0, abort_flag)) break;   // SETUP completes two phases per item
+      float g = 0.f;
+      if (row < T) {
+        g = la_s[row];
+        uint64_t a0 = m0, a1 = m1;
+        while (a0) { const int j = __ffsll((long long)a0) - 1; a0 &= a0 - 1; g += la_s[j]; }
+        while (a1) { const int j = __ffsll((long long)a1) - 1; a1 &= a1 - 1; g += la_s[64 + j]; }
+        if (row < 64) m0 |= 1ull << row; else m1 |= 1ull << (row - 64);   // M+ = M- + I
+      }
+      // ---- Q row (bf16, swizzled tile) -> fp32 -> TMEM (A operand of the prefix MMA) ----
+      if (!mbar_wait_warp(bar(QK_FULL), ph, abort_flag)) break;
+      {
+        const unsigned char* qrow = sm + kOffQ + hc * kTile + row * 128;
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          uint32_t r[32];
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            const uint4 x = *reinterpret_cast<const uint4*>(qrow + (((half * 4 + c) ^ swz) << 4));
+            const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              r[c * 8 + 2 * e] = w[e] << 16;
+              r[c * 8 + 2 * e + 1] = w[e] & 0xffff0000u;
+            }
+          }
+          tmem_st32(tmem + lane_addr + kColQf + hc * 64 + half * 32, r);
+        }
+        tmem_wait_st();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive(bar(QF_READY));
+          mbar_arrive(bar(QK_FREE));
+        }
+      }
+      // every warp needs the g_j of its column half: publish, then synchronise again
+      if (hc == 0 && row < T) g_s[row] = g;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(SETUP));
+      // ---- scores -> masked, decayed, split C ----
+      if (!mbar_wait_warp(bar(SC_DONE), ph, abort_flag)) break;
+      tc_fence_after();
+      if (!mbar_wait_warp(bar(SETUP), 1, abort_flag)) break;
+      if (hc < n_jh) {
+        const uint64_t mw = hc == 0 ? m0 : m1;
+        unsigned char* chi = sm + kOffChi + hc * kTile + row * 128;
+        unsigned char* clo = sm + kOffClo + hc * kTile + row * 128;
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          uint32_t r[32];
+          tmem_ld32(tmem + lane_addr + kColSc + hc * 64 + half * 32, r);
+          tmem_wait_ld();
+          const uint32_t bits = (uint32_t)(mw >> (half * 32));
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            uint32_t hi[4], lo[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              float cv[2];
+#pragma unroll
+              for (int t = 0; t < 2; ++t) {
+                const int jj = c * 8 + 2 * e + t;
+                const float gj = g_s[hc * 64 + half * 32 + jj];
+                const float ratio = exp2f(g - gj);   // overflow on non-ancestors is selected away
+                cv[t] = ((bits >> jj) & 1u) ? __uint_as_float(r[jj]) * ratio : 0.f;
+              }
+              const __nv_bfloat162 h2 = __floats2bfloat162_rn(cv[0], cv[1]);
+              const float2 hf = __bfloat1622float2(h2);
+              hi[e] = *reinterpret_cast<const uint32_t*>(&h2);
+              lo[e] = pack_bf16(cv[0] - hf.x, cv[1] - hf.y);
+            }
+            const uint32_t off = ((uint32_t)((half * 4 + c) ^ swz)) << 4;
+            *reinterpret_cast<uint4*>(chi + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+            *reinterpret_cast<uint4*>(clo + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+          }
+        }
+      }
+      fence_async_smem();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) {
+        mbar_arrive(bar(C_READY));
+        mbar_arrive(bar(SC_FREE));
+      }
+      // ---- O_i = P_i A1_i + A2_i ----
+      if (!mbar_wait_warp(bar(ACC_DONE), ph, abort_flag)) break;
+      tc_fence_after();
+      {
+        const float Pi = exp2f(g);
+        float* orow = p.O + (node0 + row) * 128 + hc * 64;
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          uint32_t r1[32], r2[32];
+          tmem_ld32(tmem + lane_addr + kColA1 + hc * 64 + half * 32, r1);
+          tmem_ld32(tmem + lane_addr + kColA2 + hc * 64 + half * 32, r2);
+          tmem_wait_ld();
+          if (row < T) {
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+              float4 o;
+              o.x = fmaf(Pi, __uint_as_float(r1[4 * c + 0]), __uint_as_float(r2[4 * c + 0]));
+              o.y = fmaf(Pi, __uint_as_float(r1[4 * c + 1]), __uint_as_float(r2[4 * c + 1]));
+              o.z = fmaf(Pi, __uint_as_float(r1[4 * c + 2]), __uint_as_float(r2[4 * c + 2]));
+              o.w = fmaf(Pi, __uint_as_float(r1[4 * c + 3]), __uint_as_float(r2[4 * c + 3]));
+              *reinterpret_cast<float4*>(orow + half * 32 + 4 * c) = o;
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(ACC_FREE));
+    }
+  }
+
+  // ---- teardown: every path comes here ----
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (warp == 1) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u)
+                 : "memory");
+  }
+  if (tid == 0 && *abort_flag && p.status) atomicExch(p.status, (int)TV_ERR_DEVICE_TIMEOUT);
+}
+
+// ---------------------------------------------------------------------------
+// Host side: tensor maps and launch.
+// ---------------------------------------------------------------------------
+PFN_cuTensorMapEncodeTiled get_encode() {
+  static PFN_cuTensorMapEncodeTiled fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) ==
+            cudaSuccess && qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<PFN_cuTensorMapEncodeTiled>(ptr);
+  }
+  return fn;
+}
+
+// [items][rows][cols] tensor, box {box_cols, 128, 1}, 128-byte swizzle, zero fill.
+bool make_map(CUtensorMap* map, const void* base, CUtensorMapDataType dt, int esize, uint64_t items,
+              uint64_t rows, uint64_t cols, uint32_t box_cols) {
+  PFN_cuTensorMapEncodeTiled enc = get_encode();
+  if (!enc) return false;
+  const cuuint64_t gdim[3] = {cols, rows, items};
+  const cuuint64_t gstr[2] = {cols * esize, rows * cols * esize};
+  const cuuint32_t box[3] = {box_cols, 128, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return enc(map, dt, 3, const_cast<void*>(base), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Gated rule: the correction rows are the values themselves (U = V).
+__global__ void widen_bf16_kernel(const __nv_bfloat16* __restrict__ v, float* __restrict__ U, size_t n8) {
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n8; i += (size_t)gridDim.x * blockDim.x) {
+    const uint4 x = reinterpret_cast<const uint4*>(v)[i];
+    const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+    float4 a, b;
+    a.x = __uint_as_float(w[0] << 16); a.y = __uint_as_float(w[0] & 0xffff0000u);
+    a.z = __uint_as_float(w[1] << 16); a.w = __uint_as_float(w[1] & 0xffff0000u);
+    b.x = __uint_as_float(w[2] << 16); b.y = __uint_as_float(w[2] & 0xffff0000u);
+    b.z = __uint_as_float(w[3] << 16); b.w = __uint_as_float(w[3] & 0xffff0000u);
+    reinterpret_cast<float4*>(U)[2 * i] = a;
+    reinterpret_cast<float4*>(U)[2 * i + 1] = b;
+  }
+}
+
+}  // namespace
+
+bool tv_verify_tc_supports(const VerifyArgs& a) {
+  return a.bf16 && a.dk == 128 && a.dv == 128 && a.rule == TV_GATED && a.T <= 128;
+}
+
+int tv_launch_verify_tc(const VerifyArgs& a, int32_t* status, cudaStream_t stream) {
+  if (!tv_verify_tc_supports(a)) return TV_ERR_UNSUPPORTED;
+  const uint64_t items = (uint64_t)a.L * a.B * a.H;
+  alignas(64) CUtensorMap tmQ, tmK, tmV, tmS;
+  if (!make_map(&tmQ, a.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, items, a.T, 128, 64) ||
+      !make_map(&tmK, a.k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, items, a.T, 128, 64) ||
+      !make_map(&tmV, a.v, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, items, a.T, 128, 64) ||
+      !make_map(&tmS, a.S_pre, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, 128, 128, 32))
+    return TV_ERR_CUDA;
+  static thread_local int configured_dev = -1;
+  static thread_local int sm_count = 0;
+  int dev = 0;
+  TV_CUDA_TRY(cudaGetDevice(&dev));
+  if (configured_dev != dev) {
+    TV_CUDA_TRY(cudaFuncSetAttribute(verify_tc_gated_kernel,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
+    TV_CUDA_TRY(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev));
+    configured_dev = dev;
+  }
+  TcParams p;
+  p.tree = a.tree;
+  p.n_items = (int32_t)items;
+  p.B = a.B; p.H = a.H; p.T = a.T;
+  p.alpha = a.alpha;
+  p.O = a.O;
+  p.status = status;
+  const int grid = (int)(items < (uint64_t)sm_count ? items : (uint64_t)sm_count);
+  verify_tc_gated_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tmQ, tmK, tmV, tmS, p);
+  TV_CUDA_TRY(cudaGetLastError());
+  if (a.U) {
+    const size_t n8 = items * a.T * 128 / 8;
+    const int blocks = (int)((n8 + 255) / 256 < 4096 ? (n8 + 255) / 256 : 4096);
+    widen_bf16_kernel<<<blocks, 256, 0, stream>>>(reinterpret_cast<const __nv_bfloat16*>(a.v), a.U, n8);
+    TV_CUDA_TRY(cudaGetLastError());
+  }
+  return TV_OK;
+}

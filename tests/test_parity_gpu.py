@@ -16,7 +16,16 @@ from tests import parity_util as pu
 
 pytestmark = pytest.mark.gpu
 
-IMPLS = [tv.IMPL_SIMT]
+IMPLS = [tv.IMPL_SIMT, tv.IMPL_TC]
+
+
+def _tc_ok(wl):
+    return wl.qkv_dtype == inputs.BF16 and wl.dk == 128 and wl.dv == 128 and wl.rule == inputs.GATED
+
+
+def _skip_unless_supported(wl, impl):
+    if impl == tv.IMPL_TC and not _tc_ok(wl):
+        pytest.skip("tensor-core kernel covers bf16, dk = dv = 128, gated rule")
 
 
 def _run(wl, parents, accepted, tens, tol, items=None, **kw):
@@ -34,6 +43,7 @@ def _run(wl, parents, accepted, tens, tol, items=None, **kw):
 @pytest.mark.parametrize("name", ["c1", "c2", "c3", "c4"])
 def test_workload_full(name, impl):
     wl = inputs.workload(name)
+    _skip_unless_supported(wl, impl)
     parents, accepted = inputs.make_trees(wl)
     tens = inputs.make_tensors(wl)
     _run(wl, parents, accepted, tens, wl.tol, impl=impl)
@@ -48,6 +58,7 @@ def test_c5_full_size_sampled(impl):
     """Full batch and tree size of the throughput workload, 2 layers in one
     call; the oracle checks a seeded sample of (layer, request, head) items."""
     wl = inputs.workload("c5", L=2)
+    _skip_unless_supported(wl, impl)
     parents, accepted = inputs.make_trees(wl)
     tens = [inputs.make_tensors(wl, layer=l) for l in range(wl.L)]
     stacked = {k: (None if tens[0][k] is None else torch.stack([t[k] for t in tens]))
@@ -86,6 +97,7 @@ def test_edge_shapes(case, dtype, rule, impl):
     T, dk, dv, B, H, kind, shared = case
     wl = inputs.workload("c2", T=T, dk=dk, dv=dv, B=B, H=H, rule=rule, qkv_dtype=dtype,
                          tree="frontier" if kind == "star" else kind, seed=100 + T)
+    _skip_unless_supported(wl, impl)
     parents, accepted = inputs.make_trees(wl, per_request=not shared)
     if kind == "star":
         parents[:] = -1

@@ -1,0 +1,38 @@
+"""Tensor-core verify kernel: smallest cases first, then several items per CTA."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2608_01651_b200 as tv
+from paper_2608_01651_b200 import inputs
+from tests import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("B,H,T", [(1, 1, 128), (1, 1, 64), (1, 2, 37), (4, 8, 128), (40, 16, 100)])
+def test_tc_gated(B, H, T):
+    wl = inputs.workload("c5", B=B, H=H, T=T, L=1, tree="frontier", seed=11 + T)
+    parents, accepted = inputs.make_trees(wl)
+    tens = inputs.make_tensors(wl)
+    O, U, Sn, tree = pu.gpu_round(wl, parents, accepted, tens, impl=tv.IMPL_TC, want_U=True)
+    tree.device_status()
+    ver, com = pu.oracle_round(wl, parents, accepted, tens)
+    eO, eU, eS = pu.compare(wl, O, U, Sn, ver, com)
+    print(f"TC B{B} H{H} T{T}: rel-L2 O {eO:.3e} U {eU:.3e} S {eS:.3e}")
+    assert eO <= wl.tol and eU == 0.0 and eS <= wl.tol
+
+
+def test_tc_error_budget_report():
+    """Mean and worst per-node error of the tensor-core path on c3 (printed)."""
+    wl = inputs.workload("c3", B=4)
+    parents, accepted = inputs.make_trees(wl)
+    tens = inputs.make_tensors(wl)
+    O, _, Sn, tree = pu.gpu_round(wl, parents, accepted, tens, impl=tv.IMPL_TC, want_U=False)
+    ver, com = pu.oracle_round(wl, parents, accepted, tens)
+    errs = []
+    for (b, h), (Or, _) in ver.items():
+        errs.append(np.linalg.norm(O[b, h] - Or, axis=-1) / np.linalg.norm(Or, axis=-1))
+    errs = np.concatenate(errs)
+    print(f"TC c3 per-node rel-L2: mean {errs.mean():.3e} max {errs.max():.3e}")
+    assert errs.max() <= wl.tol
