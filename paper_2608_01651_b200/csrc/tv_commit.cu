@@ -26,10 +26,6 @@ __device__ __forceinline__ float load_elem(const void* base, size_t idx) {
   return reinterpret_cast<const float*>(base)[idx];
 }
 
-struct PathInfo {
-  int len;
-};
-
 // Fills path_s[0..len) (topological order), w_s[p] = P_a / P_path[p] and *Pa_s.
 // al_s is scratch for the T decay gates (loaded by T threads in parallel so that
 // the serial suffix product below never waits on global memory).
@@ -155,6 +151,109 @@ __global__ void __launch_bounds__(kThreads) commit_factored_kernel(CommitArgs a)
   }
 }
 
+// dk = 128 fast path.  A CTA of 4 warps owns 64 consecutive rows (value
+// channels) of one state; warp w owns rows 16w..16w+15 and a lane owns one
+// float4 column, so every load and store of a warp is one contiguous 512-byte
+// row and the key row k_j[4 lane .. 4 lane + 3] stays in registers across the
+// 16 rows.  All 16 loads of a thread are in flight before anything else
+// happens; several CTAs per SM keep the stream continuous.
+constexpr int kRowThreads = 128;
+constexpr int kRowsPerCta = 64;
+
+template <bool BF16>
+__global__ void __launch_bounds__(kRowThreads) commit_factored_dk128_kernel(CommitArgs a) {
+  __shared__ int path_s[TV_MAX_NODES];
+  __shared__ float w_s[TV_MAX_NODES];
+  __shared__ float Pa_s;
+  __shared__ float al_s[TV_MAX_NODES];
+  __shared__ __align__(16) float k_s[kPathChunk][128];
+  __shared__ __align__(16) float cu_s[kPathChunk][kRowsPerCta];
+
+  const int dv = a.dv, T = a.T;
+  const int n_half = (dv + kRowsPerCta - 1) / kRowsPerCta;
+  const int item = blockIdx.x / n_half, half = blockIdx.x - item * n_half;
+  const int b = (item / a.H) % a.B;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int row0 = half * kRowsPerCta + warp * 16;
+  const size_t sbase = (size_t)item * dv * 128;
+  const float4* src = reinterpret_cast<const float4*>(a.S_pre + sbase) + (size_t)row0 * 32 + lane;
+  float4* dst = reinterpret_cast<float4*>(a.S_new + sbase) + (size_t)row0 * 32 + lane;
+
+  int acc = a.accepted[b];
+  if (acc >= T) acc = -1;
+  if (acc < 0 && a.S_new == a.S_pre) return;
+  float4 s[16];
+#pragma unroll
+  for (int e = 0; e < 16; ++e)
+    if (row0 + e < dv) s[e] = ld_stream(src + e * 32);
+  if (acc < 0) {
+#pragma unroll
+    for (int e = 0; e < 16; ++e)
+      if (row0 + e < dv) st_stream(dst + e * 32, s[e]);
+    return;
+  }
+  const int tb = a.tree.n_trees == 1 ? 0 : b;
+  const size_t node0 = (size_t)item * T;
+  const int len = build_path(a.tree, tb, T, acc, a.alpha + node0, path_s, w_s, al_s, &Pa_s);
+  const float Pa = Pa_s;
+  bool scaled = false;
+  for (int c0 = 0; c0 < len; c0 += kPathChunk) {
+    const int nc = min(kPathChunk, len - c0);
+    if (c0) __syncthreads();
+    for (int i = tid; i < nc * 32; i += kRowThreads) {   // 4 keys per thread per step
+      const int p = i >> 5, k4 = i & 31;
+      const size_t idx = (node0 + path_s[c0 + p]) * 128 + k4 * 4;
+      float4 kv;
+      if (BF16) {
+        const uint2 r = *reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(a.k) + idx);
+        kv = make_float4(__uint_as_float(r.x << 16), __uint_as_float(r.x & 0xffff0000u),
+                         __uint_as_float(r.y << 16), __uint_as_float(r.y & 0xffff0000u));
+      } else {
+        kv = *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(a.k) + idx);
+      }
+      *reinterpret_cast<float4*>(&k_s[p][k4 * 4]) = kv;
+    }
+    for (int i = tid; i < nc * kRowsPerCta; i += kRowThreads) {
+      const int p = i >> 6, r = i & 63;
+      const int vrow = half * kRowsPerCta + r;
+      float u = 0.f;
+      if (vrow < dv) {
+        const size_t idx = (node0 + path_s[c0 + p]) * dv + vrow;
+        u = a.U ? a.U[idx] : load_elem<BF16>(a.v, idx);
+      }
+      cu_s[p][r] = w_s[c0 + p] * u;
+    }
+    __syncthreads();
+    if (!scaled) {   // first use of the state: the loads have had the path build to land
+      scaled = true;
+#pragma unroll
+      for (int e = 0; e < 16; ++e) {
+        s[e].x *= Pa; s[e].y *= Pa; s[e].z *= Pa; s[e].w *= Pa;
+      }
+    }
+    for (int p = 0; p < nc; ++p) {
+      const float4 kv = *reinterpret_cast<const float4*>(&k_s[p][lane * 4]);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const float4 cu = *reinterpret_cast<const float4*>(&cu_s[p][warp * 16 + q * 4]);
+        const float c[4] = {cu.x, cu.y, cu.z, cu.w};
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+          float4& x = s[q * 4 + t];
+          x.x = fmaf(c[t], kv.x, x.x);
+          x.y = fmaf(c[t], kv.y, x.y);
+          x.z = fmaf(c[t], kv.z, x.z);
+          x.w = fmaf(c[t], kv.w, x.w);
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int e = 0; e < 16; ++e) {
+    if (row0 + e < dv) st_stream(dst + e * 32, s[e]);
+  }
+}
+
 // Delta rule without stored corrections: every row v of the [dv][dk] state
 // evolves independently along the accepted path,
 //   s <- alpha_j s;  u = beta_j (v_j[v] - s . k_j);  s <- s + u k_j,
@@ -269,7 +368,11 @@ int tv_launch_commit(const CommitArgs& a, cudaStream_t stream) {
   const int items = a.L * a.B * a.H;
   if ((size_t)a.dk * a.dv > (size_t)kMaxVec * kThreads * 4) return TV_ERR_UNSUPPORTED;
   const bool recompute = a.rule == TV_GATED_DELTA && a.U == nullptr;
-  if (!recompute) {
+  if (!recompute && a.dk == 128) {
+    const int ctas = items * ((a.dv + kRowsPerCta - 1) / kRowsPerCta);
+    if (a.bf16) commit_factored_dk128_kernel<true><<<ctas, kRowThreads, 0, stream>>>(a);
+    else commit_factored_dk128_kernel<false><<<ctas, kRowThreads, 0, stream>>>(a);
+  } else if (!recompute) {
     if (a.bf16) commit_factored_kernel<true><<<items, kThreads, 0, stream>>>(a);
     else commit_factored_kernel<false><<<items, kThreads, 0, stream>>>(a);
   } else if (a.dk == 128) {

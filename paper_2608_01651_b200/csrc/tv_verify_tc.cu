@@ -5,14 +5,17 @@
 // (Theorem 1 / Eq. 4 with U = V):
 //
 //   scores  Sc = Q K^T                 bf16 x bf16 -> fp32 in TMEM (exact products)
-//   prefix  A1 = Q S_pre^T             tf32: Q widened bf16 -> fp32 into TMEM as
-//                                      the A operand (exact), S_pre consumed as
-//                                      raw fp32 straight from the TMA buffer
-//   C_ij    = 1[j in Anc(i)+{i}] exp2(g_i - g_j) Sc_ij,  g = sum log2(alpha)
-//             over the path (decay ratio only ever taken on ancestor pairs),
-//             split into bf16 hi + lo so that C V keeps ~16 mantissa bits
-//   readout A2 = C_hi V + C_lo V       bf16 x bf16 -> fp32 in TMEM
-//   O_i     = P_i A1_i + A2_i          fp32 epilogue, P_i = exp2(g_i)
+//   prefix  acc = (2^e_i q_i) S_pre^T  tf32: q widened bf16 -> fp32 and scaled by
+//                                      a power of two (exact) into TMEM as the A
+//                                      operand; S_pre consumed as raw fp32
+//                                      straight from the TMA buffer
+//   C'_ij   = 1[j in Anc(i)+{i}] exp2(e_i - g_j) Sc_ij,  g = sum log2(alpha)
+//             over the path, e_i = round(g_i) (decay ratios only ever taken on
+//             ancestor pairs), split into bf16 hi + lo (~16 mantissa bits)
+//   readout acc += C'_hi V + C'_lo V   bf16 x bf16 -> fp32, same accumulator
+//   O_i     = exp2(g_i - e_i) acc_i    fp32 epilogue
+// The accumulator is double-buffered in TMEM: the epilogue of item n runs under
+// the MMAs of item n+1.
 //
 // S_pre (the HBM-dominant stream) goes TMA -> shared memory -> tensor core and
 // is never touched by a thread.  Nothing but O is written.
@@ -49,11 +52,11 @@ constexpr uint32_t kSmemBytes = kOffMisc + 16 + 1024;  // + alignment slack
 
 enum Bar {
   QK_FULL = 0, QK_FREE, S_FULL, S_FREE, V_FULL, V_FREE,
-  SC_DONE, SC_FREE, QF_READY, C_READY, ACC_DONE, ACC_FREE, SETUP
+  SC_DONE, SC_FREE, QF_READY, C_READY, ACC_DONE0, ACC_DONE1, ACC_FREE0, ACC_FREE1, SETUP
 };
 
-// TMEM columns
-constexpr uint32_t kColQf = 0, kColSc = 128, kColA1 = 256, kColA2 = 384;
+// TMEM columns: scaled Q (A operand), scores, two output accumulators
+constexpr uint32_t kColQf = 0, kColSc = 128, kColAcc0 = 256, kColAcc1 = 384;
 
 constexpr uint32_t kIdescBf16KK = (1u << 4) | (1u << 7) | (1u << 10) | (16u << 17) | (8u << 24);
 constexpr uint32_t kIdescBf16KMn = kIdescBf16KK | (1u << 16);
@@ -224,7 +227,8 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     mbar_init(bar(SC_DONE), 1);  mbar_init(bar(SC_FREE), kComputeWarps);
     mbar_init(bar(QF_READY), kComputeWarps);
     mbar_init(bar(C_READY), kComputeWarps);
-    mbar_init(bar(ACC_DONE), 1); mbar_init(bar(ACC_FREE), kComputeWarps);
+    mbar_init(bar(ACC_DONE0), 1); mbar_init(bar(ACC_DONE1), 1);
+    mbar_init(bar(ACC_FREE0), kComputeWarps); mbar_init(bar(ACC_FREE1), kComputeWarps);
     mbar_init(bar(SETUP), kComputeWarps);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -277,6 +281,10 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       uint32_t it = 0;
       for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++it) {
         const uint32_t ph = it & 1;
+        const uint32_t acc_col = (it & 1) ? kColAcc1 : kColAcc0;
+        const int acc_done = (it & 1) ? ACC_DONE1 : ACC_DONE0;
+        const int acc_free = (it & 1) ? ACC_FREE1 : ACC_FREE0;
+        const uint32_t ph2 = (it >> 1) & 1;   // the two accumulators alternate
         // scores = Q K^T
         if (!mbar_wait(bar(QK_FULL), ph, abort_flag)) break;
         if (!mbar_wait(bar(SC_FREE), ph ^ 1, abort_flag)) break;
@@ -289,19 +297,19 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                         desc_kmajor(sbase + kOffK + h * kTile + s * 32), kIdescBf16KK, (h | s) != 0);
         tc_commit(bar(SC_DONE));
         tc_commit(bar(QK_FREE));
-        // prefix = Q S_pre^T  (A = Q as fp32 in TMEM, B = S_pre chunks)
+        // acc = (2^e Q) S_pre^T  (A = scaled Q as fp32 in TMEM, B = S_pre chunks)
         if (!mbar_wait(bar(S_FULL), ph, abort_flag)) break;
         if (!mbar_wait(bar(QF_READY), ph, abort_flag)) break;
-        if (!mbar_wait(bar(ACC_FREE), ph ^ 1, abort_flag)) break;
+        if (!mbar_wait(bar(acc_free), ph2 ^ 1, abort_flag)) break;
         tc_fence_after();
 #pragma unroll
         for (int c = 0; c < 4; ++c)
 #pragma unroll
           for (int s = 0; s < 4; ++s)
-            mma_tf32_ts(tmem + kColA1, tmem + kColQf + c * 32 + s * 8,
+            mma_tf32_ts(tmem + acc_col, tmem + kColQf + c * 32 + s * 8,
                         desc_kmajor(sbase + kOffS + c * kTile + s * 32), kIdescTf32, (c | s) != 0);
         tc_commit(bar(S_FREE));
-        // readout = C_hi V + C_lo V
+        // acc += C'_hi V + C'_lo V
         if (!mbar_wait(bar(C_READY), ph, abort_flag)) break;
         if (!mbar_wait(bar(V_FULL), ph, abort_flag)) break;
         tc_fence_after();
@@ -309,13 +317,13 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
 #pragma unroll
           for (int s = 0; s < 4; ++s) {
             const uint64_t bdesc = desc_mnmajor(sbase + kOffV + (jh * 4 + s) * 2048, kTile);
-            mma_bf16_ss(tmem + kColA2, desc_kmajor(sbase + kOffChi + jh * kTile + s * 32), bdesc,
-                        kIdescBf16KMn, (jh | s) != 0);
-            mma_bf16_ss(tmem + kColA2, desc_kmajor(sbase + kOffClo + jh * kTile + s * 32), bdesc,
+            mma_bf16_ss(tmem + acc_col, desc_kmajor(sbase + kOffChi + jh * kTile + s * 32), bdesc,
+                        kIdescBf16KMn, 1);
+            mma_bf16_ss(tmem + acc_col, desc_kmajor(sbase + kOffClo + jh * kTile + s * 32), bdesc,
                         kIdescBf16KMn, 1);
           }
         tc_commit(bar(V_FREE));
-        tc_commit(bar(ACC_DONE));
+        tc_commit(bar(acc_done));
       }
     }
   } else {
@@ -326,33 +334,92 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     const int row = quad * 32 + lane;   // node i
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
     const uint32_t swz = (uint32_t)(row & 7);
+
+    // O_i = r_i acc_i for the item whose accumulator is `it_prev`.
+    auto final_epilogue = [&](uint32_t it_prev, size_t node0_prev, float r_prev) -> bool {
+      const int acc_done = (it_prev & 1) ? ACC_DONE1 : ACC_DONE0;
+      const int acc_free = (it_prev & 1) ? ACC_FREE1 : ACC_FREE0;
+      const uint32_t acc_col = (it_prev & 1) ? kColAcc1 : kColAcc0;
+      if (!mbar_wait_warp(bar(acc_done), (it_prev >> 1) & 1, abort_flag)) return false;
+      tc_fence_after();
+      float* orow = p.O + (node0_prev + row) * 128 + hc * 64;
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        uint32_t r1[32];
+        tmem_ld32(tmem + lane_addr + acc_col + hc * 64 + half * 32, r1);
+        tmem_wait_ld();
+        if (row < T) {
+#pragma unroll
+          for (int c = 0; c < 8; ++c) {
+            float4 o;
+            o.x = r_prev * __uint_as_float(r1[4 * c + 0]);
+            o.y = r_prev * __uint_as_float(r1[4 * c + 1]);
+            o.z = r_prev * __uint_as_float(r1[4 * c + 2]);
+            o.w = r_prev * __uint_as_float(r1[4 * c + 3]);
+            *reinterpret_cast<float4*>(orow + half * 32 + 4 * c) = o;
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(acc_free));
+      return true;
+    };
+
+    // metadata of the first item; later items are fetched one item ahead
+    uint64_t nm0 = 0, nm1 = 0;
+    float nla = 0.f;
+    auto fetch_meta = [&](int item) {
+      nm0 = 0; nm1 = 0; nla = 0.f;
+      if (item < p.n_items && row < T) {
+        const int b = (item / p.H) % p.B;
+        const int tb = p.tree.n_trees == 1 ? 0 : b;
+        const uint64_t* m = p.tree.anc + ((size_t)tb * T + row) * 2;
+        nm0 = m[0];
+        nm1 = m[1];
+        nla = log2f(p.alpha[(size_t)item * T + row]);
+      }
+    };
+    fetch_meta(blockIdx.x);
+
     uint32_t it = 0;
+    bool ok = true;
+    size_t node0_prev = 0;
+    float r_prev = 0.f;
     for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++it) {
       const uint32_t ph = it & 1;
-      const int b = (item / p.H) % p.B;
-      const int tb = p.tree.n_trees == 1 ? 0 : b;
       const size_t node0 = (size_t)item * T;
+      uint64_t m0 = nm0, m1 = nm1;
       // ---- path decay: g_i = sum of log2(alpha) over Anc(i) + {i} ----
-      uint64_t m0 = 0, m1 = 0;
-      if (row < T) {
-        const uint64_t* m = p.tree.anc + ((size_t)tb * T + row) * 2;
-        m0 = m[0];
-        m1 = m[1];
-        if (hc == 0) la_s[row] = log2f(p.alpha[node0 + row]);
-      }
+      if (hc == 0 && row < T) la_s[row] = nla;
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(SETUP));
-      if (!mbar_wait_warp(bar(SETUP), 0, abort_flag)) break;   // SETUP completes two phases per item
+      const float la_own = nla;
+      fetch_meta(item + (int)gridDim.x);   // next item's metadata rides under this item's work
+      if (!(ok = mbar_wait_warp(bar(SETUP), 0, abort_flag))) break;   // SETUP: two phases per item
       float g = 0.f;
       if (row < T) {
-        g = la_s[row];
+        g = la_own;
         uint64_t a0 = m0, a1 = m1;
         while (a0) { const int j = __ffsll((long long)a0) - 1; a0 &= a0 - 1; g += la_s[j]; }
         while (a1) { const int j = __ffsll((long long)a1) - 1; a1 &= a1 - 1; g += la_s[64 + j]; }
         if (row < 64) m0 |= 1ull << row; else m1 |= 1ull << (row - 64);   // M+ = M- + I
       }
-      // ---- Q row (bf16, swizzled tile) -> fp32 -> TMEM (A operand of the prefix MMA) ----
-      if (!mbar_wait_warp(bar(QK_FULL), ph, abort_flag)) break;
+      if (hc == 0 && row < T) g_s[row] = g;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(SETUP));
+      // Row scaling.  The accumulator holds  2^e (q_i S_pre^T) + sum_j 2^(e - g_j) s_ij v_j  and
+      // O_i = 2^(g_i - e) acc: e is an integer, so the scaled q stays exact in tf32, and the
+      // exponents e - g_j = (e - g_i) + (g_i - g_j) stay small on ancestor pairs.  Below 2^-100
+      // the prefix term is under fp32 resolution of anything it is added to and is dropped.
+      const bool tiny = g < -100.f;
+      const float e_int = tiny ? g : fminf(rintf(g), 100.f);
+      const float a_scale = tiny ? 0.f : exp2f(e_int);
+      const float r_scale = exp2f(g - e_int);
+      // ---- Q row (bf16, swizzled tile) -> scaled fp32 -> TMEM (A operand of the prefix MMA) ----
+      if (!(ok = mbar_wait_warp(bar(QK_FULL), ph, abort_flag))) break;
+      if (!(ok = mbar_wait_warp(bar(S_FREE), ph ^ 1, abort_flag))) break;   // prefix MMA of item-1 done with Qf
+      tc_fence_after();
       {
         const unsigned char* qrow = sm + kOffQ + hc * kTile + row * 128;
 #pragma unroll
@@ -364,8 +431,8 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             const uint32_t w[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-              r[c * 8 + 2 * e] = w[e] << 16;
-              r[c * 8 + 2 * e + 1] = w[e] & 0xffff0000u;
+              r[c * 8 + 2 * e] = __float_as_uint(a_scale * __uint_as_float(w[e] << 16));
+              r[c * 8 + 2 * e + 1] = __float_as_uint(a_scale * __uint_as_float(w[e] & 0xffff0000u));
             }
           }
           tmem_st32(tmem + lane_addr + kColQf + hc * 64 + half * 32, r);
@@ -378,14 +445,15 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           mbar_arrive(bar(QK_FREE));
         }
       }
-      // every warp needs the g_j of its column half: publish, then synchronise again
-      if (hc == 0 && row < T) g_s[row] = g;
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(SETUP));
-      // ---- scores -> masked, decayed, split C ----
-      if (!mbar_wait_warp(bar(SC_DONE), ph, abort_flag)) break;
+      // ---- scores -> masked, decayed, split C' ----
+      if (!(ok = mbar_wait_warp(bar(SC_DONE), ph, abort_flag))) break;
+      if (!(ok = mbar_wait_warp(bar(SETUP), 1, abort_flag))) break;
+      // the C' tiles are free once the readout MMA of the previous item has completed
+      if (it > 0) {
+        const uint32_t ip = it - 1;
+        if (!(ok = mbar_wait_warp(bar((ip & 1) ? ACC_DONE1 : ACC_DONE0), (ip >> 1) & 1, abort_flag))) break;
+      }
       tc_fence_after();
-      if (!mbar_wait_warp(bar(SETUP), 1, abort_flag)) break;
       if (hc < n_jh) {
         const uint64_t mw = hc == 0 ? m0 : m1;
         unsigned char* chi = sm + kOffChi + hc * kTile + row * 128;
@@ -406,7 +474,7 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
               for (int t = 0; t < 2; ++t) {
                 const int jj = c * 8 + 2 * e + t;
                 const float gj = g_s[hc * 64 + half * 32 + jj];
-                const float ratio = exp2f(g - gj);   // overflow on non-ancestors is selected away
+                const float ratio = exp2f(e_int - gj);   // overflow on non-ancestors is selected away
                 cv[t] = ((bits >> jj) & 1u) ? __uint_as_float(r[jj]) * ratio : 0.f;
               }
               const __nv_bfloat162 h2 = __floats2bfloat162_rn(cv[0], cv[1]);
@@ -427,35 +495,12 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         mbar_arrive(bar(C_READY));
         mbar_arrive(bar(SC_FREE));
       }
-      // ---- O_i = P_i A1_i + A2_i ----
-      if (!mbar_wait_warp(bar(ACC_DONE), ph, abort_flag)) break;
-      tc_fence_after();
-      {
-        const float Pi = exp2f(g);
-        float* orow = p.O + (node0 + row) * 128 + hc * 64;
-#pragma unroll
-        for (int half = 0; half < 2; ++half) {
-          uint32_t r1[32], r2[32];
-          tmem_ld32(tmem + lane_addr + kColA1 + hc * 64 + half * 32, r1);
-          tmem_ld32(tmem + lane_addr + kColA2 + hc * 64 + half * 32, r2);
-          tmem_wait_ld();
-          if (row < T) {
-#pragma unroll
-            for (int c = 0; c < 8; ++c) {
-              float4 o;
-              o.x = fmaf(Pi, __uint_as_float(r1[4 * c + 0]), __uint_as_float(r2[4 * c + 0]));
-              o.y = fmaf(Pi, __uint_as_float(r1[4 * c + 1]), __uint_as_float(r2[4 * c + 1]));
-              o.z = fmaf(Pi, __uint_as_float(r1[4 * c + 2]), __uint_as_float(r2[4 * c + 2]));
-              o.w = fmaf(Pi, __uint_as_float(r1[4 * c + 3]), __uint_as_float(r2[4 * c + 3]));
-              *reinterpret_cast<float4*>(orow + half * 32 + 4 * c) = o;
-            }
-          }
-        }
-      }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(ACC_FREE));
+      // ---- output rows of the previous item (its readout MMA ran under the work above) ----
+      if (it > 0 && !(ok = final_epilogue(it - 1, node0_prev, r_prev))) break;
+      node0_prev = node0;
+      r_prev = r_scale;
     }
+    if (ok && it > 0) final_epilogue(it - 1, node0_prev, r_prev);
   }
 
   // ---- teardown: every path comes here ----
