@@ -46,13 +46,15 @@ constexpr uint32_t kOffChi = kOffS + 4 * kTile;   // 2 tiles: j halves of C_hi [
 constexpr uint32_t kOffClo = kOffChi + 2 * kTile; // 2 tiles: j halves of C_lo
 constexpr uint32_t kOffG = kOffClo + 2 * kTile;   // float g[128]
 constexpr uint32_t kOffAl = kOffG + 512;          // float log2(alpha)[128]
-constexpr uint32_t kOffBar = kOffAl + 512;        // mbarriers
-constexpr uint32_t kOffMisc = kOffBar + 8 * 16;   // tmem base, abort flag
-constexpr uint32_t kSmemBytes = kOffMisc + 16 + 1024;  // + alignment slack
+constexpr uint32_t kOffF = kOffAl + 512;          // float exp2(-g)[128]
+constexpr uint32_t kOffBar = kOffF + 512;         // mbarriers
+constexpr uint32_t kOffMisc = kOffBar + 8 * 24;   // tmem base, abort flag
+constexpr uint32_t kSmemBytes = kOffMisc + 48 + 1024;  // + alignment slack
 
 enum Bar {
   QK_FULL = 0, QK_FREE, S_FULL, S_FREE, V_FULL, V_FREE,
-  SC_DONE, SC_FREE, QF_READY, C_READY, ACC_DONE0, ACC_DONE1, ACC_FREE0, ACC_FREE1, SETUP
+  SC_DONE, SC_FREE, QF_READY, C_READY, ACC_DONE0, ACC_DONE1, ACC_FREE0, ACC_FREE1, SETUP,
+  OST_READY, OST_FREE
 };
 
 // TMEM columns: scaled Q (A operand), scores, two output accumulators
@@ -119,6 +121,15 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
       " [%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
 }
+
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4}], [%1];"
+      ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
 // ---- tcgen05 ----------------------------------------------------------------
 __device__ __forceinline__ void tc_fence_before() {
@@ -188,10 +199,35 @@ __device__ __forceinline__ uint64_t desc_mnmajor(uint32_t saddr, uint32_t lbo) {
          ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
 }
 
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-  __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<uint32_t*>(&t);
+// Eight fp32 values -> bf16 hi and lo parts (hi = upper 16 bits, lo = the exact remainder cut to
+// its upper 16 bits: hi + lo carries 16 mantissa bits), stored as two 16-byte chunks.
+__device__ __forceinline__ void store_split8(unsigned char* chi, unsigned char* clo, uint32_t off,
+                                             const float* cv) {
+  uint32_t hi[4], lo[4];
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const uint32_t x0 = __float_as_uint(cv[2 * e]), x1 = __float_as_uint(cv[2 * e + 1]);
+    const uint32_t h0 = x0 & 0xffff0000u, h1 = x1 & 0xffff0000u;
+    const uint32_t l0 = __float_as_uint(cv[2 * e] - __uint_as_float(h0));
+    const uint32_t l1 = __float_as_uint(cv[2 * e + 1] - __uint_as_float(h1));
+    hi[e] = __byte_perm(x0, x1, 0x7632);   // {x0.hi16, x1.hi16}
+    lo[e] = __byte_perm(l0, l1, 0x7632);
+  }
+  *reinterpret_cast<uint4*>(chi + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+  *reinterpret_cast<uint4*>(clo + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
 }
+
+// Phase timestamps for kernel tuning: compiled out unless TV_TC_PROFILE is defined.
+#ifdef TV_TC_PROFILE
+__device__ long long* g_tc_prof = nullptr;   // [CTA 0 only][item][32] clock64 stamps
+#define TC_STAMP(it, slot)                                                        \
+  do {                                                                            \
+    if (g_tc_prof && blockIdx.x == 0 && (it) < 16 && lane == 0)                   \
+      g_tc_prof[(it) * 32 + (slot)] = clock64();                                  \
+  } while (0)
+#else
+#define TC_STAMP(it, slot) do { } while (0)
+#endif
 
 struct TcParams {
   TreeDev tree;
@@ -204,12 +240,14 @@ struct TcParams {
 __global__ void __launch_bounds__(kThreads, 1)
 verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                        const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmS,
-                       const TcParams p) {
+                       const __grid_constant__ CUtensorMap tmO, const TcParams p) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* sm = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   const uint32_t sbase = smem_u32(sm);
   float* g_s = reinterpret_cast<float*>(sm + kOffG);
   float* la_s = reinterpret_cast<float*>(sm + kOffAl);
+  float* f_s = reinterpret_cast<float*>(sm + kOffF);
+  volatile int* range_ok_s = reinterpret_cast<volatile int*>(sm + kOffMisc + 16);   // [8] per compute warp
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + kOffMisc);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + kOffMisc + 4);
   auto bar = [&](int i) { return sbase + kOffBar + 8u * i; };
@@ -230,6 +268,8 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     mbar_init(bar(ACC_DONE0), 1); mbar_init(bar(ACC_DONE1), 1);
     mbar_init(bar(ACC_FREE0), kComputeWarps); mbar_init(bar(ACC_FREE1), kComputeWarps);
     mbar_init(bar(SETUP), kComputeWarps);
+    mbar_init(bar(OST_READY), kComputeWarps);
+    mbar_init(bar(OST_FREE), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -250,6 +290,7 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++it) {
         const uint32_t ph = it & 1;
         if (!mbar_wait(bar(QK_FREE), ph ^ 1, abort_flag)) break;
+        TC_STAMP(it, 0);
         mbar_expect_tx(bar(QK_FULL), 4 * kTile);
         tma_load_3d(sbase + kOffQ, &tmQ, bar(QK_FULL), 0, 0, item);
         tma_load_3d(sbase + kOffQ + kTile, &tmQ, bar(QK_FULL), 64, 0, item);
@@ -257,12 +298,14 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         tma_load_3d(sbase + kOffK + kTile, &tmK, bar(QK_FULL), 64, 0, item);
         pend_qk = 1 + (int)ph;
         if (!mbar_wait(bar(S_FREE), ph ^ 1, abort_flag)) break;
+        TC_STAMP(it, 1);
         mbar_expect_tx(bar(S_FULL), 4 * kTile);
 #pragma unroll
         for (int c = 0; c < 4; ++c)
           tma_load_3d(sbase + kOffS + c * kTile, &tmS, bar(S_FULL), 32 * c, 0, item);
         pend_s = 1 + (int)ph;
         if (!mbar_wait(bar(V_FREE), ph ^ 1, abort_flag)) break;
+        TC_STAMP(it, 2);
         mbar_expect_tx(bar(V_FULL), 2 * kTile);
         tma_load_3d(sbase + kOffV, &tmV, bar(V_FULL), 0, 0, item);
         tma_load_3d(sbase + kOffV + kTile, &tmV, bar(V_FULL), 64, 0, item);
@@ -287,7 +330,9 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         const uint32_t ph2 = (it >> 1) & 1;   // the two accumulators alternate
         // scores = Q K^T
         if (!mbar_wait(bar(QK_FULL), ph, abort_flag)) break;
+        TC_STAMP(it, 4);
         if (!mbar_wait(bar(SC_FREE), ph ^ 1, abort_flag)) break;
+        TC_STAMP(it, 5);
         tc_fence_after();
 #pragma unroll
         for (int h = 0; h < 2; ++h)
@@ -299,8 +344,11 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         tc_commit(bar(QK_FREE));
         // acc = (2^e Q) S_pre^T  (A = scaled Q as fp32 in TMEM, B = S_pre chunks)
         if (!mbar_wait(bar(S_FULL), ph, abort_flag)) break;
+        TC_STAMP(it, 6);
         if (!mbar_wait(bar(QF_READY), ph, abort_flag)) break;
+        TC_STAMP(it, 7);
         if (!mbar_wait(bar(acc_free), ph2 ^ 1, abort_flag)) break;
+        TC_STAMP(it, 8);
         tc_fence_after();
 #pragma unroll
         for (int c = 0; c < 4; ++c)
@@ -311,7 +359,9 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         tc_commit(bar(S_FREE));
         // acc += C'_hi V + C'_lo V
         if (!mbar_wait(bar(C_READY), ph, abort_flag)) break;
+        TC_STAMP(it, 9);
         if (!mbar_wait(bar(V_FULL), ph, abort_flag)) break;
+        TC_STAMP(it, 10);
         tc_fence_after();
         for (int jh = 0; jh < n_jh; ++jh)
 #pragma unroll
@@ -324,6 +374,7 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           }
         tc_commit(bar(V_FREE));
         tc_commit(bar(acc_done));
+        TC_STAMP(it, 11);
       }
     }
   } else {
@@ -334,21 +385,24 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     const int row = quad * 32 + lane;   // node i
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
     const uint32_t swz = (uint32_t)(row & 7);
+    const bool warp_live = quad * 32 < T;   // this warp's 32 rows hold at least one node
 
-    // O_i = r_i acc_i for the item whose accumulator is `it_prev`.
-    auto final_epilogue = [&](uint32_t it_prev, size_t node0_prev, float r_prev) -> bool {
+    // O_i = r_i acc_i for the item whose accumulator is `it_prev`: TMEM -> registers -> the
+    // (now idle) C' tiles as four [128 rows][32 fp32] swizzled tiles -> one TMA store per tile
+    // (full 128-byte lines; rows past T are clipped by the tensor map).
+    auto final_epilogue = [&](uint32_t it_prev, int item_prev, float r_prev, uint32_t ost_phase) -> bool {
       const int acc_done = (it_prev & 1) ? ACC_DONE1 : ACC_DONE0;
       const int acc_free = (it_prev & 1) ? ACC_FREE1 : ACC_FREE0;
       const uint32_t acc_col = (it_prev & 1) ? kColAcc1 : kColAcc0;
       if (!mbar_wait_warp(bar(acc_done), (it_prev >> 1) & 1, abort_flag)) return false;
       tc_fence_after();
-      float* orow = p.O + (node0_prev + row) * 128 + hc * 64;
+      if (warp_live) {
 #pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        uint32_t r1[32];
-        tmem_ld32(tmem + lane_addr + acc_col + hc * 64 + half * 32, r1);
-        tmem_wait_ld();
-        if (row < T) {
+        for (int half = 0; half < 2; ++half) {
+          uint32_t r1[32];
+          tmem_ld32(tmem + lane_addr + acc_col + hc * 64 + half * 32, r1);
+          tmem_wait_ld();
+          unsigned char* orow = sm + kOffChi + (hc * 2 + half) * kTile + row * 128;
 #pragma unroll
           for (int c = 0; c < 8; ++c) {
             float4 o;
@@ -356,45 +410,58 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             o.y = r_prev * __uint_as_float(r1[4 * c + 1]);
             o.z = r_prev * __uint_as_float(r1[4 * c + 2]);
             o.w = r_prev * __uint_as_float(r1[4 * c + 3]);
-            *reinterpret_cast<float4*>(orow + half * 32 + 4 * c) = o;
+            *reinterpret_cast<float4*>(orow + (((uint32_t)c ^ swz) << 4)) = o;
           }
         }
       }
+      fence_async_smem();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar(acc_free));
-      return true;
+      if (lane == 0) {
+        mbar_arrive(bar(acc_free));
+        mbar_arrive(bar(OST_READY));
+      }
+      if (warp == 2 && lane == 0) {
+        if (mbar_wait(bar(OST_READY), ost_phase, abort_flag)) {
+#pragma unroll
+          for (int c = 0; c < 4; ++c) tma_store_3d(&tmO, sbase + kOffChi + c * kTile, 32 * c, 0, item_prev);
+          tma_store_commit();
+          tma_store_wait_read();   // the tiles may be overwritten once the store has read them
+        }
+        mbar_arrive(bar(OST_FREE));
+      }
+      return mbar_wait_warp(bar(OST_FREE), ost_phase, abort_flag);
     };
 
     // metadata of the first item; later items are fetched one item ahead
     uint64_t nm0 = 0, nm1 = 0;
-    float nla = 0.f;
+    float nal = 1.f;   // raw decay gate of the next item (log2 taken when it is used)
     auto fetch_meta = [&](int item) {
-      nm0 = 0; nm1 = 0; nla = 0.f;
+      nm0 = 0; nm1 = 0; nal = 1.f;
       if (item < p.n_items && row < T) {
         const int b = (item / p.H) % p.B;
         const int tb = p.tree.n_trees == 1 ? 0 : b;
         const uint64_t* m = p.tree.anc + ((size_t)tb * T + row) * 2;
         nm0 = m[0];
         nm1 = m[1];
-        nla = log2f(p.alpha[(size_t)item * T + row]);
+        nal = p.alpha[(size_t)item * T + row];
       }
     };
     fetch_meta(blockIdx.x);
 
     uint32_t it = 0;
     bool ok = true;
-    size_t node0_prev = 0;
+    int item_prev = 0;
     float r_prev = 0.f;
     for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++it) {
       const uint32_t ph = it & 1;
-      const size_t node0 = (size_t)item * T;
       uint64_t m0 = nm0, m1 = nm1;
+      if (warp == 4) TC_STAMP(it, 16);
       // ---- path decay: g_i = sum of log2(alpha) over Anc(i) + {i} ----
-      if (hc == 0 && row < T) la_s[row] = nla;
+      const float la_own = log2f(nal);
+      if (hc == 0 && row < T) la_s[row] = la_own;
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(SETUP));
-      const float la_own = nla;
       fetch_meta(item + (int)gridDim.x);   // next item's metadata rides under this item's work
       if (!(ok = mbar_wait_warp(bar(SETUP), 0, abort_flag))) break;   // SETUP: two phases per item
       float g = 0.f;
@@ -405,7 +472,13 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         while (a1) { const int j = __ffsll((long long)a1) - 1; a1 &= a1 - 1; g += la_s[64 + j]; }
         if (row < 64) m0 |= 1ull << row; else m1 |= 1ull << (row - 64);   // M+ = M- + I
       }
-      if (hc == 0 && row < T) g_s[row] = g;
+      if (hc == 0 && row < T) {
+        g_s[row] = g;
+        f_s[row] = exp2f(-g);
+      }
+      // exp2(e_i - g_j) = 2^e_i * 2^-g_j is safe when every |g| <= 100; otherwise take exp2 per pair
+      const bool range_ok_warp = __all_sync(0xffffffffu, row >= T || fabsf(g) <= 100.f);
+      if (lane == 0) range_ok_s[cw] = range_ok_warp;
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(SETUP));
       // Row scaling.  The accumulator holds  2^e (q_i S_pre^T) + sum_j 2^(e - g_j) s_ij v_j  and
@@ -417,10 +490,12 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       const float a_scale = tiny ? 0.f : exp2f(e_int);
       const float r_scale = exp2f(g - e_int);
       // ---- Q row (bf16, swizzled tile) -> scaled fp32 -> TMEM (A operand of the prefix MMA) ----
+      if (warp == 4) TC_STAMP(it, 17);
       if (!(ok = mbar_wait_warp(bar(QK_FULL), ph, abort_flag))) break;
       if (!(ok = mbar_wait_warp(bar(S_FREE), ph ^ 1, abort_flag))) break;   // prefix MMA of item-1 done with Qf
+      if (warp == 4) TC_STAMP(it, 18);
       tc_fence_after();
-      {
+      if (warp_live) {
         const unsigned char* qrow = sm + kOffQ + hc * kTile + row * 128;
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
@@ -438,53 +513,62 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           tmem_st32(tmem + lane_addr + kColQf + hc * 64 + half * 32, r);
         }
         tmem_wait_st();
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) {
-          mbar_arrive(bar(QF_READY));
-          mbar_arrive(bar(QK_FREE));
-        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) {
+        mbar_arrive(bar(QF_READY));
+        mbar_arrive(bar(QK_FREE));
       }
       // ---- scores -> masked, decayed, split C' ----
+      if (warp == 4) TC_STAMP(it, 19);
       if (!(ok = mbar_wait_warp(bar(SC_DONE), ph, abort_flag))) break;
+      if (warp == 4) TC_STAMP(it, 20);
       if (!(ok = mbar_wait_warp(bar(SETUP), 1, abort_flag))) break;
-      // the C' tiles are free once the readout MMA of the previous item has completed
-      if (it > 0) {
-        const uint32_t ip = it - 1;
-        if (!(ok = mbar_wait_warp(bar((ip & 1) ? ACC_DONE1 : ACC_DONE0), (ip >> 1) & 1, abort_flag))) break;
-      }
+      // ---- output rows of the previous item: its accumulator is complete once its readout MMA
+      // is, and the C' tiles it frees double as the staging area of the output store ----
+      if (it > 0 && !(ok = final_epilogue(it - 1, item_prev, r_prev, (it - 1) & 1))) break;
       tc_fence_after();
-      if (hc < n_jh) {
-        const uint64_t mw = hc == 0 ? m0 : m1;
-        unsigned char* chi = sm + kOffChi + hc * kTile + row * 128;
-        unsigned char* clo = sm + kOffClo + hc * kTile + row * 128;
+      if (warp == 4) TC_STAMP(it, 21);
+      if (warp_live) {
+        bool fast = true;
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
+        for (int w8 = 0; w8 < kComputeWarps; ++w8) fast = fast && range_ok_s[w8];
+        // this warp covers 32 n_jh of the 64 n_jh real columns, 32 at a time
+        for (int h = 0; h < n_jh; ++h) {
+          const int cbase = hc * 32 * n_jh + h * 32;     // first column j of this group
           uint32_t r[32];
-          tmem_ld32(tmem + lane_addr + kColSc + hc * 64 + half * 32, r);
+          tmem_ld32(tmem + lane_addr + kColSc + cbase, r);
           tmem_wait_ld();
-          const uint32_t bits = (uint32_t)(mw >> (half * 32));
+          const uint32_t bits = cbase < 64 ? (uint32_t)(m0 >> cbase) : (uint32_t)(m1 >> (cbase - 64));
+          unsigned char* chi = sm + kOffChi + (cbase >> 6) * kTile + row * 128;
+          unsigned char* clo = sm + kOffClo + (cbase >> 6) * kTile + row * 128;
+          const int chunk0 = (cbase & 63) >> 3;
+          if (fast) {
 #pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            uint32_t hi[4], lo[4];
+            for (int c = 0; c < 4; ++c) {
+              const float4 fa = *reinterpret_cast<const float4*>(f_s + cbase + c * 8);
+              const float4 fb = *reinterpret_cast<const float4*>(f_s + cbase + c * 8 + 4);
+              const float f8[8] = {fa.x, fa.y, fa.z, fa.w, fb.x, fb.y, fb.z, fb.w};
+              float cv[8];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              float cv[2];
-#pragma unroll
-              for (int t = 0; t < 2; ++t) {
-                const int jj = c * 8 + 2 * e + t;
-                const float gj = g_s[hc * 64 + half * 32 + jj];
-                const float ratio = exp2f(e_int - gj);   // overflow on non-ancestors is selected away
-                cv[t] = ((bits >> jj) & 1u) ? __uint_as_float(r[jj]) * ratio : 0.f;
+              for (int e = 0; e < 8; ++e) {
+                const float x = __uint_as_float(r[c * 8 + e]) * (a_scale * f8[e]);
+                cv[e] = ((bits >> (c * 8 + e)) & 1u) ? x : 0.f;   // select, never 0 * x
               }
-              const __nv_bfloat162 h2 = __floats2bfloat162_rn(cv[0], cv[1]);
-              const float2 hf = __bfloat1622float2(h2);
-              hi[e] = *reinterpret_cast<const uint32_t*>(&h2);
-              lo[e] = pack_bf16(cv[0] - hf.x, cv[1] - hf.y);
+              store_split8(chi, clo, ((uint32_t)((chunk0 + c) ^ swz)) << 4, cv);
             }
-            const uint32_t off = ((uint32_t)((half * 4 + c) ^ swz)) << 4;
-            *reinterpret_cast<uint4*>(chi + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-            *reinterpret_cast<uint4*>(clo + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+          } else {
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+              float cv[8];
+#pragma unroll
+              for (int e = 0; e < 8; ++e) {
+                const float x = __uint_as_float(r[c * 8 + e]) * exp2f(e_int - g_s[cbase + c * 8 + e]);
+                cv[e] = ((bits >> (c * 8 + e)) & 1u) ? x : 0.f;
+              }
+              store_split8(chi, clo, ((uint32_t)((chunk0 + c) ^ swz)) << 4, cv);
+            }
           }
         }
       }
@@ -495,12 +579,12 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         mbar_arrive(bar(C_READY));
         mbar_arrive(bar(SC_FREE));
       }
-      // ---- output rows of the previous item (its readout MMA ran under the work above) ----
-      if (it > 0 && !(ok = final_epilogue(it - 1, node0_prev, r_prev))) break;
-      node0_prev = node0;
+      if (warp == 4) TC_STAMP(it, 22);
+      item_prev = item;
       r_prev = r_scale;
     }
-    if (ok && it > 0) final_epilogue(it - 1, node0_prev, r_prev);
+    if (ok && it > 0) final_epilogue(it - 1, item_prev, r_prev, (it - 1) & 1);
+    if (warp == 2 && lane == 0) tma_store_wait_all();   // our stores are complete before we leave
   }
 
   // ---- teardown: every path comes here ----
@@ -562,6 +646,12 @@ __global__ void widen_bf16_kernel(const __nv_bfloat16* __restrict__ v, float* __
 
 }  // namespace
 
+#ifdef TV_TC_PROFILE
+extern "C" __attribute__((visibility("default"))) int tv_debug_set_tc_profile(long long* dev_buf) {
+  return cudaMemcpyToSymbol(g_tc_prof, &dev_buf, sizeof(dev_buf)) == cudaSuccess ? 0 : -4;
+}
+#endif
+
 bool tv_verify_tc_supports(const VerifyArgs& a) {
   return a.bf16 && a.dk == 128 && a.dv == 128 && a.rule == TV_GATED && a.T <= 128;
 }
@@ -569,11 +659,12 @@ bool tv_verify_tc_supports(const VerifyArgs& a) {
 int tv_launch_verify_tc(const VerifyArgs& a, int32_t* status, cudaStream_t stream) {
   if (!tv_verify_tc_supports(a)) return TV_ERR_UNSUPPORTED;
   const uint64_t items = (uint64_t)a.L * a.B * a.H;
-  alignas(64) CUtensorMap tmQ, tmK, tmV, tmS;
+  alignas(64) CUtensorMap tmQ, tmK, tmV, tmS, tmO;
   if (!make_map(&tmQ, a.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, items, a.T, 128, 64) ||
       !make_map(&tmK, a.k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, items, a.T, 128, 64) ||
       !make_map(&tmV, a.v, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, items, a.T, 128, 64) ||
-      !make_map(&tmS, a.S_pre, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, 128, 128, 32))
+      !make_map(&tmS, a.S_pre, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, 128, 128, 32) ||
+      !make_map(&tmO, a.O, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, a.T, 128, 32))
     return TV_ERR_CUDA;
   static thread_local int configured_dev = -1;
   static thread_local int sm_count = 0;
@@ -593,7 +684,7 @@ int tv_launch_verify_tc(const VerifyArgs& a, int32_t* status, cudaStream_t strea
   p.O = a.O;
   p.status = status;
   const int grid = (int)(items < (uint64_t)sm_count ? items : (uint64_t)sm_count);
-  verify_tc_gated_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tmQ, tmK, tmV, tmS, p);
+  verify_tc_gated_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tmQ, tmK, tmV, tmS, tmO, p);
   TV_CUDA_TRY(cudaGetLastError());
   if (a.U) {
     const size_t n8 = items * a.T * 128 / 8;

@@ -36,3 +36,19 @@ def test_tc_error_budget_report():
     errs = np.concatenate(errs)
     print(f"TC c3 per-node rel-L2: mean {errs.mean():.3e} max {errs.max():.3e}")
     assert errs.max() <= wl.tol
+
+
+@pytest.mark.parametrize("impl", [tv.IMPL_SIMT, tv.IMPL_TC])
+@pytest.mark.parametrize("tree,mu", [("chain", -2.0), ("spine", -3.0), ("frontier", 8.0)])
+def test_extreme_decay(tree, mu, impl):
+    """Strong decay (path products far below fp32 range) and no decay at all:
+    decay ratios are only ever formed on ancestor pairs, so nothing overflows."""
+    wl = inputs.workload("c5", B=2, H=2, T=128, L=1, tree=tree, seed=77, alpha_mu=mu, alpha_sd=1.0)
+    parents, accepted = inputs.make_trees(wl)
+    tens = inputs.make_tensors(wl)
+    O, U, Sn, _ = pu.gpu_round(wl, parents, accepted, tens, impl=impl, want_U=False)
+    assert np.isfinite(O).all() and np.isfinite(Sn).all()
+    ver, com = pu.oracle_round(wl, parents, accepted, tens)
+    eO, _, eS = pu.compare(wl, O, None, Sn, ver, com)
+    print(f"decay mu={mu} {tree} impl={impl}: rel-L2 O {eO:.3e} S {eS:.3e}")
+    assert eO <= wl.tol and eS <= wl.tol
