@@ -77,6 +77,15 @@ def accepted_lengths(parents, accepted):
     return np.array(out)
 
 
+def ncu_traffic(workload: str):
+    """DRAM bytes per verify launch from the committed ncu capture of this workload, if any."""
+    p = os.path.join(ROOT, "profiles", "traffic.json")
+    try:
+        return json.load(open(p)).get(workload, {}).get("tree_verify")
+    except Exception:
+        return None
+
+
 def _jsonable(o):
     return o.item() if hasattr(o, "item") else str(o)
 
@@ -350,12 +359,18 @@ def run_ours(args, wl, rank, world, local_rank):
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
-        nb = min(wl.B, 8)
-        small = inputs.workload(wl.name, B=nb, L=1, seed=wl.seed)
-        tens = inputs.make_tensors(small)
-        v, done, dt, threads = oracle_sample(small, parents[:nb] if parents.shape[0] > 1 else parents,
-                                             accepted[:nb], tens, args.cpu_budget, nb * wl.H)
-        cpu = {"value": v, "unit": "nodes/s", "cores": threads, "kind": "oracle",
+        # the oracle on whole requests of this workload, layer after layer, until the budget is spent
+        nb = min(wl.B, 32)
+        done, dt, threads, layer = 0, 0.0, 1, 0
+        while dt < args.cpu_budget and layer < 64:
+            small = inputs.workload(wl.name, B=nb, L=1, seed=wl.seed)
+            tens = inputs.make_tensors(small, layer=layer)
+            _, d1, t1, threads = oracle_sample(small, parents[:nb] if parents.shape[0] > 1 else parents,
+                                               accepted[:nb], tens, args.cpu_budget - dt, nb * wl.H)
+            done += d1
+            dt += t1
+            layer += 1
+        cpu = {"value": done * wl.T / wl.H / dt, "unit": "nodes/s", "cores": threads, "kind": "oracle",
                "sample": f"{done} (request, head) items of the workload (memoised fp64 walk of all "
                          f"{wl.T} nodes + commit), {dt:.1f} s"}
 
@@ -377,7 +392,7 @@ def run_ours(args, wl, rank, world, local_rank):
                    "frac_of_measured_copy": c_gbs / peak, "frac_of_nominal_8TBps": c_gbs / NOMINAL_HBM_GBS},
         "roofline": {"kernel": "tree_verify", "bound": "hbm", "achieved": v_gbs, "peak": peak,
                      "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": v_gbs / peak,
-                     "traffic": args.traffic},
+                     "traffic": args.traffic if args.traffic is not None else ncu_traffic(wl.name)},
         "cpu_baseline": cpu,
         "e2e": None if e2e is None else {
             "value": wl.B * wl.T * e2e_L * world / e2e[0], "unit": "nodes/s",
@@ -393,14 +408,14 @@ def run_ours(args, wl, rank, world, local_rank):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="c3", choices=sorted(DESCR))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--kernel", default="auto", choices=["auto", "simt", "tc"])
     ap.add_argument("--layers", type=int, default=0, help="override layers per step")
     ap.add_argument("--sets", type=int, default=0, help="override number of rotating input sets")
-    ap.add_argument("--cpu-budget", type=float, default=15.0)
+    ap.add_argument("--cpu-budget", type=float, default=12.0)
     ap.add_argument("--ref-items", type=int, default=8)
     ap.add_argument("--traffic", type=float, default=None,
                     help="ncu dram bytes per verify launch to echo into roofline.traffic")
