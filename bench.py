@@ -225,6 +225,30 @@ def run_reference(args, wl, rank, world):
 
 
 # --------------------------------------------------------------------------
+# Multi-GPU bookkeeping (weak scaling, no data-path collective)
+# --------------------------------------------------------------------------
+def rank_workload(wl, rank: int, layers: int = 0):
+    """Every rank verifies its own batch of requests: same shapes, its own seed."""
+    import dataclasses
+    return dataclasses.replace(wl, seed=wl.seed + 101 * rank, L=layers or wl.L)
+
+
+def max_over_ranks(values, world: int, device):
+    """Element-wise maximum of per-rank timings (the slowest rank sets the job's time)."""
+    if world <= 1:
+        return [float(v) for v in values]
+    import torch.distributed as dist
+    t = torch.tensor(list(values), device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t.tolist()]
+
+
+def job_nodes_per_step(wl, world: int) -> int:
+    """Units processed by all ranks in one step (weak scaling: per-rank work is fixed)."""
+    return wl.B * wl.T * wl.L * world
+
+
+# --------------------------------------------------------------------------
 # The CUDA path
 # --------------------------------------------------------------------------
 def run_ours(args, wl, rank, world, local_rank):
@@ -236,7 +260,7 @@ def run_ours(args, wl, rank, world, local_rank):
         raise RuntimeError("bench.py needs a CUDA device: there is no CPU fallback")
     torch.cuda.set_device(local_rank)
     dev = f"cuda:{local_rank}"
-    wl = inputs.workload(wl.name, seed=wl.seed + 101 * rank, L=args.layers or wl.L)
+    wl = rank_workload(wl, rank, args.layers)
     parents, accepted = inputs.make_trees(wl)
     acc_len = accepted_lengths(parents, accepted)
     delta = wl.rule == inputs.DELTA
@@ -339,17 +363,14 @@ def run_ours(args, wl, rank, world, local_rank):
         del hs, hO, hS
 
     # ---- max over ranks -----------------------------------------------------
-    if world > 1:
-        t = torch.tensor([total_ms, v_ms, c_ms, e2e[0] if e2e else 0.0], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, v_ms, c_ms, e2e_dt = [float(x) for x in t.tolist()]
-        if e2e:
-            e2e[0] = e2e_dt
+    total_ms, v_ms, c_ms, e2e_dt = max_over_ranks([total_ms, v_ms, c_ms, e2e[0] if e2e else 0.0], world, dev)
+    if e2e:
+        e2e[0] = e2e_dt
     if rank != 0:
         return
 
     ms_per_step = total_ms / args.steps
-    nodes_step = wl.B * wl.T * wl.L * world
+    nodes_step = job_nodes_per_step(wl, world)
     value = nodes_step / (ms_per_step * 1e-3)
     peak, peak_kind = measured_peak()
     vbytes = verify_bytes_per_layer(wl, with_U=delta)
