@@ -112,11 +112,17 @@ int tv_tree_info(const tv_tree* tree, int32_t* n_trees, int32_t* n,
  * unused entries set to -1; len is host int32 [n_req].                        */
 int tv_tree_path(const tv_tree* tree, const int32_t* accepted, int32_t n_req,
                  int32_t* path, int32_t path_stride, int32_t* len);
-/* Copy the metadata to the current device on `stream` (a cudaStream_t).  The
- * first call allocates the device mirror and a pinned staging block; later
- * calls (after tv_tree_rebuild) only copy.  The copy is asynchronous; kernels
- * launched later on the same stream see it.                                   */
+/* Put the metadata on the current device, on `stream` (a cudaStream_t): the
+ * parent arrays are staged in pinned host memory and one small kernel derives
+ * the same masks and depths on the device (Section IV-C: once per request and
+ * round, fixed buffers).  The first call allocates the device mirror and the
+ * staging block; later calls (after tv_tree_rebuild) allocate nothing.
+ * Asynchronous; kernels launched later on the same stream see the result.     */
 int tv_tree_upload(tv_tree* tree, void* stream);
+/* Copy the DEVICE-built masks and depths back to host arrays (same shapes as
+ * tv_tree_meta) and synchronise `stream`: lets a caller check them bit for bit
+ * against tv_tree_meta.                                                       */
+int tv_tree_meta_device(tv_tree* tree, uint64_t* anc, int32_t* depth, void* stream);
 /* Synchronises `stream` and reports whether any kernel launched with this tree
  * since its last upload gave up on a bounded device-side wait (a TMA or tensor-
  * core completion that never came): TV_OK or TV_ERR_DEVICE_TIMEOUT.  After a

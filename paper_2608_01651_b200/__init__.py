@@ -60,6 +60,8 @@ def lib() -> ctypes.CDLL:
     L.tv_tree_upload.argtypes = [vp, vp]
     L.tv_tree_free.argtypes = [vp]
     L.tv_tree_device_status.argtypes = [vp, vp]
+    L.tv_tree_meta_device.argtypes = [vp, vp, vp, vp]
+    L.tv_tree_meta_device.restype = ctypes.c_int
     L.tv_tree_device_status.restype = ctypes.c_int
     L.tv_tree_verify.argtypes = [vp, p(_Dims)] + [vp] * 9
     L.tv_commit_path.argtypes = [vp, p(_Dims)] + [vp] * 9
@@ -106,6 +108,14 @@ class Tree:
                "tv_tree_meta")
         return anc, depth, md
 
+    def meta_device(self, stream=None):
+        """``tv_tree_meta_device``: the masks and depths as built on the device."""
+        anc = np.zeros((self.n_trees, self.n, 2), dtype=np.uint64)
+        depth = np.zeros((self.n_trees, self.n), dtype=np.int32)
+        _check(lib().tv_tree_meta_device(self._h, anc.ctypes.data, depth.ctypes.data, _stream_ptr(stream)),
+               "tv_tree_meta_device")
+        return anc, depth
+
     @property
     def max_depth(self) -> int:
         md = ctypes.c_int32()
@@ -125,6 +135,25 @@ class Tree:
     def upload(self, stream=None):
         _check(lib().tv_tree_upload(self._h, _stream_ptr(stream)), "tv_tree_upload")
         return self
+
+    def prepare_refresh(self, parent, stream=None):
+        """``tv_tree_rebuild`` + ``tv_tree_upload`` with pre-marshalled arguments: returns a
+        callable that re-reads ``parent`` (an int32 C-contiguous numpy array that the caller
+        updates in place) and uploads the new metadata."""
+        par = np.asarray(parent)
+        if par.dtype != np.int32 or not par.flags["C_CONTIGUOUS"] or par.size != self.n_trees * self.n:
+            raise ValueError("parent must be a C-contiguous int32 array of n_trees * n entries")
+        L = lib()
+        h, pp, sp = self._h, ctypes.c_void_p(par.ctypes.data), _stream_ptr(stream)
+        rebuild, upload = L.tv_tree_rebuild, L.tv_tree_upload
+
+        def refresh(_keep=(par, self)):
+            st = rebuild(h, pp)
+            if st == 0:
+                st = upload(h, sp)
+            if st != 0:
+                raise TreeVerifyError(st, "tv_tree_rebuild/tv_tree_upload")
+        return refresh
 
     def device_status(self, stream=None):
         """``tv_tree_device_status``: synchronise and raise if a device wait timed out."""
@@ -240,6 +269,53 @@ def commit_path(tree: Tree, accepted, S_pre, k, v, alpha, beta=None, *, rule=GAT
                                 _ptr(v), _ptr(alpha), _ptr(beta), _ptr(U), _ptr(out),
                                 _stream_ptr(stream)), "tv_commit_path")
     return out
+
+
+class Prepared:
+    """A C-ABI call with its arguments marshalled once (for loops that repeat the same call:
+    validation and ctypes conversion are paid at construction, the call itself is one foreign
+    call).  Holds references to every tensor it points into."""
+
+    def __init__(self, fn, name, args, keep):
+        self._fn, self._name, self._args, self._keep = fn, name, args, keep
+
+    def __call__(self):
+        st = self._fn(*self._args)
+        if st != 0:
+            raise TreeVerifyError(st, self._name)
+
+
+def prepare_tree_verify(tree: Tree, S_pre, q, k, v, alpha, beta=None, *, rule=GATED, O=None, U=None,
+                        impl=IMPL_AUTO, stream=None) -> Prepared:
+    """``tv_tree_verify`` with pre-marshalled arguments; ``O`` (and ``U``) must be given."""
+    import torch
+    for t, n in ((S_pre, "S_pre"), (alpha, "alpha"), (beta, "beta"), (O, "O"), (U, "U")):
+        _require(t, n, torch.float32)
+    for t, n in ((q, "q"), (k, "k"), (v, "v")):
+        _require(t, n, k.dtype)
+    if O is None:
+        raise ValueError("O must be preallocated")
+    d = _dims(S_pre, k, v, rule, impl)
+    args = (tree._h, ctypes.byref(d), _ptr(S_pre), _ptr(q), _ptr(k), _ptr(v), _ptr(alpha), _ptr(beta),
+            _ptr(O), _ptr(U), _stream_ptr(stream))
+    return Prepared(lib().tv_tree_verify, "tv_tree_verify", args, (tree, d, S_pre, q, k, v, alpha, beta, O, U))
+
+
+def prepare_commit_path(tree: Tree, accepted, S_pre, k, v, alpha, beta=None, *, rule=GATED, U=None,
+                        S_new=None, stream=None) -> Prepared:
+    """``tv_commit_path`` with pre-marshalled arguments (in place when ``S_new`` is None)."""
+    import torch
+    _require(accepted, "accepted", torch.int32)
+    for t, n in ((S_pre, "S_pre"), (alpha, "alpha"), (beta, "beta"), (U, "U"), (S_new, "S_new")):
+        _require(t, n, torch.float32)
+    for t, n in ((k, "k"), (v, "v")):
+        _require(t, n, k.dtype)
+    d = _dims(S_pre, k, v, rule, IMPL_AUTO)
+    out = S_pre if S_new is None else S_new
+    args = (tree._h, ctypes.byref(d), _ptr(accepted), _ptr(S_pre), _ptr(k), _ptr(v), _ptr(alpha),
+            _ptr(beta), _ptr(U), _ptr(out), _stream_ptr(stream))
+    return Prepared(lib().tv_commit_path, "tv_commit_path", args,
+                    (tree, d, accepted, S_pre, k, v, alpha, beta, U, out))
 
 
 class Session:

@@ -151,39 +151,61 @@ TV_API int tv_tree_upload(tv_tree* t, void* stream) {
   const size_t anc_b = nn * 2 * sizeof(uint64_t), i32_b = nn * sizeof(int32_t);
   const size_t meta_b = anc_b + 2 * i32_b;
   const size_t total = ((meta_b + 15) & ~(size_t)15) + 16;  // + status word
+  const size_t slot_b = (i32_b + 255) & ~(size_t)255;       // one staged copy of the parent arrays
   int dev = 0;
   TV_CUDA_TRY(cudaGetDevice(&dev));
   if (t->d_blob && (t->device != dev || t->blob_bytes != total)) return TV_ERR_BAD_ARG;
   if (!t->d_blob) {
     TV_CUDA_TRY(cudaMalloc(&t->d_blob, total));
-    cudaError_t e = cudaMallocHost(&t->h_stage, total);
+    cudaError_t e = cudaHostAlloc(&t->h_stage, 2 * slot_b, cudaHostAllocMapped);
+    void* mapped = nullptr;
+    if (e == cudaSuccess) e = cudaHostGetDevicePointer(&mapped, t->h_stage, 0);
+    for (int i = 0; i < 2 && e == cudaSuccess; ++i)
+      e = cudaEventCreateWithFlags(&t->staged[i], cudaEventDisableTiming);
     if (e != cudaSuccess) {
       cudaFree(t->d_blob);
       t->d_blob = nullptr;
+      if (t->h_stage) cudaFreeHost(t->h_stage);
+      t->h_stage = nullptr;
       tv_set_cuda_error(e);
       return TV_ERR_CUDA;
     }
+    t->h_stage_dev = (const int32_t*)mapped;
     t->blob_bytes = total;
     t->device = dev;
     char* base = (char*)t->d_blob;
-    t->d_anc = (const uint64_t*)base;
-    t->d_depth = (const int32_t*)(base + anc_b);
-    t->d_parent = (const int32_t*)(base + anc_b + i32_b);
+    t->d_anc_w = (uint64_t*)base;
+    t->d_depth_w = (int32_t*)(base + anc_b);
+    t->d_parent_w = (int32_t*)(base + anc_b + i32_b);
+    t->d_anc = t->d_anc_w;
+    t->d_depth = t->d_depth_w;
+    t->d_parent = t->d_parent_w;
     t->d_status = (int32_t*)(base + total - 16);
   }
   cudaStream_t s = (cudaStream_t)stream;
-  // The staging block may still be in flight from an earlier upload: wait for
-  // that copy only, not for the stream.
-  if (t->staged) TV_CUDA_TRY(cudaEventSynchronize(t->staged));
-  else TV_CUDA_TRY(cudaEventCreateWithFlags(&t->staged, cudaEventDisableTiming));
-  char* hs = (char*)t->h_stage;
-  std::memcpy(hs, t->anc.data(), anc_b);
-  std::memcpy(hs + anc_b, t->depth.data(), i32_b);
-  std::memcpy(hs + anc_b + i32_b, t->parent.data(), i32_b);
-  std::memset(hs + total - 16, 0, 16);
-  TV_CUDA_TRY(cudaMemcpyAsync(t->d_blob, t->h_stage, total, cudaMemcpyHostToDevice, s));
-  TV_CUDA_TRY(cudaEventRecord(t->staged, s));
+  // The parent arrays go into one of two pinned slots; a small kernel reads the slot over the
+  // bus and derives masks and depths on the device (no copy-engine hop in front of the verify
+  // launch).  A slot is reused only after the kernel that read it two uploads ago has finished.
+  const int slot = t->stage_slot;
+  t->stage_slot ^= 1;
+  TV_CUDA_TRY(cudaEventSynchronize(t->staged[slot]));
+  std::memcpy((char*)t->h_stage + slot * slot_b, t->parent.data(), i32_b);
+  int st = tv_launch_tree_meta((const int32_t*)((const char*)t->h_stage_dev + slot * slot_b), t->n_trees,
+                               t->n, t->d_anc_w, t->d_depth_w, t->d_parent_w, t->d_status, s);
+  if (st != TV_OK) return st;
+  TV_CUDA_TRY(cudaEventRecord(t->staged[slot], s));
   t->uploaded = true;
+  return TV_OK;
+}
+
+TV_API int tv_tree_meta_device(tv_tree* t, uint64_t* anc, int32_t* depth, void* stream) {
+  if (!t) return TV_ERR_BAD_ARG;
+  if (!t->uploaded) return TV_ERR_NOT_UPLOADED;
+  const size_t nn = (size_t)t->n_trees * t->n;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (anc) TV_CUDA_TRY(cudaMemcpyAsync(anc, t->d_anc, nn * 2 * sizeof(uint64_t), cudaMemcpyDeviceToHost, s));
+  if (depth) TV_CUDA_TRY(cudaMemcpyAsync(depth, t->d_depth, nn * sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+  TV_CUDA_TRY(cudaStreamSynchronize(s));
   return TV_OK;
 }
 
@@ -200,7 +222,8 @@ TV_API int tv_tree_free(tv_tree* t) {
   if (!t) return TV_OK;
   if (t->d_blob) cudaFree(t->d_blob);
   if (t->h_stage) cudaFreeHost(t->h_stage);
-  if (t->staged) cudaEventDestroy(t->staged);
+  for (int i = 0; i < 2; ++i)
+    if (t->staged[i]) cudaEventDestroy(t->staged[i]);
   delete t;
   return TV_OK;
 }
@@ -251,9 +274,12 @@ TV_API int tv_tree_verify(const tv_tree* tree, const tv_dims* d, const float* S_
   a.L = d->L; a.B = d->B; a.H = d->H; a.T = d->T; a.dk = d->dk; a.dv = d->dv;
   a.rule = d->rule; a.bf16 = d->qkv_dtype == TV_BF16;
   a.S_pre = S_pre; a.q = q; a.k = k; a.v = v; a.alpha = alpha; a.beta = beta; a.O = O; a.U = U;
-  const bool tc_ok = tv_verify_tc_supports(a);
-  if (d->impl == TV_IMPL_TC && !tc_ok) return TV_ERR_UNSUPPORTED;
-  if (tc_ok && d->impl != TV_IMPL_SIMT) return tv_launch_verify_tc(a, tree->d_status, (cudaStream_t)stream);
+  const bool tc_gated = tv_verify_tc_supports(a), tc_delta = tv_verify_tc_delta_supports(a);
+  if (d->impl == TV_IMPL_TC && !tc_gated && !tc_delta) return TV_ERR_UNSUPPORTED;
+  if (d->impl != TV_IMPL_SIMT) {
+    if (tc_gated) return tv_launch_verify_tc(a, tree->d_status, (cudaStream_t)stream);
+    if (tc_delta) return tv_launch_verify_tc_delta(a, tree->d_status, (cudaStream_t)stream);
+  }
   return tv_launch_verify_simt(a, (cudaStream_t)stream);
 }
 

@@ -20,9 +20,14 @@ struct tv_tree {
   const uint64_t* d_anc = nullptr;
   const int32_t* d_depth = nullptr;
   const int32_t* d_parent = nullptr;
+  uint64_t* d_anc_w = nullptr;
+  int32_t* d_depth_w = nullptr;
+  int32_t* d_parent_w = nullptr;
   int32_t* d_status = nullptr;  // device status word (0 = ok), cleared by every upload
   bool uploaded = false;
-  cudaEvent_t staged = nullptr;  // completion of the last staging copy
+  cudaEvent_t staged[2] = {nullptr, nullptr};  // the device has read staging slot 0 / 1
+  const int32_t* h_stage_dev = nullptr;          // device view of the pinned staging block
+  int stage_slot = 0;
 };
 
 // Kernel-side view of the tree metadata.
@@ -65,8 +70,12 @@ void tv_set_cuda_error(cudaError_t e);
 // Launchers (each returns a tv_status; all work is asynchronous on `stream`).
 int tv_launch_verify_simt(const VerifyArgs& a, cudaStream_t stream);
 int tv_launch_commit(const CommitArgs& a, cudaStream_t stream);
+int tv_launch_tree_meta(const int32_t* parent_mapped, int32_t n_trees, int32_t n, uint64_t* anc,
+                        int32_t* depth, int32_t* parent_dev, int32_t* status, cudaStream_t stream);
 bool tv_verify_tc_supports(const VerifyArgs& a);
 int tv_launch_verify_tc(const VerifyArgs& a, int32_t* status, cudaStream_t stream);
+bool tv_verify_tc_delta_supports(const VerifyArgs& a);
+int tv_launch_verify_tc_delta(const VerifyArgs& a, int32_t* status, cudaStream_t stream);
 
 #define TV_CUDA_TRY(expr)                 \
   do {                                    \

@@ -1,0 +1,39 @@
+// Device-side tree metadata (Section IV-A Table II: Anc(i), depth; Section IV-C "Round-level
+// topology preprocessing"): one CTA per tree reads the parent array from pinned host memory
+// and writes the strict-ancestor masks, depths and a device copy of the parents.  Nodes are
+// indexed parent before child, so walking parent links from node i visits exactly Anc(i).
+#include "tv_internal.h"
+
+namespace {
+
+__global__ void __launch_bounds__(TV_MAX_NODES)
+tree_meta_kernel(const int32_t* __restrict__ parent, int32_t n, uint64_t* __restrict__ anc,
+                 int32_t* __restrict__ depth, int32_t* __restrict__ parent_dev, int32_t* status) {
+  __shared__ int32_t par_s[TV_MAX_NODES];
+  const int t = blockIdx.x, i = threadIdx.x;
+  if (i < n) par_s[i] = parent[(size_t)t * n + i];
+  if (t == 0 && i == 0) *status = 0;
+  __syncthreads();
+  if (i >= n) return;
+  uint64_t w0 = 0, w1 = 0;
+  int d = 0;
+  // the host has validated -1 <= parent[j] < j, so the walk ends within n steps
+  for (int p = par_s[i]; p >= 0 && d < n; p = par_s[p]) {
+    if (p < 64) w0 |= 1ull << p; else w1 |= 1ull << (p - 64);
+    ++d;
+  }
+  const size_t o = (size_t)t * n + i;
+  anc[2 * o] = w0;
+  anc[2 * o + 1] = w1;
+  depth[o] = d;
+  parent_dev[o] = par_s[i];
+}
+
+}  // namespace
+
+int tv_launch_tree_meta(const int32_t* parent_mapped, int32_t n_trees, int32_t n, uint64_t* anc,
+                        int32_t* depth, int32_t* parent_dev, int32_t* status, cudaStream_t stream) {
+  tree_meta_kernel<<<n_trees, TV_MAX_NODES, 0, stream>>>(parent_mapped, n, anc, depth, parent_dev, status);
+  TV_CUDA_TRY(cudaGetLastError());
+  return TV_OK;
+}

@@ -25,17 +25,14 @@
 // (the hardware's lane window of that warp) and half of the columns.
 // Every wait is an mbarrier wait with a time limit; on expiry the CTA sets the
 // status word, drains its own copies and leaves (TMEM is freed on every path).
-#include <cuda.h>
-#include <cudaTypedefs.h>
-#include <cuda_bf16.h>
-
-#include "tv_internal.h"
+#include "tv_tc_common.cuh"
 
 namespace {
 
+using namespace tvtc;
+
 constexpr int kThreads = 320;
 constexpr int kComputeWarps = 8;
-constexpr uint32_t kTile = 16384;  // one 128-row x 128-byte operand tile
 
 // shared memory map (byte offsets from the 1024-aligned base)
 constexpr uint32_t kOffQ = 0;                     // 2 tiles: k halves of Q  [128][64] bf16
@@ -60,144 +57,9 @@ enum Bar {
 // TMEM columns: scaled Q (A operand), scores, two output accumulators
 constexpr uint32_t kColQf = 0, kColSc = 128, kColAcc0 = 256, kColAcc1 = 384;
 
-constexpr uint32_t kIdescBf16KK = (1u << 4) | (1u << 7) | (1u << 10) | (16u << 17) | (8u << 24);
-constexpr uint32_t kIdescBf16KMn = kIdescBf16KK | (1u << 16);
-constexpr uint32_t kIdescTf32 = (1u << 4) | (2u << 7) | (2u << 10) | (16u << 17) | (8u << 24);
-
-constexpr long long kWaitLimitCycles = 1ll << 31;  // ~1 s
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-  return (uint32_t)__cvta_generic_to_shared(p);
-}
-
-// ---- mbarrier ---------------------------------------------------------------
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
-               : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-// Bounded wait.  Returns false when the limit ran out or another role gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  if (mbar_try(bar, parity)) return true;
-  const long long t0 = clock64();
-  for (uint32_t spin = 1;; ++spin) {
-    if (mbar_try(bar, parity)) return true;
-    if ((spin & 1023u) == 0) {
-      if (*abort_flag) return false;
-      if (clock64() - t0 > kWaitLimitCycles) {
-        *abort_flag = 1;
-        return false;
-      }
-    }
-  }
-}
-
-// Same for a whole warp: every lane gets the same answer, so that the warp never
-// splits around the warp-collective tcgen05 instructions that follow.
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  const bool ok = mbar_wait(bar, parity, abort_flag);
-  return __all_sync(0xffffffffu, ok);
-}
-
-// ---- TMA --------------------------------------------------------------------
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar,
-                                            int c0, int c1, int c2) {
-  asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
-      " [%0], [%1, {%3, %4, %5}], [%2];"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
-}
-
-__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2) {
-  asm volatile(
-      "cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4}], [%1];"
-      ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2) : "memory");
-}
-__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
-__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-
-// ---- tcgen05 ----------------------------------------------------------------
-__device__ __forceinline__ void tc_fence_before() {
-  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-}
-__device__ __forceinline__ void tc_fence_after() {
-  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-}
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
-               ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mma_bf16_ss(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc,
-                                            uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d), "l"(a), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void mma_tf32_ts(uint32_t d, uint32_t a_tmem, uint64_t b, uint32_t idesc,
-                                            uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, p;\n\t}"
-      ::"r"(d), "r"(a_tmem), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
-        "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),
-        "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]),
-        "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
-        "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
-      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
-      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]),
-        "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]),
-        "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]),
-        "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]),
-        "r"(r[29]), "r"(r[30]), "r"(r[31])
-      : "memory");
-}
-__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() {
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-}
-
-// Shared-memory matrix descriptors, 128-byte swizzle, 1024-byte swizzle atoms.
-// K-major: rows of 128 bytes, 8-row groups 1024 bytes apart.
-__device__ __forceinline__ uint64_t desc_kmajor(uint32_t saddr) {
-  return (uint64_t)((saddr & 0x3ffffu) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) |
-         (1ull << 46) | (2ull << 61);
-}
-// MN-major (V as the B operand, dv contiguous): 64-column blocks `lbo` bytes
-// apart, 8-row k groups 1024 bytes apart.
-__device__ __forceinline__ uint64_t desc_mnmajor(uint32_t saddr, uint32_t lbo) {
-  return (uint64_t)((saddr & 0x3ffffu) >> 4) | ((uint64_t)(lbo >> 4) << 16) |
-         ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
-}
+constexpr uint32_t kIdescBf16KK = idesc_bf16(128, false);
+constexpr uint32_t kIdescBf16KMn = idesc_bf16(128, true);
+constexpr uint32_t kIdescTf32 = idesc_tf32(128);
 
 // Eight fp32 values -> bf16 hi and lo parts (hi = upper 16 bits, lo = the exact remainder cut to
 // its upper 16 bits: hi + lo carries 16 mantissa bits), stored as two 16-byte chunks.
@@ -390,10 +252,26 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     // O_i = r_i acc_i for the item whose accumulator is `it_prev`: TMEM -> registers -> the
     // (now idle) C' tiles as four [128 rows][32 fp32] swizzled tiles -> one TMA store per tile
     // (full 128-byte lines; rows past T are clipped by the tensor map).
+    // T <= 64: the j >= 64 halves of the C' tiles are idle and hold the staging chunks
+    // ([64 rows][32 fp32], 8 KiB each), so staging never collides with the C' tiles of the
+    // next item and the store is only waited for one item later.  T > 64: the chunks are the
+    // four C' tiles themselves and the store must have read them before C' is rewritten.
+    const bool small = T <= 64;
+    auto stage_addr = [&](int c4) -> uint32_t {
+      return small ? kOffChi + kTile + (uint32_t)(c4 >> 1) * (kOffClo - kOffChi) + (uint32_t)(c4 & 1) * 8192u
+                   : kOffChi + (uint32_t)c4 * kTile;
+    };
     auto final_epilogue = [&](uint32_t it_prev, int item_prev, float r_prev, uint32_t ost_phase) -> bool {
       const int acc_done = (it_prev & 1) ? ACC_DONE1 : ACC_DONE0;
       const int acc_free = (it_prev & 1) ? ACC_FREE1 : ACC_FREE0;
       const uint32_t acc_col = (it_prev & 1) ? kColAcc1 : kColAcc0;
+      if (small) {
+        if (warp == 2 && lane == 0) {
+          tma_store_wait_read();          // the store of the item before has read the chunks
+          mbar_arrive(bar(OST_FREE));
+        }
+        if (!mbar_wait_warp(bar(OST_FREE), ost_phase, abort_flag)) return false;
+      }
       if (!mbar_wait_warp(bar(acc_done), (it_prev >> 1) & 1, abort_flag)) return false;
       tc_fence_after();
       if (warp_live) {
@@ -402,7 +280,7 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           uint32_t r1[32];
           tmem_ld32(tmem + lane_addr + acc_col + hc * 64 + half * 32, r1);
           tmem_wait_ld();
-          unsigned char* orow = sm + kOffChi + (hc * 2 + half) * kTile + row * 128;
+          unsigned char* orow = sm + stage_addr(hc * 2 + half) + row * 128;
 #pragma unroll
           for (int c = 0; c < 8; ++c) {
             float4 o;
@@ -424,13 +302,13 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       if (warp == 2 && lane == 0) {
         if (mbar_wait(bar(OST_READY), ost_phase, abort_flag)) {
 #pragma unroll
-          for (int c = 0; c < 4; ++c) tma_store_3d(&tmO, sbase + kOffChi + c * kTile, 32 * c, 0, item_prev);
+          for (int c = 0; c < 4; ++c) tma_store_3d(&tmO, sbase + stage_addr(c), 32 * c, 0, item_prev);
           tma_store_commit();
-          tma_store_wait_read();   // the tiles may be overwritten once the store has read them
+          if (!small) tma_store_wait_read();   // the tiles may be overwritten once the store has read them
         }
-        mbar_arrive(bar(OST_FREE));
+        if (!small) mbar_arrive(bar(OST_FREE));
       }
-      return mbar_wait_warp(bar(OST_FREE), ost_phase, abort_flag);
+      return small ? true : mbar_wait_warp(bar(OST_FREE), ost_phase, abort_flag);
     };
 
     // metadata of the first item; later items are fetched one item ahead
@@ -601,34 +479,6 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
 // ---------------------------------------------------------------------------
 // Host side: tensor maps and launch.
 // ---------------------------------------------------------------------------
-PFN_cuTensorMapEncodeTiled get_encode() {
-  static PFN_cuTensorMapEncodeTiled fn = nullptr;
-  static bool tried = false;
-  if (!tried) {
-    tried = true;
-    void* ptr = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) ==
-            cudaSuccess && qres == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<PFN_cuTensorMapEncodeTiled>(ptr);
-  }
-  return fn;
-}
-
-// [items][rows][cols] tensor, box {box_cols, 128, 1}, 128-byte swizzle, zero fill.
-bool make_map(CUtensorMap* map, const void* base, CUtensorMapDataType dt, int esize, uint64_t items,
-              uint64_t rows, uint64_t cols, uint32_t box_cols) {
-  PFN_cuTensorMapEncodeTiled enc = get_encode();
-  if (!enc) return false;
-  const cuuint64_t gdim[3] = {cols, rows, items};
-  const cuuint64_t gstr[2] = {cols * esize, rows * cols * esize};
-  const cuuint32_t box[3] = {box_cols, 128, 1};
-  const cuuint32_t estr[3] = {1, 1, 1};
-  return enc(map, dt, 3, const_cast<void*>(base), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 // Gated rule: the correction rows are the values themselves (U = V).
 __global__ void widen_bf16_kernel(const __nv_bfloat16* __restrict__ v, float* __restrict__ U, size_t n8) {
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n8; i += (size_t)gridDim.x * blockDim.x) {
@@ -659,13 +509,16 @@ bool tv_verify_tc_supports(const VerifyArgs& a) {
 int tv_launch_verify_tc(const VerifyArgs& a, int32_t* status, cudaStream_t stream) {
   if (!tv_verify_tc_supports(a)) return TV_ERR_UNSUPPORTED;
   const uint64_t items = (uint64_t)a.L * a.B * a.H;
-  alignas(64) CUtensorMap tmQ, tmK, tmV, tmS, tmO;
-  if (!make_map(&tmQ, a.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, items, a.T, 128, 64) ||
-      !make_map(&tmK, a.k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, items, a.T, 128, 64) ||
-      !make_map(&tmV, a.v, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, items, a.T, 128, 64) ||
-      !make_map(&tmS, a.S_pre, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, 128, 128, 32) ||
-      !make_map(&tmO, a.O, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, a.T, 128, 32))
-    return TV_ERR_CUDA;
+  const uint32_t orows = a.T <= 64 ? 64 : 128;   // rows of one staged output chunk
+  const void* const ptrs[5] = {a.q, a.k, a.v, a.S_pre, a.O};
+  const MapSet* ms = cached_maps(ptrs, items, a.T, 0, [&](CUtensorMap* m) {
+    return make_map(&m[0], a.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, items, a.T, 128, 64) &&
+           make_map(&m[1], a.k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, items, a.T, 128, 64) &&
+           make_map(&m[2], a.v, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, items, a.T, 128, 64) &&
+           make_map(&m[3], a.S_pre, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, 128, 128, 32) &&
+           make_map(&m[4], a.O, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, a.T, 128, 32, orows);
+  });
+  if (!ms) return TV_ERR_CUDA;
   static thread_local int configured_dev = -1;
   static thread_local int sm_count = 0;
   int dev = 0;
@@ -684,7 +537,8 @@ int tv_launch_verify_tc(const VerifyArgs& a, int32_t* status, cudaStream_t strea
   p.O = a.O;
   p.status = status;
   const int grid = (int)(items < (uint64_t)sm_count ? items : (uint64_t)sm_count);
-  verify_tc_gated_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tmQ, tmK, tmV, tmS, tmO, p);
+  verify_tc_gated_kernel<<<grid, kThreads, kSmemBytes, stream>>>(ms->map[0], ms->map[1], ms->map[2], ms->map[3],
+                                                                ms->map[4], p);
   TV_CUDA_TRY(cudaGetLastError());
   if (a.U) {
     const size_t n8 = items * a.T * 128 / 8;

@@ -19,13 +19,18 @@ pytestmark = pytest.mark.gpu
 IMPLS = [tv.IMPL_SIMT, tv.IMPL_TC]
 
 
-def _tc_ok(wl):
-    return wl.qkv_dtype == inputs.BF16 and wl.dk == 128 and wl.dv == 128 and wl.rule == inputs.GATED
+def _tc_ok(wl, parents=None):
+    if not (wl.qkv_dtype == inputs.BF16 and wl.dk == 128 and wl.dv == 128):
+        return False
+    if wl.rule == inputs.GATED:
+        return True
+    depth = max(int(inputs.node_depths(p).max()) for p in parents) if parents is not None else 0
+    return wl.T <= 64 and depth <= 15
 
 
-def _skip_unless_supported(wl, impl):
-    if impl == tv.IMPL_TC and not _tc_ok(wl):
-        pytest.skip("tensor-core kernel covers bf16, dk = dv = 128, gated rule")
+def _skip_unless_supported(wl, impl, parents=None):
+    if impl == tv.IMPL_TC and not _tc_ok(wl, parents):
+        pytest.skip("tensor-core kernels cover bf16, dk = dv = 128 (delta rule: T <= 64, depth <= 15)")
 
 
 def _run(wl, parents, accepted, tens, tol, items=None, **kw):
@@ -43,8 +48,8 @@ def _run(wl, parents, accepted, tens, tol, items=None, **kw):
 @pytest.mark.parametrize("name", ["c1", "c2", "c3", "c4"])
 def test_workload_full(name, impl):
     wl = inputs.workload(name)
-    _skip_unless_supported(wl, impl)
     parents, accepted = inputs.make_trees(wl)
+    _skip_unless_supported(wl, impl, parents)
     tens = inputs.make_tensors(wl)
     _run(wl, parents, accepted, tens, wl.tol, impl=impl)
     if wl.rule == inputs.DELTA:
@@ -97,11 +102,11 @@ def test_edge_shapes(case, dtype, rule, impl):
     T, dk, dv, B, H, kind, shared = case
     wl = inputs.workload("c2", T=T, dk=dk, dv=dv, B=B, H=H, rule=rule, qkv_dtype=dtype,
                          tree="frontier" if kind == "star" else kind, seed=100 + T)
-    _skip_unless_supported(wl, impl)
     parents, accepted = inputs.make_trees(wl, per_request=not shared)
     if kind == "star":
         parents[:] = -1
         accepted[:] = T - 1
+    _skip_unless_supported(wl, impl, parents)
     accepted[0] = -1 if T % 2 else accepted[0]          # some requests accept nothing
     tens = inputs.make_tensors(wl)
     tol = 1e-5 if dtype == inputs.F32 else 2e-3

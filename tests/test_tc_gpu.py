@@ -52,3 +52,55 @@ def test_extreme_decay(tree, mu, impl):
     eO, _, eS = pu.compare(wl, O, None, Sn, ver, com)
     print(f"decay mu={mu} {tree} impl={impl}: rel-L2 O {eO:.3e} S {eS:.3e}")
     assert eO <= wl.tol and eS <= wl.tol
+
+
+@pytest.mark.parametrize("B,H,T,tree", [(1, 1, 64, "frontier"), (1, 2, 37, "frontier"), (2, 3, 1, "chain"),
+                                         (3, 4, 16, "chain"), (16, 32, 64, "frontier"), (5, 7, 50, "levels")])
+def test_tc_delta(B, H, T, tree):
+    """Delta rule on the tensor cores: O and the corrections U against the oracle."""
+    wl = inputs.workload("c4", B=B, H=H, T=T, L=1, tree=tree, seed=23 + T)
+    parents, accepted = inputs.make_trees(wl)
+    tens = inputs.make_tensors(wl)
+    O, U, Sn, tree_h = pu.gpu_round(wl, parents, accepted, tens, impl=tv.IMPL_TC, want_U=True,
+                                    commit_with_U=True, in_place=True)
+    tree_h.device_status()
+    ver, com = pu.oracle_round(wl, parents, accepted, tens)
+    eO, eU, eS = pu.compare(wl, O, U, Sn, ver, com)
+    print(f"TC delta B{B} H{H} T{T} {tree}: rel-L2 O {eO:.3e} U {eU:.3e} S {eS:.3e}")
+    assert eO <= wl.tol and eU <= wl.tol and eS <= wl.tol
+    O2, _, _, _ = pu.gpu_round(wl, parents, accepted, tens, impl=tv.IMPL_TC, want_U=False)
+    assert np.array_equal(O2, O)          # asking for U does not change O
+
+
+def test_tc_delta_falls_back_on_deep_trees():
+    wl = inputs.workload("c4", B=1, H=2, T=40, tree="chain", seed=5)   # depth 39 > 15
+    parents, accepted = inputs.make_trees(wl)
+    tens = {k: (None if v is None else v.cuda()) for k, v in inputs.make_tensors(wl).items()}
+    tree = tv.tree_build(parents).upload()
+    with pytest.raises(tv.TreeVerifyError) as e:
+        tv.tree_verify(tree, tens["S_pre"], tens["q"], tens["k"], tens["v"], tens["alpha"], tens["beta"],
+                       rule=tv.DELTA, impl=tv.IMPL_TC)
+    assert e.value.status == -3
+    O = tv.tree_verify(tree, tens["S_pre"], tens["q"], tens["k"], tens["v"], tens["alpha"], tens["beta"],
+                       rule=tv.DELTA)            # AUTO takes the SIMT kernel
+    torch.cuda.synchronize()
+    assert torch.isfinite(O).all()
+
+
+@pytest.mark.parametrize("name", ["c1", "c2", "c3", "c5"])
+def test_device_built_metadata_bit_exact(name):
+    """Masks and depths derived by the device kernel equal the host's and the oracle's."""
+    from oracle import tree_oracle as orc
+    wl = inputs.workload(name)
+    parents, _ = inputs.make_trees(wl)
+    tree = tv.tree_build(parents).upload()
+    anc_d, depth_d = tree.meta_device()
+    anc_h, depth_h, _ = tree.meta()
+    assert anc_d.tobytes() == anc_h.tobytes() and depth_d.tobytes() == depth_h.tobytes()
+    for t in (0, len(parents) - 1):
+        oanc, odepth, _ = orc.tree_metadata(parents[t])
+        assert anc_d[t].tobytes() == oanc.tobytes() and depth_d[t].tobytes() == odepth.tobytes()
+    tree.rebuild(parents[::-1].copy()).upload()       # new topology, same buffers
+    anc_d2, depth_d2 = tree.meta_device()
+    anc_h2, depth_h2, _ = tree.meta()
+    assert anc_d2.tobytes() == anc_h2.tobytes() and depth_d2.tobytes() == depth_h2.tobytes()
