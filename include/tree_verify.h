@@ -51,6 +51,7 @@ extern "C" {
 
 #define TV_MAX_NODES 128   /* T <= 128: ancestor sets are 128-bit masks   */
 #define TV_MAX_DIM   128   /* dk, dv <= 128, multiples of 4               */
+#define TV_STATIC_MAX_TREES 128  /* capacity of tv_tree_verify_static       */
 
 typedef enum tv_status {
   TV_OK = 0,
@@ -60,7 +61,8 @@ typedef enum tv_status {
   TV_ERR_CUDA = -4,           /* a CUDA runtime call failed (tv_last_cuda_error)*/
   TV_ERR_NOT_UPLOADED = -5,   /* tree metadata not on the device yet            */
   TV_ERR_DEVICE_TIMEOUT = -6, /* a bounded device-side wait ran out             */
-  TV_ERR_NOMEM = -7
+  TV_ERR_NOMEM = -7,
+  TV_ERR_TOO_LARGE = -8       /* size beyond a fixed, documented capacity       */
 } tv_status;
 
 enum { TV_GATED = 0, TV_GATED_DELTA = 1 };  /* update rule                      */
@@ -147,6 +149,42 @@ int tv_tree_verify(const tv_tree* tree, const tv_dims* dims,
                    const float* alpha /*dev*/, const float* beta /*dev or NULL*/,
                    float* O /*dev*/, float* U /*dev or NULL*/,
                    void* stream);
+
+/* ---- verification without any allocation ------------------------------------
+ * (The paper has no counterpart: this entry exists for this library's users.)
+ *
+ * Some callers may not allocate device or pinned memory at all: code inside a
+ * CUDA-graph capture, a serving loop whose memory was carved up at start-up,
+ * a plug-in in a process that owns the allocator, or a latency-critical path
+ * that cannot afford the implicit synchronisation of an allocation.  The
+ * regular path allocates in tv_tree_build and in the first tv_tree_upload.
+ * This call does the same verification as tv_tree_verify but takes the parent
+ * arrays straight from DEVICE memory (int32 [n_trees][T], n_trees = 1 or B, as
+ * a drafter running on the GPU leaves them) and keeps the derived masks and
+ * depths in a fixed array inside the library's device image: 384 KiB that
+ * every GPU which loads the library holds until the process exits.  It calls
+ * no cudaMalloc/cudaFree and no allocating library routine.
+ *
+ * Limits: n_trees <= TV_STATIC_MAX_TREES and T <= TV_MAX_NODES, otherwise
+ * TV_ERR_TOO_LARGE / TV_ERR_UNSUPPORTED is returned and nothing is launched.
+ * The delta rule runs on the general fp32 kernel here (the tree depth is not
+ * known on the host).
+ * The first call on each device looks up the device address of that array
+ * (with that device current); make that first call outside any stream capture.
+ * All calls share the array and it keeps the last call's metadata (the part a
+ * call needs is rewritten, and its status word cleared, by the call itself):
+ * two calls whose kernels may overlap on the GPU -- different streams without
+ * ordering -- race on it; calls on one stream are safe.
+ * The parents cannot be validated on the host: a parent outside [-1, i) is
+ * treated as -1 and TV_ERR_INVALID_TREE is written to *status; a device-side
+ * wait that ran out writes TV_ERR_DEVICE_TIMEOUT.  status is a DEVICE int32
+ * that the caller zeroes beforehand, or NULL.                                 */
+int tv_tree_verify_static(const int32_t* parent /*dev*/, int32_t n_trees, const tv_dims* dims,
+                          const float* S_pre /*dev*/,
+                          const void* q /*dev*/, const void* k /*dev*/, const void* v /*dev*/,
+                          const float* alpha /*dev*/, const float* beta /*dev or NULL*/,
+                          float* O /*dev*/, float* U /*dev or NULL*/,
+                          int32_t* status /*dev or NULL*/, void* stream);
 
 /* ---- accepted-path commit (Section IV-D Eq. 10; Lemma 1 Eq. 3) -------------
  *

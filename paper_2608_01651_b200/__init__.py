@@ -17,6 +17,7 @@ GATED, DELTA = 0, 1
 F32, BF16 = 0, 1
 IMPL_AUTO, IMPL_SIMT, IMPL_TC = 0, 1, 2
 MAX_NODES = 128
+STATIC_MAX_TREES = 128
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libtreeverify.so")
@@ -65,6 +66,8 @@ def lib() -> ctypes.CDLL:
     L.tv_tree_device_status.restype = ctypes.c_int
     L.tv_tree_verify.argtypes = [vp, p(_Dims)] + [vp] * 9
     L.tv_commit_path.argtypes = [vp, p(_Dims)] + [vp] * 9
+    L.tv_tree_verify_static.argtypes = [vp, i32, p(_Dims)] + [vp] * 10
+    L.tv_tree_verify_static.restype = ctypes.c_int
     L.tv_session_create.argtypes = [p(_Dims), i32, p(vp)]
     L.tv_session_round.argtypes = [vp] + [vp] * 11
     L.tv_session_free.argtypes = [vp]
@@ -269,6 +272,29 @@ def commit_path(tree: Tree, accepted, S_pre, k, v, alpha, beta=None, *, rule=GAT
                                 _ptr(v), _ptr(alpha), _ptr(beta), _ptr(U), _ptr(out),
                                 _stream_ptr(stream)), "tv_commit_path")
     return out
+
+
+def tree_verify_static(parent, S_pre, q, k, v, alpha, beta=None, *, rule=GATED, O, U=None, status=None,
+                       impl=IMPL_AUTO, stream=None):
+    """``tv_tree_verify_static``: verification for callers that must not allocate.
+
+    ``parent`` is a CUDA int32 tensor [n_trees, T] (n_trees = 1 or B); ``O`` (and ``U``,
+    ``status`` if wanted) are preallocated CUDA tensors.  Nothing is allocated here or in the
+    library: the tree metadata lives in a fixed device array (at most 128 trees of 128 nodes).
+    """
+    import torch
+    _require(parent, "parent", torch.int32)
+    _require(status, "status", torch.int32)
+    for t, n in ((S_pre, "S_pre"), (alpha, "alpha"), (beta, "beta"), (O, "O"), (U, "U")):
+        _require(t, n, torch.float32)
+    for t, n in ((q, "q"), (k, "k"), (v, "v")):
+        _require(t, n, k.dtype)
+    d = _dims(S_pre, k, v, rule, impl)
+    n_trees = parent.shape[0] if parent.dim() == 2 else 1
+    _check(lib().tv_tree_verify_static(_ptr(parent), n_trees, ctypes.byref(d), _ptr(S_pre), _ptr(q),
+                                       _ptr(k), _ptr(v), _ptr(alpha), _ptr(beta), _ptr(O), _ptr(U),
+                                       _ptr(status), _stream_ptr(stream)), "tv_tree_verify_static")
+    return O
 
 
 class Prepared:

@@ -21,6 +21,7 @@ TV_API const char* tv_strerror(int s) {
     case TV_ERR_NOT_UPLOADED: return "tree metadata not uploaded to the device";
     case TV_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait ran out";
     case TV_ERR_NOMEM: return "out of memory";
+    case TV_ERR_TOO_LARGE: return "size beyond the fixed capacity of this entry point";
     default: return "unknown status";
   }
 }
