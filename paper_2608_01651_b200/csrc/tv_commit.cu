@@ -254,6 +254,207 @@ __global__ void __launch_bounds__(kRowThreads) commit_factored_dk128_kernel(Comm
   }
 }
 
+// Persistent version of the dk = 128 row-owner kernel for accepted paths of at most 16 nodes
+// and batches of at most 256 requests.  A CTA walks units of 64 state rows; the accepted node
+// and path mask of every request are read once per CTA, and while the 16 loads of unit n are
+// in flight the path of unit n+1 is worked out (nodes from the mask bits, suffix products
+// P_a/P_j by a warp scan) and its key / value rows are fetched into registers, to be staged in
+// the other half of a double buffer after unit n has been updated.  No unit waits on a chain of
+// dependent global loads.
+#ifndef TV_STREAM_CTAS
+#define TV_STREAM_CTAS 5
+#endif
+constexpr int kStreamMaxB = 256;
+constexpr int kStreamMaxLen = 16;
+
+template <bool BF16>
+__global__ void __launch_bounds__(kRowThreads, TV_STREAM_CTAS) commit_stream_dk128_kernel(CommitArgs a) {
+  __shared__ int acc_s[kStreamMaxB];
+  __shared__ uint64_t mask_s[kStreamMaxB][2];
+  __shared__ __align__(16) float k_s[2][kStreamMaxLen][128];
+  __shared__ __align__(16) float cu_s[2][kStreamMaxLen][kRowsPerCta];
+  __shared__ int node_s[2][kStreamMaxLen];
+  __shared__ float w_s[2][kStreamMaxLen];
+  __shared__ float Pa_s[2];
+  __shared__ int len_s[2];
+
+  const int dv = a.dv, T = a.T;
+  const int n_half = dv / kRowsPerCta;
+  const int n_units = a.L * a.B * a.H * n_half;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const bool in_place = a.S_new == a.S_pre;
+
+  for (int b = tid; b < a.B; b += kRowThreads) {
+    int acc = a.accepted[b];
+    if (acc >= T) acc = -1;
+    acc_s[b] = acc;
+    uint64_t m0 = 0, m1 = 0;
+    if (acc >= 0) {
+      const int tb = a.tree.n_trees == 1 ? 0 : b;
+      const uint64_t* m = a.tree.anc + ((size_t)tb * T + acc) * 2;
+      m0 = m[0];
+      m1 = m[1];
+      if (acc < 64) m0 |= 1ull << acc; else m1 |= 1ull << (acc - 64);
+    }
+    mask_s[b][0] = m0;
+    mask_s[b][1] = m1;
+  }
+  __syncthreads();
+
+  auto req_of = [&](int u) { return ((u / n_half) / a.H) % a.B; };
+  auto next_live = [&](int u) {   // first unit >= u (in this CTA's stride) that has work to do
+    while (u < n_units && in_place && acc_s[req_of(u)] < 0) u += gridDim.x;
+    return u;
+  };
+
+  // path of unit u into buffer nb: nodes, weights P_a/P_j, P_a, length (warp 0)
+  auto path_nodes = [&](int u, int nb) {
+    if (warp != 0) return;
+    const int b = req_of(u);
+    const uint64_t m0 = mask_s[b][0], m1 = mask_s[b][1];
+    const int c0 = __popcll(m0);
+    const int len = min(c0 + __popcll(m1), kStreamMaxLen);
+    int node = 0;
+    float al = 1.f;
+    if (lane < len) {
+      uint64_t w = lane < c0 ? m0 : m1;
+      const int r = lane < c0 ? lane : lane - c0;
+      for (int i = 0; i < r; ++i) w &= w - 1;
+      node = __ffsll((long long)w) - 1 + (lane < c0 ? 0 : 64);
+      al = a.alpha[(size_t)(u / n_half) * T + node];
+    }
+    float incl = al;   // product of alpha over path positions >= lane
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const float up = __shfl_down_sync(0xffffffffu, incl, o);
+      if (lane + o < 32) incl *= up;
+    }
+    const float nxt = __shfl_down_sync(0xffffffffu, incl, 1);
+    if (lane < kStreamMaxLen) {
+      node_s[nb][lane] = node;
+      w_s[nb][lane] = lane + 1 < 32 ? nxt : 1.f;
+    }
+    if (lane == 0) {
+      Pa_s[nb] = incl;
+      len_s[nb] = len;
+    }
+  };
+
+  // key / value rows of unit u's path: 4 x 16 keys and 8 values per thread, in registers
+  uint2 kreg[4];
+  uint2 kreg2[4];
+  float ureg[8];
+  auto fetch_rows = [&](int u, int nb) {
+    const int item = u / n_half, half = u - item * n_half;
+    const size_t node0 = (size_t)item * T;
+    const int len = len_s[nb];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int i = tid + q * kRowThreads;          // (p, k4) = (i / 32, i % 32)
+      const int p = i >> 5, k4 = i & 31;
+      kreg[q] = make_uint2(0u, 0u);
+      kreg2[q] = make_uint2(0u, 0u);
+      if (p < len) {
+        const size_t idx = (node0 + node_s[nb][p]) * 128 + k4 * 4;
+        if (BF16) {
+          kreg[q] = *reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(a.k) + idx);
+        } else {
+          const uint4 r = *reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(a.k) + idx);
+          kreg[q] = make_uint2(r.x, r.y);
+          kreg2[q] = make_uint2(r.z, r.w);
+        }
+      }
+    }
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      const int i = tid + q * kRowThreads;          // (p, r) = (i / 64, i % 64)
+      const int p = i >> 6, r = i & 63;
+      ureg[q] = 0.f;
+      if (p < len) {
+        const size_t idx = (node0 + node_s[nb][p]) * dv + half * kRowsPerCta + r;
+        ureg[q] = a.U ? a.U[idx] : load_elem<BF16>(a.v, idx);
+      }
+    }
+  };
+  auto stage_rows = [&](int nb) {
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int i = tid + q * kRowThreads;
+      const int p = i >> 5, k4 = i & 31;
+      float4 kv;
+      if (BF16) {
+        kv = make_float4(__uint_as_float(kreg[q].x << 16), __uint_as_float(kreg[q].x & 0xffff0000u),
+                         __uint_as_float(kreg[q].y << 16), __uint_as_float(kreg[q].y & 0xffff0000u));
+      } else {
+        kv = make_float4(__uint_as_float(kreg[q].x), __uint_as_float(kreg[q].y),
+                         __uint_as_float(kreg2[q].x), __uint_as_float(kreg2[q].y));
+      }
+      *reinterpret_cast<float4*>(&k_s[nb][p][k4 * 4]) = kv;
+    }
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      const int i = tid + q * kRowThreads;
+      const int p = i >> 6, r = i & 63;
+      cu_s[nb][p][r] = w_s[nb][p] * ureg[q];
+    }
+  };
+
+  int u = next_live(blockIdx.x);
+  if (u >= n_units) return;
+  path_nodes(u, 0);
+  __syncthreads();
+  fetch_rows(u, 0);
+  stage_rows(0);
+  __syncthreads();
+
+  for (int n = 0; u < n_units; ++n) {
+    const int cb = n & 1, nb = cb ^ 1;
+    const int un = next_live(u + gridDim.x);
+    // a. the 16 loads of this unit
+    const int row0 = warp * 16;
+    const float4* src = reinterpret_cast<const float4*>(a.S_pre) + ((size_t)u * kRowsPerCta + row0) * 32 + lane;
+    float4* dst = reinterpret_cast<float4*>(a.S_new) + ((size_t)u * kRowsPerCta + row0) * 32 + lane;
+    float4 s[16];
+#pragma unroll
+    for (int e = 0; e < 16; ++e) s[e] = ld_stream(src + e * 32);
+    // b-d. the path of the next unit, and its rows into registers
+    if (un < n_units) path_nodes(un, nb);
+    __syncthreads();
+    if (un < n_units) fetch_rows(un, nb);
+    // e. update and store this unit
+    const float Pa = Pa_s[cb];
+    const int len = len_s[cb];
+    if (len > 0) {
+#pragma unroll
+      for (int e = 0; e < 16; ++e) {
+        s[e].x *= Pa; s[e].y *= Pa; s[e].z *= Pa; s[e].w *= Pa;
+      }
+      for (int p = 0; p < len; ++p) {
+        const float4 kv = *reinterpret_cast<const float4*>(&k_s[cb][p][lane * 4]);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const float4 cu = *reinterpret_cast<const float4*>(&cu_s[cb][p][warp * 16 + q * 4]);
+          const float c[4] = {cu.x, cu.y, cu.z, cu.w};
+#pragma unroll
+          for (int t = 0; t < 4; ++t) {
+            float4& x = s[q * 4 + t];
+            x.x = fmaf(c[t], kv.x, x.x);
+            x.y = fmaf(c[t], kv.y, x.y);
+            x.z = fmaf(c[t], kv.z, x.z);
+            x.w = fmaf(c[t], kv.w, x.w);
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int e = 0; e < 16; ++e) st_stream(dst + e * 32, s[e]);
+    // f. the next unit's rows into the other buffer
+    if (un < n_units) stage_rows(nb);
+    __syncthreads();
+    u = un;
+  }
+}
+
 // Delta rule without stored corrections: every row v of the [dv][dk] state
 // evolves independently along the accepted path,
 //   s <- alpha_j s;  u = beta_j (v_j[v] - s . k_j);  s <- s + u k_j,
@@ -368,7 +569,20 @@ int tv_launch_commit(const CommitArgs& a, cudaStream_t stream) {
   const int items = a.L * a.B * a.H;
   if ((size_t)a.dk * a.dv > (size_t)kMaxVec * kThreads * 4) return TV_ERR_UNSUPPORTED;
   const bool recompute = a.rule == TV_GATED_DELTA && a.U == nullptr;
-  if (!recompute && a.dk == 128) {
+  static thread_local int sm_count = 0;
+  if (!sm_count) {
+    int dev = 0;
+    TV_CUDA_TRY(cudaGetDevice(&dev));
+    TV_CUDA_TRY(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev));
+  }
+  const int units = a.dv % kRowsPerCta == 0 ? items * (a.dv / kRowsPerCta) : 0;
+  // the persistent kernel pays a prologue per CTA: worth it from about six units per CTA on
+  if (!recompute && a.dk == 128 && units >= 6 * TV_STREAM_CTAS * sm_count && a.B <= kStreamMaxB &&
+      a.tree.max_depth_all < kStreamMaxLen) {
+    const int ctas = TV_STREAM_CTAS * sm_count;
+    if (a.bf16) commit_stream_dk128_kernel<true><<<ctas, kRowThreads, 0, stream>>>(a);
+    else commit_stream_dk128_kernel<false><<<ctas, kRowThreads, 0, stream>>>(a);
+  } else if (!recompute && a.dk == 128) {
     const int ctas = items * ((a.dv + kRowsPerCta - 1) / kRowsPerCta);
     if (a.bf16) commit_factored_dk128_kernel<true><<<ctas, kRowThreads, 0, stream>>>(a);
     else commit_factored_dk128_kernel<false><<<ctas, kRowThreads, 0, stream>>>(a);

@@ -153,3 +153,22 @@ def test_argument_errors_on_device():
                        S_new=flat[64:].view_as(S))
     assert e.value.status == -1
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("rule", [inputs.GATED, inputs.DELTA])
+def test_commit_many_units_per_cta(rule):
+    """Enough states that the persistent commit kernel is the one that runs (several units per
+    CTA, mixed accepted / rejected requests, in place and out of place), checked on samples."""
+    wl = inputs.workload("c3", B=160, H=32, T=24, L=1, rule=rule, seed=321)
+    parents, accepted = inputs.make_trees(wl)
+    tens = inputs.make_tensors(wl)
+    items = [(b, h) for b in (0, 1, 7, 63, 159) for h in (0, 31)]
+    for in_place in (True, False):
+        O, U, Sn, _ = pu.gpu_round(wl, parents, accepted, tens, want_U=True, commit_with_U=True,
+                                   in_place=in_place)
+        ver, com = pu.oracle_round(wl, parents, accepted, tens, items=items)
+        eO, eU, eS = pu.compare(wl, O, U, Sn, ver, com)
+        assert eO <= wl.tol and eU <= wl.tol and eS <= wl.tol, (eO, eU, eS)
+        dead = [b for b in range(wl.B) if accepted[b] < 0]
+        assert dead, "the workload should reject some requests"
+        assert np.array_equal(Sn[dead[0]], tens["S_pre"][dead[0]].double().numpy())
