@@ -12,19 +12,22 @@
 // any descendant refer to the same node p_s.  Row i of W = C N D_beta and of
 // A = N D_beta come from ONE back-substitution each on the path-restricted unit
 // lower-triangular system (w L = c, x L = e_d; L = I + G on the path): d^2/2
-// FMAs per row, no T x T product, no Neumann rounds, no level barriers.
+// FMAs per row, no T x T product, no Neumann rounds, no level barriers.  All
+// decay factors are exp2 of differences of log-gate prefix sums along the row's
+// own path, i.e. only ever formed on ancestor pairs.
 //
 // Tile rows 0..63 carry the O problem of node i, rows 64..127 the U problem of
-// node i (the M = 128 MMA shape is otherwise half empty at T <= 64):
-//     Sc1 = Q K^T, Sc2 = K K^T                 (bf16, N = 64)        -> TMEM
-//     rows of [W ; A] and [W D_P ; A D_P]      (fp32 threads)        -> bf16 hi/lo tiles
-//     D1  = [W D_P ; A D_P] K                  (bf16, K as MN-major B)
-//     Qf  = [D_P Q - D1 ; -D1]                 (fp32 -> TMEM, tf32 A operand)
-//     acc = Qf S_pre^T + [W ; A] V             (tf32 + bf16 hi/lo)
+// node i (the M = 128 MMA shape is otherwise half empty at T <= 64).  Q and K
+// are stacked in one operand tile [Q ; K]:
+//     Sc  = [Q ; K] K^T   (bf16, N = 64)   rows 0..63 = Q K^T, rows 64..127 = K K^T
+//     E1: path-sparse raw rows of C and G; E2: back-substitution, operand tiles
+//     Qf  = [diag(P) | -(W D_P)] [Q ; K]   rows 0..63  = Q_eff      (bf16 hi/lo,
+//           [   0    | -(A D_P)] [Q ; K]   rows 64..127 = -K_eff     result in TMEM)
+//     acc = Qf S_pre^T (tf32, A operand straight from TMEM) + [W ; A] V (bf16 hi/lo)
 //     O = acc[0..63], U = acc[64..127]
-// S_pre goes TMA -> shared memory -> tensor core untouched; O leaves through
-// swizzled staging tiles and a TMA store.  Every wait is a bounded mbarrier
-// wait (status word on expiry); no TMA multicast.
+// S_pre goes TMA -> shared memory -> tensor core untouched; O and U leave
+// through swizzled staging chunks and TMA stores.  Every wait is a bounded
+// mbarrier wait (status word on expiry); no TMA multicast.
 #include "tv_tc_common.cuh"
 
 namespace {
@@ -35,32 +38,32 @@ constexpr int kThreads = 320;
 constexpr int kComputeWarps = 8;
 constexpr int kSlots = 16;     // path slots per node: depth <= 15
 constexpr int kRows = 64;      // T <= 64
+constexpr int kLd = 17;        // row stride of the slot tables (floats): conflict-free per slot
+constexpr int kLdP = 20;       // row stride of the path table (bytes)
 
-// shared memory map (bytes from the 1024-aligned base); operand tiles are 128 x 128 B,
-// TMA fills rows 0..63 only; the upper halves (rows 64..127) hold scratch and staging
-constexpr uint32_t kOffQ = 0;                    // 2 k-halves of Q; upper halves: O staging 0,1
-constexpr uint32_t kOffK = 2 * kTile;            // 2 k-halves of K; upper halves: O staging 2,3
-constexpr uint32_t kOffV = 4 * kTile;            // 2 dv-halves of V; upper halves: scratch
-constexpr uint32_t kOffS = 6 * kTile;            // 4 k-chunks of S_pre [128 v][32] f32
-constexpr uint32_t kOffW = 10 * kTile;           // [W;A] hi, lo, [W D_P;A D_P] hi, lo: [128][64] bf16
-constexpr int kLd = 17;                          // row stride of the slot tables (floats): no bank
-                                                 // conflict when 32 nodes touch the same slot
-constexpr int kLdP = 20;                         // row stride of the path table (bytes)
-constexpr uint32_t kOffGs = kOffV + 8192;        // float Gs[64][kLd]: G_{i,p_s}
-constexpr uint32_t kOffCs = kOffV + kTile + 8192;  // float Cs[64][kLd]: C_{i,p_s}
+// shared memory map (bytes from the 1024-aligned base); 14 tiles of 128 rows x 128 B
+constexpr uint32_t kOffQK = 0;                   // 2 k-halves: rows 0..63 Q, rows 64..127 K
+constexpr uint32_t kOffV = 2 * kTile;            // 2 dv-halves of V (rows 0..63); upper halves: scratch
+constexpr uint32_t kOffS = 4 * kTile;            // 4 k-chunks of S_pre [128 v][32] f32
+constexpr uint32_t kOffAq = 8 * kTile;           // hi, lo of [diag(P) ; 0]          [128][64] bf16
+constexpr uint32_t kOffAk = 10 * kTile;          // hi, lo of [-(W D_P) ; -(A D_P)]  [128][64] bf16
+constexpr uint32_t kOffW = 12 * kTile;           // hi, lo of [W ; A]                [128][64] bf16
+constexpr uint32_t kOffStage = kOffAk;           // 8 output chunks of 8 KiB (O: 0..3, U: 4..7)
+constexpr uint32_t kOffGs = kOffV + 8192;        // float Gs[64][kLd]: raw K K^T on the path
+constexpr uint32_t kOffCs = kOffV + kTile + 8192;  // float Cs[64][kLd]: raw Q K^T on the path
 constexpr uint32_t kOffPs = kOffCs + 4352;       // uint8 Ps[64][kLdP]: path nodes
-constexpr uint32_t kOffSmall = kOffPs + 1280;    // float g, f, la, be, P [64] each
+constexpr uint32_t kOffSmall = kOffPs + 1280;    // float la[64] (log2 alpha), be[64]
 constexpr uint32_t kOffBar = 14 * kTile;
 constexpr uint32_t kOffMisc = kOffBar + 8 * 24;
 constexpr uint32_t kSmemBytes = kOffMisc + 64 + 1024;
 
 enum Bar {
   QK_FULL = 0, QK_FREE, S_FULL, S_FREE, V_FULL, V_FREE,
-  G_DONE, G_FREE, W_READY, D1_DONE, QF_READY, ACC_DONE, ACC_FREE, SETUP, E1_SYNC,
+  G_DONE, G_FREE, W_READY, D1_DONE, ACC_DONE, ACC_FREE, SETUP, E1_SYNC,
   OST_READY, OST_FREE
 };
 
-constexpr uint32_t kColQf = 0, kColSc1 = 128, kColSc2 = 192, kColD1 = 256, kColAcc = 384;
+constexpr uint32_t kColSc = 0, kColQf = 128, kColAcc = 256;
 
 // Phase timestamps for kernel tuning: compiled out unless TV_TC_PROFILE is defined.
 #ifdef TV_TC_PROFILE
@@ -79,16 +82,9 @@ struct DeltaParams {
   int32_t n_items, B, H, T;
   const float* alpha;
   const float* beta;
-  float* U;        // [items][T][128] or nullptr
+  int32_t want_U;
   int32_t* status;
 };
-
-// fp32 -> tf32 with round-to-nearest (the tensor core would otherwise cut the low 13 bits)
-__device__ __forceinline__ uint32_t to_tf32_rn(float x) {
-  uint32_t r;
-  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
-  return r;
-}
 
 // bf16 hi/lo parts of x (hi = upper 16 bits, lo = upper 16 bits of the exact remainder)
 __device__ __forceinline__ void split_bf16(float x, uint16_t& hi, uint16_t& lo) {
@@ -98,41 +94,39 @@ __device__ __forceinline__ void split_bf16(float x, uint16_t& hi, uint16_t& lo) 
   lo = (uint16_t)(__float_as_uint(x - __uint_as_float(h)) >> 16);
 }
 
+// DMAX: compile-time bound on the tree depth (8 covers draft trees, 15 the rest), so that the
+// per-row triangular solve is straight-line code whose loads all issue up front.
+template <int DMAX>
 __global__ void __launch_bounds__(kThreads, 1)
 verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                        const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmS,
-                       const __grid_constant__ CUtensorMap tmO, const DeltaParams p) {
+                       const __grid_constant__ CUtensorMap tmO, const __grid_constant__ CUtensorMap tmU,
+                       const DeltaParams p) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* sm = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   const uint32_t sbase = smem_u32(sm);
   float* Gs = reinterpret_cast<float*>(sm + kOffGs);
   float* Cs = reinterpret_cast<float*>(sm + kOffCs);
   uint8_t* Ps = reinterpret_cast<uint8_t*>(sm + kOffPs);
-  float* g_s = reinterpret_cast<float*>(sm + kOffSmall);
-  float* f_s = g_s + kRows;
-  float* la_s = f_s + kRows;
+  float* la_s = reinterpret_cast<float*>(sm + kOffSmall);
   float* be_s = la_s + kRows;
-  float* P_s = be_s + kRows;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + kOffMisc);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + kOffMisc + 4);
-  volatile int* range_ok_s = reinterpret_cast<volatile int*>(sm + kOffMisc + 16);
   auto bar = [&](int i) { return sbase + kOffBar + 8u * i; };
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int T = p.T;
-  const bool want_U = p.U != nullptr;
-  const int dmax = p.tree.max_depth_all;   // <= 15, the same for every thread
+  const bool want_U = p.want_U != 0;
 
   if (tid == 0) {
     abort_flag[0] = 0;
     abort_flag[1] = 0;
-    mbar_init(bar(QK_FULL), 1);  mbar_init(bar(QK_FREE), 1 + kComputeWarps);
+    mbar_init(bar(QK_FULL), 1);  mbar_init(bar(QK_FREE), 1);
     mbar_init(bar(S_FULL), 1);   mbar_init(bar(S_FREE), 1);
     mbar_init(bar(V_FULL), 1);   mbar_init(bar(V_FREE), 1);
     mbar_init(bar(G_DONE), 1);   mbar_init(bar(G_FREE), kComputeWarps);
     mbar_init(bar(W_READY), kComputeWarps);
     mbar_init(bar(D1_DONE), 1);
-    mbar_init(bar(QF_READY), kComputeWarps);
     mbar_init(bar(ACC_DONE), 1); mbar_init(bar(ACC_FREE), kComputeWarps);
     mbar_init(bar(SETUP), kComputeWarps);
     mbar_init(bar(E1_SYNC), kComputeWarps);
@@ -151,18 +145,18 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   const uint32_t tmem = *tmem_slot;
 
   if (warp == 0) {
-    // ===================== TMA producer =====================
     if (lane == 0) {
+      // ===================== TMA producer =====================
       int pend_qk = 0, pend_s = 0, pend_v = 0;
       uint32_t it = 0;
       for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++it) {
         const uint32_t ph = it & 1;
         if (!mbar_wait(bar(QK_FREE), ph ^ 1, abort_flag)) break;
         mbar_expect_tx(bar(QK_FULL), 4 * 8192);
-        tma_load_3d(sbase + kOffQ, &tmQ, bar(QK_FULL), 0, 0, item);
-        tma_load_3d(sbase + kOffQ + kTile, &tmQ, bar(QK_FULL), 64, 0, item);
-        tma_load_3d(sbase + kOffK, &tmK, bar(QK_FULL), 0, 0, item);
-        tma_load_3d(sbase + kOffK + kTile, &tmK, bar(QK_FULL), 64, 0, item);
+        tma_load_3d(sbase + kOffQK, &tmQ, bar(QK_FULL), 0, 0, item);
+        tma_load_3d(sbase + kOffQK + kTile, &tmQ, bar(QK_FULL), 64, 0, item);
+        tma_load_3d(sbase + kOffQK + 8192, &tmK, bar(QK_FULL), 0, 0, item);
+        tma_load_3d(sbase + kOffQK + kTile + 8192, &tmK, bar(QK_FULL), 64, 0, item);
         pend_qk = 1 + (int)ph;
         if (!mbar_wait(bar(S_FREE), ph ^ 1, abort_flag)) break;
         mbar_expect_tx(bar(S_FULL), 4 * kTile);
@@ -181,6 +175,24 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         if (pend_s) mbar_wait(bar(S_FULL), pend_s - 1, abort_flag + 1);
         if (pend_v) mbar_wait(bar(V_FULL), pend_v - 1, abort_flag + 1);
       }
+    } else if (lane == 1) {
+      // ===================== output stores =====================
+      // Staged chunks of item k leave by TMA; OST_FREE(k) tells the compute warps that the
+      // chunks (which alias the Ak / W operand tiles) have been read and may be rewritten.
+      uint32_t it = 0;
+      for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++it) {
+        if (!mbar_wait(bar(OST_READY), it & 1, abort_flag)) break;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) tma_store_3d(&tmO, sbase + kOffStage + c * 8192, 32 * c, 0, item);
+        if (want_U) {
+#pragma unroll
+          for (int c = 0; c < 4; ++c) tma_store_3d(&tmU, sbase + kOffStage + (4 + c) * 8192, 32 * c, 0, item);
+        }
+        tma_store_commit();
+        tma_store_wait_read();
+        mbar_arrive(bar(OST_FREE));
+      }
+      tma_store_wait_all();
     }
   } else if (warp == 1) {
     // ===================== MMA issuer =====================
@@ -191,7 +203,7 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       uint32_t it = 0;
       for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++it) {
         const uint32_t ph = it & 1;
-        // Gram tiles: Sc1 = Q K^T, Sc2 = K K^T (N = 64: only nodes j < 64 exist)
+        // Sc = [Q ; K] K^T
         if (!mbar_wait(bar(QK_FULL), ph, abort_flag)) break;
         TCD_STAMP(it, 4);
         if (!mbar_wait(bar(G_FREE), ph ^ 1, abort_flag)) break;
@@ -199,31 +211,30 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
 #pragma unroll
         for (int h = 0; h < 2; ++h)
 #pragma unroll
-          for (int s = 0; s < 4; ++s) {
-            const uint64_t kd = desc_kmajor(sbase + kOffK + h * kTile + s * 32);
-            mma_bf16_ss(tmem + kColSc1, desc_kmajor(sbase + kOffQ + h * kTile + s * 32), kd, kIdGram,
-                        (h | s) != 0);
-            mma_bf16_ss(tmem + kColSc2, kd, kd, kIdGram, (h | s) != 0);
-          }
+          for (int s = 0; s < 4; ++s)
+            mma_bf16_ss(tmem + kColSc, desc_kmajor(sbase + kOffQK + h * kTile + s * 32),
+                        desc_kmajor(sbase + kOffQK + h * kTile + 8192 + s * 32), kIdGram, (h | s) != 0);
         tc_commit(bar(G_DONE));
-        // D1 = [W D_P ; A D_P] K   (A operand: hi/lo tiles, K extent 64; B: K tiles, MN-major)
+        // Qf = [diag(P) | -(W D_P)] [Q ; K]  (rows 64..127: [0 | -(A D_P)])
         if (!mbar_wait(bar(W_READY), ph, abort_flag)) break;
         TCD_STAMP(it, 5);
         tc_fence_after();
 #pragma unroll
-        for (int s = 0; s < 4; ++s) {
-          const uint64_t bdesc = desc_mnmajor(sbase + kOffK + s * 2048, kTile);
-          mma_bf16_ss(tmem + kColD1, desc_kmajor(sbase + kOffW + 2 * kTile + s * 32), bdesc, kIdMn, s != 0);
-          mma_bf16_ss(tmem + kColD1, desc_kmajor(sbase + kOffW + 3 * kTile + s * 32), bdesc, kIdMn, 1);
-        }
+        for (int part = 0; part < 2; ++part)      // hi, lo
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const uint32_t a_tile = (j < 4 ? kOffAq : kOffAk) + part * kTile + (j & 3) * 32;
+            mma_bf16_ss(tmem + kColQf, desc_kmajor(sbase + a_tile),
+                        desc_mnmajor(sbase + kOffQK + j * 2048, kTile), kIdMn, (part | j) != 0);
+          }
         tc_commit(bar(D1_DONE));
         tc_commit(bar(QK_FREE));
-        // acc = Qf S_pre^T
+        // acc = Qf S_pre^T: Qf must be complete in TMEM before it is read as the A operand
+        if (!mbar_wait(bar(D1_DONE), ph, abort_flag)) break;
         if (!mbar_wait(bar(S_FULL), ph, abort_flag)) break;
         TCD_STAMP(it, 6);
-        if (!mbar_wait(bar(QF_READY), ph, abort_flag)) break;
-        TCD_STAMP(it, 7);
         if (!mbar_wait(bar(ACC_FREE), ph ^ 1, abort_flag)) break;
+        TCD_STAMP(it, 7);
         tc_fence_after();
 #pragma unroll
         for (int c = 0; c < 4; ++c)
@@ -251,15 +262,23 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     // ===================== compute warps =====================
     const int cw = warp - 2;
     const int quad = warp & 3;
-    const int hc = cw >> 2;                 // column half handled by this warp
+    const int hc = cw >> 2;                 // which of the two threads of a row
     const int row = quad * 32 + lane;       // tile row
     const int node = row & 63;              // tree node of this row
     const int part = row >> 6;              // 0: O problem, 1: U problem
-    const bool live = node < T && (part == 0 || want_U);             // this row carries a problem
-    const bool warp_live = (quad & 1) * 32 < T && (part == 0 || want_U);   // same for the whole warp: the
-                                                                     // tcgen05.ld/st below are warp-wide
+    const bool rows_live = (quad & 1) * 32 < T;                  // warp-uniform: some row of the warp is a node
+    const bool live = node < T && (part == 0 || want_U);         // this row carries a problem
+    const bool warp_live = rows_live && (part == 0 || want_U);   // same, for the warp-wide tcgen05.ld/st
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
     const uint32_t swz = (uint32_t)(row & 7);
+    const uint32_t nswz = (uint32_t)(node & 7);
+
+    // the [diag(P) ; 0] tiles are zero except for the diagonal, which E2 rewrites per item
+    {
+      const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+      uint4* aq = reinterpret_cast<uint4*>(sm + kOffAq);
+      for (int i = tid - 64; i < (int)(2 * kTile / 16); i += kComputeWarps * 32) aq[i] = z;
+    }
 
     uint64_t nm = 0;
     float nal = 1.f, nbe = 0.f;
@@ -275,15 +294,10 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     };
     fetch_meta(blockIdx.x);
 
-    // Output of the previous item: acc rows 0..63 -> O (staging tiles + TMA store),
-    // rows 64..127 -> U (plain stores, off the critical path).
-    auto final_epilogue = [&](uint32_t it_prev, int item_prev) -> bool {
-      if (warp == 2 && lane == 0) {
-        tma_store_wait_read();            // the store of the item before has read the staging tiles
-        mbar_arrive(bar(OST_FREE));
-      }
+    // acc rows 0..63 -> O chunks 0..3, rows 64..127 -> U chunks 4..7 (the chunks alias the Ak / W
+    // tiles, which are idle between the readout MMA of item k and E2 of item k+1)
+    auto final_epilogue = [&](uint32_t it_prev) -> bool {
       if (!mbar_wait_warp(bar(ACC_DONE), it_prev & 1, abort_flag)) return false;
-      if (!mbar_wait_warp(bar(OST_FREE), it_prev & 1, abort_flag)) return false;
       tc_fence_after();
       if (warp_live) {
 #pragma unroll
@@ -291,21 +305,11 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           uint32_t r1[32];
           tmem_ld32(tmem + lane_addr + kColAcc + hc * 64 + half * 32, r1);
           tmem_wait_ld();
-          if (!live) continue;
-          if (part == 0) {
-            const int c4 = hc * 2 + half;   // 32-column chunk -> upper half of Q0, Q1, K0, K1 tiles
-            unsigned char* orow = sm + kOffQ + c4 * kTile + 8192 + node * 128;
+          unsigned char* orow = sm + kOffStage + (part * 4 + hc * 2 + half) * 8192 + node * 128;
 #pragma unroll
-            for (int c = 0; c < 8; ++c)
-              *reinterpret_cast<uint4*>(orow + (((uint32_t)c ^ swz) << 4)) =
-                  make_uint4(r1[4 * c], r1[4 * c + 1], r1[4 * c + 2], r1[4 * c + 3]);
-          } else {
-            float* urow = p.U + ((size_t)item_prev * T + node) * 128 + hc * 64 + half * 32;
-#pragma unroll
-            for (int c = 0; c < 8; ++c)
-              *reinterpret_cast<uint4*>(urow + 4 * c) =
-                  make_uint4(r1[4 * c], r1[4 * c + 1], r1[4 * c + 2], r1[4 * c + 3]);
-          }
+          for (int c = 0; c < 8; ++c)
+            *reinterpret_cast<uint4*>(orow + (((uint32_t)c ^ nswz) << 4)) =
+                make_uint4(r1[4 * c], r1[4 * c + 1], r1[4 * c + 2], r1[4 * c + 3]);
         }
       }
       fence_async_smem();
@@ -315,83 +319,44 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         mbar_arrive(bar(ACC_FREE));
         mbar_arrive(bar(OST_READY));
       }
-      if (warp == 2 && lane == 0) {
-        if (mbar_wait(bar(OST_READY), it_prev & 1, abort_flag)) {
-#pragma unroll
-          for (int c = 0; c < 4; ++c)
-            tma_store_3d(&tmO, sbase + kOffQ + c * kTile + 8192, 32 * c, 0, item_prev);
-          tma_store_commit();
-        }
-      }
       return true;
     };
 
     uint32_t it = 0;
     bool ok = true;
-    int item_prev = 0;
     for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++it) {
       const uint32_t ph = it & 1;
       if (warp == 4) TCD_STAMP(it, 16);
-      const uint64_t m = nm;                                  // strict ancestors
-      const float be = nbe;
-      const float la_own = log2f(nal);
-      const bool writer = part == 0 && hc == 0 && node < T;   // one thread per node fills the tables
-      if (writer) { la_s[node] = la_own; be_s[node] = be; }
+      // ---- per-node tables of this item ----
+      const uint64_t m = node < T ? nm : 0ull;                // strict ancestors
+      if (part == 0 && hc == 0 && node < T) {
+        la_s[node] = log2f(nal);
+        be_s[node] = nbe;
+      }
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(SETUP));
       fetch_meta(item + (int)gridDim.x);
-      if (!(ok = mbar_wait_warp(bar(SETUP), 0, abort_flag))) break;
-      float g = 0.f;
-      if (node < T) {
-        g = la_own;
-        uint64_t a0 = m;
-        while (a0) { const int j = __ffsll((long long)a0) - 1; a0 &= a0 - 1; g += la_s[j]; }
-      }
-      const float Pi = exp2f(g);
-      if (writer) { g_s[node] = g; f_s[node] = exp2f(-g); P_s[node] = Pi; }
-      const bool range_ok_warp = __all_sync(0xffffffffu, node >= T || fabsf(g) <= 100.f);
-      if (lane == 0) range_ok_s[cw] = range_ok_warp;
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(SETUP));
       const int depth = __popcll(m);
-      const uint64_t mplus = m | (1ull << node);
 
-      // ---- E1: path-sparse rows of C (from Q K^T) and G (from K K^T) ----
-      if (warp == 4) TCD_STAMP(it, 17);
+      // ---- E1: raw path-sparse rows: part 0 <- Q K^T (path incl. the node), part 1 <- K K^T ----
       if (!(ok = mbar_wait_warp(bar(G_DONE), ph, abort_flag))) break;
       if (warp == 4) TCD_STAMP(it, 18);
-      if (!(ok = mbar_wait_warp(bar(SETUP), 1, abort_flag))) break;
       tc_fence_after();
-      bool fast = true;
+      if (rows_live) {
+        const uint64_t sel = node < T ? (part == 0 ? (m | (1ull << node)) : m) : 0ull;
+        float* dst = (part == 0 ? Cs : Gs) + node * kLd;
+        const int cbase = hc * 32;
+        const uint32_t bits = (uint32_t)(sel >> cbase);
+        const int base = hc ? __popc((uint32_t)sel) : 0;      // slots taken by columns 0..31
+        uint32_t r[32];
+        tmem_ld32(tmem + lane_addr + kColSc + cbase, r);
+        tmem_wait_ld();
 #pragma unroll
-      for (int w8 = 0; w8 < kComputeWarps; ++w8) fast = fast && range_ok_s[w8];
-      if (part == 0 && warp_live) {
-        const uint64_t sel = node < T ? (hc == 0 ? mplus : m) : 0ull;
-        float* dst = (hc == 0 ? Cs : Gs) + node * kLd;
-        const float lead = (hc == 0 ? 1.f : be) * (fast ? Pi : 1.f);
-#pragma unroll 1
-        for (int half = 0; half < 2; ++half) {
-          uint32_t r[32];
-          tmem_ld32(tmem + lane_addr + (hc == 0 ? kColSc1 : kColSc2) + half * 32, r);
-          tmem_wait_ld();
-          const uint32_t bits = (uint32_t)(sel >> (half * 32));
-          const int base = half ? __popc((uint32_t)sel) : 0;   // slots taken by columns 0..31
-          // Every column is independent: its slot is the number of selected columns before it.
-#pragma unroll
-          for (int q4 = 0; q4 < 8; ++q4) {
-            const float4 f4 = *reinterpret_cast<const float4*>((fast ? f_s : g_s) + half * 32 + q4 * 4);
-            const float fv[4] = {f4.x, f4.y, f4.z, f4.w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const int jj = q4 * 4 + e;
-              const float ratio = fast ? fv[e] : exp2f(g - fv[e]);   // P_i / P_j (times P_i in `lead`)
-              const float val = lead * ratio * __uint_as_float(r[jj]);
-              // unselected columns land in the padding slot of the row: no branch, no predicate
-              const int slot = ((bits >> jj) & 1u) ? base + __popc(bits & ((1u << jj) - 1u)) : kSlots;
-              dst[slot] = val;
-              if (hc == 0) Ps[node * kLdP + slot] = (uint8_t)(half * 32 + jj);
-            }
-          }
+        for (int jj = 0; jj < 32; ++jj) {
+          // unselected columns land in the padding slot of the row: no branch, no predicate
+          const int slot = ((bits >> jj) & 1u) ? base + __popc(bits & ((1u << jj) - 1u)) : kSlots;
+          dst[slot] = __uint_as_float(r[jj]);
+          if (part == 0) Ps[node * kLdP + slot] = (uint8_t)(cbase + jj);
         }
       }
       tc_fence_before();
@@ -401,120 +366,90 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         mbar_arrive(bar(E1_SYNC));
       }
       if (warp == 4) TCD_STAMP(it, 19);
+      // ---- output of the previous item (its MMAs ran under E1 above) ----
+      if (it > 0 && !(ok = final_epilogue(it - 1))) break;
+      if (warp == 4) TCD_STAMP(it, 17);
+      if (!(ok = mbar_wait_warp(bar(SETUP), ph, abort_flag))) break;
       if (!(ok = mbar_wait_warp(bar(E1_SYNC), ph, abort_flag))) break;
       if (warp == 4) TCD_STAMP(it, 20);
 
-      // ---- E2: one back-substitution per row on the path system, then the operand tiles ----
-      if (hc == 0 && live) {
-        // path nodes and the right-hand side into registers (16 slots, statically indexed)
+      // ---- E2: decay factors, one back-substitution per row, operand tiles ----
+      constexpr int NS = DMAX + 1;                            // path slots in use
+      int path[NS];
+      float gp[NS], bt[NS], vec[NS];
+      float gi = 0.f;
+      if (live) {
         const uint32_t* pw = reinterpret_cast<const uint32_t*>(Ps + node * kLdP);
         const uint32_t pword[4] = {pw[0], pw[1], pw[2], pw[3]};
-        int path[kSlots];
+        float run = 0.f;
 #pragma unroll
-        for (int s2 = 0; s2 < kSlots; ++s2) path[s2] = (pword[s2 >> 2] >> ((s2 & 3) * 8)) & 0xff;
-        float vec[kSlots];
-        if (part == 0) {
-#pragma unroll
-          for (int s2 = 0; s2 < kSlots; ++s2) vec[s2] = s2 <= depth ? Cs[node * kLd + s2] : 0.f;
-        } else {
-#pragma unroll
-          for (int s2 = 0; s2 < kSlots; ++s2) vec[s2] = s2 == depth ? 1.f : 0.f;   // x L = e_d
+        for (int s2 = 0; s2 < NS; ++s2) {
+          path[s2] = (pword[s2 >> 2] >> ((s2 & 3) * 8)) & 63;
+          const bool on = s2 <= depth;
+          const float la = la_s[path[s2]], b2 = be_s[path[s2]];
+          bt[s2] = on ? b2 : 0.f;
+          run += on ? la : 0.f;      // log2 of P at path node s2
+          gp[s2] = run;
+          if (s2 == depth) gi = run;
         }
-        if (warp == 4) TCD_STAMP(it, 25);
-        // w_s = c_s - sum_{t > s} w_t G_{p_t, p_s}, from the node upwards
 #pragma unroll
-        for (int s2 = kSlots - 2; s2 >= 0; --s2) {
-          if (s2 < dmax) {                                    // CTA-uniform bound
-            // slots past the node's depth hold vec = 0 and a deselected G: loads carry no predicate
-            float acc = vec[s2];
+        for (int s2 = 0; s2 < NS; ++s2) {
+          const float c = Cs[node * kLd + s2];
+          if (part == 0) vec[s2] = s2 <= depth ? c * exp2f(gi - gp[s2]) : 0.f;   // C_{i,p_s}
+          else vec[s2] = s2 == depth ? 1.f : 0.f;                               // x L = e_d
+        }
+        // w_s = c_s - sum_{t > s} w_t G_{p_t,p_s},  G_{p_t,p_s} = beta_t 2^(gp_t - gp_s) k_t.k_s;
+        // slots past the node's depth carry vec = 0 and a deselected G, so nothing is predicated
 #pragma unroll
-            for (int t = s2 + 1; t < kSlots; ++t) {
-              const float gts = Gs[(path[t] & 63) * kLd + s2];
-              acc = fmaf(-vec[t], t <= depth ? gts : 0.f, acc);
-            }
-            if (s2 < depth) vec[s2] = acc;
+        for (int s2 = NS - 2; s2 >= 0; --s2) {
+          float acc = vec[s2];
+#pragma unroll
+          for (int t = s2 + 1; t < NS; ++t) {
+            const float gts = Gs[path[t] * kLd + s2] * (bt[t] * exp2f(gp[t] - gp[s2]));
+            acc = fmaf(-vec[t], t <= depth ? gts : 0.f, acc);
           }
+          if (s2 < depth) vec[s2] = acc;
         }
-        if (warp == 4) TCD_STAMP(it, 26);
-        unsigned char* trow = sm + kOffW + row * 128;
+      }
+      // The tiles alias the staged output chunks of the previous item: its stores must have read
+      // them (they did so under the solve above).
+      if (it > 0 && !(ok = mbar_wait_warp(bar(OST_FREE), (it - 1) & 1, abort_flag))) break;
+      if (live) {
+        // hc 0 writes the [W ; A] tiles, hc 1 the -[W D_P ; A D_P] tiles (and the diagonal of P)
+        unsigned char* trow = sm + (hc == 0 ? kOffW : kOffAk) + row * 128;
         const uint4 z = make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
-        for (int tile = 0; tile < 4; ++tile)
+        for (int tile = 0; tile < 2; ++tile)
 #pragma unroll
           for (int c = 0; c < 8; ++c)
             *reinterpret_cast<uint4*>(trow + tile * kTile + (((uint32_t)c ^ swz) << 4)) = z;
-        if (warp == 4) TCD_STAMP(it, 27);
 #pragma unroll
-        for (int s2 = 0; s2 < kSlots; ++s2) {
-          if (s2 <= dmax && s2 <= depth) {
+        for (int s2 = 0; s2 < NS; ++s2) {
+          if (s2 <= depth) {
             const int j = path[s2];
-            const float wv = vec[s2] * be_s[j];                // row of W = C N D_beta (or A = N D_beta)
-            const float wp = wv * P_s[j];                      // row of W D_P (or A D_P)
+            const float wv = vec[s2] * bt[s2];                        // W = C N D_beta (or A = N D_beta)
+            const float val = hc == 0 ? wv : -(wv * exp2f(gp[s2]));   // ... times P_{p_s}, negated
             const uint32_t off = ((((uint32_t)j >> 3) ^ swz) << 4) + ((uint32_t)j & 7u) * 2u;
             uint16_t hi, lo;
-            split_bf16(wv, hi, lo);
+            split_bf16(val, hi, lo);
             *reinterpret_cast<uint16_t*>(trow + off) = hi;
             *reinterpret_cast<uint16_t*>(trow + kTile + off) = lo;
-            split_bf16(wp, hi, lo);
-            *reinterpret_cast<uint16_t*>(trow + 2 * kTile + off) = hi;
-            *reinterpret_cast<uint16_t*>(trow + 3 * kTile + off) = lo;
           }
         }
+        if (part == 0 && hc == 1) {
+          uint16_t hi, lo;
+          split_bf16(exp2f(gi), hi, lo);                              // P_i on the diagonal
+          const uint32_t off = row * 128 + ((((uint32_t)node >> 3) ^ swz) << 4) + ((uint32_t)node & 7u) * 2u;
+          *reinterpret_cast<uint16_t*>(sm + kOffAq + off) = hi;
+          *reinterpret_cast<uint16_t*>(sm + kOffAq + kTile + off) = lo;
+        }
       }
-      if (warp == 4) TCD_STAMP(it, 28);
       fence_async_smem();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(W_READY));
       if (warp == 4) TCD_STAMP(it, 21);
-
-      // ---- output of the previous item, under the D1 MMA of this one ----
-      if (it > 0 && !(ok = final_epilogue(it - 1, item_prev))) break;
-
-      // ---- E3: Qf = [D_P Q - D1 ; -D1] -> TMEM (A operand of the state contraction) ----
-      if (warp == 4) TCD_STAMP(it, 22);
-      if (!(ok = mbar_wait_warp(bar(D1_DONE), ph, abort_flag))) break;
-      if (warp == 4) TCD_STAMP(it, 23);
-      tc_fence_after();
-      if (warp_live) {
-        const unsigned char* qrow = sm + kOffQ + hc * kTile + node * 128;
-        const uint32_t qswz = (uint32_t)(node & 7);
-#pragma unroll
-        for (int half = 0; half < 2; ++half) {
-          uint32_t r[32];
-          tmem_ld32(tmem + lane_addr + kColD1 + hc * 64 + half * 32, r);
-          tmem_wait_ld();
-          if (part == 0) {
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-              const uint4 x = *reinterpret_cast<const uint4*>(qrow + (((half * 4 + c) ^ qswz) << 4));
-              const uint32_t w[4] = {x.x, x.y, x.z, x.w};
-#pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                r[c * 8 + 2 * e] = to_tf32_rn(
-                    fmaf(Pi, __uint_as_float(w[e] << 16), -__uint_as_float(r[c * 8 + 2 * e])));
-                r[c * 8 + 2 * e + 1] = to_tf32_rn(
-                    fmaf(Pi, __uint_as_float(w[e] & 0xffff0000u), -__uint_as_float(r[c * 8 + 2 * e + 1])));
-              }
-            }
-          } else {
-#pragma unroll
-            for (int e = 0; e < 32; ++e) r[e] = to_tf32_rn(-__uint_as_float(r[e]));
-          }
-          tmem_st32(tmem + lane_addr + kColQf + hc * 64 + half * 32, r);
-        }
-        tmem_wait_st();
-      }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) {
-        mbar_arrive(bar(QF_READY));
-        mbar_arrive(bar(QK_FREE));
-      }
-      item_prev = item;
-      if (warp == 4) TCD_STAMP(it, 24);
     }
-    if (ok && it > 0) final_epilogue(it - 1, item_prev);
-    if (warp == 2 && lane == 0) tma_store_wait_all();
+    if (ok && it > 0) final_epilogue(it - 1);
   }
 
   tc_fence_before();
@@ -543,6 +478,8 @@ bool tv_verify_tc_delta_supports(const VerifyArgs& a) {
 int tv_launch_verify_tc_delta(const VerifyArgs& a, int32_t* status, cudaStream_t stream) {
   if (!tv_verify_tc_delta_supports(a)) return TV_ERR_UNSUPPORTED;
   const uint64_t items = (uint64_t)a.L * a.B * a.H;
+  // the U map is only used when U is requested; O stands in otherwise
+  float* Uout = a.U ? a.U : a.O;
   const void* const ptrs[5] = {a.q, a.k, a.v, a.S_pre, a.O};
   const MapSet* ms = cached_maps(ptrs, items, a.T, 1, [&](CUtensorMap* m) {
     return make_map(&m[0], a.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, items, a.T, 128, 64, 64) &&
@@ -551,13 +488,19 @@ int tv_launch_verify_tc_delta(const VerifyArgs& a, int32_t* status, cudaStream_t
            make_map(&m[3], a.S_pre, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, 128, 128, 32, 128) &&
            make_map(&m[4], a.O, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, a.T, 128, 32, 64);
   });
-  if (!ms) return TV_ERR_CUDA;
+  const void* const uptrs[5] = {Uout, nullptr, nullptr, nullptr, nullptr};
+  const MapSet* mu = cached_maps(uptrs, items, a.T, 2, [&](CUtensorMap* m) {
+    return make_map(&m[0], Uout, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, a.T, 128, 32, 64);
+  });
+  if (!ms || !mu) return TV_ERR_CUDA;
   static thread_local int configured_dev = -1;
   static thread_local int sm_count = 0;
   int dev = 0;
   TV_CUDA_TRY(cudaGetDevice(&dev));
   if (configured_dev != dev) {
-    TV_CUDA_TRY(cudaFuncSetAttribute(verify_tc_delta_kernel,
+    TV_CUDA_TRY(cudaFuncSetAttribute(verify_tc_delta_kernel<8>,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
+    TV_CUDA_TRY(cudaFuncSetAttribute(verify_tc_delta_kernel<15>,
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
     TV_CUDA_TRY(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev));
     configured_dev = dev;
@@ -568,11 +511,15 @@ int tv_launch_verify_tc_delta(const VerifyArgs& a, int32_t* status, cudaStream_t
   p.B = a.B; p.H = a.H; p.T = a.T;
   p.alpha = a.alpha;
   p.beta = a.beta;
-  p.U = a.U;
+  p.want_U = a.U != nullptr;
   p.status = status;
   const int grid = (int)(items < (uint64_t)sm_count ? items : (uint64_t)sm_count);
-  verify_tc_delta_kernel<<<grid, kThreads, kSmemBytes, stream>>>(ms->map[0], ms->map[1], ms->map[2], ms->map[3],
-                                                                ms->map[4], p);
+  if (a.tree.max_depth_all <= 8)
+    verify_tc_delta_kernel<8><<<grid, kThreads, kSmemBytes, stream>>>(ms->map[0], ms->map[1], ms->map[2],
+                                                                   ms->map[3], ms->map[4], mu->map[0], p);
+  else
+    verify_tc_delta_kernel<15><<<grid, kThreads, kSmemBytes, stream>>>(ms->map[0], ms->map[1], ms->map[2],
+                                                                    ms->map[3], ms->map[4], mu->map[0], p);
   TV_CUDA_TRY(cudaGetLastError());
   return TV_OK;
 }
