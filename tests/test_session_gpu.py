@@ -1,0 +1,65 @@
+"""Host-buffer round (tv_session_round) and pre-marshalled calls against the oracle."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2608_01651_b200 as tv
+from paper_2608_01651_b200 import inputs
+from tests import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("name,B,H,L", [("c3", 3, 4, 2), ("c4", 2, 4, 1), ("c1", 1, 4, 1)])
+def test_session_round_matches_oracle(name, B, H, L):
+    wl = inputs.workload(name, B=B, H=H, L=L)
+    parents, accepted = inputs.make_trees(wl)
+    layers = [inputs.make_tensors(wl, layer=l) for l in range(L)]
+    host = {k: (None if layers[0][k] is None else torch.stack([x[k] for x in layers]).pin_memory())
+            for k in layers[0]}
+    O = torch.empty(L, B, H, wl.T, wl.dv).pin_memory()
+    S_new = torch.empty_like(host["S_pre"]).pin_memory()
+    sess = tv.Session(L, B, H, wl.T, wl.dk, wl.dv, rule=wl.rule, qkv_dtype=wl.qkv_dtype)
+    S0 = host["S_pre"].clone()
+    for _ in range(2):   # a session is reusable; the host state is not modified
+        sess.round(parents, accepted, host["S_pre"], host["q"], host["k"], host["v"], host["alpha"],
+                   host["beta"], O, S_new)
+    assert torch.equal(host["S_pre"], S0)
+    On, Sn = O.double().numpy(), S_new.double().numpy()
+    for l in range(L):
+        ver, com = pu.oracle_round(wl, parents, accepted, host, layer=l)
+        eO, _, eS = pu.compare(wl, On, None, Sn, ver, com, layer=l)
+        assert eO <= wl.tol and eS <= wl.tol, (l, eO, eS)
+    sess.free()
+    with pytest.raises(tv.TreeVerifyError):     # malformed tree is refused before any copy
+        bad = parents.copy()
+        bad[0, 1] = 5
+        s2 = tv.Session(L, B, H, wl.T, wl.dk, wl.dv, rule=wl.rule, qkv_dtype=wl.qkv_dtype)
+        s2.round(bad, accepted, host["S_pre"], host["q"], host["k"], host["v"], host["alpha"],
+                 host["beta"], O, S_new)
+
+
+def test_prepared_calls_equal_direct_calls():
+    wl = inputs.workload("c3", B=4, H=4)
+    parents, accepted = inputs.make_trees(wl)
+    t = {k: (None if v is None else v.cuda()) for k, v in inputs.make_tensors(wl).items()}
+    tree = tv.tree_build(parents).upload()
+    acc = torch.from_numpy(accepted).cuda()
+    O1 = tv.tree_verify(tree, t["S_pre"], t["q"], t["k"], t["v"], t["alpha"])
+    S1 = torch.empty_like(t["S_pre"])
+    tv.commit_path(tree, acc, t["S_pre"], t["k"], t["v"], t["alpha"], S_new=S1)
+    par = np.ascontiguousarray(parents, dtype=np.int32)
+    refresh = tree.prepare_refresh(par)
+    O2 = torch.empty_like(O1)
+    S2 = torch.empty_like(S1)
+    ver = tv.prepare_tree_verify(tree, t["S_pre"], t["q"], t["k"], t["v"], t["alpha"], O=O2)
+    com = tv.prepare_commit_path(tree, acc, t["S_pre"], t["k"], t["v"], t["alpha"], S_new=S2)
+    for _ in range(2):
+        refresh(); ver(); com()
+    torch.cuda.synchronize()
+    assert torch.equal(O1, O2) and torch.equal(S1, S2)
+    # the refresh re-reads the caller's parent array: a new topology changes the result
+    par[:] = inputs.make_trees(inputs.workload("c3", B=4, H=4, seed=99))[0]
+    refresh(); ver()
+    torch.cuda.synchronize()
+    assert not torch.equal(O1, O2)
