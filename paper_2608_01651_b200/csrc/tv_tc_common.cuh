@@ -188,6 +188,27 @@ inline bool make_map(CUtensorMap* map, const void* base, CUtensorMapDataType dt,
 }
 
 
+// Programmatic dependent launch: the kernel may start while the kernel in front of it on the
+// stream is still running, provided that kernel released its dependents early; whatever reads
+// that kernel's output first passes grid_dependency_wait().
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <class... KArgs, class... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), int grid, int block, size_t smem,
+                                    cudaStream_t stream, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3((unsigned)block);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // Tensor maps depend only on base pointers and shapes: a serving loop calls with the same
 // buffers round after round, so the five encodes of a launch are cached per thread.
 struct MapSet {

@@ -325,6 +325,9 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         nal = p.alpha[(size_t)item * T + row];
       }
     };
+    // the tree metadata may still be on its way (dependent launch): everything above and the
+    // operand loads of the producer warp do not depend on it
+    grid_dependency_wait();
     fetch_meta(blockIdx.x);
 
     uint32_t it = 0;
@@ -537,9 +540,8 @@ int tv_launch_verify_tc(const VerifyArgs& a, int32_t* status, cudaStream_t strea
   p.O = a.O;
   p.status = status;
   const int grid = (int)(items < (uint64_t)sm_count ? items : (uint64_t)sm_count);
-  verify_tc_gated_kernel<<<grid, kThreads, kSmemBytes, stream>>>(ms->map[0], ms->map[1], ms->map[2], ms->map[3],
-                                                                ms->map[4], p);
-  TV_CUDA_TRY(cudaGetLastError());
+  TV_CUDA_TRY(launch_dependent(verify_tc_gated_kernel, grid, kThreads, kSmemBytes, stream, ms->map[0],
+                               ms->map[1], ms->map[2], ms->map[3], ms->map[4], p));
   if (a.U) {
     const size_t n8 = items * a.T * 128 / 8;
     const int blocks = (int)((n8 + 255) / 256 < 4096 ? (n8 + 255) / 256 : 4096);

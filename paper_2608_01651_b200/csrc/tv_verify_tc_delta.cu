@@ -292,6 +292,7 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         nbe = p.beta[(size_t)item * T + node];
       }
     };
+    grid_dependency_wait();   // tree metadata comes from the kernel in front (dependent launch)
     fetch_meta(blockIdx.x);
 
     // acc rows 0..63 -> O chunks 0..3, rows 64..127 -> U chunks 4..7 (the chunks alias the Ak / W
@@ -515,11 +516,11 @@ int tv_launch_verify_tc_delta(const VerifyArgs& a, int32_t* status, cudaStream_t
   p.status = status;
   const int grid = (int)(items < (uint64_t)sm_count ? items : (uint64_t)sm_count);
   if (a.tree.max_depth_all <= 8)
-    verify_tc_delta_kernel<8><<<grid, kThreads, kSmemBytes, stream>>>(ms->map[0], ms->map[1], ms->map[2],
-                                                                   ms->map[3], ms->map[4], mu->map[0], p);
+    TV_CUDA_TRY(launch_dependent(verify_tc_delta_kernel<8>, grid, kThreads, kSmemBytes, stream, ms->map[0],
+                                 ms->map[1], ms->map[2], ms->map[3], ms->map[4], mu->map[0], p));
   else
-    verify_tc_delta_kernel<15><<<grid, kThreads, kSmemBytes, stream>>>(ms->map[0], ms->map[1], ms->map[2],
-                                                                    ms->map[3], ms->map[4], mu->map[0], p);
+    TV_CUDA_TRY(launch_dependent(verify_tc_delta_kernel<15>, grid, kThreads, kSmemBytes, stream, ms->map[0],
+                                 ms->map[1], ms->map[2], ms->map[3], ms->map[4], mu->map[0], p));
   TV_CUDA_TRY(cudaGetLastError());
   return TV_OK;
 }
