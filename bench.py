@@ -47,7 +47,7 @@ DESCR = {
 
 
 # --------------------------------------------------------------------------
-# Algorithmic bytes (what the method must move; the design doc states the formulae)
+# Algorithmic bytes: what the method must move per launch (state once, q/k/v once, outputs once)
 # --------------------------------------------------------------------------
 def verify_bytes_per_layer(wl, with_U: bool) -> int:
     eb = 2 if wl.qkv_dtype == inputs.BF16 else 4
@@ -114,7 +114,7 @@ class ClockSampler:
         try:
             self.p = subprocess.Popen(
                 ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                 "-i", str(index), "-lms", "100"], stdout=self.f, stderr=subprocess.DEVNULL)
+                 "-i", str(index), "-lms", "20"], stdout=self.f, stderr=subprocess.DEVNULL)
         except Exception:
             self.p = None
 
@@ -433,7 +433,7 @@ def run_ours(args, wl, rank, world, local_rank):
             "h2d_bytes_per_step": int(e2e[1]), "d2h_bytes_per_step": int(e2e[2]),
             "steps": e2e[3], "layers": e2e_L,
             "call": "tv_session_round (pinned host buffers in, O and S_new out)"},
-        "gpu_launches": args.steps * (wl.L + 1),
+        "gpu_launches": args.steps * (wl.L + 2),   # per step: metadata kernel, L verify, one commit
         "clocks": clocks,
     }
     print(json.dumps(line, default=_jsonable), flush=True)
@@ -442,7 +442,7 @@ def run_ours(args, wl, rank, world, local_rank):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="c3", choices=sorted(DESCR))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])

@@ -11,8 +11,8 @@ tree_meta_kernel(const int32_t* __restrict__ parent, int32_t n, uint64_t* __rest
                  int32_t* __restrict__ depth, int32_t* __restrict__ parent_dev, int32_t* status) {
   __shared__ int32_t par_s[TV_MAX_NODES];
   const int t = blockIdx.x, i = threadIdx.x;
-  // a verify kernel launched behind this one may start its operand loads now; it waits for
-  // this grid to finish before it reads the metadata
+  // a verify kernel launched behind this one may be scheduled now and set itself up; it waits
+  // for this grid to finish before it reads global memory
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (i < n) par_s[i] = parent[(size_t)t * n + i];
   if (t == 0 && i == 0) *status = 0;

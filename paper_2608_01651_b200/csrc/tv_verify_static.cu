@@ -32,8 +32,8 @@ tree_meta_static_kernel(const int32_t* __restrict__ parent, int32_t n, uint64_t*
                         int32_t* scratch_status, int32_t* user_status) {
   __shared__ int32_t par_s[TV_MAX_NODES];
   const int t = blockIdx.x, i = threadIdx.x;
-  // a verify kernel launched behind this one may start its operand loads now; it waits for
-  // this grid to finish before it reads the metadata
+  // a verify kernel launched behind this one may be scheduled now and set itself up; it waits
+  // for this grid to finish before it reads global memory
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   bool bad = false;
   if (i < n) {

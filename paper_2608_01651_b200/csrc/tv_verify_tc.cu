@@ -149,6 +149,7 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     if (lane == 0) {
       int pend_qk = 0, pend_s = 0, pend_v = 0;
       uint32_t it = 0;
+      grid_dependency_wait();   // inputs may come from the kernel in front (dependent launch)
       for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++it) {
         const uint32_t ph = it & 1;
         if (!mbar_wait(bar(QK_FREE), ph ^ 1, abort_flag)) break;
@@ -325,8 +326,8 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         nal = p.alpha[(size_t)item * T + row];
       }
     };
-    // the tree metadata may still be on its way (dependent launch): everything above and the
-    // operand loads of the producer warp do not depend on it
+    // dependent launch: barrier set-up and the TMEM allocation above ran under the tail of the
+    // kernel in front; everything that reads global memory waits for it here
     grid_dependency_wait();
     fetch_meta(blockIdx.x);
 

@@ -149,6 +149,7 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       // ===================== TMA producer =====================
       int pend_qk = 0, pend_s = 0, pend_v = 0;
       uint32_t it = 0;
+      grid_dependency_wait();   // inputs may come from the kernel in front (dependent launch)
       for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++it) {
         const uint32_t ph = it & 1;
         if (!mbar_wait(bar(QK_FREE), ph ^ 1, abort_flag)) break;
