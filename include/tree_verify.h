@@ -130,6 +130,11 @@ int tv_tree_meta_device(tv_tree* tree, uint64_t* anc, int32_t* depth, void* stre
  * core completion that never came): TV_OK or TV_ERR_DEVICE_TIMEOUT.  After a
  * timeout the outputs of that launch are undefined; the context stays usable. */
 int tv_tree_device_status(tv_tree* tree, void* stream);
+/* Self-test of that mechanism: launches one CTA that waits, with a limit of a
+ * few milliseconds, on a barrier nothing ever signals, and writes what the
+ * kernels would report (TV_ERR_DEVICE_TIMEOUT) to the DEVICE int32 *status.
+ * Nothing faults or hangs; the context stays usable.                          */
+int tv_selftest_wait_timeout(int32_t* status /*dev*/, void* stream);
 int tv_tree_free(tv_tree* tree);
 
 /* ---- verification (Section IV-A Theorem 1, Eq. 2; Eq. 4; Lemma 2 Eq. 5) ----

@@ -61,6 +61,8 @@ def lib() -> ctypes.CDLL:
     L.tv_tree_upload.argtypes = [vp, vp]
     L.tv_tree_free.argtypes = [vp]
     L.tv_tree_device_status.argtypes = [vp, vp]
+    L.tv_selftest_wait_timeout.argtypes = [vp, vp]
+    L.tv_selftest_wait_timeout.restype = ctypes.c_int
     L.tv_tree_meta_device.argtypes = [vp, vp, vp, vp]
     L.tv_tree_meta_device.restype = ctypes.c_int
     L.tv_tree_device_status.restype = ctypes.c_int
@@ -295,6 +297,11 @@ def tree_verify_static(parent, S_pre, q, k, v, alpha, beta=None, *, rule=GATED, 
                                        _ptr(k), _ptr(v), _ptr(alpha), _ptr(beta), _ptr(O), _ptr(U),
                                        _ptr(status), _stream_ptr(stream)), "tv_tree_verify_static")
     return O
+
+
+def selftest_wait_timeout(status, stream=None):
+    """``tv_selftest_wait_timeout``: make a bounded device wait run out; ``status`` is a CUDA int32[1]."""
+    _check(lib().tv_selftest_wait_timeout(_ptr(status), _stream_ptr(stream)), "tv_selftest_wait_timeout")
 
 
 class Prepared:

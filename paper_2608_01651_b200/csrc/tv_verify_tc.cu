@@ -506,6 +506,32 @@ extern "C" __attribute__((visibility("default"))) int tv_debug_set_tc_profile(lo
 }
 #endif
 
+// Self-test of the bounded wait every tensor-core kernel relies on: one CTA waits, with a short
+// limit, on a barrier that nothing ever arrives at, then reports and returns like the kernels do.
+namespace {
+__global__ void wait_timeout_selftest_kernel(int32_t* status) {
+  __shared__ uint64_t bar_mem;
+  __shared__ int abort_flag;
+  const uint32_t bar = smem_u32(&bar_mem);
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    mbar_init(bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  const bool ok = mbar_wait_warp(bar, 0, &abort_flag, 1ll << 22);   // ~2 ms, never satisfied
+  __syncthreads();
+  if (threadIdx.x == 0) atomicExch(status, ok ? (int)TV_OK : (int)TV_ERR_DEVICE_TIMEOUT);
+}
+}  // namespace
+
+extern "C" __attribute__((visibility("default"))) int tv_selftest_wait_timeout(int32_t* status, void* stream) {
+  if (!status || ((uintptr_t)status & 3)) return TV_ERR_BAD_ARG;
+  wait_timeout_selftest_kernel<<<1, 64, 0, (cudaStream_t)stream>>>(status);
+  TV_CUDA_TRY(cudaGetLastError());
+  return TV_OK;
+}
+
 bool tv_verify_tc_supports(const VerifyArgs& a) {
   return a.bf16 && a.dk == 128 && a.dv == 128 && a.rule == TV_GATED && a.T <= 128;
 }

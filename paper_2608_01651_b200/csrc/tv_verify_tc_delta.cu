@@ -86,6 +86,14 @@ struct DeltaParams {
   int32_t* status;
 };
 
+// 2^x in one MUFU instruction (2 ulp; denormal results flush to zero, which is what a decay
+// factor below 2^-126 should do).  The decay exponents are sums of log2(alpha) along a path.
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
 // bf16 hi/lo parts of x (hi = upper 16 bits, lo = upper 16 bits of the exact remainder)
 __device__ __forceinline__ void split_bf16(float x, uint16_t& hi, uint16_t& lo) {
   const uint32_t b = __float_as_uint(x);
@@ -397,7 +405,7 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
 #pragma unroll
         for (int s2 = 0; s2 < NS; ++s2) {
           const float c = Cs[node * kLd + s2];
-          if (part == 0) vec[s2] = s2 <= depth ? c * exp2f(gi - gp[s2]) : 0.f;   // C_{i,p_s}
+          if (part == 0) vec[s2] = s2 <= depth ? c * fast_exp2(gi - gp[s2]) : 0.f;   // C_{i,p_s}
           else vec[s2] = s2 == depth ? 1.f : 0.f;                               // x L = e_d
         }
         // w_s = c_s - sum_{t > s} w_t G_{p_t,p_s},  G_{p_t,p_s} = beta_t 2^(gp_t - gp_s) k_t.k_s;
@@ -407,7 +415,7 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           float acc = vec[s2];
 #pragma unroll
           for (int t = s2 + 1; t < NS; ++t) {
-            const float gts = Gs[path[t] * kLd + s2] * (bt[t] * exp2f(gp[t] - gp[s2]));
+            const float gts = Gs[path[t] * kLd + s2] * (bt[t] * fast_exp2(gp[t] - gp[s2]));
             acc = fmaf(-vec[t], t <= depth ? gts : 0.f, acc);
           }
           if (s2 < depth) vec[s2] = acc;
@@ -430,7 +438,7 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           if (s2 <= depth) {
             const int j = path[s2];
             const float wv = vec[s2] * bt[s2];                        // W = C N D_beta (or A = N D_beta)
-            const float val = hc == 0 ? wv : -(wv * exp2f(gp[s2]));   // ... times P_{p_s}, negated
+            const float val = hc == 0 ? wv : -(wv * fast_exp2(gp[s2]));   // ... times P_{p_s}, negated
             const uint32_t off = ((((uint32_t)j >> 3) ^ swz) << 4) + ((uint32_t)j & 7u) * 2u;
             uint16_t hi, lo;
             split_bf16(val, hi, lo);
@@ -440,7 +448,7 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         }
         if (part == 0 && hc == 1) {
           uint16_t hi, lo;
-          split_bf16(exp2f(gi), hi, lo);                              // P_i on the diagonal
+          split_bf16(fast_exp2(gi), hi, lo);                              // P_i on the diagonal
           const uint32_t off = row * 128 + ((((uint32_t)node >> 3) ^ swz) << 4) + ((uint32_t)node & 7u) * 2u;
           *reinterpret_cast<uint16_t*>(sm + kOffAq + off) = hi;
           *reinterpret_cast<uint16_t*>(sm + kOffAq + kTile + off) = lo;

@@ -63,3 +63,19 @@ def test_prepared_calls_equal_direct_calls():
     refresh(); ver()
     torch.cuda.synchronize()
     assert not torch.equal(O1, O2)
+
+
+def test_bounded_device_wait_reports_and_context_survives():
+    """A wait that nothing satisfies runs out after its limit: the kernel reports a timeout
+    status and returns; later launches on the same context work."""
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    tv.selftest_wait_timeout(status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == -6
+    wl = inputs.workload("c2", B=1, H=2, T=20)
+    parents, accepted = inputs.make_trees(wl)
+    t = {k: (None if v is None else v.cuda()) for k, v in inputs.make_tensors(wl).items()}
+    tree = tv.tree_build(parents).upload()
+    O = tv.tree_verify(tree, t["S_pre"], t["q"], t["k"], t["v"], t["alpha"])
+    tree.device_status()                      # no timeout in a real launch
+    assert torch.isfinite(O).all()
