@@ -1,0 +1,87 @@
+"""CPU fp64 oracle for the tree-parallel causal convolution front end (Stage 1).
+
+TEST INFRASTRUCTURE ONLY (see tree_oracle.py): numpy, float64, imported only by
+tests, the smoke check and the benchmark's CPU-baseline leg.
+
+What it computes.  Section II-A: a linear-attention layer forms q, k and v by
+passing its projected inputs through a short causal depthwise convolution.
+Section IV-C, Stage 1: under a proposal tree the taps of that convolution for a
+node are the node's ancestors along its root-to-node path (then the committed
+context), not its neighbours in the flattened order, and the stage applies the
+convolution, the bias and SiLU in one pass:
+
+    y_i[c] = SiLU( bias[c] + sum_{r=0}^{W-1} w[c][W-1-r] * in_r(i)[c] )
+
+where in_0(i) = x_i, in_1(i) = x_pi(i), in_2(i) = x_pi(pi(i)), ... and, once
+the path reaches the virtual root, the sequence continues into the committed
+context: ctx[W-2] is the token just before the tree, ctx[W-3] the one before
+it, and so on (ctx has W-1 rows, oldest first).  w[c][W-1] multiplies the
+current token (the usual causal depthwise layout), SiLU(z) = z / (1 + e^-z).
+
+Readings of what the paper leaves open, fixed here and listed in the design doc:
+the channel order is [q heads | k heads | v heads]; "normalization ... folded
+into these stages" is read as an optional L2 normalisation of each q and k head
+vector after SiLU, x / sqrt(sum x^2 + eps); the gate formulas are not given by
+the paper and are not part of this operator.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+
+def silu(z):
+    return z / (1.0 + np.exp(-z))
+
+
+def conv_inputs_for_node(x, ctx, parent, i, W):
+    """The W inputs [in_0, ..., in_{W-1}] of node i: itself, then its ancestors
+    from the nearest upwards, then the context from its newest row backwards."""
+    rows = []
+    j = int(i)
+    while j >= 0 and len(rows) < W:
+        rows.append(x[j])
+        j = int(parent[j])
+    back = ctx.shape[0] - 1
+    while len(rows) < W:
+        rows.append(ctx[back])
+        back -= 1
+    return rows
+
+
+def tree_conv(x, ctx, weight, bias, parent):
+    """x [T, C], ctx [W-1, C], weight [C, W], bias [C] or None -> y [T, C]."""
+    T, C = x.shape
+    W = weight.shape[1]
+    y = np.zeros((T, C))
+    for i in range(T):
+        rows = conv_inputs_for_node(x, ctx, parent, i, W)
+        z = np.zeros(C) if bias is None else np.array(bias, dtype=np.float64)
+        for r in range(W):
+            z = z + weight[:, W - 1 - r] * rows[r]
+        y[i] = silu(z)
+    return y
+
+
+def split_heads(y, H, dk, dv, normalize_qk=False, eps=1e-6):
+    """[T, H(2dk+dv)] -> q [H,T,dk], k [H,T,dk], v [H,T,dv] (channel order q|k|v)."""
+    T = y.shape[0]
+    q = y[:, :H * dk].reshape(T, H, dk).transpose(1, 0, 2).copy()
+    k = y[:, H * dk:2 * H * dk].reshape(T, H, dk).transpose(1, 0, 2).copy()
+    v = y[:, 2 * H * dk:].reshape(T, H, dv).transpose(1, 0, 2).copy()
+    if normalize_qk:
+        q = q / np.sqrt((q * q).sum(-1, keepdims=True) + eps)
+        k = k / np.sqrt((k * k).sum(-1, keepdims=True) + eps)
+    return q, k, v
+
+
+def tree_conv_batch(x, ctx, weight, bias, parents, H, dk, dv, normalize_qk=False, eps=1e-6):
+    """x [B,T,C], ctx [B,W-1,C] -> q,k [B,H,T,dk], v [B,H,T,dv]."""
+    B = x.shape[0]
+    qs, ks, vs = [], [], []
+    for b in range(B):
+        par = parents[0] if parents.shape[0] == 1 else parents[b]
+        y = tree_conv(np.asarray(x[b], np.float64), np.asarray(ctx[b], np.float64),
+                      np.asarray(weight, np.float64), None if bias is None else np.asarray(bias, np.float64), par)
+        q, k, v = split_heads(y, H, dk, dv, normalize_qk, eps)
+        qs.append(q); ks.append(k); vs.append(v)
+    return np.stack(qs), np.stack(ks), np.stack(vs)
