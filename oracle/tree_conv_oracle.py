@@ -85,3 +85,37 @@ def tree_conv_batch(x, ctx, weight, bias, parents, H, dk, dv, normalize_qk=False
         q, k, v = split_heads(y, H, dk, dv, normalize_qk, eps)
         qs.append(q); ks.append(k); vs.append(v)
     return np.stack(qs), np.stack(ks), np.stack(vs)
+
+
+def gate_prep(a, b, A_log, dt_bias):
+    """Gate preparation of Stage 1.  The paper names the step and gives no formula; this is the
+    parameterisation of the Gated DeltaNet publication it cites for the layer:
+
+        gamma = exp( -exp(A_log[h]) * softplus(a + dt_bias[h]) )      (decay, in (0, 1])
+        beta  = 1 / (1 + exp(-b))                                     (write strength, in (0, 1))
+
+    a, b [T, H] -> gamma, beta [H, T] (head-major, the layout the verification stage reads).
+    """
+    a = np.asarray(a, np.float64)
+    b = np.asarray(b, np.float64)
+    z = a + np.asarray(dt_bias, np.float64)[None, :]
+    softplus = np.maximum(z, 0.0) + np.log1p(np.exp(-np.abs(z)))
+    gamma = np.exp(-np.exp(np.asarray(A_log, np.float64))[None, :] * softplus)
+    beta = 1.0 / (1.0 + np.exp(-b))
+    return gamma.T.copy(), beta.T.copy()
+
+
+def conv_commit(x, ctx, parent, accepted):
+    """Context rows after the accepted path is committed: the last W-1 rows of the sequence
+    [ctx rows, x along the accepted root-to-node path].  accepted = -1 keeps ctx.
+    (Implied by Section IV-D's commit for a layer whose front end is the convolution: the next
+    round's taps must be the committed tokens; the paper does not spell it out.)"""
+    path = []
+    j = int(accepted)
+    while j >= 0:
+        path.append(j)
+        j = int(parent[j])
+    path.reverse()
+    seq = np.concatenate([ctx, x[path]]) if path else np.array(ctx, copy=True)
+    keep = ctx.shape[0]
+    return seq[seq.shape[0] - keep:].copy()

@@ -102,3 +102,57 @@ def test_head_split_and_normalisation():
     assert np.allclose(np.linalg.norm(qn, axis=-1), 1.0) and np.allclose(np.linalg.norm(kn, axis=-1), 1.0)
     assert np.array_equal(vn, v)
     assert np.allclose(qn * np.linalg.norm(q, axis=-1, keepdims=True), q)
+
+
+def test_gate_prep_closed_forms_and_library():
+    import torch
+    rng = np.random.default_rng(6)
+    T, H = 7, 3
+    a = rng.normal(size=(T, H)) * 3; b = rng.normal(size=(T, H)) * 3
+    A_log = rng.uniform(-1, 2, size=H); dt_bias = rng.uniform(-4, 1, size=H)
+    gamma, beta = cv.gate_prep(a, b, A_log, dt_bias)
+    assert gamma.shape == (H, T) and beta.shape == (H, T)
+    sp = torch.nn.functional.softplus(torch.tensor(a + dt_bias), threshold=1e9).numpy()
+    assert np.allclose(gamma.T, np.exp(-np.exp(A_log) * sp), rtol=1e-13)
+    assert np.allclose(beta.T, torch.sigmoid(torch.tensor(b)).numpy(), rtol=1e-13)
+    # closed forms: softplus(0) = ln 2, sigmoid(0) = 1/2, sigmoid(x) + sigmoid(-x) = 1
+    g0, b0 = cv.gate_prep(np.zeros((1, 1)), np.zeros((1, 1)), np.array([0.0]), np.array([0.0]))
+    assert np.isclose(g0[0, 0], 0.5, rtol=1e-15) and b0[0, 0] == 0.5      # exp(-ln 2)
+    _, bm = cv.gate_prep(a, -b, A_log, dt_bias)
+    assert np.allclose(beta + bm, 1.0, rtol=1e-14)
+    # large arguments: softplus(z) -> z, no overflow
+    g1, _ = cv.gate_prep(np.full((1, 1), 800.0), np.zeros((1, 1)), np.array([-3.0]), np.array([0.0]))
+    assert np.isclose(g1[0, 0], np.exp(-np.exp(-3.0) * 800.0), rtol=1e-13)
+    assert np.all(gamma > 0) and np.all(gamma <= 1)
+
+
+def test_conv_commit_continues_the_linear_sequence():
+    """After committing a path, a follow-up chain convolved with the new context equals the
+    library convolution over [old context, accepted tokens, new tokens]."""
+    rng = np.random.default_rng(7)
+    T, C, W = 12, 4, 4
+    par = rand_tree(T, rng)
+    x = rng.normal(size=(T, C)); ctx = rng.normal(size=(W - 1, C))
+    w = rng.normal(size=(C, W)); bias = rng.normal(size=C)
+    depth = np.zeros(T, dtype=int)
+    for i in range(T):
+        depth[i] = 0 if par[i] < 0 else depth[par[i]] + 1
+    for acc in (-1, int(np.argmin(depth)), int(np.argmax(depth)), T - 1):
+        new_ctx = cv.conv_commit(x, ctx, par, acc)
+        assert new_ctx.shape == ctx.shape
+        path = []
+        j = acc
+        while j >= 0:
+            path.append(j); j = par[j]
+        path.reverse()
+        x2 = rng.normal(size=(5, C))
+        y2 = cv.tree_conv(x2, new_ctx, w, bias, np.arange(-1, 4))
+        seq = np.concatenate([ctx, x[path], x2])
+        for c in range(C):
+            z = np.convolve(seq[:, c], w[c, ::-1])[len(seq) - 5:len(seq)] + bias[c]
+            assert np.allclose(y2[:, c], z / (1 + np.exp(-z)), rtol=1e-12, atol=1e-13)
+    assert np.array_equal(cv.conv_commit(x, ctx, par, -1), ctx)
+    # a path shorter than the window keeps the newest old rows
+    root_child = int(np.argmin(depth))
+    nc = cv.conv_commit(x, ctx, par, root_child)
+    assert np.array_equal(nc[-1], x[root_child]) and np.array_equal(nc[:-1], ctx[1:])
