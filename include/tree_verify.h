@@ -231,6 +231,60 @@ int tv_session_round(tv_session* s, const int32_t* parent /*[n_trees][T]*/,
                      float* O, float* S_new, void* stream);
 int tv_session_free(tv_session* s);
 
+/* ---- Stage 1: tree-parallel convolution and gate preparation (Section II-A,
+ * Section IV-C "Stage 1") -----------------------------------------------------
+ * The layer's front end: a short causal depthwise convolution whose taps for a
+ * tree node are the node itself and its nearest ancestors along the
+ * root-to-node path, continued into the committed context once the path ends,
+ * followed by bias and SiLU.  One layer per call.  With C = H*(2*dk+dv) and the
+ * channel order [q heads | k heads | v heads] (head-major inside each block):
+ *
+ *   y[b][i][c] = SiLU( bias[c] + sum_{r<W} weight[c][W-1-r] * in_r(b,i)[c] ),
+ *   in_0 = x[b][i], in_1 = x[b][pi(i)], ...; past the root: ctx[b][W-2],
+ *   ctx[b][W-3], ...                          SiLU(z) = z / (1 + exp(-z))
+ *
+ * and y is written head-major, in the layout tv_tree_verify reads:
+ *   q, k [B][H][T][dk], v [B][H][T][dv].  normalize_qk != 0 divides every q and
+ *   k head vector by sqrt(sum of squares + eps) (the paper folds
+ *   "normalisation" into its stages without a formula; this is the reading).
+ * Gate preparation (optional: pass gate_a == NULL to skip).  The paper names the
+ * step only; the formulas are those of the Gated DeltaNet layer it cites:
+ *   alpha[b][h][i] = exp(-exp(A_log[h]) * softplus(gate_a[b][i][h] + dt_bias[h]))
+ *   beta [b][h][i] = 1 / (1 + exp(-gate_b[b][i][h]))      (gate_b may be NULL)
+ *
+ * Device pointers, all owned by the caller, none retained:
+ *   x      [B][T][C]   io_dtype        ctx    [B][W-1][C] io_dtype, oldest row first
+ *   weight [C][W]      float           bias   [C] float or NULL
+ *   gate_a, gate_b [B][T][H] io_dtype  A_log, dt_bias [H] float
+ *   q, k, v            io_dtype        alpha, beta [B][H][T] float
+ * x, ctx, q, k, v 16-byte aligned; dk, dv multiples of 8 (bf16) or 4 (float),
+ * at most 256; 1 <= W <= TV_CONV_MAX_TAPS; T <= TV_MAX_NODES.  The tree must be
+ * uploaded (1 tree shared by all requests, or B trees).  Outputs must not alias
+ * inputs.  Asynchronous on `stream`; returns a tv_status, launches nothing on
+ * an error. */
+#define TV_CONV_MAX_TAPS 8
+typedef struct tv_conv_dims {
+  int32_t B, H, T, dk, dv;
+  int32_t W;             /* taps, including the current token           */
+  int32_t io_dtype;      /* tv_dtype of x, ctx, gate_a, gate_b, q, k, v  */
+  int32_t normalize_qk;  /* 0 / 1                                        */
+  float eps;             /* added under the square root                  */
+} tv_conv_dims;
+
+int tv_tree_conv(const tv_tree* tree, const tv_conv_dims* dims, const void* x, const void* ctx,
+                 const float* weight, const float* bias, const void* gate_a, const void* gate_b,
+                 const float* A_log, const float* dt_bias, void* q, void* k, void* v,
+                 float* alpha, float* beta, void* stream);
+
+/* The convolution's context after the accepted path is committed (the
+ * counterpart, for the front end, of Section IV-D's state commit; implied, not
+ * spelled out, by the paper): ctx_new[b] = the last W-1 rows of
+ * [ctx[b] rows, x[b] along the accepted root-to-node path].  accepted[b] = -1
+ * keeps ctx[b].  accepted [B] int32 (device), ctx_new [B][W-1][C] io_dtype;
+ * ctx_new == ctx (in place) is allowed, partial overlap is not. */
+int tv_conv_commit(const tv_tree* tree, const tv_conv_dims* dims, const int32_t* accepted,
+                   const void* x, const void* ctx, void* ctx_new, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -38,6 +38,11 @@ class _Dims(ctypes.Structure):
                 ("L", "B", "H", "T", "dk", "dv", "rule", "qkv_dtype", "impl")]
 
 
+class _ConvDims(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in
+                ("B", "H", "T", "dk", "dv", "W", "io_dtype", "normalize_qk")] + [("eps", ctypes.c_float)]
+
+
 def lib() -> ctypes.CDLL:
     """Load libtreeverify.so; raises if it has not been built."""
     global _lib
@@ -70,6 +75,10 @@ def lib() -> ctypes.CDLL:
     L.tv_commit_path.argtypes = [vp, p(_Dims)] + [vp] * 9
     L.tv_tree_verify_static.argtypes = [vp, i32, p(_Dims)] + [vp] * 10
     L.tv_tree_verify_static.restype = ctypes.c_int
+    L.tv_tree_conv.argtypes = [vp, p(_ConvDims)] + [vp] * 14
+    L.tv_conv_commit.argtypes = [vp, p(_ConvDims)] + [vp] * 5
+    L.tv_tree_conv.restype = ctypes.c_int
+    L.tv_conv_commit.restype = ctypes.c_int
     L.tv_session_create.argtypes = [p(_Dims), i32, p(vp)]
     L.tv_session_round.argtypes = [vp] + [vp] * 11
     L.tv_session_free.argtypes = [vp]
@@ -297,6 +306,84 @@ def tree_verify_static(parent, S_pre, q, k, v, alpha, beta=None, *, rule=GATED, 
                                        _ptr(k), _ptr(v), _ptr(alpha), _ptr(beta), _ptr(O), _ptr(U),
                                        _ptr(status), _stream_ptr(stream)), "tv_tree_verify_static")
     return O
+
+
+def _conv_dims(x, H, dk, dv, W, normalize_qk, eps) -> _ConvDims:
+    import torch
+    if x.dim() != 3 or x.shape[2] != H * (2 * dk + dv):
+        raise ValueError("x must be [B, T, H*(2*dk+dv)]")
+    if x.dtype == torch.bfloat16:
+        dt = BF16
+    elif x.dtype == torch.float32:
+        dt = F32
+    else:
+        raise ValueError("x must be float32 or bfloat16")
+    return _ConvDims(x.shape[0], H, x.shape[1], dk, dv, W, dt, int(bool(normalize_qk)), float(eps))
+
+
+def _conv_args(tree, x, ctx, weight, bias, H, dk, dv, gate_a, gate_b, A_log, dt_bias, normalize_qk, eps,
+               q, k, v, alpha, beta, stream):
+    import torch
+    for t, n in ((x, "x"), (ctx, "ctx"), (gate_a, "gate_a"), (gate_b, "gate_b"), (q, "q"), (k, "k"), (v, "v")):
+        _require(t, n, x.dtype)
+    for t, n in ((weight, "weight"), (bias, "bias"), (A_log, "A_log"), (dt_bias, "dt_bias"),
+                 (alpha, "alpha"), (beta, "beta")):
+        _require(t, n, torch.float32)
+    if weight.dim() != 2 or weight.shape[0] != x.shape[2]:
+        raise ValueError("weight must be [C, W]")
+    W = weight.shape[1]
+    if W > 1 and (ctx is None or tuple(ctx.shape) != (x.shape[0], W - 1, x.shape[2])):
+        raise ValueError("ctx must be [B, W-1, C]")
+    d = _conv_dims(x, H, dk, dv, W, normalize_qk, eps)
+    args = (tree._h, ctypes.byref(d), _ptr(x), _ptr(ctx), _ptr(weight), _ptr(bias), _ptr(gate_a), _ptr(gate_b),
+            _ptr(A_log), _ptr(dt_bias), _ptr(q), _ptr(k), _ptr(v), _ptr(alpha), _ptr(beta), _stream_ptr(stream))
+    keep = (tree, d, x, ctx, weight, bias, gate_a, gate_b, A_log, dt_bias, q, k, v, alpha, beta)
+    return args, keep
+
+
+def tree_conv(tree: Tree, x, ctx, weight, bias=None, *, H, dk, dv, gate_a=None, gate_b=None, A_log=None,
+              dt_bias=None, normalize_qk=False, eps=1e-6, q=None, k=None, v=None, alpha=None, beta=None,
+              stream=None):
+    """``tv_tree_conv``: tree-parallel causal convolution + bias + SiLU (+ q/k normalisation, + gates).
+
+    ``x`` [B,T,C], ``ctx`` [B,W-1,C], ``weight`` f32 [C,W]; returns ``(q, k, v)`` head-major, and
+    ``(q, k, v, alpha, beta)`` when ``gate_a`` is given (``beta`` None without ``gate_b``).
+    """
+    import torch
+    B, T = x.shape[0], x.shape[1]
+    q = torch.empty(B, H, T, dk, device=x.device, dtype=x.dtype) if q is None else q
+    k = torch.empty(B, H, T, dk, device=x.device, dtype=x.dtype) if k is None else k
+    v = torch.empty(B, H, T, dv, device=x.device, dtype=x.dtype) if v is None else v
+    if gate_a is not None and alpha is None:
+        alpha = torch.empty(B, H, T, device=x.device, dtype=torch.float32)
+    if gate_b is not None and beta is None:
+        beta = torch.empty(B, H, T, device=x.device, dtype=torch.float32)
+    args, _keep = _conv_args(tree, x, ctx, weight, bias, H, dk, dv, gate_a, gate_b, A_log, dt_bias,
+                             normalize_qk, eps, q, k, v, alpha, beta, stream)
+    _check(lib().tv_tree_conv(*args), "tv_tree_conv")
+    return (q, k, v) if gate_a is None else (q, k, v, alpha, beta)
+
+
+def prepare_tree_conv(tree: Tree, x, ctx, weight, bias=None, *, H, dk, dv, gate_a=None, gate_b=None,
+                      A_log=None, dt_bias=None, normalize_qk=False, eps=1e-6, q, k, v, alpha=None, beta=None,
+                      stream=None) -> "Prepared":
+    """``tv_tree_conv`` with pre-marshalled arguments; outputs must be given."""
+    args, keep = _conv_args(tree, x, ctx, weight, bias, H, dk, dv, gate_a, gate_b, A_log, dt_bias,
+                            normalize_qk, eps, q, k, v, alpha, beta, stream)
+    return Prepared(lib().tv_tree_conv, "tv_tree_conv", args, keep)
+
+
+def conv_commit(tree: Tree, accepted, x, ctx, *, H, dk, dv, ctx_new=None, stream=None):
+    """``tv_conv_commit``: context rows after the accepted path (in place when ``ctx_new`` is None)."""
+    import torch
+    _require(accepted, "accepted", torch.int32)
+    for t, n in ((x, "x"), (ctx, "ctx"), (ctx_new, "ctx_new")):
+        _require(t, n, x.dtype)
+    out = ctx if ctx_new is None else ctx_new
+    d = _conv_dims(x, H, dk, dv, ctx.shape[1] + 1, False, 0.0)
+    _check(lib().tv_conv_commit(tree._h, ctypes.byref(d), _ptr(accepted), _ptr(x), _ptr(ctx), _ptr(out),
+                                _stream_ptr(stream)), "tv_conv_commit")
+    return out
 
 
 def selftest_wait_timeout(status, stream=None):

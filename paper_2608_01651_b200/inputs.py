@@ -267,6 +267,30 @@ def make_tensors(wl: Workload, layer: int = 0, device: str = "cpu") -> dict:
             "beta": None if beta is None else beta.contiguous()}
 
 
+def make_conv_inputs(wl: Workload, layer: int = 0, device: str = "cpu", W: int = 4) -> dict:
+    """Draw one layer's front-end inputs: projected activations ``x`` [B,T,C] and context rows
+    ``ctx`` [B,W-1,C] in the workload's dtype (C = H(2dk+dv), channel order q|k|v), a depthwise
+    filter ``weight`` f32 [C,W] and ``bias`` f32 [C], gate pre-activations ``gate_a``, ``gate_b``
+    [B,T,H] in the workload's dtype, and the per-head gate parameters ``A_log``, ``dt_bias`` f32 [H]
+    drawn so that the decay lands in the same range as ``make_tensors`` draws it directly."""
+    g = torch.Generator(device=device)
+    g.manual_seed(wl.seed * 1000003 + layer * 7919 + 4241)
+    B, H, T, dk, dv = wl.B, wl.H, wl.T, wl.dk, wl.dv
+    C = H * (2 * dk + dv)
+
+    def randn(*shape):
+        return torch.randn(*shape, generator=g, device=device, dtype=torch.float32)
+
+    def rand(*shape):
+        return torch.rand(*shape, generator=g, device=device, dtype=torch.float32)
+
+    dt = wl.torch_dtype
+    return {"x": randn(B, T, C).to(dt).contiguous(), "ctx": randn(B, W - 1, C).to(dt).contiguous(),
+            "weight": (randn(C, W) / W ** 0.5).contiguous(), "bias": (0.1 * randn(C)).contiguous(),
+            "gate_a": randn(B, T, H).to(dt).contiguous(), "gate_b": randn(B, T, H).to(dt).contiguous(),
+            "A_log": (-2.0 + 2.5 * rand(H)).contiguous(), "dt_bias": (-3.0 + 2.0 * rand(H)).contiguous()}
+
+
 def to_f64(t):
     """Widen exactly the values the GPU receives to float64 numpy."""
     if t is None:
