@@ -257,7 +257,7 @@ int tv_session_free(tv_session* s);
  *   weight [C][W]      float           bias   [C] float or NULL
  *   gate_a, gate_b [B][T][H] io_dtype  A_log, dt_bias [H] float
  *   q, k, v            io_dtype        alpha, beta [B][H][T] float
- * x, ctx, q, k, v 16-byte aligned; dk, dv multiples of 8 (bf16) or 4 (float),
+ * x, ctx, weight, bias, q, k, v 16-byte aligned; dk, dv multiples of 8 (bf16) or 4 (float),
  * at most 256; 1 <= W <= TV_CONV_MAX_TAPS; T <= TV_MAX_NODES.  The tree must be
  * uploaded (1 tree shared by all requests, or B trees).  Outputs must not alias
  * inputs.  Asynchronous on `stream`; returns a tv_status, launches nothing on

@@ -2,19 +2,25 @@
 // + bias + SiLU, optional q/k normalisation, gate preparation, and the head-major layout the
 // verification kernels read -- one pass over the projected activations.
 //
-// The work is a gather along parent links with W taps per output and no reuse beyond the tile,
-// so it is bound by HBM: x is read once, q/k/v are written once.  One CTA owns one
-// (request, head, q|k|v) slice: T rows of d channels.  It stages the slice (plus the W-1 context
-// rows) in shared memory with 16-byte streaming loads, derives each node's W tap rows from the
-// parent array once, and then one warp per node row gathers the taps from shared memory, so a
-// row's sum of squares (for the normalisation) is a warp reduction and the row leaves as one
-// contiguous store.
+// Traffic is minimal (x is read once, q/k/v are written once), but per output element the
+// operator needs W unpack+multiply-add pairs, a SiLU (two special-function operations) and its
+// share of the row normalisation: about 20 instructions per 4 bytes moved, so on this GPU the
+// kernel is bound by instruction issue before it is bound by HBM.  The design therefore spends
+// its effort on instructions per element: persistent CTAs walk (request, head, q|k|v) slices so
+// that the filter stays in registers, rows arrive by cp.async one item ahead, each node's W tap
+// rows are derived from the parent array once per item into a table of shared-memory offsets,
+// and a half-warp owns a node row (8 channels per lane), so a row's sum of squares is a 4-step
+// shuffle reduction and the row leaves as contiguous 16-byte stores.
 #include <cuda_bf16.h>
 
 #include "tv_internal.h"
 
 namespace {
 
+// Two CTAs per SM (up to 128 registers, no spills) with the row loop unrolled twice measured
+// faster than three CTAs at 80 registers: the kernel is bound by instruction issue, not by occupancy.
+constexpr int kConvMinBlocks = 2;
+constexpr int kConvUnroll = 2;
 constexpr int kConvThreads = 256;
 constexpr int kConvWarps = kConvThreads / 32;
 constexpr int kMaxConvDim = 256;
@@ -23,6 +29,7 @@ struct ConvArgs {
   const int32_t* parent;  // [n_trees][T]
   int32_t n_trees;
   int32_t B, H, T, dk, dv, W, normalize;
+  int32_t single;  // one row buffer only (two do not fit): no prefetch of the next item's rows
   float eps;
   const void* x;      // [B][T][C]
   const void* ctx;    // [B][W-1][C]
@@ -39,14 +46,6 @@ struct ConvArgs {
   float* beta;
 };
 
-__device__ __forceinline__ uint4 ld_stream16(const void* p) {
-  uint4 r;
-  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
-               : "l"(p));
-  return r;
-}
-
 // For memory the same kernel also writes (the in-place context commit): a coherent load that the
 // compiler may not reorder against the stores.
 __device__ __forceinline__ uint4 ld_ordered16(const void* p) {
@@ -61,176 +60,329 @@ __device__ __forceinline__ uint4 ld_ordered16(const void* p) {
 __device__ __forceinline__ float to_f32(float v) { return v; }
 __device__ __forceinline__ float to_f32(__nv_bfloat16 v) { return __bfloat162float(v); }
 
-// four consecutive channels of one staged row
-__device__ __forceinline__ void load4(const float* row, int c, float (&o)[4]) {
-  const float4 t = *reinterpret_cast<const float4*>(row + c);
-  o[0] = t.x; o[1] = t.y; o[2] = t.z; o[3] = t.w;
-}
-__device__ __forceinline__ void load4(const __nv_bfloat16* row, int c, float (&o)[4]) {
-  const uint2 t = *reinterpret_cast<const uint2*>(row + c);
-  o[0] = __uint_as_float(t.x << 16);
-  o[1] = __uint_as_float(t.x & 0xffff0000u);
-  o[2] = __uint_as_float(t.y << 16);
-  o[3] = __uint_as_float(t.y & 0xffff0000u);
-}
-__device__ __forceinline__ void store4(float* dst, const float (&y)[4]) {
-  asm volatile("st.global.L1::no_allocate.v4.f32 [%0], {%1,%2,%3,%4};" ::"l"(dst), "f"(y[0]),
-               "f"(y[1]), "f"(y[2]), "f"(y[3])
-               : "memory");
-}
-__device__ __forceinline__ void store4(__nv_bfloat16* dst, const float (&y)[4]) {
-  const __nv_bfloat162 lo = __floats2bfloat162_rn(y[0], y[1]);
-  const __nv_bfloat162 hi = __floats2bfloat162_rn(y[2], y[3]);
-  asm volatile("st.global.L1::no_allocate.v2.u32 [%0], {%1,%2};" ::"l"(dst),
-               "r"(*reinterpret_cast<const uint32_t*>(&lo)),
-               "r"(*reinterpret_cast<const uint32_t*>(&hi))
-               : "memory");
+// Lane geometry.  A node row of one 128-channel chunk is handled by 16 lanes with 8 channels
+// each, as two groups of four.  bf16: the groups are adjacent (one 16-byte shared-memory read
+// per tap and one 16-byte store).  f32: the groups sit 64 channels apart, so that each of the
+// two 16-byte reads of a half-warp covers 256 contiguous bytes (no bank conflict).
+template <typename IO> struct Geo;
+template <> struct Geo<__nv_bfloat16> {
+  static __device__ __forceinline__ int g0(int l16) { return 8 * l16; }
+  static __device__ __forceinline__ int g1(int l16) { return 8 * l16 + 4; }
+};
+template <> struct Geo<float> {
+  static __device__ __forceinline__ int g0(int l16) { return 4 * l16; }
+  static __device__ __forceinline__ int g1(int l16) { return 64 + 4 * l16; }
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ uint4 lds16(uint32_t addr) {
+  uint4 r;
+  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "r"(addr));
+  return r;
 }
 
-// SiLU(z) = z / (1 + e^-z).  e^-z overflows to +inf for z < -88 and the quotient is then -0.
-__device__ __forceinline__ float silu(float z) { return __fdividef(z, 1.0f + __expf(-z)); }
+// The eight staged values of this lane for one tap row; a0 / a1 are the shared-memory byte
+// addresses of the lane's two channel groups in that row (bf16 reads both with one load).
+__device__ __forceinline__ void load8(const __nv_bfloat16*, uint32_t a0, uint32_t, float (&o)[8]) {
+  const uint4 t = lds16(a0);
+  o[0] = __uint_as_float(t.x << 16); o[1] = __uint_as_float(t.x & 0xffff0000u);
+  o[2] = __uint_as_float(t.y << 16); o[3] = __uint_as_float(t.y & 0xffff0000u);
+  o[4] = __uint_as_float(t.z << 16); o[5] = __uint_as_float(t.z & 0xffff0000u);
+  o[6] = __uint_as_float(t.w << 16); o[7] = __uint_as_float(t.w & 0xffff0000u);
+}
+__device__ __forceinline__ void load8(const float*, uint32_t a0, uint32_t a1, float (&o)[8]) {
+  const uint4 a = lds16(a0), b = lds16(a1);
+  o[0] = __uint_as_float(a.x); o[1] = __uint_as_float(a.y); o[2] = __uint_as_float(a.z); o[3] = __uint_as_float(a.w);
+  o[4] = __uint_as_float(b.x); o[5] = __uint_as_float(b.y); o[6] = __uint_as_float(b.z); o[7] = __uint_as_float(b.w);
+}
+__device__ __forceinline__ void store8(__nv_bfloat16* row, int g0, int, bool live0, bool, const float (&y)[8]) {
+  uint32_t p[4];
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const __nv_bfloat162 t = __floats2bfloat162_rn(y[2 * e], y[2 * e + 1]);
+    p[e] = *reinterpret_cast<const uint32_t*>(&t);
+  }
+  if (live0)
+    asm volatile("st.global.L1::no_allocate.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(row + g0), "r"(p[0]), "r"(p[1]),
+                 "r"(p[2]), "r"(p[3])
+                 : "memory");
+}
+__device__ __forceinline__ void store8(float* row, int g0, int g1, bool live0, bool live1, const float (&y)[8]) {
+  if (live0)
+    asm volatile("st.global.L1::no_allocate.v4.f32 [%0], {%1,%2,%3,%4};" ::"l"(row + g0), "f"(y[0]), "f"(y[1]),
+                 "f"(y[2]), "f"(y[3])
+                 : "memory");
+  if (live1)
+    asm volatile("st.global.L1::no_allocate.v4.f32 [%0], {%1,%2,%3,%4};" ::"l"(row + g1), "f"(y[4]), "f"(y[5]),
+                 "f"(y[6]), "f"(y[7])
+                 : "memory");
+}
+
+// SiLU(z) = z / (1 + e^-z) in five instructions.  e^-z overflows to +inf for z < -88; its
+// reciprocal is then 0 and the product -0.
+__device__ __forceinline__ float silu(float z) {
+  float e, r;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(z * -1.4426950408889634f));
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(1.0f + e));
+  return z * r;
+}
+__device__ __forceinline__ float rsqrt_fast(float x) {
+  float r;
+  asm("rsqrt.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+  return r;
+}
 
 __device__ __forceinline__ float softplus(float z) {
   return fmaxf(z, 0.0f) + log1pf(expf(-fabsf(z)));
 }
 
-// Shared memory: [T+W-1][d] staged rows (context rows first, oldest first, then the nodes),
-// then the parent array, then 8 tap-row bytes per node.
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async4(uint32_t dst, const void* src) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() {
+  asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+}
+
+// Work items are (slice, request) pairs, slice-major, where a slice is one head's q, k or v
+// channels; a CTA walks a contiguous range of them, so its filter registers are reloaded only
+// when the slice changes.  Shared memory, every block on a 16-byte boundary:
+//   2 x [T+W-1][d] staged rows (context rows first, oldest first, then the nodes),
+//   2 x [T] parents, 2 x [T][WP] byte offsets of each node's tap rows (WP = 4 or 8).
+// While item n is computed, the rows of item n+1 and the parents of item n+2 are in flight
+// (cp.async) and the tap table of item n+1 is derived: one __syncthreads per item.
+struct ConvItem {
+  int slice, b, kind, h, d, c0;
+};
+
 template <typename IO, int W, int NJ>
-__global__ void __launch_bounds__(kConvThreads)
+__global__ void __launch_bounds__(kConvThreads, (NJ == 1 && W <= 4) ? kConvMinBlocks : 1)
 tree_conv_kernel(const ConvArgs a) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   constexpr int VEC = 16 / (int)sizeof(IO);
-  const int T = a.T, H = a.H;
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int slice = blockIdx.x % (3 * H), b = blockIdx.x / (3 * H);
-  const int kind = slice / H, h = slice - kind * H;  // 0 q, 1 k, 2 v
-  const int d = kind == 2 ? a.dv : a.dk;
-  const int C = H * (2 * a.dk + a.dv);
-  const int c0 = kind == 0 ? h * a.dk : kind == 1 ? (H + h) * a.dk : 2 * H * a.dk + h * a.dv;
-  const int dmax = a.dk > a.dv ? a.dk : a.dv;
-  const int rows = T + W - 1;
+  constexpr int WP = W <= 4 ? 4 : 8;
+  const int T = a.T, H = a.H, B = a.B, dk = a.dk, dv = a.dv;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, l16 = lane & 15, half = lane >> 4;
+  const int C = H * (2 * dk + dv);
+  const int dmax = dk > dv ? dk : dv;
+  const int Tp = (T + 3) & ~3;
+  const bool single = a.single != 0;
 
-  IO* xs = reinterpret_cast<IO*>(smem_raw);
-  int32_t* par_s = reinterpret_cast<int32_t*>(smem_raw + (size_t)(T + W - 1) * dmax * sizeof(IO));
-  unsigned char* taps_s = reinterpret_cast<unsigned char*>(par_s + ((T + 1) & ~1));
+  const uint32_t buf_bytes = (uint32_t)(T + W - 1) * dmax * sizeof(IO);
+  const uint32_t xs_u32 = smem_u32(smem_raw);
+  int32_t* par_s = reinterpret_cast<int32_t*>(smem_raw + (single ? 1 : 2) * (size_t)buf_bytes);  // [2][Tp]
+  uint32_t* taps_s = reinterpret_cast<uint32_t*>(par_s + 2 * Tp);                                // [2][T][WP]
+  const uint32_t par_u32 = smem_u32(par_s), taps_u32 = smem_u32(taps_s);
 
-  if (tid < T) par_s[tid] = a.parent[(size_t)(a.n_trees == 1 ? 0 : b) * T + tid];
+  const long long n_items = 3LL * H * B;
+  const int first = (int)(n_items * blockIdx.x / gridDim.x);
+  const int last = (int)(n_items * (blockIdx.x + 1) / gridDim.x);
+  if (first >= last) return;
 
-  // ---- stage the slice: all loads of a batch are issued before the first store
-  {
-    const int vpr = d / VEC, total = rows * vpr;
-    const IO* xb = reinterpret_cast<const IO*>(a.x) + (size_t)b * T * C + c0;
-    const IO* cb = reinterpret_cast<const IO*>(a.ctx) + (size_t)b * (W - 1) * C + c0;
-    for (int base = 0; base < total; base += 4 * kConvThreads) {
-      uint4 r[4];
+  // item cursors advance without divisions
+  auto set_slice = [&](ConvItem& it) {
+    it.kind = it.slice / H;
+    it.h = it.slice - it.kind * H;
+    it.d = it.kind == 2 ? dv : dk;
+    it.c0 = it.kind == 0 ? it.h * dk : it.kind == 1 ? (H + it.h) * dk : 2 * H * dk + it.h * dv;
+  };
+  auto advance = [&](ConvItem& it) {
+    if (++it.b == B) {
+      it.b = 0;
+      ++it.slice;
+      set_slice(it);
+    }
+  };
+  ConvItem cur;
+  cur.slice = first / B;
+  cur.b = first - cur.slice * B;
+  set_slice(cur);
+  ConvItem nxt = cur;
+  advance(nxt);
+  int b2 = nxt.b + 1 == B ? 0 : nxt.b + 1;  // request of the item after next
+
+  // This thread's share of a row block: 16-byte vector tid, tid + 256, ... of [rows][d/VEC];
+  // 256 consecutive vectors advance (rstep rows, cstep vectors).  Recomputed when d changes.
+  int g_d = -1, vpr = 1, rstep = 0, cstep = 0, row0 = 0, cv0 = 0;
+  auto set_geometry = [&](int d) {
+    g_d = d;
+    vpr = d / VEC;
+    rstep = kConvThreads / vpr;
+    cstep = kConvThreads - rstep * vpr;
+    row0 = tid / vpr;
+    cv0 = tid - row0 * vpr;
+  };
+  auto fetch_parents = [&](int b, int slot) {
+    if (tid < T)
+      cp_async4(par_u32 + (uint32_t)(slot * Tp + tid) * 4, a.parent + (size_t)(a.n_trees == 1 ? 0 : b) * T + tid);
+  };
+  auto fetch_rows = [&](const ConvItem& it, int slot) {
+    if (it.d != g_d) set_geometry(it.d);
+    const IO* xb = reinterpret_cast<const IO*>(a.x) + (size_t)it.b * T * C + it.c0;
+    const IO* cb = reinterpret_cast<const IO*>(a.ctx) + (size_t)it.b * (W - 1) * C + it.c0;
+    const uint32_t dctx = xs_u32 + (uint32_t)slot * buf_bytes;
+    const uint32_t dx = dctx + (uint32_t)((W - 1) * it.d * sizeof(IO));
+    int row = row0, cv = cv0;
+    while (row < W - 1) {  // context rows
+      cp_async16(dctx + (uint32_t)((row * it.d + cv * VEC) * sizeof(IO)), cb + (row * C + cv * VEC));
+      row += rstep;
+      cv += cstep;
+      if (cv >= vpr) { cv -= vpr; ++row; }
+    }
+    row = row0;
+    cv = cv0;
+    while (row < T) {  // node rows
+      cp_async16(dx + (uint32_t)((row * it.d + cv * VEC) * sizeof(IO)), xb + (row * C + cv * VEC));
+      row += rstep;
+      cv += cstep;
+      if (cv >= vpr) { cv -= vpr; ++row; }
+    }
+  };
+  auto build_taps = [&](const ConvItem& it, int slot) {
+    if (tid < T) {
+      const uint32_t row_bytes = (uint32_t)it.d * sizeof(IO);
+      const int32_t* par = par_s + slot * Tp;
+      int j = tid, ctx_row = W - 2;
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int idx = base + u * kConvThreads + tid;
-        if (idx < total) {
-          const int row = idx / vpr, col = (idx - row * vpr) * VEC;
-          const IO* src = row < W - 1 ? cb + (size_t)row * C + col : xb + (size_t)(row - (W - 1)) * C + col;
-          r[u] = ld_stream16(src);
+      for (int r = 0; r < W; ++r) {
+        int row;
+        if (j >= 0) {
+          row = W - 1 + j;
+          j = par[j];
+        } else {
+          row = ctx_row--;
+        }
+        taps_s[(slot * T + tid) * WP + r] = (uint32_t)row * row_bytes;
+      }
+    }
+  };
+
+  // ---- prologue: parents of the first two items, rows of the first, taps of the first
+  fetch_parents(cur.b, 0);
+  if (first + 1 < last) fetch_parents(nxt.b, 1);
+  if (!single) fetch_rows(cur, 0);
+  cp_async_wait_all();
+  __syncthreads();
+  build_taps(cur, 0);
+
+  // Dead channel groups (past the slice's width) keep zero weights and read the row's first
+  // bytes, so the row loop is straight-line code; only their store is predicated off.
+  float wreg[NJ][W][8], breg[NJ][8];
+  bool live0[NJ], live1[NJ];
+  uint32_t off0[NJ], off1[NJ];
+  int loaded_slice = -1;
+  const float eps = a.eps;
+  const bool want_norm = a.normalize != 0;
+
+  for (int item = first; item < last; ++item) {
+    const int s = (item - first) & 1, xs_slot = single ? 0 : s;
+    // rows of this item and parents of the next have landed; everyone is done with the last item
+    cp_async_wait_all();
+    __syncthreads();
+    if (single) {
+      fetch_rows(cur, 0);
+      cp_async_wait_all();
+      __syncthreads();
+    }
+    if (item + 1 < last) {
+      if (!single) fetch_rows(nxt, s ^ 1);
+      if (item + 2 < last) fetch_parents(b2, s);
+      build_taps(nxt, s ^ 1);
+    }
+    const int d = cur.d, c0 = cur.c0;
+
+    // ---- this lane's filter taps and bias, when the slice changes
+    if (cur.slice != loaded_slice) {
+      loaded_slice = cur.slice;
+#pragma unroll
+      for (int j = 0; j < NJ; ++j) {
+        const int g0 = 128 * j + Geo<IO>::g0(l16), g1 = 128 * j + Geo<IO>::g1(l16);
+        live0[j] = g0 < d;
+        live1[j] = g1 < d;
+        off0[j] = live0[j] ? (uint32_t)(g0 * sizeof(IO)) : 0u;
+        off1[j] = live1[j] ? (uint32_t)(g1 * sizeof(IO)) : 0u;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const int c = e < 4 ? g0 + e : g1 + e - 4;
+          const bool live = e < 4 ? live0[j] : live1[j];
+          breg[j][e] = live && a.bias ? __ldg(a.bias + c0 + c) : 0.0f;
+#pragma unroll
+          for (int r = 0; r < W; ++r)
+            wreg[j][r][e] = live ? __ldg(a.weight + (size_t)(c0 + c) * W + (W - 1 - r)) : 0.0f;
         }
       }
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int idx = base + u * kConvThreads + tid;
-        if (idx < total) {
-          const int row = idx / vpr, col = (idx - row * vpr) * VEC;
-          *reinterpret_cast<uint4*>(xs + (size_t)row * d + col) = r[u];
-        }
+    }
+
+    // ---- gate preparation for this (request, head): done with the q slice
+    if (cur.kind == 0 && a.gate_a != nullptr && tid < T) {
+      const size_t gi = ((size_t)cur.b * T + tid) * H + cur.h, go = ((size_t)cur.b * H + cur.h) * T + tid;
+      const float ga = to_f32(reinterpret_cast<const IO*>(a.gate_a)[gi]);
+      a.alpha[go] = expf(-expf(__ldg(a.A_log + cur.h)) * softplus(ga + __ldg(a.dt_bias + cur.h)));
+      if (a.gate_b != nullptr) {
+        const float gb = to_f32(reinterpret_cast<const IO*>(a.gate_b)[gi]);
+        a.beta[go] = 1.0f / (1.0f + expf(-gb));
       }
     }
-  }
 
-  // ---- this lane's filter taps and bias: channels 4*lane + 128*j
-  float wreg[NJ][W][4], breg[NJ][4];
-#pragma unroll
-  for (int j = 0; j < NJ; ++j) {
-    const int c = 4 * lane + 128 * j;
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const bool live = c + e < d;
-      breg[j][e] = live && a.bias ? __ldg(a.bias + c0 + c + e) : 0.0f;
-#pragma unroll
-      for (int r = 0; r < W; ++r)
-        wreg[j][r][e] = live ? __ldg(a.weight + (size_t)(c0 + c + e) * W + (W - 1 - r)) : 0.0f;
-    }
-  }
-
-  // ---- gate preparation for this (request, head): done by the q slice
-  if (kind == 0 && a.gate_a != nullptr && tid < T) {
-    const size_t gi = ((size_t)b * T + tid) * H + h, go = ((size_t)b * H + h) * T + tid;
-    const float ga = to_f32(reinterpret_cast<const IO*>(a.gate_a)[gi]);
-    a.alpha[go] = expf(-expf(__ldg(a.A_log + h)) * softplus(ga + __ldg(a.dt_bias + h)));
-    if (a.gate_b != nullptr) {
-      const float gb = to_f32(reinterpret_cast<const IO*>(a.gate_b)[gi]);
-      a.beta[go] = 1.0f / (1.0f + expf(-gb));
-    }
-  }
-  __syncthreads();
-
-  // ---- tap rows of every node: itself, its ancestors, then the context from its newest row
-  if (tid < T) {
-    int j = tid, ctx_row = W - 2;
-#pragma unroll
-    for (int r = 0; r < W; ++r) {
-      int row;
-      if (j >= 0) {
-        row = W - 1 + j;
-        j = par_s[j];
-      } else {
-        row = ctx_row--;
-      }
-      taps_s[tid * 8 + r] = (unsigned char)row;
-    }
-  }
-  __syncthreads();
-
-  // ---- one warp per node row
-  IO* out = reinterpret_cast<IO*>(kind == 0 ? a.q : kind == 1 ? a.k : a.v) + ((size_t)b * H + h) * T * d;
-  const bool norm = a.normalize && kind < 2;
-#pragma unroll 2
-  for (int i = warp; i < T; i += kConvWarps) {
-    const uint2 tw = *reinterpret_cast<const uint2*>(taps_s + i * 8);
-    float y[NJ][4];
-    float ss = 0.0f;
+    // ---- each half-warp takes one node row at a time (the last row is repeated, unstored,
+    // when T is odd)
+    IO* out = reinterpret_cast<IO*>(cur.kind == 0 ? a.q : cur.kind == 1 ? a.k : a.v) +
+              ((size_t)cur.b * H + cur.h) * T * d;
+    const bool norm = want_norm && cur.kind < 2;
+    const uint32_t xs_item = xs_u32 + (uint32_t)xs_slot * buf_bytes;
+    const uint32_t taps_item = taps_u32 + (uint32_t)(s * T) * (WP * 4);
+    uint32_t base0[NJ], base1[NJ];
 #pragma unroll
     for (int j = 0; j < NJ; ++j) {
-      const int c = 4 * lane + 128 * j;
+      base0[j] = xs_item + off0[j];
+      base1[j] = xs_item + off1[j];
+    }
+#pragma unroll kConvUnroll
+    for (int i0 = 2 * warp; i0 < T; i0 += 2 * kConvWarps) {
+      const bool row_live = i0 + half < T;
+      const int i = row_live ? i0 + half : T - 1;
+      uint32_t tap[WP];
+      {
+        const uint4 t0 = lds16(taps_item + (uint32_t)i * (WP * 4));
+        tap[0] = t0.x; tap[1] = t0.y; tap[2] = t0.z; tap[3] = t0.w;
+        if constexpr (WP == 8) {
+          const uint4 t1 = lds16(taps_item + (uint32_t)i * (WP * 4) + 16);
+          tap[4] = t1.x; tap[5] = t1.y; tap[6] = t1.z; tap[7] = t1.w;
+        }
+      }
+      float y[NJ][8];
+      float ss = 0.0f;
 #pragma unroll
-      for (int e = 0; e < 4; ++e) y[j][e] = breg[j][e];
-      if (c < d) {
+      for (int j = 0; j < NJ; ++j) {
 #pragma unroll
         for (int r = 0; r < W; ++r) {
-          const uint32_t row = ((r < 4 ? tw.x : tw.y) >> (8 * (r & 3))) & 0xffu;
-          float in[4];
-          load4(xs + (size_t)row * d, c, in);
+          float in[8];
+          load8((const IO*)nullptr, base0[j] + tap[r], base1[j] + tap[r], in);
 #pragma unroll
-          for (int e = 0; e < 4; ++e) y[j][e] = fmaf(wreg[j][r][e], in[e], y[j][e]);
+          for (int e = 0; e < 8; ++e) y[j][e] = fmaf(wreg[j][r][e], in[e], r == 0 ? breg[j][e] : y[j][e]);
         }
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
+        for (int e = 0; e < 8; ++e) {
           y[j][e] = silu(y[j][e]);
           ss = fmaf(y[j][e], y[j][e], ss);
         }
       }
+#pragma unroll
+      for (int o = 8; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+      const float sc = norm ? rsqrt_fast(ss + eps) : 1.0f;
+#pragma unroll
+      for (int j = 0; j < NJ; ++j) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) y[j][e] *= sc;
+        store8(out + (uint32_t)(i * d + 128 * j), Geo<IO>::g0(l16), Geo<IO>::g1(l16), row_live && live0[j],
+               row_live && live1[j], y[j]);
+      }
     }
-    if (norm) {
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-      const float sc = 1.0f / sqrtf(ss + a.eps);
-#pragma unroll
-      for (int j = 0; j < NJ; ++j)
-#pragma unroll
-        for (int e = 0; e < 4; ++e) y[j][e] *= sc;
-    }
-#pragma unroll
-    for (int j = 0; j < NJ; ++j) {
-      const int c = 4 * lane + 128 * j;
-      if (c < d) store4(out + (size_t)i * d + c, y[j]);
-    }
+    cur = nxt;
+    advance(nxt);
+    b2 = b2 + 1 == B ? 0 : b2 + 1;
   }
 }
 
@@ -284,13 +436,24 @@ int check_conv(const tv_tree* t, const tv_conv_dims* d) {
 }
 
 template <typename IO, int W>
-int launch_conv(const ConvArgs& a, cudaStream_t stream) {
+int launch_conv(const ConvArgs& a_in, cudaStream_t stream) {
+  ConvArgs a = a_in;
   const int dmax = a.dk > a.dv ? a.dk : a.dv;
-  const size_t smem = (size_t)(a.T + W - 1) * dmax * sizeof(IO) + (size_t)((a.T + 1) & ~1) * 4 + (size_t)a.T * 8;
-  const unsigned grid = (unsigned)a.B * 3u * (unsigned)a.H;
+  const size_t buf = (size_t)(a.T + W - 1) * dmax * sizeof(IO);
+  const size_t tables = 2 * ((size_t)((a.T + 3) & ~3) * 4 + (size_t)a.T * (W <= 4 ? 4 : 8) * 4);
+  a.single = 2 * buf + tables > 200 * 1024;
+  const size_t smem = (a.single ? 1 : 2) * buf + tables;
+  int dev = 0, sms = 0;
+  TV_CUDA_TRY(cudaGetDevice(&dev));
+  TV_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
   auto go = [&](auto kernel) -> int {
     if (smem > 48 * 1024)
       TV_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    int per_sm = 0;
+    TV_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kConvThreads, smem));
+    if (per_sm < 1) return TV_ERR_UNSUPPORTED;
+    const long long items = 3LL * a.H * a.B, slots = (long long)sms * per_sm;
+    const unsigned grid = (unsigned)(items < slots ? items : slots);
     kernel<<<grid, kConvThreads, smem, stream>>>(a);
     TV_CUDA_TRY(cudaGetLastError());
     return TV_OK;
@@ -357,7 +520,7 @@ TV_API int tv_tree_conv(const tv_tree* tree, const tv_conv_dims* d, const void* 
   if (gate_a && (!A_log || !dt_bias || !alpha)) return TV_ERR_BAD_ARG;
   if (gate_b && (!gate_a || !beta)) return TV_ERR_BAD_ARG;
   if (!aligned16(x) || !aligned16(ctx) || !aligned16(q) || !aligned16(k) || !aligned16(v) ||
-      ((uintptr_t)weight & 3) || ((uintptr_t)bias & 3) || ((uintptr_t)alpha & 3) || ((uintptr_t)beta & 3) ||
+      !aligned16(weight) || !aligned16(bias) || ((uintptr_t)alpha & 3) || ((uintptr_t)beta & 3) ||
       ((uintptr_t)A_log & 3) || ((uintptr_t)dt_bias & 3))
     return TV_ERR_BAD_ARG;
   const uintptr_t esz = d->io_dtype == TV_BF16 ? 2 : 4;
