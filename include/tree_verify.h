@@ -25,7 +25,8 @@
  *     S_pre, S_new : float  [L][B][H][dv][dk]   (the serving cache layout
  *                    "[H, dv, dk]" of Section IV-D, i.e. the transpose of the
  *                    paper's S in R^{dk x dv})
- *     q, k         : float or bf16 [L][B][H][T][dk]
+ *     q, k         : float or bf16 [L][B][H][T][dk]   ([L][B][Hk][T][dk] with
+ *                    grouped key heads, see tv_dims.Hk)
  *     v            : float or bf16 [L][B][H][T][dv]
  *     alpha, beta  : float  [L][B][H][T]
  *     O, U         : float  [L][B][H][T][dv]
@@ -78,6 +79,10 @@ typedef struct tv_dims {
   int32_t impl;        /* TV_IMPL_AUTO picks the tensor-core kernel when the
                           shape allows it (bf16, dk = dv = 128) and the SIMT
                           fp32 kernel otherwise                                 */
+  int32_t Hk;          /* grouped key heads (Section IV-D: a K factor shared by
+                          several state heads is stored once): q and k have Hk
+                          heads, [L][B][Hk][T][dk], and state head h reads
+                          q/k head h / (H / Hk).  0 means Hk = H; H % Hk == 0. */
 } tv_dims;
 
 const char* tv_strerror(int status);

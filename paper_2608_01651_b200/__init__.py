@@ -35,7 +35,7 @@ class TreeVerifyError(RuntimeError):
 
 class _Dims(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in
-                ("L", "B", "H", "T", "dk", "dv", "rule", "qkv_dtype", "impl")]
+                ("L", "B", "H", "T", "dk", "dv", "rule", "qkv_dtype", "impl", "Hk")]
 
 
 class _ConvDims(ctypes.Structure):
@@ -227,7 +227,10 @@ def _dims(S_pre, k, v, rule, impl) -> _Dims:
         dt = F32
     else:
         raise ValueError("q/k/v must be float32 or bfloat16")
-    return _Dims(L, B, H, T, dk, dv, rule, dt, impl)
+    Hk = k.shape[-3]
+    if H % Hk:
+        raise ValueError("the number of state heads must be a multiple of the number of key heads")
+    return _Dims(L, B, H, T, dk, dv, rule, dt, impl, 0 if Hk == H else Hk)
 
 
 def _require(t, name, dtype=None):
@@ -442,8 +445,8 @@ class Session:
     """Handle of a ``tv_session``: device copies for host-buffer rounds."""
 
     def __init__(self, L, B, H, T, dk, dv, *, rule=GATED, qkv_dtype=BF16, n_trees=None,
-                 impl=IMPL_AUTO):
-        self.dims = _Dims(L, B, H, T, dk, dv, rule, qkv_dtype, impl)
+                 impl=IMPL_AUTO, Hk=None):
+        self.dims = _Dims(L, B, H, T, dk, dv, rule, qkv_dtype, impl, 0 if Hk in (None, H) else Hk)
         self._h = ctypes.c_void_p()
         _check(lib().tv_session_create(ctypes.byref(self.dims), B if n_trees is None else n_trees,
                                        ctypes.byref(self._h)), "tv_session_create")

@@ -244,6 +244,7 @@ static int check_common(const tv_tree* t, const tv_dims* d) {
   if (d->qkv_dtype == TV_BF16 && ((d->dk & 7) || (d->dv & 7))) return TV_ERR_UNSUPPORTED;
   if (t->n != d->T) return TV_ERR_BAD_ARG;
   if (t->n_trees != 1 && t->n_trees != d->B) return TV_ERR_BAD_ARG;
+  if (d->Hk < 0 || d->Hk > d->H || (d->Hk > 0 && d->H % d->Hk != 0)) return TV_ERR_BAD_ARG;
   if ((int64_t)d->L * d->B * d->H > 0x7fffffffLL) return TV_ERR_UNSUPPORTED;
   if (!t->uploaded) return TV_ERR_NOT_UPLOADED;
   return TV_OK;
@@ -273,7 +274,7 @@ TV_API int tv_tree_verify(const tv_tree* tree, const tv_dims* d, const float* S_
   VerifyArgs a;
   a.tree = tree_dev(tree);
   a.L = d->L; a.B = d->B; a.H = d->H; a.T = d->T; a.dk = d->dk; a.dv = d->dv;
-  a.rule = d->rule; a.bf16 = d->qkv_dtype == TV_BF16;
+  a.rule = d->rule; a.bf16 = d->qkv_dtype == TV_BF16; a.Hk = d->Hk ? d->Hk : d->H;
   a.S_pre = S_pre; a.q = q; a.k = k; a.v = v; a.alpha = alpha; a.beta = beta; a.O = O; a.U = U;
   const bool tc_gated = tv_verify_tc_supports(a), tc_delta = tv_verify_tc_delta_supports(a);
   if (d->impl == TV_IMPL_TC && !tc_gated && !tc_delta) return TV_ERR_UNSUPPORTED;
@@ -305,7 +306,7 @@ TV_API int tv_commit_path(const tv_tree* tree, const tv_dims* d, const int32_t* 
   CommitArgs a;
   a.tree = tree_dev(tree);
   a.L = d->L; a.B = d->B; a.H = d->H; a.T = d->T; a.dk = d->dk; a.dv = d->dv;
-  a.rule = d->rule; a.bf16 = d->qkv_dtype == TV_BF16;
+  a.rule = d->rule; a.bf16 = d->qkv_dtype == TV_BF16; a.Hk = d->Hk ? d->Hk : d->H;
   a.accepted = accepted; a.S_pre = S_pre; a.k = k; a.v = v; a.alpha = alpha; a.beta = beta;
   a.U = U; a.S_new = S_new;
   return tv_launch_commit(a, (cudaStream_t)stream);

@@ -107,6 +107,7 @@ __global__ void __launch_bounds__(kThreads) commit_factored_kernel(CommitArgs a)
   }
   const int tb = a.tree.n_trees == 1 ? 0 : b;
   const size_t node0 = (size_t)item * T;  // first node row of this (l, b, h)
+  const size_t qk0 = (size_t)tv_qk_item(item, a.H, a.Hk) * T;  // first key row (grouped key heads)
   const int len = build_path(a.tree, tb, T, acc, a.alpha + node0, path_s, w_s, al_s, &Pa_s);
   const float Pa = Pa_s;
 #pragma unroll
@@ -119,7 +120,7 @@ __global__ void __launch_bounds__(kThreads) commit_factored_kernel(CommitArgs a)
     __syncthreads();
     for (int i = tid; i < nc * dk; i += kThreads) {
       const int p = i / dk, kk = i - p * dk;
-      k_s[p][kk] = load_elem<BF16>(a.k, (node0 + path_s[c0 + p]) * dk + kk);
+      k_s[p][kk] = load_elem<BF16>(a.k, (qk0 + path_s[c0 + p]) * dk + kk);
     }
     for (int i = tid; i < nc * dv; i += kThreads) {
       const int p = i / dv, vv = i - p * dv;
@@ -194,6 +195,7 @@ __global__ void __launch_bounds__(kRowThreads) commit_factored_dk128_kernel(Comm
   }
   const int tb = a.tree.n_trees == 1 ? 0 : b;
   const size_t node0 = (size_t)item * T;
+  const size_t qk0 = (size_t)tv_qk_item(item, a.H, a.Hk) * T;
   const int len = build_path(a.tree, tb, T, acc, a.alpha + node0, path_s, w_s, al_s, &Pa_s);
   const float Pa = Pa_s;
   bool scaled = false;
@@ -202,7 +204,7 @@ __global__ void __launch_bounds__(kRowThreads) commit_factored_dk128_kernel(Comm
     if (c0) __syncthreads();
     for (int i = tid; i < nc * 32; i += kRowThreads) {   // 4 keys per thread per step
       const int p = i >> 5, k4 = i & 31;
-      const size_t idx = (node0 + path_s[c0 + p]) * 128 + k4 * 4;
+      const size_t idx = (qk0 + path_s[c0 + p]) * 128 + k4 * 4;
       float4 kv;
       if (BF16) {
         const uint2 r = *reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(a.k) + idx);
@@ -347,6 +349,7 @@ __global__ void __launch_bounds__(kRowThreads, TV_STREAM_CTAS) commit_stream_dk1
   auto fetch_rows = [&](int u, int nb) {
     const int item = u / n_half, half = u - item * n_half;
     const size_t node0 = (size_t)item * T;
+    const size_t qk0 = (size_t)tv_qk_item(item, a.H, a.Hk) * T;
     const int len = len_s[nb];
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
@@ -355,7 +358,7 @@ __global__ void __launch_bounds__(kRowThreads, TV_STREAM_CTAS) commit_stream_dk1
       kreg[q] = make_uint2(0u, 0u);
       kreg2[q] = make_uint2(0u, 0u);
       if (p < len) {
-        const size_t idx = (node0 + node_s[nb][p]) * 128 + k4 * 4;
+        const size_t idx = (qk0 + node_s[nb][p]) * 128 + k4 * 4;
         if (BF16) {
           kreg[q] = *reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(a.k) + idx);
         } else {
@@ -492,6 +495,7 @@ __global__ void __launch_bounds__(kThreads) commit_delta_rows_kernel(CommitArgs 
   }
   const int tb = a.tree.n_trees == 1 ? 0 : b;
   const size_t node0 = (size_t)item * T;
+  const size_t qk0 = (size_t)tv_qk_item(item, a.H, a.Hk) * T;
   const int len = build_path(a.tree, tb, T, acc, a.alpha + node0, path_s, w_s, al_s, &Pa_s);
 
   float s[kRowsPerWarp][NPL];
@@ -514,7 +518,7 @@ __global__ void __launch_bounds__(kThreads) commit_delta_rows_kernel(CommitArgs 
     __syncthreads();
     for (int i = tid; i < nc * DK; i += kThreads) {
       const int p = i / DK, kk = i - p * DK;
-      k_s[p][kk] = load_elem<BF16>(a.k, (node0 + path_s[c0 + p]) * DK + kk);
+      k_s[p][kk] = load_elem<BF16>(a.k, (qk0 + path_s[c0 + p]) * DK + kk);
     }
     for (int i = tid; i < nc * dv; i += kThreads) {
       const int p = i / dv, vv = i - p * dv;

@@ -42,6 +42,7 @@ struct TreeDev {
 struct VerifyArgs {
   TreeDev tree;
   int32_t L, B, H, T, dk, dv, rule, bf16;
+  int32_t Hk;  // q/k heads (H % Hk == 0); state head h reads q/k head h / (H / Hk)
   const float* S_pre;
   const void* q;
   const void* k;
@@ -55,6 +56,7 @@ struct VerifyArgs {
 struct CommitArgs {
   TreeDev tree;
   int32_t L, B, H, T, dk, dv, rule, bf16;
+  int32_t Hk;
   const int32_t* accepted;
   const float* S_pre;
   const void* k;
@@ -64,6 +66,13 @@ struct CommitArgs {
   const float* U;
   float* S_new;
 };
+
+// Index of the q/k item (layer, request, key head) that state item (layer, request, head) reads.
+__host__ __device__ inline int tv_qk_item(int item, int H, int Hk) {
+  if (Hk == H) return item;
+  const int lb = item / H, h = item - lb * H;
+  return lb * Hk + h / (H / Hk);
+}
 
 void tv_set_cuda_error(cudaError_t e);
 

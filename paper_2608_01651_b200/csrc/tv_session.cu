@@ -35,7 +35,11 @@ TV_API int tv_session_create(const tv_dims* d, int32_t n_trees, tv_session** out
   const size_t items = (size_t)d->L * d->B * d->H;
   s->eb = d->qkv_dtype == TV_BF16 ? 2 : 4;
   s->nS = items * d->dv * d->dk;
-  s->nQ = items * d->T * d->dk;
+  if (d->Hk < 0 || d->Hk > d->H || (d->Hk > 0 && d->H % d->Hk != 0)) {
+    delete s;
+    return TV_ERR_BAD_ARG;
+  }
+  s->nQ = (size_t)d->L * d->B * (d->Hk ? d->Hk : d->H) * d->T * d->dk;
   s->nV = items * d->T * d->dv;
   s->nG = items * d->T;
   const bool delta = d->rule == TV_GATED_DELTA;

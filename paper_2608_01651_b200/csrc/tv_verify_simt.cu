@@ -84,7 +84,7 @@ struct Smem {
 //   mode 1 (A = K): U_s[i][v] = beta_i (v_i[v] - P_i acc)
 template <bool BF16, int MODE>
 __device__ __forceinline__ void dense_pass(const VerifyArgs& a, const Smem& sm, const void* A,
-                                           size_t node0, float* Og) {
+                                           size_t arow0, size_t node0, float* Og) {
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
   const int T = a.T, dk = a.dk, dv = a.dv;
   float acc[8][8];
@@ -98,7 +98,7 @@ __device__ __forceinline__ void dense_pass(const VerifyArgs& a, const Smem& sm, 
     for (int idx = tid; idx < TV_MAX_NODES * kKC; idx += kThreads) {
       const int i = idx >> 5, kk = idx & 31;
       float x = 0.f;
-      if (i < T && k0 + kk < dk) x = load_elem<BF16>(A, (node0 + i) * dk + k0 + kk);
+      if (i < T && k0 + kk < dk) x = load_elem<BF16>(A, (arow0 + i) * dk + k0 + kk);
       sm.A_s[i * kALD + kk] = x;
     }
     __syncthreads();
@@ -162,6 +162,7 @@ __global__ void __launch_bounds__(kThreads) verify_simt_kernel(VerifyArgs a) {
   const int tb = a.tree.n_trees == 1 ? 0 : b;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const size_t node0 = (size_t)item * T;
+  const size_t qk0 = (size_t)tv_qk_item(item, a.H, a.Hk) * T;  // first q/k row (grouped key heads)
   const float* Sg = a.S_pre + (size_t)item * dv * dk;
   float* Og = a.O + node0 * dv;
 
@@ -194,8 +195,8 @@ __global__ void __launch_bounds__(kThreads) verify_simt_kernel(VerifyArgs a) {
   __syncthreads();
 
   // 3. dense part
-  dense_pass<BF16, 0>(a, sm, a.q, node0, Og);
-  if (DELTA) dense_pass<BF16, 1>(a, sm, a.k, node0, Og);
+  dense_pass<BF16, 0>(a, sm, a.q, qk0, node0, Og);
+  if (DELTA) dense_pass<BF16, 1>(a, sm, a.k, qk0, node0, Og);
   __syncthreads();
 
   const int nk = dk >> 2;  // lanes holding 4 consecutive k elements
@@ -207,13 +208,13 @@ __global__ void __launch_bounds__(kThreads) verify_simt_kernel(VerifyArgs a) {
       for (int i = warp; i < T; i += kWarps) {
         if (sm.depth_s[i] != lev) continue;
         float4 ki = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (lane < nk) ki = load4<BF16>(a.k, (node0 + i) * dk + lane * 4);
+        if (lane < nk) ki = load4<BF16>(a.k, (qk0 + i) * dk + lane * 4);
         float acc[4] = {0.f, 0.f, 0.f, 0.f};
         uint64_t m0 = sm.anc_s[2 * i], m1 = sm.anc_s[2 * i + 1];
         float w = sm.alpha_s[i];  // P_i / P_parent(i)
         for (int j = pop_highest(m0, m1); j >= 0; j = pop_highest(m0, m1)) {
           float4 kj = make_float4(0.f, 0.f, 0.f, 0.f);
-          if (lane < nk) kj = load4<BF16>(a.k, (node0 + j) * dk + lane * 4);
+          if (lane < nk) kj = load4<BF16>(a.k, (qk0 + j) * dk + lane * 4);
           const float dot = warp_sum(ki.x * kj.x + ki.y * kj.y + ki.z * kj.z + ki.w * kj.w);
           const float g = w * dot;
 #pragma unroll
@@ -237,14 +238,14 @@ __global__ void __launch_bounds__(kThreads) verify_simt_kernel(VerifyArgs a) {
   // 5. sparse readout: O_i += sum_j C_ij u_j
   for (int i = warp; i < T; i += kWarps) {
     float4 qi = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (lane < nk) qi = load4<BF16>(a.q, (node0 + i) * dk + lane * 4);
+    if (lane < nk) qi = load4<BF16>(a.q, (qk0 + i) * dk + lane * 4);
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
     uint64_t m0 = sm.anc_s[2 * i], m1 = sm.anc_s[2 * i + 1];
     float w = 1.f;
     int j = i;
     while (j >= 0) {
       float4 kj = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (lane < nk) kj = load4<BF16>(a.k, (node0 + j) * dk + lane * 4);
+      if (lane < nk) kj = load4<BF16>(a.k, (qk0 + j) * dk + lane * 4);
       const float dot = warp_sum(qi.x * kj.x + qi.y * kj.y + qi.z * kj.z + qi.w * kj.w);
       const float c = w * dot;
 #pragma unroll

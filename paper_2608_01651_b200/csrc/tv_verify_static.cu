@@ -100,6 +100,7 @@ int tv_tree_verify_static(const int32_t* parent, int32_t n_trees, const tv_dims*
   if (d->impl != TV_IMPL_AUTO && d->impl != TV_IMPL_SIMT && d->impl != TV_IMPL_TC) return TV_ERR_BAD_ARG;
   if (d->rule == TV_GATED_DELTA && !beta) return TV_ERR_BAD_ARG;
   if (n_trees != 1 && n_trees != d->B) return TV_ERR_BAD_ARG;
+  if (d->Hk < 0 || d->Hk > d->H || (d->Hk > 0 && d->H % d->Hk != 0)) return TV_ERR_BAD_ARG;
   // beyond the fixed scratch: refuse, never spill into an allocation
   if (n_trees > kMaxTrees) return TV_ERR_TOO_LARGE;
   if (d->T > TV_MAX_NODES || d->dk > TV_MAX_DIM || d->dv > TV_MAX_DIM) return TV_ERR_UNSUPPORTED;
@@ -136,7 +137,7 @@ int tv_tree_verify_static(const int32_t* parent, int32_t n_trees, const tv_dims*
   a.tree.n_trees = n_trees;
   a.tree.max_depth_all = TV_MAX_NODES - 1;   // not known on the host
   a.L = d->L; a.B = d->B; a.H = d->H; a.T = d->T; a.dk = d->dk; a.dv = d->dv;
-  a.rule = d->rule; a.bf16 = d->qkv_dtype == TV_BF16;
+  a.rule = d->rule; a.bf16 = d->qkv_dtype == TV_BF16; a.Hk = d->Hk ? d->Hk : d->H;
   a.S_pre = S_pre; a.q = q; a.k = k; a.v = v; a.alpha = alpha; a.beta = beta; a.O = O; a.U = U;
   const bool tc_gated = tv_verify_tc_supports(a);
   if (d->impl == TV_IMPL_TC && !tc_gated) return TV_ERR_UNSUPPORTED;

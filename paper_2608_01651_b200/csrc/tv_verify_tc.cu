@@ -94,6 +94,7 @@ __device__ long long* g_tc_prof = nullptr;   // [CTA 0 only][item][32] clock64 s
 struct TcParams {
   TreeDev tree;
   int32_t n_items, B, H, T;
+  int32_t Hk;  // q/k heads (grouped key heads); H when not grouped
   const float* alpha;
   float* O;
   int32_t* status;
@@ -155,10 +156,11 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         if (!mbar_wait(bar(QK_FREE), ph ^ 1, abort_flag)) break;
         TC_STAMP(it, 0);
         mbar_expect_tx(bar(QK_FULL), 4 * kTile);
-        tma_load_3d(sbase + kOffQ, &tmQ, bar(QK_FULL), 0, 0, item);
-        tma_load_3d(sbase + kOffQ + kTile, &tmQ, bar(QK_FULL), 64, 0, item);
-        tma_load_3d(sbase + kOffK, &tmK, bar(QK_FULL), 0, 0, item);
-        tma_load_3d(sbase + kOffK + kTile, &tmK, bar(QK_FULL), 64, 0, item);
+        const int qk = tv_qk_item(item, p.H, p.Hk);
+        tma_load_3d(sbase + kOffQ, &tmQ, bar(QK_FULL), 0, 0, qk);
+        tma_load_3d(sbase + kOffQ + kTile, &tmQ, bar(QK_FULL), 64, 0, qk);
+        tma_load_3d(sbase + kOffK, &tmK, bar(QK_FULL), 0, 0, qk);
+        tma_load_3d(sbase + kOffK + kTile, &tmK, bar(QK_FULL), 64, 0, qk);
         pend_qk = 1 + (int)ph;
         if (!mbar_wait(bar(S_FREE), ph ^ 1, abort_flag)) break;
         TC_STAMP(it, 1);
@@ -541,9 +543,10 @@ int tv_launch_verify_tc(const VerifyArgs& a, int32_t* status, cudaStream_t strea
   const uint64_t items = (uint64_t)a.L * a.B * a.H;
   const uint32_t orows = a.T <= 64 ? 64 : 128;   // rows of one staged output chunk
   const void* const ptrs[5] = {a.q, a.k, a.v, a.S_pre, a.O};
-  const MapSet* ms = cached_maps(ptrs, items, a.T, 0, [&](CUtensorMap* m) {
-    return make_map(&m[0], a.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, items, a.T, 128, 64) &&
-           make_map(&m[1], a.k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, items, a.T, 128, 64) &&
+  const uint64_t qk_items = (uint64_t)a.L * a.B * a.Hk;
+  const MapSet* ms = cached_maps(ptrs, items, a.T, a.Hk << 8, [&](CUtensorMap* m) {
+    return make_map(&m[0], a.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, qk_items, a.T, 128, 64) &&
+           make_map(&m[1], a.k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, qk_items, a.T, 128, 64) &&
            make_map(&m[2], a.v, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, items, a.T, 128, 64) &&
            make_map(&m[3], a.S_pre, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, 128, 128, 32) &&
            make_map(&m[4], a.O, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, a.T, 128, 32, orows);
@@ -562,7 +565,7 @@ int tv_launch_verify_tc(const VerifyArgs& a, int32_t* status, cudaStream_t strea
   TcParams p;
   p.tree = a.tree;
   p.n_items = (int32_t)items;
-  p.B = a.B; p.H = a.H; p.T = a.T;
+  p.B = a.B; p.H = a.H; p.T = a.T; p.Hk = a.Hk;
   p.alpha = a.alpha;
   p.O = a.O;
   p.status = status;

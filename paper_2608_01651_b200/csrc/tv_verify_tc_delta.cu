@@ -80,6 +80,7 @@ __device__ long long* g_tcd_prof = nullptr;
 struct DeltaParams {
   TreeDev tree;
   int32_t n_items, B, H, T;
+  int32_t Hk;  // q/k heads (grouped key heads); H when not grouped
   const float* alpha;
   const float* beta;
   int32_t want_U;
@@ -162,10 +163,11 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         const uint32_t ph = it & 1;
         if (!mbar_wait(bar(QK_FREE), ph ^ 1, abort_flag)) break;
         mbar_expect_tx(bar(QK_FULL), 4 * 8192);
-        tma_load_3d(sbase + kOffQK, &tmQ, bar(QK_FULL), 0, 0, item);
-        tma_load_3d(sbase + kOffQK + kTile, &tmQ, bar(QK_FULL), 64, 0, item);
-        tma_load_3d(sbase + kOffQK + 8192, &tmK, bar(QK_FULL), 0, 0, item);
-        tma_load_3d(sbase + kOffQK + kTile + 8192, &tmK, bar(QK_FULL), 64, 0, item);
+        const int qk = tv_qk_item(item, p.H, p.Hk);
+        tma_load_3d(sbase + kOffQK, &tmQ, bar(QK_FULL), 0, 0, qk);
+        tma_load_3d(sbase + kOffQK + kTile, &tmQ, bar(QK_FULL), 64, 0, qk);
+        tma_load_3d(sbase + kOffQK + 8192, &tmK, bar(QK_FULL), 0, 0, qk);
+        tma_load_3d(sbase + kOffQK + kTile + 8192, &tmK, bar(QK_FULL), 64, 0, qk);
         pend_qk = 1 + (int)ph;
         if (!mbar_wait(bar(S_FREE), ph ^ 1, abort_flag)) break;
         mbar_expect_tx(bar(S_FULL), 4 * kTile);
@@ -491,9 +493,10 @@ int tv_launch_verify_tc_delta(const VerifyArgs& a, int32_t* status, cudaStream_t
   // the U map is only used when U is requested; O stands in otherwise
   float* Uout = a.U ? a.U : a.O;
   const void* const ptrs[5] = {a.q, a.k, a.v, a.S_pre, a.O};
-  const MapSet* ms = cached_maps(ptrs, items, a.T, 1, [&](CUtensorMap* m) {
-    return make_map(&m[0], a.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, items, a.T, 128, 64, 64) &&
-           make_map(&m[1], a.k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, items, a.T, 128, 64, 64) &&
+  const uint64_t qk_items = (uint64_t)a.L * a.B * a.Hk;
+  const MapSet* ms = cached_maps(ptrs, items, a.T, 1 | (a.Hk << 8), [&](CUtensorMap* m) {
+    return make_map(&m[0], a.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, qk_items, a.T, 128, 64, 64) &&
+           make_map(&m[1], a.k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, qk_items, a.T, 128, 64, 64) &&
            make_map(&m[2], a.v, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, items, a.T, 128, 64, 64) &&
            make_map(&m[3], a.S_pre, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, 128, 128, 32, 128) &&
            make_map(&m[4], a.O, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, a.T, 128, 32, 64);
@@ -518,7 +521,7 @@ int tv_launch_verify_tc_delta(const VerifyArgs& a, int32_t* status, cudaStream_t
   DeltaParams p;
   p.tree = a.tree;
   p.n_items = (int32_t)items;
-  p.B = a.B; p.H = a.H; p.T = a.T;
+  p.B = a.B; p.H = a.H; p.T = a.T; p.Hk = a.Hk;
   p.alpha = a.alpha;
   p.beta = a.beta;
   p.want_U = a.U != nullptr;
