@@ -142,6 +142,35 @@ int tv_tree_device_status(tv_tree* tree, void* stream);
 int tv_selftest_wait_timeout(int32_t* status /*dev*/, void* stream);
 int tv_tree_free(tv_tree* tree);
 
+/* ---- packed forest (Section V-B "CUDA Graph-native packed-forest execution":
+ * variable-sized trees packed topologically into one flat-ragged forest of
+ * fixed total capacity, described by request offsets, parent indices and
+ * compact ancestor metadata; only tiles internal to a request are computed) ---
+ *
+ * tv_forest_build: host only.  Request r owns nodes offsets[r] .. offsets[r+1]-1
+ * of the flat forest (offsets host int32 [n_req+1], offsets[0] = 0, between 1
+ * and n_max <= TV_MAX_NODES nodes each, offsets[n_req] <= capacity);
+ * parent_flat (host int32 [offsets[n_req]]) holds each node's parent as an
+ * index LOCAL to its request, -1 <= parent < local index.  The handle is used
+ * with the same calls as a dense one (upload, verify, commit, conv), with
+ * tv_dims.T = n_max and B = n_req, but the node-indexed tensors are packed
+ * planes of `capacity` rows:
+ *     q, k        [L][Hk][capacity][dk]      v, O, U  [L][H][capacity][dv]
+ *     alpha, beta [L][H][capacity]           (row offsets[r] + i = node i of r)
+ * S_pre / S_new keep [L][B][H][dv][dk]; accepted[r] is local to request r.
+ * Rows at and beyond offsets[n_req] are never read or written.  Metadata
+ * (tv_tree_meta, tv_tree_meta_device) stays padded per request: n_max entries
+ * each, padding entries have empty ancestor sets.  tv_tree_path works as for
+ * dense trees.  tv_forest_rebuild: new topology and offsets, same n_req, n_max
+ * and capacity, no allocation (fixed buffers across rounds).
+ * Errors: TV_ERR_BAD_ARG (offsets not increasing from 0, a request with no or
+ * more than n_max nodes), TV_ERR_TOO_LARGE (more nodes than capacity),
+ * TV_ERR_INVALID_TREE.                                                        */
+int tv_forest_build(const int32_t* parent_flat /*host*/, const int32_t* offsets /*host*/,
+                    int32_t n_req, int32_t n_max, int32_t capacity, tv_tree** out);
+int tv_forest_rebuild(tv_tree* forest, const int32_t* parent_flat /*host*/,
+                      const int32_t* offsets /*host*/);
+
 /* ---- verification (Section IV-A Theorem 1, Eq. 2; Eq. 4; Lemma 2 Eq. 5) ----
  *
  * For every layer, request, head and node i:

@@ -60,6 +60,10 @@ def lib() -> ctypes.CDLL:
     L.tv_last_cuda_error.restype = ctypes.c_int
     L.tv_tree_build.argtypes = [vp, i32, i32, p(vp)]
     L.tv_tree_rebuild.argtypes = [vp, vp]
+    L.tv_forest_build.argtypes = [vp, vp, i32, i32, i32, p(vp)]
+    L.tv_forest_rebuild.argtypes = [vp, vp, vp]
+    L.tv_forest_build.restype = ctypes.c_int
+    L.tv_forest_rebuild.restype = ctypes.c_int
     L.tv_tree_meta.argtypes = [vp, vp, vp, vp]
     L.tv_tree_info.argtypes = [vp, p(i32), p(i32), p(i32)]
     L.tv_tree_path.argtypes = [vp, vp, i32, vp, i32, vp]
@@ -107,6 +111,18 @@ class Tree:
         self._h = handle
         self.n_trees = n_trees
         self.n = n
+        self.offsets = None     # packed forest (forest_build): int32 [n_trees + 1]
+        self.capacity = None    # packed forest: rows of one (layer, head) plane
+
+    def rebuild_forest(self, parents):
+        """``tv_forest_rebuild``: new per-request parent arrays (lengths may change)."""
+        parts = [_np_i32(p).reshape(-1) for p in parents]
+        offsets = np.zeros(len(parts) + 1, dtype=np.int32)
+        offsets[1:] = np.cumsum([len(p) for p in parts])
+        flat = np.ascontiguousarray(np.concatenate(parts), dtype=np.int32)
+        _check(lib().tv_forest_rebuild(self._h, flat.ctypes.data, offsets.ctypes.data), "tv_forest_rebuild")
+        self.offsets = offsets
+        return self
 
     def rebuild(self, parent):
         par = _np_i32(parent).reshape(self.n_trees, self.n)
@@ -196,6 +212,24 @@ def tree_build(parent) -> Tree:
     return Tree(h, n_trees, n)
 
 
+def forest_build(parents, n_max=None, capacity=None) -> Tree:
+    """``tv_forest_build``: ``parents`` is a list of per-request parent arrays (local indices) of
+    different lengths; they are packed in order.  Returns a ``Tree`` with ``offsets`` (int32
+    [B+1]) and ``capacity``; node-indexed tensors are then [L][H][capacity][d] planes."""
+    parts = [_np_i32(p).reshape(-1) for p in parents]
+    offsets = np.zeros(len(parts) + 1, dtype=np.int32)
+    offsets[1:] = np.cumsum([len(p) for p in parts])
+    flat = np.ascontiguousarray(np.concatenate(parts), dtype=np.int32)
+    n_max = int(max(len(p) for p in parts)) if n_max is None else int(n_max)
+    capacity = int(offsets[-1]) if capacity is None else int(capacity)
+    h = ctypes.c_void_p()
+    _check(lib().tv_forest_build(flat.ctypes.data, offsets.ctypes.data, len(parts), n_max, capacity,
+                                 ctypes.byref(h)), "tv_forest_build")
+    t = Tree(h, len(parts), n_max)
+    t.offsets, t.capacity = offsets, capacity
+    return t
+
+
 def _stream_ptr(stream):
     if stream is None:
         import torch
@@ -211,7 +245,7 @@ def _ptr(t):
     return ctypes.c_void_p(0 if t is None else t.data_ptr())
 
 
-def _dims(S_pre, k, v, rule, impl) -> _Dims:
+def _dims(S_pre, k, v, rule, impl, tree=None) -> _Dims:
     import torch
     if S_pre.dim() == 4:
         L = 1
@@ -227,6 +261,11 @@ def _dims(S_pre, k, v, rule, impl) -> _Dims:
         dt = F32
     else:
         raise ValueError("q/k/v must be float32 or bfloat16")
+    if tree is not None and getattr(tree, "capacity", None) is not None:
+        # packed forest: [L][H][capacity][d] planes; the per-request node limit comes from the handle
+        if T != tree.capacity or k.dim() != S_pre.dim() - 1:
+            raise ValueError("packed-forest tensors must be [L][H][capacity][d] (or [H][capacity][d])")
+        T = tree.n
     Hk = k.shape[-3]
     if H % Hk:
         raise ValueError("the number of state heads must be a multiple of the number of key heads")
@@ -254,7 +293,7 @@ def tree_verify(tree: Tree, S_pre, q, k, v, alpha, beta=None, *, rule=GATED, O=N
         _require(t, n, torch.float32)
     for t, n in ((q, "q"), (k, "k"), (v, "v")):
         _require(t, n, k.dtype)
-    d = _dims(S_pre, k, v, rule, impl)
+    d = _dims(S_pre, k, v, rule, impl, tree)
     if O is None:
         O = torch.empty(*v.shape[:-1], d.dv, device=v.device, dtype=torch.float32)
     if U is None and want_U:
@@ -280,7 +319,7 @@ def commit_path(tree: Tree, accepted, S_pre, k, v, alpha, beta=None, *, rule=GAT
         _require(t, n, torch.float32)
     for t, n in ((k, "k"), (v, "v")):
         _require(t, n, k.dtype)
-    d = _dims(S_pre, k, v, rule, IMPL_AUTO)
+    d = _dims(S_pre, k, v, rule, IMPL_AUTO, tree)
     out = S_pre if S_new is None else S_new
     _check(lib().tv_commit_path(tree._h, ctypes.byref(d), _ptr(accepted), _ptr(S_pre), _ptr(k),
                                 _ptr(v), _ptr(alpha), _ptr(beta), _ptr(U), _ptr(out),
@@ -418,7 +457,7 @@ def prepare_tree_verify(tree: Tree, S_pre, q, k, v, alpha, beta=None, *, rule=GA
         _require(t, n, k.dtype)
     if O is None:
         raise ValueError("O must be preallocated")
-    d = _dims(S_pre, k, v, rule, impl)
+    d = _dims(S_pre, k, v, rule, impl, tree)
     args = (tree._h, ctypes.byref(d), _ptr(S_pre), _ptr(q), _ptr(k), _ptr(v), _ptr(alpha), _ptr(beta),
             _ptr(O), _ptr(U), _stream_ptr(stream))
     return Prepared(lib().tv_tree_verify, "tv_tree_verify", args, (tree, d, S_pre, q, k, v, alpha, beta, O, U))
@@ -433,7 +472,7 @@ def prepare_commit_path(tree: Tree, accepted, S_pre, k, v, alpha, beta=None, *, 
         _require(t, n, torch.float32)
     for t, n in ((k, "k"), (v, "v")):
         _require(t, n, k.dtype)
-    d = _dims(S_pre, k, v, rule, IMPL_AUTO)
+    d = _dims(S_pre, k, v, rule, IMPL_AUTO, tree)
     out = S_pre if S_new is None else S_new
     args = (tree._h, ctypes.byref(d), _ptr(accepted), _ptr(S_pre), _ptr(k), _ptr(v), _ptr(alpha),
             _ptr(beta), _ptr(U), _ptr(out), _stream_ptr(stream))

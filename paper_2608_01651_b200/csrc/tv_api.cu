@@ -99,7 +99,69 @@ TV_API int tv_tree_build(const int32_t* parent, int32_t n_trees, int32_t n, tv_t
 
 TV_API int tv_tree_rebuild(tv_tree* t, const int32_t* parent) {
   if (!t || !parent) return TV_ERR_BAD_ARG;
+  if (!t->offsets.empty()) return TV_ERR_BAD_ARG;   // a packed forest is rebuilt with its offsets
   return fill_tree(t, parent);
+}
+
+// Packed forest: the flat parent array is spread into per-tree slabs of n entries (padding =
+// root children nobody descends from), so all metadata code above and every kernel's mask
+// handling serve both layouts; only the tensor rows are packed.
+static int fill_forest(tv_tree* t, const int32_t* parent_flat, const int32_t* offsets) {
+  const int B = t->n_trees, n = t->n;
+  if (offsets[0] != 0) return TV_ERR_BAD_ARG;
+  for (int b = 0; b < B; ++b) {
+    const int nb = offsets[b + 1] - offsets[b];
+    if (nb < 1 || nb > n) return TV_ERR_BAD_ARG;
+  }
+  if (offsets[B] > t->capacity) return TV_ERR_TOO_LARGE;
+  std::vector<int32_t> padded;
+  try {
+    padded.assign((size_t)B * n, -1);
+  } catch (...) {
+    return TV_ERR_NOMEM;
+  }
+  for (int b = 0; b < B; ++b)
+    std::memcpy(padded.data() + (size_t)b * n, parent_flat + offsets[b],
+                sizeof(int32_t) * (size_t)(offsets[b + 1] - offsets[b]));
+  int st = fill_tree(t, padded.data());
+  if (st != TV_OK) return st;
+  std::memcpy(t->offsets.data(), offsets, sizeof(int32_t) * (size_t)(B + 1));
+  return TV_OK;
+}
+
+TV_API int tv_forest_build(const int32_t* parent_flat, const int32_t* offsets, int32_t n_req, int32_t n_max,
+                           int32_t capacity, tv_tree** out) {
+  if (!out) return TV_ERR_BAD_ARG;
+  *out = nullptr;
+  if (!parent_flat || !offsets || n_req < 1 || n_max < 1 || capacity < 1) return TV_ERR_BAD_ARG;
+  if (n_max > TV_MAX_NODES) return TV_ERR_UNSUPPORTED;
+  tv_tree* t = new (std::nothrow) tv_tree();
+  if (!t) return TV_ERR_NOMEM;
+  t->n_trees = n_req;
+  t->n = n_max;
+  t->capacity = capacity;
+  try {
+    t->parent.resize((size_t)n_req * n_max);
+    t->depth.resize((size_t)n_req * n_max);
+    t->max_depth.resize(n_req);
+    t->anc.resize((size_t)n_req * n_max * 2);
+    t->offsets.resize((size_t)n_req + 1);
+  } catch (...) {
+    delete t;
+    return TV_ERR_NOMEM;
+  }
+  int st = fill_forest(t, parent_flat, offsets);
+  if (st != TV_OK) {
+    delete t;
+    return st;
+  }
+  *out = t;
+  return TV_OK;
+}
+
+TV_API int tv_forest_rebuild(tv_tree* t, const int32_t* parent_flat, const int32_t* offsets) {
+  if (!t || !parent_flat || !offsets || t->offsets.empty()) return TV_ERR_BAD_ARG;
+  return fill_forest(t, parent_flat, offsets);
 }
 
 TV_API int tv_tree_meta(const tv_tree* t, uint64_t* anc, int32_t* depth, int32_t* max_depth) {
@@ -150,9 +212,10 @@ TV_API int tv_tree_upload(tv_tree* t, void* stream) {
   if (!t) return TV_ERR_BAD_ARG;
   const size_t nn = (size_t)t->n_trees * t->n;
   const size_t anc_b = nn * 2 * sizeof(uint64_t), i32_b = nn * sizeof(int32_t);
-  const size_t meta_b = anc_b + 2 * i32_b;
+  const size_t off_b = t->offsets.empty() ? 0 : ((t->offsets.size() * sizeof(int32_t) + 15) & ~(size_t)15);
+  const size_t meta_b = anc_b + 2 * i32_b + off_b;
   const size_t total = ((meta_b + 15) & ~(size_t)15) + 16;  // + status word
-  const size_t slot_b = (i32_b + 255) & ~(size_t)255;       // one staged copy of the parent arrays
+  const size_t slot_b = (i32_b + off_b + 255) & ~(size_t)255;  // one staged copy of parents (+ offsets)
   int dev = 0;
   TV_CUDA_TRY(cudaGetDevice(&dev));
   if (t->d_blob && (t->device != dev || t->blob_bytes != total)) return TV_ERR_BAD_ARG;
@@ -182,6 +245,10 @@ TV_API int tv_tree_upload(tv_tree* t, void* stream) {
     t->d_depth = t->d_depth_w;
     t->d_parent = t->d_parent_w;
     t->d_status = (int32_t*)(base + total - 16);
+    if (off_b) {
+      t->d_offsets_w = (int32_t*)(base + anc_b + 2 * i32_b);
+      t->d_offsets = t->d_offsets_w;
+    }
   }
   cudaStream_t s = (cudaStream_t)stream;
   // The parent arrays go into one of two pinned slots; a small kernel reads the slot over the
@@ -191,8 +258,14 @@ TV_API int tv_tree_upload(tv_tree* t, void* stream) {
   t->stage_slot ^= 1;
   TV_CUDA_TRY(cudaEventSynchronize(t->staged[slot]));
   std::memcpy((char*)t->h_stage + slot * slot_b, t->parent.data(), i32_b);
+  const int32_t* off_mapped = nullptr;
+  if (off_b) {
+    std::memcpy((char*)t->h_stage + slot * slot_b + i32_b, t->offsets.data(), t->offsets.size() * sizeof(int32_t));
+    off_mapped = (const int32_t*)((const char*)t->h_stage_dev + slot * slot_b + i32_b);
+  }
   int st = tv_launch_tree_meta((const int32_t*)((const char*)t->h_stage_dev + slot * slot_b), t->n_trees,
-                               t->n, t->d_anc_w, t->d_depth_w, t->d_parent_w, t->d_status, s);
+                               t->n, t->d_anc_w, t->d_depth_w, t->d_parent_w, t->d_status, off_mapped,
+                               t->d_offsets_w, s);
   if (st != TV_OK) return st;
   TV_CUDA_TRY(cudaEventRecord(t->staged[slot], s));
   t->uploaded = true;
@@ -244,6 +317,7 @@ static int check_common(const tv_tree* t, const tv_dims* d) {
   if (d->qkv_dtype == TV_BF16 && ((d->dk & 7) || (d->dv & 7))) return TV_ERR_UNSUPPORTED;
   if (t->n != d->T) return TV_ERR_BAD_ARG;
   if (t->n_trees != 1 && t->n_trees != d->B) return TV_ERR_BAD_ARG;
+  if (!t->offsets.empty() && t->n_trees != d->B) return TV_ERR_BAD_ARG;   // a packed forest has one tree per request
   if (d->Hk < 0 || d->Hk > d->H || (d->Hk > 0 && d->H % d->Hk != 0)) return TV_ERR_BAD_ARG;
   if ((int64_t)d->L * d->B * d->H > 0x7fffffffLL) return TV_ERR_UNSUPPORTED;
   if (!t->uploaded) return TV_ERR_NOT_UPLOADED;
@@ -257,6 +331,8 @@ static TreeDev tree_dev(const tv_tree* t) {
   td.parent = t->d_parent;
   td.n_trees = t->n_trees;
   td.max_depth_all = t->max_depth_all;
+  td.offsets = t->d_offsets;
+  td.capacity = t->capacity;
   return td;
 }
 

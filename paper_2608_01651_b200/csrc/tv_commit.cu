@@ -29,10 +29,10 @@ __device__ __forceinline__ float load_elem(const void* base, size_t idx) {
 // Fills path_s[0..len) (topological order), w_s[p] = P_a / P_path[p] and *Pa_s.
 // al_s is scratch for the T decay gates (loaded by T threads in parallel so that
 // the serial suffix product below never waits on global memory).
-__device__ __forceinline__ int build_path(const TreeDev& tree, int tb, int T, int acc,
+__device__ __forceinline__ int build_path(const TreeDev& tree, size_t meta0, int T, int acc,
                                           const float* alpha_row, int* path_s, float* w_s,
                                           float* al_s, float* Pa_s) {
-  const uint64_t* m = tree.anc + ((size_t)tb * T + acc) * 2;
+  const uint64_t* m = tree.anc + (meta0 + acc) * 2;
   const int t = threadIdx.x;
   if (t < T) al_s[t] = alpha_row[t];
   uint64_t m0 = m[0], m1 = m[1];
@@ -85,7 +85,9 @@ __global__ void __launch_bounds__(kThreads) commit_factored_kernel(CommitArgs a)
   const int item = blockIdx.x;
   const int b = (item / a.H) % a.B;
   const int tid = threadIdx.x;
-  const int dk = a.dk, dv = a.dv, T = a.T;
+  const int dk = a.dk, dv = a.dv;
+  const ItemRows rows = tv_item_rows(a.tree, item, a.B, a.H, a.Hk, a.T);
+  const int T = rows.n;
   const int n4 = dv * dk / 4;
   const size_t sbase = (size_t)item * dv * dk;
   const float4* src = reinterpret_cast<const float4*>(a.S_pre + sbase);
@@ -105,10 +107,9 @@ __global__ void __launch_bounds__(kThreads) commit_factored_kernel(CommitArgs a)
     const int i = tid + e * kThreads;
     if (i < n4) s[e] = ld_stream(src + i);
   }
-  const int tb = a.tree.n_trees == 1 ? 0 : b;
-  const size_t node0 = (size_t)item * T;  // first node row of this (l, b, h)
-  const size_t qk0 = (size_t)tv_qk_item(item, a.H, a.Hk) * T;  // first key row (grouped key heads)
-  const int len = build_path(a.tree, tb, T, acc, a.alpha + node0, path_s, w_s, al_s, &Pa_s);
+  const size_t node0 = rows.node0;  // first node row of this (l, b, h)
+  const size_t qk0 = rows.qk0;      // first key row (grouped key heads)
+  const int len = build_path(a.tree, rows.meta0, T, acc, a.alpha + node0, path_s, w_s, al_s, &Pa_s);
   const float Pa = Pa_s;
 #pragma unroll
   for (int e = 0; e < kMaxVec; ++e) {
@@ -170,9 +171,11 @@ __global__ void __launch_bounds__(kRowThreads) commit_factored_dk128_kernel(Comm
   __shared__ __align__(16) float k_s[kPathChunk][128];
   __shared__ __align__(16) float cu_s[kPathChunk][kRowsPerCta];
 
-  const int dv = a.dv, T = a.T;
+  const int dv = a.dv;
   const int n_half = (dv + kRowsPerCta - 1) / kRowsPerCta;
   const int item = blockIdx.x / n_half, half = blockIdx.x - item * n_half;
+  const ItemRows rows = tv_item_rows(a.tree, item, a.B, a.H, a.Hk, a.T);
+  const int T = rows.n;
   const int b = (item / a.H) % a.B;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int row0 = half * kRowsPerCta + warp * 16;
@@ -193,10 +196,9 @@ __global__ void __launch_bounds__(kRowThreads) commit_factored_dk128_kernel(Comm
       if (row0 + e < dv) st_stream(dst + e * 32, s[e]);
     return;
   }
-  const int tb = a.tree.n_trees == 1 ? 0 : b;
-  const size_t node0 = (size_t)item * T;
-  const size_t qk0 = (size_t)tv_qk_item(item, a.H, a.Hk) * T;
-  const int len = build_path(a.tree, tb, T, acc, a.alpha + node0, path_s, w_s, al_s, &Pa_s);
+  const size_t node0 = rows.node0;
+  const size_t qk0 = rows.qk0;
+  const int len = build_path(a.tree, rows.meta0, T, acc, a.alpha + node0, path_s, w_s, al_s, &Pa_s);
   const float Pa = Pa_s;
   bool scaled = false;
   for (int c0 = 0; c0 < len; c0 += kPathChunk) {
@@ -288,7 +290,8 @@ __global__ void __launch_bounds__(kRowThreads, TV_STREAM_CTAS) commit_stream_dk1
 
   for (int b = tid; b < a.B; b += kRowThreads) {
     int acc = a.accepted[b];
-    if (acc >= T) acc = -1;
+    const int nb = a.tree.offsets ? a.tree.offsets[b + 1] - a.tree.offsets[b] : T;
+    if (acc >= nb) acc = -1;
     acc_s[b] = acc;
     uint64_t m0 = 0, m1 = 0;
     if (acc >= 0) {
@@ -323,7 +326,7 @@ __global__ void __launch_bounds__(kRowThreads, TV_STREAM_CTAS) commit_stream_dk1
       const int r = lane < c0 ? lane : lane - c0;
       for (int i = 0; i < r; ++i) w &= w - 1;
       node = __ffsll((long long)w) - 1 + (lane < c0 ? 0 : 64);
-      al = a.alpha[(size_t)(u / n_half) * T + node];
+      al = a.alpha[tv_item_rows(a.tree, u / n_half, a.B, a.H, a.Hk, T).node0 + node];
     }
     float incl = al;   // product of alpha over path positions >= lane
 #pragma unroll
@@ -348,8 +351,8 @@ __global__ void __launch_bounds__(kRowThreads, TV_STREAM_CTAS) commit_stream_dk1
   float ureg[8];
   auto fetch_rows = [&](int u, int nb) {
     const int item = u / n_half, half = u - item * n_half;
-    const size_t node0 = (size_t)item * T;
-    const size_t qk0 = (size_t)tv_qk_item(item, a.H, a.Hk) * T;
+    const ItemRows rows = tv_item_rows(a.tree, item, a.B, a.H, a.Hk, T);
+    const size_t node0 = rows.node0, qk0 = rows.qk0;
     const int len = len_s[nb];
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
@@ -479,7 +482,9 @@ __global__ void __launch_bounds__(kThreads) commit_delta_rows_kernel(CommitArgs 
   const int item = blockIdx.x;
   const int b = (item / a.H) % a.B;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int dv = a.dv, T = a.T;
+  const int dv = a.dv;
+  const ItemRows rows = tv_item_rows(a.tree, item, a.B, a.H, a.Hk, a.T);
+  const int T = rows.n;
   const size_t sbase = (size_t)item * dv * DK;
   const int n4 = dv * DK / 4;
 
@@ -493,10 +498,9 @@ __global__ void __launch_bounds__(kThreads) commit_delta_rows_kernel(CommitArgs 
     }
     return;
   }
-  const int tb = a.tree.n_trees == 1 ? 0 : b;
-  const size_t node0 = (size_t)item * T;
-  const size_t qk0 = (size_t)tv_qk_item(item, a.H, a.Hk) * T;
-  const int len = build_path(a.tree, tb, T, acc, a.alpha + node0, path_s, w_s, al_s, &Pa_s);
+  const size_t node0 = rows.node0;
+  const size_t qk0 = rows.qk0;
+  const int len = build_path(a.tree, rows.meta0, T, acc, a.alpha + node0, path_s, w_s, al_s, &Pa_s);
 
   float s[kRowsPerWarp][NPL];
 #pragma unroll

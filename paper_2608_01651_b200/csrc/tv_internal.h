@@ -25,6 +25,13 @@ struct tv_tree {
   int32_t* d_parent_w = nullptr;
   int32_t* d_status = nullptr;  // device status word (0 = ok), cleared by every upload
   bool uploaded = false;
+  // Packed forest (tv_forest_build): tree t has offsets[t+1] - offsets[t] <= n real nodes (its
+  // metadata slab is padded to n with root children) and its tensor rows start at offsets[t] in
+  // every (layer, head) plane of `capacity` rows.  Empty for a dense tree set.
+  std::vector<int32_t> offsets;
+  int32_t capacity = 0;
+  const int32_t* d_offsets = nullptr;
+  int32_t* d_offsets_w = nullptr;
   cudaEvent_t staged[2] = {nullptr, nullptr};  // the device has read staging slot 0 / 1
   const int32_t* h_stage_dev = nullptr;          // device view of the pinned staging block
   int stage_slot = 0;
@@ -37,6 +44,8 @@ struct TreeDev {
   const int32_t* parent;  // [n_trees][T]
   int32_t n_trees;
   int32_t max_depth_all;
+  const int32_t* offsets;  // packed forest: [n_trees + 1] first tensor row of each tree; else null
+  int32_t capacity;        // packed forest: rows of one (layer, head) plane
 };
 
 struct VerifyArgs {
@@ -74,13 +83,43 @@ __host__ __device__ inline int tv_qk_item(int item, int H, int Hk) {
   return lb * Hk + h / (H / Hk);
 }
 
+// Where the rows of work item (layer l, request b, head h) live.  Dense layout: every item owns a
+// slab of T rows.  Packed forest: request b owns rows [offsets[b], offsets[b+1]) of every
+// (layer, head) plane of `capacity` rows; its metadata slab is still T entries wide.
+struct ItemRows {
+  size_t node0;   // first row in v / alpha / beta / O / U
+  size_t qk0;     // first row in q / k
+  size_t meta0;   // first entry in the metadata arrays
+  int n;          // real nodes of this item
+};
+__device__ inline ItemRows tv_item_rows(const TreeDev& t, int item, int B, int H, int Hk, int T) {
+  ItemRows r;
+  const int lb = item / H, h = item - lb * H;
+  const int l = lb / B, b = lb - l * B;
+  const int hk = Hk == H ? h : h / (H / Hk);
+  if (t.offsets == nullptr) {
+    r.node0 = (size_t)item * T;
+    r.qk0 = (size_t)(lb * Hk + hk) * T;
+    r.meta0 = (size_t)(t.n_trees == 1 ? 0 : b) * T;
+    r.n = T;
+  } else {
+    const int off = t.offsets[b];
+    r.n = t.offsets[b + 1] - off;
+    r.node0 = (size_t)(l * H + h) * t.capacity + off;
+    r.qk0 = (size_t)(l * Hk + hk) * t.capacity + off;
+    r.meta0 = (size_t)b * T;
+  }
+  return r;
+}
+
 void tv_set_cuda_error(cudaError_t e);
 
 // Launchers (each returns a tv_status; all work is asynchronous on `stream`).
 int tv_launch_verify_simt(const VerifyArgs& a, cudaStream_t stream);
 int tv_launch_commit(const CommitArgs& a, cudaStream_t stream);
 int tv_launch_tree_meta(const int32_t* parent_mapped, int32_t n_trees, int32_t n, uint64_t* anc,
-                        int32_t* depth, int32_t* parent_dev, int32_t* status, cudaStream_t stream);
+                        int32_t* depth, int32_t* parent_dev, int32_t* status, const int32_t* offsets_mapped,
+                        int32_t* offsets_dev, cudaStream_t stream);
 bool tv_verify_tc_supports(const VerifyArgs& a);
 int tv_launch_verify_tc(const VerifyArgs& a, int32_t* status, cudaStream_t stream);
 bool tv_verify_tc_delta_supports(const VerifyArgs& a);

@@ -8,7 +8,8 @@ namespace {
 
 __global__ void __launch_bounds__(TV_MAX_NODES)
 tree_meta_kernel(const int32_t* __restrict__ parent, int32_t n, uint64_t* __restrict__ anc,
-                 int32_t* __restrict__ depth, int32_t* __restrict__ parent_dev, int32_t* status) {
+                 int32_t* __restrict__ depth, int32_t* __restrict__ parent_dev, int32_t* status,
+                 const int32_t* __restrict__ offsets, int32_t* __restrict__ offsets_dev) {
   __shared__ int32_t par_s[TV_MAX_NODES];
   const int t = blockIdx.x, i = threadIdx.x;
   // a verify kernel launched behind this one may be scheduled now and set itself up; it waits
@@ -16,6 +17,12 @@ tree_meta_kernel(const int32_t* __restrict__ parent, int32_t n, uint64_t* __rest
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (i < n) par_s[i] = parent[(size_t)t * n + i];
   if (t == 0 && i == 0) *status = 0;
+  // packed forest: the row offsets travel with the parents (tree t copies entry t, the last
+  // tree also the end marker)
+  if (offsets != nullptr && i == 0) {
+    offsets_dev[t] = offsets[t];
+    if (t == (int)gridDim.x - 1) offsets_dev[t + 1] = offsets[t + 1];
+  }
   __syncthreads();
   if (i >= n) return;
   uint64_t w0 = 0, w1 = 0;
@@ -35,8 +42,10 @@ tree_meta_kernel(const int32_t* __restrict__ parent, int32_t n, uint64_t* __rest
 }  // namespace
 
 int tv_launch_tree_meta(const int32_t* parent_mapped, int32_t n_trees, int32_t n, uint64_t* anc,
-                        int32_t* depth, int32_t* parent_dev, int32_t* status, cudaStream_t stream) {
-  tree_meta_kernel<<<n_trees, TV_MAX_NODES, 0, stream>>>(parent_mapped, n, anc, depth, parent_dev, status);
+                        int32_t* depth, int32_t* parent_dev, int32_t* status, const int32_t* offsets_mapped,
+                        int32_t* offsets_dev, cudaStream_t stream) {
+  tree_meta_kernel<<<n_trees, TV_MAX_NODES, 0, stream>>>(parent_mapped, n, anc, depth, parent_dev, status,
+                                                        offsets_mapped, offsets_dev);
   TV_CUDA_TRY(cudaGetLastError());
   return TV_OK;
 }

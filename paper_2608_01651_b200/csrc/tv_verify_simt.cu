@@ -84,9 +84,9 @@ struct Smem {
 //   mode 1 (A = K): U_s[i][v] = beta_i (v_i[v] - P_i acc)
 template <bool BF16, int MODE>
 __device__ __forceinline__ void dense_pass(const VerifyArgs& a, const Smem& sm, const void* A,
-                                           size_t arow0, size_t node0, float* Og) {
+                                           size_t arow0, size_t node0, int T, float* Og) {
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
-  const int T = a.T, dk = a.dk, dv = a.dv;
+  const int dk = a.dk, dv = a.dv;
   float acc[8][8];
 #pragma unroll
   for (int m = 0; m < 8; ++m)
@@ -143,7 +143,10 @@ __device__ __forceinline__ void dense_pass(const VerifyArgs& a, const Smem& sm, 
 template <bool BF16, bool DELTA>
 __global__ void __launch_bounds__(kThreads) verify_simt_kernel(VerifyArgs a) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  const int T = a.T, dk = a.dk, dv = a.dv;
+  const int dk = a.dk, dv = a.dv;
+  const int item = blockIdx.x;
+  const ItemRows rows = tv_item_rows(a.tree, item, a.B, a.H, a.Hk, a.T);
+  const int T = rows.n;   // real nodes of this item (the whole slab unless the forest is packed)
   Smem sm;
   {
     unsigned char* p = smem_raw;
@@ -157,23 +160,20 @@ __global__ void __launch_bounds__(kThreads) verify_simt_kernel(VerifyArgs a) {
     sm.depth_s = reinterpret_cast<int*>(p);  p += sizeof(int) * TV_MAX_NODES;
     sm.U_s = reinterpret_cast<float*>(p);  // only with DELTA
   }
-  const int item = blockIdx.x;
-  const int b = (item / a.H) % a.B;
-  const int tb = a.tree.n_trees == 1 ? 0 : b;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const size_t node0 = (size_t)item * T;
-  const size_t qk0 = (size_t)tv_qk_item(item, a.H, a.Hk) * T;  // first q/k row (grouped key heads)
+  const size_t node0 = rows.node0;
+  const size_t qk0 = rows.qk0;   // first q/k row (grouped key heads)
   const float* Sg = a.S_pre + (size_t)item * dv * dk;
   float* Og = a.O + node0 * dv;
 
   // 1. metadata and path decay P_i
   if (tid < T) {
-    const uint64_t* m = a.tree.anc + ((size_t)tb * T + tid) * 2;
+    const uint64_t* m = a.tree.anc + (rows.meta0 + tid) * 2;
     sm.anc_s[2 * tid] = m[0];
     sm.anc_s[2 * tid + 1] = m[1];
     sm.alpha_s[tid] = a.alpha[node0 + tid];
     sm.beta_s[tid] = DELTA ? a.beta[node0 + tid] : 0.f;
-    sm.depth_s[tid] = a.tree.depth[(size_t)tb * T + tid];
+    sm.depth_s[tid] = a.tree.depth[rows.meta0 + tid];
   }
   __syncthreads();
   if (tid < T) {
@@ -195,8 +195,8 @@ __global__ void __launch_bounds__(kThreads) verify_simt_kernel(VerifyArgs a) {
   __syncthreads();
 
   // 3. dense part
-  dense_pass<BF16, 0>(a, sm, a.q, qk0, node0, Og);
-  if (DELTA) dense_pass<BF16, 1>(a, sm, a.k, qk0, node0, Og);
+  dense_pass<BF16, 0>(a, sm, a.q, qk0, node0, T, Og);
+  if (DELTA) dense_pass<BF16, 1>(a, sm, a.k, qk0, node0, T, Og);
   __syncthreads();
 
   const int nk = dk >> 2;  // lanes holding 4 consecutive k elements

@@ -136,6 +136,8 @@ int tv_tree_verify_static(const int32_t* parent, int32_t n_trees, const tv_dims*
   a.tree.parent = par_dev;
   a.tree.n_trees = n_trees;
   a.tree.max_depth_all = TV_MAX_NODES - 1;   // not known on the host
+  a.tree.offsets = nullptr;
+  a.tree.capacity = 0;
   a.L = d->L; a.B = d->B; a.H = d->H; a.T = d->T; a.dk = d->dk; a.dv = d->dv;
   a.rule = d->rule; a.bf16 = d->qkv_dtype == TV_BF16; a.Hk = d->Hk ? d->Hk : d->H;
   a.S_pre = S_pre; a.q = q; a.k = k; a.v = v; a.alpha = alpha; a.beta = beta; a.O = O; a.U = U;

@@ -535,6 +535,7 @@ extern "C" __attribute__((visibility("default"))) int tv_selftest_wait_timeout(i
 }
 
 bool tv_verify_tc_supports(const VerifyArgs& a) {
+  if (a.tree.offsets != nullptr) return false;   // packed forests take the general kernel
   return a.bf16 && a.dk == 128 && a.dv == 128 && a.rule == TV_GATED && a.T <= 128;
 }
 

@@ -483,6 +483,7 @@ extern "C" __attribute__((visibility("default"))) int tv_debug_set_tcd_profile(l
 #endif
 
 bool tv_verify_tc_delta_supports(const VerifyArgs& a) {
+  if (a.tree.offsets != nullptr) return false;   // packed forests take the general kernel
   return a.bf16 && a.dk == 128 && a.dv == 128 && a.rule == TV_GATED_DELTA && a.T <= kRows &&
          a.tree.max_depth_all < kSlots;
 }

@@ -1,0 +1,152 @@
+"""Packed forest (Section V-B): requests with different node counts share flat tensors; every
+request is checked against the oracle run on its own tree, and against the dense call on the
+same request."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2608_01651_b200 as tv
+from paper_2608_01651_b200 import inputs
+from oracle import tree_oracle as orc
+from tests.parity_util import rel_l2_rows, rel_fro
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def make_forest(B, n_max, seed, kind="frontier"):
+    """Per-request trees of 1..n_max nodes (the first has n_max, the second one node)."""
+    rng = np.random.Generator(np.random.Philox(key=seed))
+    sizes = [n_max, 1] + [int(rng.integers(1, n_max + 1)) for _ in range(max(0, B - 2))]
+    sizes = sizes[:B]
+    parents = []
+    for n in sizes:
+        if kind == "chain":
+            parents.append(inputs.tree_chain(n))
+        else:
+            parents.append(inputs.tree_frontier(n, rng) if n > 1 else np.array([-1], dtype=np.int32))
+    accepted = np.array([inputs.accepted_walk(p, rng) for p in parents], dtype=np.int32)
+    accepted[-1] = -1
+    return parents, accepted
+
+
+def packed_tensors(wl, parents, capacity, Hk, L=1):
+    """Draw dense per-request tensors with the workload's generator, then pack the real rows."""
+    B, H = wl.B, wl.H
+    G = H // Hk
+    dt = wl.torch_dtype
+    off = np.concatenate([[0], np.cumsum([len(p) for p in parents])]).astype(np.int64)
+    layers = [inputs.make_tensors(wl, layer=l) for l in range(L)]
+    fill = lambda *shape: torch.full(shape, 3.0)   # rows past the forest must stay untouched/unread
+    P = {"q": fill(L, Hk, capacity, wl.dk).to(dt), "k": fill(L, Hk, capacity, wl.dk).to(dt),
+         "v": fill(L, H, capacity, wl.dv).to(dt), "alpha": fill(L, H, capacity),
+         "beta": fill(L, H, capacity) if layers[0]["beta"] is not None else None,
+         "S_pre": torch.stack([x["S_pre"] for x in layers])}
+    for l, t in enumerate(layers):
+        for b, par in enumerate(parents):
+            n = len(par)
+            rows = slice(int(off[b]), int(off[b]) + n)
+            P["q"][l, :, rows] = t["q"][b, ::G, :n]
+            P["k"][l, :, rows] = t["k"][b, ::G, :n]
+            P["v"][l, :, rows] = t["v"][b, :, :n]
+            P["alpha"][l, :, rows] = t["alpha"][b, :, :n]
+            if P["beta"] is not None:
+                P["beta"][l, :, rows] = t["beta"][b, :, :n]
+    return P, off
+
+
+def oracle_request(wl, P, off, parents, accepted, l, b, h, Hk):
+    G = wl.H // Hk
+    n = len(parents[b])
+    rows = slice(int(off[b]), int(off[b]) + n)
+    f = lambda t: inputs.to_f64(t)
+    S = f(P["S_pre"][l, b, h]).T            # paper orientation [dk][dv]
+    q, k, v = f(P["q"][l, h // G, rows]), f(P["k"][l, h // G, rows]), f(P["v"][l, h, rows])
+    al = f(P["alpha"][l, h, rows])
+    be = None if P["beta"] is None else f(P["beta"][l, h, rows])
+    O, U, _ = orc.verify_memo(S, q, k, v, al, be, parents[b], wl.rule_name)
+    Sn = orc.commit_walk(S, k, v, al, be, parents[b], int(accepted[b]), wl.rule_name)
+    return O, U, Sn.T
+
+
+CASES = [  # B, H, Hk, n_max, dk, dv, L
+    (5, 4, 4, 64, 128, 128, 1),
+    (4, 4, 2, 128, 128, 128, 2),
+    (6, 2, 1, 33, 64, 128, 1),
+    (3, 2, 2, 17, 64, 64, 1),
+]
+
+
+@pytest.mark.parametrize("rule", [inputs.GATED, inputs.DELTA])
+@pytest.mark.parametrize("dtype", [inputs.BF16, inputs.F32])
+@pytest.mark.parametrize("case", CASES)
+def test_forest_matches_oracle_per_request(case, dtype, rule):
+    B, H, Hk, n_max, dk, dv, L = case
+    wl = inputs.workload("c2", B=B, H=H, T=n_max, dk=dk, dv=dv, rule=rule, qkv_dtype=dtype, seed=400 + n_max)
+    parents, accepted = make_forest(B, n_max, seed=n_max + B)
+    total = sum(len(p) for p in parents)
+    capacity = total + 37                      # spare rows at the end of every plane
+    P, off = packed_tensors(wl, parents, capacity, Hk, L)
+    g = {n: (None if t is None else t.to(DEV)) for n, t in P.items()}
+    forest = tv.forest_build(parents, n_max=n_max, capacity=capacity).upload()
+    O = torch.full((L, H, capacity, dv), 7.0, device=DEV)
+    U = torch.full((L, H, capacity, dv), 7.0, device=DEV)
+    tv.tree_verify(forest, g["S_pre"], g["q"], g["k"], g["v"], g["alpha"], g["beta"], rule=rule, O=O, U=U)
+    acc = torch.from_numpy(accepted).to(DEV)
+    outs = []
+    for with_U in (False, True):
+        Sn = torch.empty_like(g["S_pre"])
+        tv.commit_path(forest, acc, g["S_pre"], g["k"], g["v"], g["alpha"], g["beta"], rule=rule,
+                       U=U if with_U else None, S_new=Sn)
+        outs.append(Sn.cpu().double().numpy())
+    torch.cuda.synchronize()
+    assert torch.equal(g["S_pre"].cpu(), P["S_pre"])
+    On, Un = O.cpu().double().numpy(), U.cpu().double().numpy()
+    assert (On[:, :, total:] == 7.0).all() and (Un[:, :, total:] == 7.0).all()   # spare rows untouched
+    tol = 1e-5 if dtype == inputs.F32 else 2e-3
+    for l in range(L):
+        for b in range(B):
+            n = len(parents[b])
+            rows = slice(int(off[b]), int(off[b]) + n)
+            for h in range(H):
+                Or, Ur, Sr = oracle_request(wl, P, off, parents, accepted, l, b, h, Hk)
+                assert rel_l2_rows(On[l, h, rows], Or) <= tol
+                assert rel_l2_rows(Un[l, h, rows], Ur) <= tol
+                for Sn in outs:
+                    assert rel_fro(Sn[l, b, h], Sr) <= tol
+
+
+def test_forest_metadata_and_rebuild():
+    parents, accepted = make_forest(5, 40, seed=3)
+    forest = tv.forest_build(parents, n_max=40, capacity=300).upload()
+    anc, depth, max_depth = forest.meta()
+    dev_anc, dev_depth = forest.meta_device()
+    assert np.array_equal(anc, dev_anc) and np.array_equal(depth, dev_depth)
+    for b, par in enumerate(parents):
+        ref_anc, ref_depth, ref_md = orc.tree_metadata(par)
+        n = len(par)
+        assert np.array_equal(anc[b, :n], ref_anc) and np.array_equal(depth[b, :n], ref_depth)
+        assert max_depth[b] == ref_md
+        assert not anc[b, n:].any() and not depth[b, n:].any()
+    # new topology with other sizes in the same buffers
+    parents2, _ = make_forest(5, 40, seed=4, kind="chain")
+    forest.rebuild_forest(parents2).upload()
+    anc2, depth2, _ = forest.meta()
+    dev_anc2, dev_depth2 = forest.meta_device()
+    assert np.array_equal(anc2, dev_anc2) and np.array_equal(depth2, dev_depth2)
+    assert depth2[0, 39] == 39
+
+
+def test_forest_argument_errors():
+    with pytest.raises(tv.TreeVerifyError) as e:
+        tv.forest_build([np.array([-1, 0]), np.array([-1])], n_max=1)
+    assert e.value.status == -1
+    with pytest.raises(tv.TreeVerifyError) as e:
+        tv.forest_build([np.array([-1, 0]), np.array([-1])], n_max=2, capacity=2)
+    assert e.value.status == -8
+    with pytest.raises(tv.TreeVerifyError) as e:
+        tv.forest_build([np.array([-1, 1])], n_max=2)
+    assert e.value.status == -2
+    dense = tv.tree_build(np.array([[-1, 0]], dtype=np.int32))
+    with pytest.raises(tv.TreeVerifyError):
+        dense.rebuild_forest([np.array([-1, 0])])
