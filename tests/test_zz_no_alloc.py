@@ -97,6 +97,11 @@ def test_static_call_allocates_nothing():
     O = torch.empty(wl.B, wl.H, wl.T, wl.dv, device="cuda")
     tv.tree_verify_static(par, t["S_pre"], t["q"], t["k"], t["v"], t["alpha"], O=O)   # loads the kernels
     torch.cuda.synchronize()
+    # handles left over from earlier tests free their device memory when they are collected:
+    # do that now, not between the two readings
+    import gc
+    gc.collect()
+    torch.cuda.synchronize()
     free0, _ = torch.cuda.mem_get_info()
     alloc0 = torch.cuda.memory_allocated()
     for _ in range(3):
