@@ -294,6 +294,115 @@ def time_stage1(tv, wl, tree, dev, stream, iters: int, W: int = 4):
             "launches": iters, "l2": f"{n_sets} rotating input set(s)"}
 
 
+def run_packed(args, wl, local_rank):
+    """The same step on a packed forest: every request keeps a random prefix of its tree (between
+    a quarter and all of its nodes), the node rows of all requests share flat planes.  One GPU;
+    prints a line of its own (not the headline configuration)."""
+    import paper_2608_01651_b200 as tv
+
+    tv.lib()
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    if args.layers:
+        wl = dataclasses.replace(wl, L=args.layers)
+    parents, _ = inputs.make_trees(wl)
+    rng = np.random.Generator(np.random.Philox(key=wl.seed + 77))
+    sizes = [wl.T] + [int(rng.integers(max(1, wl.T // 4), wl.T + 1)) for _ in range(wl.B - 1)]
+    trees = [np.ascontiguousarray(parents[b if parents.shape[0] > 1 else 0][:n]) for b, n in enumerate(sizes)]
+    accepted = np.array([inputs.accepted_walk(t, rng) for t in trees], dtype=np.int32)
+    offsets = np.zeros(wl.B + 1, dtype=np.int32)
+    offsets[1:] = np.cumsum(sizes)
+    total, cap = int(offsets[-1]), wl.B * wl.T
+    flat = np.ascontiguousarray(np.concatenate(trees), dtype=np.int32)
+    rows = torch.from_numpy(np.concatenate([b * wl.T + np.arange(n) for b, n in enumerate(sizes)])).to(dev)
+    delta = wl.rule == inputs.DELTA
+    eb = 2 if wl.qkv_dtype == inputs.BF16 else 4
+
+    def pack(t):   # dense [L,B,H,T,...] -> planes [L,H,cap,...] holding the kept rows first
+        t = t.transpose(1, 2)
+        t = t.reshape(t.shape[0], t.shape[1], wl.B * wl.T, *t.shape[4:])
+        out = torch.zeros_like(t)
+        out[:, :, :total] = t.index_select(2, rows)
+        return out.contiguous()
+
+    set_bytes = wl.L * (wl.B * wl.H * 4 * wl.dk * wl.dv + wl.H * total * (eb * (2 * wl.dk + wl.dv) + 4 * wl.dv))
+    n_sets = args.sets or max(2, min(8, int(np.ceil(4 * L2_BYTES / set_bytes))))
+    stream = torch.cuda.current_stream()
+    forest = tv.forest_build(trees, n_max=wl.T, capacity=cap)
+    acc_dev = torch.from_numpy(accepted).to(dev)
+    calls = []
+    for s in range(n_sets):
+        layers = [inputs.make_tensors(wl, layer=s * wl.L + l, device=dev) for l in range(wl.L)]
+        st = {k: (None if layers[0][k] is None else torch.stack([x[k] for x in layers])) for k in layers[0]}
+        del layers
+        P = {k: (None if st[k] is None else pack(st[k].unsqueeze(-1)).squeeze(-1) if k in ("alpha", "beta")
+                 else pack(st[k])) for k in ("q", "k", "v", "alpha", "beta")}
+        O = torch.empty(wl.L, wl.H, cap, wl.dv, device=dev, dtype=torch.float32)
+        U = torch.empty_like(O) if delta else None
+        ver = [tv.prepare_tree_verify(forest.upload(), st["S_pre"][l], P["q"][l], P["k"][l], P["v"][l],
+                                      P["alpha"][l], None if P["beta"] is None else P["beta"][l], rule=wl.rule,
+                                      O=O[l], U=None if U is None else U[l], stream=stream) for l in range(wl.L)]
+        com = tv.prepare_commit_path(forest, acc_dev, st["S_pre"], P["k"], P["v"], P["alpha"], P["beta"],
+                                     rule=wl.rule, U=U, stream=stream)
+        calls.append((ver, com, st, P, O, U))
+    refresh = forest.prepare_refresh_forest(flat, offsets, stream)
+    probe = max(1, args.probe_every)
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    pool = [(ev(), ev(), ev()) for _ in range(args.steps // probe + 1)]
+    used = []
+
+    def step(i, record):
+        ver, com = calls[i % n_sets][:2]
+        refresh()
+        if record:
+            e0, e1, e2 = pool[len(used)]
+            e0.record(stream)
+        for c in ver:
+            c()
+        if record:
+            e1.record(stream)
+        com()
+        if record:
+            e2.record(stream)
+            used.append((e0, e1, e2))
+
+    for i in range(max(3, args.warmup)):
+        step(i, False)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local_rank)
+    t0, t1 = ev(), ev()
+    t0.record(stream)
+    for i in range(args.steps):
+        step(i, i % probe == 0)
+    t1.record(stream)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = t0.elapsed_time(t1) / args.steps
+    v_ms = float(np.mean([a.elapsed_time(b) for a, b, _ in used])) / wl.L
+    c_ms = float(np.mean([b.elapsed_time(c) for _, b, c in used]))
+    peak, peak_kind = measured_peak()
+    vbytes = (wl.B * wl.H * 4 * wl.dk * wl.dv
+              + wl.H * total * (eb * (2 * wl.dk + wl.dv) + 4 + (4 if delta else 0) + 4 * wl.dv * (2 if delta else 1)))
+    v_gbs = vbytes / (v_ms * 1e-3) / 1e9
+    line = {
+        "metric": "verified_tree_nodes_per_s_per_layer", "value": total * wl.L / (ms * 1e-3), "unit": "nodes/s",
+        "n_gpus": 1, "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": DESCR[wl.name] + f"; PACKED FOREST: {total} nodes in {wl.B} requests of "
+                               f"{min(sizes)}..{max(sizes)} nodes, planes of {cap} rows",
+                   "layers_per_step": wl.L,
+                   "step": "tv_forest_rebuild+upload, tree_verify per layer, commit_path over all layers (in place)",
+                   "l2": f"{n_sets} rotating input set(s)"},
+        "verify": {"ms_per_layer": v_ms, "nodes_per_s_per_layer": total / (v_ms * 1e-3), "bytes": vbytes,
+                   "algorithmic_GBps": v_gbs, "frac_of_measured_copy": v_gbs / peak},
+        "commit": {"ms": c_ms},
+        "roofline": {"kernel": "tree_verify (packed)", "bound": "hbm", "achieved": v_gbs, "peak": peak,
+                     "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": v_gbs / peak, "traffic": None},
+        "cpu_baseline": None, "e2e": None, "gpu_launches": args.steps * (wl.L + 2), "clocks": clocks,
+    }
+    print(json.dumps(line, default=_jsonable), flush=True)
+
+
 def run_ours(args, wl, rank, world, local_rank):
     import paper_2608_01651_b200 as tv
     import torch.distributed as dist
@@ -506,6 +615,8 @@ def main():
                     help="ncu dram bytes per verify launch to echo into roofline.traffic")
     ap.add_argument("--probe-every", type=int, default=8,
                     help="record per-kernel CUDA events on every n-th timed step")
+    ap.add_argument("--packed", action="store_true",
+                    help="run the step on a packed forest of requests with different node counts (1 GPU)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-stage1", action="store_true")
     ap.add_argument("--stage1-iters", type=int, default=48)
@@ -520,6 +631,10 @@ def main():
 
     if args.impl == "reference":
         run_reference(args, wl, rank, world)
+        return
+    if args.packed:
+        if rank == 0:
+            run_packed(args, wl, local_rank)
         return
     if world > 1:
         import torch.distributed as dist

@@ -185,6 +185,25 @@ class Tree:
                 raise TreeVerifyError(st, "tv_tree_rebuild/tv_tree_upload")
         return refresh
 
+    def prepare_refresh_forest(self, parent_flat, offsets, stream=None):
+        """``tv_forest_rebuild`` + ``tv_tree_upload`` with pre-marshalled arguments; the caller
+        updates the two int32 arrays in place between calls."""
+        flat, off = np.asarray(parent_flat), np.asarray(offsets)
+        for a in (flat, off):
+            if a.dtype != np.int32 or not a.flags["C_CONTIGUOUS"]:
+                raise ValueError("parent_flat and offsets must be C-contiguous int32 arrays")
+        L = lib()
+        h, pp, po, sp = self._h, ctypes.c_void_p(flat.ctypes.data), ctypes.c_void_p(off.ctypes.data), _stream_ptr(stream)
+        rebuild, upload = L.tv_forest_rebuild, L.tv_tree_upload
+
+        def refresh(_keep=(flat, off, self)):
+            st = rebuild(h, pp, po)
+            if st == 0:
+                st = upload(h, sp)
+            if st != 0:
+                raise TreeVerifyError(st, "tv_forest_rebuild/tv_tree_upload")
+        return refresh
+
     def device_status(self, stream=None):
         """``tv_tree_device_status``: synchronise and raise if a device wait timed out."""
         _check(lib().tv_tree_device_status(self._h, _stream_ptr(stream)), "tv_tree_device_status")

@@ -98,12 +98,40 @@ struct TcParams {
   const float* alpha;
   float* O;
   int32_t* status;
+  // packed forest only: request b owns rows offsets[b] .. offsets[b+1]-1 of every plane of
+  // `capacity` rows; T is then the per-request node limit (width of the metadata slabs)
+  const int32_t* offsets;
+  int32_t capacity;
 };
 
+// (layer, request, head) of an item and, for a packed forest, where its rows live
+struct PackedItem {
+  int b, plane_v, plane_qk, row0, n;
+};
+__device__ __forceinline__ PackedItem packed_item(const TcParams& p, int item) {
+  PackedItem r;
+  const int lb = item / p.H, h = item - lb * p.H;
+  const int l = lb / p.B;
+  r.b = lb - l * p.B;
+  r.plane_v = l * p.H + h;
+  r.plane_qk = l * p.Hk + (p.Hk == p.H ? h : h / (p.H / p.Hk));
+  r.row0 = p.offsets[r.b];
+  r.n = p.offsets[r.b + 1] - r.row0;
+  return r;
+}
+
+// PACKED = packed forest: q/k/v/O are planes of `capacity` rows and an item's rows start at its
+// request's offset.  Loads take the fixed box at that offset (rows past the request belong to
+// other requests and are masked like padding); stores are cut to the request's node count:
+// 8-row-aligned part by TMA boxes of 64/32/16/8 rows (tmO, tmO32, tmO16, tmO8), the last < 8
+// rows straight from registers.  The dense instantiation ignores the three extra maps.
+template <bool PACKED>
 __global__ void __launch_bounds__(kThreads, 1)
 verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                        const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmS,
-                       const __grid_constant__ CUtensorMap tmO, const TcParams p) {
+                       const __grid_constant__ CUtensorMap tmO, const __grid_constant__ CUtensorMap tmO32,
+                       const __grid_constant__ CUtensorMap tmO16, const __grid_constant__ CUtensorMap tmO8,
+                       const TcParams p) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* sm = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   const uint32_t sbase = smem_u32(sm);
@@ -155,12 +183,20 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         const uint32_t ph = it & 1;
         if (!mbar_wait(bar(QK_FREE), ph ^ 1, abort_flag)) break;
         TC_STAMP(it, 0);
-        mbar_expect_tx(bar(QK_FULL), 4 * kTile);
-        const int qk = tv_qk_item(item, p.H, p.Hk);
-        tma_load_3d(sbase + kOffQ, &tmQ, bar(QK_FULL), 0, 0, qk);
-        tma_load_3d(sbase + kOffQ + kTile, &tmQ, bar(QK_FULL), 64, 0, qk);
-        tma_load_3d(sbase + kOffK, &tmK, bar(QK_FULL), 0, 0, qk);
-        tma_load_3d(sbase + kOffK + kTile, &tmK, bar(QK_FULL), 64, 0, qk);
+        // packed forest: boxes of 64 rows (per-request limit <= 64) or 128 rows at the request's offset
+        const uint32_t box_bytes = PACKED ? (T <= 64 ? kTile / 2 : kTile) : kTile;
+        int qk = 0, vplane = item, y0 = 0;
+        if constexpr (PACKED) {
+          const PackedItem pi = packed_item(p, item);
+          qk = pi.plane_qk; vplane = pi.plane_v; y0 = pi.row0;
+        } else {
+          qk = tv_qk_item(item, p.H, p.Hk);
+        }
+        mbar_expect_tx(bar(QK_FULL), 4 * box_bytes);
+        tma_load_3d(sbase + kOffQ, &tmQ, bar(QK_FULL), 0, y0, qk);
+        tma_load_3d(sbase + kOffQ + kTile, &tmQ, bar(QK_FULL), 64, y0, qk);
+        tma_load_3d(sbase + kOffK, &tmK, bar(QK_FULL), 0, y0, qk);
+        tma_load_3d(sbase + kOffK + kTile, &tmK, bar(QK_FULL), 64, y0, qk);
         pend_qk = 1 + (int)ph;
         if (!mbar_wait(bar(S_FREE), ph ^ 1, abort_flag)) break;
         TC_STAMP(it, 1);
@@ -171,9 +207,9 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         pend_s = 1 + (int)ph;
         if (!mbar_wait(bar(V_FREE), ph ^ 1, abort_flag)) break;
         TC_STAMP(it, 2);
-        mbar_expect_tx(bar(V_FULL), 2 * kTile);
-        tma_load_3d(sbase + kOffV, &tmV, bar(V_FULL), 0, 0, item);
-        tma_load_3d(sbase + kOffV + kTile, &tmV, bar(V_FULL), 64, 0, item);
+        mbar_expect_tx(bar(V_FULL), 2 * box_bytes);
+        tma_load_3d(sbase + kOffV, &tmV, bar(V_FULL), 0, y0, vplane);
+        tma_load_3d(sbase + kOffV + kTile, &tmV, bar(V_FULL), 64, y0, vplane);
         pend_v = 1 + (int)ph;
       }
       if (*abort_flag) {
@@ -264,7 +300,8 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       return small ? kOffChi + kTile + (uint32_t)(c4 >> 1) * (kOffClo - kOffChi) + (uint32_t)(c4 & 1) * 8192u
                    : kOffChi + (uint32_t)c4 * kTile;
     };
-    auto final_epilogue = [&](uint32_t it_prev, int item_prev, float r_prev, uint32_t ost_phase) -> bool {
+    auto final_epilogue = [&](uint32_t it_prev, int item_prev, float r_prev, uint32_t ost_phase,
+                              const PackedItem& pk_prev) -> bool {
       const int acc_done = (it_prev & 1) ? ACC_DONE1 : ACC_DONE0;
       const int acc_free = (it_prev & 1) ? ACC_FREE1 : ACC_FREE0;
       const uint32_t acc_col = (it_prev & 1) ? kColAcc1 : kColAcc0;
@@ -284,6 +321,11 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           tmem_ld32(tmem + lane_addr + acc_col + hc * 64 + half * 32, r1);
           tmem_wait_ld();
           unsigned char* orow = sm + stage_addr(hc * 2 + half) + row * 128;
+          // packed forest: the rows after the last full group of 8 leave from registers
+          const bool tail_row = PACKED && row >= (pk_prev.n & ~7) && row < pk_prev.n;
+          float* otail = nullptr;
+          if constexpr (PACKED)
+            otail = p.O + ((size_t)pk_prev.plane_v * p.capacity + pk_prev.row0 + row) * 128 + hc * 64 + half * 32;
 #pragma unroll
           for (int c = 0; c < 8; ++c) {
             float4 o;
@@ -292,6 +334,7 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             o.z = r_prev * __uint_as_float(r1[4 * c + 2]);
             o.w = r_prev * __uint_as_float(r1[4 * c + 3]);
             *reinterpret_cast<float4*>(orow + (((uint32_t)c ^ swz) << 4)) = o;
+            if (tail_row) *reinterpret_cast<float4*>(otail + 4 * c) = o;
           }
         }
       }
@@ -304,8 +347,28 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       }
       if (warp == 2 && lane == 0) {
         if (mbar_wait(bar(OST_READY), ost_phase, abort_flag)) {
+          if constexpr (PACKED) {
+            // groups of 8 rows, largest boxes first; staging rows r.. start on a 1024-byte
+            // boundary, so the swizzle phase of a partial box equals that of the full tile
+            const int full = pk_prev.n & ~7;
+            int r = 0;
+            auto put = [&](const CUtensorMap* m, int rows_box) {
+              while (full - r >= rows_box) {
 #pragma unroll
-          for (int c = 0; c < 4; ++c) tma_store_3d(&tmO, sbase + stage_addr(c), 32 * c, 0, item_prev);
+                for (int c = 0; c < 4; ++c)
+                  tma_store_3d(m, sbase + stage_addr(c) + (uint32_t)r * 128u, 32 * c, pk_prev.row0 + r,
+                               pk_prev.plane_v);
+                r += rows_box;
+              }
+            };
+            put(&tmO, 64);
+            put(&tmO32, 32);
+            put(&tmO16, 16);
+            put(&tmO8, 8);
+          } else {
+#pragma unroll
+            for (int c = 0; c < 4; ++c) tma_store_3d(&tmO, sbase + stage_addr(c), 32 * c, 0, item_prev);
+          }
           tma_store_commit();
           if (!small) tma_store_wait_read();   // the tiles may be overwritten once the store has read them
         }
@@ -317,9 +380,20 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     // metadata of the first item; later items are fetched one item ahead
     uint64_t nm0 = 0, nm1 = 0;
     float nal = 1.f;   // raw decay gate of the next item (log2 taken when it is used)
+    PackedItem npk = {0, 0, 0, 0, T};   // packed forest: rows of the next item
     auto fetch_meta = [&](int item) {
       nm0 = 0; nm1 = 0; nal = 1.f;
-      if (item < p.n_items && row < T) {
+      if constexpr (PACKED) {
+        if (item < p.n_items) {
+          npk = packed_item(p, item);
+          if (row < npk.n) {
+            const uint64_t* m = p.tree.anc + ((size_t)npk.b * T + row) * 2;
+            nm0 = m[0];
+            nm1 = m[1];
+            nal = p.alpha[(size_t)npk.plane_v * p.capacity + npk.row0 + row];
+          }
+        }
+      } else if (item < p.n_items && row < T) {
         const int b = (item / p.H) % p.B;
         const int tb = p.tree.n_trees == 1 ? 0 : b;
         const uint64_t* m = p.tree.anc + ((size_t)tb * T + row) * 2;
@@ -337,31 +411,35 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     bool ok = true;
     int item_prev = 0;
     float r_prev = 0.f;
+    PackedItem pk = npk, pk_prev = npk;
+    const int total_rows = PACKED ? p.offsets[p.B] : 0;   // rows at and past this one hold no node
     for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++it) {
       const uint32_t ph = it & 1;
       uint64_t m0 = nm0, m1 = nm1;
+      pk = npk;
+      const int Tb = PACKED ? pk.n : T;   // real nodes of this item
       if (warp == 4) TC_STAMP(it, 16);
       // ---- path decay: g_i = sum of log2(alpha) over Anc(i) + {i} ----
       const float la_own = log2f(nal);
-      if (hc == 0 && row < T) la_s[row] = la_own;
+      if (hc == 0 && row < Tb) la_s[row] = la_own;
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(SETUP));
       fetch_meta(item + (int)gridDim.x);   // next item's metadata rides under this item's work
       if (!(ok = mbar_wait_warp(bar(SETUP), 0, abort_flag))) break;   // SETUP: two phases per item
       float g = 0.f;
-      if (row < T) {
+      if (row < Tb) {
         g = la_own;
         uint64_t a0 = m0, a1 = m1;
         while (a0) { const int j = __ffsll((long long)a0) - 1; a0 &= a0 - 1; g += la_s[j]; }
         while (a1) { const int j = __ffsll((long long)a1) - 1; a1 &= a1 - 1; g += la_s[64 + j]; }
         if (row < 64) m0 |= 1ull << row; else m1 |= 1ull << (row - 64);   // M+ = M- + I
       }
-      if (hc == 0 && row < T) {
+      if (hc == 0 && row < Tb) {
         g_s[row] = g;
         f_s[row] = exp2f(-g);
       }
       // exp2(e_i - g_j) = 2^e_i * 2^-g_j is safe when every |g| <= 100; otherwise take exp2 per pair
-      const bool range_ok_warp = __all_sync(0xffffffffu, row >= T || fabsf(g) <= 100.f);
+      const bool range_ok_warp = __all_sync(0xffffffffu, row >= Tb || fabsf(g) <= 100.f);
       if (lane == 0) range_ok_s[cw] = range_ok_warp;
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(SETUP));
@@ -411,7 +489,7 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       if (!(ok = mbar_wait_warp(bar(SETUP), 1, abort_flag))) break;
       // ---- output rows of the previous item: its accumulator is complete once its readout MMA
       // is, and the C' tiles it frees double as the staging area of the output store ----
-      if (it > 0 && !(ok = final_epilogue(it - 1, item_prev, r_prev, (it - 1) & 1))) break;
+      if (it > 0 && !(ok = final_epilogue(it - 1, item_prev, r_prev, (it - 1) & 1, pk_prev))) break;
       tc_fence_after();
       if (warp == 4) TC_STAMP(it, 21);
       if (warp_live) {
@@ -456,6 +534,19 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           }
         }
       }
+      if constexpr (PACKED) {
+        // A box that reaches past the last node of the forest brings rows nobody wrote: zero them
+        // in the V tiles (0 x garbage would not be 0); K and Q rows are masked by selection.
+        const int box_rows = T <= 64 ? 64 : 128;
+        if (pk.row0 + box_rows > total_rows) {
+          if (!(ok = mbar_wait_warp(bar(V_FULL), ph, abort_flag))) break;
+          if (row >= total_rows - pk.row0 && row < box_rows) {
+            uint4* vrow = reinterpret_cast<uint4*>(sm + kOffV + hc * kTile + row * 128);
+#pragma unroll
+            for (int c = 0; c < 8; ++c) vrow[c] = make_uint4(0u, 0u, 0u, 0u);
+          }
+        }
+      }
       fence_async_smem();
       tc_fence_before();
       __syncwarp();
@@ -466,8 +557,9 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       if (warp == 4) TC_STAMP(it, 22);
       item_prev = item;
       r_prev = r_scale;
+      pk_prev = pk;
     }
-    if (ok && it > 0) final_epilogue(it - 1, item_prev, r_prev, (it - 1) & 1);
+    if (ok && it > 0) final_epilogue(it - 1, item_prev, r_prev, (it - 1) & 1, pk_prev);
     if (warp == 2 && lane == 0) tma_store_wait_all();   // our stores are complete before we leave
   }
 
@@ -497,6 +589,27 @@ __global__ void widen_bf16_kernel(const __nv_bfloat16* __restrict__ v, float* __
     b.z = __uint_as_float(w[3] << 16); b.w = __uint_as_float(w[3] & 0xffff0000u);
     reinterpret_cast<float4*>(U)[2 * i] = a;
     reinterpret_cast<float4*>(U)[2 * i + 1] = b;
+  }
+}
+
+// Packed forest: only the rows that hold nodes, plane by plane.
+__global__ void widen_bf16_rows_kernel(const __nv_bfloat16* __restrict__ v, float* __restrict__ U, size_t planes,
+                                       size_t capacity, const int32_t* __restrict__ offsets, int n_req) {
+  const size_t n8 = (size_t)offsets[n_req] * 128 / 8;   // 16-byte groups of one plane that hold nodes
+  for (size_t pl = blockIdx.y; pl < planes; pl += gridDim.y) {
+    const uint4* src = reinterpret_cast<const uint4*>(v + pl * capacity * 128);
+    float4* dst = reinterpret_cast<float4*>(U + pl * capacity * 128);
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n8; i += (size_t)gridDim.x * blockDim.x) {
+      const uint4 x = src[i];
+      const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+      float4 a, b;
+      a.x = __uint_as_float(w[0] << 16); a.y = __uint_as_float(w[0] & 0xffff0000u);
+      a.z = __uint_as_float(w[1] << 16); a.w = __uint_as_float(w[1] & 0xffff0000u);
+      b.x = __uint_as_float(w[2] << 16); b.y = __uint_as_float(w[2] & 0xffff0000u);
+      b.z = __uint_as_float(w[3] << 16); b.w = __uint_as_float(w[3] & 0xffff0000u);
+      dst[2 * i] = a;
+      dst[2 * i + 1] = b;
+    }
   }
 }
 
@@ -535,30 +648,56 @@ extern "C" __attribute__((visibility("default"))) int tv_selftest_wait_timeout(i
 }
 
 bool tv_verify_tc_supports(const VerifyArgs& a) {
-  if (a.tree.offsets != nullptr) return false;   // packed forests take the general kernel
   return a.bf16 && a.dk == 128 && a.dv == 128 && a.rule == TV_GATED && a.T <= 128;
 }
 
 int tv_launch_verify_tc(const VerifyArgs& a, int32_t* status, cudaStream_t stream) {
   if (!tv_verify_tc_supports(a)) return TV_ERR_UNSUPPORTED;
+  const bool packed = a.tree.offsets != nullptr;
   const uint64_t items = (uint64_t)a.L * a.B * a.H;
+  const uint64_t qk_items = (uint64_t)a.L * a.B * a.Hk;
   const uint32_t orows = a.T <= 64 ? 64 : 128;   // rows of one staged output chunk
   const void* const ptrs[5] = {a.q, a.k, a.v, a.S_pre, a.O};
-  const uint64_t qk_items = (uint64_t)a.L * a.B * a.Hk;
-  const MapSet* ms = cached_maps(ptrs, items, a.T, a.Hk << 8, [&](CUtensorMap* m) {
-    return make_map(&m[0], a.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, qk_items, a.T, 128, 64) &&
-           make_map(&m[1], a.k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, qk_items, a.T, 128, 64) &&
-           make_map(&m[2], a.v, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, items, a.T, 128, 64) &&
-           make_map(&m[3], a.S_pre, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, 128, 128, 32) &&
-           make_map(&m[4], a.O, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, a.T, 128, 32, orows);
-  });
-  if (!ms) return TV_ERR_CUDA;
+  const MapSet* ms = nullptr;
+  const MapSet* mo = nullptr;   // packed forest: output boxes of 32, 16 and 8 rows
+  if (!packed) {
+    ms = cached_maps(ptrs, items, a.T, a.Hk << 8, [&](CUtensorMap* m) {
+      return make_map(&m[0], a.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, qk_items, a.T, 128, 64) &&
+             make_map(&m[1], a.k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, qk_items, a.T, 128, 64) &&
+             make_map(&m[2], a.v, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, items, a.T, 128, 64) &&
+             make_map(&m[3], a.S_pre, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, 128, 128, 32) &&
+             make_map(&m[4], a.O, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, a.T, 128, 32, orows);
+    });
+    mo = ms;
+  } else {
+    // planes of `capacity` rows; loads in boxes of 64 or 128 rows, stores in boxes of 64/32/16/8
+    const uint64_t cap = (uint64_t)a.tree.capacity;
+    const uint64_t pv = (uint64_t)a.L * a.H, pqk = (uint64_t)a.L * a.Hk;
+    const uint32_t lrows = a.T <= 64 ? 64 : 128;
+    const uint64_t key = (cap << 24) ^ items;
+    ms = cached_maps(ptrs, key, a.T, 4 | (a.Hk << 8), [&](CUtensorMap* m) {
+      return make_map(&m[0], a.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, pqk, cap, 128, 64, lrows) &&
+             make_map(&m[1], a.k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, pqk, cap, 128, 64, lrows) &&
+             make_map(&m[2], a.v, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, pv, cap, 128, 64, lrows) &&
+             make_map(&m[3], a.S_pre, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, 128, 128, 32) &&
+             make_map(&m[4], a.O, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, pv, cap, 128, 32, 64);
+    });
+    const void* const optrs[5] = {a.O, nullptr, nullptr, nullptr, nullptr};
+    mo = cached_maps(optrs, key, a.T, 5, [&](CUtensorMap* m) {
+      return make_map(&m[0], a.O, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, pv, cap, 128, 32, 32) &&
+             make_map(&m[1], a.O, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, pv, cap, 128, 32, 16) &&
+             make_map(&m[2], a.O, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, pv, cap, 128, 32, 8);
+    });
+  }
+  if (!ms || !mo) return TV_ERR_CUDA;
   static thread_local int configured_dev = -1;
   static thread_local int sm_count = 0;
   int dev = 0;
   TV_CUDA_TRY(cudaGetDevice(&dev));
   if (configured_dev != dev) {
-    TV_CUDA_TRY(cudaFuncSetAttribute(verify_tc_gated_kernel,
+    TV_CUDA_TRY(cudaFuncSetAttribute(verify_tc_gated_kernel<false>,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
+    TV_CUDA_TRY(cudaFuncSetAttribute(verify_tc_gated_kernel<true>,
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
     TV_CUDA_TRY(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev));
     configured_dev = dev;
@@ -570,9 +709,24 @@ int tv_launch_verify_tc(const VerifyArgs& a, int32_t* status, cudaStream_t strea
   p.alpha = a.alpha;
   p.O = a.O;
   p.status = status;
+  p.offsets = a.tree.offsets;
+  p.capacity = a.tree.capacity;
   const int grid = (int)(items < (uint64_t)sm_count ? items : (uint64_t)sm_count);
-  TV_CUDA_TRY(launch_dependent(verify_tc_gated_kernel, grid, kThreads, kSmemBytes, stream, ms->map[0],
-                               ms->map[1], ms->map[2], ms->map[3], ms->map[4], p));
+  if (packed) {
+    TV_CUDA_TRY(launch_dependent(verify_tc_gated_kernel<true>, grid, kThreads, kSmemBytes, stream, ms->map[0],
+                                 ms->map[1], ms->map[2], ms->map[3], ms->map[4], mo->map[0], mo->map[1],
+                                 mo->map[2], p));
+    if (a.U) {
+      const size_t planes = (size_t)a.L * a.H;
+      widen_bf16_rows_kernel<<<dim3(64, (unsigned)(planes < 65535 ? planes : 65535)), 256, 0, stream>>>(
+          reinterpret_cast<const __nv_bfloat16*>(a.v), a.U, planes, (size_t)a.tree.capacity, a.tree.offsets, a.B);
+      TV_CUDA_TRY(cudaGetLastError());
+    }
+    return TV_OK;
+  }
+  TV_CUDA_TRY(launch_dependent(verify_tc_gated_kernel<false>, grid, kThreads, kSmemBytes, stream, ms->map[0],
+                               ms->map[1], ms->map[2], ms->map[3], ms->map[4], ms->map[4], ms->map[4],
+                               ms->map[4], p));
   if (a.U) {
     const size_t n8 = items * a.T * 128 / 8;
     const int blocks = (int)((n8 + 255) / 256 < 4096 ? (n8 + 255) / 256 : 4096);

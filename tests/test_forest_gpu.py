@@ -37,7 +37,7 @@ def packed_tensors(wl, parents, capacity, Hk, L=1):
     dt = wl.torch_dtype
     off = np.concatenate([[0], np.cumsum([len(p) for p in parents])]).astype(np.int64)
     layers = [inputs.make_tensors(wl, layer=l) for l in range(L)]
-    fill = lambda *shape: torch.full(shape, 3.0)   # rows past the forest must stay untouched/unread
+    fill = lambda *shape: torch.full(shape, float("nan"))   # rows past the forest: whatever is read there must not matter
     P = {"q": fill(L, Hk, capacity, wl.dk).to(dt), "k": fill(L, Hk, capacity, wl.dk).to(dt),
          "v": fill(L, H, capacity, wl.dv).to(dt), "alpha": fill(L, H, capacity),
          "beta": fill(L, H, capacity) if layers[0]["beta"] is not None else None,
@@ -74,13 +74,16 @@ CASES = [  # B, H, Hk, n_max, dk, dv, L
     (4, 4, 2, 128, 128, 128, 2),
     (6, 2, 1, 33, 64, 128, 1),
     (3, 2, 2, 17, 64, 64, 1),
+    (9, 2, 2, 8, 128, 128, 1),
+    (40, 2, 2, 70, 128, 128, 1),
 ]
 
 
+@pytest.mark.parametrize("impl", [tv.IMPL_AUTO, tv.IMPL_SIMT])
 @pytest.mark.parametrize("rule", [inputs.GATED, inputs.DELTA])
 @pytest.mark.parametrize("dtype", [inputs.BF16, inputs.F32])
 @pytest.mark.parametrize("case", CASES)
-def test_forest_matches_oracle_per_request(case, dtype, rule):
+def test_forest_matches_oracle_per_request(case, dtype, rule, impl):
     B, H, Hk, n_max, dk, dv, L = case
     wl = inputs.workload("c2", B=B, H=H, T=n_max, dk=dk, dv=dv, rule=rule, qkv_dtype=dtype, seed=400 + n_max)
     parents, accepted = make_forest(B, n_max, seed=n_max + B)
@@ -91,7 +94,8 @@ def test_forest_matches_oracle_per_request(case, dtype, rule):
     forest = tv.forest_build(parents, n_max=n_max, capacity=capacity).upload()
     O = torch.full((L, H, capacity, dv), 7.0, device=DEV)
     U = torch.full((L, H, capacity, dv), 7.0, device=DEV)
-    tv.tree_verify(forest, g["S_pre"], g["q"], g["k"], g["v"], g["alpha"], g["beta"], rule=rule, O=O, U=U)
+    tv.tree_verify(forest, g["S_pre"], g["q"], g["k"], g["v"], g["alpha"], g["beta"], rule=rule, O=O, U=U,
+                   impl=impl)
     acc = torch.from_numpy(accepted).to(DEV)
     outs = []
     for with_U in (False, True):
@@ -100,6 +104,7 @@ def test_forest_matches_oracle_per_request(case, dtype, rule):
                        U=U if with_U else None, S_new=Sn)
         outs.append(Sn.cpu().double().numpy())
     torch.cuda.synchronize()
+    forest.device_status()          # raises if a bounded device wait ran out
     assert torch.equal(g["S_pre"].cpu(), P["S_pre"])
     On, Un = O.cpu().double().numpy(), U.cpu().double().numpy()
     assert (On[:, :, total:] == 7.0).all() and (Un[:, :, total:] == 7.0).all()   # spare rows untouched
@@ -114,6 +119,25 @@ def test_forest_matches_oracle_per_request(case, dtype, rule):
                 assert rel_l2_rows(Un[l, h, rows], Ur) <= tol
                 for Sn in outs:
                     assert rel_fro(Sn[l, b, h], Sr) <= tol
+
+
+def test_forest_takes_the_tensor_core_kernel():
+    """Gated rule, bf16, dk = dv = 128: IMPL_TC must accept a packed forest (and the delta rule,
+    which has no packed tensor-core kernel, must decline rather than fall back silently)."""
+    wl = inputs.workload("c2", B=4, H=2, T=64, seed=11)
+    parents, _ = make_forest(4, 64, seed=12)
+    cap = sum(len(p) for p in parents)
+    P, _ = packed_tensors(wl, parents, cap, 2)
+    g = {n: (None if t is None else t.to(DEV)) for n, t in P.items()}
+    forest = tv.forest_build(parents, n_max=64, capacity=cap).upload()
+    O1 = tv.tree_verify(forest, g["S_pre"], g["q"], g["k"], g["v"], g["alpha"], impl=tv.IMPL_TC)
+    O2 = tv.tree_verify(forest, g["S_pre"], g["q"], g["k"], g["v"], g["alpha"], impl=tv.IMPL_SIMT)
+    torch.cuda.synchronize()
+    assert rel_fro(O1.cpu().double().numpy(), O2.cpu().double().numpy()) < 2e-3
+    with pytest.raises(tv.TreeVerifyError) as e:
+        tv.tree_verify(forest, g["S_pre"], g["q"], g["k"], g["v"], g["alpha"], torch.ones_like(g["alpha"]),
+                       rule=inputs.DELTA, impl=tv.IMPL_TC)
+    assert e.value.status == -3
 
 
 def test_forest_metadata_and_rebuild():
