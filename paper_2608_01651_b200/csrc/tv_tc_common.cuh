@@ -190,6 +190,23 @@ inline bool make_map(CUtensorMap* map, const void* base, CUtensorMapDataType dt,
 }
 
 
+// (layer, request, head) of a work item and, for a packed forest, where its rows live: request b
+// owns rows offsets[b] .. offsets[b+1]-1 of every (layer, head) plane.
+struct PackedItem {
+  int b, plane_v, plane_qk, row0, n;
+};
+__device__ __forceinline__ PackedItem packed_item(const int32_t* offsets, int B, int H, int Hk, int item) {
+  PackedItem r;
+  const int lb = item / H, h = item - lb * H;
+  const int l = lb / B;
+  r.b = lb - l * B;
+  r.plane_v = l * H + h;
+  r.plane_qk = l * Hk + (Hk == H ? h : h / (H / Hk));
+  r.row0 = offsets[r.b];
+  r.n = offsets[r.b + 1] - r.row0;
+  return r;
+}
+
 // Programmatic dependent launch: the kernel may start while the kernel in front of it on the
 // stream is still running, provided that kernel released its dependents early; whatever reads
 // that kernel's output first passes grid_dependency_wait().

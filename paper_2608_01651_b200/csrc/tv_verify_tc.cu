@@ -104,20 +104,8 @@ struct TcParams {
   int32_t capacity;
 };
 
-// (layer, request, head) of an item and, for a packed forest, where its rows live
-struct PackedItem {
-  int b, plane_v, plane_qk, row0, n;
-};
 __device__ __forceinline__ PackedItem packed_item(const TcParams& p, int item) {
-  PackedItem r;
-  const int lb = item / p.H, h = item - lb * p.H;
-  const int l = lb / p.B;
-  r.b = lb - l * p.B;
-  r.plane_v = l * p.H + h;
-  r.plane_qk = l * p.Hk + (p.Hk == p.H ? h : h / (p.H / p.Hk));
-  r.row0 = p.offsets[r.b];
-  r.n = p.offsets[r.b + 1] - r.row0;
-  return r;
+  return tvtc::packed_item(p.offsets, p.B, p.H, p.Hk, item);
 }
 
 // PACKED = packed forest: q/k/v/O are planes of `capacity` rows and an item's rows start at its

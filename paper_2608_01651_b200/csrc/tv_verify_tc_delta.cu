@@ -85,6 +85,12 @@ struct DeltaParams {
   const float* beta;
   int32_t want_U;
   int32_t* status;
+  // packed forest only (see tv_verify_tc.cu): row offsets of the requests, rows per plane, and the
+  // outputs as plain pointers for the rows that leave from registers
+  const int32_t* offsets;
+  int32_t capacity;
+  float* O;
+  float* U;
 };
 
 // 2^x in one MUFU instruction (2 ulp; denormal results flush to zero, which is what a decay
@@ -105,12 +111,21 @@ __device__ __forceinline__ void split_bf16(float x, uint16_t& hi, uint16_t& lo) 
 
 // DMAX: compile-time bound on the tree depth (8 covers draft trees, 15 the rest), so that the
 // per-row triangular solve is straight-line code whose loads all issue up front.
-template <int DMAX>
+// PACKED = packed forest: loads take the 64-row box at the request's offset, stores are cut to
+// the request's node count (TMA boxes of 64/32/16/8 rows, then a register tail), and operand
+// rows past the last node of the forest are zeroed in shared memory before they meet a zero
+// coefficient.  The dense instantiation is given the 64-row maps for all box sizes and ignores them.
+struct OutMaps {
+  CUtensorMap m64, m32, m16, m8;
+};
+template <int DMAX, bool PACKED>
 __global__ void __launch_bounds__(kThreads, 1)
 verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                        const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmS,
-                       const __grid_constant__ CUtensorMap tmO, const __grid_constant__ CUtensorMap tmU,
+                       const __grid_constant__ OutMaps mapsO, const __grid_constant__ OutMaps mapsU,
                        const DeltaParams p) {
+  const CUtensorMap& tmO = mapsO.m64;
+  const CUtensorMap& tmU = mapsU.m64;
   extern __shared__ unsigned char smem_raw[];
   unsigned char* sm = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   const uint32_t sbase = smem_u32(sm);
@@ -163,11 +178,17 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         const uint32_t ph = it & 1;
         if (!mbar_wait(bar(QK_FREE), ph ^ 1, abort_flag)) break;
         mbar_expect_tx(bar(QK_FULL), 4 * 8192);
-        const int qk = tv_qk_item(item, p.H, p.Hk);
-        tma_load_3d(sbase + kOffQK, &tmQ, bar(QK_FULL), 0, 0, qk);
-        tma_load_3d(sbase + kOffQK + kTile, &tmQ, bar(QK_FULL), 64, 0, qk);
-        tma_load_3d(sbase + kOffQK + 8192, &tmK, bar(QK_FULL), 0, 0, qk);
-        tma_load_3d(sbase + kOffQK + kTile + 8192, &tmK, bar(QK_FULL), 64, 0, qk);
+        int qk = 0, vplane = item, y0 = 0;
+        if constexpr (PACKED) {
+          const PackedItem pi = packed_item(p.offsets, p.B, p.H, p.Hk, item);
+          qk = pi.plane_qk; vplane = pi.plane_v; y0 = pi.row0;
+        } else {
+          qk = tv_qk_item(item, p.H, p.Hk);
+        }
+        tma_load_3d(sbase + kOffQK, &tmQ, bar(QK_FULL), 0, y0, qk);
+        tma_load_3d(sbase + kOffQK + kTile, &tmQ, bar(QK_FULL), 64, y0, qk);
+        tma_load_3d(sbase + kOffQK + 8192, &tmK, bar(QK_FULL), 0, y0, qk);
+        tma_load_3d(sbase + kOffQK + kTile + 8192, &tmK, bar(QK_FULL), 64, y0, qk);
         pend_qk = 1 + (int)ph;
         if (!mbar_wait(bar(S_FREE), ph ^ 1, abort_flag)) break;
         mbar_expect_tx(bar(S_FULL), 4 * kTile);
@@ -177,8 +198,8 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         pend_s = 1 + (int)ph;
         if (!mbar_wait(bar(V_FREE), ph ^ 1, abort_flag)) break;
         mbar_expect_tx(bar(V_FULL), 2 * 8192);
-        tma_load_3d(sbase + kOffV, &tmV, bar(V_FULL), 0, 0, item);
-        tma_load_3d(sbase + kOffV + kTile, &tmV, bar(V_FULL), 64, 0, item);
+        tma_load_3d(sbase + kOffV, &tmV, bar(V_FULL), 0, y0, vplane);
+        tma_load_3d(sbase + kOffV + kTile, &tmV, bar(V_FULL), 64, y0, vplane);
         pend_v = 1 + (int)ph;
       }
       if (*abort_flag) {
@@ -193,11 +214,34 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       uint32_t it = 0;
       for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++it) {
         if (!mbar_wait(bar(OST_READY), it & 1, abort_flag)) break;
+        if constexpr (PACKED) {
+          // groups of 8 rows, largest boxes first (staging rows start on 1024-byte boundaries)
+          const PackedItem pi = packed_item(p.offsets, p.B, p.H, p.Hk, item);
+          const int full = pi.n & ~7;
+          for (int part = 0; part < (want_U ? 2 : 1); ++part) {
+            const OutMaps& mm = part == 0 ? mapsO : mapsU;
+            int r = 0;
+            auto put = [&](const CUtensorMap* m, int rows_box) {
+              while (full - r >= rows_box) {
 #pragma unroll
-        for (int c = 0; c < 4; ++c) tma_store_3d(&tmO, sbase + kOffStage + c * 8192, 32 * c, 0, item);
-        if (want_U) {
+                for (int c = 0; c < 4; ++c)
+                  tma_store_3d(m, sbase + kOffStage + (part * 4 + c) * 8192 + (uint32_t)r * 128u, 32 * c,
+                               pi.row0 + r, pi.plane_v);
+                r += rows_box;
+              }
+            };
+            put(&mm.m64, 64);
+            put(&mm.m32, 32);
+            put(&mm.m16, 16);
+            put(&mm.m8, 8);
+          }
+        } else {
 #pragma unroll
-          for (int c = 0; c < 4; ++c) tma_store_3d(&tmU, sbase + kOffStage + (4 + c) * 8192, 32 * c, 0, item);
+          for (int c = 0; c < 4; ++c) tma_store_3d(&tmO, sbase + kOffStage + c * 8192, 32 * c, 0, item);
+          if (want_U) {
+#pragma unroll
+            for (int c = 0; c < 4; ++c) tma_store_3d(&tmU, sbase + kOffStage + (4 + c) * 8192, 32 * c, 0, item);
+          }
         }
         tma_store_commit();
         tma_store_wait_read();
@@ -293,9 +337,20 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
 
     uint64_t nm = 0;
     float nal = 1.f, nbe = 0.f;
+    PackedItem npk = {0, 0, 0, 0, T};   // packed forest: rows of the next item
     auto fetch_meta = [&](int item) {
       nm = 0; nal = 1.f; nbe = 0.f;
-      if (item < p.n_items && node < T) {
+      if constexpr (PACKED) {
+        if (item < p.n_items) {
+          npk = packed_item(p.offsets, p.B, p.H, p.Hk, item);
+          if (node < npk.n) {
+            const size_t r = (size_t)npk.plane_v * p.capacity + npk.row0 + node;
+            nm = p.tree.anc[((size_t)npk.b * T + node) * 2];
+            nal = p.alpha[r];
+            nbe = p.beta[r];
+          }
+        }
+      } else if (item < p.n_items && node < T) {
         const int b = (item / p.H) % p.B;
         const int tb = p.tree.n_trees == 1 ? 0 : b;
         nm = p.tree.anc[((size_t)tb * T + node) * 2];
@@ -308,7 +363,7 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
 
     // acc rows 0..63 -> O chunks 0..3, rows 64..127 -> U chunks 4..7 (the chunks alias the Ak / W
     // tiles, which are idle between the readout MMA of item k and E2 of item k+1)
-    auto final_epilogue = [&](uint32_t it_prev) -> bool {
+    auto final_epilogue = [&](uint32_t it_prev, const PackedItem& pk_prev) -> bool {
       if (!mbar_wait_warp(bar(ACC_DONE), it_prev & 1, abort_flag)) return false;
       tc_fence_after();
       if (warp_live) {
@@ -318,10 +373,18 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           tmem_ld32(tmem + lane_addr + kColAcc + hc * 64 + half * 32, r1);
           tmem_wait_ld();
           unsigned char* orow = sm + kOffStage + (part * 4 + hc * 2 + half) * 8192 + node * 128;
+          // packed forest: the rows after the last full group of 8 leave from registers
+          const bool tail_row = PACKED && node >= (pk_prev.n & ~7) && node < pk_prev.n;
+          float* otail = nullptr;
+          if constexpr (PACKED)
+            otail = (part == 0 ? p.O : p.U) +
+                    ((size_t)pk_prev.plane_v * p.capacity + pk_prev.row0 + node) * 128 + hc * 64 + half * 32;
 #pragma unroll
-          for (int c = 0; c < 8; ++c)
-            *reinterpret_cast<uint4*>(orow + (((uint32_t)c ^ nswz) << 4)) =
-                make_uint4(r1[4 * c], r1[4 * c + 1], r1[4 * c + 2], r1[4 * c + 3]);
+          for (int c = 0; c < 8; ++c) {
+            const uint4 o4 = make_uint4(r1[4 * c], r1[4 * c + 1], r1[4 * c + 2], r1[4 * c + 3]);
+            *reinterpret_cast<uint4*>(orow + (((uint32_t)c ^ nswz) << 4)) = o4;
+            if (tail_row) *reinterpret_cast<uint4*>(otail + 4 * c) = o4;
+          }
         }
       }
       fence_async_smem();
@@ -336,12 +399,17 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
 
     uint32_t it = 0;
     bool ok = true;
+    PackedItem pk = npk, pk_prev = npk;
+    const int total_rows = PACKED ? p.offsets[p.B] : 0;   // rows at and past this one hold no node
     for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++it) {
       const uint32_t ph = it & 1;
+      pk = npk;
+      const int Tb = PACKED ? pk.n : T;                       // real nodes of this item
+      const bool live_i = live && node < Tb;
       if (warp == 4) TCD_STAMP(it, 16);
       // ---- per-node tables of this item ----
-      const uint64_t m = node < T ? nm : 0ull;                // strict ancestors
-      if (part == 0 && hc == 0 && node < T) {
+      const uint64_t m = node < Tb ? nm : 0ull;               // strict ancestors
+      if (part == 0 && hc == 0 && node < Tb) {
         la_s[node] = log2f(nal);
         be_s[node] = nbe;
       }
@@ -355,7 +423,7 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       if (warp == 4) TCD_STAMP(it, 18);
       tc_fence_after();
       if (rows_live) {
-        const uint64_t sel = node < T ? (part == 0 ? (m | (1ull << node)) : m) : 0ull;
+        const uint64_t sel = node < Tb ? (part == 0 ? (m | (1ull << node)) : m) : 0ull;
         float* dst = (part == 0 ? Cs : Gs) + node * kLd;
         const int cbase = hc * 32;
         const uint32_t bits = (uint32_t)(sel >> cbase);
@@ -379,7 +447,7 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       }
       if (warp == 4) TCD_STAMP(it, 19);
       // ---- output of the previous item (its MMAs ran under E1 above) ----
-      if (it > 0 && !(ok = final_epilogue(it - 1))) break;
+      if (it > 0 && !(ok = final_epilogue(it - 1, pk_prev))) break;
       if (warp == 4) TCD_STAMP(it, 17);
       if (!(ok = mbar_wait_warp(bar(SETUP), ph, abort_flag))) break;
       if (!(ok = mbar_wait_warp(bar(E1_SYNC), ph, abort_flag))) break;
@@ -390,7 +458,7 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       int path[NS];
       float gp[NS], bt[NS], vec[NS];
       float gi = 0.f;
-      if (live) {
+      if (live_i) {
         const uint32_t* pw = reinterpret_cast<const uint32_t*>(Ps + node * kLdP);
         const uint32_t pword[4] = {pw[0], pw[1], pw[2], pw[3]};
         float run = 0.f;
@@ -426,7 +494,24 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       // The tiles alias the staged output chunks of the previous item: its stores must have read
       // them (they did so under the solve above).
       if (it > 0 && !(ok = mbar_wait_warp(bar(OST_FREE), (it - 1) & 1, abort_flag))) break;
-      if (live) {
+      if constexpr (PACKED) {
+        // A box that reaches past the last node of the forest brings rows nobody wrote.  They only
+        // ever meet zero coefficients, but 0 x garbage need not be 0: zero them.  The Gram MMA has
+        // finished with Q and K (G_DONE above); V is waited for here.
+        if (pk.row0 + kRows > total_rows) {
+          if (!(ok = mbar_wait_warp(bar(V_FULL), ph, abort_flag))) break;
+          if (node >= total_rows - pk.row0 && !(part == 1 && hc == 1)) {
+            const uint32_t base = part == 1 ? kOffV : hc == 0 ? kOffQK : kOffQK + 8192;
+            const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+            for (int tile = 0; tile < 2; ++tile)
+#pragma unroll
+              for (int c = 0; c < 8; ++c)
+                *reinterpret_cast<uint4*>(sm + base + tile * kTile + node * 128 + c * 16) = z;
+          }
+        }
+      }
+      if (live_i) {
         // hc 0 writes the [W ; A] tiles, hc 1 the -[W D_P ; A D_P] tiles (and the diagonal of P)
         unsigned char* trow = sm + (hc == 0 ? kOffW : kOffAk) + row * 128;
         const uint4 z = make_uint4(0u, 0u, 0u, 0u);
@@ -460,8 +545,9 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(W_READY));
       if (warp == 4) TCD_STAMP(it, 21);
+      pk_prev = pk;
     }
-    if (ok && it > 0) final_epilogue(it - 1);
+    if (ok && it > 0) final_epilogue(it - 1, pk_prev);
   }
 
   tc_fence_before();
@@ -483,38 +569,80 @@ extern "C" __attribute__((visibility("default"))) int tv_debug_set_tcd_profile(l
 #endif
 
 bool tv_verify_tc_delta_supports(const VerifyArgs& a) {
-  if (a.tree.offsets != nullptr) return false;   // packed forests take the general kernel
   return a.bf16 && a.dk == 128 && a.dv == 128 && a.rule == TV_GATED_DELTA && a.T <= kRows &&
          a.tree.max_depth_all < kSlots;
 }
 
 int tv_launch_verify_tc_delta(const VerifyArgs& a, int32_t* status, cudaStream_t stream) {
   if (!tv_verify_tc_delta_supports(a)) return TV_ERR_UNSUPPORTED;
+  const bool packed = a.tree.offsets != nullptr;
   const uint64_t items = (uint64_t)a.L * a.B * a.H;
-  // the U map is only used when U is requested; O stands in otherwise
+  // the U maps are only used when U is requested; O stands in otherwise
   float* Uout = a.U ? a.U : a.O;
   const void* const ptrs[5] = {a.q, a.k, a.v, a.S_pre, a.O};
-  const uint64_t qk_items = (uint64_t)a.L * a.B * a.Hk;
-  const MapSet* ms = cached_maps(ptrs, items, a.T, 1 | (a.Hk << 8), [&](CUtensorMap* m) {
-    return make_map(&m[0], a.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, qk_items, a.T, 128, 64, 64) &&
-           make_map(&m[1], a.k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, qk_items, a.T, 128, 64, 64) &&
-           make_map(&m[2], a.v, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, items, a.T, 128, 64, 64) &&
-           make_map(&m[3], a.S_pre, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, 128, 128, 32, 128) &&
-           make_map(&m[4], a.O, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, a.T, 128, 32, 64);
-  });
   const void* const uptrs[5] = {Uout, nullptr, nullptr, nullptr, nullptr};
-  const MapSet* mu = cached_maps(uptrs, items, a.T, 2, [&](CUtensorMap* m) {
-    return make_map(&m[0], Uout, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, a.T, 128, 32, 64);
-  });
-  if (!ms || !mu) return TV_ERR_CUDA;
+  const uint64_t qk_items = (uint64_t)a.L * a.B * a.Hk;
+  const MapSet* ms = nullptr;   // q, k, v, S, O (64-row boxes)
+  const MapSet* mu = nullptr;   // U (64-row boxes)
+  const MapSet* mo2 = nullptr;  // packed forest: O boxes of 32, 16, 8 rows
+  const MapSet* mu2 = nullptr;  // packed forest: U boxes of 32, 16, 8 rows
+  if (!packed) {
+    ms = cached_maps(ptrs, items, a.T, 1 | (a.Hk << 8), [&](CUtensorMap* m) {
+      return make_map(&m[0], a.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, qk_items, a.T, 128, 64, 64) &&
+             make_map(&m[1], a.k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, qk_items, a.T, 128, 64, 64) &&
+             make_map(&m[2], a.v, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, items, a.T, 128, 64, 64) &&
+             make_map(&m[3], a.S_pre, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, 128, 128, 32, 128) &&
+             make_map(&m[4], a.O, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, a.T, 128, 32, 64);
+    });
+    mu = cached_maps(uptrs, items, a.T, 2, [&](CUtensorMap* m) {
+      return make_map(&m[0], Uout, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, a.T, 128, 32, 64);
+    });
+  } else {
+    const uint64_t cap = (uint64_t)a.tree.capacity;
+    const uint64_t pv = (uint64_t)a.L * a.H, pqk = (uint64_t)a.L * a.Hk;
+    const uint64_t key = (cap << 24) ^ items;
+    ms = cached_maps(ptrs, key, a.T, 6 | (a.Hk << 8), [&](CUtensorMap* m) {
+      return make_map(&m[0], a.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, pqk, cap, 128, 64, 64) &&
+             make_map(&m[1], a.k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, pqk, cap, 128, 64, 64) &&
+             make_map(&m[2], a.v, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, pv, cap, 128, 64, 64) &&
+             make_map(&m[3], a.S_pre, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, 128, 128, 32, 128) &&
+             make_map(&m[4], a.O, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, pv, cap, 128, 32, 64);
+    });
+    auto small_boxes = [&](float* base) {
+      return [=](CUtensorMap* m) {
+        return make_map(&m[0], base, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, pv, cap, 128, 32, 32) &&
+               make_map(&m[1], base, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, pv, cap, 128, 32, 16) &&
+               make_map(&m[2], base, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, pv, cap, 128, 32, 8) &&
+               make_map(&m[3], base, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, pv, cap, 128, 32, 64);
+      };
+    };
+    const void* const optrs[5] = {a.O, nullptr, nullptr, nullptr, (const void*)1};
+    const void* const u2ptrs[5] = {Uout, nullptr, nullptr, nullptr, (const void*)2};
+    mo2 = cached_maps(optrs, key, a.T, 7, small_boxes(a.O));
+    mu2 = cached_maps(u2ptrs, key, a.T, 7, small_boxes(Uout));
+    mu = mu2;
+  }
+  if (!ms || !mu || (packed && (!mo2 || !mu2))) return TV_ERR_CUDA;
+  OutMaps mapsO, mapsU;
+  if (packed) {
+    mapsO.m64 = ms->map[4]; mapsO.m32 = mo2->map[0]; mapsO.m16 = mo2->map[1]; mapsO.m8 = mo2->map[2];
+    mapsU.m64 = mu2->map[3]; mapsU.m32 = mu2->map[0]; mapsU.m16 = mu2->map[1]; mapsU.m8 = mu2->map[2];
+  } else {
+    mapsO.m64 = mapsO.m32 = mapsO.m16 = mapsO.m8 = ms->map[4];
+    mapsU.m64 = mapsU.m32 = mapsU.m16 = mapsU.m8 = mu->map[0];
+  }
   static thread_local int configured_dev = -1;
   static thread_local int sm_count = 0;
   int dev = 0;
   TV_CUDA_TRY(cudaGetDevice(&dev));
   if (configured_dev != dev) {
-    TV_CUDA_TRY(cudaFuncSetAttribute(verify_tc_delta_kernel<8>,
+    TV_CUDA_TRY(cudaFuncSetAttribute(verify_tc_delta_kernel<8, false>,
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
-    TV_CUDA_TRY(cudaFuncSetAttribute(verify_tc_delta_kernel<15>,
+    TV_CUDA_TRY(cudaFuncSetAttribute(verify_tc_delta_kernel<15, false>,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
+    TV_CUDA_TRY(cudaFuncSetAttribute(verify_tc_delta_kernel<8, true>,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
+    TV_CUDA_TRY(cudaFuncSetAttribute(verify_tc_delta_kernel<15, true>,
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
     TV_CUDA_TRY(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev));
     configured_dev = dev;
@@ -527,13 +655,20 @@ int tv_launch_verify_tc_delta(const VerifyArgs& a, int32_t* status, cudaStream_t
   p.beta = a.beta;
   p.want_U = a.U != nullptr;
   p.status = status;
+  p.offsets = a.tree.offsets;
+  p.capacity = a.tree.capacity;
+  p.O = a.O;
+  p.U = Uout;
   const int grid = (int)(items < (uint64_t)sm_count ? items : (uint64_t)sm_count);
-  if (a.tree.max_depth_all <= 8)
-    TV_CUDA_TRY(launch_dependent(verify_tc_delta_kernel<8>, grid, kThreads, kSmemBytes, stream, ms->map[0],
-                                 ms->map[1], ms->map[2], ms->map[3], ms->map[4], mu->map[0], p));
+  const bool shallow = a.tree.max_depth_all <= 8;
+  auto launch = [&](auto kernel) {
+    return launch_dependent(kernel, grid, kThreads, kSmemBytes, stream, ms->map[0], ms->map[1], ms->map[2],
+                            ms->map[3], mapsO, mapsU, p);
+  };
+  if (packed)
+    TV_CUDA_TRY(shallow ? launch(verify_tc_delta_kernel<8, true>) : launch(verify_tc_delta_kernel<15, true>));
   else
-    TV_CUDA_TRY(launch_dependent(verify_tc_delta_kernel<15>, grid, kThreads, kSmemBytes, stream, ms->map[0],
-                                 ms->map[1], ms->map[2], ms->map[3], ms->map[4], mu->map[0], p));
+    TV_CUDA_TRY(shallow ? launch(verify_tc_delta_kernel<8, false>) : launch(verify_tc_delta_kernel<15, false>));
   TV_CUDA_TRY(cudaGetLastError());
   return TV_OK;
 }

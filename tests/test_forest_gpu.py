@@ -121,23 +121,35 @@ def test_forest_matches_oracle_per_request(case, dtype, rule, impl):
                     assert rel_fro(Sn[l, b, h], Sr) <= tol
 
 
-def test_forest_takes_the_tensor_core_kernel():
-    """Gated rule, bf16, dk = dv = 128: IMPL_TC must accept a packed forest (and the delta rule,
-    which has no packed tensor-core kernel, must decline rather than fall back silently)."""
-    wl = inputs.workload("c2", B=4, H=2, T=64, seed=11)
-    parents, _ = make_forest(4, 64, seed=12)
-    cap = sum(len(p) for p in parents)
+@pytest.mark.parametrize("rule", [inputs.GATED, inputs.DELTA])
+def test_forest_takes_the_tensor_core_kernels(rule):
+    """bf16, dk = dv = 128: IMPL_TC must accept a packed forest for both rules (no silent fallback)
+    and agree with the general kernel."""
+    wl = inputs.workload("c2", B=5, H=2, T=64, rule=rule, seed=11)
+    parents, _ = make_forest(5, 64, seed=12)
+    cap = sum(len(p) for p in parents) + 3
     P, _ = packed_tensors(wl, parents, cap, 2)
     g = {n: (None if t is None else t.to(DEV)) for n, t in P.items()}
     forest = tv.forest_build(parents, n_max=64, capacity=cap).upload()
-    O1 = tv.tree_verify(forest, g["S_pre"], g["q"], g["k"], g["v"], g["alpha"], impl=tv.IMPL_TC)
-    O2 = tv.tree_verify(forest, g["S_pre"], g["q"], g["k"], g["v"], g["alpha"], impl=tv.IMPL_SIMT)
-    torch.cuda.synchronize()
-    assert rel_fro(O1.cpu().double().numpy(), O2.cpu().double().numpy()) < 2e-3
-    with pytest.raises(tv.TreeVerifyError) as e:
-        tv.tree_verify(forest, g["S_pre"], g["q"], g["k"], g["v"], g["alpha"], torch.ones_like(g["alpha"]),
-                       rule=inputs.DELTA, impl=tv.IMPL_TC)
-    assert e.value.status == -3
+    outs = []
+    for impl in (tv.IMPL_TC, tv.IMPL_SIMT):
+        O = torch.zeros(1, 2, cap, 128, device=DEV)
+        U = torch.zeros_like(O)
+        tv.tree_verify(forest, g["S_pre"], g["q"], g["k"], g["v"], g["alpha"], g["beta"], rule=rule, O=O, U=U,
+                       impl=impl)
+        torch.cuda.synchronize()
+        outs.append((O.cpu().double().numpy(), U.cpu().double().numpy()))
+    forest.device_status()
+    assert rel_fro(outs[0][0], outs[1][0]) < 2e-3 and rel_fro(outs[0][1], outs[1][1]) < 2e-3
+    # deeper than the tensor-core delta kernel's path tables: declined, not faked
+    if rule == inputs.DELTA:
+        deep = tv.forest_build([inputs.tree_chain(40)], n_max=64, capacity=64).upload()
+        one = {n: (None if t is None else t[:, :1].contiguous() if n == "S_pre" else t) for n, t in g.items()}
+        with pytest.raises(tv.TreeVerifyError) as e:
+            tv.tree_verify(deep, one["S_pre"], g["q"][:, :, :64].contiguous(), g["k"][:, :, :64].contiguous(),
+                           g["v"][:, :, :64].contiguous(), g["alpha"][:, :, :64].contiguous(),
+                           g["beta"][:, :, :64].contiguous(), rule=rule, impl=tv.IMPL_TC)
+        assert e.value.status == -3
 
 
 def test_forest_metadata_and_rebuild():
