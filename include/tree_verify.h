@@ -293,7 +293,11 @@ int tv_session_free(tv_session* s);
  *   q, k, v            io_dtype        alpha, beta [B][H][T] float
  * x, ctx, weight, bias, q, k, v 16-byte aligned; dk, dv multiples of 8 (bf16) or 4 (float),
  * at most 256; 1 <= W <= TV_CONV_MAX_TAPS; T <= TV_MAX_NODES.  The tree must be
- * uploaded (1 tree shared by all requests, or B trees).  Outputs must not alias
+ * uploaded (1 tree shared by all requests, or B trees).  With a packed forest
+ * (tv_forest_build; T = n_max, B = n_req) the node-indexed tensors are packed
+ * like those of tv_tree_verify: x [capacity][C], gate_a, gate_b [capacity][H]
+ * (row offsets[r] + i = node i of request r), q, k, v [H][capacity][d],
+ * alpha, beta [H][capacity]; ctx keeps [B][W-1][C].  Outputs must not alias
  * inputs.  Asynchronous on `stream`; returns a tv_status, launches nothing on
  * an error. */
 #define TV_CONV_MAX_TAPS 8

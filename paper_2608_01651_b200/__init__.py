@@ -369,8 +369,16 @@ def tree_verify_static(parent, S_pre, q, k, v, alpha, beta=None, *, rule=GATED, 
     return O
 
 
-def _conv_dims(x, H, dk, dv, W, normalize_qk, eps) -> _ConvDims:
+def _conv_dims(x, H, dk, dv, W, normalize_qk, eps, tree=None) -> _ConvDims:
     import torch
+    if tree is not None and tree.capacity is not None:
+        # packed forest: x is [capacity, C]; request count and node limit come from the handle
+        if x.dim() != 2 or x.shape[0] != tree.capacity or x.shape[1] != H * (2 * dk + dv):
+            raise ValueError("packed-forest x must be [capacity, H*(2*dk+dv)]")
+        dt = BF16 if x.dtype == torch.bfloat16 else F32 if x.dtype == torch.float32 else None
+        if dt is None:
+            raise ValueError("x must be float32 or bfloat16")
+        return _ConvDims(tree.n_trees, H, tree.n, dk, dv, W, dt, int(bool(normalize_qk)), float(eps))
     if x.dim() != 3 or x.shape[2] != H * (2 * dk + dv):
         raise ValueError("x must be [B, T, H*(2*dk+dv)]")
     if x.dtype == torch.bfloat16:
@@ -390,12 +398,13 @@ def _conv_args(tree, x, ctx, weight, bias, H, dk, dv, gate_a, gate_b, A_log, dt_
     for t, n in ((weight, "weight"), (bias, "bias"), (A_log, "A_log"), (dt_bias, "dt_bias"),
                  (alpha, "alpha"), (beta, "beta")):
         _require(t, n, torch.float32)
-    if weight.dim() != 2 or weight.shape[0] != x.shape[2]:
+    if weight.dim() != 2 or weight.shape[0] != x.shape[-1]:
         raise ValueError("weight must be [C, W]")
     W = weight.shape[1]
-    if W > 1 and (ctx is None or tuple(ctx.shape) != (x.shape[0], W - 1, x.shape[2])):
+    n_req = tree.n_trees if tree.capacity is not None else x.shape[0]
+    if W > 1 and (ctx is None or tuple(ctx.shape) != (n_req, W - 1, x.shape[-1])):
         raise ValueError("ctx must be [B, W-1, C]")
-    d = _conv_dims(x, H, dk, dv, W, normalize_qk, eps)
+    d = _conv_dims(x, H, dk, dv, W, normalize_qk, eps, tree)
     args = (tree._h, ctypes.byref(d), _ptr(x), _ptr(ctx), _ptr(weight), _ptr(bias), _ptr(gate_a), _ptr(gate_b),
             _ptr(A_log), _ptr(dt_bias), _ptr(q), _ptr(k), _ptr(v), _ptr(alpha), _ptr(beta), _stream_ptr(stream))
     keep = (tree, d, x, ctx, weight, bias, gate_a, gate_b, A_log, dt_bias, q, k, v, alpha, beta)
@@ -411,14 +420,14 @@ def tree_conv(tree: Tree, x, ctx, weight, bias=None, *, H, dk, dv, gate_a=None, 
     ``(q, k, v, alpha, beta)`` when ``gate_a`` is given (``beta`` None without ``gate_b``).
     """
     import torch
-    B, T = x.shape[0], x.shape[1]
-    q = torch.empty(B, H, T, dk, device=x.device, dtype=x.dtype) if q is None else q
-    k = torch.empty(B, H, T, dk, device=x.device, dtype=x.dtype) if k is None else k
-    v = torch.empty(B, H, T, dv, device=x.device, dtype=x.dtype) if v is None else v
+    lead = (H, tree.capacity) if tree.capacity is not None else (x.shape[0], H, x.shape[1])
+    q = torch.empty(*lead, dk, device=x.device, dtype=x.dtype) if q is None else q
+    k = torch.empty(*lead, dk, device=x.device, dtype=x.dtype) if k is None else k
+    v = torch.empty(*lead, dv, device=x.device, dtype=x.dtype) if v is None else v
     if gate_a is not None and alpha is None:
-        alpha = torch.empty(B, H, T, device=x.device, dtype=torch.float32)
+        alpha = torch.empty(*lead, device=x.device, dtype=torch.float32)
     if gate_b is not None and beta is None:
-        beta = torch.empty(B, H, T, device=x.device, dtype=torch.float32)
+        beta = torch.empty(*lead, device=x.device, dtype=torch.float32)
     args, _keep = _conv_args(tree, x, ctx, weight, bias, H, dk, dv, gate_a, gate_b, A_log, dt_bias,
                              normalize_qk, eps, q, k, v, alpha, beta, stream)
     _check(lib().tv_tree_conv(*args), "tv_tree_conv")
@@ -441,7 +450,7 @@ def conv_commit(tree: Tree, accepted, x, ctx, *, H, dk, dv, ctx_new=None, stream
     for t, n in ((x, "x"), (ctx, "ctx"), (ctx_new, "ctx_new")):
         _require(t, n, x.dtype)
     out = ctx if ctx_new is None else ctx_new
-    d = _conv_dims(x, H, dk, dv, ctx.shape[1] + 1, False, 0.0)
+    d = _conv_dims(x, H, dk, dv, ctx.shape[1] + 1, False, 0.0, tree)
     _check(lib().tv_conv_commit(tree._h, ctypes.byref(d), _ptr(accepted), _ptr(x), _ptr(ctx), _ptr(out),
                                 _stream_ptr(stream)), "tv_conv_commit")
     return out

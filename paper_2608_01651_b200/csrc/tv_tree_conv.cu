@@ -27,6 +27,8 @@ constexpr int kMaxConvDim = 256;
 
 struct ConvArgs {
   const int32_t* parent;  // [n_trees][T]
+  const int32_t* offsets; // packed forest: [B + 1] first row of each request (x rows and output planes); else null
+  int32_t capacity;       // packed forest: rows of one output plane
   int32_t n_trees;
   int32_t B, H, T, dk, dv, W, normalize;
   int32_t single;  // one row buffer only (two do not fit): no prefetch of the next item's rows
@@ -155,6 +157,9 @@ __device__ __forceinline__ void cp_async_wait_all() {
 // (cp.async) and the tap table of item n+1 is derived: one __syncthreads per item.
 struct ConvItem {
   int slice, b, kind, h, d, c0;
+  int n;          // node rows of this request
+  int row0;       // first row of the request in x and in the gate inputs
+  size_t orow0;   // first row of this (request, head) in q/k/v and in the gate outputs
 };
 
 template <typename IO, int W, int NJ>
@@ -188,17 +193,32 @@ tree_conv_kernel(const ConvArgs a) {
     it.d = it.kind == 2 ? dv : dk;
     it.c0 = it.kind == 0 ? it.h * dk : it.kind == 1 ? (H + it.h) * dk : 2 * H * dk + it.h * dv;
   };
+  // dense: request b owns rows b*T .. of x and the slab (b, h) of every output; packed forest:
+  // rows offsets[b] .. of x and of every head's plane of `capacity` rows
+  auto set_request = [&](ConvItem& it) {
+    if (a.offsets == nullptr) {
+      it.n = T;
+      it.row0 = it.b * T;
+      it.orow0 = ((size_t)it.b * H + it.h) * T;
+    } else if (it.slice < 3 * H) {
+      it.row0 = a.offsets[it.b];
+      it.n = a.offsets[it.b + 1] - it.row0;
+      it.orow0 = (size_t)it.h * a.capacity + it.row0;
+    }
+  };
   auto advance = [&](ConvItem& it) {
     if (++it.b == B) {
       it.b = 0;
       ++it.slice;
       set_slice(it);
     }
+    set_request(it);
   };
   ConvItem cur;
   cur.slice = first / B;
   cur.b = first - cur.slice * B;
   set_slice(cur);
+  set_request(cur);
   ConvItem nxt = cur;
   advance(nxt);
   int b2 = nxt.b + 1 == B ? 0 : nxt.b + 1;  // request of the item after next
@@ -220,7 +240,7 @@ tree_conv_kernel(const ConvArgs a) {
   };
   auto fetch_rows = [&](const ConvItem& it, int slot) {
     if (it.d != g_d) set_geometry(it.d);
-    const IO* xb = reinterpret_cast<const IO*>(a.x) + (size_t)it.b * T * C + it.c0;
+    const IO* xb = reinterpret_cast<const IO*>(a.x) + (size_t)it.row0 * C + it.c0;
     const IO* cb = reinterpret_cast<const IO*>(a.ctx) + (size_t)it.b * (W - 1) * C + it.c0;
     const uint32_t dctx = xs_u32 + (uint32_t)slot * buf_bytes;
     const uint32_t dx = dctx + (uint32_t)((W - 1) * it.d * sizeof(IO));
@@ -233,7 +253,7 @@ tree_conv_kernel(const ConvArgs a) {
     }
     row = row0;
     cv = cv0;
-    while (row < T) {  // node rows
+    while (row < it.n) {  // node rows
       cp_async16(dx + (uint32_t)((row * it.d + cv * VEC) * sizeof(IO)), xb + (row * C + cv * VEC));
       row += rstep;
       cv += cstep;
@@ -241,7 +261,7 @@ tree_conv_kernel(const ConvArgs a) {
     }
   };
   auto build_taps = [&](const ConvItem& it, int slot) {
-    if (tid < T) {
+    if (tid < it.n) {
       const uint32_t row_bytes = (uint32_t)it.d * sizeof(IO);
       const int32_t* par = par_s + slot * Tp;
       int j = tid, ctx_row = W - 2;
@@ -316,8 +336,8 @@ tree_conv_kernel(const ConvArgs a) {
     }
 
     // ---- gate preparation for this (request, head): done with the q slice
-    if (cur.kind == 0 && a.gate_a != nullptr && tid < T) {
-      const size_t gi = ((size_t)cur.b * T + tid) * H + cur.h, go = ((size_t)cur.b * H + cur.h) * T + tid;
+    if (cur.kind == 0 && a.gate_a != nullptr && tid < cur.n) {
+      const size_t gi = ((size_t)cur.row0 + tid) * H + cur.h, go = cur.orow0 + tid;
       const float ga = to_f32(reinterpret_cast<const IO*>(a.gate_a)[gi]);
       a.alpha[go] = expf(-expf(__ldg(a.A_log + cur.h)) * softplus(ga + __ldg(a.dt_bias + cur.h)));
       if (a.gate_b != nullptr) {
@@ -328,8 +348,8 @@ tree_conv_kernel(const ConvArgs a) {
 
     // ---- each half-warp takes one node row at a time (the last row is repeated, unstored,
     // when T is odd)
-    IO* out = reinterpret_cast<IO*>(cur.kind == 0 ? a.q : cur.kind == 1 ? a.k : a.v) +
-              ((size_t)cur.b * H + cur.h) * T * d;
+    IO* out = reinterpret_cast<IO*>(cur.kind == 0 ? a.q : cur.kind == 1 ? a.k : a.v) + cur.orow0 * d;
+    const int Tn = cur.n;
     const bool norm = want_norm && cur.kind < 2;
     const uint32_t xs_item = xs_u32 + (uint32_t)xs_slot * buf_bytes;
     const uint32_t taps_item = taps_u32 + (uint32_t)(s * T) * (WP * 4);
@@ -340,9 +360,9 @@ tree_conv_kernel(const ConvArgs a) {
       base1[j] = xs_item + off1[j];
     }
 #pragma unroll kConvUnroll
-    for (int i0 = 2 * warp; i0 < T; i0 += 2 * kConvWarps) {
-      const bool row_live = i0 + half < T;
-      const int i = row_live ? i0 + half : T - 1;
+    for (int i0 = 2 * warp; i0 < Tn; i0 += 2 * kConvWarps) {
+      const bool row_live = i0 + half < Tn;
+      const int i = row_live ? i0 + half : Tn - 1;
       uint32_t tap[WP];
       {
         const uint4 t0 = lds16(taps_item + (uint32_t)i * (WP * 4));
@@ -391,16 +411,19 @@ tree_conv_kernel(const ConvArgs a) {
 // ctx_new may be ctx itself.
 template <typename IO, int W>
 __global__ void __launch_bounds__(kConvThreads)
-conv_commit_kernel(const int32_t* __restrict__ parent, int32_t n_trees, const int32_t* __restrict__ accepted,
-                   int32_t T, int32_t C, const IO* x, const IO* ctx, IO* ctx_new) {
+conv_commit_kernel(const int32_t* __restrict__ parent, int32_t n_trees, const int32_t* __restrict__ offsets,
+                   const int32_t* __restrict__ accepted, int32_t T, int32_t C, const IO* x, const IO* ctx,
+                   IO* ctx_new) {
   constexpr int VEC = 16 / (int)sizeof(IO);
   const int b = blockIdx.y;
   const int col = (blockIdx.x * kConvThreads + threadIdx.x) * VEC;
   if (col >= C) return;
   int acc = accepted[b];
-  if (acc >= T) acc = -1;
+  const int row0 = offsets ? offsets[b] : b * T;                     // packed forest: the request's first x row
+  const int nb = offsets ? offsets[b + 1] - offsets[b] : T;
+  if (acc >= nb) acc = -1;
   const int32_t* par = parent + (size_t)(n_trees == 1 ? 0 : b) * T;
-  const IO* xb = x + (size_t)b * T * C + col;
+  const IO* xb = x + (size_t)row0 * C + col;
   const IO* cb = ctx + (size_t)b * (W - 1) * C + col;
   uint4 vals[W > 1 ? W - 1 : 1];
   int j = acc, back = W - 2;
@@ -430,6 +453,7 @@ int check_conv(const tv_tree* t, const tv_conv_dims* d) {
   if ((d->dk & m) || (d->dv & m)) return TV_ERR_UNSUPPORTED;
   if (t->n != d->T) return TV_ERR_BAD_ARG;
   if (t->n_trees != 1 && t->n_trees != d->B) return TV_ERR_BAD_ARG;
+  if (!t->offsets.empty() && t->n_trees != d->B) return TV_ERR_BAD_ARG;
   if ((int64_t)d->B * d->H * 3 > 0x7fffffffLL || d->B > 65535) return TV_ERR_UNSUPPORTED;
   if (!t->uploaded) return TV_ERR_NOT_UPLOADED;
   return TV_OK;
@@ -482,7 +506,7 @@ int launch_conv_commit(const tv_tree* t, const tv_conv_dims* d, const int32_t* a
   constexpr int VEC = 16 / (int)sizeof(IO);
   const int C = d->H * (2 * d->dk + d->dv);
   dim3 grid((unsigned)((C / VEC + kConvThreads - 1) / kConvThreads), (unsigned)d->B);
-  conv_commit_kernel<IO, W><<<grid, kConvThreads, 0, s>>>(t->d_parent, t->n_trees, accepted, d->T, C,
+  conv_commit_kernel<IO, W><<<grid, kConvThreads, 0, s>>>(t->d_parent, t->n_trees, t->d_offsets, accepted, d->T, C,
                                                          (const IO*)x, (const IO*)ctx, (IO*)ctx_new);
   TV_CUDA_TRY(cudaGetLastError());
   return TV_OK;
@@ -528,6 +552,7 @@ TV_API int tv_tree_conv(const tv_tree* tree, const tv_conv_dims* d, const void* 
   if (q == x || k == x || v == x || q == k || q == v || k == v) return TV_ERR_BAD_ARG;
   ConvArgs a;
   a.parent = tree->d_parent; a.n_trees = tree->n_trees;
+  a.offsets = tree->d_offsets; a.capacity = tree->capacity;
   a.B = d->B; a.H = d->H; a.T = d->T; a.dk = d->dk; a.dv = d->dv; a.W = d->W;
   a.normalize = d->normalize_qk != 0; a.eps = d->eps;
   a.x = x; a.ctx = ctx; a.weight = weight; a.bias = bias; a.gate_a = gate_a; a.gate_b = gate_b;

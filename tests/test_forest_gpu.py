@@ -186,3 +186,57 @@ def test_forest_argument_errors():
     dense = tv.tree_build(np.array([[-1, 0]], dtype=np.int32))
     with pytest.raises(tv.TreeVerifyError):
         dense.rebuild_forest([np.array([-1, 0])])
+
+
+@pytest.mark.parametrize("dtype", [inputs.BF16, inputs.F32])
+@pytest.mark.parametrize("W", [2, 4])
+def test_forest_stage1_conv_and_context_commit(dtype, W):
+    """Stage 1 on a packed forest: x rows packed, outputs in the planes the verify kernels read."""
+    from oracle import tree_conv_oracle as cv
+    H, dk, dv, n_max = 3, 64, 40, 48
+    parents, accepted = make_forest(6, n_max, seed=21 + W)
+    B = len(parents)
+    total = sum(len(p) for p in parents)
+    cap = total + 5
+    C = H * (2 * dk + dv)
+    dt = torch.bfloat16 if dtype == inputs.BF16 else torch.float32
+    gen = torch.Generator().manual_seed(7 + W)
+    x = torch.full((cap, C), float("nan")).to(dt)
+    x[:total] = torch.randn(total, C, generator=gen).to(dt)
+    ga = torch.full((cap, H), float("nan")).to(dt)
+    gb = torch.full((cap, H), float("nan")).to(dt)
+    ga[:total] = torch.randn(total, H, generator=gen).to(dt)
+    gb[:total] = torch.randn(total, H, generator=gen).to(dt)
+    ctx = torch.randn(B, W - 1, C, generator=gen).to(dt)
+    weight = torch.randn(C, W, generator=gen) / W ** 0.5
+    bias = 0.1 * torch.randn(C, generator=gen)
+    A_log = -2 + 2.5 * torch.rand(H, generator=gen)
+    dt_bias = -3 + 2 * torch.rand(H, generator=gen)
+    forest = tv.forest_build(parents, n_max=n_max, capacity=cap).upload()
+    out = {n: torch.full((H, cap, d), 9.0, device=DEV, dtype=dt) for n, d in (("q", dk), ("k", dk), ("v", dv))}
+    al = torch.full((H, cap), 9.0, device=DEV)
+    be = torch.full((H, cap), 9.0, device=DEV)
+    tv.tree_conv(forest, x.to(DEV), ctx.to(DEV), weight.to(DEV), bias.to(DEV), H=H, dk=dk, dv=dv,
+                 gate_a=ga.to(DEV), gate_b=gb.to(DEV), A_log=A_log.to(DEV), dt_bias=dt_bias.to(DEV),
+                 normalize_qk=True, q=out["q"], k=out["k"], v=out["v"], alpha=al, beta=be)
+    ctx_new = tv.conv_commit(forest, torch.from_numpy(accepted).to(DEV), x.to(DEV), ctx.to(DEV).clone(),
+                             H=H, dk=dk, dv=dv)
+    torch.cuda.synchronize()
+    rtol, atol = (2.0 ** -8, 2e-6) if dtype == inputs.BF16 else (1e-5, 1e-6)
+    f = inputs.to_f64
+    off = 0
+    for b, par in enumerate(parents):
+        n = len(par)
+        rows = slice(off, off + n)
+        y = cv.tree_conv(f(x[rows]), f(ctx[b]), f(weight), f(bias), par)
+        for name, ref in zip(("q", "k", "v"), cv.split_heads(y, H, dk, dv, normalize_qk=True, eps=1e-6)):
+            got = out[name][:, rows].cpu().double().numpy()
+            assert (np.abs(got - ref) <= rtol * np.abs(ref) + atol).all(), (name, b)
+        ra, rb = cv.gate_prep(f(ga[rows]), f(gb[rows]), f(A_log), f(dt_bias))
+        assert np.allclose(al[:, rows].cpu().double().numpy(), ra, rtol=5e-6)
+        assert np.allclose(be[:, rows].cpu().double().numpy(), rb, rtol=5e-6)
+        ref_ctx = cv.conv_commit(f(x[rows]), f(ctx[b]), par, int(accepted[b]))
+        assert np.array_equal(ctx_new[b].cpu().double().numpy(), ref_ctx)
+        off += n
+    for t in list(out.values()) + [al, be]:
+        assert bool((t[:, total:] == 9.0).all())      # rows past the forest untouched
