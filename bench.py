@@ -380,6 +380,27 @@ def run_packed(args, wl, local_rank):
     ms = t0.elapsed_time(t1) / args.steps
     v_ms = float(np.mean([a.elapsed_time(b) for a, b, _ in used])) / wl.L
     c_ms = float(np.mean([b.elapsed_time(c) for _, b, c in used]))
+    # ---- the budget selector that would produce such a forest on the GPU, timed on its own:
+    # candidates = the full trees, synthetic draft probabilities, budget = the packed node count
+    cand = torch.from_numpy(np.ascontiguousarray(
+        np.stack([parents[b if parents.shape[0] > 1 else 0] for b in range(wl.B)]), dtype=np.int32)).to(dev)
+    cand[:, 0] = -1
+    probs = torch.rand(wl.B, wl.T, device=dev) * 0.9 + 0.1
+    sel_forest = tv.forest_build([np.array([-1], dtype=np.int32)] * wl.B, n_max=wl.T, capacity=cap)
+    for _ in range(3):
+        sel = tv.budget_select(cand, probs, total, stream=stream)
+        sel_forest.upload_device(sel["parent_packed"], sel["offsets"], max_depth_bound=wl.T - 1, stream=stream)
+    torch.cuda.synchronize()
+    s0, s1 = ev(), ev()
+    n_sel = 50
+    s0.record(stream)
+    for _ in range(n_sel):
+        sel = tv.budget_select(cand, probs, total, stream=stream)
+        sel_forest.upload_device(sel["parent_packed"], sel["offsets"], max_depth_bound=wl.T - 1, stream=stream)
+    s1.record(stream)
+    torch.cuda.synchronize()
+    sel_ms = s0.elapsed_time(s1) / n_sel
+
     peak, peak_kind = measured_peak()
     vbytes = (wl.B * wl.H * 4 * wl.dk * wl.dv
               + wl.H * total * (eb * (2 * wl.dk + wl.dv) + 4 + (4 if delta else 0) + 4 * wl.dv * (2 if delta else 1)))
@@ -396,6 +417,8 @@ def run_packed(args, wl, local_rank):
         "verify": {"ms_per_layer": v_ms, "nodes_per_s_per_layer": total / (v_ms * 1e-3), "bytes": vbytes,
                    "algorithmic_GBps": v_gbs, "frac_of_measured_copy": v_gbs / peak},
         "commit": {"ms": c_ms},
+        "selector": {"ms": sel_ms, "launches": 4, "candidates": wl.B * wl.T, "budget": total,
+                     "what": "tv_budget_select (3 kernels) + tv_forest_upload_device (1 kernel), no host sync"},
         "roofline": {"kernel": "tree_verify (packed)", "bound": "hbm", "achieved": v_gbs, "peak": peak,
                      "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": v_gbs / peak, "traffic": None},
         "cpu_baseline": None, "e2e": None, "gpu_launches": args.steps * (wl.L + 2), "clocks": clocks,

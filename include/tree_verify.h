@@ -171,6 +171,41 @@ int tv_forest_build(const int32_t* parent_flat /*host*/, const int32_t* offsets 
 int tv_forest_rebuild(tv_tree* forest, const int32_t* parent_flat /*host*/,
                       const int32_t* offsets /*host*/);
 
+/* ---- batch-wide utility allocation (Section V-A "Batch-wide utility
+ * allocation") and device-side forest materialisation (Section V-B) ----------
+ * Every request brings a candidate tree of n_cand <= TV_MAX_NODES nodes (node 0
+ * = the tree's root, parent -1; -1 <= parent[i] < i) and the drafter's
+ * conditional probability p_draft of every node, 0 <= p <= 1.  tv_budget_select
+ * scores node v by rho(v) = rho(parent(v)) * p_draft(v) (float32, one rounding
+ * per edge; rho of a root child is its own p), keeps the root of every tree
+ * and, of all other nodes of the batch, the budget - n_req highest rho (ties:
+ * lower (request, node) index first), and packs the kept nodes request by
+ * request in their original order:
+ *   rho           float [n_req][n_cand]
+ *   counts        int32 [n_req]     kept nodes per request (the budget q_r)
+ *   offsets       int32 [n_req+1]   prefix sums of counts
+ *   parent_packed int32 [n_req][n_cand]  parents renumbered locally, padded with -1
+ *   node_id       int32 [budget]    r * n_cand + i of every packed row, -1 past the forest
+ * All pointers are DEVICE pointers (4-byte aligned; workspace 16-byte aligned,
+ * tv_budget_workspace_bytes(n_req, n_cand) bytes); nothing is allocated and the
+ * host is not synchronised.  *status (device int32, may be NULL) receives
+ * TV_ERR_INVALID_TREE if a parent is out of range (it is then treated as -1).
+ * n_req <= 1024, n_req <= budget.  parent_packed and offsets are exactly what
+ * tv_forest_upload_device reads: it derives the masks and depths of a forest
+ * handle (tv_forest_build with the same n_req, n_max = n_cand, capacity >=
+ * budget) from DEVICE memory, with no host copy.  max_depth_bound must bound the
+ * depth of every candidate tree (kernel choice depends on it; a wrong bound
+ * gives wrong results).  After it the handle's host-side metadata is stale:
+ * tv_tree_meta and tv_tree_path return TV_ERR_UNSUPPORTED until the next
+ * tv_forest_rebuild + tv_tree_upload.                                          */
+size_t tv_budget_workspace_bytes(int32_t n_req, int32_t n_cand);
+int tv_budget_select(const int32_t* parent /*dev*/, const float* p_draft /*dev*/, int32_t n_req,
+                     int32_t n_cand, int32_t budget, float* rho, int32_t* counts, int32_t* offsets,
+                     int32_t* parent_packed, int32_t* node_id, void* workspace, int32_t* status,
+                     void* stream);
+int tv_forest_upload_device(tv_tree* forest, const int32_t* parent_padded /*dev*/,
+                            const int32_t* offsets /*dev*/, int32_t max_depth_bound, void* stream);
+
 /* ---- verification (Section IV-A Theorem 1, Eq. 2; Eq. 4; Lemma 2 Eq. 5) ----
  *
  * For every layer, request, head and node i:

@@ -62,6 +62,12 @@ def lib() -> ctypes.CDLL:
     L.tv_tree_rebuild.argtypes = [vp, vp]
     L.tv_forest_build.argtypes = [vp, vp, i32, i32, i32, p(vp)]
     L.tv_forest_rebuild.argtypes = [vp, vp, vp]
+    L.tv_budget_workspace_bytes.argtypes = [i32, i32]
+    L.tv_budget_workspace_bytes.restype = ctypes.c_size_t
+    L.tv_budget_select.argtypes = [vp, vp, i32, i32, i32] + [vp] * 8
+    L.tv_budget_select.restype = ctypes.c_int
+    L.tv_forest_upload_device.argtypes = [vp, vp, vp, i32, vp]
+    L.tv_forest_upload_device.restype = ctypes.c_int
     L.tv_forest_build.restype = ctypes.c_int
     L.tv_forest_rebuild.restype = ctypes.c_int
     L.tv_tree_meta.argtypes = [vp, vp, vp, vp]
@@ -185,6 +191,16 @@ class Tree:
                 raise TreeVerifyError(st, "tv_tree_rebuild/tv_tree_upload")
         return refresh
 
+    def upload_device(self, parent_padded, offsets, max_depth_bound, stream=None):
+        """``tv_forest_upload_device``: metadata from CUDA int32 tensors (as ``budget_select`` leaves
+        them); the host-side metadata of the handle is stale afterwards."""
+        import torch
+        _require(parent_padded, "parent_padded", torch.int32)
+        _require(offsets, "offsets", torch.int32)
+        _check(lib().tv_forest_upload_device(self._h, _ptr(parent_padded), _ptr(offsets), int(max_depth_bound),
+                                             _stream_ptr(stream)), "tv_forest_upload_device")
+        return self
+
     def prepare_refresh_forest(self, parent_flat, offsets, stream=None):
         """``tv_forest_rebuild`` + ``tv_tree_upload`` with pre-marshalled arguments; the caller
         updates the two int32 arrays in place between calls."""
@@ -247,6 +263,29 @@ def forest_build(parents, n_max=None, capacity=None) -> Tree:
     t = Tree(h, len(parts), n_max)
     t.offsets, t.capacity = offsets, capacity
     return t
+
+
+def budget_select(parent, p_draft, budget, *, status=None, stream=None):
+    """``tv_budget_select``: ``parent`` int32 and ``p_draft`` float32 CUDA tensors [B, Tc].  Returns a
+    dict of CUDA tensors: rho, counts, offsets, parent_packed, node_id."""
+    import torch
+    _require(parent, "parent", torch.int32)
+    _require(p_draft, "p_draft", torch.float32)
+    _require(status, "status", torch.int32)
+    B, Tc = parent.shape
+    dev = parent.device
+    out = {"rho": torch.empty(B, Tc, device=dev, dtype=torch.float32),
+           "counts": torch.empty(B, device=dev, dtype=torch.int32),
+           "offsets": torch.empty(B + 1, device=dev, dtype=torch.int32),
+           "parent_packed": torch.empty(B, Tc, device=dev, dtype=torch.int32),
+           "node_id": torch.empty(int(budget), device=dev, dtype=torch.int32)}
+    ws = torch.empty(lib().tv_budget_workspace_bytes(B, Tc), device=dev, dtype=torch.uint8)
+    _check(lib().tv_budget_select(_ptr(parent), _ptr(p_draft), B, Tc, int(budget), _ptr(out["rho"]),
+                                  _ptr(out["counts"]), _ptr(out["offsets"]), _ptr(out["parent_packed"]),
+                                  _ptr(out["node_id"]), _ptr(ws), _ptr(status), _stream_ptr(stream)),
+           "tv_budget_select")
+    out["_workspace"] = ws   # keep it alive until the stream has run the kernels
+    return out
 
 
 def _stream_ptr(stream):

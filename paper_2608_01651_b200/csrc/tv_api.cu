@@ -67,6 +67,7 @@ static int fill_tree(tv_tree* t, const int32_t* parent) {
   std::memcpy(t->parent.data(), parent, sizeof(int32_t) * (size_t)t->n_trees * n);
   t->max_depth_all = md_all;
   t->uploaded = false;
+  t->host_meta_valid = true;
   return TV_OK;
 }
 
@@ -166,6 +167,7 @@ TV_API int tv_forest_rebuild(tv_tree* t, const int32_t* parent_flat, const int32
 
 TV_API int tv_tree_meta(const tv_tree* t, uint64_t* anc, int32_t* depth, int32_t* max_depth) {
   if (!t) return TV_ERR_BAD_ARG;
+  if (!t->host_meta_valid) return TV_ERR_UNSUPPORTED;   // topology came from the device
   if (anc) std::memcpy(anc, t->anc.data(), t->anc.size() * sizeof(uint64_t));
   if (depth) std::memcpy(depth, t->depth.data(), t->depth.size() * sizeof(int32_t));
   if (max_depth) std::memcpy(max_depth, t->max_depth.data(), t->max_depth.size() * sizeof(int32_t));
@@ -183,6 +185,7 @@ TV_API int tv_tree_info(const tv_tree* t, int32_t* n_trees, int32_t* n, int32_t*
 TV_API int tv_tree_path(const tv_tree* t, const int32_t* accepted, int32_t n_req, int32_t* path,
                  int32_t path_stride, int32_t* len) {
   if (!t || !accepted || !path || !len || n_req < 0) return TV_ERR_BAD_ARG;
+  if (!t->host_meta_valid) return TV_ERR_UNSUPPORTED;   // topology came from the device
   if (path_stride < t->max_depth_all + 1) return TV_ERR_BAD_ARG;
   if (t->n_trees != 1 && n_req > t->n_trees) return TV_ERR_BAD_ARG;
   for (int r = 0; r < n_req; ++r)
@@ -208,48 +211,64 @@ TV_API int tv_tree_path(const tv_tree* t, const int32_t* accepted, int32_t n_req
   return TV_OK;
 }
 
-TV_API int tv_tree_upload(tv_tree* t, void* stream) {
-  if (!t) return TV_ERR_BAD_ARG;
+// Device mirror of the metadata (masks | depths | parents | offsets | status word) and the two
+// pinned staging slots; allocated by the first upload, reused by every later one.
+struct BlobLayout {
+  size_t anc_b, i32_b, off_b, total, slot_b;
+};
+static BlobLayout blob_layout(const tv_tree* t) {
+  BlobLayout L;
   const size_t nn = (size_t)t->n_trees * t->n;
-  const size_t anc_b = nn * 2 * sizeof(uint64_t), i32_b = nn * sizeof(int32_t);
-  const size_t off_b = t->offsets.empty() ? 0 : ((t->offsets.size() * sizeof(int32_t) + 15) & ~(size_t)15);
-  const size_t meta_b = anc_b + 2 * i32_b + off_b;
-  const size_t total = ((meta_b + 15) & ~(size_t)15) + 16;  // + status word
-  const size_t slot_b = (i32_b + off_b + 255) & ~(size_t)255;  // one staged copy of parents (+ offsets)
+  L.anc_b = nn * 2 * sizeof(uint64_t);
+  L.i32_b = nn * sizeof(int32_t);
+  L.off_b = t->offsets.empty() ? 0 : ((t->offsets.size() * sizeof(int32_t) + 15) & ~(size_t)15);
+  const size_t meta_b = L.anc_b + 2 * L.i32_b + L.off_b;
+  L.total = ((meta_b + 15) & ~(size_t)15) + 16;                 // + status word
+  L.slot_b = (L.i32_b + L.off_b + 255) & ~(size_t)255;          // one staged copy of parents (+ offsets)
+  return L;
+}
+static int ensure_device(tv_tree* t, const BlobLayout& L) {
   int dev = 0;
   TV_CUDA_TRY(cudaGetDevice(&dev));
-  if (t->d_blob && (t->device != dev || t->blob_bytes != total)) return TV_ERR_BAD_ARG;
-  if (!t->d_blob) {
-    TV_CUDA_TRY(cudaMalloc(&t->d_blob, total));
-    cudaError_t e = cudaHostAlloc(&t->h_stage, 2 * slot_b, cudaHostAllocMapped);
-    void* mapped = nullptr;
-    if (e == cudaSuccess) e = cudaHostGetDevicePointer(&mapped, t->h_stage, 0);
-    for (int i = 0; i < 2 && e == cudaSuccess; ++i)
-      e = cudaEventCreateWithFlags(&t->staged[i], cudaEventDisableTiming);
-    if (e != cudaSuccess) {
-      cudaFree(t->d_blob);
-      t->d_blob = nullptr;
-      if (t->h_stage) cudaFreeHost(t->h_stage);
-      t->h_stage = nullptr;
-      tv_set_cuda_error(e);
-      return TV_ERR_CUDA;
-    }
-    t->h_stage_dev = (const int32_t*)mapped;
-    t->blob_bytes = total;
-    t->device = dev;
-    char* base = (char*)t->d_blob;
-    t->d_anc_w = (uint64_t*)base;
-    t->d_depth_w = (int32_t*)(base + anc_b);
-    t->d_parent_w = (int32_t*)(base + anc_b + i32_b);
-    t->d_anc = t->d_anc_w;
-    t->d_depth = t->d_depth_w;
-    t->d_parent = t->d_parent_w;
-    t->d_status = (int32_t*)(base + total - 16);
-    if (off_b) {
-      t->d_offsets_w = (int32_t*)(base + anc_b + 2 * i32_b);
-      t->d_offsets = t->d_offsets_w;
-    }
+  if (t->d_blob && (t->device != dev || t->blob_bytes != L.total)) return TV_ERR_BAD_ARG;
+  if (t->d_blob) return TV_OK;
+  TV_CUDA_TRY(cudaMalloc(&t->d_blob, L.total));
+  cudaError_t e = cudaHostAlloc(&t->h_stage, 2 * L.slot_b, cudaHostAllocMapped);
+  void* mapped = nullptr;
+  if (e == cudaSuccess) e = cudaHostGetDevicePointer(&mapped, t->h_stage, 0);
+  for (int i = 0; i < 2 && e == cudaSuccess; ++i)
+    e = cudaEventCreateWithFlags(&t->staged[i], cudaEventDisableTiming);
+  if (e != cudaSuccess) {
+    cudaFree(t->d_blob);
+    t->d_blob = nullptr;
+    if (t->h_stage) cudaFreeHost(t->h_stage);
+    t->h_stage = nullptr;
+    tv_set_cuda_error(e);
+    return TV_ERR_CUDA;
   }
+  t->h_stage_dev = (const int32_t*)mapped;
+  t->blob_bytes = L.total;
+  t->device = dev;
+  char* base = (char*)t->d_blob;
+  t->d_anc_w = (uint64_t*)base;
+  t->d_depth_w = (int32_t*)(base + L.anc_b);
+  t->d_parent_w = (int32_t*)(base + L.anc_b + L.i32_b);
+  t->d_anc = t->d_anc_w;
+  t->d_depth = t->d_depth_w;
+  t->d_parent = t->d_parent_w;
+  t->d_status = (int32_t*)(base + L.total - 16);
+  if (L.off_b) {
+    t->d_offsets_w = (int32_t*)(base + L.anc_b + 2 * L.i32_b);
+    t->d_offsets = t->d_offsets_w;
+  }
+  return TV_OK;
+}
+
+TV_API int tv_tree_upload(tv_tree* t, void* stream) {
+  if (!t) return TV_ERR_BAD_ARG;
+  const BlobLayout L = blob_layout(t);
+  int st = ensure_device(t, L);
+  if (st != TV_OK) return st;
   cudaStream_t s = (cudaStream_t)stream;
   // The parent arrays go into one of two pinned slots; a small kernel reads the slot over the
   // bus and derives masks and depths on the device (no copy-engine hop in front of the verify
@@ -257,18 +276,38 @@ TV_API int tv_tree_upload(tv_tree* t, void* stream) {
   const int slot = t->stage_slot;
   t->stage_slot ^= 1;
   TV_CUDA_TRY(cudaEventSynchronize(t->staged[slot]));
-  std::memcpy((char*)t->h_stage + slot * slot_b, t->parent.data(), i32_b);
+  std::memcpy((char*)t->h_stage + slot * L.slot_b, t->parent.data(), L.i32_b);
   const int32_t* off_mapped = nullptr;
-  if (off_b) {
-    std::memcpy((char*)t->h_stage + slot * slot_b + i32_b, t->offsets.data(), t->offsets.size() * sizeof(int32_t));
-    off_mapped = (const int32_t*)((const char*)t->h_stage_dev + slot * slot_b + i32_b);
+  if (L.off_b) {
+    std::memcpy((char*)t->h_stage + slot * L.slot_b + L.i32_b, t->offsets.data(),
+                t->offsets.size() * sizeof(int32_t));
+    off_mapped = (const int32_t*)((const char*)t->h_stage_dev + slot * L.slot_b + L.i32_b);
   }
-  int st = tv_launch_tree_meta((const int32_t*)((const char*)t->h_stage_dev + slot * slot_b), t->n_trees,
-                               t->n, t->d_anc_w, t->d_depth_w, t->d_parent_w, t->d_status, off_mapped,
-                               t->d_offsets_w, s);
+  st = tv_launch_tree_meta((const int32_t*)((const char*)t->h_stage_dev + slot * L.slot_b), t->n_trees, t->n,
+                           t->d_anc_w, t->d_depth_w, t->d_parent_w, t->d_status, off_mapped, t->d_offsets_w, s);
   if (st != TV_OK) return st;
   TV_CUDA_TRY(cudaEventRecord(t->staged[slot], s));
   t->uploaded = true;
+  t->host_meta_valid = true;
+  return TV_OK;
+}
+
+// The same metadata from DEVICE-resident parents and offsets (as tv_budget_select leaves them):
+// no host copy, no synchronisation.  The host-side metadata of the handle is then stale.
+TV_API int tv_forest_upload_device(tv_tree* t, const int32_t* parent_padded, const int32_t* offsets,
+                                   int32_t max_depth_bound, void* stream) {
+  if (!t || !parent_padded || !offsets || t->offsets.empty()) return TV_ERR_BAD_ARG;
+  if (max_depth_bound < 0 || max_depth_bound >= t->n) return TV_ERR_BAD_ARG;
+  if (((uintptr_t)parent_padded | (uintptr_t)offsets) & 3) return TV_ERR_BAD_ARG;
+  const BlobLayout L = blob_layout(t);
+  int st = ensure_device(t, L);
+  if (st != TV_OK) return st;
+  st = tv_launch_tree_meta(parent_padded, t->n_trees, t->n, t->d_anc_w, t->d_depth_w, t->d_parent_w, t->d_status,
+                           offsets, t->d_offsets_w, (cudaStream_t)stream);
+  if (st != TV_OK) return st;
+  t->max_depth_all = max_depth_bound;
+  t->uploaded = true;
+  t->host_meta_valid = false;
   return TV_OK;
 }
 

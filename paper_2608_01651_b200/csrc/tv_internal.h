@@ -25,6 +25,7 @@ struct tv_tree {
   int32_t* d_parent_w = nullptr;
   int32_t* d_status = nullptr;  // device status word (0 = ok), cleared by every upload
   bool uploaded = false;
+  bool host_meta_valid = true;   // false after tv_forest_upload_device: the topology lives on the device only
   // Packed forest (tv_forest_build): tree t has offsets[t+1] - offsets[t] <= n real nodes (its
   // metadata slab is padded to n with root children) and its tensor rows start at offsets[t] in
   // every (layer, head) plane of `capacity` rows.  Empty for a dense tree set.

@@ -15,7 +15,12 @@ tree_meta_kernel(const int32_t* __restrict__ parent, int32_t n, uint64_t* __rest
   // a verify kernel launched behind this one may be scheduled now and set itself up; it waits
   // for this grid to finish before it reads global memory
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  if (i < n) par_s[i] = parent[(size_t)t * n + i];
+  if (i < n) {
+    // host-built trees are validated there; device-built ones (tv_forest_upload_device) are not:
+    // an out-of-range parent is treated as a child of the virtual root so the walk stays in bounds
+    const int p = parent[(size_t)t * n + i];
+    par_s[i] = (p < -1 || p >= i) ? -1 : p;
+  }
   if (t == 0 && i == 0) *status = 0;
   // packed forest: the row offsets travel with the parents (tree t copies entry t, the last
   // tree also the end marker)
