@@ -18,6 +18,7 @@ algorithmic HBM GB/s of the verify kernel against the measured copy peak;
 from __future__ import annotations
 
 import argparse
+import dataclasses
 import json
 import os
 import subprocess
@@ -387,15 +388,16 @@ def run_packed(args, wl, local_rank):
     cand[:, 0] = -1
     probs = torch.rand(wl.B, wl.T, device=dev) * 0.9 + 0.1
     sel_forest = tv.forest_build([np.array([-1], dtype=np.int32)] * wl.B, n_max=wl.T, capacity=cap)
+    sel = None
     for _ in range(3):
-        sel = tv.budget_select(cand, probs, total, stream=stream)
+        sel = tv.budget_select(cand, probs, total, stream=stream, out=sel)
         sel_forest.upload_device(sel["parent_packed"], sel["offsets"], max_depth_bound=wl.T - 1, stream=stream)
     torch.cuda.synchronize()
     s0, s1 = ev(), ev()
     n_sel = 50
     s0.record(stream)
     for _ in range(n_sel):
-        sel = tv.budget_select(cand, probs, total, stream=stream)
+        sel = tv.budget_select(cand, probs, total, stream=stream, out=sel)
         sel_forest.upload_device(sel["parent_packed"], sel["offsets"], max_depth_bound=wl.T - 1, stream=stream)
     s1.record(stream)
     torch.cuda.synchronize()

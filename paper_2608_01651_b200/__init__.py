@@ -265,15 +265,24 @@ def forest_build(parents, n_max=None, capacity=None) -> Tree:
     return t
 
 
-def budget_select(parent, p_draft, budget, *, status=None, stream=None):
+def budget_select(parent, p_draft, budget, *, status=None, stream=None, out=None):
     """``tv_budget_select``: ``parent`` int32 and ``p_draft`` float32 CUDA tensors [B, Tc].  Returns a
-    dict of CUDA tensors: rho, counts, offsets, parent_packed, node_id."""
+    dict of CUDA tensors: rho, counts, offsets, parent_packed, node_id (``out``: the dict of an
+    earlier call with the same sizes, to reuse its tensors)."""
     import torch
     _require(parent, "parent", torch.int32)
     _require(p_draft, "p_draft", torch.float32)
     _require(status, "status", torch.int32)
     B, Tc = parent.shape
     dev = parent.device
+    if out is not None:
+        if out["node_id"].numel() != int(budget) or tuple(out["rho"].shape) != (B, Tc):
+            raise ValueError("out does not match these sizes")
+        _check(lib().tv_budget_select(_ptr(parent), _ptr(p_draft), B, Tc, int(budget), _ptr(out["rho"]),
+                                      _ptr(out["counts"]), _ptr(out["offsets"]), _ptr(out["parent_packed"]),
+                                      _ptr(out["node_id"]), _ptr(out["_workspace"]), _ptr(status),
+                                      _stream_ptr(stream)), "tv_budget_select")
+        return out
     out = {"rho": torch.empty(B, Tc, device=dev, dtype=torch.float32),
            "counts": torch.empty(B, device=dev, dtype=torch.int32),
            "offsets": torch.empty(B + 1, device=dev, dtype=torch.int32),
