@@ -112,3 +112,76 @@ def test_gpu_resident_round(rule):
             assert rel_l2_rows(On[h, rows], Or) <= 2e-3
             assert rel_l2_rows(Un[h, rows], Ur) <= 2e-3
             assert rel_fro(Snn[b, h], Sr) <= 2e-3
+
+
+def test_round_replays_from_a_cuda_graph_with_a_new_topology():
+    """Section V-B: fixed addresses and kernel shapes, topology and node allocation change from
+    round to round.  One round (select -> metadata -> verify -> commit) is captured once and
+    replayed after the candidate trees, the probabilities and the tensors changed in place; the
+    replay must equal an ordinary run on the new inputs."""
+    B, H, Tc, budget = 8, 2, 64, 300
+    wl = inputs.workload("c2", B=B, H=H, T=Tc, seed=31)
+    forest = tv.forest_build([np.array([-1], dtype=np.int32)] * B, n_max=Tc, capacity=budget)
+    par_d = torch.empty(B, Tc, dtype=torch.int32, device=DEV)
+    p_d = torch.empty(B, Tc, dtype=torch.float32, device=DEV)
+    planes = {"q": torch.empty(H, budget, 128, device=DEV, dtype=torch.bfloat16)}
+    planes["k"] = torch.empty_like(planes["q"])
+    planes["v"] = torch.empty_like(planes["q"])
+    planes["alpha"] = torch.empty(H, budget, device=DEV)
+    S = torch.empty(B, H, 128, 128, device=DEV)
+    S_new = torch.empty_like(S)
+    O = torch.empty(H, budget, 128, device=DEV)
+    acc = torch.zeros(B, dtype=torch.int32, device=DEV)      # node 0 (the root) of every request
+    sel = None
+
+    def load_inputs(seed):
+        par, p = candidates(B, Tc, seed=seed)
+        par_d.copy_(torch.from_numpy(par)); p_d.copy_(torch.from_numpy(p))
+        t = inputs.make_tensors(inputs.workload("c2", B=B, H=H, T=Tc, seed=seed))
+        S.copy_(t["S_pre"])
+        for n in ("q", "k", "v", "alpha"):     # candidate tensors land in the packed planes below
+            planes[n].zero_()
+        return par, p, t
+
+    def round_(stream):
+        nonlocal sel
+        sel = tv.budget_select(par_d, p_d, budget, stream=stream, out=sel)
+        forest.upload_device(sel["parent_packed"], sel["offsets"], max_depth_bound=8, stream=stream)
+        tv.tree_verify(forest, S, planes["q"], planes["k"], planes["v"], planes["alpha"], O=O, stream=stream)
+        tv.commit_path(forest, acc, S, planes["k"], planes["v"], planes["alpha"], S_new=S_new, stream=stream)
+
+    def fill_planes(par, p, t):
+        ref = bo.select(par, p, budget)
+        ids = torch.from_numpy(ref["node_id"][:int(ref["offsets"][-1])].astype(np.int64)).to(DEV)
+        n = ids.numel()
+        for name in ("q", "k", "v", "alpha"):
+            x = t[name].to(DEV)
+            flat = x.transpose(0, 1).reshape(H, B * Tc, *x.shape[3:])
+            planes[name][:, :n] = flat.index_select(1, ids)
+
+    stream = torch.cuda.Stream()
+    # warm-up outside the capture: allocations, attribute calls and tensor-map encodes happen here
+    par, p, t = load_inputs(101)
+    fill_planes(par, p, t)
+    with torch.cuda.stream(stream):
+        round_(stream)
+    stream.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=stream):
+        round_(stream)
+    # new round: other trees, probabilities and tensors at the same addresses
+    par, p, t = load_inputs(202)
+    fill_planes(par, p, t)
+    torch.cuda.synchronize()
+    graph.replay()
+    torch.cuda.synchronize()
+    O_graph, S_graph, off_graph = O.clone(), S_new.clone(), sel["offsets"].clone()
+    O.zero_(); S_new.zero_()
+    with torch.cuda.stream(stream):
+        round_(stream)
+    stream.synchronize()
+    assert torch.equal(off_graph, sel["offsets"])
+    n = int(off_graph[-1].item())
+    assert torch.equal(O_graph[:, :n], O[:, :n]) and torch.equal(S_graph, S_new)
+    ref = bo.select(par, p, budget)
+    assert np.array_equal(off_graph.cpu().numpy(), ref["offsets"])
