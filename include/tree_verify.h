@@ -342,6 +342,11 @@ typedef struct tv_conv_dims {
   int32_t io_dtype;      /* tv_dtype of x, ctx, gate_a, gate_b, q, k, v  */
   int32_t normalize_qk;  /* 0 / 1                                        */
   float eps;             /* added under the square root                  */
+  int32_t impl;          /* TV_IMPL_AUTO / TV_IMPL_SIMT: the CUDA-core kernel.
+                            TV_IMPL_TC: a variant with the taps as mma.sync tiles
+                            (filter split into three bf16 pieces), for bf16 heads
+                            of 128 channels and W <= 4 only (TV_ERR_UNSUPPORTED
+                            otherwise); measured slower, kept for comparison  */
 } tv_conv_dims;
 
 int tv_tree_conv(const tv_tree* tree, const tv_conv_dims* dims, const void* x, const void* ctx,

@@ -40,7 +40,8 @@ class _Dims(ctypes.Structure):
 
 class _ConvDims(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in
-                ("B", "H", "T", "dk", "dv", "W", "io_dtype", "normalize_qk")] + [("eps", ctypes.c_float)]
+                ("B", "H", "T", "dk", "dv", "W", "io_dtype", "normalize_qk")] + [("eps", ctypes.c_float),
+                                                                                   ("impl", ctypes.c_int32)]
 
 
 def lib() -> ctypes.CDLL:
@@ -417,7 +418,7 @@ def tree_verify_static(parent, S_pre, q, k, v, alpha, beta=None, *, rule=GATED, 
     return O
 
 
-def _conv_dims(x, H, dk, dv, W, normalize_qk, eps, tree=None) -> _ConvDims:
+def _conv_dims(x, H, dk, dv, W, normalize_qk, eps, tree=None, impl=IMPL_AUTO) -> _ConvDims:
     import torch
     if tree is not None and tree.capacity is not None:
         # packed forest: x is [capacity, C]; request count and node limit come from the handle
@@ -426,7 +427,7 @@ def _conv_dims(x, H, dk, dv, W, normalize_qk, eps, tree=None) -> _ConvDims:
         dt = BF16 if x.dtype == torch.bfloat16 else F32 if x.dtype == torch.float32 else None
         if dt is None:
             raise ValueError("x must be float32 or bfloat16")
-        return _ConvDims(tree.n_trees, H, tree.n, dk, dv, W, dt, int(bool(normalize_qk)), float(eps))
+        return _ConvDims(tree.n_trees, H, tree.n, dk, dv, W, dt, int(bool(normalize_qk)), float(eps), int(impl))
     if x.dim() != 3 or x.shape[2] != H * (2 * dk + dv):
         raise ValueError("x must be [B, T, H*(2*dk+dv)]")
     if x.dtype == torch.bfloat16:
@@ -435,11 +436,11 @@ def _conv_dims(x, H, dk, dv, W, normalize_qk, eps, tree=None) -> _ConvDims:
         dt = F32
     else:
         raise ValueError("x must be float32 or bfloat16")
-    return _ConvDims(x.shape[0], H, x.shape[1], dk, dv, W, dt, int(bool(normalize_qk)), float(eps))
+    return _ConvDims(x.shape[0], H, x.shape[1], dk, dv, W, dt, int(bool(normalize_qk)), float(eps), int(impl))
 
 
 def _conv_args(tree, x, ctx, weight, bias, H, dk, dv, gate_a, gate_b, A_log, dt_bias, normalize_qk, eps,
-               q, k, v, alpha, beta, stream):
+               q, k, v, alpha, beta, stream, impl=IMPL_AUTO):
     import torch
     for t, n in ((x, "x"), (ctx, "ctx"), (gate_a, "gate_a"), (gate_b, "gate_b"), (q, "q"), (k, "k"), (v, "v")):
         _require(t, n, x.dtype)
@@ -452,7 +453,7 @@ def _conv_args(tree, x, ctx, weight, bias, H, dk, dv, gate_a, gate_b, A_log, dt_
     n_req = tree.n_trees if tree.capacity is not None else x.shape[0]
     if W > 1 and (ctx is None or tuple(ctx.shape) != (n_req, W - 1, x.shape[-1])):
         raise ValueError("ctx must be [B, W-1, C]")
-    d = _conv_dims(x, H, dk, dv, W, normalize_qk, eps, tree)
+    d = _conv_dims(x, H, dk, dv, W, normalize_qk, eps, tree, impl)
     args = (tree._h, ctypes.byref(d), _ptr(x), _ptr(ctx), _ptr(weight), _ptr(bias), _ptr(gate_a), _ptr(gate_b),
             _ptr(A_log), _ptr(dt_bias), _ptr(q), _ptr(k), _ptr(v), _ptr(alpha), _ptr(beta), _stream_ptr(stream))
     keep = (tree, d, x, ctx, weight, bias, gate_a, gate_b, A_log, dt_bias, q, k, v, alpha, beta)
@@ -461,7 +462,7 @@ def _conv_args(tree, x, ctx, weight, bias, H, dk, dv, gate_a, gate_b, A_log, dt_
 
 def tree_conv(tree: Tree, x, ctx, weight, bias=None, *, H, dk, dv, gate_a=None, gate_b=None, A_log=None,
               dt_bias=None, normalize_qk=False, eps=1e-6, q=None, k=None, v=None, alpha=None, beta=None,
-              stream=None):
+              stream=None, impl=IMPL_AUTO):
     """``tv_tree_conv``: tree-parallel causal convolution + bias + SiLU (+ q/k normalisation, + gates).
 
     ``x`` [B,T,C], ``ctx`` [B,W-1,C], ``weight`` f32 [C,W]; returns ``(q, k, v)`` head-major, and
@@ -477,17 +478,17 @@ def tree_conv(tree: Tree, x, ctx, weight, bias=None, *, H, dk, dv, gate_a=None, 
     if gate_b is not None and beta is None:
         beta = torch.empty(*lead, device=x.device, dtype=torch.float32)
     args, _keep = _conv_args(tree, x, ctx, weight, bias, H, dk, dv, gate_a, gate_b, A_log, dt_bias,
-                             normalize_qk, eps, q, k, v, alpha, beta, stream)
+                             normalize_qk, eps, q, k, v, alpha, beta, stream, impl)
     _check(lib().tv_tree_conv(*args), "tv_tree_conv")
     return (q, k, v) if gate_a is None else (q, k, v, alpha, beta)
 
 
 def prepare_tree_conv(tree: Tree, x, ctx, weight, bias=None, *, H, dk, dv, gate_a=None, gate_b=None,
                       A_log=None, dt_bias=None, normalize_qk=False, eps=1e-6, q, k, v, alpha=None, beta=None,
-                      stream=None) -> "Prepared":
+                      stream=None, impl=IMPL_AUTO) -> "Prepared":
     """``tv_tree_conv`` with pre-marshalled arguments; outputs must be given."""
     args, keep = _conv_args(tree, x, ctx, weight, bias, H, dk, dv, gate_a, gate_b, A_log, dt_bias,
-                            normalize_qk, eps, q, k, v, alpha, beta, stream)
+                            normalize_qk, eps, q, k, v, alpha, beta, stream, impl)
     return Prepared(lib().tv_tree_conv, "tv_tree_conv", args, keep)
 
 

@@ -40,7 +40,8 @@ def close(got, ref, dtype, what, scale=1.0):
     assert err.max() <= 0, f"{what}: worst excess {err.max():.3e} at {np.unravel_index(err.argmax(), err.shape)}"
 
 
-def run_case(wl, parents, W=4, normalize=False, gates=True, gate_b=True, bias=True, scale=1.0, requests=None):
+def run_case(wl, parents, W=4, normalize=False, gates=True, gate_b=True, bias=True, scale=1.0, requests=None,
+             impl=tv.IMPL_AUTO):
     ci = inputs.make_conv_inputs(wl, layer=0, device="cpu", W=W)
     if scale != 1.0:
         ci["x"] = (ci["x"].float() * scale).to(ci["x"].dtype)
@@ -58,7 +59,7 @@ def run_case(wl, parents, W=4, normalize=False, gates=True, gate_b=True, bias=Tr
                  H=H, dk=dk, dv=dv, gate_a=g["gate_a"] if gates else None,
                  gate_b=g["gate_b"] if gates and gate_b else None, A_log=g["A_log"], dt_bias=g["dt_bias"],
                  normalize_qk=normalize, eps=1e-6, q=q, k=k, v=v, alpha=al if gates else None,
-                 beta=be if gates and gate_b else None)
+                 beta=be if gates and gate_b else None, impl=impl)
     torch.cuda.synchronize()
     assert torch.equal(g["x"], x0)
     for buf, t in ((qb, q), (kb, k), (vb, v), (ab, al), (bb, be)):
@@ -86,11 +87,29 @@ def run_case(wl, parents, W=4, normalize=False, gates=True, gate_b=True, bias=Tr
     return g, tree
 
 
+@pytest.mark.parametrize("impl", [tv.IMPL_AUTO, tv.IMPL_SIMT])
 @pytest.mark.parametrize("name", ["c1", "c2", "c3", "c4"])
-def test_workloads(name):
+def test_workloads(name, impl):
     wl = inputs.workload(name)
     parents, _ = inputs.make_trees(wl)
-    run_case(wl, parents, W=4, normalize=(name in ("c2", "c4")))
+    run_case(wl, parents, W=4, normalize=(name in ("c2", "c4")), impl=impl)
+
+
+@pytest.mark.parametrize("T", [1, 7, 16, 17, 63, 64, 65, 100, 128])
+@pytest.mark.parametrize("W", [1, 2, 3, 4])
+def test_tensor_core_kernel_shapes(T, W):
+    """bf16, 128-channel heads, W <= 4: the mma kernel, forced (IMPL_TC), over tile-edge sizes."""
+    wl = dataclasses.replace(inputs.workload("c2"), B=3, H=2, T=T, seed=900 + T + W)
+    parents, _ = inputs.make_trees(wl)
+    run_case(wl, parents, W=W, normalize=bool(T & 1), gate_b=bool(W & 1), bias=W != 3, impl=tv.IMPL_TC)
+
+
+def test_tensor_core_kernel_declines_other_shapes():
+    wl = dataclasses.replace(inputs.workload("c2"), B=1, H=2, T=16, dk=64, dv=128)
+    parents, _ = inputs.make_trees(wl)
+    with pytest.raises(tv.TreeVerifyError) as e:
+        run_case(wl, parents, W=4, impl=tv.IMPL_TC)
+    assert e.value.status == -3
 
 
 def test_c5_sampled_requests():
