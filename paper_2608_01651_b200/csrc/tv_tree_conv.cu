@@ -261,11 +261,13 @@ tree_conv_kernel(const ConvArgs a) {
       if (cv >= vpr) { cv -= vpr; ++row; }
     }
   };
+  // (the last warps do this, the first ones prepare the gates: neither is late at the barrier)
   auto build_taps = [&](const ConvItem& it, int slot) {
-    if (tid < it.n) {
+    const int node = kConvThreads - 1 - tid;
+    if (node < it.n) {
       const uint32_t row_bytes = (uint32_t)it.d * sizeof(IO);
       const int32_t* par = par_s + slot * Tp;
-      int j = tid, ctx_row = W - 2;
+      int j = node, ctx_row = W - 2;
 #pragma unroll
       for (int r = 0; r < W; ++r) {
         int row;
@@ -275,7 +277,7 @@ tree_conv_kernel(const ConvArgs a) {
         } else {
           row = ctx_row--;
         }
-        taps_s[(slot * T + tid) * WP + r] = (uint32_t)row * row_bytes;
+        taps_s[(slot * T + node) * WP + r] = (uint32_t)row * row_bytes;
       }
     }
   };
