@@ -16,7 +16,7 @@ path, the kept nodes of a request form a prefix-closed subtree.  A count per req
 budget q_b; the kept nodes are packed request by request, in their original order, into one flat
 forest (Section V-B), with parents renumbered locally.
 
-Precision and ties (fixed here, listed in the design doc): rho is computed in float32 by the
+Precision and ties (the paper is silent; fixed here): rho is computed in float32 by the
 recurrence above (one rounding per edge, parent before child), which is what decides the
 selection; equal rho are ordered by (request, node) index, lower first.  Roots rank above
 everything.  A non-root child of the virtual root (parent -1 at index > 0) is a sibling tree of

@@ -18,7 +18,7 @@ context: ctx[W-2] is the token just before the tree, ctx[W-3] the one before
 it, and so on (ctx has W-1 rows, oldest first).  w[c][W-1] multiplies the
 current token (the usual causal depthwise layout), SiLU(z) = z / (1 + e^-z).
 
-Readings of what the paper leaves open, fixed here and listed in the design doc:
+Readings of what the paper leaves open, fixed here:
 the channel order is [q heads | k heads | v heads]; "normalization ... folded
 into these stages" is read as an optional L2 normalisation of each q and k head
 vector after SiLU, x / sqrt(sum x^2 + eps); the gate formulas are not given by
