@@ -19,10 +19,10 @@ it, and so on (ctx has W-1 rows, oldest first).  w[c][W-1] multiplies the
 current token (the usual causal depthwise layout), SiLU(z) = z / (1 + e^-z).
 
 Readings of what the paper leaves open, fixed here:
-the channel order is [q heads | k heads | v heads]; "normalization ... folded
-into these stages" is read as an optional L2 normalisation of each q and k head
-vector after SiLU, x / sqrt(sum x^2 + eps); the gate formulas are not given by
-the paper and are not part of this operator.
+the channel order is [q heads | k heads | v heads]; the normalisation that the
+paper folds into its stages without a formula is read as an optional L2
+normalisation of each q and k head vector after SiLU, x / sqrt(sum x^2 + eps);
+the gate formulas are not given by the paper either (see gate_prep below).
 """
 from __future__ import annotations
 
