@@ -286,11 +286,14 @@ int tv_commit_path(const tv_tree* tree, const tv_dims* dims,
  * whose tensors live in HOST memory (pinned memory makes the copies
  * asynchronous).  A session owns device copies sized for `dims` (allocated
  * once by tv_session_create on the current device; n_trees is 1 or B).
- * tv_session_round copies parent/accepted/S_pre/q/k/v/alpha/beta to the device
- * on `stream`, verifies, commits in place on the device copy (the delta rule
- * commits from the corrections U that verify wrote), copies O and S_new back
- * and synchronises the stream before returning.  All pointers are host
- * pointers in the layouts above; beta may be NULL for TV_GATED.               */
+ * tv_session_round copies parent/accepted/S_pre/q/k/v/alpha/beta to the device,
+ * verifies, commits in place on the device copy (the delta rule commits from
+ * the corrections U that verify wrote), copies O and S_new back and
+ * synchronises before returning.  The requests are handled in up to four
+ * groups on two streams of the session's own (ordered after the work already
+ * queued on `stream`, and `stream` waits for them), so that the copies in, the
+ * kernels and the copies out of different groups overlap.  All pointers are
+ * host pointers in the layouts above; beta may be NULL for TV_GATED.           */
 typedef struct tv_session tv_session;
 int tv_session_create(const tv_dims* dims, int32_t n_trees, tv_session** out);
 int tv_session_round(tv_session* s, const int32_t* parent /*[n_trees][T]*/,

@@ -1,20 +1,34 @@
 // Host-buffer round: the whole hot path (tree_build -> tree_verify ->
 // commit_path) for callers whose tensors live in host memory.  A session owns
 // the device copies; a round moves the inputs in, runs the same entry points
-// a device-resident caller uses, and moves O and S_new out.
+// a device-resident caller uses, and moves O and S_new out, group of requests
+// by group of requests so that transfers and kernels overlap.
 #include <new>
 
 #include "tv_internal.h"
 
-struct tv_session {
-  tv_dims dims;
-  int32_t n_trees = 0;
+// The batch is cut into up to kMaxChunks groups of requests that alternate between two internal
+// streams: while one group computes and returns its outputs, the next group's inputs arrive, so
+// the host->device and device->host copies (separate copy engines) overlap each other and the
+// kernels.  Requests are independent (Section IV-B), so the groups need no exchange.
+constexpr int kMaxChunks = 4;
+
+struct tv_chunk {
+  int32_t b0 = 0, nb = 0;     // requests [b0, b0 + nb)
   tv_tree* tree = nullptr;
-  char* d_base = nullptr;
   float *S = nullptr, *alpha = nullptr, *beta = nullptr, *O = nullptr, *U = nullptr;
   void *q = nullptr, *k = nullptr, *v = nullptr;
   int32_t* accepted = nullptr;
-  size_t nS = 0, nQ = 0, nV = 0, nG = 0, eb = 0;
+};
+
+struct tv_session {
+  tv_dims dims;
+  int32_t n_trees = 0, n_chunks = 0;
+  tv_chunk chunk[kMaxChunks];
+  char* d_base = nullptr;
+  size_t eb = 0;
+  cudaStream_t side[2] = {nullptr, nullptr};
+  cudaEvent_t start = nullptr, done[2] = {nullptr, nullptr};
 };
 
 static size_t up256(size_t x) { return (x + 255) & ~(size_t)255; }
@@ -23,46 +37,63 @@ static size_t up256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 extern "C" {
 
+TV_API int tv_session_free(tv_session* s);
+
 TV_API int tv_session_create(const tv_dims* d, int32_t n_trees, tv_session** out) {
   if (!out) return TV_ERR_BAD_ARG;
   *out = nullptr;
   if (!d || (n_trees != 1 && n_trees != d->B)) return TV_ERR_BAD_ARG;
   if (d->L < 1 || d->B < 1 || d->H < 1 || d->T < 1 || d->T > TV_MAX_NODES) return TV_ERR_BAD_ARG;
+  if (d->Hk < 0 || d->Hk > d->H || (d->Hk > 0 && d->H % d->Hk != 0)) return TV_ERR_BAD_ARG;
   tv_session* s = new (std::nothrow) tv_session();
   if (!s) return TV_ERR_NOMEM;
   s->dims = *d;
   s->n_trees = n_trees;
-  const size_t items = (size_t)d->L * d->B * d->H;
   s->eb = d->qkv_dtype == TV_BF16 ? 2 : 4;
-  s->nS = items * d->dv * d->dk;
-  if (d->Hk < 0 || d->Hk > d->H || (d->Hk > 0 && d->H % d->Hk != 0)) {
-    delete s;
-    return TV_ERR_BAD_ARG;
-  }
-  s->nQ = (size_t)d->L * d->B * (d->Hk ? d->Hk : d->H) * d->T * d->dk;
-  s->nV = items * d->T * d->dv;
-  s->nG = items * d->T;
+  s->n_chunks = d->B < kMaxChunks ? d->B : kMaxChunks;
   const bool delta = d->rule == TV_GATED_DELTA;
+  const size_t Hk = d->Hk ? d->Hk : d->H;
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off += up256(bytes); return o; };
-  const size_t oS = take(s->nS * 4), oq = take(s->nQ * s->eb), ok = take(s->nQ * s->eb),
-               ov = take(s->nV * s->eb), oa = take(s->nG * 4), ob = take(s->nG * 4),
-               oO = take(s->nV * 4), oU = take(delta ? s->nV * 4 : 0), oacc = take((size_t)d->B * 4);
+  size_t o[kMaxChunks][9];
+  for (int c = 0; c < s->n_chunks; ++c) {
+    tv_chunk& ch = s->chunk[c];
+    ch.b0 = (int32_t)((int64_t)d->B * c / s->n_chunks);
+    ch.nb = (int32_t)((int64_t)d->B * (c + 1) / s->n_chunks) - ch.b0;
+    const size_t items = (size_t)d->L * ch.nb * d->H, qitems = (size_t)d->L * ch.nb * Hk;
+    o[c][0] = take(items * d->dv * d->dk * 4);
+    o[c][1] = take(qitems * d->T * d->dk * s->eb);
+    o[c][2] = take(qitems * d->T * d->dk * s->eb);
+    o[c][3] = take(items * d->T * d->dv * s->eb);
+    o[c][4] = take(items * d->T * 4);
+    o[c][5] = take(items * d->T * 4);
+    o[c][6] = take(items * d->T * d->dv * 4);
+    o[c][7] = take(delta ? items * d->T * d->dv * 4 : 0);
+    o[c][8] = take((size_t)ch.nb * 4);
+  }
   cudaError_t e = cudaMalloc((void**)&s->d_base, off);
+  for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
+    e = cudaStreamCreateWithFlags(&s->side[i], cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&s->done[i], cudaEventDisableTiming);
+  }
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&s->start, cudaEventDisableTiming);
   if (e != cudaSuccess) {
     tv_set_cuda_error(e);
-    delete s;
+    tv_session_free(s);
     return TV_ERR_CUDA;
   }
-  s->S = (float*)(s->d_base + oS);
-  s->q = s->d_base + oq;
-  s->k = s->d_base + ok;
-  s->v = s->d_base + ov;
-  s->alpha = (float*)(s->d_base + oa);
-  s->beta = delta ? (float*)(s->d_base + ob) : nullptr;
-  s->O = (float*)(s->d_base + oO);
-  s->U = delta ? (float*)(s->d_base + oU) : nullptr;
-  s->accepted = (int32_t*)(s->d_base + oacc);
+  for (int c = 0; c < s->n_chunks; ++c) {
+    tv_chunk& ch = s->chunk[c];
+    ch.S = (float*)(s->d_base + o[c][0]);
+    ch.q = s->d_base + o[c][1];
+    ch.k = s->d_base + o[c][2];
+    ch.v = s->d_base + o[c][3];
+    ch.alpha = (float*)(s->d_base + o[c][4]);
+    ch.beta = delta ? (float*)(s->d_base + o[c][5]) : nullptr;
+    ch.O = (float*)(s->d_base + o[c][6]);
+    ch.U = delta ? (float*)(s->d_base + o[c][7]) : nullptr;
+    ch.accepted = (int32_t*)(s->d_base + o[c][8]);
+  }
   *out = s;
   return TV_OK;
 }
@@ -78,34 +109,69 @@ TV_API int tv_session_round(tv_session* s, const int32_t* parent, const int32_t*
   if (delta && !beta) return TV_ERR_BAD_ARG;
   for (int b = 0; b < d.B; ++b)
     if (accepted[b] < -1 || accepted[b] >= d.T) return TV_ERR_BAD_ARG;
-  int st;
-  if (!s->tree) st = tv_tree_build(parent, s->n_trees, d.T, &s->tree);
-  else st = tv_tree_rebuild(s->tree, parent);
-  if (st != TV_OK) return st;
-  cudaStream_t cs = (cudaStream_t)stream;
-  st = tv_tree_upload(s->tree, stream);
-  if (st != TV_OK) return st;
-  TV_CUDA_TRY(cudaMemcpyAsync(s->S, S_pre, s->nS * 4, cudaMemcpyHostToDevice, cs));
-  TV_CUDA_TRY(cudaMemcpyAsync(s->q, q, s->nQ * s->eb, cudaMemcpyHostToDevice, cs));
-  TV_CUDA_TRY(cudaMemcpyAsync(s->k, k, s->nQ * s->eb, cudaMemcpyHostToDevice, cs));
-  TV_CUDA_TRY(cudaMemcpyAsync(s->v, v, s->nV * s->eb, cudaMemcpyHostToDevice, cs));
-  TV_CUDA_TRY(cudaMemcpyAsync(s->alpha, alpha, s->nG * 4, cudaMemcpyHostToDevice, cs));
-  if (delta) TV_CUDA_TRY(cudaMemcpyAsync(s->beta, beta, s->nG * 4, cudaMemcpyHostToDevice, cs));
-  TV_CUDA_TRY(cudaMemcpyAsync(s->accepted, accepted, (size_t)d.B * 4, cudaMemcpyHostToDevice, cs));
-  st = tv_tree_verify(s->tree, &d, s->S, s->q, s->k, s->v, s->alpha, s->beta, s->O, s->U, stream);
-  if (st != TV_OK) return st;
-  st = tv_commit_path(s->tree, &d, s->accepted, s->S, s->k, s->v, s->alpha, s->beta, s->U, s->S,
-                      stream);
-  if (st != TV_OK) return st;
-  TV_CUDA_TRY(cudaMemcpyAsync(O, s->O, s->nV * 4, cudaMemcpyDeviceToHost, cs));
-  TV_CUDA_TRY(cudaMemcpyAsync(S_new, s->S, s->nS * 4, cudaMemcpyDeviceToHost, cs));
-  TV_CUDA_TRY(cudaStreamSynchronize(cs));
+  const size_t Hk = d.Hk ? d.Hk : d.H;
+  // bytes of one request of one layer in each tensor
+  const size_t rS = (size_t)d.H * d.dv * d.dk * 4, rQ = Hk * d.T * d.dk * s->eb, rV = (size_t)d.H * d.T * d.dv * s->eb,
+               rG = (size_t)d.H * d.T * 4, rO = (size_t)d.H * d.T * d.dv * 4;
+  cudaStream_t user = (cudaStream_t)stream;
+  TV_CUDA_TRY(cudaEventRecord(s->start, user));
+  for (int i = 0; i < 2; ++i) TV_CUDA_TRY(cudaStreamWaitEvent(s->side[i], s->start, 0));
+  for (int c = 0; c < s->n_chunks; ++c) {
+    tv_chunk& ch = s->chunk[c];
+    cudaStream_t cs = s->side[c & 1];
+    const int32_t* par = s->n_trees == 1 ? parent : parent + (size_t)ch.b0 * d.T;
+    const int32_t nt = s->n_trees == 1 ? 1 : ch.nb;
+    int st = ch.tree ? tv_tree_rebuild(ch.tree, par) : tv_tree_build(par, nt, d.T, &ch.tree);
+    if (st != TV_OK) return st;
+    st = tv_tree_upload(ch.tree, cs);
+    if (st != TV_OK) return st;
+    auto h2d = [&](void* dst, const void* src, size_t per_req) -> cudaError_t {
+      for (int l = 0; l < d.L; ++l) {   // the group's requests are contiguous within a layer
+        cudaError_t e = cudaMemcpyAsync((char*)dst + (size_t)l * ch.nb * per_req,
+                                        (const char*)src + ((size_t)l * d.B + ch.b0) * per_req,
+                                        (size_t)ch.nb * per_req, cudaMemcpyHostToDevice, cs);
+        if (e != cudaSuccess) return e;
+      }
+      return cudaSuccess;
+    };
+    TV_CUDA_TRY(h2d(ch.S, S_pre, rS));
+    TV_CUDA_TRY(h2d(ch.q, q, rQ));
+    TV_CUDA_TRY(h2d(ch.k, k, rQ));
+    TV_CUDA_TRY(h2d(ch.v, v, rV));
+    TV_CUDA_TRY(h2d(ch.alpha, alpha, rG));
+    if (delta) TV_CUDA_TRY(h2d(ch.beta, beta, rG));
+    TV_CUDA_TRY(cudaMemcpyAsync(ch.accepted, accepted + ch.b0, (size_t)ch.nb * 4, cudaMemcpyHostToDevice, cs));
+    tv_dims dc = d;
+    dc.B = ch.nb;
+    st = tv_tree_verify(ch.tree, &dc, ch.S, ch.q, ch.k, ch.v, ch.alpha, ch.beta, ch.O, ch.U, cs);
+    if (st != TV_OK) return st;
+    st = tv_commit_path(ch.tree, &dc, ch.accepted, ch.S, ch.k, ch.v, ch.alpha, ch.beta, ch.U, ch.S, cs);
+    if (st != TV_OK) return st;
+    for (int l = 0; l < d.L; ++l) {
+      TV_CUDA_TRY(cudaMemcpyAsync((char*)O + ((size_t)l * d.B + ch.b0) * rO, (char*)ch.O + (size_t)l * ch.nb * rO,
+                                  (size_t)ch.nb * rO, cudaMemcpyDeviceToHost, cs));
+      TV_CUDA_TRY(cudaMemcpyAsync((char*)S_new + ((size_t)l * d.B + ch.b0) * rS,
+                                  (char*)ch.S + (size_t)l * ch.nb * rS, (size_t)ch.nb * rS,
+                                  cudaMemcpyDeviceToHost, cs));
+    }
+  }
+  for (int i = 0; i < 2; ++i) {
+    TV_CUDA_TRY(cudaEventRecord(s->done[i], s->side[i]));
+    TV_CUDA_TRY(cudaStreamWaitEvent(user, s->done[i], 0));
+  }
+  TV_CUDA_TRY(cudaStreamSynchronize(user));
   return TV_OK;
 }
 
 TV_API int tv_session_free(tv_session* s) {
   if (!s) return TV_OK;
-  if (s->tree) tv_tree_free(s->tree);
+  for (int c = 0; c < kMaxChunks; ++c)
+    if (s->chunk[c].tree) tv_tree_free(s->chunk[c].tree);
+  for (int i = 0; i < 2; ++i) {
+    if (s->side[i]) cudaStreamDestroy(s->side[i]);
+    if (s->done[i]) cudaEventDestroy(s->done[i]);
+  }
+  if (s->start) cudaEventDestroy(s->start);
   if (s->d_base) cudaFree(s->d_base);
   delete s;
   return TV_OK;
