@@ -393,6 +393,8 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     // dependent launch: barrier set-up and the TMEM allocation above ran under the tail of the
     // kernel in front; everything that reads global memory waits for it here
     grid_dependency_wait();
+    // the commit kernel behind this one may be scheduled as SMs drain (it orders itself)
+    if (warp == 2 && lane == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     fetch_meta(blockIdx.x);
 
     uint32_t it = 0;

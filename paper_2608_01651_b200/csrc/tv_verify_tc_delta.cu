@@ -359,6 +359,8 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       }
     };
     grid_dependency_wait();   // tree metadata comes from the kernel in front (dependent launch)
+    // the commit kernel behind this one may be scheduled as SMs drain (it orders itself)
+    if (warp == 2 && lane == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     fetch_meta(blockIdx.x);
 
     // acc rows 0..63 -> O chunks 0..3, rows 64..127 -> U chunks 4..7 (the chunks alias the Ak / W
