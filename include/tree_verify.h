@@ -270,7 +270,13 @@ int tv_tree_verify_static(const int32_t* parent /*dev*/, int32_t n_trees, const 
  * outside [-1, T) are treated as -1.  U: the corrections written by
  * tv_tree_verify, or NULL -- then TV_GATED uses u_j = v_j and TV_GATED_DELTA
  * re-derives u_j along the accepted path from S_pre (needs dk in {64,128}).
- * S_new may alias S_pre exactly (in place) or not overlap it at all.          */
+ * S_new may alias S_pre exactly (in place) or not overlap it at all.
+ * Stream order: when the call directly follows tv_tree_verify on the same
+ * stream, the commit grid may be scheduled while the verify kernel drains and
+ * read S_pre and accepted early; it reads U and writes S_new only after that
+ * kernel has completed.  (Behind any other work it starts after that work, as
+ * usual.)  So accepted, S_pre, k, v, alpha must not be outputs of the
+ * tv_tree_verify call in front of it -- U is the only one that may be.        */
 int tv_commit_path(const tv_tree* tree, const tv_dims* dims,
                    const int32_t* accepted /*dev [B]*/,
                    const float* S_pre /*dev*/,
