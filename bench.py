@@ -522,8 +522,8 @@ def run_ours(args, wl, rank, world, local_rank):
 
     # ---- the verify kernel alone, launches back to back over the rotating sets: what the events
     # inside the step above cannot separate from launch latency (they sit between two launches)
-    n_b2b = 48
-    for i in range(n_sets):
+    n_b2b = 0 if args.no_b2b else 48
+    for i in range(n_sets if n_b2b else 0):
         calls[i][0][0]()
     torch.cuda.synchronize()
     b0, b1 = ev(), ev()
@@ -533,7 +533,7 @@ def run_ours(args, wl, rank, world, local_rank):
         ver[i % len(ver)]()
     b1.record(stream)
     torch.cuda.synchronize()
-    v_b2b_ms = b0.elapsed_time(b1) / n_b2b
+    v_b2b_ms = b0.elapsed_time(b1) / n_b2b if n_b2b else float("nan")
 
     # ---- Stage 1 (tree convolution + SiLU + normalisation + gates), timed on its own --------
     # Not part of the step above (the metric is defined on verify + commit); one launch per layer
@@ -661,6 +661,7 @@ def main():
                     help="run the step on a packed forest of requests with different node counts (1 GPU)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-stage1", action="store_true")
+    ap.add_argument("--no-b2b", action="store_true", help="skip the back-to-back verify timing")
     ap.add_argument("--stage1-iters", type=int, default=48)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
