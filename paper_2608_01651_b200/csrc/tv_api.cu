@@ -270,6 +270,16 @@ TV_API int tv_tree_upload(tv_tree* t, void* stream) {
   int st = ensure_device(t, L);
   if (st != TV_OK) return st;
   cudaStream_t s = (cudaStream_t)stream;
+  if (tv_tree_meta_fits_params(t->n_trees, t->n, !t->offsets.empty())) {
+    // small tree sets: the parents ride in the launch itself
+    st = tv_launch_tree_meta_params(t->parent.data(), t->n_trees, t->n, t->d_anc_w, t->d_depth_w, t->d_parent_w,
+                                    t->d_status, t->offsets.empty() ? nullptr : t->offsets.data(),
+                                    t->d_offsets_w, s);
+    if (st != TV_OK) return st;
+    t->uploaded = true;
+    t->host_meta_valid = true;
+    return TV_OK;
+  }
   // The parent arrays go into one of two pinned slots; a small kernel reads the slot over the
   // bus and derives masks and depths on the device (no copy-engine hop in front of the verify
   // launch).  A slot is reused only after the kernel that read it two uploads ago has finished.

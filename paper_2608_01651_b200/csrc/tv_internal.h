@@ -121,6 +121,11 @@ int tv_launch_commit(const CommitArgs& a, cudaStream_t stream);
 int tv_launch_tree_meta(const int32_t* parent_mapped, int32_t n_trees, int32_t n, uint64_t* anc,
                         int32_t* depth, int32_t* parent_dev, int32_t* status, const int32_t* offsets_mapped,
                         int32_t* offsets_dev, cudaStream_t stream);
+// Host parents carried in the kernel parameters (small tree sets): no staging, no read over the bus.
+bool tv_tree_meta_fits_params(int32_t n_trees, int32_t n, bool has_offsets);
+int tv_launch_tree_meta_params(const int32_t* parent_host, int32_t n_trees, int32_t n, uint64_t* anc,
+                               int32_t* depth, int32_t* parent_dev, int32_t* status, const int32_t* offsets_host,
+                               int32_t* offsets_dev, cudaStream_t stream);
 bool tv_verify_tc_supports(const VerifyArgs& a);
 int tv_launch_verify_tc(const VerifyArgs& a, int32_t* status, cudaStream_t stream);
 bool tv_verify_tc_delta_supports(const VerifyArgs& a);

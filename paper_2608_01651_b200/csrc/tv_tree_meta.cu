@@ -44,7 +44,78 @@ tree_meta_kernel(const int32_t* __restrict__ parent, int32_t n, uint64_t* __rest
   parent_dev[o] = par_s[i];
 }
 
+// The same derivation with the parents carried in the kernel's PARAMETERS (one byte per node,
+// -1..127), for tree sets small enough to fit: the launch itself brings the data, so the kernel
+// does not start with a read over the bus.
+template <int NB>
+struct ParentBytes {
+  int8_t p[NB];
+};
+struct OffsetWords {
+  int32_t o[TV_MAX_NODES + 1 + 3];   // up to 128 requests + end marker
+};
+
+template <int NB>
+__global__ void __launch_bounds__(TV_MAX_NODES)
+tree_meta_param_kernel(const __grid_constant__ ParentBytes<NB> pb, const __grid_constant__ OffsetWords off,
+                       int32_t has_offsets, int32_t n, uint64_t* __restrict__ anc, int32_t* __restrict__ depth,
+                       int32_t* __restrict__ parent_dev, int32_t* status, int32_t* __restrict__ offsets_dev) {
+  __shared__ int32_t par_s[TV_MAX_NODES];
+  const int t = blockIdx.x, i = threadIdx.x;
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // as in the kernel above
+  if (i < n) par_s[i] = pb.p[t * n + i];
+  if (t == 0 && i == 0) *status = 0;
+  if (has_offsets && i == 0) {
+    offsets_dev[t] = off.o[t];
+    if (t == (int)gridDim.x - 1) offsets_dev[t + 1] = off.o[t + 1];
+  }
+  __syncthreads();
+  if (i >= n) return;
+  uint64_t w0 = 0, w1 = 0;
+  int d = 0;
+  for (int p = par_s[i]; p >= 0 && d < n; p = par_s[p]) {
+    if (p < 64) w0 |= 1ull << p; else w1 |= 1ull << (p - 64);
+    ++d;
+  }
+  const size_t o = (size_t)t * n + i;
+  anc[2 * o] = w0;
+  anc[2 * o + 1] = w1;
+  depth[o] = d;
+  parent_dev[o] = par_s[i];
+}
+
+template <int NB>
+int launch_param(const int32_t* parent_host, int32_t n_trees, int32_t n, uint64_t* anc, int32_t* depth,
+                 int32_t* parent_dev, int32_t* status, const int32_t* offsets_host, int32_t* offsets_dev,
+                 cudaStream_t stream) {
+  ParentBytes<NB> pb;
+  const int nn = n_trees * n;
+  for (int i = 0; i < nn; ++i) pb.p[i] = (int8_t)parent_host[i];   // validated: -1 <= parent < 128
+  OffsetWords off;
+  if (offsets_host)
+    for (int i = 0; i <= n_trees; ++i) off.o[i] = offsets_host[i];
+  tree_meta_param_kernel<NB><<<n_trees, TV_MAX_NODES, 0, stream>>>(pb, off, offsets_host != nullptr, n, anc, depth,
+                                                                  parent_dev, status, offsets_dev);
+  TV_CUDA_TRY(cudaGetLastError());
+  return TV_OK;
+}
+
 }  // namespace
+
+bool tv_tree_meta_fits_params(int32_t n_trees, int32_t n, bool has_offsets) {
+  return (int64_t)n_trees * n <= 16384 && (!has_offsets || n_trees <= TV_MAX_NODES);
+}
+
+int tv_launch_tree_meta_params(const int32_t* parent_host, int32_t n_trees, int32_t n, uint64_t* anc,
+                               int32_t* depth, int32_t* parent_dev, int32_t* status, const int32_t* offsets_host,
+                               int32_t* offsets_dev, cudaStream_t stream) {
+  const int nn = n_trees * n;
+  if (nn <= 2048)
+    return launch_param<2048>(parent_host, n_trees, n, anc, depth, parent_dev, status, offsets_host, offsets_dev,
+                              stream);
+  return launch_param<16384>(parent_host, n_trees, n, anc, depth, parent_dev, status, offsets_host, offsets_dev,
+                             stream);
+}
 
 int tv_launch_tree_meta(const int32_t* parent_mapped, int32_t n_trees, int32_t n, uint64_t* anc,
                         int32_t* depth, int32_t* parent_dev, int32_t* status, const int32_t* offsets_mapped,

@@ -240,3 +240,17 @@ def test_forest_stage1_conv_and_context_commit(dtype, W):
         off += n
     for t in list(out.values()) + [al, be]:
         assert bool((t[:, total:] == 9.0).all())      # rows past the forest untouched
+
+
+@pytest.mark.parametrize("n_trees,n", [(200, 100), (129, 128), (16, 128)])
+def test_metadata_upload_paths_agree_with_the_host(n_trees, n):
+    """Small tree sets ride in the kernel parameters, large ones are staged through pinned memory:
+    both must reproduce the host-built masks and depths bit for bit (and survive a rebuild)."""
+    rng = np.random.Generator(np.random.Philox(key=n_trees))
+    for trial in range(3):
+        par = np.stack([inputs.tree_frontier(n, rng) for _ in range(n_trees)]).astype(np.int32)
+        tree = tv.tree_build(par) if trial == 0 else tree.rebuild(par)
+        tree.upload()
+        anc, depth, _ = tree.meta()
+        danc, ddepth = tree.meta_device()
+        assert np.array_equal(anc, danc) and np.array_equal(depth, ddepth)
