@@ -119,12 +119,14 @@ int tv_tree_info(const tv_tree* tree, int32_t* n_trees, int32_t* n,
  * unused entries set to -1; len is host int32 [n_req].                        */
 int tv_tree_path(const tv_tree* tree, const int32_t* accepted, int32_t n_req,
                  int32_t* path, int32_t path_stride, int32_t* len);
-/* Put the metadata on the current device, on `stream` (a cudaStream_t): the
- * parent arrays are staged in pinned host memory and one small kernel derives
- * the same masks and depths on the device (Section IV-C: once per request and
- * round, fixed buffers).  The first call allocates the device mirror and the
- * staging block; later calls (after tv_tree_rebuild) allocate nothing.
- * Asynchronous; kernels launched later on the same stream see the result.     */
+/* Put the metadata on the current device, on `stream` (a cudaStream_t): one
+ * small kernel derives the same masks and depths on the device from the parent
+ * arrays (Section IV-C: once per request and round, fixed buffers).  Tree sets
+ * of up to 16384 nodes travel in that kernel's parameters; larger ones are
+ * staged in pinned host memory that the kernel reads.  The first call allocates
+ * the device mirror (and, for large sets, the staging block); later calls
+ * (after tv_tree_rebuild) allocate nothing.  Asynchronous; kernels launched
+ * later on the same stream see the result.                                     */
 int tv_tree_upload(tv_tree* tree, void* stream);
 /* Copy the DEVICE-built masks and depths back to host arrays (same shapes as
  * tv_tree_meta) and synchronise `stream`: lets a caller check them bit for bit
