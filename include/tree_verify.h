@@ -124,8 +124,8 @@ int tv_tree_path(const tv_tree* tree, const int32_t* accepted, int32_t n_req,
  * arrays (Section IV-C: once per request and round, fixed buffers).  Tree sets
  * of up to 16384 nodes travel in that kernel's parameters; larger ones are
  * staged in pinned host memory that the kernel reads.  The first call allocates
- * the device mirror (and, for large sets, the staging block); later calls
- * (after tv_tree_rebuild) allocate nothing.  Asynchronous; kernels launched
+ * the device mirror and the staging block; later calls (after tv_tree_rebuild)
+ * allocate nothing.  Asynchronous; kernels launched
  * later on the same stream see the result.                                     */
 int tv_tree_upload(tv_tree* tree, void* stream);
 /* Copy the DEVICE-built masks and depths back to host arrays (same shapes as
