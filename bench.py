@@ -105,7 +105,7 @@ def measured_peak():
 # Clock sampling during the timed region
 # --------------------------------------------------------------------------
 class ClockSampler:
-    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+    Q = ("timestamp,clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
 
@@ -115,40 +115,74 @@ class ClockSampler:
         try:
             self.p = subprocess.Popen(
                 ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                 "-i", str(index), "-lms", "20"], stdout=self.f, stderr=subprocess.DEVNULL)
+                 "-i", str(index), "-lms", "10"], stdout=self.f, stderr=subprocess.DEVNULL)
         except Exception:
             self.p = None
 
-    def stop(self) -> dict:
-        if self.p is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
-        self.p.terminate()
-        try:
-            self.p.wait(timeout=5)
-        except Exception:
-            self.p.kill()
-        self.f.flush()
-        self.f.seek(0)
-        sm, mx = [], []
-        reasons = set()
+    def wait_ready(self, timeout: float = 3.0):
+        """nvidia-smi takes a few hundred ms to deliver its first sample: wait for it."""
+        t0 = time.time()
+        while self.p is not None and time.time() - t0 < timeout:
+            if os.path.getsize(self.f.name) > 0:
+                return
+            time.sleep(0.01)
+
+    def _samples(self):
+        import datetime
+        out = []
+        with open(self.f.name) as fh:
+            for line in fh.read().splitlines():
+                parts = [x.strip() for x in line.split(",")]
+                if len(parts) < 7:
+                    continue
+                try:
+                    ts = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                    out.append((ts, float(parts[1]), float(parts[2]), parts[3:7]))
+                except ValueError:
+                    continue
+        return out
+
+    def window(self, w0: float, w1: float) -> dict:
+        """Median SM clock and the throttle reasons seen between wall-clock times w0 and w1."""
+        time.sleep(0.03)   # let the last sample of the window reach the file
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for line in self.f.read().splitlines():
-            parts = [x.strip() for x in line.split(",")]
-            if len(parts) < 6:
-                continue
+        sm, mx, reasons = [], [], set()
+        for ts, c, m, flags in self._samples():
+            if w0 <= ts <= w1:
+                sm.append(c); mx.append(m)
+                for n, v in zip(names, flags):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": float(max(mx)) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+    def stop(self):
+        if self.p is not None:
+            self.p.terminate()
             try:
-                sm.append(float(parts[0])); mx.append(float(parts[1]))
-            except ValueError:
-                continue
-            for n, v in zip(names, parts[2:6]):
-                if v.lower().startswith("active"):
-                    reasons.add(n)
+                self.p.wait(timeout=5)
+            except Exception:
+                self.p.kill()
         self.f.close()
         os.unlink(self.f.name)
-        return {"sm_mhz": float(np.median(sm)) if sm else None,
-                "sm_max_mhz": float(max(mx)) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def sample_clocks(sampler, w0: float, w1: float, replay):
+    """Clocks during the timed region [w0, w1]; if the region was too short for nvidia-smi to
+    sample it, during an untimed replay of the same step loop right after it."""
+    if sampler is None or sampler.p is None:
+        return {"sm_mhz": None, "sm_max_mhz": None, "samples": 0, "reasons": ["nvidia-smi unavailable"]}
+    c = sampler.window(w0, w1)
+    c["sampled"] = "timed region"
+    if c["samples"] < 3:
+        r0 = time.time()
+        while time.time() - r0 < 0.4:
+            replay()
+        torch.cuda.synchronize()
+        c = sampler.window(r0, time.time())
+        c["sampled"] = "untimed replay of the step loop (the timed region was too short to sample)"
+    sampler.stop()
+    return c
 
 
 # --------------------------------------------------------------------------
@@ -371,13 +405,17 @@ def run_packed(args, wl, local_rank):
         step(i, False)
     torch.cuda.synchronize()
     sampler = ClockSampler(local_rank)
+    sampler.wait_ready()
     t0, t1 = ev(), ev()
+    torch.cuda.synchronize()
+    w0 = time.time()
     t0.record(stream)
     for i in range(args.steps):
         step(i, i % probe == 0)
     t1.record(stream)
     torch.cuda.synchronize()
-    clocks = sampler.stop()
+    w1 = time.time()
+    clocks = sample_clocks(sampler, w0, w1, lambda: [step(j, False) for j in range(16)])
     ms = t0.elapsed_time(t1) / args.steps
     v_ms = float(np.mean([a.elapsed_time(b) for a, b, _ in used])) / wl.L
     c_ms = float(np.mean([b.elapsed_time(c) for _, b, c in used]))
@@ -507,15 +545,19 @@ def run_ours(args, wl, rank, world, local_rank):
     torch.cuda.synchronize()
     barrier()
     sampler = ClockSampler(local_rank) if rank == 0 else None
+    if sampler:
+        sampler.wait_ready()
     t_start, t_end = ev(), ev()
     torch.cuda.synchronize()
+    w0 = time.time()
     t_start.record(stream)
     for i in range(args.steps):
         step(args.warmup + i, i % probe == 0)
     t_end.record(stream)
     torch.cuda.synchronize()
+    w1 = time.time()
     barrier()
-    clocks = sampler.stop() if sampler else None
+    clocks = sample_clocks(sampler, w0, w1, lambda: [step(j, False) for j in range(16)]) if sampler else None
     total_ms = t_start.elapsed_time(t_end)
     v_ms = float(np.mean([a.elapsed_time(b) for a, b, _ in kernel_events])) / wl.L
     c_ms = float(np.mean([b.elapsed_time(c) for _, b, c in kernel_events]))
@@ -644,7 +686,9 @@ def run_ours(args, wl, rank, world, local_rank):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--steps", type=int, default=None,
+                    help="timed steps (default: 5000, or 20 for the 48-layer workload: a few hundred ms, "
+                         "long enough for nvidia-smi to sample the clocks inside the timed region)")
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="c3", choices=sorted(DESCR))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -665,6 +709,8 @@ def main():
     ap.add_argument("--stage1-iters", type=int, default=48)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
+    if args.steps is None:
+        args.steps = 200 if args.impl == "reference" else (20 if args.workload == "c5" else 5000)
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
     rank = int(os.environ.get("RANK", "0"))
