@@ -21,10 +21,14 @@
 // are stacked in one operand tile [Q ; K]:
 //     Sc  = [Q ; K] K^T   (bf16, N = 64)   rows 0..63 = Q K^T, rows 64..127 = K K^T
 //     E1: path-sparse raw rows of C and G; E2: back-substitution, operand tiles
-//     Qf  = [diag(P) | -(W D_P)] [Q ; K]   rows 0..63  = Q_eff      (bf16 hi/lo,
-//           [   0    | -(A D_P)] [Q ; K]   rows 64..127 = -K_eff     result in TMEM)
+//     Qf  = D_P Q   (rows 0..63; written to TMEM by the threads that know P_i, in fp32)
+//         + [-(W D_P) ; -(A D_P)] K        rows 0..63 = Q_eff, rows 64..127 = -K_eff
+//           (bf16 hi/lo coefficients, accumulated into the same TMEM columns)
 //     acc = Qf S_pre^T (tf32, A operand straight from TMEM) + [W ; A] V (bf16 hi/lo)
 //     O = acc[0..63], U = acc[64..127]
+// The [Q ; K] tile is double-buffered and its Gram product is issued one item ahead, so the load
+// and the product of item n+1 run under the row solve of item n; what bounds an item is then the
+// CUDA-core chain E1 -> output staging of the previous item -> E2 (about 4.5 us).
 // S_pre goes TMA -> shared memory -> tensor core untouched; O and U leave
 // through swizzled staging chunks and TMA stores.  Every wait is a bounded
 // mbarrier wait (status word on expiry); no TMA multicast.
@@ -42,10 +46,10 @@ constexpr int kLd = 17;        // row stride of the slot tables (floats): confli
 constexpr int kLdP = 20;       // row stride of the path table (bytes)
 
 // shared memory map (bytes from the 1024-aligned base); 14 tiles of 128 rows x 128 B
-constexpr uint32_t kOffQK = 0;                   // 2 k-halves: rows 0..63 Q, rows 64..127 K
+constexpr uint32_t kOffQK = 0;                   // buffer 0 of [Q ; K]: 2 k-halves, rows 0..63 Q, rows 64..127 K
 constexpr uint32_t kOffV = 2 * kTile;            // 2 dv-halves of V (rows 0..63); upper halves: scratch
 constexpr uint32_t kOffS = 4 * kTile;            // 4 k-chunks of S_pre [128 v][32] f32
-constexpr uint32_t kOffAq = 8 * kTile;           // hi, lo of [diag(P) ; 0]          [128][64] bf16
+constexpr uint32_t kOffQK1 = 8 * kTile;          // buffer 1 of [Q ; K] (items alternate between the two)
 constexpr uint32_t kOffAk = 10 * kTile;          // hi, lo of [-(W D_P) ; -(A D_P)]  [128][64] bf16
 constexpr uint32_t kOffW = 12 * kTile;           // hi, lo of [W ; A]                [128][64] bf16
 constexpr uint32_t kOffStage = kOffAk;           // 8 output chunks of 8 KiB (O: 0..3, U: 4..7)
@@ -60,7 +64,7 @@ constexpr uint32_t kSmemBytes = kOffMisc + 64 + 1024;
 enum Bar {
   QK_FULL = 0, QK_FREE, S_FULL, S_FREE, V_FULL, V_FREE,
   G_DONE, G_FREE, W_READY, D1_DONE, ACC_DONE, ACC_FREE, SETUP, E1_SYNC,
-  OST_READY, OST_FREE
+  OST_READY, OST_FREE, QK_FULL1, QK_FREE1
 };
 
 constexpr uint32_t kColSc = 0, kColQf = 128, kColAcc = 256;
@@ -146,6 +150,7 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     abort_flag[0] = 0;
     abort_flag[1] = 0;
     mbar_init(bar(QK_FULL), 1);  mbar_init(bar(QK_FREE), 1);
+    mbar_init(bar(QK_FULL1), 1); mbar_init(bar(QK_FREE1), 1);
     mbar_init(bar(S_FULL), 1);   mbar_init(bar(S_FREE), 1);
     mbar_init(bar(V_FULL), 1);   mbar_init(bar(V_FREE), 1);
     mbar_init(bar(G_DONE), 1);   mbar_init(bar(G_FREE), kComputeWarps);
@@ -171,13 +176,19 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   if (warp == 0) {
     if (lane == 0) {
       // ===================== TMA producer =====================
-      int pend_qk = 0, pend_s = 0, pend_v = 0;
+      int pend_qk = 0, pend_qk_bar = QK_FULL, pend_s = 0, pend_v = 0;
       uint32_t it = 0;
       grid_dependency_wait();   // inputs may come from the kernel in front (dependent launch)
       for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++it) {
         const uint32_t ph = it & 1;
-        if (!mbar_wait(bar(QK_FREE), ph ^ 1, abort_flag)) break;
-        mbar_expect_tx(bar(QK_FULL), 4 * 8192);
+        // [Q ; K] is double-buffered: item it uses buffer it & 1, each buffer's barriers flip
+        // every second item
+        const int qb = (int)(it & 1);
+        const uint32_t qph = (it >> 1) & 1;
+        const uint32_t qk_base = qb ? kOffQK1 : kOffQK;
+        const int qfull = qb ? QK_FULL1 : QK_FULL, qfree = qb ? QK_FREE1 : QK_FREE;
+        if (!mbar_wait(bar(qfree), qph ^ 1, abort_flag)) break;
+        mbar_expect_tx(bar(qfull), 4 * 8192);
         int qk = 0, vplane = item, y0 = 0;
         if constexpr (PACKED) {
           const PackedItem pi = packed_item(p.offsets, p.B, p.H, p.Hk, item);
@@ -185,11 +196,12 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         } else {
           qk = tv_qk_item(item, p.H, p.Hk);
         }
-        tma_load_3d(sbase + kOffQK, &tmQ, bar(QK_FULL), 0, y0, qk);
-        tma_load_3d(sbase + kOffQK + kTile, &tmQ, bar(QK_FULL), 64, y0, qk);
-        tma_load_3d(sbase + kOffQK + 8192, &tmK, bar(QK_FULL), 0, y0, qk);
-        tma_load_3d(sbase + kOffQK + kTile + 8192, &tmK, bar(QK_FULL), 64, y0, qk);
-        pend_qk = 1 + (int)ph;
+        tma_load_3d(sbase + qk_base, &tmQ, bar(qfull), 0, y0, qk);
+        tma_load_3d(sbase + qk_base + kTile, &tmQ, bar(qfull), 64, y0, qk);
+        tma_load_3d(sbase + qk_base + 8192, &tmK, bar(qfull), 0, y0, qk);
+        tma_load_3d(sbase + qk_base + kTile + 8192, &tmK, bar(qfull), 64, y0, qk);
+        pend_qk_bar = qfull;
+        pend_qk = 1 + (int)qph;
         if (!mbar_wait(bar(S_FREE), ph ^ 1, abort_flag)) break;
         mbar_expect_tx(bar(S_FULL), 4 * kTile);
 #pragma unroll
@@ -203,7 +215,7 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         pend_v = 1 + (int)ph;
       }
       if (*abort_flag) {
-        if (pend_qk) mbar_wait(bar(QK_FULL), pend_qk - 1, abort_flag + 1);
+        if (pend_qk) mbar_wait(bar(pend_qk_bar), pend_qk - 1, abort_flag + 1);
         if (pend_s) mbar_wait(bar(S_FULL), pend_s - 1, abort_flag + 1);
         if (pend_v) mbar_wait(bar(V_FULL), pend_v - 1, abort_flag + 1);
       }
@@ -255,35 +267,42 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       constexpr uint32_t kIdGram = idesc_bf16(64, false);
       constexpr uint32_t kIdMn = idesc_bf16(128, true);
       constexpr uint32_t kIdTf32 = idesc_tf32(128);
-      uint32_t it = 0;
-      for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++it) {
-        const uint32_t ph = it & 1;
-        // Sc = [Q ; K] K^T
-        if (!mbar_wait(bar(QK_FULL), ph, abort_flag)) break;
-        TCD_STAMP(it, 4);
-        if (!mbar_wait(bar(G_FREE), ph ^ 1, abort_flag)) break;
+      // Sc = [Q ; K] K^T of local item j, issued one item ahead of the rest of the chain so that
+      // it runs under the row solve of the item before
+      const uint32_t n_local = p.n_items > (int)blockIdx.x
+                                   ? (uint32_t)((p.n_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x) : 0u;
+      auto gram = [&](uint32_t j) -> bool {
+        const uint32_t qk_base = (j & 1) ? kOffQK1 : kOffQK;
+        if (!mbar_wait(bar((j & 1) ? QK_FULL1 : QK_FULL), (j >> 1) & 1, abort_flag)) return false;
+        TCD_STAMP(j, 4);
+        if (!mbar_wait(bar(G_FREE), (j & 1) ^ 1, abort_flag)) return false;   // score columns read by E1 of j-1
         tc_fence_after();
 #pragma unroll
         for (int h = 0; h < 2; ++h)
 #pragma unroll
           for (int s = 0; s < 4; ++s)
-            mma_bf16_ss(tmem + kColSc, desc_kmajor(sbase + kOffQK + h * kTile + s * 32),
-                        desc_kmajor(sbase + kOffQK + h * kTile + 8192 + s * 32), kIdGram, (h | s) != 0);
+            mma_bf16_ss(tmem + kColSc, desc_kmajor(sbase + qk_base + h * kTile + s * 32),
+                        desc_kmajor(sbase + qk_base + h * kTile + 8192 + s * 32), kIdGram, (h | s) != 0);
         tc_commit(bar(G_DONE));
-        // Qf = [diag(P) | -(W D_P)] [Q ; K]  (rows 64..127: [0 | -(A D_P)])
+        return true;
+      };
+      bool mma_ok = n_local == 0 || gram(0);
+      for (uint32_t it = 0; mma_ok && it < n_local; ++it) {
+        const uint32_t ph = it & 1;
+        const uint32_t qk_base = (it & 1) ? kOffQK1 : kOffQK;
+        if (it + 1 < n_local && !gram(it + 1)) break;
+        // Qf += -(W D_P) K  (rows 64..127: -(A D_P) K); the compute warps initialised Qf with D_P Q
         if (!mbar_wait(bar(W_READY), ph, abort_flag)) break;
         TCD_STAMP(it, 5);
         tc_fence_after();
 #pragma unroll
         for (int part = 0; part < 2; ++part)      // hi, lo
 #pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const uint32_t a_tile = (j < 4 ? kOffAq : kOffAk) + part * kTile + (j & 3) * 32;
-            mma_bf16_ss(tmem + kColQf, desc_kmajor(sbase + a_tile),
-                        desc_mnmajor(sbase + kOffQK + j * 2048, kTile), kIdMn, (part | j) != 0);
-          }
+          for (int j = 4; j < 8; ++j)             // the K rows of the stacked tile
+            mma_bf16_ss(tmem + kColQf, desc_kmajor(sbase + kOffAk + part * kTile + (j & 3) * 32),
+                        desc_mnmajor(sbase + qk_base + j * 2048, kTile), kIdMn, 1);
         tc_commit(bar(D1_DONE));
-        tc_commit(bar(QK_FREE));
+        tc_commit(bar((it & 1) ? QK_FREE1 : QK_FREE));
         // acc = Qf S_pre^T: Qf must be complete in TMEM before it is read as the A operand
         if (!mbar_wait(bar(D1_DONE), ph, abort_flag)) break;
         if (!mbar_wait(bar(S_FULL), ph, abort_flag)) break;
@@ -327,13 +346,6 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
     const uint32_t swz = (uint32_t)(row & 7);
     const uint32_t nswz = (uint32_t)(node & 7);
-
-    // the [diag(P) ; 0] tiles are zero except for the diagonal, which E2 rewrites per item
-    {
-      const uint4 z = make_uint4(0u, 0u, 0u, 0u);
-      uint4* aq = reinterpret_cast<uint4*>(sm + kOffAq);
-      for (int i = tid - 64; i < (int)(2 * kTile / 16); i += kComputeWarps * 32) aq[i] = z;
-    }
 
     uint64_t nm = 0;
     float nal = 1.f, nbe = 0.f;
@@ -408,6 +420,10 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       pk = npk;
       const int Tb = PACKED ? pk.n : T;                       // real nodes of this item
       const bool live_i = live && node < Tb;
+      // Every warp has finished the row solve of the previous item (it read the slot tables and
+      // the per-node tables that this item is about to overwrite; with the Gram product issued one
+      // item ahead, nothing else would hold a fast warp back).
+      if (it > 0 && !(ok = mbar_wait_warp(bar(W_READY), (it - 1) & 1, abort_flag))) break;
       if (warp == 4) TCD_STAMP(it, 16);
       // ---- per-node tables of this item ----
       const uint64_t m = node < Tb ? nm : 0ull;               // strict ancestors
@@ -503,7 +519,8 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         if (pk.row0 + kRows > total_rows) {
           if (!(ok = mbar_wait_warp(bar(V_FULL), ph, abort_flag))) break;
           if (node >= total_rows - pk.row0 && !(part == 1 && hc == 1)) {
-            const uint32_t base = part == 1 ? kOffV : hc == 0 ? kOffQK : kOffQK + 8192;
+            const uint32_t qk_base = (it & 1) ? kOffQK1 : kOffQK;
+            const uint32_t base = part == 1 ? kOffV : hc == 0 ? qk_base : qk_base + 8192;
             const uint4 z = make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
             for (int tile = 0; tile < 2; ++tile)
@@ -514,7 +531,7 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         }
       }
       if (live_i) {
-        // hc 0 writes the [W ; A] tiles, hc 1 the -[W D_P ; A D_P] tiles (and the diagonal of P)
+        // hc 0 writes the [W ; A] tiles, hc 1 the -[W D_P ; A D_P] tiles
         unsigned char* trow = sm + (hc == 0 ? kOffW : kOffAk) + row * 128;
         const uint4 z = make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
@@ -535,14 +552,36 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             *reinterpret_cast<uint16_t*>(trow + kTile + off) = lo;
           }
         }
-        if (part == 0 && hc == 1) {
-          uint16_t hi, lo;
-          split_bf16(fast_exp2(gi), hi, lo);                              // P_i on the diagonal
-          const uint32_t off = row * 128 + ((((uint32_t)node >> 3) ^ swz) << 4) + ((uint32_t)node & 7u) * 2u;
-          *reinterpret_cast<uint16_t*>(sm + kOffAq + off) = hi;
-          *reinterpret_cast<uint16_t*>(sm + kOffAq + kTile + off) = lo;
-        }
       }
+      // Qf starts as D_P Q (rows of the O problem; P_i in full fp32) or 0 (rows of the U problem):
+      // the key-product MMA accumulates -(W D_P) K on top.  The state MMA of the previous item
+      // must have read the old Qf first.
+      if (it > 0 && !(ok = mbar_wait_warp(bar(S_FREE), (it - 1) & 1, abort_flag))) break;
+      // the Q rows are read by these threads: observe the load's barrier themselves
+      if (!(ok = mbar_wait_warp(bar((it & 1) ? QK_FULL1 : QK_FULL), (it >> 1) & 1, abort_flag))) break;
+      if (warp_live) {
+        const bool use_q = live_i && part == 0;
+        const float Pi = use_q ? fast_exp2(gi) : 0.f;
+        const unsigned char* qrow = sm + ((it & 1) ? kOffQK1 : kOffQK) + hc * kTile + node * 128;
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          uint32_t r[32];
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            const uint4 x = *reinterpret_cast<const uint4*>(qrow + (((uint32_t)(half * 4 + c) ^ nswz) << 4));
+            const uint32_t w4[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              // select, never 0 * x: rows past the request may hold anything
+              r[c * 8 + 2 * e] = use_q ? __float_as_uint(Pi * __uint_as_float(w4[e] << 16)) : 0u;
+              r[c * 8 + 2 * e + 1] = use_q ? __float_as_uint(Pi * __uint_as_float(w4[e] & 0xffff0000u)) : 0u;
+            }
+          }
+          tmem_st32(tmem + lane_addr + kColQf + hc * 64 + half * 32, r);
+        }
+        tmem_wait_st();
+      }
+      tc_fence_before();
       fence_async_smem();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(W_READY));
