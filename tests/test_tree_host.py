@@ -128,3 +128,43 @@ def test_library_exports_every_declared_symbol():
     L = tv.lib()
     for n in names:
         assert hasattr(L, n), f"{n} declared in tree_verify.h but not exported"
+
+
+def test_forest_build_host_metadata_and_errors():
+    """tv_forest_build is host-only: per-request metadata equals the oracle's on each tree, padding
+    entries are empty, paths come out per request, malformed input is refused with the right code."""
+    from oracle import tree_oracle as orc
+    rng = np.random.default_rng(11)
+    trees = []
+    for n in (1, 7, 40, 23):
+        par = np.full(n, -1, dtype=np.int32)
+        for i in range(1, n):
+            par[i] = rng.integers(-1, i)
+        trees.append(par)
+    f = tv.forest_build(trees, n_max=40, capacity=100)
+    assert f.n_trees == 4 and f.n == 40 and f.capacity == 100
+    assert f.offsets.tolist() == [0, 1, 8, 48, 71]
+    anc, depth, md = f.meta()
+    for b, par in enumerate(trees):
+        ra, rd, rm = orc.tree_metadata(par)
+        n = len(par)
+        assert np.array_equal(anc[b, :n], ra) and np.array_equal(depth[b, :n], rd) and md[b] == rm
+        assert not anc[b, n:].any() and not depth[b, n:].any()
+    acc = np.array([0, 6, -1, 22], dtype=np.int32)
+    path, ln = f.path(acc)
+    for b, par in enumerate(trees):
+        ref = orc.path_to(par, int(acc[b])) if acc[b] >= 0 else []
+        assert path[b, :ln[b]].tolist() == list(ref) and ln[b] == len(ref)
+    f.rebuild_forest(trees[::-1][1:] + [trees[0]])       # other sizes, same shape limits
+    assert f.offsets.tolist() == [0, 40, 47, 48, 49]
+    for bad, code in (([np.array([-1, 0]), np.array([], dtype=np.int32)], -1),      # empty request
+                      ([np.array([-1, 2, 0])], -2)):                                  # parent after child
+        with pytest.raises(tv.TreeVerifyError) as e:
+            tv.forest_build(bad, n_max=8, capacity=16)
+        assert e.value.status == code
+    with pytest.raises(tv.TreeVerifyError) as e:
+        tv.forest_build(trees, n_max=39)
+    assert e.value.status == -1
+    with pytest.raises(tv.TreeVerifyError) as e:
+        tv.forest_build(trees, n_max=40, capacity=70)
+    assert e.value.status == -8
