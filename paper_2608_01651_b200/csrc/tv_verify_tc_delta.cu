@@ -13,8 +13,9 @@
 // A = N D_beta come from ONE back-substitution each on the path-restricted unit
 // lower-triangular system (w L = c, x L = e_d; L = I + G on the path): d^2/2
 // FMAs per row, no T x T product, no Neumann rounds, no level barriers.  All
-// decay factors are exp2 of differences of log-gate prefix sums along the row's
-// own path, i.e. only ever formed on ancestor pairs.
+// decay factors are products of alpha over a stretch of the row's own path
+// (P_t / P_s for ancestors s < t, never a quotient of two underflowing
+// numbers), built up one factor at a time beside the back-substitution.
 //
 // Tile rows 0..63 carry the O problem of node i, rows 64..127 the U problem of
 // node i (the M = 128 MMA shape is otherwise half empty at T <= 64).  Q and K
@@ -28,7 +29,9 @@
 //     O = acc[0..63], U = acc[64..127]
 // The [Q ; K] tile is double-buffered and its Gram product is issued one item ahead, so the load
 // and the product of item n+1 run under the row solve of item n; what bounds an item is then the
-// CUDA-core chain E1 -> output staging of the previous item -> E2 (about 4.5 us).
+// CUDA-core chain of the eight compute warps: E1 -> path gather -> output staging of the previous
+// item -> back-substitution -> Qf initialisation -> operand tiles.  Loads, MMA issue, output
+// stores and the per-item tables (masks, gates) each have a warp of their own.
 // S_pre goes TMA -> shared memory -> tensor core untouched; O and U leave
 // through swizzled staging chunks and TMA stores.  Every wait is a bounded
 // mbarrier wait (status word on expiry); no TMA multicast.
@@ -38,7 +41,7 @@ namespace {
 
 using namespace tvtc;
 
-constexpr int kThreads = 320;
+constexpr int kThreads = 384;     // producer, MMA issuer, 8 compute warps, output-store warp, metadata warp
 constexpr int kComputeWarps = 8;
 constexpr int kSlots = 16;     // path slots per node: depth <= 15
 constexpr int kRows = 64;      // T <= 64
@@ -56,15 +59,16 @@ constexpr uint32_t kOffStage = kOffAk;           // 8 output chunks of 8 KiB (O:
 constexpr uint32_t kOffGs = kOffV + 8192;        // float Gs[64][kLd]: raw K K^T on the path
 constexpr uint32_t kOffCs = kOffV + kTile + 8192;  // float Cs[64][kLd]: raw Q K^T on the path
 constexpr uint32_t kOffPs = kOffCs + 4352;       // uint8 Ps[64][kLdP]: path nodes
-constexpr uint32_t kOffSmall = kOffPs + 1280;    // float la[64] (log2 alpha), be[64]
+constexpr uint32_t kOffSmall = kOffPs + 1280;    // 2 buffers x {float al[64] (alpha), be[64] (beta)}
+constexpr uint32_t kOffMeta = kOffGs + 4352;     // 2 buffers x uint64 strict-ancestor mask [64]
 constexpr uint32_t kOffBar = 14 * kTile;
 constexpr uint32_t kOffMisc = kOffBar + 8 * 24;
 constexpr uint32_t kSmemBytes = kOffMisc + 64 + 1024;
 
 enum Bar {
   QK_FULL = 0, QK_FREE, S_FULL, S_FREE, V_FULL, V_FREE,
-  G_DONE, G_FREE, W_READY, D1_DONE, ACC_DONE, ACC_FREE, SETUP, E1_SYNC,
-  OST_READY, OST_FREE, QK_FULL1, QK_FREE1
+  G_DONE, G_FREE, W_READY, D1_DONE, ACC_DONE, ACC_FREE, E1_SYNC,
+  OST_READY, OST_FREE, QK_FULL1, QK_FREE1, META_FULL, META_FULL1, META_FREE, META_FREE1
 };
 
 constexpr uint32_t kColSc = 0, kColQf = 128, kColAcc = 256;
@@ -97,14 +101,6 @@ struct DeltaParams {
   float* U;
 };
 
-// 2^x in one MUFU instruction (2 ulp; denormal results flush to zero, which is what a decay
-// factor below 2^-126 should do).  The decay exponents are sums of log2(alpha) along a path.
-__device__ __forceinline__ float fast_exp2(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-
 // bf16 hi/lo parts of x (hi = upper 16 bits, lo = upper 16 bits of the exact remainder)
 __device__ __forceinline__ void split_bf16(float x, uint16_t& hi, uint16_t& lo) {
   const uint32_t b = __float_as_uint(x);
@@ -136,8 +132,8 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   float* Gs = reinterpret_cast<float*>(sm + kOffGs);
   float* Cs = reinterpret_cast<float*>(sm + kOffCs);
   uint8_t* Ps = reinterpret_cast<uint8_t*>(sm + kOffPs);
-  float* la_s = reinterpret_cast<float*>(sm + kOffSmall);
-  float* be_s = la_s + kRows;
+  float* tab_s = reinterpret_cast<float*>(sm + kOffSmall);       // [2][la[64], be[64]]
+  uint64_t* mask_s = reinterpret_cast<uint64_t*>(sm + kOffMeta);   // [2][64]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + kOffMisc);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + kOffMisc + 4);
   auto bar = [&](int i) { return sbase + kOffBar + 8u * i; };
@@ -157,7 +153,8 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     mbar_init(bar(W_READY), kComputeWarps);
     mbar_init(bar(D1_DONE), 1);
     mbar_init(bar(ACC_DONE), 1); mbar_init(bar(ACC_FREE), kComputeWarps);
-    mbar_init(bar(SETUP), kComputeWarps);
+    mbar_init(bar(META_FULL), 1);  mbar_init(bar(META_FULL1), 1);
+    mbar_init(bar(META_FREE), kComputeWarps); mbar_init(bar(META_FREE1), kComputeWarps);
     mbar_init(bar(E1_SYNC), kComputeWarps);
     mbar_init(bar(OST_READY), kComputeWarps);
     mbar_init(bar(OST_FREE), 1);
@@ -219,47 +216,6 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         if (pend_s) mbar_wait(bar(S_FULL), pend_s - 1, abort_flag + 1);
         if (pend_v) mbar_wait(bar(V_FULL), pend_v - 1, abort_flag + 1);
       }
-    } else if (lane == 1) {
-      // ===================== output stores =====================
-      // Staged chunks of item k leave by TMA; OST_FREE(k) tells the compute warps that the
-      // chunks (which alias the Ak / W operand tiles) have been read and may be rewritten.
-      uint32_t it = 0;
-      for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++it) {
-        if (!mbar_wait(bar(OST_READY), it & 1, abort_flag)) break;
-        if constexpr (PACKED) {
-          // groups of 8 rows, largest boxes first (staging rows start on 1024-byte boundaries)
-          const PackedItem pi = packed_item(p.offsets, p.B, p.H, p.Hk, item);
-          const int full = pi.n & ~7;
-          for (int part = 0; part < (want_U ? 2 : 1); ++part) {
-            const OutMaps& mm = part == 0 ? mapsO : mapsU;
-            int r = 0;
-            auto put = [&](const CUtensorMap* m, int rows_box) {
-              while (full - r >= rows_box) {
-#pragma unroll
-                for (int c = 0; c < 4; ++c)
-                  tma_store_3d(m, sbase + kOffStage + (part * 4 + c) * 8192 + (uint32_t)r * 128u, 32 * c,
-                               pi.row0 + r, pi.plane_v);
-                r += rows_box;
-              }
-            };
-            put(&mm.m64, 64);
-            put(&mm.m32, 32);
-            put(&mm.m16, 16);
-            put(&mm.m8, 8);
-          }
-        } else {
-#pragma unroll
-          for (int c = 0; c < 4; ++c) tma_store_3d(&tmO, sbase + kOffStage + c * 8192, 32 * c, 0, item);
-          if (want_U) {
-#pragma unroll
-            for (int c = 0; c < 4; ++c) tma_store_3d(&tmU, sbase + kOffStage + (4 + c) * 8192, 32 * c, 0, item);
-          }
-        }
-        tma_store_commit();
-        tma_store_wait_read();
-        mbar_arrive(bar(OST_FREE));
-      }
-      tma_store_wait_all();
     }
   } else if (warp == 1) {
     // ===================== MMA issuer =====================
@@ -332,6 +288,91 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         TCD_STAMP(it, 9);
       }
     }
+  } else if (warp == kComputeWarps + 2) {
+    if (lane == 0) {
+      // ===================== output stores =====================
+      // Staged chunks of item k leave by TMA; OST_FREE(k) tells the compute warps that the
+      // chunks (which alias the Ak / W operand tiles) have been read and may be rewritten.
+      uint32_t it = 0;
+      for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++it) {
+        if (!mbar_wait(bar(OST_READY), it & 1, abort_flag)) break;
+        if constexpr (PACKED) {
+          // groups of 8 rows, largest boxes first (staging rows start on 1024-byte boundaries)
+          const PackedItem pi = packed_item(p.offsets, p.B, p.H, p.Hk, item);
+          const int full = pi.n & ~7;
+          for (int part = 0; part < (want_U ? 2 : 1); ++part) {
+            const OutMaps& mm = part == 0 ? mapsO : mapsU;
+            int r = 0;
+            auto put = [&](const CUtensorMap* m, int rows_box) {
+              while (full - r >= rows_box) {
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                  tma_store_3d(m, sbase + kOffStage + (part * 4 + c) * 8192 + (uint32_t)r * 128u, 32 * c,
+                               pi.row0 + r, pi.plane_v);
+                r += rows_box;
+              }
+            };
+            put(&mm.m64, 64);
+            put(&mm.m32, 32);
+            put(&mm.m16, 16);
+            put(&mm.m8, 8);
+          }
+        } else {
+#pragma unroll
+          for (int c = 0; c < 4; ++c) tma_store_3d(&tmO, sbase + kOffStage + c * 8192, 32 * c, 0, item);
+          if (want_U) {
+#pragma unroll
+            for (int c = 0; c < 4; ++c) tma_store_3d(&tmU, sbase + kOffStage + (4 + c) * 8192, 32 * c, 0, item);
+          }
+        }
+        tma_store_commit();
+        tma_store_wait_read();
+        mbar_arrive(bar(OST_FREE));
+      }
+      tma_store_wait_all();
+    }
+  } else if (warp == kComputeWarps + 3) {
+    // ===================== metadata warp =====================
+    // Item j's strict-ancestor masks, alpha and beta go to buffer j & 1 while the compute
+    // warps work on item j-1; the buffer is free once they have finished item j-2.
+    grid_dependency_wait();   // tree metadata and gates may come from the kernels in front
+    uint32_t j = 0;
+    for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++j) {
+      const uint32_t buf = j & 1, use = j >> 1;
+      if (use > 0 && !mbar_wait_warp(bar(buf ? META_FREE1 : META_FREE), (use - 1) & 1, abort_flag)) break;
+      int n = T, tb = 0;
+      size_t g0 = (size_t)item * T;                     // first gate of the item
+      if constexpr (PACKED) {
+        const PackedItem pi = packed_item(p.offsets, p.B, p.H, p.Hk, item);
+        n = pi.n;
+        tb = pi.b;
+        g0 = (size_t)pi.plane_v * p.capacity + pi.row0;
+      } else {
+        tb = p.tree.n_trees == 1 ? 0 : (item / p.H) % p.B;
+      }
+      float* tab = tab_s + buf * (2 * kRows);
+      // all six loads first: one trip to memory, not one per table
+      uint64_t mk[2] = {0ull, 0ull};
+      float al[2] = {1.f, 1.f}, be[2] = {0.f, 0.f};
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int nd = lane + 32 * h;
+        if (nd < n) {
+          mk[h] = __ldg(reinterpret_cast<const unsigned long long*>(p.tree.anc) + ((size_t)tb * T + nd) * 2);
+          al[h] = __ldg(p.alpha + g0 + nd);
+          be[h] = __ldg(p.beta + g0 + nd);
+        }
+      }
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int nd = lane + 32 * h;
+        mask_s[buf * kRows + nd] = mk[h];
+        tab[nd] = al[h];
+        tab[kRows + nd] = be[h];
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(buf ? META_FULL1 : META_FULL));
+    }
   } else {
     // ===================== compute warps =====================
     const int cw = warp - 2;
@@ -347,33 +388,18 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     const uint32_t swz = (uint32_t)(row & 7);
     const uint32_t nswz = (uint32_t)(node & 7);
 
-    uint64_t nm = 0;
-    float nal = 1.f, nbe = 0.f;
+    // Ancestor masks, alpha and beta of every item are put into shared memory by the
+    // metadata warp, one item ahead (META_FULL / META_FREE, two buffers).
     PackedItem npk = {0, 0, 0, 0, T};   // packed forest: rows of the next item
-    auto fetch_meta = [&](int item) {
-      nm = 0; nal = 1.f; nbe = 0.f;
+    auto next_rows = [&](int item) {
       if constexpr (PACKED) {
-        if (item < p.n_items) {
-          npk = packed_item(p.offsets, p.B, p.H, p.Hk, item);
-          if (node < npk.n) {
-            const size_t r = (size_t)npk.plane_v * p.capacity + npk.row0 + node;
-            nm = p.tree.anc[((size_t)npk.b * T + node) * 2];
-            nal = p.alpha[r];
-            nbe = p.beta[r];
-          }
-        }
-      } else if (item < p.n_items && node < T) {
-        const int b = (item / p.H) % p.B;
-        const int tb = p.tree.n_trees == 1 ? 0 : b;
-        nm = p.tree.anc[((size_t)tb * T + node) * 2];
-        nal = p.alpha[(size_t)item * T + node];
-        nbe = p.beta[(size_t)item * T + node];
+        if (item < p.n_items) npk = packed_item(p.offsets, p.B, p.H, p.Hk, item);
       }
     };
     grid_dependency_wait();   // tree metadata comes from the kernel in front (dependent launch)
     // the commit kernel behind this one may be scheduled as SMs drain (it orders itself)
     if (warp == 2 && lane == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    fetch_meta(blockIdx.x);
+    next_rows(blockIdx.x);
 
     // acc rows 0..63 -> O chunks 0..3, rows 64..127 -> U chunks 4..7 (the chunks alias the Ak / W
     // tiles, which are idle between the readout MMA of item k and E2 of item k+1)
@@ -425,15 +451,12 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       // item ahead, nothing else would hold a fast warp back).
       if (it > 0 && !(ok = mbar_wait_warp(bar(W_READY), (it - 1) & 1, abort_flag))) break;
       if (warp == 4) TCD_STAMP(it, 16);
-      // ---- per-node tables of this item ----
-      const uint64_t m = node < Tb ? nm : 0ull;               // strict ancestors
-      if (part == 0 && hc == 0 && node < Tb) {
-        la_s[node] = log2f(nal);
-        be_s[node] = nbe;
-      }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(SETUP));
-      fetch_meta(item + (int)gridDim.x);
+      // ---- per-node tables of this item (written by the metadata warp) ----
+      if (!(ok = mbar_wait_warp(bar(ph ? META_FULL1 : META_FULL), (it >> 1) & 1, abort_flag))) break;
+      const uint64_t m = node < Tb ? mask_s[ph * kRows + node] : 0ull;   // strict ancestors
+      const float* al_s = tab_s + ph * (2 * kRows);
+      const float* be_s = al_s + kRows;
+      next_rows(item + (int)gridDim.x);
       const int depth = __popcll(m);
 
       // ---- E1: raw path-sparse rows: part 0 <- Q K^T (path incl. the node), part 1 <- K K^T ----
@@ -452,6 +475,7 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
 #pragma unroll
         for (int jj = 0; jj < 32; ++jj) {
           // unselected columns land in the padding slot of the row: no branch, no predicate
+          // (predicated stores of the selected columns only were measured slower)
           const int slot = ((bits >> jj) & 1u) ? base + __popc(bits & ((1u << jj) - 1u)) : kSlots;
           dst[slot] = __uint_as_float(r[jj]);
           if (part == 0) Ps[node * kLdP + slot] = (uint8_t)(cbase + jj);
@@ -464,54 +488,94 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         mbar_arrive(bar(E1_SYNC));
       }
       if (warp == 4) TCD_STAMP(it, 19);
-      // ---- output of the previous item (its MMAs ran under E1 above) ----
-      if (it > 0 && !(ok = final_epilogue(it - 1, pk_prev))) break;
-      if (warp == 4) TCD_STAMP(it, 17);
-      if (!(ok = mbar_wait_warp(bar(SETUP), ph, abort_flag))) break;
       if (!(ok = mbar_wait_warp(bar(E1_SYNC), ph, abort_flag))) break;
       if (warp == 4) TCD_STAMP(it, 20);
 
       // ---- E2: decay factors, one back-substitution per row, operand tiles ----
       constexpr int NS = DMAX + 1;                            // path slots in use
       int path[NS];
-      float gp[NS], bt[NS], vec[NS];
-      float gi = 0.f;
+      float al[NS], bt[NS], pre[NS], vec[NS];
+      float Pi = 1.f;                                         // P_i: product of alpha along the path
       if (live_i) {
         const uint32_t* pw = reinterpret_cast<const uint32_t*>(Ps + node * kLdP);
         const uint32_t pword[4] = {pw[0], pw[1], pw[2], pw[3]};
-        float run = 0.f;
 #pragma unroll
         for (int s2 = 0; s2 < NS; ++s2) {
           path[s2] = (pword[s2 >> 2] >> ((s2 & 3) * 8)) & 63;
           const bool on = s2 <= depth;
-          const float la = la_s[path[s2]], b2 = be_s[path[s2]];
+          const float a2 = al_s[path[s2]], b2 = be_s[path[s2]];
+          al[s2] = on ? a2 : 1.f;    // slots past the node count as no decay
           bt[s2] = on ? b2 : 0.f;
-          run += on ? la : 0.f;      // log2 of P at path node s2
-          gp[s2] = run;
-          if (s2 == depth) gi = run;
+          Pi *= al[s2];
+          pre[s2] = Pi;              // P at path node s2
         }
+      }
+      if (warp == 4) TCD_STAMP(it, 22);
+      // ---- output of the previous item: its MMAs ran under E1 and the gather above, so the
+      // accumulator is complete by now; the TMA stores that take the staged chunks away read them
+      // under the back-substitution and the Qf initialisation below ----
+      if (it > 0 && !(ok = final_epilogue(it - 1, pk_prev))) break;
+      if (warp == 4) TCD_STAMP(it, 17);
+      if (live_i) {
+        // C_{i,p_s} = (q_i . k_{p_s}) P_i / P_{p_s}: the ratio is the product of alpha over the
+        // slots after s, built up from the node's own slot backwards
+        float sfx = 1.f;
 #pragma unroll
-        for (int s2 = 0; s2 < NS; ++s2) {
+        for (int s2 = NS - 1; s2 >= 0; --s2) {
           const float c = Cs[node * kLd + s2];
-          if (part == 0) vec[s2] = s2 <= depth ? c * fast_exp2(gi - gp[s2]) : 0.f;   // C_{i,p_s}
+          if (part == 0) vec[s2] = s2 <= depth ? c * sfx : 0.f;
           else vec[s2] = s2 == depth ? 1.f : 0.f;                               // x L = e_d
+          sfx *= al[s2];
         }
-        // w_s = c_s - sum_{t > s} w_t G_{p_t,p_s},  G_{p_t,p_s} = beta_t 2^(gp_t - gp_s) k_t.k_s;
-        // slots past the node's depth carry vec = 0 and a deselected G, so nothing is predicated
+        // w_s = c_s - sum_{t > s} w_t G_{p_t,p_s},  G_{p_t,p_s} = beta_t (P_{p_t} / P_{p_s}) k_t.k_s;
+        // rr[t] holds P_{p_t} / P_{p_s} = alpha_{s+1} ... alpha_t for the current s and grows by one
+        // factor per step.  Slots past the node's depth carry vec = 0 and a deselected G, so nothing
+        // is predicated.
+        float rr[NS];
 #pragma unroll
         for (int s2 = NS - 2; s2 >= 0; --s2) {
           float acc = vec[s2];
 #pragma unroll
           for (int t = s2 + 1; t < NS; ++t) {
-            const float gts = Gs[path[t] * kLd + s2] * (bt[t] * fast_exp2(gp[t] - gp[s2]));
+            rr[t] = t == s2 + 1 ? al[t] : rr[t] * al[s2 + 1];
+            const float gts = Gs[path[t] * kLd + s2] * (bt[t] * rr[t]);
             acc = fmaf(-vec[t], t <= depth ? gts : 0.f, acc);
           }
           if (s2 < depth) vec[s2] = acc;
         }
       }
+      // Qf starts as D_P Q (rows of the O problem; P_i in full fp32) or 0 (rows of the U problem):
+      // the key-product MMA accumulates -(W D_P) K on top.  The state MMA of the previous item
+      // must have read the old Qf first.
+      if (it > 0 && !(ok = mbar_wait_warp(bar(S_FREE), (it - 1) & 1, abort_flag))) break;
+      // the Q rows are read by these threads: observe the load's barrier themselves
+      if (!(ok = mbar_wait_warp(bar((it & 1) ? QK_FULL1 : QK_FULL), (it >> 1) & 1, abort_flag))) break;
+      if (warp_live) {
+        const bool use_q = live_i && part == 0;
+        const unsigned char* qrow = sm + ((it & 1) ? kOffQK1 : kOffQK) + hc * kTile + node * 128;
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          uint32_t r[32];
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            const uint4 x = *reinterpret_cast<const uint4*>(qrow + (((uint32_t)(half * 4 + c) ^ nswz) << 4));
+            const uint32_t w4[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              // select, never 0 * x: rows past the request may hold anything
+              r[c * 8 + 2 * e] = use_q ? __float_as_uint(Pi * __uint_as_float(w4[e] << 16)) : 0u;
+              r[c * 8 + 2 * e + 1] = use_q ? __float_as_uint(Pi * __uint_as_float(w4[e] & 0xffff0000u)) : 0u;
+            }
+          }
+          tmem_st32(tmem + lane_addr + kColQf + hc * 64 + half * 32, r);
+        }
+        tmem_wait_st();
+      }
+      if (warp == 4) TCD_STAMP(it, 25);
       // The tiles alias the staged output chunks of the previous item: its stores must have read
-      // them (they did so under the solve above).
+      // them (they did so under the Qf initialisation above).
       if (it > 0 && !(ok = mbar_wait_warp(bar(OST_FREE), (it - 1) & 1, abort_flag))) break;
+      if (warp == 4) TCD_STAMP(it, 23);
       if constexpr (PACKED) {
         // A box that reaches past the last node of the forest brings rows nobody wrote.  They only
         // ever meet zero coefficients, but 0 x garbage need not be 0: zero them.  The Gram MMA has
@@ -544,7 +608,7 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           if (s2 <= depth) {
             const int j = path[s2];
             const float wv = vec[s2] * bt[s2];                        // W = C N D_beta (or A = N D_beta)
-            const float val = hc == 0 ? wv : -(wv * fast_exp2(gp[s2]));   // ... times P_{p_s}, negated
+            const float val = hc == 0 ? wv : -(wv * pre[s2]);            // ... times P_{p_s}, negated
             const uint32_t off = ((((uint32_t)j >> 3) ^ swz) << 4) + ((uint32_t)j & 7u) * 2u;
             uint16_t hi, lo;
             split_bf16(val, hi, lo);
@@ -553,38 +617,14 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           }
         }
       }
-      // Qf starts as D_P Q (rows of the O problem; P_i in full fp32) or 0 (rows of the U problem):
-      // the key-product MMA accumulates -(W D_P) K on top.  The state MMA of the previous item
-      // must have read the old Qf first.
-      if (it > 0 && !(ok = mbar_wait_warp(bar(S_FREE), (it - 1) & 1, abort_flag))) break;
-      // the Q rows are read by these threads: observe the load's barrier themselves
-      if (!(ok = mbar_wait_warp(bar((it & 1) ? QK_FULL1 : QK_FULL), (it >> 1) & 1, abort_flag))) break;
-      if (warp_live) {
-        const bool use_q = live_i && part == 0;
-        const float Pi = use_q ? fast_exp2(gi) : 0.f;
-        const unsigned char* qrow = sm + ((it & 1) ? kOffQK1 : kOffQK) + hc * kTile + node * 128;
-#pragma unroll
-        for (int half = 0; half < 2; ++half) {
-          uint32_t r[32];
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            const uint4 x = *reinterpret_cast<const uint4*>(qrow + (((uint32_t)(half * 4 + c) ^ nswz) << 4));
-            const uint32_t w4[4] = {x.x, x.y, x.z, x.w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              // select, never 0 * x: rows past the request may hold anything
-              r[c * 8 + 2 * e] = use_q ? __float_as_uint(Pi * __uint_as_float(w4[e] << 16)) : 0u;
-              r[c * 8 + 2 * e + 1] = use_q ? __float_as_uint(Pi * __uint_as_float(w4[e] & 0xffff0000u)) : 0u;
-            }
-          }
-          tmem_st32(tmem + lane_addr + kColQf + hc * 64 + half * 32, r);
-        }
-        tmem_wait_st();
-      }
+      if (warp == 4) TCD_STAMP(it, 24);
       tc_fence_before();
       fence_async_smem();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar(W_READY));
+      if (lane == 0) {
+        mbar_arrive(bar(W_READY));
+        mbar_arrive(bar(ph ? META_FREE1 : META_FREE));   // this item's tables may be overwritten
+      }
       if (warp == 4) TCD_STAMP(it, 21);
       pk_prev = pk;
     }
