@@ -297,10 +297,11 @@ int tv_commit_path(const tv_tree* tree, const tv_dims* dims,
  * tv_session_round copies parent/accepted/S_pre/q/k/v/alpha/beta to the device,
  * verifies, commits in place on the device copy (the delta rule commits from
  * the corrections U that verify wrote), copies O and S_new back and
- * synchronises before returning.  The requests are handled in up to four
- * groups on two streams of the session's own (ordered after the work already
- * queued on `stream`, and `stream` waits for them), so that the copies in, the
- * kernels and the copies out of different groups overlap.  All pointers are
+ * synchronises before returning.  The requests are handled in up to eight
+ * groups that flow through three streams of the session's own -- copies in,
+ * kernels, copies out, chained by events per group; all ordered after the work
+ * already queued on `stream`, and `stream` waits for them -- so that the
+ * copies in, the kernels and the copies out of different groups overlap.  All pointers are
  * host pointers in the layouts above; beta may be NULL for TV_GATED.           */
 typedef struct tv_session tv_session;
 int tv_session_create(const tv_dims* dims, int32_t n_trees, tv_session** out);
