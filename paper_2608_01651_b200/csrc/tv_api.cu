@@ -401,11 +401,13 @@ TV_API int tv_tree_verify(const tv_tree* tree, const tv_dims* d, const float* S_
   a.L = d->L; a.B = d->B; a.H = d->H; a.T = d->T; a.dk = d->dk; a.dv = d->dv;
   a.rule = d->rule; a.bf16 = d->qkv_dtype == TV_BF16; a.Hk = d->Hk ? d->Hk : d->H;
   a.S_pre = S_pre; a.q = q; a.k = k; a.v = v; a.alpha = alpha; a.beta = beta; a.O = O; a.U = U;
-  const bool tc_gated = tv_verify_tc_supports(a), tc_delta = tv_verify_tc_delta_supports(a);
-  if (d->impl == TV_IMPL_TC && !tc_gated && !tc_delta) return TV_ERR_UNSUPPORTED;
+  const bool tc_gated = tv_verify_tc_supports(a), tc_delta = tv_verify_tc_delta_supports(a),
+             tc_delta128 = tv_verify_tc_delta128_supports(a);
+  if (d->impl == TV_IMPL_TC && !tc_gated && !tc_delta && !tc_delta128) return TV_ERR_UNSUPPORTED;
   if (d->impl != TV_IMPL_SIMT) {
     if (tc_gated) return tv_launch_verify_tc(a, tree->d_status, (cudaStream_t)stream);
     if (tc_delta) return tv_launch_verify_tc_delta(a, tree->d_status, (cudaStream_t)stream);
+    if (tc_delta128) return tv_launch_verify_tc_delta128(a, tree->d_status, (cudaStream_t)stream);
   }
   return tv_launch_verify_simt(a, (cudaStream_t)stream);
 }

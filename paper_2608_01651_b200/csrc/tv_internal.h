@@ -130,6 +130,8 @@ bool tv_verify_tc_supports(const VerifyArgs& a);
 int tv_launch_verify_tc(const VerifyArgs& a, int32_t* status, cudaStream_t stream);
 bool tv_verify_tc_delta_supports(const VerifyArgs& a);
 int tv_launch_verify_tc_delta(const VerifyArgs& a, int32_t* status, cudaStream_t stream);
+bool tv_verify_tc_delta128_supports(const VerifyArgs& a);   // 64 < T <= 128, dense layout
+int tv_launch_verify_tc_delta128(const VerifyArgs& a, int32_t* status, cudaStream_t stream);
 
 #define TV_CUDA_TRY(expr)                 \
   do {                                    \

@@ -1,0 +1,575 @@
+// Tree verification of the gated delta rule on the tensor cores for trees of 65..128 nodes
+// (bf16 q/k/v, fp32 state, dk = dv = 128, tree depth <= 15, dense batch layout).
+//
+// Same algebra as tv_verify_tc_delta.cu (Theorem 1, Eq. 2, regrouped so that the state is
+// contracted once; Lemma 2/3 for N = (I+G)^-1; one back-substitution per row on the
+// path-restricted triangular system):
+//     O = Q_eff S_pre^T + W V,   Q_eff = D_P Q - (W D_P) K,   W = C N D_beta
+//     U = A V - K_eff S_pre^T,   K_eff = (A D_P) K,           A = N D_beta
+// With up to 128 nodes the 2T row problems no longer fit one M = 128 tile, and the T x T
+// coefficient matrices no longer fit shared memory next to Q, K, V and S_pre.  The item is
+// therefore worked on in two ROW BLOCKS of 64 nodes (block 0: nodes 0..63, block 1: nodes
+// 64..127; tile rows 0..63 = O problems, rows 64..127 = U problems of the block's nodes), and
+// every coefficient matrix is built and consumed in COLUMN HALVES of 64 ancestors through one
+// [128 x 64] bf16 hi/lo tile pair.  Nodes are numbered parent before child, so block 0 only has
+// ancestors in column half 0; block 1 has them in both.  Per block:
+//     Sc   = [Q_b ; K_b] K^T             (Gram rows of the block against all earlier nodes)
+//     E1:    path-sparse raw rows of C (block rows) and G (kept for all 128 nodes)
+//     solve: one back-substitution per row, decay ratios as running products of alpha
+//     Qf   = D_P Q_b (written to TMEM by the compute warps)
+//          + sum over column halves h of [-(W D_P) ; -(A D_P)]_h K_h          (bf16 hi/lo)
+//     acc  = Qf S_pre^T (tf32, A operand from TMEM) + sum over h of [W ; A]_h V_h
+//     O rows and U rows of the block leave from registers.
+// The Gram products of both blocks are issued as soon as Q and K have landed; the output of a
+// block is read out after the row solve of the next block (of the next item for block 1), when
+// its MMAs are long complete.  Eleven warps: TMA producer, MMA issuer, eight compute warps, one
+// warp that stages the next item's ancestor masks and gates.  Every wait is a bounded mbarrier wait; no TMA multicast.
+#include "tv_tc_common.cuh"
+
+namespace {
+
+using namespace tvtc;
+
+constexpr int kThreads = 352;
+constexpr int kComputeWarps = 8;
+constexpr int kSlots = 16;     // path slots per node: depth <= 15
+constexpr int kNodes = 128;    // T <= 128
+constexpr int kBlk = 64;       // nodes per row block
+constexpr int kLd = 17;        // row stride of the slot tables (floats): conflict-free per slot
+constexpr int kLdP = 20;       // row stride of the path table (bytes)
+
+// shared memory map (bytes from the 1024-aligned base); 12 tiles of 128 rows x 128 B, then tables
+constexpr uint32_t kOffQK0 = 0;                  // [Q_0 ; K_0]: 2 dk-halves, rows 0..63 Q, rows 64..127 K
+constexpr uint32_t kOffQK1 = 2 * kTile;          // [Q_1 ; K_1]
+constexpr uint32_t kOffV = 4 * kTile;            // 2 dv-halves of V, rows = nodes 0..127
+constexpr uint32_t kOffS = 6 * kTile;            // 4 k-chunks of S_pre [128 v][32] f32
+constexpr uint32_t kOffCoef = 10 * kTile;        // hi, lo of the current coefficient tile [128][64] bf16
+constexpr uint32_t kOffGs = 12 * kTile;          // float Gs[128][kLd]: raw K K^T on the path, all nodes
+constexpr uint32_t kOffCs = kOffGs + 8704;       // float Cs[64][kLd]: raw Q K^T on the path, block rows
+constexpr uint32_t kOffPs = kOffCs + 4352;       // uint8 Ps[64][kLdP]: path nodes of the block's rows
+constexpr uint32_t kOffTab = kOffPs + 1280;      // 2 buffers x {float alpha[128], beta[128]}
+constexpr uint32_t kOffMask = kOffTab + 2048;    // 2 buffers x [128] x {uint64 lo, hi} strict ancestors
+constexpr uint32_t kOffBar = kOffMask + 4096;
+constexpr uint32_t kOffMisc = kOffBar + 8 * 32;
+constexpr uint32_t kSmemBytes = kOffMisc + 64 + 1024;
+
+enum Bar {
+  QK_FULL = 0, QK_FREE, S_FULL, S_FREE, V_FULL, V_FREE,
+  GD0, GD1, GF0, GF1, TILE_READY, TILE_FREE, D1_DONE, QF_FREE, ACC_DONE, ACC_FREE, E1_SYNC,
+  META_FULL, META_FULL1, META_FREE, META_FREE1
+};
+
+constexpr uint32_t kColSc0 = 0, kColQf = 128, kColAcc = 256, kColSc1 = 384;
+
+struct Delta128Params {
+  TreeDev tree;
+  int32_t n_items, B, H, T;
+  int32_t Hk;  // q/k heads (grouped key heads); H when not grouped
+  const float* alpha;
+  const float* beta;
+  int32_t want_U;
+  int32_t* status;
+  float* O;
+  float* U;
+};
+
+// bf16 hi/lo parts of x (hi = upper 16 bits, lo = upper 16 bits of the exact remainder)
+__device__ __forceinline__ void split_bf16(float x, uint16_t& hi, uint16_t& lo) {
+  const uint32_t b = __float_as_uint(x);
+  const uint32_t h = b & 0xffff0000u;
+  hi = (uint16_t)(h >> 16);
+  lo = (uint16_t)(__float_as_uint(x - __uint_as_float(h)) >> 16);
+}
+
+// DMAX: compile-time bound on the tree depth (8 covers draft trees, 15 the rest), so that the
+// per-row triangular solve is straight-line code whose loads all issue up front.
+template <int DMAX>
+__global__ void __launch_bounds__(kThreads, 1)
+verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                          const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmS,
+                          const Delta128Params p) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* sm = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  const uint32_t sbase = smem_u32(sm);
+  float* Gs = reinterpret_cast<float*>(sm + kOffGs);
+  float* Cs = reinterpret_cast<float*>(sm + kOffCs);
+  uint8_t* Ps = reinterpret_cast<uint8_t*>(sm + kOffPs);
+  float* tab_s = reinterpret_cast<float*>(sm + kOffTab);              // [2][alpha[128], beta[128]]
+  ulonglong2* mask_s = reinterpret_cast<ulonglong2*>(sm + kOffMask);  // [2][128]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + kOffMisc);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + kOffMisc + 4);
+  auto bar = [&](int i) { return sbase + kOffBar + 8u * i; };
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int T = p.T;
+  const bool want_U = p.want_U != 0;
+
+  if (tid == 0) {
+    abort_flag[0] = 0;
+    abort_flag[1] = 0;
+    mbar_init(bar(QK_FULL), 1);  mbar_init(bar(QK_FREE), 1 + kComputeWarps);
+    mbar_init(bar(S_FULL), 1);   mbar_init(bar(S_FREE), 1);
+    mbar_init(bar(V_FULL), 1);   mbar_init(bar(V_FREE), 1);
+    mbar_init(bar(GD0), 1);      mbar_init(bar(GD1), 1);
+    mbar_init(bar(GF0), kComputeWarps); mbar_init(bar(GF1), kComputeWarps);
+    mbar_init(bar(TILE_READY), kComputeWarps); mbar_init(bar(TILE_FREE), 1);
+    mbar_init(bar(D1_DONE), 1);  mbar_init(bar(QF_FREE), 1);
+    mbar_init(bar(ACC_DONE), 1); mbar_init(bar(ACC_FREE), kComputeWarps);
+    mbar_init(bar(E1_SYNC), kComputeWarps);
+    mbar_init(bar(META_FULL), 1);  mbar_init(bar(META_FULL1), 1);
+    mbar_init(bar(META_FREE), kComputeWarps); mbar_init(bar(META_FREE1), kComputeWarps);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(tmem_slot)), "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      // ===================== TMA producer =====================
+      int pend_qk = 0, pend_s = 0, pend_v = 0;
+      uint32_t it = 0;
+      grid_dependency_wait();   // inputs may come from the kernel in front (dependent launch)
+      for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++it) {
+        const uint32_t ph = it & 1;
+        const int qk = tv_qk_item(item, p.H, p.Hk);
+        if (!mbar_wait(bar(QK_FREE), ph ^ 1, abort_flag)) break;
+        mbar_expect_tx(bar(QK_FULL), 8 * 8192);
+#pragma unroll
+        for (int h = 0; h < 2; ++h)        // row block
+#pragma unroll
+          for (int d = 0; d < 2; ++d) {    // dk half
+            const uint32_t dst = sbase + (h ? kOffQK1 : kOffQK0) + d * kTile;
+            tma_load_3d(dst, &tmQ, bar(QK_FULL), 64 * d, 64 * h, qk);
+            tma_load_3d(dst + 8192, &tmK, bar(QK_FULL), 64 * d, 64 * h, qk);
+          }
+        pend_qk = 1 + (int)ph;
+        if (!mbar_wait(bar(S_FREE), ph ^ 1, abort_flag)) break;
+        mbar_expect_tx(bar(S_FULL), 4 * kTile);
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+          tma_load_3d(sbase + kOffS + c * kTile, &tmS, bar(S_FULL), 32 * c, 0, item);
+        pend_s = 1 + (int)ph;
+        if (!mbar_wait(bar(V_FREE), ph ^ 1, abort_flag)) break;
+        mbar_expect_tx(bar(V_FULL), 4 * 8192);
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+#pragma unroll
+          for (int d = 0; d < 2; ++d)
+            tma_load_3d(sbase + kOffV + d * kTile + h * 8192, &tmV, bar(V_FULL), 64 * d, 64 * h, item);
+        pend_v = 1 + (int)ph;
+      }
+      if (*abort_flag) {
+        if (pend_qk) mbar_wait(bar(QK_FULL), pend_qk - 1, abort_flag + 1);
+        if (pend_s) mbar_wait(bar(S_FULL), pend_s - 1, abort_flag + 1);
+        if (pend_v) mbar_wait(bar(V_FULL), pend_v - 1, abort_flag + 1);
+      }
+    }
+  } else if (warp == 1) {
+    // ===================== MMA issuer =====================
+    if (lane == 0) {
+      constexpr uint32_t kIdGram = idesc_bf16(64, false);
+      constexpr uint32_t kIdMn = idesc_bf16(128, true);
+      constexpr uint32_t kIdTf32 = idesc_tf32(128);
+      uint32_t it = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; ok && item < p.n_items; item += gridDim.x, ++it) {
+        const uint32_t ph = it & 1;
+        // ---- Gram products of both row blocks: Sc_b = [Q_b ; K_b] K^T over the columns 0..64(b+1) ----
+        if (!(ok = mbar_wait(bar(QK_FULL), ph, abort_flag))) break;
+        if (!(ok = mbar_wait(bar(GF0), ph ^ 1, abort_flag))) break;   // score columns read by E1 of the item before
+        tc_fence_after();
+#pragma unroll
+        for (int d = 0; d < 2; ++d)
+#pragma unroll
+          for (int s = 0; s < 4; ++s)
+            mma_bf16_ss(tmem + kColSc0, desc_kmajor(sbase + kOffQK0 + d * kTile + s * 32),
+                        desc_kmajor(sbase + kOffQK0 + d * kTile + 8192 + s * 32), kIdGram, (d | s) != 0);
+        tc_commit(bar(GD0));
+        if (!(ok = mbar_wait(bar(GF1), ph ^ 1, abort_flag))) break;
+        tc_fence_after();
+#pragma unroll
+        for (int nh = 0; nh < 2; ++nh)   // column half = K rows of block nh
+#pragma unroll
+          for (int d = 0; d < 2; ++d)
+#pragma unroll
+            for (int s = 0; s < 4; ++s)
+              mma_bf16_ss(tmem + kColSc1 + 64 * nh, desc_kmajor(sbase + kOffQK1 + d * kTile + s * 32),
+                          desc_kmajor(sbase + (nh ? kOffQK1 : kOffQK0) + d * kTile + 8192 + s * 32), kIdGram,
+                          (d | s) != 0);
+        tc_commit(bar(GD1));
+
+        for (int b = 0; ok && b < 2; ++b) {
+          // ---- Qf += [-(W D_P) ; -(A D_P)]_h K_h, one coefficient tile per column half ----
+          for (int h = 0; h <= b; ++h) {
+            const uint32_t j = b == 0 ? 0u : 2u + h;   // build number within the item (6 builds)
+            if (!(ok = mbar_wait(bar(TILE_READY), j & 1, abort_flag))) break;
+            tc_fence_after();
+            const uint32_t kb = h ? kOffQK1 : kOffQK0;
+#pragma unroll
+            for (int part = 0; part < 2; ++part)      // hi, lo
+#pragma unroll
+              for (int s = 0; s < 4; ++s)             // 16 ancestors per step: the K rows of the stacked tile
+                mma_bf16_ss(tmem + kColQf, desc_kmajor(sbase + kOffCoef + part * kTile + s * 32),
+                            desc_mnmajor(sbase + kb + (4 + s) * 2048, kTile), kIdMn, 1);
+            tc_commit(bar(TILE_FREE));
+          }
+          if (!ok) break;
+          tc_commit(bar(D1_DONE));
+          if (b == 1) tc_commit(bar(QK_FREE));
+          // acc = Qf S_pre^T: Qf must be complete in TMEM before it is read as the A operand
+          if (!(ok = mbar_wait(bar(D1_DONE), (uint32_t)b, abort_flag))) break;
+          if (b == 0 && !(ok = mbar_wait(bar(S_FULL), ph, abort_flag))) break;
+          if (!(ok = mbar_wait(bar(ACC_FREE), (uint32_t)b ^ 1, abort_flag))) break;   // read-out of the block before
+          tc_fence_after();
+#pragma unroll
+          for (int c = 0; c < 4; ++c)
+#pragma unroll
+            for (int s = 0; s < 4; ++s)
+              mma_tf32_ts(tmem + kColAcc, tmem + kColQf + c * 32 + s * 8,
+                          desc_kmajor(sbase + kOffS + c * kTile + s * 32), kIdTf32, (c | s) != 0);
+          tc_commit(bar(QF_FREE));
+          if (b == 1) tc_commit(bar(S_FREE));
+          // ---- acc += [W ; A]_h V_h ----
+          if (b == 0 && !(ok = mbar_wait(bar(V_FULL), ph, abort_flag))) break;
+          for (int h = 0; h <= b; ++h) {
+            const uint32_t j = b == 0 ? 1u : 4u + h;
+            if (!(ok = mbar_wait(bar(TILE_READY), j & 1, abort_flag))) break;
+            tc_fence_after();
+#pragma unroll
+            for (int s = 0; s < 4; ++s) {
+              const uint64_t bdesc = desc_mnmajor(sbase + kOffV + (4 * h + s) * 2048, kTile);
+              mma_bf16_ss(tmem + kColAcc, desc_kmajor(sbase + kOffCoef + s * 32), bdesc, kIdMn, 1);
+              mma_bf16_ss(tmem + kColAcc, desc_kmajor(sbase + kOffCoef + kTile + s * 32), bdesc, kIdMn, 1);
+            }
+            tc_commit(bar(TILE_FREE));
+          }
+          if (!ok) break;
+          tc_commit(bar(ACC_DONE));
+          if (b == 1) tc_commit(bar(V_FREE));
+        }
+      }
+    }
+  } else if (warp == kComputeWarps + 2) {
+    // ===================== metadata warp =====================
+    // Item j's strict-ancestor masks, alpha and beta go to buffer j & 1 while the compute warps
+    // work on item j-1; the buffer is free once they have finished item j-2.
+    grid_dependency_wait();   // tree metadata and gates may come from the kernels in front
+    uint32_t j = 0;
+    for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++j) {
+      const uint32_t buf = j & 1, use = j >> 1;
+      if (use > 0 && !mbar_wait_warp(bar(buf ? META_FREE1 : META_FREE), (use - 1) & 1, abort_flag)) break;
+      const int tb = p.tree.n_trees == 1 ? 0 : (item / p.H) % p.B;
+      const size_t g0 = (size_t)item * T;   // first gate of the item
+      float* tab = tab_s + buf * (2 * kNodes);
+      // all loads first: one trip to memory, not one per table
+      ulonglong2 mk[4];
+      float al[4], be[4];
+#pragma unroll
+      for (int h = 0; h < 4; ++h) {
+        const int nd = lane + 32 * h;
+        mk[h] = make_ulonglong2(0ull, 0ull);
+        al[h] = 1.f;
+        be[h] = 0.f;
+        if (nd < T) {
+          mk[h] = __ldg(reinterpret_cast<const ulonglong2*>(p.tree.anc) + (size_t)tb * T + nd);
+          al[h] = __ldg(p.alpha + g0 + nd);
+          be[h] = __ldg(p.beta + g0 + nd);
+        }
+      }
+#pragma unroll
+      for (int h = 0; h < 4; ++h) {
+        const int nd = lane + 32 * h;
+        mask_s[buf * kNodes + nd] = mk[h];
+        tab[nd] = al[h];
+        tab[kNodes + nd] = be[h];
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(buf ? META_FULL1 : META_FULL));
+    }
+  } else if (warp >= 2 && warp < 2 + kComputeWarps) {
+    // ===================== compute warps =====================
+    const int cw = warp - 2;
+    const int quad = warp & 3;
+    const int hc = cw >> 2;                 // which of the two threads of a row
+    const int row = quad * 32 + lane;       // tile row
+    const int rn = row & 63;                // node of this row within its block
+    const int part = row >> 6;              // 0: O problem, 1: U problem
+    const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+    const uint32_t swz = (uint32_t)(row & 7);
+    const uint32_t nswz = (uint32_t)(rn & 7);
+
+    grid_dependency_wait();   // nothing is read before the kernels in front have finished
+    // the commit kernel behind this one may be scheduled as SMs drain (it orders itself)
+    if (warp == 2 && lane == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
+    // acc rows 0..63 -> O rows, rows 64..127 -> U rows of block pb of item pitem, straight from
+    // registers (each thread owns 64 consecutive floats of one row)
+    auto read_out = [&](int pitem, int pb) -> bool {
+      if (!mbar_wait_warp(bar(ACC_DONE), (uint32_t)pb, abort_flag)) return false;
+      tc_fence_after();
+      const int nd = kBlk * pb + rn;
+      if (kBlk * pb + (quad & 1) * 32 < T && (part == 0 || want_U)) {   // warp-uniform
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          uint32_t r1[32];
+          tmem_ld32(tmem + lane_addr + kColAcc + hc * 64 + half * 32, r1);
+          tmem_wait_ld();
+          if (nd < T) {
+            float4* o = reinterpret_cast<float4*>((part == 0 ? p.O : p.U) + ((size_t)pitem * T + nd) * 128 + hc * 64 +
+                                                  half * 32);
+#pragma unroll
+            for (int c = 0; c < 8; ++c)
+              __stcs(o + c, make_float4(__uint_as_float(r1[4 * c]), __uint_as_float(r1[4 * c + 1]),
+                                        __uint_as_float(r1[4 * c + 2]), __uint_as_float(r1[4 * c + 3])));
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(ACC_FREE));
+      return true;
+    };
+
+    uint32_t it = 0;
+    bool ok = true;
+    int pitem = -1, pb = 0;   // block whose output is still in TMEM
+    for (int item = blockIdx.x; ok && item < p.n_items; item += gridDim.x, ++it) {
+      const uint32_t ph = it & 1;
+      const float* al_s = tab_s + ph * (2 * kNodes);
+      const float* be_s = al_s + kNodes;
+      for (int b = 0; b < 2; ++b) {
+        // Every warp has finished the row solve and the tiles of the block before (they read the
+        // slot tables that this block overwrites): the last build of a block has an odd number.
+        if (pitem >= 0 && !(ok = mbar_wait_warp(bar(TILE_READY), 1u, abort_flag))) break;
+        if (b == 0 && !(ok = mbar_wait_warp(bar(ph ? META_FULL1 : META_FULL), (it >> 1) & 1, abort_flag))) break;
+        const int nd = kBlk * b + rn;                              // tree node of this row
+        const bool rows_live = kBlk * b + (quad & 1) * 32 < T;     // warp-uniform: some row of the warp is a node
+        const bool live_i = nd < T && (part == 0 || want_U);       // this row carries a problem
+        const bool warp_live = rows_live && (part == 0 || want_U); // same, for the warp-wide tcgen05.ld/st
+        const ulonglong2 mrec = mask_s[ph * kNodes + nd];
+        const uint64_t m0 = nd < T ? mrec.x : 0ull, m1 = nd < T ? mrec.y : 0ull;   // strict ancestors
+        const int depth = __popcll(m0) + __popcll(m1);
+
+        // ---- E1: raw path-sparse rows: part 0 <- Q K^T (path incl. the node), part 1 <- K K^T ----
+        if (!(ok = mbar_wait_warp(bar(b ? GD1 : GD0), ph, abort_flag))) break;
+        tc_fence_after();
+        if (rows_live) {
+          uint64_t s0 = m0, s1 = m1;
+          if (part == 0 && nd < T) {
+            if (nd < 64) s0 |= 1ull << nd; else s1 |= 1ull << (nd - 64);
+          }
+          float* dst = part == 0 ? Cs + rn * kLd : Gs + nd * kLd;
+          for (int c = 0; c <= b; ++c) {
+            const int cb = hc * 32 * (b + 1) + 32 * c;   // first column of this chunk of 32
+            const uint32_t bits = cb < 64 ? (uint32_t)(s0 >> cb) : (uint32_t)(s1 >> (cb - 64));
+            const int base = cb < 64 ? __popcll(s0 & ((1ull << cb) - 1ull))
+                                     : __popcll(s0) + __popcll(s1 & ((1ull << (cb - 64)) - 1ull));
+            uint32_t r[32];
+            tmem_ld32(tmem + lane_addr + (b ? kColSc1 : kColSc0) + cb, r);
+            tmem_wait_ld();
+#pragma unroll
+            for (int jj = 0; jj < 32; ++jj) {
+              // unselected columns land in the padding slot of the row: no branch, no predicate
+              const int slot = ((bits >> jj) & 1u) ? base + __popc(bits & ((1u << jj) - 1u)) : kSlots;
+              dst[slot] = __uint_as_float(r[jj]);
+              if (part == 0) Ps[rn * kLdP + slot] = (uint8_t)(cb + jj);
+            }
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive(bar(b ? GF1 : GF0));
+          mbar_arrive(bar(E1_SYNC));
+        }
+        if (!(ok = mbar_wait_warp(bar(E1_SYNC), (uint32_t)b, abort_flag))) break;
+
+        // ---- E2: decay factors, one back-substitution per row ----
+        constexpr int NS = DMAX + 1;                            // path slots in use
+        int path[NS];
+        float al[NS], bt[NS], pre[NS], vec[NS];
+        float Pi = 1.f;                                         // P_i: product of alpha along the path
+        if (live_i) {
+          const uint32_t* pw = reinterpret_cast<const uint32_t*>(Ps + rn * kLdP);
+          const uint32_t pword[4] = {pw[0], pw[1], pw[2], pw[3]};
+#pragma unroll
+          for (int s2 = 0; s2 < NS; ++s2) {
+            path[s2] = (pword[s2 >> 2] >> ((s2 & 3) * 8)) & 127;
+            const bool on = s2 <= depth;
+            const float a2 = al_s[path[s2]], b2 = be_s[path[s2]];
+            al[s2] = on ? a2 : 1.f;    // slots past the node count as no decay
+            bt[s2] = on ? b2 : 0.f;
+            Pi *= al[s2];
+            pre[s2] = Pi;              // P at path node s2
+          }
+        }
+        // ---- output of the block before: its MMAs ran under E1 and the gather above ----
+        if (pitem >= 0 && !(ok = read_out(pitem, pb))) break;
+        if (live_i) {
+          // C_{i,p_s} = (q_i . k_{p_s}) P_i / P_{p_s}: the ratio is the product of alpha over the
+          // slots after s, built up from the node's own slot backwards
+          float sfx = 1.f;
+#pragma unroll
+          for (int s2 = NS - 1; s2 >= 0; --s2) {
+            const float c = Cs[rn * kLd + s2];
+            if (part == 0) vec[s2] = s2 <= depth ? c * sfx : 0.f;
+            else vec[s2] = s2 == depth ? 1.f : 0.f;                               // x L = e_d
+            sfx *= al[s2];
+          }
+          // w_s = c_s - sum_{t > s} w_t G_{p_t,p_s},  G_{p_t,p_s} = beta_t (P_{p_t} / P_{p_s}) k_t.k_s;
+          // rr[t] holds P_{p_t} / P_{p_s} for the current s and grows by one factor per step
+          float rr[NS];
+#pragma unroll
+          for (int s2 = NS - 2; s2 >= 0; --s2) {
+            float acc = vec[s2];
+#pragma unroll
+            for (int t = s2 + 1; t < NS; ++t) {
+              rr[t] = t == s2 + 1 ? al[t] : rr[t] * al[s2 + 1];
+              const float gts = Gs[path[t] * kLd + s2] * (bt[t] * rr[t]);
+              acc = fmaf(-vec[t], t <= depth ? gts : 0.f, acc);
+            }
+            if (s2 < depth) vec[s2] = acc;
+          }
+        }
+        // ---- Qf starts as D_P Q (rows of the O problem; P_i in full fp32) or 0 (rows of the U
+        // problem); the state MMA of the block before must have read the old Qf first ----
+        if (!(ok = mbar_wait_warp(bar(QF_FREE), (uint32_t)b ^ 1, abort_flag))) break;
+        // the Q rows are read by these threads: observe the load's barrier themselves
+        if (!(ok = mbar_wait_warp(bar(QK_FULL), ph, abort_flag))) break;
+        if (warp_live) {
+          const bool use_q = live_i && part == 0;
+          const unsigned char* qrow = sm + (b ? kOffQK1 : kOffQK0) + hc * kTile + rn * 128;
+#pragma unroll
+          for (int half = 0; half < 2; ++half) {
+            uint32_t r[32];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+              const uint4 x = *reinterpret_cast<const uint4*>(qrow + (((uint32_t)(half * 4 + c) ^ nswz) << 4));
+              const uint32_t w4[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                // select, never 0 * x: rows past the tree may hold anything
+                r[c * 8 + 2 * e] = use_q ? __float_as_uint(Pi * __uint_as_float(w4[e] << 16)) : 0u;
+                r[c * 8 + 2 * e + 1] = use_q ? __float_as_uint(Pi * __uint_as_float(w4[e] & 0xffff0000u)) : 0u;
+              }
+            }
+            tmem_st32(tmem + lane_addr + kColQf + hc * 64 + half * 32, r);
+          }
+          tmem_wait_st();
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (b == 1 && lane == 0) mbar_arrive(bar(QK_FREE));   // Q rows of the item are not read again
+
+        // ---- coefficient tiles, one column half of one matrix at a time: thread hc = 0 writes the
+        // hi tile, hc = 1 the lo tile of its row ----
+        const int n_builds = b ? 4 : 2;
+        for (int q = 0; q < n_builds; ++q) {
+          const uint32_t j = b ? 2u + q : (uint32_t)q;    // build number within the item
+          const bool isW = b ? q >= 2 : q == 1;           // [W ; A] for V, else -[W D_P ; A D_P] for K
+          const int h = b ? (q & 1) : 0;                  // column half: ancestors 64 h .. 64 h + 63
+          // the MMAs that read the tile of the build before have completed
+          if (!(ok = mbar_wait_warp(bar(TILE_FREE), (j & 1) ^ 1, abort_flag))) break;
+          if (live_i) {
+            unsigned char* trow = sm + kOffCoef + hc * kTile + row * 128;
+            const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+            for (int c = 0; c < 8; ++c) *reinterpret_cast<uint4*>(trow + (((uint32_t)c ^ swz) << 4)) = z;
+#pragma unroll
+            for (int s2 = 0; s2 < NS; ++s2) {
+              if (s2 <= depth && (path[s2] >> 6) == h) {
+                const uint32_t jn = (uint32_t)path[s2] & 63u;
+                const float wv = vec[s2] * bt[s2];                   // W = C N D_beta (or A = N D_beta)
+                const float val = isW ? wv : -(wv * pre[s2]);        // ... times P_{p_s}, negated
+                const uint32_t off = (((jn >> 3) ^ swz) << 4) + (jn & 7u) * 2u;
+                uint16_t hi, lo;
+                split_bf16(val, hi, lo);
+                *reinterpret_cast<uint16_t*>(trow + off) = hc == 0 ? hi : lo;
+              }
+            }
+          }
+          fence_async_smem();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar(TILE_READY));
+        }
+        if (!ok) break;
+        if (b == 1) {
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar(ph ? META_FREE1 : META_FREE));   // this item's tables may be overwritten
+        }
+        pitem = item;
+        pb = b;
+      }
+    }
+    if (ok && pitem >= 0) read_out(pitem, pb);
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (warp == 1) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u)
+                 : "memory");
+  }
+  if (tid == 0 && *abort_flag && p.status) atomicExch(p.status, (int)TV_ERR_DEVICE_TIMEOUT);
+}
+
+}  // namespace
+
+bool tv_verify_tc_delta128_supports(const VerifyArgs& a) {
+  return a.bf16 && a.dk == 128 && a.dv == 128 && a.rule == TV_GATED_DELTA && a.T > kBlk && a.T <= kNodes &&
+         a.tree.max_depth_all < kSlots && a.tree.offsets == nullptr;
+}
+
+int tv_launch_verify_tc_delta128(const VerifyArgs& a, int32_t* status, cudaStream_t stream) {
+  if (!tv_verify_tc_delta128_supports(a)) return TV_ERR_UNSUPPORTED;
+  const uint64_t items = (uint64_t)a.L * a.B * a.H;
+  const uint64_t qk_items = (uint64_t)a.L * a.B * a.Hk;
+  const void* const ptrs[5] = {a.q, a.k, a.v, a.S_pre, nullptr};
+  // q, k, v in boxes of 64 rows x 64 columns (rows past T read as zero), S_pre in 4 chunks of 32 columns
+  const MapSet* ms = cached_maps(ptrs, items, a.T, 9 | (a.Hk << 8), [&](CUtensorMap* m) {
+    return make_map(&m[0], a.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, qk_items, a.T, 128, 64, 64) &&
+           make_map(&m[1], a.k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, qk_items, a.T, 128, 64, 64) &&
+           make_map(&m[2], a.v, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, items, a.T, 128, 64, 64) &&
+           make_map(&m[3], a.S_pre, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, 128, 128, 32, 128);
+  });
+  if (!ms) return TV_ERR_CUDA;
+  static thread_local int configured_dev = -1;
+  static thread_local int sm_count = 0;
+  int dev = 0;
+  TV_CUDA_TRY(cudaGetDevice(&dev));
+  if (configured_dev != dev) {
+    TV_CUDA_TRY(cudaFuncSetAttribute(verify_tc_delta128_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)kSmemBytes));
+    TV_CUDA_TRY(cudaFuncSetAttribute(verify_tc_delta128_kernel<15>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)kSmemBytes));
+    TV_CUDA_TRY(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev));
+    configured_dev = dev;
+  }
+  Delta128Params p;
+  p.tree = a.tree;
+  p.n_items = (int32_t)items;
+  p.B = a.B; p.H = a.H; p.T = a.T; p.Hk = a.Hk;
+  p.alpha = a.alpha;
+  p.beta = a.beta;
+  p.want_U = a.U != nullptr;
+  p.status = status;
+  p.O = a.O;
+  p.U = a.U ? a.U : a.O;   // never written when U is not requested
+  const int grid = (int)(items < (uint64_t)sm_count ? items : (uint64_t)sm_count);
+  if (a.tree.max_depth_all <= 8)
+    TV_CUDA_TRY(launch_dependent(verify_tc_delta128_kernel<8>, grid, kThreads, kSmemBytes, stream, ms->map[0],
+                                 ms->map[1], ms->map[2], ms->map[3], p));
+  else
+    TV_CUDA_TRY(launch_dependent(verify_tc_delta128_kernel<15>, grid, kThreads, kSmemBytes, stream, ms->map[0],
+                                 ms->map[1], ms->map[2], ms->map[3], p));
+  TV_CUDA_TRY(cudaGetLastError());
+  return TV_OK;
+}

@@ -72,6 +72,57 @@ def test_tc_delta(B, H, T, tree):
     assert np.array_equal(O2, O)          # asking for U does not change O
 
 
+@pytest.mark.parametrize("B,H,T,tree", [(1, 1, 128, "frontier"), (1, 2, 65, "frontier"), (2, 3, 96, "binary"),
+                                         (3, 2, 127, "frontier"), (8, 32, 128, "frontier"), (2, 2, 100, "spine")])
+def test_tc_delta_large_trees(B, H, T, tree):
+    """Delta rule, 64 < T <= 128: the two-row-block tensor-core kernel against the oracle, O and U,
+    per-request trees; asking for U must not change O."""
+    wl = inputs.workload("c4", B=B, H=H, T=T, L=1, tree=tree, seed=41 + T)
+    parents, accepted = inputs.make_trees(wl)
+    assert max(int(inputs.node_depths(par).max()) for par in parents) <= 15   # what the kernel takes
+    tens = inputs.make_tensors(wl)
+    O, U, Sn, tree_h = pu.gpu_round(wl, parents, accepted, tens, impl=tv.IMPL_TC, want_U=True,
+                                    commit_with_U=True, in_place=True)
+    tree_h.device_status()
+    ver, com = pu.oracle_round(wl, parents, accepted, tens)
+    eO, eU, eS = pu.compare(wl, O, U, Sn, ver, com)
+    print(f"TC delta (large trees) B{B} H{H} T{T} {tree}: rel-L2 O {eO:.3e} U {eU:.3e} S {eS:.3e}")
+    assert eO <= wl.tol and eU <= wl.tol and eS <= wl.tol
+    O2, _, _, _ = pu.gpu_round(wl, parents, accepted, tens, impl=tv.IMPL_TC, want_U=False)
+    assert np.array_equal(O2, O)          # asking for U does not change O
+    O3, _, _, _ = pu.gpu_round(wl, parents, accepted, tens, impl=tv.IMPL_TC, want_U=True)
+    assert np.array_equal(O3, O)          # run to run identical
+
+
+@pytest.mark.parametrize("T", [64, 128])
+def test_tc_delta_depth_15(T):
+    """Trees of depth 9..15 take the deeper instantiation of the row solve (both tree sizes)."""
+    B, H = 3, 2
+    wl = inputs.workload("c4", B=B, H=H, T=T, L=1, seed=97 + T)
+    rng = np.random.default_rng(5 + T)
+    parents = np.zeros((B, T), dtype=np.int32)
+    for b in range(B):
+        par, dep = [-1], [0]
+        for i in range(1, T):
+            if i <= 15:
+                p = i - 1                                   # a spine down to depth 15
+            else:
+                p = int(rng.choice([j for j in range(i) if dep[j] < 15]))
+            par.append(p)
+            dep.append(dep[p] + 1)
+        assert max(dep) == 15
+        parents[b] = par
+    accepted = np.array([15, T - 1, -1], dtype=np.int32)
+    tens = inputs.make_tensors(wl)
+    O, U, Sn, tree_h = pu.gpu_round(wl, parents, accepted, tens, impl=tv.IMPL_TC, want_U=True,
+                                    commit_with_U=True, in_place=True)
+    tree_h.device_status()
+    ver, com = pu.oracle_round(wl, parents, accepted, tens)
+    eO, eU, eS = pu.compare(wl, O, U, Sn, ver, com)
+    print(f"TC delta depth 15, T{T}: rel-L2 O {eO:.3e} U {eU:.3e} S {eS:.3e}")
+    assert eO <= wl.tol and eU <= wl.tol and eS <= wl.tol
+
+
 def test_tc_delta_falls_back_on_deep_trees():
     wl = inputs.workload("c4", B=1, H=2, T=40, tree="chain", seed=5)   # depth 39 > 15
     parents, accepted = inputs.make_trees(wl)
