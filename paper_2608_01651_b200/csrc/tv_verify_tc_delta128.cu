@@ -1,5 +1,5 @@
 // Tree verification of the gated delta rule on the tensor cores for trees of 65..128 nodes
-// (bf16 q/k/v, fp32 state, dk = dv = 128, tree depth <= 15, dense batch layout).
+// (bf16 q/k/v, fp32 state, dk = dv = 128, tree depth <= 15; dense batches and packed forests).
 //
 // Same algebra as tv_verify_tc_delta.cu (Theorem 1, Eq. 2, regrouped so that the state is
 // contracted once; Lemma 2/3 for N = (I+G)^-1; one back-substitution per row on the
@@ -49,7 +49,8 @@ constexpr uint32_t kOffCs = kOffGs + 8704;       // float Cs[64][kLd]: raw Q K^T
 constexpr uint32_t kOffPs = kOffCs + 4352;       // uint8 Ps[64][kLdP]: path nodes of the block's rows
 constexpr uint32_t kOffTab = kOffPs + 1280;      // 2 buffers x {float alpha[128], beta[128]}
 constexpr uint32_t kOffMask = kOffTab + 2048;    // 2 buffers x [128] x {uint64 lo, hi} strict ancestors
-constexpr uint32_t kOffBar = kOffMask + 4096;
+constexpr uint32_t kOffItem = kOffMask + 4096;   // 2 buffers x {nodes, first output row (2 words), spare}
+constexpr uint32_t kOffBar = kOffItem + 64;
 constexpr uint32_t kOffMisc = kOffBar + 8 * 32;
 constexpr uint32_t kSmemBytes = kOffMisc + 64 + 1024;
 
@@ -71,6 +72,9 @@ struct Delta128Params {
   int32_t* status;
   float* O;
   float* U;
+  // packed forest only: row offsets of the requests and rows per (layer, head) plane
+  const int32_t* offsets;
+  int32_t capacity;
 };
 
 // bf16 hi/lo parts of x (hi = upper 16 bits, lo = upper 16 bits of the exact remainder)
@@ -83,7 +87,11 @@ __device__ __forceinline__ void split_bf16(float x, uint16_t& hi, uint16_t& lo) 
 
 // DMAX: compile-time bound on the tree depth (8 covers draft trees, 15 the rest), so that the
 // per-row triangular solve is straight-line code whose loads all issue up front.
-template <int DMAX>
+// PACKED = packed forest: request b owns rows offsets[b] .. offsets[b+1]-1 of every plane; loads
+// take 64-row boxes at the request's offset, rows past the request's node count are not worked on
+// or stored, and operand rows past the last node of the forest are zeroed in shared memory before
+// they meet a zero coefficient.
+template <int DMAX, bool PACKED>
 __global__ void __launch_bounds__(kThreads, 1)
 verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                           const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmS,
@@ -96,6 +104,7 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
   uint8_t* Ps = reinterpret_cast<uint8_t*>(sm + kOffPs);
   float* tab_s = reinterpret_cast<float*>(sm + kOffTab);              // [2][alpha[128], beta[128]]
   ulonglong2* mask_s = reinterpret_cast<ulonglong2*>(sm + kOffMask);  // [2][128]
+  int32_t* item_s = reinterpret_cast<int32_t*>(sm + kOffItem);        // [2][4]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + kOffMisc);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + kOffMisc + 4);
   auto bar = [&](int i) { return sbase + kOffBar + 8u * i; };
@@ -138,7 +147,13 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
       grid_dependency_wait();   // inputs may come from the kernel in front (dependent launch)
       for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++it) {
         const uint32_t ph = it & 1;
-        const int qk = tv_qk_item(item, p.H, p.Hk);
+        int qk = 0, vplane = item, y0 = 0;
+        if constexpr (PACKED) {
+          const PackedItem pi = packed_item(p.offsets, p.B, p.H, p.Hk, item);
+          qk = pi.plane_qk; vplane = pi.plane_v; y0 = pi.row0;
+        } else {
+          qk = tv_qk_item(item, p.H, p.Hk);
+        }
         if (!mbar_wait(bar(QK_FREE), ph ^ 1, abort_flag)) break;
         mbar_expect_tx(bar(QK_FULL), 8 * 8192);
 #pragma unroll
@@ -146,8 +161,8 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
 #pragma unroll
           for (int d = 0; d < 2; ++d) {    // dk half
             const uint32_t dst = sbase + (h ? kOffQK1 : kOffQK0) + d * kTile;
-            tma_load_3d(dst, &tmQ, bar(QK_FULL), 64 * d, 64 * h, qk);
-            tma_load_3d(dst + 8192, &tmK, bar(QK_FULL), 64 * d, 64 * h, qk);
+            tma_load_3d(dst, &tmQ, bar(QK_FULL), 64 * d, y0 + 64 * h, qk);
+            tma_load_3d(dst + 8192, &tmK, bar(QK_FULL), 64 * d, y0 + 64 * h, qk);
           }
         pend_qk = 1 + (int)ph;
         if (!mbar_wait(bar(S_FREE), ph ^ 1, abort_flag)) break;
@@ -162,7 +177,7 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
         for (int h = 0; h < 2; ++h)
 #pragma unroll
           for (int d = 0; d < 2; ++d)
-            tma_load_3d(sbase + kOffV + d * kTile + h * 8192, &tmV, bar(V_FULL), 64 * d, 64 * h, item);
+            tma_load_3d(sbase + kOffV + d * kTile + h * 8192, &tmV, bar(V_FULL), 64 * d, y0 + 64 * h, vplane);
         pend_v = 1 + (int)ph;
       }
       if (*abort_flag) {
@@ -265,8 +280,16 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
     for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++j) {
       const uint32_t buf = j & 1, use = j >> 1;
       if (use > 0 && !mbar_wait_warp(bar(buf ? META_FREE1 : META_FREE), (use - 1) & 1, abort_flag)) break;
-      const int tb = p.tree.n_trees == 1 ? 0 : (item / p.H) % p.B;
-      const size_t g0 = (size_t)item * T;   // first gate of the item
+      int n = T, tb = 0;
+      size_t g0 = (size_t)item * T;   // first gate (and first output row) of the item
+      if constexpr (PACKED) {
+        const PackedItem pi = packed_item(p.offsets, p.B, p.H, p.Hk, item);
+        n = pi.n;
+        tb = pi.b;
+        g0 = (size_t)pi.plane_v * p.capacity + pi.row0;
+      } else {
+        tb = p.tree.n_trees == 1 ? 0 : (item / p.H) % p.B;
+      }
       float* tab = tab_s + buf * (2 * kNodes);
       // all loads first: one trip to memory, not one per table
       ulonglong2 mk[4];
@@ -277,7 +300,7 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
         mk[h] = make_ulonglong2(0ull, 0ull);
         al[h] = 1.f;
         be[h] = 0.f;
-        if (nd < T) {
+        if (nd < n) {
           mk[h] = __ldg(reinterpret_cast<const ulonglong2*>(p.tree.anc) + (size_t)tb * T + nd);
           al[h] = __ldg(p.alpha + g0 + nd);
           be[h] = __ldg(p.beta + g0 + nd);
@@ -289,6 +312,11 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
         mask_s[buf * kNodes + nd] = mk[h];
         tab[nd] = al[h];
         tab[kNodes + nd] = be[h];
+      }
+      if (lane == 0) {
+        item_s[buf * 4 + 0] = n;
+        item_s[buf * 4 + 1] = (int32_t)(g0 & 0xffffffffu);
+        item_s[buf * 4 + 2] = (int32_t)(g0 >> 32);
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(buf ? META_FULL1 : META_FULL));
@@ -309,25 +337,27 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
     // the commit kernel behind this one may be scheduled as SMs drain (it orders itself)
     if (warp == 2 && lane == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
-    // acc rows 0..63 -> O rows, rows 64..127 -> U rows of block pb of item pitem, straight from
-    // registers (each thread owns 64 consecutive floats of one row)
-    auto read_out = [&](int pitem, int pb) -> bool {
+    // acc rows 0..63 -> O rows, rows 64..127 -> U rows of block pb of an item with pn nodes whose
+    // output rows start at row prow0: straight from registers, 32 bytes per store (each thread owns
+    // 64 consecutive floats of one row, so every store fills a whole sector)
+    auto read_out = [&](size_t prow0, int pn, int pb) -> bool {
       if (!mbar_wait_warp(bar(ACC_DONE), (uint32_t)pb, abort_flag)) return false;
       tc_fence_after();
       const int nd = kBlk * pb + rn;
-      if (kBlk * pb + (quad & 1) * 32 < T && (part == 0 || want_U)) {   // warp-uniform
+      if (kBlk * pb + (quad & 1) * 32 < pn && (part == 0 || want_U)) {   // warp-uniform
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
           uint32_t r1[32];
           tmem_ld32(tmem + lane_addr + kColAcc + hc * 64 + half * 32, r1);
           tmem_wait_ld();
-          if (nd < T) {
-            float4* o = reinterpret_cast<float4*>((part == 0 ? p.O : p.U) + ((size_t)pitem * T + nd) * 128 + hc * 64 +
-                                                  half * 32);
+          if (nd < pn) {
+            float* o = (part == 0 ? p.O : p.U) + (prow0 + nd) * 128 + hc * 64 + half * 32;
 #pragma unroll
-            for (int c = 0; c < 8; ++c)
-              __stcs(o + c, make_float4(__uint_as_float(r1[4 * c]), __uint_as_float(r1[4 * c + 1]),
-                                        __uint_as_float(r1[4 * c + 2]), __uint_as_float(r1[4 * c + 3])));
+            for (int c = 0; c < 4; ++c)
+              asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(o + 8 * c), "r"(r1[8 * c]),
+                           "r"(r1[8 * c + 1]), "r"(r1[8 * c + 2]), "r"(r1[8 * c + 3]), "r"(r1[8 * c + 4]),
+                           "r"(r1[8 * c + 5]), "r"(r1[8 * c + 6]), "r"(r1[8 * c + 7])
+                           : "memory");
           }
         }
       }
@@ -336,10 +366,14 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
       if (lane == 0) mbar_arrive(bar(ACC_FREE));
       return true;
     };
+    const int total_rows = PACKED ? p.offsets[p.B] : 0;   // rows at and past this one hold no node
 
     uint32_t it = 0;
     bool ok = true;
-    int pitem = -1, pb = 0;   // block whose output is still in TMEM
+    int pn = -1, pb = 0;      // block whose output is still in TMEM: nodes of its item, block,
+    size_t prow0 = 0;         // first output row of its item
+    int Tn = T;               // nodes of the current item
+    size_t row0 = 0;          // its first gate / output row
     for (int item = blockIdx.x; ok && item < p.n_items; item += gridDim.x, ++it) {
       const uint32_t ph = it & 1;
       const float* al_s = tab_s + ph * (2 * kNodes);
@@ -347,14 +381,18 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
       for (int b = 0; b < 2; ++b) {
         // Every warp has finished the row solve and the tiles of the block before (they read the
         // slot tables that this block overwrites): the last build of a block has an odd number.
-        if (pitem >= 0 && !(ok = mbar_wait_warp(bar(TILE_READY), 1u, abort_flag))) break;
-        if (b == 0 && !(ok = mbar_wait_warp(bar(ph ? META_FULL1 : META_FULL), (it >> 1) & 1, abort_flag))) break;
+        if (pn >= 0 && !(ok = mbar_wait_warp(bar(TILE_READY), 1u, abort_flag))) break;
+        if (b == 0) {
+          if (!(ok = mbar_wait_warp(bar(ph ? META_FULL1 : META_FULL), (it >> 1) & 1, abort_flag))) break;
+          Tn = item_s[ph * 4];
+          row0 = (size_t)(uint32_t)item_s[ph * 4 + 1] | (size_t)(uint32_t)item_s[ph * 4 + 2] << 32;
+        }
         const int nd = kBlk * b + rn;                              // tree node of this row
-        const bool rows_live = kBlk * b + (quad & 1) * 32 < T;     // warp-uniform: some row of the warp is a node
-        const bool live_i = nd < T && (part == 0 || want_U);       // this row carries a problem
+        const bool rows_live = kBlk * b + (quad & 1) * 32 < Tn;    // warp-uniform: some row of the warp is a node
+        const bool live_i = nd < Tn && (part == 0 || want_U);      // this row carries a problem
         const bool warp_live = rows_live && (part == 0 || want_U); // same, for the warp-wide tcgen05.ld/st
         const ulonglong2 mrec = mask_s[ph * kNodes + nd];
-        const uint64_t m0 = nd < T ? mrec.x : 0ull, m1 = nd < T ? mrec.y : 0ull;   // strict ancestors
+        const uint64_t m0 = nd < Tn ? mrec.x : 0ull, m1 = nd < Tn ? mrec.y : 0ull;   // strict ancestors
         const int depth = __popcll(m0) + __popcll(m1);
 
         // ---- E1: raw path-sparse rows: part 0 <- Q K^T (path incl. the node), part 1 <- K K^T ----
@@ -362,7 +400,7 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
         tc_fence_after();
         if (rows_live) {
           uint64_t s0 = m0, s1 = m1;
-          if (part == 0 && nd < T) {
+          if (part == 0 && nd < Tn) {
             if (nd < 64) s0 |= 1ull << nd; else s1 |= 1ull << (nd - 64);
           }
           float* dst = part == 0 ? Cs + rn * kLd : Gs + nd * kLd;
@@ -391,6 +429,27 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
         }
         if (!(ok = mbar_wait_warp(bar(E1_SYNC), (uint32_t)b, abort_flag))) break;
 
+        if constexpr (PACKED) {
+          // A box that reaches past the last node of the forest brings rows nobody wrote.  They only
+          // ever meet zero coefficients, but 0 x garbage need not be 0: zero the K and V rows (the B
+          // operands of the coefficient MMAs) once both Gram products have read K.
+          const int lim = total_rows - (int)(row0 % (size_t)p.capacity);   // rows of the box that exist
+          if (b == 0 && lim < kNodes) {
+            if (!(ok = mbar_wait_warp(bar(GD1), ph, abort_flag))) break;
+            if (!(ok = mbar_wait_warp(bar(V_FULL), ph, abort_flag))) break;
+            if (row >= lim) {   // thread (row, hc): dk-half hc of K row `row`, dv-half hc of V row `row`
+              unsigned char* krow = sm + (row >> 6 ? kOffQK1 : kOffQK0) + hc * kTile + 8192 + (row & 63) * 128;
+              unsigned char* vrow = sm + kOffV + hc * kTile + row * 128;
+              const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+              for (int c = 0; c < 8; ++c) {
+                *reinterpret_cast<uint4*>(krow + c * 16) = z;
+                *reinterpret_cast<uint4*>(vrow + c * 16) = z;
+              }
+            }
+          }
+        }
+
         // ---- E2: decay factors, one back-substitution per row ----
         constexpr int NS = DMAX + 1;                            // path slots in use
         int path[NS];
@@ -411,7 +470,7 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
           }
         }
         // ---- output of the block before: its MMAs ran under E1 and the gather above ----
-        if (pitem >= 0 && !(ok = read_out(pitem, pb))) break;
+        if (pn >= 0 && !(ok = read_out(prow0, pn, pb))) break;
         if (live_i) {
           // C_{i,p_s} = (q_i . k_{p_s}) P_i / P_{p_s}: the ratio is the product of alpha over the
           // slots after s, built up from the node's own slot backwards
@@ -504,11 +563,12 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
           __syncwarp();
           if (lane == 0) mbar_arrive(bar(ph ? META_FREE1 : META_FREE));   // this item's tables may be overwritten
         }
-        pitem = item;
+        pn = Tn;
+        prow0 = row0;
         pb = b;
       }
     }
-    if (ok && pitem >= 0) read_out(pitem, pb);
+    if (ok && pn >= 0) read_out(prow0, pn, pb);
   }
 
   tc_fence_before();
@@ -525,31 +585,49 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
 
 bool tv_verify_tc_delta128_supports(const VerifyArgs& a) {
   return a.bf16 && a.dk == 128 && a.dv == 128 && a.rule == TV_GATED_DELTA && a.T > kBlk && a.T <= kNodes &&
-         a.tree.max_depth_all < kSlots && a.tree.offsets == nullptr;
+         a.tree.max_depth_all < kSlots;
 }
 
 int tv_launch_verify_tc_delta128(const VerifyArgs& a, int32_t* status, cudaStream_t stream) {
   if (!tv_verify_tc_delta128_supports(a)) return TV_ERR_UNSUPPORTED;
   const uint64_t items = (uint64_t)a.L * a.B * a.H;
   const uint64_t qk_items = (uint64_t)a.L * a.B * a.Hk;
+  const bool packed = a.tree.offsets != nullptr;
   const void* const ptrs[5] = {a.q, a.k, a.v, a.S_pre, nullptr};
-  // q, k, v in boxes of 64 rows x 64 columns (rows past T read as zero), S_pre in 4 chunks of 32 columns
-  const MapSet* ms = cached_maps(ptrs, items, a.T, 9 | (a.Hk << 8), [&](CUtensorMap* m) {
-    return make_map(&m[0], a.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, qk_items, a.T, 128, 64, 64) &&
-           make_map(&m[1], a.k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, qk_items, a.T, 128, 64, 64) &&
-           make_map(&m[2], a.v, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, items, a.T, 128, 64, 64) &&
-           make_map(&m[3], a.S_pre, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, 128, 128, 32, 128);
-  });
+  // q, k, v in boxes of 64 rows x 64 columns (rows past the tensor read as zero), S_pre in 4 chunks
+  // of 32 columns; a packed forest addresses (layer, head) planes of `capacity` rows
+  const MapSet* ms = nullptr;
+  if (!packed) {
+    ms = cached_maps(ptrs, items, a.T, 9 | (a.Hk << 8), [&](CUtensorMap* m) {
+      return make_map(&m[0], a.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, qk_items, a.T, 128, 64, 64) &&
+             make_map(&m[1], a.k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, qk_items, a.T, 128, 64, 64) &&
+             make_map(&m[2], a.v, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, items, a.T, 128, 64, 64) &&
+             make_map(&m[3], a.S_pre, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, 128, 128, 32, 128);
+    });
+  } else {
+    const uint64_t cap = (uint64_t)a.tree.capacity;
+    const uint64_t pv = (uint64_t)a.L * a.H, pqk = (uint64_t)a.L * a.Hk;
+    ms = cached_maps(ptrs, (cap << 24) ^ items, a.T, 10 | (a.Hk << 8), [&](CUtensorMap* m) {
+      return make_map(&m[0], a.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, pqk, cap, 128, 64, 64) &&
+             make_map(&m[1], a.k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, pqk, cap, 128, 64, 64) &&
+             make_map(&m[2], a.v, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, pv, cap, 128, 64, 64) &&
+             make_map(&m[3], a.S_pre, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, 128, 128, 32, 128);
+    });
+  }
   if (!ms) return TV_ERR_CUDA;
   static thread_local int configured_dev = -1;
   static thread_local int sm_count = 0;
   int dev = 0;
   TV_CUDA_TRY(cudaGetDevice(&dev));
   if (configured_dev != dev) {
-    TV_CUDA_TRY(cudaFuncSetAttribute(verify_tc_delta128_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)kSmemBytes));
-    TV_CUDA_TRY(cudaFuncSetAttribute(verify_tc_delta128_kernel<15>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)kSmemBytes));
+    TV_CUDA_TRY(cudaFuncSetAttribute(verify_tc_delta128_kernel<8, false>,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
+    TV_CUDA_TRY(cudaFuncSetAttribute(verify_tc_delta128_kernel<15, false>,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
+    TV_CUDA_TRY(cudaFuncSetAttribute(verify_tc_delta128_kernel<8, true>,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
+    TV_CUDA_TRY(cudaFuncSetAttribute(verify_tc_delta128_kernel<15, true>,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
     TV_CUDA_TRY(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev));
     configured_dev = dev;
   }
@@ -564,12 +642,17 @@ int tv_launch_verify_tc_delta128(const VerifyArgs& a, int32_t* status, cudaStrea
   p.O = a.O;
   p.U = a.U ? a.U : a.O;   // never written when U is not requested
   const int grid = (int)(items < (uint64_t)sm_count ? items : (uint64_t)sm_count);
-  if (a.tree.max_depth_all <= 8)
-    TV_CUDA_TRY(launch_dependent(verify_tc_delta128_kernel<8>, grid, kThreads, kSmemBytes, stream, ms->map[0],
-                                 ms->map[1], ms->map[2], ms->map[3], p));
+  p.offsets = a.tree.offsets;
+  p.capacity = a.tree.capacity;
+  const bool shallow = a.tree.max_depth_all <= 8;
+  auto launch = [&](auto kernel) {
+    return launch_dependent(kernel, grid, kThreads, kSmemBytes, stream, ms->map[0], ms->map[1], ms->map[2],
+                            ms->map[3], p);
+  };
+  if (packed)
+    TV_CUDA_TRY(shallow ? launch(verify_tc_delta128_kernel<8, true>) : launch(verify_tc_delta128_kernel<15, true>));
   else
-    TV_CUDA_TRY(launch_dependent(verify_tc_delta128_kernel<15>, grid, kThreads, kSmemBytes, stream, ms->map[0],
-                                 ms->map[1], ms->map[2], ms->map[3], p));
+    TV_CUDA_TRY(shallow ? launch(verify_tc_delta128_kernel<8, false>) : launch(verify_tc_delta128_kernel<15, false>));
   TV_CUDA_TRY(cudaGetLastError());
   return TV_OK;
 }

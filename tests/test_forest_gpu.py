@@ -121,16 +121,17 @@ def test_forest_matches_oracle_per_request(case, dtype, rule, impl):
                     assert rel_fro(Sn[l, b, h], Sr) <= tol
 
 
+@pytest.mark.parametrize("n_max", [64, 128])
 @pytest.mark.parametrize("rule", [inputs.GATED, inputs.DELTA])
-def test_forest_takes_the_tensor_core_kernels(rule):
-    """bf16, dk = dv = 128: IMPL_TC must accept a packed forest for both rules (no silent fallback)
-    and agree with the general kernel."""
-    wl = inputs.workload("c2", B=5, H=2, T=64, rule=rule, seed=11)
-    parents, _ = make_forest(5, 64, seed=12)
+def test_forest_takes_the_tensor_core_kernels(rule, n_max):
+    """bf16, dk = dv = 128: IMPL_TC must accept a packed forest for both rules and both tree-size
+    classes (no silent fallback) and agree with the general kernel."""
+    wl = inputs.workload("c2", B=5, H=2, T=n_max, rule=rule, seed=11)
+    parents, _ = make_forest(5, n_max, seed=12)
     cap = sum(len(p) for p in parents) + 3
     P, _ = packed_tensors(wl, parents, cap, 2)
     g = {n: (None if t is None else t.to(DEV)) for n, t in P.items()}
-    forest = tv.forest_build(parents, n_max=64, capacity=cap).upload()
+    forest = tv.forest_build(parents, n_max=n_max, capacity=cap).upload()
     outs = []
     for impl in (tv.IMPL_TC, tv.IMPL_SIMT):
         O = torch.zeros(1, 2, cap, 128, device=DEV)
@@ -142,7 +143,7 @@ def test_forest_takes_the_tensor_core_kernels(rule):
     forest.device_status()
     assert rel_fro(outs[0][0], outs[1][0]) < 2e-3 and rel_fro(outs[0][1], outs[1][1]) < 2e-3
     # deeper than the tensor-core delta kernel's path tables: declined, not faked
-    if rule == inputs.DELTA:
+    if rule == inputs.DELTA and n_max == 64:
         deep = tv.forest_build([inputs.tree_chain(40)], n_max=64, capacity=64).upload()
         one = {n: (None if t is None else t[:, :1].contiguous() if n == "S_pre" else t) for n, t in g.items()}
         with pytest.raises(tv.TreeVerifyError) as e:
