@@ -39,6 +39,29 @@ def test_session_round_matches_oracle(name, B, H, L):
                  host["beta"], O, S_new)
 
 
+@pytest.mark.parametrize("name,B,T", [("c4", 24, 64), ("c4", 12, 128), ("c3", 40, 64)])
+def test_session_round_in_several_groups(name, B, T):
+    """Enough traffic for three or more request groups (copy-in, kernel and copy-out streams chained
+    per group): sampled items of every group against the oracle, all outputs finite."""
+    H = 32
+    wl = inputs.workload(name, B=B, H=H, T=T, L=1, seed=61 + B)
+    parents, accepted = inputs.make_trees(wl)
+    t = inputs.make_tensors(wl)
+    host = {k: (None if v is None else v.unsqueeze(0).contiguous().pin_memory()) for k, v in t.items()}
+    O = torch.full((1, B, H, T, wl.dv), float("nan")).pin_memory()
+    S_new = torch.full_like(host["S_pre"], float("nan")).pin_memory()
+    sess = tv.Session(1, B, H, T, wl.dk, wl.dv, rule=wl.rule, qkv_dtype=wl.qkv_dtype)
+    sess.round(parents, accepted, host["S_pre"], host["q"], host["k"], host["v"], host["alpha"], host["beta"],
+               O, S_new)
+    sess.free()
+    assert torch.isfinite(O).all() and torch.isfinite(S_new).all()     # every group wrote its rows
+    rng = np.random.default_rng(B)
+    items = [(int(b), int(rng.integers(H))) for b in sorted({0, B - 1, *rng.integers(0, B, 6).tolist()})]
+    ver, com = pu.oracle_round(wl, parents, accepted, host, items=items, layer=0)
+    eO, _, eS = pu.compare(wl, O.double().numpy(), None, S_new.double().numpy(), ver, com, layer=0)
+    assert eO <= wl.tol and eS <= wl.tol, (eO, eS)
+
+
 def test_prepared_calls_equal_direct_calls():
     wl = inputs.workload("c3", B=4, H=4)
     parents, accepted = inputs.make_trees(wl)
