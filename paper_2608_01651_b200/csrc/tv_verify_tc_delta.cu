@@ -58,9 +58,9 @@ constexpr uint32_t kOffW = 12 * kTile;           // hi, lo of [W ; A]           
 constexpr uint32_t kOffStage = kOffAk;           // 8 output chunks of 8 KiB (O: 0..3, U: 4..7)
 constexpr uint32_t kOffGs = kOffV + 8192;        // float Gs[64][kLd]: raw K K^T on the path
 constexpr uint32_t kOffCs = kOffV + kTile + 8192;  // float Cs[64][kLd]: raw Q K^T on the path
-constexpr uint32_t kOffPs = kOffCs + 4352;       // uint8 Ps[64][kLdP]: path nodes
-constexpr uint32_t kOffSmall = kOffPs + 1280;    // 2 buffers x {float al[64] (alpha), be[64] (beta)}
+constexpr uint32_t kOffSmall = kOffCs + 4352;    // 2 buffers x {float al[64] (alpha), be[64] (beta)}
 constexpr uint32_t kOffMeta = kOffGs + 4352;     // 2 buffers x uint64 strict-ancestor mask [64]
+constexpr uint32_t kOffPs = kOffMeta + 1024;     // 2 buffers x uint8 Ps[64][kLdP]: path nodes in slot order
 constexpr uint32_t kOffBar = 14 * kTile;
 constexpr uint32_t kOffMisc = kOffBar + 8 * 24;
 constexpr uint32_t kSmemBytes = kOffMisc + 64 + 1024;
@@ -131,7 +131,7 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   const uint32_t sbase = smem_u32(sm);
   float* Gs = reinterpret_cast<float*>(sm + kOffGs);
   float* Cs = reinterpret_cast<float*>(sm + kOffCs);
-  uint8_t* Ps = reinterpret_cast<uint8_t*>(sm + kOffPs);
+  uint8_t* Ps_all = reinterpret_cast<uint8_t*>(sm + kOffPs);     // [2][64][kLdP]
   float* tab_s = reinterpret_cast<float*>(sm + kOffSmall);       // [2][la[64], be[64]]
   uint64_t* mask_s = reinterpret_cast<uint64_t*>(sm + kOffMeta);   // [2][64]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + kOffMisc);
@@ -369,6 +369,14 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         mask_s[buf * kRows + nd] = mk[h];
         tab[nd] = al[h];
         tab[kRows + nd] = be[h];
+        // the node's path in slot order: the set bits of (ancestors | self) from the lowest up
+        // (nodes are numbered parent before child); slots past the node's depth are never used
+        uint8_t* prow = Ps_all + (buf * kRows + nd) * kLdP;
+        uint64_t rest = nd < n ? (mk[h] | (1ull << nd)) : 0ull;
+        for (int s2 = 0; rest != 0ull && s2 < kSlots; ++s2) {
+          prow[s2] = (uint8_t)(__ffsll((long long)rest) - 1);
+          rest &= rest - 1;
+        }
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(buf ? META_FULL1 : META_FULL));
@@ -478,7 +486,6 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           // (predicated stores of the selected columns only were measured slower)
           const int slot = ((bits >> jj) & 1u) ? base + __popc(bits & ((1u << jj) - 1u)) : kSlots;
           dst[slot] = __uint_as_float(r[jj]);
-          if (part == 0) Ps[node * kLdP + slot] = (uint8_t)(cbase + jj);
         }
       }
       tc_fence_before();
@@ -497,7 +504,7 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       float al[NS], bt[NS], pre[NS], vec[NS];
       float Pi = 1.f;                                         // P_i: product of alpha along the path
       if (live_i) {
-        const uint32_t* pw = reinterpret_cast<const uint32_t*>(Ps + node * kLdP);
+        const uint32_t* pw = reinterpret_cast<const uint32_t*>(Ps_all + (ph * kRows + node) * kLdP);
         const uint32_t pword[4] = {pw[0], pw[1], pw[2], pw[3]};
 #pragma unroll
         for (int s2 = 0; s2 < NS; ++s2) {

@@ -46,8 +46,8 @@ constexpr uint32_t kOffS = 6 * kTile;            // 4 k-chunks of S_pre [128 v][
 constexpr uint32_t kOffCoef = 10 * kTile;        // hi, lo of the current coefficient tile [128][64] bf16
 constexpr uint32_t kOffGs = 12 * kTile;          // float Gs[128][kLd]: raw K K^T on the path, all nodes
 constexpr uint32_t kOffCs = kOffGs + 8704;       // float Cs[64][kLd]: raw Q K^T on the path, block rows
-constexpr uint32_t kOffPs = kOffCs + 4352;       // uint8 Ps[64][kLdP]: path nodes of the block's rows
-constexpr uint32_t kOffTab = kOffPs + 1280;      // 2 buffers x {float alpha[128], beta[128]}
+constexpr uint32_t kOffPs = kOffCs + 4352;       // 2 buffers x uint8 Ps[128][kLdP]: path nodes in slot order
+constexpr uint32_t kOffTab = kOffPs + 5120;      // 2 buffers x {float alpha[128], beta[128]}
 constexpr uint32_t kOffMask = kOffTab + 2048;    // 2 buffers x [128] x {uint64 lo, hi} strict ancestors
 constexpr uint32_t kOffItem = kOffMask + 4096;   // 2 buffers x {nodes, first output row (2 words), spare}
 constexpr uint32_t kOffBar = kOffItem + 64;
@@ -113,7 +113,7 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
   const uint32_t sbase = smem_u32(sm);
   float* Gs = reinterpret_cast<float*>(sm + kOffGs);
   float* Cs = reinterpret_cast<float*>(sm + kOffCs);
-  uint8_t* Ps = reinterpret_cast<uint8_t*>(sm + kOffPs);
+  uint8_t* Ps_all = reinterpret_cast<uint8_t*>(sm + kOffPs);          // [2][128][kLdP]
   float* tab_s = reinterpret_cast<float*>(sm + kOffTab);              // [2][alpha[128], beta[128]]
   ulonglong2* mask_s = reinterpret_cast<ulonglong2*>(sm + kOffMask);  // [2][128]
   int32_t* item_s = reinterpret_cast<int32_t*>(sm + kOffItem);        // [2][4]
@@ -324,6 +324,23 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
         mask_s[buf * kNodes + nd] = mk[h];
         tab[nd] = al[h];
         tab[kNodes + nd] = be[h];
+        // the node's path in slot order: the set bits of (ancestors | self) from the lowest up
+        // (nodes are numbered parent before child); slots past the node's depth are never used
+        uint8_t* prow = Ps_all + (buf * kNodes + nd) * kLdP;
+        uint64_t r0 = 0ull, r1 = 0ull;
+        if (nd < n) {
+          r0 = mk[h].x | (nd < 64 ? 1ull << nd : 0ull);
+          r1 = mk[h].y | (nd >= 64 ? 1ull << (nd - 64) : 0ull);
+        }
+        int s2 = 0;
+        for (; r0 != 0ull && s2 < kSlots; ++s2) {
+          prow[s2] = (uint8_t)(__ffsll((long long)r0) - 1);
+          r0 &= r0 - 1;
+        }
+        for (; r1 != 0ull && s2 < kSlots; ++s2) {
+          prow[s2] = (uint8_t)(64 + __ffsll((long long)r1) - 1);
+          r1 &= r1 - 1;
+        }
       }
       if (lane == 0) {
         item_s[buf * 4 + 0] = n;
@@ -431,7 +448,6 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
               // unselected columns land in the padding slot of the row: no branch, no predicate
               const int slot = ((bits >> jj) & 1u) ? base + __popc(bits & ((1u << jj) - 1u)) : kSlots;
               dst[slot] = __uint_as_float(r[jj]);
-              if (part == 0) Ps[rn * kLdP + slot] = (uint8_t)(cb + jj);
             }
           }
         }
@@ -472,7 +488,7 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
         float al[NS], bt[NS], pre[NS], vec[NS];
         float Pi = 1.f;                                         // P_i: product of alpha along the path
         if (live_i) {
-          const uint32_t* pw = reinterpret_cast<const uint32_t*>(Ps + rn * kLdP);
+          const uint32_t* pw = reinterpret_cast<const uint32_t*>(Ps_all + (ph * kNodes + nd) * kLdP);
           const uint32_t pword[4] = {pw[0], pw[1], pw[2], pw[3]};
 #pragma unroll
           for (int s2 = 0; s2 < NS; ++s2) {
