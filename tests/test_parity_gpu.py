@@ -78,6 +78,23 @@ def test_c5_full_size_sampled(impl):
         assert eO <= wl.tol and eS <= wl.tol, (eO, eS)
 
 
+def test_delta_128_nodes_full_batch_sampled():
+    """The delta rule at the batch and tree size of the throughput workload (4096 items of 128
+    nodes, 27.7 per CTA of the two-row-block tensor-core kernel), O, U and the committed state on a
+    seeded sample of items."""
+    wl = inputs.workload("c5", L=1, rule=inputs.DELTA, seed=1234)
+    parents, accepted = inputs.make_trees(wl)
+    tens = inputs.make_tensors(wl)
+    O, U, Sn, tree = pu.gpu_round(wl, parents, accepted, tens, impl=tv.IMPL_TC, want_U=True, commit_with_U=True)
+    tree.device_status()
+    rng = np.random.default_rng(7)
+    items = [(int(rng.integers(wl.B)), int(rng.integers(wl.H))) for _ in range(10)]
+    items += [(0, 0), (wl.B - 1, wl.H - 1)]
+    ver, com = pu.oracle_round(wl, parents, accepted, tens, items=items)
+    eO, eU, eS = pu.compare(wl, O, U, Sn, ver, com)
+    assert eO <= wl.tol and eU <= wl.tol and eS <= wl.tol, (eO, eU, eS)
+
+
 EDGE = [
     # T, dk, dv, B, H, tree, shared tree
     (1, 64, 64, 2, 2, "chain", False),
