@@ -699,8 +699,9 @@ def main():
     ap.add_argument("--ref-items", type=int, default=8)
     ap.add_argument("--traffic", type=float, default=None,
                     help="ncu dram bytes per verify launch to echo into roofline.traffic")
-    ap.add_argument("--probe-every", type=int, default=8,
-                    help="record per-kernel CUDA events on every n-th timed step")
+    ap.add_argument("--probe-every", type=int, default=0,
+                    help="record per-kernel CUDA events on every n-th timed step "
+                         "(0: every 8th, or steps/64 if that is larger: about 64 samples)")
     ap.add_argument("--packed", action="store_true",
                     help="run the step on a packed forest of requests with different node counts (1 GPU)")
     ap.add_argument("--no-e2e", action="store_true")
@@ -712,6 +713,8 @@ def main():
     if args.steps is None:
         args.steps = 200 if args.impl == "reference" else (20 if args.workload == "c5" else 5000)
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.probe_every <= 0:
+        args.probe_every = max(8, args.steps // 64)
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
