@@ -471,7 +471,9 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       if (!(ok = mbar_wait_warp(bar(G_DONE), ph, abort_flag))) break;
       if (warp == 4) TCD_STAMP(it, 18);
       tc_fence_after();
-      if (rows_live) {
+      // A node's ancestors have smaller numbers than the node: the rows of nodes 0..31 select
+      // nothing among the columns 32..63, and the warp that would scan them skips the chunk.
+      if (rows_live && !(hc == 1 && (quad & 1) == 0)) {
         const uint64_t sel = node < Tb ? (part == 0 ? (m | (1ull << node)) : m) : 0ull;
         float* dst = (part == 0 ? Cs : Gs) + node * kLd;
         const int cbase = hc * 32;

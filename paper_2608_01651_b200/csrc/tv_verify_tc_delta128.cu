@@ -437,6 +437,9 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
           float* dst = part == 0 ? Cs + rn * kLd : Gs + nd * kLd;
           for (int c = 0; c <= b; ++c) {
             const int cb = hc * 32 * (b + 1) + 32 * c;   // first column of this chunk of 32
+            // ancestors have smaller numbers than the node: nothing to select at or past the
+            // column after the warp's last node
+            if (cb > kBlk * b + (quad & 1) * 32 + 31) continue;
             const uint32_t bits = cb < 64 ? (uint32_t)(s0 >> cb) : (uint32_t)(s1 >> (cb - 64));
             const int base = cb < 64 ? __popcll(s0 & ((1ull << cb) - 1ull))
                                      : __popcll(s0) + __popcll(s1 & ((1ull << (cb - 64)) - 1ull));
