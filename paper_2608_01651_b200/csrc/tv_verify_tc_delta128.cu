@@ -19,18 +19,20 @@
 //     Qf   = D_P Q_b (written to TMEM by the compute warps)
 //          + sum over column halves h of [-(W D_P) ; -(A D_P)]_h K_h          (bf16 hi/lo)
 //     acc  = Qf S_pre^T (tf32, A operand from TMEM) + sum over h of [W ; A]_h V_h
-//     O rows and U rows of the block leave from registers.
+//     O rows and U rows of the block leave half by TMA (staged in the idle coefficient tiles),
+//     half from registers (packed forests: all from registers).
 // The Gram products of both blocks are issued as soon as Q and K have landed; the output of a
 // block is read out after the row solve of the next block (of the next item for block 1), when
-// its MMAs are long complete.  Eleven warps: TMA producer, MMA issuer, eight compute warps, one
-// warp that stages the next item's ancestor masks and gates.  Every wait is a bounded mbarrier wait; no TMA multicast.
+// its MMAs are long complete.  Twelve warps: TMA producer, MMA issuer, eight compute warps, one
+// warp that stages the next item's ancestor masks, gates and path tables, one that issues the
+// output stores.  Every wait is a bounded mbarrier wait; no TMA multicast.
 #include "tv_tc_common.cuh"
 
 namespace {
 
 using namespace tvtc;
 
-constexpr int kThreads = 352;
+constexpr int kThreads = 384;
 constexpr int kComputeWarps = 8;
 constexpr int kSlots = 16;     // path slots per node: depth <= 15
 constexpr int kNodes = 128;    // T <= 128
@@ -57,7 +59,7 @@ constexpr uint32_t kSmemBytes = kOffMisc + 64 + 1024;
 enum Bar {
   QK_FULL = 0, QK_FREE, S_FULL, S_FREE, V_FULL, V_FREE,
   GD0, GD1, GF0, GF1, TILE_READY, TILE_FREE, D1_DONE, QF_FREE, ACC_DONE, ACC_FREE, E1_SYNC,
-  META_FULL, META_FULL1, META_FREE, META_FREE1
+  META_FULL, META_FULL1, META_FREE, META_FREE1, OST_READY, OST_FREE
 };
 
 constexpr uint32_t kColSc0 = 0, kColQf = 128, kColAcc = 256, kColSc1 = 384;
@@ -107,6 +109,7 @@ template <int DMAX, bool PACKED>
 __global__ void __launch_bounds__(kThreads, 1)
 verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                           const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmS,
+                          const __grid_constant__ CUtensorMap tmO, const __grid_constant__ CUtensorMap tmU,
                           const Delta128Params p) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* sm = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -139,6 +142,7 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
     mbar_init(bar(E1_SYNC), kComputeWarps);
     mbar_init(bar(META_FULL), 1);  mbar_init(bar(META_FULL1), 1);
     mbar_init(bar(META_FREE), kComputeWarps); mbar_init(bar(META_FREE1), kComputeWarps);
+    mbar_init(bar(OST_READY), kComputeWarps); mbar_init(bar(OST_FREE), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -350,6 +354,32 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(buf ? META_FULL1 : META_FULL));
     }
+  } else if (warp == kComputeWarps + 3) {
+    // ===================== output stores (dense layout) =====================
+    // Half of every block's output (columns 0..31 and 64..95 of its O and U rows) is staged in the
+    // coefficient tiles, which are idle between the last MMA of a block and the first tile of the
+    // next, and leaves by TMA; OST_FREE tells the compute warps that the tiles may be rewritten.
+    // The other half leaves from registers.  Rows past the tree are clipped by the TMA unit.
+    if constexpr (!PACKED) {
+      if (lane == 0) {
+        uint32_t r = 0;
+        bool ok = true;
+        for (int item = blockIdx.x; ok && item < p.n_items; item += gridDim.x) {
+          for (int b = 0; b < 2; ++b, ++r) {
+            if (!(ok = mbar_wait(bar(OST_READY), r & 1, abort_flag))) break;
+#pragma unroll
+            for (int hc2 = 0; hc2 < 2; ++hc2) {
+              tma_store_3d(&tmO, sbase + kOffCoef + hc2 * 8192, 64 * hc2, kBlk * b, item);
+              if (want_U) tma_store_3d(&tmU, sbase + kOffCoef + (2 + hc2) * 8192, 64 * hc2, kBlk * b, item);
+            }
+            tma_store_commit();
+            tma_store_wait_read();
+            mbar_arrive(bar(OST_FREE));
+          }
+        }
+        tma_store_wait_all();
+      }
+    }
   } else if (warp >= 2 && warp < 2 + kComputeWarps) {
     // ===================== compute warps =====================
     const int cw = warp - 2;
@@ -367,8 +397,12 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
     if (warp == 2 && lane == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     // acc rows 0..63 -> O rows, rows 64..127 -> U rows of block pb of an item with pn nodes whose
-    // output rows start at row prow0: straight from registers, 32 bytes per store (each thread owns
-    // 64 consecutive floats of one row, so every store fills a whole sector)
+    // output rows start at row prow0.  Each thread owns 64 consecutive floats of one row.  Dense
+    // layout: the first 32 go to a swizzled staging chunk in the (idle) coefficient tiles and leave
+    // by TMA, the other 32 leave from registers in 32-byte stores (whole sectors); a warp-wide
+    // register store touches 32 different lines and keeps the load/store unit busy for as many
+    // cycles, so halving them is what this buys.  Packed forest: both halves from registers, rows
+    // past the request skipped.
     auto read_out = [&](size_t prow0, int pn, int pb) -> bool {
       if (!mbar_wait_warp(bar(ACC_DONE), (uint32_t)pb, abort_flag)) return false;
       tc_fence_after();
@@ -379,7 +413,13 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
           uint32_t r1[32];
           tmem_ld32(tmem + lane_addr + kColAcc + hc * 64 + half * 32, r1);
           tmem_wait_ld();
-          if (nd < pn) {
+          if (!PACKED && half == 0) {
+            unsigned char* orow = sm + kOffCoef + (part * 2 + hc) * 8192 + rn * 128;
+#pragma unroll
+            for (int c = 0; c < 8; ++c)
+              *reinterpret_cast<uint4*>(orow + (((uint32_t)c ^ nswz) << 4)) =
+                  make_uint4(r1[4 * c], r1[4 * c + 1], r1[4 * c + 2], r1[4 * c + 3]);
+          } else if (nd < pn) {
             float* o = (part == 0 ? p.O : p.U) + (prow0 + nd) * 128 + hc * 64 + half * 32;
 #pragma unroll
             for (int c = 0; c < 4; ++c)
@@ -390,15 +430,20 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
           }
         }
       }
+      if (!PACKED) fence_async_smem();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar(ACC_FREE));
+      if (lane == 0) {
+        mbar_arrive(bar(ACC_FREE));
+        if (!PACKED) mbar_arrive(bar(OST_READY));
+      }
       return true;
     };
     const int total_rows = PACKED ? p.offsets[p.B] : 0;   // rows at and past this one hold no node
 
     uint32_t it = 0;
     bool ok = true;
+    uint32_t n_read = 0;      // read-outs done so far (one per block, from the second block on)
     int pn = -1, pb = 0;      // block whose output is still in TMEM: nodes of its item, block,
     size_t prow0 = 0;         // first output row of its item
     int Tn = T;               // nodes of the current item
@@ -506,7 +551,10 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
         }
         // ---- output of the block before: its MMAs ran under E1 and the gather above ----
         D128_STAMP(2 * it + b, 4);
-        if (pn >= 0 && !(ok = read_out(prow0, pn, pb))) break;
+        if (pn >= 0) {
+          if (!(ok = read_out(prow0, pn, pb))) break;
+          ++n_read;
+        }
         D128_STAMP(2 * it + b, 5);
         if (live_i) {
           // C_{i,p_s} = (q_i . k_{p_s}) P_i / P_{p_s}: the ratio is the product of alpha over the
@@ -568,6 +616,8 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
         // ---- coefficient tiles, one column half of one matrix at a time: thread hc = 0 writes the
         // hi tile, hc = 1 the lo tile of its row ----
         D128_STAMP(2 * it + b, 7);
+        // the staged half of the block read out above has left the coefficient tiles
+        if (!PACKED && n_read > 0 && !(ok = mbar_wait_warp(bar(OST_FREE), (n_read - 1) & 1, abort_flag))) break;
         const int n_builds = b ? 4 : 2;
         for (int q = 0; q < n_builds; ++q) {
           const uint32_t j = b ? 2u + q : (uint32_t)q;    // build number within the item
@@ -640,7 +690,10 @@ int tv_launch_verify_tc_delta128(const VerifyArgs& a, int32_t* status, cudaStrea
   const uint64_t items = (uint64_t)a.L * a.B * a.H;
   const uint64_t qk_items = (uint64_t)a.L * a.B * a.Hk;
   const bool packed = a.tree.offsets != nullptr;
-  const void* const ptrs[5] = {a.q, a.k, a.v, a.S_pre, nullptr};
+  float* Uout = a.U ? a.U : a.O;   // never written when U is not requested
+  const void* const ptrs[5] = {a.q, a.k, a.v, a.S_pre, a.O};
+  const void* const uptrs[5] = {Uout, nullptr, nullptr, nullptr, (const void*)3};
+  const MapSet* mu = nullptr;   // dense layout: U in boxes of 64 rows x 32 columns
   // q, k, v in boxes of 64 rows x 64 columns (rows past the tensor read as zero), S_pre in 4 chunks
   // of 32 columns; a packed forest addresses (layer, head) planes of `capacity` rows
   const MapSet* ms = nullptr;
@@ -649,8 +702,13 @@ int tv_launch_verify_tc_delta128(const VerifyArgs& a, int32_t* status, cudaStrea
       return make_map(&m[0], a.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, qk_items, a.T, 128, 64, 64) &&
              make_map(&m[1], a.k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, qk_items, a.T, 128, 64, 64) &&
              make_map(&m[2], a.v, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, items, a.T, 128, 64, 64) &&
-             make_map(&m[3], a.S_pre, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, 128, 128, 32, 128);
+             make_map(&m[3], a.S_pre, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, 128, 128, 32, 128) &&
+             make_map(&m[4], a.O, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, a.T, 128, 32, 64);
     });
+    mu = cached_maps(uptrs, items, a.T, 11, [&](CUtensorMap* m) {
+      return make_map(&m[0], Uout, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, a.T, 128, 32, 64);
+    });
+    if (!mu) return TV_ERR_CUDA;
   } else {
     const uint64_t cap = (uint64_t)a.tree.capacity;
     const uint64_t pv = (uint64_t)a.L * a.H, pqk = (uint64_t)a.L * a.Hk;
@@ -687,14 +745,15 @@ int tv_launch_verify_tc_delta128(const VerifyArgs& a, int32_t* status, cudaStrea
   p.want_U = a.U != nullptr;
   p.status = status;
   p.O = a.O;
-  p.U = a.U ? a.U : a.O;   // never written when U is not requested
+  p.U = Uout;
   const int grid = (int)(items < (uint64_t)sm_count ? items : (uint64_t)sm_count);
   p.offsets = a.tree.offsets;
   p.capacity = a.tree.capacity;
   const bool shallow = a.tree.max_depth_all <= 8;
   auto launch = [&](auto kernel) {
+    // packed forests store from registers only: the output maps are placeholders there
     return launch_dependent(kernel, grid, kThreads, kSmemBytes, stream, ms->map[0], ms->map[1], ms->map[2],
-                            ms->map[3], p);
+                            ms->map[3], packed ? ms->map[3] : ms->map[4], packed ? ms->map[3] : mu->map[0], p);
   };
   if (packed)
     TV_CUDA_TRY(shallow ? launch(verify_tc_delta128_kernel<8, true>) : launch(verify_tc_delta128_kernel<15, true>));
