@@ -123,6 +123,21 @@ def test_tc_delta_depth_15(T):
     assert eO <= wl.tol and eU <= wl.tol and eS <= wl.tol
 
 
+@pytest.mark.parametrize("T", [64, 100, 128])
+def test_tc_delta_run_to_run_identical(T):
+    """Several items per CTA, U requested and not, repeated: O and U identical bit for bit.  (A slot
+    table overwritten by a fast warp while a slow one still read it once showed up exactly here.)"""
+    wl = inputs.workload("c4", B=16, H=32, T=T, L=1, tree="frontier", seed=23 + T)
+    parents, accepted = inputs.make_trees(wl)
+    tens = inputs.make_tensors(wl)
+    outs = [pu.gpu_round(wl, parents, accepted, tens, impl=tv.IMPL_TC, want_U=w)[:2]
+            for w in (True, True, False, False, True, False)]
+    for O, U in outs[1:]:
+        assert np.array_equal(O, outs[0][0])
+        if U is not None:
+            assert np.array_equal(U, outs[0][1])
+
+
 def test_tc_delta_falls_back_on_deep_trees():
     wl = inputs.workload("c4", B=1, H=2, T=40, tree="chain", seed=5)   # depth 39 > 15
     parents, accepted = inputs.make_trees(wl)
