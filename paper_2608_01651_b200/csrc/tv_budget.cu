@@ -91,7 +91,9 @@ budget_select_kernel(const uint32_t* __restrict__ key, int32_t N, int32_t K, int
   __shared__ int need_s;
   __shared__ int warp_tot[32];
   __shared__ int total_s;
+  __shared__ int cnt_s[kSelThreads];   // kept nodes per request (B <= kSelThreads)
   const int tid = threadIdx.x;
+  cnt_s[tid] = 0;
   if (tid == 0) {
     prefix_s = 0;
     need_s = K;
@@ -107,11 +109,16 @@ budget_select_kernel(const uint32_t* __restrict__ key, int32_t N, int32_t K, int
       if (pass == 0 || (k >> (shift + 8)) == prefix) atomicAdd(&hist[(k >> shift) & 255u], 1);
     }
     __syncthreads();
-    if (tid == 0) {
-      int need = need_s, d = 255;
-      while (d > 0 && hist[d] < need) need -= hist[d--];
-      prefix_s = (prefix << 8) | (uint32_t)d;
-      need_s = need;   // how many keys with this prefix still have to be taken
+    // the digit whose bucket holds the need-th largest key: thread t looks at digit 255 - t and
+    // at the number of keys in the higher buckets (a prefix sum over the CTA, not a serial walk)
+    {
+      const int need = need_s;
+      const int mine = tid < 256 ? hist[255 - tid] : 0;
+      const int above = block_exclusive_scan(mine, warp_tot, &total_s);
+      if (tid < 256 && above < need && above + mine >= need) {
+        prefix_s = (prefix << 8) | (uint32_t)(255 - tid);
+        need_s = need - above;   // how many keys with this prefix still have to be taken
+      }
     }
     __syncthreads();
   }
@@ -128,12 +135,11 @@ budget_select_kernel(const uint32_t* __restrict__ key, int32_t N, int32_t K, int
     bool take = k > tau;
     if (k == tau) take = before++ < need;
     keep[i] = take ? 1 : 0;
+    if (take) atomicAdd(&cnt_s[i / Tc], 1);
   }
   __syncthreads();
   // ---- per-request counts and their exclusive prefix sums (B <= kSelThreads) ----
-  int c = 0;
-  if (tid < B)
-    for (int i = 0; i < Tc; ++i) c += keep[(size_t)tid * Tc + i];
+  const int c = tid < B ? cnt_s[tid] : 0;
   const int off = block_exclusive_scan(c, warp_tot, &total_s);
   if (tid < B) {
     counts[tid] = c;
