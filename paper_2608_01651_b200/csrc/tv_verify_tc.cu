@@ -31,7 +31,7 @@ namespace {
 
 using namespace tvtc;
 
-constexpr int kThreads = 320;
+constexpr int kThreads = 352;     // producer, MMA issuer, 8 compute warps, output-store warp
 constexpr int kComputeWarps = 8;
 
 // shared memory map (byte offsets from the 1024-aligned base)
@@ -266,6 +266,50 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         TC_STAMP(it, 11);
       }
     }
+  } else if (warp == kComputeWarps + 2) {
+    // ===================== output stores =====================
+    // The staged chunks of an item leave by TMA once all compute warps have written them
+    // (OST_READY); OST_FREE tells them that the chunks have been read.  T <= 64: the chunks are
+    // not the C' tiles, and OST_FREE phase k says that the store of item k-1 is read (phase 0
+    // is given away up front).  T > 64: phase k = the store of item k.
+    if (lane == 0) {
+      const bool small = T <= 64;
+      auto stage_addr = [&](int c4) -> uint32_t {
+        return small ? kOffChi + kTile + (uint32_t)(c4 >> 1) * (kOffClo - kOffChi) + (uint32_t)(c4 & 1) * 8192u
+                     : kOffChi + (uint32_t)c4 * kTile;
+      };
+      if (small) mbar_arrive(bar(OST_FREE));
+      uint32_t it = 0;
+      for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++it) {
+        if (!mbar_wait(bar(OST_READY), it & 1, abort_flag)) break;
+        if constexpr (PACKED) {
+          // groups of 8 rows, largest boxes first; staging rows r.. start on a 1024-byte
+          // boundary, so the swizzle phase of a partial box equals that of the full tile
+          const PackedItem pk = packed_item(p, item);
+          const int full = pk.n & ~7;
+          int r = 0;
+          auto put = [&](const CUtensorMap* m, int rows_box) {
+            while (full - r >= rows_box) {
+#pragma unroll
+              for (int c = 0; c < 4; ++c)
+                tma_store_3d(m, sbase + stage_addr(c) + (uint32_t)r * 128u, 32 * c, pk.row0 + r, pk.plane_v);
+              r += rows_box;
+            }
+          };
+          put(&tmO, 64);
+          put(&tmO32, 32);
+          put(&tmO16, 16);
+          put(&tmO8, 8);
+        } else {
+#pragma unroll
+          for (int c = 0; c < 4; ++c) tma_store_3d(&tmO, sbase + stage_addr(c), 32 * c, 0, item);
+        }
+        tma_store_commit();
+        tma_store_wait_read();
+        mbar_arrive(bar(OST_FREE));
+      }
+      tma_store_wait_all();   // our stores are complete before we leave
+    }
   } else {
     // ===================== compute warps =====================
     const int cw = warp - 2;
@@ -293,13 +337,8 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       const int acc_done = (it_prev & 1) ? ACC_DONE1 : ACC_DONE0;
       const int acc_free = (it_prev & 1) ? ACC_FREE1 : ACC_FREE0;
       const uint32_t acc_col = (it_prev & 1) ? kColAcc1 : kColAcc0;
-      if (small) {
-        if (warp == 2 && lane == 0) {
-          tma_store_wait_read();          // the store of the item before has read the chunks
-          mbar_arrive(bar(OST_FREE));
-        }
-        if (!mbar_wait_warp(bar(OST_FREE), ost_phase, abort_flag)) return false;
-      }
+      // T <= 64: the store of the item before has read the staging chunks
+      if (small && !mbar_wait_warp(bar(OST_FREE), ost_phase, abort_flag)) return false;
       if (!mbar_wait_warp(bar(acc_done), (it_prev >> 1) & 1, abort_flag)) return false;
       tc_fence_after();
       if (warp_live) {
@@ -332,35 +371,6 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       if (lane == 0) {
         mbar_arrive(bar(acc_free));
         mbar_arrive(bar(OST_READY));
-      }
-      if (warp == 2 && lane == 0) {
-        if (mbar_wait(bar(OST_READY), ost_phase, abort_flag)) {
-          if constexpr (PACKED) {
-            // groups of 8 rows, largest boxes first; staging rows r.. start on a 1024-byte
-            // boundary, so the swizzle phase of a partial box equals that of the full tile
-            const int full = pk_prev.n & ~7;
-            int r = 0;
-            auto put = [&](const CUtensorMap* m, int rows_box) {
-              while (full - r >= rows_box) {
-#pragma unroll
-                for (int c = 0; c < 4; ++c)
-                  tma_store_3d(m, sbase + stage_addr(c) + (uint32_t)r * 128u, 32 * c, pk_prev.row0 + r,
-                               pk_prev.plane_v);
-                r += rows_box;
-              }
-            };
-            put(&tmO, 64);
-            put(&tmO32, 32);
-            put(&tmO16, 16);
-            put(&tmO8, 8);
-          } else {
-#pragma unroll
-            for (int c = 0; c < 4; ++c) tma_store_3d(&tmO, sbase + stage_addr(c), 32 * c, 0, item_prev);
-          }
-          tma_store_commit();
-          if (!small) tma_store_wait_read();   // the tiles may be overwritten once the store has read them
-        }
-        if (!small) mbar_arrive(bar(OST_FREE));
       }
       return small ? true : mbar_wait_warp(bar(OST_FREE), ost_phase, abort_flag);
     };
@@ -550,7 +560,6 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       pk_prev = pk;
     }
     if (ok && it > 0) final_epilogue(it - 1, item_prev, r_prev, (it - 1) & 1, pk_prev);
-    if (warp == 2 && lane == 0) tma_store_wait_all();   // our stores are complete before we leave
   }
 
   // ---- teardown: every path comes here ----
