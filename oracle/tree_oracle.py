@@ -10,8 +10,8 @@ states.
 Notation is the paper's (Section II-B Eq. 1, Section IV-A Table II):
 one state head keeps ``S`` of shape ``[dk, dv]``; node ``i`` of the proposal
 tree has parent ``pi(i)``; ``parent[i] == -1`` marks a child of the virtual
-root whose state is the committed ``S_pre`` (Table II: "pi(i)=0 for a root
-child and S_0 = S_pre").  Nodes are indexed parent before child (Section IV-A,
+root whose state is the committed ``S_pre`` (Table II gives a root child the
+parent index 0 and defines the state of index 0 as S_pre).  Nodes are indexed parent before child (Section IV-A,
 text after Theorem 1).  Row ``i`` of ``Q, K`` is ``q_i, k_i`` (``[T, dk]``),
 row ``i`` of ``V, U, O`` is ``v_i, u_i, o_i`` (``[T, dv]``); ``gamma`` is the
 decay gate and ``beta`` the write gate (``[T]``).
@@ -28,7 +28,9 @@ Two update rules are covered:
 Pins (tests/test_oracle_pins.py): a hand-worked example, Theorem 1 evaluated
 densely, Eq. 4, Lemma 3, Eq. 10, the masked linear-attention special case,
 delta-rule retrieval, beta = 0, chain = sequential decoding, sibling
-independence, brute force over every tree of up to five nodes.
+independence, brute force over every tree of up to five nodes, and, for the
+batch wrappers at the end of this file, the hand examples laid out in the
+library's transposed state layout with dk != dv and per-request trees.
 """
 from __future__ import annotations
 

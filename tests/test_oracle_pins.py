@@ -310,3 +310,84 @@ def test_state_and_factor_sizes_match_table_one():
     assert 82 <= 4.7e9 / 57e6 < 83 and 99 <= 14.1e9 / 142e6 < 100
     # Eq. 9: one factorised node costs Theta(H (dk+dv+1)) elements, a snapshot H dk dv
     assert (H * dk * dv) / (H * (dk + dv + 1)) > 60
+
+
+# ---- the batch wrappers: library layout S^ = S^T [B,H,dv,dk], tree pick per request ----------
+def _hand_batch(rule, per_request_trees):
+    """The hand-worked examples laid out as the library stores them, with dk = 2 != dv = 3.
+
+    Every value channel of the recurrence evolves on its own and linearly in (its column of
+    S_pre, its column of V) (Sec. IV-B: value channels are independent), so a third channel
+    2*c0 - c1 must come out as 2*out0 - out1, and head 1 (S_pre and V scaled by -1/2) as -1/2
+    of head 0.  Request 1 uses either the same tree or the root-child variant of the second
+    golden file, whose node 1 differs.  All expected values trace back to the hand examples.
+    """
+    g = json.load(open(os.path.join(GOLD, "hand_example.json")))
+    g2 = json.load(open(os.path.join(GOLD, "hand_example_root_child.json")))
+    widen = lambda rows: [[r[0], r[1], 2 * r[0] - r[1]] for r in rows]        # [.., 2] -> [.., 3]
+    S3, V3 = widen(g["S_pre"]), widen(g["V"])                                  # [dk][3], [T][3]
+    B, H, T, dk, dv = 2, 2, 3, 2, 3
+    scale = [1.0, -0.5]
+    S_hat = np.zeros((B, H, dv, dk)); q = np.zeros((B, H, T, dk)); k = np.zeros((B, H, T, dk))
+    v = np.zeros((B, H, T, dv)); gamma = np.zeros((B, H, T)); beta = np.zeros((B, H, T))
+    for b in range(B):
+        for h in range(H):
+            for c in range(dv):
+                for kk in range(dk):
+                    S_hat[b, h, c, kk] = scale[h] * S3[kk][c]      # transposed by hand
+            for i in range(T):
+                for kk in range(dk):
+                    q[b, h, i, kk] = g["Q"][i][kk]
+                    k[b, h, i, kk] = g["K"][i][kk]
+                for c in range(dv):
+                    v[b, h, i, c] = scale[h] * V3[i][c]
+                gamma[b, h, i] = g["gamma"][i]
+                beta[b, h, i] = g["beta"][i]
+    parents = np.array([g["parent"], g2["parent"]]) if per_request_trees else np.array([g["parent"]])
+    # expected per request: rows of O, U and the per-node states [dk][dv], widened to 3 channels
+    exp = []
+    for b in range(B):
+        O = [list(r) for r in g[rule]["O"]]
+        U = [list(r) for r in (g[rule]["U"] if rule == "delta" else g["V"])]
+        St = [g[rule][f"S_{i}"] for i in range(T)]
+        if per_request_trees and b == 1:
+            O[1] = list(g2[rule]["O_1"])
+            if rule == "delta":
+                U[1] = list(g2[rule]["U_1"])
+            St[1] = g2[rule]["S_1"]
+        exp.append((widen(O), widen(U), [widen(s) for s in St]))
+    return (S_hat, q, k, v, gamma, beta, parents), exp, scale, widen(g["S_pre"])
+
+
+@pytest.mark.parametrize("rule", ["gated", "delta"])
+@pytest.mark.parametrize("per_request_trees", [False, True])
+@pytest.mark.parametrize("memo", [True, False])
+def test_verify_batch_layout_and_tree_pick(rule, per_request_trees, memo):
+    (S_hat, q, k, v, gamma, beta, parents), exp, scale, _ = _hand_batch(rule, per_request_trees)
+    out = orc.verify_batch(S_hat, q, k, v, gamma, None if rule == "gated" else beta, parents, rule, memo=memo)
+    assert sorted(out) == [(b, h) for b in range(2) for h in range(2)]
+    for (b, h), (O, U) in out.items():
+        Oe, Ue, _ = exp[b]
+        assert O.shape == (3, 3) and U.shape == (3, 3)
+        assert np.array_equal(O, scale[h] * np.array(Oe)), (b, h)
+        assert np.array_equal(U, scale[h] * np.array(Ue)), (b, h)
+    # the item list restricts the work and keeps the indexing
+    one = orc.verify_batch(S_hat, q, k, v, gamma, beta, parents, rule, memo=memo, items=[(1, 1)])
+    assert list(one) == [(1, 1)] and np.array_equal(one[(1, 1)][0], out[(1, 1)][0])
+
+
+@pytest.mark.parametrize("rule", ["gated", "delta"])
+@pytest.mark.parametrize("per_request_trees", [False, True])
+def test_commit_batch_layout_and_tree_pick(rule, per_request_trees):
+    (S_hat, q, k, v, gamma, beta, parents), exp, scale, S3 = _hand_batch(rule, per_request_trees)
+    for accepted in ([2, 1], [1, -1], [-1, 0]):
+        out = orc.commit_batch(S_hat, k, v, gamma, None if rule == "gated" else beta, parents, accepted, rule)
+        for (b, h), Sn in out.items():
+            a = accepted[b]
+            S_paper = S3 if a < 0 else exp[b][2][a]                  # [dk][dv]
+            want = np.zeros((3, 2))
+            for c in range(3):
+                for kk in range(2):
+                    want[c, kk] = scale[h] * S_paper[kk][c]          # library layout [dv][dk]
+            assert Sn.shape == (3, 2)
+            assert np.array_equal(Sn, want), (accepted, b, h)
