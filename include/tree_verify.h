@@ -137,7 +137,9 @@ int tv_tree_meta_device(tv_tree* tree, uint64_t* anc, int32_t* depth, void* stre
 /* Synchronises `stream` and reports whether any kernel launched with this tree
  * since its last upload gave up on a bounded device-side wait (a TMA or tensor-
  * core completion that never came): TV_OK or TV_ERR_DEVICE_TIMEOUT.  After a
- * timeout the outputs of that launch are undefined; the context stays usable. */
+ * timeout the outputs of that launch are undefined; the context stays usable.
+ * TV_ERR_UNSUPPORTED: the trees of the last tv_forest_upload_device were deeper
+ * than the bound that call was given.                                         */
 int tv_tree_device_status(tv_tree* tree, void* stream);
 /* Self-test of that mechanism: launches one CTA that waits, with a limit of a
  * few milliseconds, on a barrier nothing ever signals, and writes what the
@@ -198,8 +200,11 @@ int tv_forest_rebuild(tv_tree* forest, const int32_t* parent_flat /*host*/,
  * tv_forest_upload_device reads: it derives the masks and depths of a forest
  * handle (tv_forest_build with the same n_req, n_max = n_cand, capacity >=
  * budget) from DEVICE memory, with no host copy.  max_depth_bound must bound the
- * depth of every candidate tree (kernel choice depends on it; a wrong bound
- * gives wrong results).  After it the handle's host-side metadata is stale:
+ * depth of every candidate tree (the kernel choice depends on it).  The device
+ * checks it: a node with more ancestors keeps only its nearest max_depth_bound
+ * of them, so every kernel stays within its tables, the results of that round
+ * are not the tree's, and tv_tree_device_status returns TV_ERR_UNSUPPORTED
+ * until the next upload.  After it the handle's host-side metadata is stale:
  * tv_tree_meta and tv_tree_path return TV_ERR_UNSUPPORTED until the next
  * tv_forest_rebuild + tv_tree_upload.                                          */
 size_t tv_budget_workspace_bytes(int32_t n_req, int32_t n_cand);
@@ -275,12 +280,13 @@ int tv_tree_verify_static(const int32_t* parent /*dev*/, int32_t n_trees, const 
  * tv_tree_verify, or NULL -- then TV_GATED uses u_j = v_j and TV_GATED_DELTA
  * re-derives u_j along the accepted path from S_pre (needs dk in {64,128}).
  * S_new may alias S_pre exactly (in place) or not overlap it at all.
- * Stream order: when the call directly follows tv_tree_verify on the same
- * stream, the commit grid may be scheduled while the verify kernel drains and
- * read S_pre and accepted early; it reads U and writes S_new only after that
- * kernel has completed.  (Behind any other work it starts after that work, as
- * usual.)  So accepted, S_pre, k, v, alpha must not be outputs of the
- * tv_tree_verify call in front of it -- U is the only one that may be.        */
+ * Stream order: when the call directly follows tv_tree_verify, tv_tree_upload
+ * or tv_forest_upload_device on the same stream, the commit grid may be
+ * scheduled while that kernel drains and read S_pre and accepted early; it
+ * reads the tree metadata and U, and writes S_new, only after that kernel has
+ * completed.  (Behind any other work it starts after that work, as usual.)  So
+ * accepted and S_pre must not be outputs of the library call in front of it --
+ * U and the tree metadata are the only ones that may be.                      */
 int tv_commit_path(const tv_tree* tree, const tv_dims* dims,
                    const int32_t* accepted /*dev [B]*/,
                    const float* S_pre /*dev*/,
@@ -356,11 +362,8 @@ typedef struct tv_conv_dims {
   int32_t io_dtype;      /* tv_dtype of x, ctx, gate_a, gate_b, q, k, v  */
   int32_t normalize_qk;  /* 0 / 1                                        */
   float eps;             /* added under the square root                  */
-  int32_t impl;          /* TV_IMPL_AUTO / TV_IMPL_SIMT: the CUDA-core kernel.
-                            TV_IMPL_TC: a variant with the taps as mma.sync tiles
-                            (filter split into three bf16 pieces), for bf16 heads
-                            of 128 channels and W <= 4 only (TV_ERR_UNSUPPORTED
-                            otherwise); measured slower, kept for comparison  */
+  int32_t impl;          /* TV_IMPL_AUTO / TV_IMPL_SIMT: the CUDA-core kernel (the only
+                            one); TV_IMPL_TC returns TV_ERR_UNSUPPORTED      */
 } tv_conv_dims;
 
 int tv_tree_conv(const tv_tree* tree, const tv_conv_dims* dims, const void* x, const void* ctx,

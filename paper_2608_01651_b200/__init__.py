@@ -412,6 +412,10 @@ def tree_verify_static(parent, S_pre, q, k, v, alpha, beta=None, *, rule=GATED, 
         _require(t, n, k.dtype)
     d = _dims(S_pre, k, v, rule, impl)
     n_trees = parent.shape[0] if parent.dim() == 2 else 1
+    if parent.dim() not in (1, 2) or parent.shape[-1] != d.T:
+        raise ValueError("parent must be [T] or [n_trees, T] with T = the node count of q/k/v")
+    if n_trees not in (1, d.B):
+        raise ValueError("parent must hold one tree or one tree per request")
     _check(lib().tv_tree_verify_static(_ptr(parent), n_trees, ctypes.byref(d), _ptr(S_pre), _ptr(q),
                                        _ptr(k), _ptr(v), _ptr(alpha), _ptr(beta), _ptr(O), _ptr(U),
                                        _ptr(status), _stream_ptr(stream)), "tv_tree_verify_static")

@@ -213,6 +213,12 @@ TV_API int tv_tree_path(const tv_tree* t, const int32_t* accepted, int32_t n_req
 
 // Device mirror of the metadata (masks | depths | parents | offsets | status word) and the two
 // pinned staging slots; allocated by the first upload, reused by every later one.
+// Upload generations count 1, 2, ... and wrap long before the sign bit (0 = "never").
+static int32_t next_gen(tv_tree* t) {
+  t->upload_gen = t->upload_gen % 0x3fffffff + 1;
+  return t->upload_gen;
+}
+
 struct BlobLayout {
   size_t anc_b, i32_b, off_b, total, slot_b;
 };
@@ -233,7 +239,8 @@ static int ensure_device(tv_tree* t, const BlobLayout& L) {
   if (t->d_blob && (t->device != dev || t->blob_bytes != L.total)) return TV_ERR_BAD_ARG;
   if (t->d_blob) return TV_OK;
   TV_CUDA_TRY(cudaMalloc(&t->d_blob, L.total));
-  cudaError_t e = cudaHostAlloc(&t->h_stage, 2 * L.slot_b, cudaHostAllocMapped);
+  cudaError_t e = cudaMemset((char*)t->d_blob + L.total - 16, 0, 16);   // status words start at zero
+  if (e == cudaSuccess) e = cudaHostAlloc(&t->h_stage, 2 * L.slot_b, cudaHostAllocMapped);
   void* mapped = nullptr;
   if (e == cudaSuccess) e = cudaHostGetDevicePointer(&mapped, t->h_stage, 0);
   for (int i = 0; i < 2 && e == cudaSuccess; ++i)
@@ -276,6 +283,7 @@ TV_API int tv_tree_upload(tv_tree* t, void* stream) {
                                     t->d_status, t->offsets.empty() ? nullptr : t->offsets.data(),
                                     t->d_offsets_w, s);
     if (st != TV_OK) return st;
+    next_gen(t);   // host-built trees cannot break a depth bound: only the generation moves on
     t->uploaded = true;
     t->host_meta_valid = true;
     return TV_OK;
@@ -294,7 +302,8 @@ TV_API int tv_tree_upload(tv_tree* t, void* stream) {
     off_mapped = (const int32_t*)((const char*)t->h_stage_dev + slot * L.slot_b + L.i32_b);
   }
   st = tv_launch_tree_meta((const int32_t*)((const char*)t->h_stage_dev + slot * L.slot_b), t->n_trees, t->n,
-                           t->d_anc_w, t->d_depth_w, t->d_parent_w, t->d_status, off_mapped, t->d_offsets_w, s);
+                           t->d_anc_w, t->d_depth_w, t->d_parent_w, t->d_status, off_mapped, t->d_offsets_w, t->n,
+                           next_gen(t), s);
   if (st != TV_OK) return st;
   TV_CUDA_TRY(cudaEventRecord(t->staged[slot], s));
   t->uploaded = true;
@@ -313,7 +322,7 @@ TV_API int tv_forest_upload_device(tv_tree* t, const int32_t* parent_padded, con
   int st = ensure_device(t, L);
   if (st != TV_OK) return st;
   st = tv_launch_tree_meta(parent_padded, t->n_trees, t->n, t->d_anc_w, t->d_depth_w, t->d_parent_w, t->d_status,
-                           offsets, t->d_offsets_w, (cudaStream_t)stream);
+                           offsets, t->d_offsets_w, max_depth_bound, next_gen(t), (cudaStream_t)stream);
   if (st != TV_OK) return st;
   t->max_depth_all = max_depth_bound;
   t->uploaded = true;
@@ -335,10 +344,12 @@ TV_API int tv_tree_meta_device(tv_tree* t, uint64_t* anc, int32_t* depth, void* 
 TV_API int tv_tree_device_status(tv_tree* t, void* stream) {
   if (!t) return TV_ERR_BAD_ARG;
   if (!t->d_status) return TV_ERR_NOT_UPLOADED;
-  int32_t st = 0;
-  TV_CUDA_TRY(cudaMemcpyAsync(&st, t->d_status, sizeof(st), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+  int32_t st[2] = {0, 0};
+  TV_CUDA_TRY(cudaMemcpyAsync(st, t->d_status, sizeof(st), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
   TV_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
-  return st == 0 ? TV_OK : TV_ERR_DEVICE_TIMEOUT;
+  if (st[0] != 0) return TV_ERR_DEVICE_TIMEOUT;
+  if (st[1] != 0 && st[1] == t->upload_gen) return TV_ERR_UNSUPPORTED;   // trees deeper than the stated bound
+  return TV_OK;
 }
 
 TV_API int tv_tree_free(tv_tree* t) {

@@ -174,8 +174,6 @@ __global__ void __launch_bounds__(kRowThreads) commit_factored_dk128_kernel(Comm
   const int dv = a.dv;
   const int n_half = (dv + kRowsPerCta - 1) / kRowsPerCta;
   const int item = blockIdx.x / n_half, half = blockIdx.x - item * n_half;
-  const ItemRows rows = tv_item_rows(a.tree, item, a.B, a.H, a.Hk, a.T);
-  const int T = rows.n;
   const int b = (item / a.H) % a.B;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int row0 = half * kRowsPerCta + warp * 16;
@@ -184,17 +182,23 @@ __global__ void __launch_bounds__(kRowThreads) commit_factored_dk128_kernel(Comm
   float4* dst = reinterpret_cast<float4*>(a.S_new + sbase) + (size_t)row0 * 32 + lane;
 
   int acc = a.accepted[b];
-  if (acc >= T) acc = -1;
+  if (acc >= a.T) acc = -1;
   if (acc < 0 && a.S_new == a.S_pre) return;
   float4 s[16];
 #pragma unroll
   for (int e = 0; e < 16; ++e)
     if (row0 + e < dv) s[e] = ld_stream(src + e * 32);
-  // Dependent launch: this grid may have started under the tail of the verify kernel in front
-  // of it.  S_pre and the accepted nodes are older than that kernel; everything it writes (U)
-  // is read, and everything it reads that we write (S in place) is written, after this point.
+  // Dependent launch: this grid may have started under the tail of the kernel in front of it
+  // (a verify kernel, or the tree-metadata kernel when no verify call sits in between).  S_pre
+  // and the accepted nodes are older than either; everything those kernels write -- U, and the
+  // tree metadata including the request offsets of a packed forest -- is read, and everything
+  // they read that we write (S in place) is written, after this point.
   asm volatile("griddepcontrol.wait;" ::: "memory");
+  const ItemRows rows = tv_item_rows(a.tree, item, a.B, a.H, a.Hk, a.T);
+  const int T = rows.n;
+  if (acc >= T) acc = -1;   // packed forest: beyond this request's node count
   if (acc < 0) {
+    if (a.S_new == a.S_pre) return;
 #pragma unroll
     for (int e = 0; e < 16; ++e)
       if (row0 + e < dv) st_stream(dst + e * 32, s[e]);

@@ -23,7 +23,9 @@ struct tv_tree {
   uint64_t* d_anc_w = nullptr;
   int32_t* d_depth_w = nullptr;
   int32_t* d_parent_w = nullptr;
-  int32_t* d_status = nullptr;  // device status word (0 = ok), cleared by every upload
+  int32_t* d_status = nullptr;  // device status: [0] timeout flag (0 = ok), cleared by every upload;
+                                // [1] generation of the last upload whose trees broke their depth bound
+  int32_t upload_gen = 0;       // generation of the latest upload (counts from 1)
   bool uploaded = false;
   bool host_meta_valid = true;   // false after tv_forest_upload_device: the topology lives on the device only
   // Packed forest (tv_forest_build): tree t has offsets[t+1] - offsets[t] <= n real nodes (its
@@ -120,7 +122,7 @@ int tv_launch_verify_simt(const VerifyArgs& a, cudaStream_t stream);
 int tv_launch_commit(const CommitArgs& a, cudaStream_t stream);
 int tv_launch_tree_meta(const int32_t* parent_mapped, int32_t n_trees, int32_t n, uint64_t* anc,
                         int32_t* depth, int32_t* parent_dev, int32_t* status, const int32_t* offsets_mapped,
-                        int32_t* offsets_dev, cudaStream_t stream);
+                        int32_t* offsets_dev, int32_t depth_bound, int32_t generation, cudaStream_t stream);
 // Host parents carried in the kernel parameters (small tree sets): no staging, no read over the bus.
 bool tv_tree_meta_fits_params(int32_t n_trees, int32_t n, bool has_offsets);
 int tv_launch_tree_meta_params(const int32_t* parent_host, int32_t n_trees, int32_t n, uint64_t* anc,

@@ -126,6 +126,12 @@ TV_API int tv_session_round(tv_session* s, const int32_t* parent, const int32_t*
   if (delta && !beta) return TV_ERR_BAD_ARG;
   for (int b = 0; b < d.B; ++b)
     if (accepted[b] < -1 || accepted[b] >= d.T) return TV_ERR_BAD_ARG;
+  // malformed trees are refused before anything is queued
+  for (size_t t = 0; t < (size_t)s->n_trees; ++t)
+    for (int i = 0; i < d.T; ++i) {
+      const int32_t p = parent[t * d.T + i];
+      if (p < -1 || p >= i) return TV_ERR_INVALID_TREE;
+    }
   const size_t Hk = d.Hk ? d.Hk : d.H;
   // bytes of one request of one layer in each tensor
   const size_t rS = (size_t)d.H * d.dv * d.dk * 4, rQ = Hk * d.T * d.dk * s->eb, rV = (size_t)d.H * d.T * d.dv * s->eb,
@@ -134,12 +140,27 @@ TV_API int tv_session_round(tv_session* s, const int32_t* parent, const int32_t*
   TV_CUDA_TRY(cudaEventRecord(s->start, user));
   for (int i = 0; i < 3; ++i) TV_CUDA_TRY(cudaStreamWaitEvent(s->side[i], s->start, 0));
   cudaStream_t in = s->side[0], cs = s->side[1], out = s->side[2];
+  // From here on copies to and from the caller's host buffers may be in flight: an error return
+  // first waits for everything already queued on the three streams, so that the caller never
+  // gets control back (and never frees the session) under running work.
+  auto fail = [&](int status) {
+    for (int i = 0; i < 3; ++i) cudaStreamSynchronize(s->side[i]);
+    return status;
+  };
+#define TV_ROUND_TRY(expr)                \
+  do {                                    \
+    cudaError_t e__ = (expr);             \
+    if (e__ != cudaSuccess) {             \
+      tv_set_cuda_error(e__);             \
+      return fail(TV_ERR_CUDA);           \
+    }                                     \
+  } while (0)
   for (int c = 0; c < s->n_chunks; ++c) {
     tv_chunk& ch = s->chunk[c];
     const int32_t* par = s->n_trees == 1 ? parent : parent + (size_t)ch.b0 * d.T;
     const int32_t nt = s->n_trees == 1 ? 1 : ch.nb;
     int st = ch.tree ? tv_tree_rebuild(ch.tree, par) : tv_tree_build(par, nt, d.T, &ch.tree);
-    if (st != TV_OK) return st;
+    if (st != TV_OK) return fail(st);
     auto h2d = [&](void* dst, const void* src, size_t per_req) -> cudaError_t {
       for (int l = 0; l < d.L; ++l) {   // the group's requests are contiguous within a layer
         cudaError_t e = cudaMemcpyAsync((char*)dst + (size_t)l * ch.nb * per_req,
@@ -149,39 +170,40 @@ TV_API int tv_session_round(tv_session* s, const int32_t* parent, const int32_t*
       }
       return cudaSuccess;
     };
-    TV_CUDA_TRY(h2d(ch.S, S_pre, rS));
-    TV_CUDA_TRY(h2d(ch.q, q, rQ));
-    TV_CUDA_TRY(h2d(ch.k, k, rQ));
-    TV_CUDA_TRY(h2d(ch.v, v, rV));
-    TV_CUDA_TRY(h2d(ch.alpha, alpha, rG));
-    if (delta) TV_CUDA_TRY(h2d(ch.beta, beta, rG));
-    TV_CUDA_TRY(cudaMemcpyAsync(ch.accepted, accepted + ch.b0, (size_t)ch.nb * 4, cudaMemcpyHostToDevice, in));
-    TV_CUDA_TRY(cudaEventRecord(s->in_done[c], in));
-    TV_CUDA_TRY(cudaStreamWaitEvent(cs, s->in_done[c], 0));
+    TV_ROUND_TRY(h2d(ch.S, S_pre, rS));
+    TV_ROUND_TRY(h2d(ch.q, q, rQ));
+    TV_ROUND_TRY(h2d(ch.k, k, rQ));
+    TV_ROUND_TRY(h2d(ch.v, v, rV));
+    TV_ROUND_TRY(h2d(ch.alpha, alpha, rG));
+    if (delta) TV_ROUND_TRY(h2d(ch.beta, beta, rG));
+    TV_ROUND_TRY(cudaMemcpyAsync(ch.accepted, accepted + ch.b0, (size_t)ch.nb * 4, cudaMemcpyHostToDevice, in));
+    TV_ROUND_TRY(cudaEventRecord(s->in_done[c], in));
+    TV_ROUND_TRY(cudaStreamWaitEvent(cs, s->in_done[c], 0));
     st = tv_tree_upload(ch.tree, cs);
-    if (st != TV_OK) return st;
+    if (st != TV_OK) return fail(st);
     tv_dims dc = d;
     dc.B = ch.nb;
     st = tv_tree_verify(ch.tree, &dc, ch.S, ch.q, ch.k, ch.v, ch.alpha, ch.beta, ch.O, ch.U, cs);
-    if (st != TV_OK) return st;
+    if (st != TV_OK) return fail(st);
     st = tv_commit_path(ch.tree, &dc, ch.accepted, ch.S, ch.k, ch.v, ch.alpha, ch.beta, ch.U, ch.S, cs);
-    if (st != TV_OK) return st;
-    TV_CUDA_TRY(cudaEventRecord(s->k_done[c], cs));
-    TV_CUDA_TRY(cudaStreamWaitEvent(out, s->k_done[c], 0));
+    if (st != TV_OK) return fail(st);
+    TV_ROUND_TRY(cudaEventRecord(s->k_done[c], cs));
+    TV_ROUND_TRY(cudaStreamWaitEvent(out, s->k_done[c], 0));
     for (int l = 0; l < d.L; ++l) {
-      TV_CUDA_TRY(cudaMemcpyAsync((char*)O + ((size_t)l * d.B + ch.b0) * rO, (char*)ch.O + (size_t)l * ch.nb * rO,
+      TV_ROUND_TRY(cudaMemcpyAsync((char*)O + ((size_t)l * d.B + ch.b0) * rO, (char*)ch.O + (size_t)l * ch.nb * rO,
                                   (size_t)ch.nb * rO, cudaMemcpyDeviceToHost, out));
-      TV_CUDA_TRY(cudaMemcpyAsync((char*)S_new + ((size_t)l * d.B + ch.b0) * rS,
+      TV_ROUND_TRY(cudaMemcpyAsync((char*)S_new + ((size_t)l * d.B + ch.b0) * rS,
                                   (char*)ch.S + (size_t)l * ch.nb * rS, (size_t)ch.nb * rS,
                                   cudaMemcpyDeviceToHost, out));
     }
   }
   for (int i = 0; i < 3; ++i) {
-    TV_CUDA_TRY(cudaEventRecord(s->done[i], s->side[i]));
-    TV_CUDA_TRY(cudaStreamWaitEvent(user, s->done[i], 0));
+    TV_ROUND_TRY(cudaEventRecord(s->done[i], s->side[i]));
+    TV_ROUND_TRY(cudaStreamWaitEvent(user, s->done[i], 0));
   }
-  TV_CUDA_TRY(cudaStreamSynchronize(user));
+  TV_ROUND_TRY(cudaStreamSynchronize(user));
   return TV_OK;
+#undef TV_ROUND_TRY
 }
 
 TV_API int tv_session_free(tv_session* s) {

@@ -31,7 +31,6 @@ struct ConvArgs {
   int32_t capacity;       // packed forest: rows of one output plane
   int32_t n_trees;
   int32_t B, H, T, dk, dv, W, normalize;
-  int32_t use_mma;     // take the mma.sync kernel (explicit request only: it is not the faster one)
   int32_t single;  // one row buffer only (two do not fit): no prefetch of the next item's rows
   float eps;
   const void* x;      // [B][T][C]
@@ -415,296 +414,6 @@ tree_conv_kernel(const ConvArgs a) {
   }
 }
 
-// ---------------------------------------------------------------------------------------------
-// bf16, 128-channel slices, W <= 4: the same operator with the tap sum on the tensor cores.
-// Measured SLOWER than the kernel above (c3: 49.6 vs 49.3 us, c5: 449 vs 224 us per layer) and
-// therefore only run on explicit request (TV_IMPL_TC): it removes the unpack and multiply-add
-// instructions of the taps, but SiLU, normalisation, rounding and staging are what is left and
-// they cost as much; at T > 64 the outputs held in registers across the normalisation barrier
-// (64 per thread) leave room for one CTA per SM only.  Kept as the record of that experiment.
-//
-// The SIMT kernel above spends 4 unpack + 4 FMA instructions per output on the taps.  Here a warp
-// owns 16 channels (two blocks of 8) and walks 16-node row tiles with mma.sync.m16n8k16: the A
-// fragment IS the gather -- each of its 32-bit registers is two adjacent bf16 channels of one
-// tap row, loaded straight from the staged rows by the row's tap offset -- and the B fragment is
-// the filter as a block-diagonal [k = (tap, channel')][channel] matrix (non-zero where channel'
-// = channel), split into three bf16 pieces (hi + mid + lo = w to 2^-27) so that the fp32 filter
-// loses nothing.  Products
-// bf16 x bf16 are exact and accumulate in fp32; the accumulator starts at the bias.  That is
-// 8 shared loads + 6 MMAs per 16 x 8 outputs instead of 1024 unpack/FMA instructions; SiLU, the
-// sum of squares and the scaling stay on the CUDA cores, the rows leave through a staging tile as
-// whole 16-byte vectors.  Staged rows are 272 bytes apart (256 + 16) so that the fragment loads
-// of eight different tap rows fall into different banks.
-constexpr int kMmaRowB = 272;
-
-__device__ __forceinline__ uint32_t lds32(uint32_t addr) {
-  uint32_t r;
-  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(r) : "r"(addr));
-  return r;
-}
-__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-
-// NT = 16-row tiles per item (4: T <= 64, 8: T <= 128)
-template <int W, int NT>
-__global__ void __launch_bounds__(kConvThreads, NT == 4 ? 2 : 1)
-tree_conv_mma_kernel(const ConvArgs a) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  using IO = __nv_bfloat16;
-  constexpr int KS = (W + 1) / 2;   // k-steps of 16 = two taps x 8 channels
-  const int T = a.T, H = a.H, B = a.B;
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t4 = lane & 3;
-  const int C = H * 384;
-  const int Tp = (T + 3) & ~3;
-
-  const uint32_t buf_bytes = (uint32_t)(T + W - 1) * kMmaRowB;
-  const uint32_t xs_u32 = smem_u32(smem_raw);
-  constexpr int Tpad = NT * 16;   // tiles may reach past T: staging and partial sums are sized for them
-  const uint32_t ys_u32 = xs_u32 + 2 * buf_bytes;                       // [Tpad][272] output staging
-  unsigned char* after = smem_raw + 2 * (size_t)buf_bytes + (size_t)Tpad * kMmaRowB;
-  int32_t* par_s = reinterpret_cast<int32_t*>(after);                   // [2][Tp]
-  uint32_t* taps_s = reinterpret_cast<uint32_t*>(par_s + 2 * Tp);       // [2][T][4]
-  float* part_s = reinterpret_cast<float*>(taps_s + 2 * T * 4);         // [Tpad][8]
-  float* inv_s = part_s + Tpad * 8;                                     // [Tpad]
-  const uint32_t par_u32 = smem_u32(par_s), taps_u32 = smem_u32(taps_s);
-
-  const long long n_items = 3LL * H * B;
-  const int first = (int)(n_items * blockIdx.x / gridDim.x);
-  const int last = (int)(n_items * (blockIdx.x + 1) / gridDim.x);
-  if (first >= last) return;
-
-  auto set_slice = [&](ConvItem& it) {
-    it.kind = it.slice / H;
-    it.h = it.slice - it.kind * H;
-    it.d = 128;
-    it.c0 = it.slice * 128;   // q heads | k heads | v heads, 128 channels each
-  };
-  auto set_request = [&](ConvItem& it) {
-    if (a.offsets == nullptr) {
-      it.n = T;
-      it.row0 = it.b * T;
-      it.orow0 = ((size_t)it.b * H + it.h) * T;
-    } else if (it.slice < 3 * H) {
-      it.row0 = a.offsets[it.b];
-      it.n = a.offsets[it.b + 1] - it.row0;
-      it.orow0 = (size_t)it.h * a.capacity + it.row0;
-    }
-  };
-  auto advance = [&](ConvItem& it) {
-    if (++it.b == B) {
-      it.b = 0;
-      ++it.slice;
-      set_slice(it);
-    }
-    set_request(it);
-  };
-  ConvItem cur;
-  cur.slice = first / B;
-  cur.b = first - cur.slice * B;
-  set_slice(cur);
-  set_request(cur);
-  ConvItem nxt = cur;
-  advance(nxt);
-  int b2 = nxt.b + 1 == B ? 0 : nxt.b + 1;
-
-  // 16 vectors of 16 bytes per staged row: thread tid copies vector tid & 15 of rows tid >> 4, +16, ...
-  const int frow = tid >> 4, fcol = (tid & 15) * 8;
-  auto fetch_parents = [&](int b, int slot) {
-    if (tid < T)
-      cp_async4(par_u32 + (uint32_t)(slot * Tp + tid) * 4, a.parent + (size_t)(a.n_trees == 1 ? 0 : b) * T + tid);
-  };
-  auto fetch_rows = [&](const ConvItem& it, int slot) {
-    const IO* xb = reinterpret_cast<const IO*>(a.x) + (size_t)it.row0 * C + it.c0 + fcol;
-    const IO* cb = reinterpret_cast<const IO*>(a.ctx) + (size_t)it.b * (W - 1) * C + it.c0 + fcol;
-    const uint32_t dctx = xs_u32 + (uint32_t)slot * buf_bytes + (uint32_t)fcol * 2u;
-    const uint32_t dx = dctx + (uint32_t)((W - 1) * kMmaRowB);
-    for (int row = frow; row < W - 1; row += 16) cp_async16(dctx + (uint32_t)(row * kMmaRowB), cb + row * C);
-    for (int row = frow; row < it.n; row += 16) cp_async16(dx + (uint32_t)(row * kMmaRowB), xb + row * C);
-  };
-  auto build_taps = [&](const ConvItem& it, int slot) {
-    if (tid < it.n) {
-      const int32_t* par = par_s + slot * Tp;
-      int j = tid, ctx_row = W - 2, row = 0;
-#pragma unroll
-      for (int r = 0; r < 4; ++r) {
-        if (r < W) {
-          if (j >= 0) {
-            row = W - 1 + j;
-            j = par[j];
-          } else {
-            row = ctx_row--;
-          }
-        }   // taps past the filter width repeat the last row (their weights are zero)
-        taps_s[(slot * T + tid) * 4 + r] = (uint32_t)(row * kMmaRowB);
-      }
-    }
-  };
-
-  fetch_parents(cur.b, 0);
-  if (first + 1 < last) fetch_parents(nxt.b, 1);
-  fetch_rows(cur, 0);
-  cp_async_wait_all();
-  __syncthreads();
-  build_taps(cur, 0);
-
-  // filter of this warp's two channel blocks as B fragments (hi and lo), bias as accumulator init
-  uint32_t bhi[2][KS][2], bmid[2][KS][2], blo[2][KS][2];
-  float bias0[2], bias1[2];
-  int loaded_slice = -1;
-  const float eps = a.eps;
-  const bool want_norm = a.normalize != 0;
-
-  for (int item = first; item < last; ++item) {
-    const int s = (item - first) & 1;
-    // rows of this item and parents of the next have landed; the staging tile is free again
-    cp_async_wait_all();
-    __syncthreads();
-    if (item + 1 < last) {
-      fetch_rows(nxt, s ^ 1);
-      if (item + 2 < last) fetch_parents(b2, s);
-      build_taps(nxt, s ^ 1);
-    }
-    const int n = cur.n;
-
-    if (cur.slice != loaded_slice) {
-      loaded_slice = cur.slice;
-#pragma unroll
-      for (int nb = 0; nb < 2; ++nb) {
-        const int cb = cur.c0 + 16 * warp + 8 * nb;
-        bias0[nb] = a.bias ? __ldg(a.bias + cb + 2 * t4) : 0.f;
-        bias1[nb] = a.bias ? __ldg(a.bias + cb + 2 * t4 + 1) : 0.f;
-        // B[k = (tap, c')][col = g] is non-zero only for c' = g: this lane holds k = 2*t4, 2*t4 + 1
-        const bool lo_half = 2 * t4 == g, hi_half = 2 * t4 + 1 == g;
-#pragma unroll
-        for (int ks = 0; ks < KS; ++ks)
-#pragma unroll
-          for (int j = 0; j < 2; ++j) {
-            const int r = 2 * ks + j;   // tap
-            float w = 0.f;
-            if (r < W && (lo_half || hi_half)) w = __ldg(a.weight + (size_t)(cb + g) * W + (W - 1 - r));
-            // w = hi + mid + lo to 2^-27 |w|: three round-to-nearest bf16 pieces, exact remainders
-            const __nv_bfloat16 p0 = __float2bfloat16_rn(w);
-            const float r1 = w - __bfloat162float(p0);
-            const __nv_bfloat16 p1 = __float2bfloat16_rn(r1);
-            const __nv_bfloat16 p2 = __float2bfloat16_rn(r1 - __bfloat162float(p1));
-            const uint32_t h16 = __bfloat16_as_ushort(p0), m16 = __bfloat16_as_ushort(p1), l16 = __bfloat16_as_ushort(p2);
-            bhi[nb][ks][j] = lo_half ? h16 : hi_half ? h16 << 16 : 0u;
-            bmid[nb][ks][j] = lo_half ? m16 : hi_half ? m16 << 16 : 0u;
-            blo[nb][ks][j] = lo_half ? l16 : hi_half ? l16 << 16 : 0u;
-          }
-      }
-    }
-
-    // ---- gate preparation for this (request, head), done with the q slice: the inputs are
-    // requested here and used after the row loop, so nobody waits for them at the next barrier
-    const bool do_gates = cur.kind == 0 && a.gate_a != nullptr && tid < cur.n;
-    float gate_in_a = 0.f, gate_in_b = 0.f, gate_A = 0.f, gate_dt = 0.f;
-    if (do_gates) {
-      const size_t gi = ((size_t)cur.row0 + tid) * H + cur.h;
-      gate_in_a = to_f32(reinterpret_cast<const IO*>(a.gate_a)[gi]);
-      if (a.gate_b != nullptr) gate_in_b = to_f32(reinterpret_cast<const IO*>(a.gate_b)[gi]);
-      gate_A = __ldg(a.A_log + cur.h);
-      gate_dt = __ldg(a.dt_bias + cur.h);
-    }
-
-    // ---- tiles of 16 node rows: taps on the tensor cores, SiLU and squares on the CUDA cores
-    const bool norm = want_norm && cur.kind < 2;
-    const uint32_t xs_item = xs_u32 + (uint32_t)s * buf_bytes + (uint32_t)((16 * warp + 2 * t4) * 2);
-    const uint32_t taps_item = taps_u32 + (uint32_t)(s * T) * 16u;
-    float y[NT][2][4];
-#pragma unroll
-    for (int ti = 0; ti < NT; ++ti) {
-      if (ti * 16 < n) {   // uniform
-        const int r0 = min(ti * 16 + g, n - 1), r1 = min(ti * 16 + g + 8, n - 1);
-        const uint4 t0 = lds16(taps_item + (uint32_t)r0 * 16u), t1 = lds16(taps_item + (uint32_t)r1 * 16u);
-        const uint32_t tap0[4] = {t0.x, t0.y, t0.z, t0.w}, tap1[4] = {t1.x, t1.y, t1.z, t1.w};
-        float ss0 = 0.f, ss1 = 0.f;
-#pragma unroll
-        for (int nb = 0; nb < 2; ++nb) {
-          float c[4] = {bias0[nb], bias1[nb], bias0[nb], bias1[nb]};
-#pragma unroll
-          for (int ks = 0; ks < KS; ++ks) {
-            uint32_t af[4];
-            af[0] = lds32(xs_item + tap0[2 * ks] + 16 * nb);
-            af[1] = lds32(xs_item + tap1[2 * ks] + 16 * nb);
-            af[2] = lds32(xs_item + tap0[2 * ks + 1] + 16 * nb);
-            af[3] = lds32(xs_item + tap1[2 * ks + 1] + 16 * nb);
-            mma_bf16_16816(c, af, bhi[nb][ks][0], bhi[nb][ks][1]);
-            mma_bf16_16816(c, af, bmid[nb][ks][0], bmid[nb][ks][1]);
-            mma_bf16_16816(c, af, blo[nb][ks][0], blo[nb][ks][1]);
-          }
-#pragma unroll
-          for (int e = 0; e < 4; ++e) y[ti][nb][e] = silu(c[e]);
-          ss0 = fmaf(y[ti][nb][0], y[ti][nb][0], fmaf(y[ti][nb][1], y[ti][nb][1], ss0));
-          ss1 = fmaf(y[ti][nb][2], y[ti][nb][2], fmaf(y[ti][nb][3], y[ti][nb][3], ss1));
-        }
-        if (norm) {   // uniform: this warp's 16 channels of rows g and g + 8
-          ss0 += __shfl_xor_sync(0xffffffffu, ss0, 1);
-          ss1 += __shfl_xor_sync(0xffffffffu, ss1, 1);
-          ss0 += __shfl_xor_sync(0xffffffffu, ss0, 2);
-          ss1 += __shfl_xor_sync(0xffffffffu, ss1, 2);
-          if (t4 == 0) {
-            part_s[(ti * 16 + g) * 8 + warp] = ss0;
-            part_s[(ti * 16 + g + 8) * 8 + warp] = ss1;
-          }
-        }
-      }
-    }
-    if (norm) {   // uniform over the CTA
-      __syncthreads();
-      if (tid < n) {
-        const float4 p0 = *reinterpret_cast<const float4*>(part_s + tid * 8);
-        const float4 p1 = *reinterpret_cast<const float4*>(part_s + tid * 8 + 4);
-        inv_s[tid] = rsqrt_fast(((p0.x + p0.y) + (p0.z + p0.w)) + ((p1.x + p1.y) + (p1.z + p1.w)) + eps);
-      }
-      __syncthreads();
-    }
-    // ---- scale, round, stage
-#pragma unroll
-    for (int ti = 0; ti < NT; ++ti) {
-      if (ti * 16 < n) {
-        const int r0 = ti * 16 + g, r1 = r0 + 8;
-        const float s0 = norm ? inv_s[r0] : 1.0f, s1 = norm ? inv_s[r1] : 1.0f;
-#pragma unroll
-        for (int nb = 0; nb < 2; ++nb) {
-          const __nv_bfloat162 v0 = __floats2bfloat162_rn(y[ti][nb][0] * s0, y[ti][nb][1] * s0);
-          const __nv_bfloat162 v1 = __floats2bfloat162_rn(y[ti][nb][2] * s1, y[ti][nb][3] * s1);
-          const uint32_t col = (uint32_t)((16 * warp + 8 * nb + 2 * t4) * 2);
-          asm volatile("st.shared.u32 [%0], %1;" ::"r"(ys_u32 + (uint32_t)r0 * kMmaRowB + col),
-                       "r"(*reinterpret_cast<const uint32_t*>(&v0)) : "memory");
-          asm volatile("st.shared.u32 [%0], %1;" ::"r"(ys_u32 + (uint32_t)r1 * kMmaRowB + col),
-                       "r"(*reinterpret_cast<const uint32_t*>(&v1)) : "memory");
-        }
-      }
-    }
-    __syncthreads();
-    // ---- rows leave as whole 16-byte vectors, coalesced
-    {
-      unsigned char* out = reinterpret_cast<unsigned char*>(cur.kind == 0 ? a.q : cur.kind == 1 ? a.k : a.v) +
-                           cur.orow0 * 256;
-      for (int idx = tid; idx < n * 16; idx += kConvThreads) {
-        const int row = idx >> 4, v = idx & 15;
-        const uint4 x = lds16(ys_u32 + (uint32_t)row * kMmaRowB + (uint32_t)v * 16u);
-        asm volatile("st.global.L1::no_allocate.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(out + (size_t)idx * 16), "r"(x.x),
-                     "r"(x.y), "r"(x.z), "r"(x.w)
-                     : "memory");
-      }
-    }
-    if (do_gates) {
-      const size_t go = cur.orow0 + tid;
-      a.alpha[go] = expf(-expf(gate_A) * softplus(gate_in_a + gate_dt));
-      if (a.gate_b != nullptr) a.beta[go] = 1.0f / (1.0f + expf(-gate_in_b));
-    }
-    cur = nxt;
-    advance(nxt);
-    b2 = b2 + 1 == B ? 0 : b2 + 1;
-  }
-}
-
 // Context rows after the commit: one thread per 16-byte channel vector reads its W-1 source
 // values (accepted node and its ancestors first, then the old context) before it writes any, so
 // ctx_new may be ctx itself.
@@ -747,8 +456,7 @@ int check_conv(const tv_tree* t, const tv_conv_dims* d) {
   if (d->B < 1 || d->H < 1 || d->T < 1 || d->dk < 1 || d->dv < 1 || d->W < 1) return TV_ERR_BAD_ARG;
   if (d->io_dtype != TV_F32 && d->io_dtype != TV_BF16) return TV_ERR_BAD_ARG;
   if (d->impl != TV_IMPL_AUTO && d->impl != TV_IMPL_SIMT && d->impl != TV_IMPL_TC) return TV_ERR_BAD_ARG;
-  if (d->impl == TV_IMPL_TC && !(d->io_dtype == TV_BF16 && d->dk == 128 && d->dv == 128 && d->W <= 4))
-    return TV_ERR_UNSUPPORTED;
+  if (d->impl == TV_IMPL_TC) return TV_ERR_UNSUPPORTED;   // no tensor-core form of this operator
   if (d->T > TV_MAX_NODES || d->dk > kMaxConvDim || d->dv > kMaxConvDim || d->W > TV_CONV_MAX_TAPS)
     return TV_ERR_UNSUPPORTED;
   const int m = d->io_dtype == TV_BF16 ? 7 : 3;
@@ -787,39 +495,8 @@ int launch_conv(const ConvArgs& a_in, cudaStream_t stream) {
   return dmax <= 128 ? go(tree_conv_kernel<IO, W, 1>) : go(tree_conv_kernel<IO, W, 2>);
 }
 
-// bf16 slices of 128 channels with at most 4 taps: the tensor-core kernel
-template <int W>
-int launch_conv_mma(const ConvArgs& a, cudaStream_t stream) {
-  const int NT = a.T <= 64 ? 4 : 8, Tpad = NT * 16, Tp = (a.T + 3) & ~3;
-  const size_t smem = 2 * (size_t)(a.T + W - 1) * kMmaRowB + (size_t)Tpad * kMmaRowB + 2 * (size_t)Tp * 4 +
-                      2 * (size_t)a.T * 16 + (size_t)Tpad * 9 * 4;
-  int dev = 0, sms = 0;
-  TV_CUDA_TRY(cudaGetDevice(&dev));
-  TV_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-  auto go = [&](auto kernel) -> int {
-    if (smem > 48 * 1024)
-      TV_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    int per_sm = 0;
-    TV_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kConvThreads, smem));
-    if (per_sm < 1) return TV_ERR_UNSUPPORTED;
-    const long long items = 3LL * a.H * a.B, slots = (long long)sms * per_sm;
-    kernel<<<(unsigned)(items < slots ? items : slots), kConvThreads, smem, stream>>>(a);
-    TV_CUDA_TRY(cudaGetLastError());
-    return TV_OK;
-  };
-  return NT == 4 ? go(tree_conv_mma_kernel<W, 4>) : go(tree_conv_mma_kernel<W, 8>);
-}
-
 template <typename IO>
 int launch_conv_w(const ConvArgs& a, cudaStream_t s) {
-  if (sizeof(IO) == 2 && a.dk == 128 && a.dv == 128 && a.W <= 4 && a.use_mma) {
-    switch (a.W) {
-      case 1: return launch_conv_mma<1>(a, s);
-      case 2: return launch_conv_mma<2>(a, s);
-      case 3: return launch_conv_mma<3>(a, s);
-      case 4: return launch_conv_mma<4>(a, s);
-    }
-  }
   switch (a.W) {
     case 1: return launch_conv<IO, 1>(a, s);
     case 2: return launch_conv<IO, 2>(a, s);
@@ -886,7 +563,6 @@ TV_API int tv_tree_conv(const tv_tree* tree, const tv_conv_dims* d, const void* 
   ConvArgs a;
   a.parent = tree->d_parent; a.n_trees = tree->n_trees;
   a.offsets = tree->d_offsets; a.capacity = tree->capacity;
-  a.use_mma = d->impl == TV_IMPL_TC;
   a.B = d->B; a.H = d->H; a.T = d->T; a.dk = d->dk; a.dv = d->dv; a.W = d->W;
   a.normalize = d->normalize_qk != 0; a.eps = d->eps;
   a.x = x; a.ctx = ctx; a.weight = weight; a.bias = bias; a.gate_a = gate_a; a.gate_b = gate_b;

@@ -9,7 +9,8 @@ namespace {
 __global__ void __launch_bounds__(TV_MAX_NODES)
 tree_meta_kernel(const int32_t* __restrict__ parent, int32_t n, uint64_t* __restrict__ anc,
                  int32_t* __restrict__ depth, int32_t* __restrict__ parent_dev, int32_t* status,
-                 const int32_t* __restrict__ offsets, int32_t* __restrict__ offsets_dev) {
+                 const int32_t* __restrict__ offsets, int32_t* __restrict__ offsets_dev,
+                 int32_t depth_bound, int32_t generation) {
   __shared__ int32_t par_s[TV_MAX_NODES];
   const int t = blockIdx.x, i = threadIdx.x;
   // a verify kernel launched behind this one may be scheduled now and set itself up; it waits
@@ -32,11 +33,17 @@ tree_meta_kernel(const int32_t* __restrict__ parent, int32_t n, uint64_t* __rest
   if (i >= n) return;
   uint64_t w0 = 0, w1 = 0;
   int d = 0;
-  // the host has validated -1 <= parent[j] < j, so the walk ends within n steps
-  for (int p = par_s[i]; p >= 0 && d < n; p = par_s[p]) {
+  // -1 <= parent[j] < j holds by now, so the walk ends within n steps.  The caller's depth bound
+  // picked the kernels that will read these masks: a node deeper than that keeps its nearest
+  // depth_bound ancestors only (every mask then fits those kernels' tables) and the upload is
+  // marked as failed -- status[1] receives the generation of this upload (all CTAs write the same value),
+  // which needs no clearing and so no ordering between the CTAs of this grid.
+  int p = par_s[i];
+  for (; p >= 0 && d < depth_bound; p = par_s[p]) {
     if (p < 64) w0 |= 1ull << p; else w1 |= 1ull << (p - 64);
     ++d;
   }
+  if (p >= 0) atomicExch(status + 1, generation);
   const size_t o = (size_t)t * n + i;
   anc[2 * o] = w0;
   anc[2 * o + 1] = w1;
@@ -119,9 +126,9 @@ int tv_launch_tree_meta_params(const int32_t* parent_host, int32_t n_trees, int3
 
 int tv_launch_tree_meta(const int32_t* parent_mapped, int32_t n_trees, int32_t n, uint64_t* anc,
                         int32_t* depth, int32_t* parent_dev, int32_t* status, const int32_t* offsets_mapped,
-                        int32_t* offsets_dev, cudaStream_t stream) {
+                        int32_t* offsets_dev, int32_t depth_bound, int32_t generation, cudaStream_t stream) {
   tree_meta_kernel<<<n_trees, TV_MAX_NODES, 0, stream>>>(parent_mapped, n, anc, depth, parent_dev, status,
-                                                        offsets_mapped, offsets_dev);
+                                                        offsets_mapped, offsets_dev, depth_bound, generation);
   TV_CUDA_TRY(cudaGetLastError());
   return TV_OK;
 }

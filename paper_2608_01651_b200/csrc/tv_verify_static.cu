@@ -125,11 +125,6 @@ int tv_tree_verify_static(const int32_t* parent, int32_t n_trees, const tv_dims*
   int32_t* par_dev = reinterpret_cast<int32_t*>(base + kAncBytes + kI32Bytes);
   int32_t* scratch_status = reinterpret_cast<int32_t*>(base + kAncBytes + 2 * kI32Bytes);
 
-  cudaStream_t s = (cudaStream_t)stream;
-  tree_meta_static_kernel<<<n_trees, TV_MAX_NODES, 0, s>>>(parent, d->T, anc, depth, par_dev,
-                                                          scratch_status, status);
-  TV_CUDA_TRY(cudaGetLastError());
-
   VerifyArgs a;
   a.tree.anc = anc;
   a.tree.depth = depth;
@@ -141,8 +136,15 @@ int tv_tree_verify_static(const int32_t* parent, int32_t n_trees, const tv_dims*
   a.L = d->L; a.B = d->B; a.H = d->H; a.T = d->T; a.dk = d->dk; a.dv = d->dv;
   a.rule = d->rule; a.bf16 = d->qkv_dtype == TV_BF16; a.Hk = d->Hk ? d->Hk : d->H;
   a.S_pre = S_pre; a.q = q; a.k = k; a.v = v; a.alpha = alpha; a.beta = beta; a.O = O; a.U = U;
+  // every refusal comes before the first launch: an error return has touched nothing, not even
+  // the scratch that all calls share
   const bool tc_gated = tv_verify_tc_supports(a);
   if (d->impl == TV_IMPL_TC && !tc_gated) return TV_ERR_UNSUPPORTED;
+
+  cudaStream_t s = (cudaStream_t)stream;
+  tree_meta_static_kernel<<<n_trees, TV_MAX_NODES, 0, s>>>(parent, d->T, anc, depth, par_dev,
+                                                          scratch_status, status);
+  TV_CUDA_TRY(cudaGetLastError());
   int st;
   if (tc_gated && d->impl != TV_IMPL_SIMT) st = tv_launch_verify_tc(a, scratch_status, s);
   else st = tv_launch_verify_simt(a, s);

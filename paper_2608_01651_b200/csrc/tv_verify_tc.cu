@@ -79,18 +79,6 @@ __device__ __forceinline__ void store_split8(unsigned char* chi, unsigned char* 
   *reinterpret_cast<uint4*>(clo + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
 }
 
-// Phase timestamps for kernel tuning: compiled out unless TV_TC_PROFILE is defined.
-#ifdef TV_TC_PROFILE
-__device__ long long* g_tc_prof = nullptr;   // [CTA 0 only][item][32] clock64 stamps
-#define TC_STAMP(it, slot)                                                        \
-  do {                                                                            \
-    if (g_tc_prof && blockIdx.x == 0 && (it) < 16 && lane == 0)                   \
-      g_tc_prof[(it) * 32 + (slot)] = clock64();                                  \
-  } while (0)
-#else
-#define TC_STAMP(it, slot) do { } while (0)
-#endif
-
 struct TcParams {
   TreeDev tree;
   int32_t n_items, B, H, T;
@@ -170,7 +158,6 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++it) {
         const uint32_t ph = it & 1;
         if (!mbar_wait(bar(QK_FREE), ph ^ 1, abort_flag)) break;
-        TC_STAMP(it, 0);
         // packed forest: boxes of 64 rows (per-request limit <= 64) or 128 rows at the request's offset
         const uint32_t box_bytes = PACKED ? (T <= 64 ? kTile / 2 : kTile) : kTile;
         int qk = 0, vplane = item, y0 = 0;
@@ -187,14 +174,12 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         tma_load_3d(sbase + kOffK + kTile, &tmK, bar(QK_FULL), 64, y0, qk);
         pend_qk = 1 + (int)ph;
         if (!mbar_wait(bar(S_FREE), ph ^ 1, abort_flag)) break;
-        TC_STAMP(it, 1);
         mbar_expect_tx(bar(S_FULL), 4 * kTile);
 #pragma unroll
         for (int c = 0; c < 4; ++c)
           tma_load_3d(sbase + kOffS + c * kTile, &tmS, bar(S_FULL), 32 * c, 0, item);
         pend_s = 1 + (int)ph;
         if (!mbar_wait(bar(V_FREE), ph ^ 1, abort_flag)) break;
-        TC_STAMP(it, 2);
         mbar_expect_tx(bar(V_FULL), 2 * box_bytes);
         tma_load_3d(sbase + kOffV, &tmV, bar(V_FULL), 0, y0, vplane);
         tma_load_3d(sbase + kOffV + kTile, &tmV, bar(V_FULL), 64, y0, vplane);
@@ -219,9 +204,7 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         const uint32_t ph2 = (it >> 1) & 1;   // the two accumulators alternate
         // scores = Q K^T
         if (!mbar_wait(bar(QK_FULL), ph, abort_flag)) break;
-        TC_STAMP(it, 4);
         if (!mbar_wait(bar(SC_FREE), ph ^ 1, abort_flag)) break;
-        TC_STAMP(it, 5);
         tc_fence_after();
 #pragma unroll
         for (int h = 0; h < 2; ++h)
@@ -233,11 +216,8 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         tc_commit(bar(QK_FREE));
         // acc = (2^e Q) S_pre^T  (A = scaled Q as fp32 in TMEM, B = S_pre chunks)
         if (!mbar_wait(bar(S_FULL), ph, abort_flag)) break;
-        TC_STAMP(it, 6);
         if (!mbar_wait(bar(QF_READY), ph, abort_flag)) break;
-        TC_STAMP(it, 7);
         if (!mbar_wait(bar(acc_free), ph2 ^ 1, abort_flag)) break;
-        TC_STAMP(it, 8);
         tc_fence_after();
 #pragma unroll
         for (int c = 0; c < 4; ++c)
@@ -248,9 +228,7 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         tc_commit(bar(S_FREE));
         // acc += C'_hi V + C'_lo V
         if (!mbar_wait(bar(C_READY), ph, abort_flag)) break;
-        TC_STAMP(it, 9);
         if (!mbar_wait(bar(V_FULL), ph, abort_flag)) break;
-        TC_STAMP(it, 10);
         tc_fence_after();
         for (int jh = 0; jh < n_jh; ++jh)
 #pragma unroll
@@ -263,7 +241,6 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           }
         tc_commit(bar(V_FREE));
         tc_commit(bar(acc_done));
-        TC_STAMP(it, 11);
       }
     }
   } else if (warp == kComputeWarps + 2) {
@@ -418,7 +395,6 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       uint64_t m0 = nm0, m1 = nm1;
       pk = npk;
       const int Tb = PACKED ? pk.n : T;   // real nodes of this item
-      if (warp == 4) TC_STAMP(it, 16);
       // ---- path decay: g_i = sum of log2(alpha) over Anc(i) + {i} ----
       const float la_own = log2f(nal);
       if (hc == 0 && row < Tb) la_s[row] = la_own;
@@ -452,10 +428,8 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       const float a_scale = tiny ? 0.f : exp2f(e_int);
       const float r_scale = exp2f(g - e_int);
       // ---- Q row (bf16, swizzled tile) -> scaled fp32 -> TMEM (A operand of the prefix MMA) ----
-      if (warp == 4) TC_STAMP(it, 17);
       if (!(ok = mbar_wait_warp(bar(QK_FULL), ph, abort_flag))) break;
       if (!(ok = mbar_wait_warp(bar(S_FREE), ph ^ 1, abort_flag))) break;   // prefix MMA of item-1 done with Qf
-      if (warp == 4) TC_STAMP(it, 18);
       tc_fence_after();
       if (warp_live) {
         const unsigned char* qrow = sm + kOffQ + hc * kTile + row * 128;
@@ -483,15 +457,12 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         mbar_arrive(bar(QK_FREE));
       }
       // ---- scores -> masked, decayed, split C' ----
-      if (warp == 4) TC_STAMP(it, 19);
       if (!(ok = mbar_wait_warp(bar(SC_DONE), ph, abort_flag))) break;
-      if (warp == 4) TC_STAMP(it, 20);
       if (!(ok = mbar_wait_warp(bar(SETUP), 1, abort_flag))) break;
       // ---- output rows of the previous item: its accumulator is complete once its readout MMA
       // is, and the C' tiles it frees double as the staging area of the output store ----
       if (it > 0 && !(ok = final_epilogue(it - 1, item_prev, r_prev, (it - 1) & 1, pk_prev))) break;
       tc_fence_after();
-      if (warp == 4) TC_STAMP(it, 21);
       if (warp_live) {
         bool fast = true;
 #pragma unroll
@@ -554,7 +525,6 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         mbar_arrive(bar(C_READY));
         mbar_arrive(bar(SC_FREE));
       }
-      if (warp == 4) TC_STAMP(it, 22);
       item_prev = item;
       r_prev = r_scale;
       pk_prev = pk;
@@ -613,12 +583,6 @@ __global__ void widen_bf16_rows_kernel(const __nv_bfloat16* __restrict__ v, floa
 }
 
 }  // namespace
-
-#ifdef TV_TC_PROFILE
-extern "C" __attribute__((visibility("default"))) int tv_debug_set_tc_profile(long long* dev_buf) {
-  return cudaMemcpyToSymbol(g_tc_prof, &dev_buf, sizeof(dev_buf)) == cudaSuccess ? 0 : -4;
-}
-#endif
 
 // Self-test of the bounded wait every tensor-core kernel relies on: one CTA waits, with a short
 // limit, on a barrier that nothing ever arrives at, then reports and returns like the kernels do.

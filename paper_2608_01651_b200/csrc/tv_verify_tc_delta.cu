@@ -73,18 +73,6 @@ enum Bar {
 
 constexpr uint32_t kColSc = 0, kColQf = 128, kColAcc = 256;
 
-// Phase timestamps for kernel tuning: compiled out unless TV_TC_PROFILE is defined.
-#ifdef TV_TC_PROFILE
-__device__ long long* g_tcd_prof = nullptr;
-#define TCD_STAMP(it, slot)                                                       \
-  do {                                                                            \
-    if (g_tcd_prof && blockIdx.x == 0 && (it) < 16 && lane == 0)                  \
-      g_tcd_prof[(it) * 32 + (slot)] = clock64();                                 \
-  } while (0)
-#else
-#define TCD_STAMP(it, slot) do { } while (0)
-#endif
-
 struct DeltaParams {
   TreeDev tree;
   int32_t n_items, B, H, T;
@@ -230,7 +218,6 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       auto gram = [&](uint32_t j) -> bool {
         const uint32_t qk_base = (j & 1) ? kOffQK1 : kOffQK;
         if (!mbar_wait(bar((j & 1) ? QK_FULL1 : QK_FULL), (j >> 1) & 1, abort_flag)) return false;
-        TCD_STAMP(j, 4);
         if (!mbar_wait(bar(G_FREE), (j & 1) ^ 1, abort_flag)) return false;   // score columns read by E1 of j-1
         tc_fence_after();
 #pragma unroll
@@ -249,7 +236,6 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         if (it + 1 < n_local && !gram(it + 1)) break;
         // Qf += -(W D_P) K  (rows 64..127: -(A D_P) K); the compute warps initialised Qf with D_P Q
         if (!mbar_wait(bar(W_READY), ph, abort_flag)) break;
-        TCD_STAMP(it, 5);
         tc_fence_after();
 #pragma unroll
         for (int part = 0; part < 2; ++part)      // hi, lo
@@ -262,9 +248,7 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         // acc = Qf S_pre^T: Qf must be complete in TMEM before it is read as the A operand
         if (!mbar_wait(bar(D1_DONE), ph, abort_flag)) break;
         if (!mbar_wait(bar(S_FULL), ph, abort_flag)) break;
-        TCD_STAMP(it, 6);
         if (!mbar_wait(bar(ACC_FREE), ph ^ 1, abort_flag)) break;
-        TCD_STAMP(it, 7);
         tc_fence_after();
 #pragma unroll
         for (int c = 0; c < 4; ++c)
@@ -275,7 +259,6 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         tc_commit(bar(S_FREE));
         // acc += [W ; A] V
         if (!mbar_wait(bar(V_FULL), ph, abort_flag)) break;
-        TCD_STAMP(it, 8);
         tc_fence_after();
 #pragma unroll
         for (int s = 0; s < 4; ++s) {
@@ -285,7 +268,6 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         }
         tc_commit(bar(V_FREE));
         tc_commit(bar(ACC_DONE));
-        TCD_STAMP(it, 9);
       }
     }
   } else if (warp == kComputeWarps + 2) {
@@ -458,7 +440,6 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       // the per-node tables that this item is about to overwrite; with the Gram product issued one
       // item ahead, nothing else would hold a fast warp back).
       if (it > 0 && !(ok = mbar_wait_warp(bar(W_READY), (it - 1) & 1, abort_flag))) break;
-      if (warp == 4) TCD_STAMP(it, 16);
       // ---- per-node tables of this item (written by the metadata warp) ----
       if (!(ok = mbar_wait_warp(bar(ph ? META_FULL1 : META_FULL), (it >> 1) & 1, abort_flag))) break;
       const uint64_t m = node < Tb ? mask_s[ph * kRows + node] : 0ull;   // strict ancestors
@@ -469,7 +450,6 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
 
       // ---- E1: raw path-sparse rows: part 0 <- Q K^T (path incl. the node), part 1 <- K K^T ----
       if (!(ok = mbar_wait_warp(bar(G_DONE), ph, abort_flag))) break;
-      if (warp == 4) TCD_STAMP(it, 18);
       tc_fence_after();
       // A node's ancestors have smaller numbers than the node: the rows of nodes 0..31 select
       // nothing among the columns 32..63, and the warp that would scan them skips the chunk.
@@ -496,9 +476,7 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         mbar_arrive(bar(G_FREE));
         mbar_arrive(bar(E1_SYNC));
       }
-      if (warp == 4) TCD_STAMP(it, 19);
       if (!(ok = mbar_wait_warp(bar(E1_SYNC), ph, abort_flag))) break;
-      if (warp == 4) TCD_STAMP(it, 20);
 
       // ---- E2: decay factors, one back-substitution per row, operand tiles ----
       constexpr int NS = DMAX + 1;                            // path slots in use
@@ -519,12 +497,10 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           pre[s2] = Pi;              // P at path node s2
         }
       }
-      if (warp == 4) TCD_STAMP(it, 22);
       // ---- output of the previous item: its MMAs ran under E1 and the gather above, so the
       // accumulator is complete by now; the TMA stores that take the staged chunks away read them
       // under the back-substitution and the Qf initialisation below ----
       if (it > 0 && !(ok = final_epilogue(it - 1, pk_prev))) break;
-      if (warp == 4) TCD_STAMP(it, 17);
       if (live_i) {
         // C_{i,p_s} = (q_i . k_{p_s}) P_i / P_{p_s}: the ratio is the product of alpha over the
         // slots after s, built up from the node's own slot backwards
@@ -580,11 +556,9 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         }
         tmem_wait_st();
       }
-      if (warp == 4) TCD_STAMP(it, 25);
       // The tiles alias the staged output chunks of the previous item: its stores must have read
       // them (they did so under the Qf initialisation above).
       if (it > 0 && !(ok = mbar_wait_warp(bar(OST_FREE), (it - 1) & 1, abort_flag))) break;
-      if (warp == 4) TCD_STAMP(it, 23);
       if constexpr (PACKED) {
         // A box that reaches past the last node of the forest brings rows nobody wrote.  They only
         // ever meet zero coefficients, but 0 x garbage need not be 0: zero them.  The Gram MMA has
@@ -626,7 +600,6 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           }
         }
       }
-      if (warp == 4) TCD_STAMP(it, 24);
       tc_fence_before();
       fence_async_smem();
       __syncwarp();
@@ -634,7 +607,6 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         mbar_arrive(bar(W_READY));
         mbar_arrive(bar(ph ? META_FREE1 : META_FREE));   // this item's tables may be overwritten
       }
-      if (warp == 4) TCD_STAMP(it, 21);
       pk_prev = pk;
     }
     if (ok && it > 0) final_epilogue(it - 1, pk_prev);
@@ -651,12 +623,6 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
 }
 
 }  // namespace
-
-#ifdef TV_TC_PROFILE
-extern "C" __attribute__((visibility("default"))) int tv_debug_set_tcd_profile(long long* dev_buf) {
-  return cudaMemcpyToSymbol(g_tcd_prof, &dev_buf, sizeof(dev_buf)) == cudaSuccess ? 0 : -4;
-}
-#endif
 
 bool tv_verify_tc_delta_supports(const VerifyArgs& a) {
   return a.bf16 && a.dk == 128 && a.dv == 128 && a.rule == TV_GATED_DELTA && a.T <= kRows &&

@@ -64,18 +64,6 @@ enum Bar {
 
 constexpr uint32_t kColSc0 = 0, kColQf = 128, kColAcc = 256, kColSc1 = 384;
 
-// Phase timestamps for kernel tuning: compiled out unless TV_TC_PROFILE is defined.
-#ifdef TV_TC_PROFILE
-__device__ long long* g_d128_prof = nullptr;
-#define D128_STAMP(blk, slot)                                                      \
-  do {                                                                            \
-    if (g_d128_prof && blockIdx.x == 0 && (blk) < 16 && warp == 4 && lane == 0)   \
-      g_d128_prof[(blk) * 32 + (slot)] = clock64();                               \
-  } while (0)
-#else
-#define D128_STAMP(blk, slot) do { } while (0)
-#endif
-
 struct Delta128Params {
   TreeDev tree;
   int32_t n_items, B, H, T;
@@ -461,7 +449,6 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
           Tn = item_s[ph * 4];
           row0 = (size_t)(uint32_t)item_s[ph * 4 + 1] | (size_t)(uint32_t)item_s[ph * 4 + 2] << 32;
         }
-        D128_STAMP(2 * it + b, 0);
         const int nd = kBlk * b + rn;                              // tree node of this row
         const bool rows_live = kBlk * b + (quad & 1) * 32 < Tn;    // warp-uniform: some row of the warp is a node
         const bool live_i = nd < Tn && (part == 0 || want_U);      // this row carries a problem
@@ -472,7 +459,6 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
 
         // ---- E1: raw path-sparse rows: part 0 <- Q K^T (path incl. the node), part 1 <- K K^T ----
         if (!(ok = mbar_wait_warp(bar(b ? GD1 : GD0), ph, abort_flag))) break;
-        D128_STAMP(2 * it + b, 1);
         tc_fence_after();
         if (rows_live) {
           uint64_t s0 = m0, s1 = m1;
@@ -505,9 +491,7 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
           mbar_arrive(bar(b ? GF1 : GF0));
           mbar_arrive(bar(E1_SYNC));
         }
-        D128_STAMP(2 * it + b, 2);
         if (!(ok = mbar_wait_warp(bar(E1_SYNC), (uint32_t)b, abort_flag))) break;
-        D128_STAMP(2 * it + b, 3);
 
         if constexpr (PACKED) {
           // A box that reaches past the last node of the forest brings rows nobody wrote.  They only
@@ -550,12 +534,10 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
           }
         }
         // ---- output of the block before: its MMAs ran under E1 and the gather above ----
-        D128_STAMP(2 * it + b, 4);
         if (pn >= 0) {
           if (!(ok = read_out(prow0, pn, pb))) break;
           ++n_read;
         }
-        D128_STAMP(2 * it + b, 5);
         if (live_i) {
           // C_{i,p_s} = (q_i . k_{p_s}) P_i / P_{p_s}: the ratio is the product of alpha over the
           // slots after s, built up from the node's own slot backwards
@@ -584,7 +566,6 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
         }
         // ---- Qf starts as D_P Q (rows of the O problem; P_i in full fp32) or 0 (rows of the U
         // problem); the state MMA of the block before must have read the old Qf first ----
-        D128_STAMP(2 * it + b, 6);
         if (!(ok = mbar_wait_warp(bar(QF_FREE), (uint32_t)b ^ 1, abort_flag))) break;
         // the Q rows are read by these threads: observe the load's barrier themselves
         if (!(ok = mbar_wait_warp(bar(QK_FULL), ph, abort_flag))) break;
@@ -615,7 +596,6 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
 
         // ---- coefficient tiles, one column half of one matrix at a time: thread hc = 0 writes the
         // hi tile, hc = 1 the lo tile of its row ----
-        D128_STAMP(2 * it + b, 7);
         // the staged half of the block read out above has left the coefficient tiles
         if (!PACKED && n_read > 0 && !(ok = mbar_wait_warp(bar(OST_FREE), (n_read - 1) & 1, abort_flag))) break;
         const int n_builds = b ? 4 : 2;
@@ -625,7 +605,6 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
           const int h = b ? (q & 1) : 0;                  // column half: ancestors 64 h .. 64 h + 63
           // the MMAs that read the tile of the build before have completed
           if (!(ok = mbar_wait_warp(bar(TILE_FREE), (j & 1) ^ 1, abort_flag))) break;
-          D128_STAMP(2 * it + b, 8 + 2 * q);
           if (live_i) {
             unsigned char* trow = sm + kOffCoef + hc * kTile + row * 128;
             const uint4 z = make_uint4(0u, 0u, 0u, 0u);
@@ -647,7 +626,6 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
           fence_async_smem();
           __syncwarp();
           if (lane == 0) mbar_arrive(bar(TILE_READY));
-          D128_STAMP(2 * it + b, 9 + 2 * q);
         }
         if (!ok) break;
         if (b == 1) {
@@ -673,12 +651,6 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
 }
 
 }  // namespace
-
-#ifdef TV_TC_PROFILE
-extern "C" __attribute__((visibility("default"))) int tv_debug_set_d128_profile(long long* dev_buf) {
-  return cudaMemcpyToSymbol(g_d128_prof, &dev_buf, sizeof(dev_buf)) == cudaSuccess ? 0 : -4;
-}
-#endif
 
 bool tv_verify_tc_delta128_supports(const VerifyArgs& a) {
   return a.bf16 && a.dk == 128 && a.dv == 128 && a.rule == TV_GATED_DELTA && a.T > kBlk && a.T <= kNodes &&

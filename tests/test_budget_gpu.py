@@ -185,3 +185,40 @@ def test_round_replays_from_a_cuda_graph_with_a_new_topology():
     assert torch.equal(O_graph[:, :n], O[:, :n]) and torch.equal(S_graph, S_new)
     ref = bo.select(par, p, budget)
     assert np.array_equal(off_graph.cpu().numpy(), ref["offsets"])
+
+
+def test_depth_bound_is_checked_on_the_device():
+    """tv_forest_upload_device is told a bound on the tree depth (it picks the kernels).  A forest
+    that is deeper is reported by tv_tree_device_status and its masks are cut to the bound, so the
+    delta-rule tensor-core kernel that the bound selected stays inside its tables; the next upload
+    with an honest bound clears the report."""
+    B, n = 3, 40
+    chains = np.tile(np.arange(-1, n - 1, dtype=np.int32), (B, 1))          # depth n - 1 = 39
+    offsets = torch.arange(0, (B + 1) * n, n, dtype=torch.int32, device=DEV)
+    forest = tv.forest_build([np.array([-1], dtype=np.int32)] * B, n_max=n, capacity=B * n)
+    par_d = torch.from_numpy(chains).to(DEV)
+    forest.upload_device(par_d, offsets, max_depth_bound=8)
+    anc, depth = forest.meta_device()
+    assert int(depth.max()) == 8
+    assert all(bin(int(anc[b, i, 0])).count("1") == min(i, 8) for b in range(B) for i in range(n))
+    with pytest.raises(tv.TreeVerifyError) as e:
+        forest.device_status()
+    assert e.value.status == -3
+    # the kernels chosen for depth <= 8 run on those masks without leaving their tables
+    wl = inputs.workload("c4", B=B, H=2, T=n, seed=3)
+    t = {k: (None if v is None else v.to(DEV)) for k, v in inputs.make_tensors(wl).items()}
+    plane = lambda x: x.transpose(0, 1).reshape(x.shape[1], B * n, *x.shape[3:]).contiguous()
+    O = torch.empty(2, B * n, 128, device=DEV)
+    tv.tree_verify(forest, t["S_pre"], plane(t["q"]), plane(t["k"]), plane(t["v"]), plane(t["alpha"]),
+                   plane(t["beta"]), rule=inputs.DELTA, O=O, impl=tv.IMPL_TC)
+    torch.cuda.synchronize()
+    assert torch.isfinite(O).all()
+    # an honest bound: same handle, report gone, full masks
+    forest.upload_device(par_d, offsets, max_depth_bound=n - 1)
+    forest.device_status()
+    anc, depth = forest.meta_device()
+    assert int(depth.max()) == n - 1
+    # and a host-side rebuild after a failed device upload starts clean as well
+    forest.upload_device(par_d, offsets, max_depth_bound=2)
+    forest.rebuild_forest([c for c in chains]).upload()
+    forest.device_status()

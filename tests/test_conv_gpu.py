@@ -97,15 +97,16 @@ def test_workloads(name, impl):
 
 @pytest.mark.parametrize("T", [1, 7, 16, 17, 63, 64, 65, 100, 128])
 @pytest.mark.parametrize("W", [1, 2, 3, 4])
-def test_tensor_core_kernel_shapes(T, W):
-    """bf16, 128-channel heads, W <= 4: the mma kernel, forced (IMPL_TC), over tile-edge sizes."""
+def test_bf16_head128_tile_edges(T, W):
+    """bf16, 128-channel heads, W <= 4 (the shape of the workloads) over tile-edge node counts."""
     wl = dataclasses.replace(inputs.workload("c2"), B=3, H=2, T=T, seed=900 + T + W)
     parents, _ = inputs.make_trees(wl)
-    run_case(wl, parents, W=W, normalize=bool(T & 1), gate_b=bool(W & 1), bias=W != 3, impl=tv.IMPL_TC)
+    run_case(wl, parents, W=W, normalize=bool(T & 1), gate_b=bool(W & 1), bias=W != 3)
 
 
-def test_tensor_core_kernel_declines_other_shapes():
-    wl = dataclasses.replace(inputs.workload("c2"), B=1, H=2, T=16, dk=64, dv=128)
+def test_no_tensor_core_form():
+    """IMPL_TC is refused: the operator has no tensor-core kernel and never falls back silently."""
+    wl = dataclasses.replace(inputs.workload("c2"), B=1, H=2, T=16)
     parents, _ = inputs.make_trees(wl)
     with pytest.raises(tv.TreeVerifyError) as e:
         run_case(wl, parents, W=4, impl=tv.IMPL_TC)

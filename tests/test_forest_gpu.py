@@ -255,3 +255,35 @@ def test_metadata_upload_paths_agree_with_the_host(n_trees, n):
         anc, depth, _ = tree.meta()
         danc, ddepth = tree.meta_device()
         assert np.array_equal(anc, danc) and np.array_equal(depth, ddepth)
+
+
+def test_commit_right_behind_a_forest_upload():
+    """tv_commit_path directly behind tv_forest_rebuild + tv_tree_upload on the same stream, with
+    no verify call in between: the commit grid may be scheduled while the metadata kernel still
+    runs, and must not read the request offsets (or anything else that kernel writes) before that
+    kernel is complete.  The handle first holds another forest, so stale offsets would put every
+    request's rows in the wrong place."""
+    B, H, n_max = 48, 8, 64
+    wl = inputs.workload("c2", B=B, H=H, T=n_max, seed=77)
+    first, _ = make_forest(B, n_max, seed=5)
+    first = first[::-1]                                   # other sizes per request than `parents`
+    parents, accepted = make_forest(B, n_max, seed=6)
+    accepted = np.array([len(p) - 1 for p in parents], dtype=np.int32)   # last node: needs the right row count
+    cap = B * n_max
+    P, off = packed_tensors(wl, parents, cap, H)
+    g = {n: (None if t is None else t.to(DEV)) for n, t in P.items()}
+    acc = torch.from_numpy(accepted).to(DEV)
+    forest = tv.forest_build(first, n_max=n_max, capacity=cap).upload()
+    torch.cuda.synchronize()
+    for _ in range(3):
+        forest.rebuild_forest(first).upload()
+        torch.cuda.synchronize()
+        Sn = torch.empty_like(g["S_pre"])
+        forest.rebuild_forest(parents).upload()
+        tv.commit_path(forest, acc, g["S_pre"], g["k"], g["v"], g["alpha"], None, S_new=Sn)
+        torch.cuda.synchronize()
+        Snn = Sn.cpu().double().numpy()
+        for b in range(0, B, 5):
+            for h in (0, H - 1):
+                Sr = oracle_request(wl, P, off, parents, accepted, 0, b, h, H)[2]
+                assert rel_fro(Snn[0, b, h], Sr) <= 2e-3, (b, h)

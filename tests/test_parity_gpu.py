@@ -25,12 +25,12 @@ def _tc_ok(wl, parents=None):
     if wl.rule == inputs.GATED:
         return True
     depth = max(int(inputs.node_depths(p).max()) for p in parents) if parents is not None else 0
-    return wl.T <= 64 and depth <= 15
+    return depth <= 15
 
 
 def _skip_unless_supported(wl, impl, parents=None):
     if impl == tv.IMPL_TC and not _tc_ok(wl, parents):
-        pytest.skip("tensor-core kernels cover bf16, dk = dv = 128 (delta rule: T <= 64, depth <= 15)")
+        pytest.skip("tensor-core kernels cover bf16, dk = dv = 128 (delta rule: tree depth <= 15)")
 
 
 def _run(wl, parents, accepted, tens, tol, items=None, **kw):

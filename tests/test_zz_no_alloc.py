@@ -3,8 +3,8 @@
 Collected last on purpose (file name): it is an addition beside the paper's path, and a run
 that stops at the first failure should already have run every other test.  The new entry is
 called through the C ABI and compared with the regular entry point (tv_tree_build +
-tv_tree_upload + tv_tree_verify) on the same inputs, twice in a row, because the fixed
-device array it works in keeps the previous call's contents.
+tv_tree_upload + tv_tree_verify) and with the fp64 oracle on the same inputs, twice in a row,
+because the fixed device array it works in keeps the previous call's contents.
 """
 import numpy as np
 import pytest
@@ -12,6 +12,7 @@ import torch
 
 import paper_2608_01651_b200 as tv
 from paper_2608_01651_b200 import inputs
+from tests import parity_util as pu
 
 pytestmark = pytest.mark.gpu
 
@@ -50,7 +51,8 @@ def test_static_matches_regular_entry_point_twice(name, B, H):
     for round_ in range(2):
         wl_r = inputs.workload(name, B=B, H=H, seed=wl.seed + 50 * round_)
         parents, _ = inputs.make_trees(wl_r)
-        t = dev(inputs.make_tensors(wl_r))
+        t_cpu = inputs.make_tensors(wl_r)
+        t = dev(t_cpu)
         want_U = wl.rule == inputs.DELTA
         O_ref, U_ref = _regular(wl_r, parents, t, want_U)
         O, U = _static(wl_r, torch.from_numpy(parents).cuda(), t, want_U)
@@ -62,6 +64,14 @@ def test_static_matches_regular_entry_point_twice(name, B, H):
             assert _close(U, U_ref, wl.tol)
         if wl.rule == inputs.GATED:
             assert torch.equal(O, O_ref)
+        # and directly against the oracle, on every (request, head)
+        ver, _ = pu.oracle_round(wl_r, parents, np.full(B, -1), t_cpu)
+        On = O.cpu().double().numpy()
+        Un = None if U is None else U.cpu().double().numpy()
+        for (b, h), (Or, Ur) in ver.items():
+            assert pu.rel_l2_rows(On[b, h], Or) <= wl.tol
+            if want_U:
+                assert pu.rel_l2_rows(Un[b, h], Ur) <= wl.tol
 
 
 def test_static_shared_tree_capacity_and_bad_parents():
