@@ -466,6 +466,206 @@ def run_packed(args, wl, local_rank):
     print(json.dumps(line, default=_jsonable), flush=True)
 
 
+class StepRig:
+    """One workload resident on the device: rotating input sets (so that consecutive steps never
+    find their inputs in L2: every set is larger than 4x L2, or there are several), the calls
+    marshalled once per set, and the step itself."""
+
+    def __init__(self, tv, wl, dev, stream, impl, n_sets=0):
+        self.tv, self.wl, self.stream = tv, wl, stream
+        self.parents, self.accepted = inputs.make_trees(wl)
+        self.acc_len = accepted_lengths(self.parents, self.accepted)
+        delta = wl.rule == inputs.DELTA
+        eb = 2 if wl.qkv_dtype == inputs.BF16 else 4
+        self.set_bytes = wl.L * wl.B * wl.H * (4 * wl.dk * wl.dv + eb * wl.T * (2 * wl.dk + wl.dv)
+                                               + 4 * wl.T * wl.dv)
+        if not n_sets:
+            n_sets = 1 if self.set_bytes > 4 * L2_BYTES else max(2, min(8, int(np.ceil(4 * L2_BYTES / self.set_bytes))))
+        self.n_sets = n_sets
+        self.sets = []
+        for s in range(n_sets):
+            layers = [inputs.make_tensors(wl, layer=s * wl.L + l, device=dev) for l in range(wl.L)]
+            st = {k: (None if layers[0][k] is None else torch.stack([x[k] for x in layers]))
+                  for k in layers[0]}
+            del layers
+            st["O"] = torch.empty(wl.L, wl.B, wl.H, wl.T, wl.dv, device=dev, dtype=torch.float32)
+            st["U"] = torch.empty_like(st["O"]) if delta else None
+            self.sets.append(st)
+        self.acc_dev = torch.from_numpy(self.accepted).to(dev)
+        self.tree = tv.tree_build(self.parents)
+        self.calls = []
+        for st in self.sets:
+            ver = [tv.prepare_tree_verify(self.tree, st["S_pre"][l], st["q"][l], st["k"][l], st["v"][l],
+                                          st["alpha"][l], None if st["beta"] is None else st["beta"][l],
+                                          rule=wl.rule, O=st["O"][l],
+                                          U=None if st["U"] is None else st["U"][l], impl=impl, stream=stream)
+                   for l in range(wl.L)]
+            com = tv.prepare_commit_path(self.tree, self.acc_dev, st["S_pre"], st["k"], st["v"], st["alpha"],
+                                         st["beta"], rule=wl.rule, U=st["U"], stream=stream)
+            self.calls.append((ver, com))
+        self.refresh = self.tree.prepare_refresh(np.ascontiguousarray(self.parents, dtype=np.int32), stream)
+        self.vbytes = verify_bytes_per_layer(wl, with_U=delta)
+        self.cbytes = commit_bytes_per_layer(wl, self.acc_len, with_U=delta) * wl.L
+
+    # the whole hot path: tree_build + upload, L verify launches, one commit over all layers
+    def step(self, i):
+        ver, com = self.calls[i % self.n_sets]
+        self.refresh()
+        for call in ver:
+            call()
+        com()
+
+    def step_without_commit(self, i):
+        self.refresh()
+        for call in self.calls[i % self.n_sets][0]:
+            call()
+
+    def verify_only(self, i):          # one launch per call, layers and sets in rotation
+        ver = self.calls[i % self.n_sets][0]
+        ver[(i // self.n_sets) % len(ver)]()
+
+    def commit_only(self, i):
+        self.calls[i % self.n_sets][1]()
+
+
+def _ev():
+    return torch.cuda.Event(enable_timing=True)
+
+
+def time_loop(stream, n, body, warm=3):
+    """Average device time of body(i) over n calls: two events, nothing recorded in between."""
+    for i in range(warm):
+        body(i)
+    torch.cuda.synchronize()
+    e0, e1 = _ev(), _ev()
+    e0.record(stream)
+    for i in range(n):
+        body(warm + i)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / n
+
+
+def kernel_split(rig, step_ms, n, peak):
+    """Per-kernel times WITHOUT events between launches (an event between two launches costs a
+    bubble and undoes the dependent launches): the loop 'metadata + verify' is timed next to the
+    full step, the commit's share is the difference, so verify + commit = step by construction.
+    The back-to-back loops give each kernel alone (launch gaps included, no dependency on the
+    metadata kernel)."""
+    wl, stream = rig.wl, rig.stream
+    upto_verify = time_loop(stream, n, rig.step_without_commit)
+    v_b2b = time_loop(stream, max(n, 16) * min(wl.L, 4), rig.verify_only, warm=max(3, rig.n_sets))
+    c_b2b = time_loop(stream, max(n, 16), rig.commit_only, warm=max(3, rig.n_sets))
+    v_ms = upto_verify / wl.L
+    c_ms = max(step_ms - upto_verify, 0.0)
+    gbs = lambda nbytes, ms: nbytes / (ms * 1e-3) / 1e9 if ms > 0 else 0.0
+    verify = {"ms_per_layer": v_ms,
+              "what": "tree_build + upload + L verify launches, over L; no events between launches",
+              "nodes_per_s_per_layer": wl.B * wl.T / (v_ms * 1e-3),
+              "bytes_per_layer": rig.vbytes, "algorithmic_GBps": gbs(rig.vbytes, v_ms),
+              "frac_of_measured_copy": gbs(rig.vbytes, v_ms) / peak,
+              "frac_of_nominal_8TBps": gbs(rig.vbytes, v_ms) / NOMINAL_HBM_GBS,
+              "back_to_back_ms": v_b2b,
+              "back_to_back_frac_of_measured_copy": gbs(rig.vbytes, v_b2b) / peak,
+              "back_to_back_frac_of_nominal_8TBps": gbs(rig.vbytes, v_b2b) / NOMINAL_HBM_GBS}
+    commit = {"ms": c_ms, "what": "step minus (tree_build + upload + L verify launches)",
+              "bytes": rig.cbytes, "algorithmic_GBps": gbs(rig.cbytes, c_ms),
+              "frac_of_measured_copy": gbs(rig.cbytes, c_ms) / peak,
+              "frac_of_nominal_8TBps": gbs(rig.cbytes, c_ms) / NOMINAL_HBM_GBS,
+              "back_to_back_ms": c_b2b,
+              "back_to_back_frac_of_measured_copy": gbs(rig.cbytes, c_b2b) / peak,
+              "back_to_back_frac_of_nominal_8TBps": gbs(rig.cbytes, c_b2b) / NOMINAL_HBM_GBS}
+    return verify, commit
+
+
+def parity_check(rig, layers, n_items, seed=11):
+    """One more round of the step exactly as timed (same calls, same launch configuration, commit
+    in place), with O, U and S_new of sampled (layer, request, head) items compared with the fp64
+    oracle run on the values that sit in device memory.  Outside every timed region."""
+    from oracle import tree_oracle as orc
+    wl = rig.wl
+    st = rig.sets[0]
+    rng = np.random.default_rng(seed)
+    items = []
+    for l in layers:
+        picks = {(0, 0), (wl.B - 1, wl.H - 1)}
+        while len(picks) < min(n_items, wl.B * wl.H):
+            picks.add((int(rng.integers(wl.B)), int(rng.integers(wl.H))))
+        items += [(l, b, h) for (b, h) in sorted(picks)]
+    S0 = {it: st["S_pre"][it].clone() for it in items}          # the state before this round
+    rig.step(0)
+    torch.cuda.synchronize()
+    rig.tree.device_status()
+    f = inputs.to_f64
+    eO = eU = eS = 0.0
+    for (l, b, h) in items:
+        par = rig.parents[b if rig.parents.shape[0] > 1 else 0][None]
+        one = lambda t: None if t is None else f(t[l, b, h].cpu())[None, None]
+        S_hat, q, k, v, al, be = (f(S0[(l, b, h)].cpu())[None, None], one(st["q"]), one(st["k"]), one(st["v"]),
+                                  one(st["alpha"]), one(st["beta"]))
+        Or, Ur = orc.verify_batch(S_hat, q, k, v, al, be, par, wl.rule_name)[(0, 0)]
+        Sr = orc.commit_batch(S_hat, k, v, al, be, par, [int(rig.accepted[b])], wl.rule_name)[(0, 0)]
+        rel = lambda x, r: float((np.linalg.norm(x - r, axis=-1) / np.maximum(np.linalg.norm(r, axis=-1), 1e-300)).max())
+        eO = max(eO, rel(f(st["O"][l, b, h].cpu()), Or))
+        if st["U"] is not None:
+            eU = max(eU, rel(f(st["U"][l, b, h].cpu()), Ur))
+        Sn = f(st["S_pre"][l, b, h].cpu())
+        eS = max(eS, float(np.linalg.norm(Sn - Sr) / max(np.linalg.norm(Sr), 1e-300)))
+    return {"max_rel_l2_O": eO, "max_rel_l2_U": eU if st["U"] is not None else None, "max_rel_fro_S": eS,
+            "tol": wl.tol, "ok": bool(max(eO, eU, eS) <= wl.tol), "layers": list(layers), "items": len(items),
+            "against": "fp64 oracle (per-node path walk) on the device-resident values, after the timed region"}
+
+
+def throughput_scale(tv, dev, stream, impl, layers, steps, peak, check):
+    """The 48-layer workload at a reduced layer count (same kernels, same per-layer work, one input
+    set larger than 4x L2): verify and commit against both peaks, driver-visible in the default run."""
+    wl = inputs.workload("c5", L=layers)
+    rig = StepRig(tv, wl, dev, stream, impl, n_sets=1)
+    step_ms = time_loop(stream, steps, rig.step)
+    verify, commit = kernel_split(rig, step_ms, steps, peak)
+    out = {"workload": DESCR["c5"] + f" -- run with {layers} of its 48 layers "
+                       f"({rig.set_bytes / 2**30:.1f} GiB resident, one input set > 4x L2)",
+           "steps": steps, "ms_per_step": step_ms, "nodes_per_s_per_layer": wl.B * wl.T * wl.L / (step_ms * 1e-3),
+           "verify": verify, "commit": commit}
+    if check:
+        out["parity"] = parity_check(rig, sorted({0, layers // 2, layers - 1}), 6)
+    del rig
+    torch.cuda.empty_cache()
+    return out
+
+
+def small_config_latency(tv, dev, stream, impl, name, launches=100):
+    """c1 / c2 are launch- and latency-bound (their ideal traffic time is a fraction of a
+    microsecond): report them as latency.  Every launch (or whole step) sits between its own pair
+    of events; 'warm' = back to back on the same buffers (resident in L2), 'cold' = a buffer
+    larger than L2 is overwritten before every launch."""
+    wl = inputs.workload(name)
+    rig = StepRig(tv, wl, dev, stream, impl, n_sets=1)
+    flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=dev)
+
+    def series(body, cold):
+        ts = []
+        for i in range(launches + 5):
+            if cold:
+                flush.fill_(i & 0xff)
+            e0, e1 = _ev(), _ev()
+            e0.record(stream)
+            body(i)
+            e1.record(stream)
+            ts.append((e0, e1))
+        torch.cuda.synchronize()
+        us = np.array([a.elapsed_time(b) * 1e3 for a, b in ts[5:]])
+        return {"median": float(np.median(us)), "min": float(us.min())}
+
+    out = {"workload": DESCR[name], "launches": launches, "unit": "us"}
+    rig.step(0)
+    torch.cuda.synchronize()
+    for key, body in (("verify", rig.verify_only), ("commit", rig.commit_only), ("step", rig.step)):
+        out[key] = {"l2_warm": series(body, False), "l2_cold": series(body, True)}
+    del rig, flush
+    return out
+
+
 def run_ours(args, wl, rank, world, local_rank):
     import paper_2608_01651_b200 as tv
     import torch.distributed as dist
@@ -476,106 +676,48 @@ def run_ours(args, wl, rank, world, local_rank):
     torch.cuda.set_device(local_rank)
     dev = f"cuda:{local_rank}"
     wl = rank_workload(wl, rank, args.layers)
-    parents, accepted = inputs.make_trees(wl)
-    acc_len = accepted_lengths(parents, accepted)
     delta = wl.rule == inputs.DELTA
     impl = {"auto": tv.IMPL_AUTO, "simt": tv.IMPL_SIMT, "tc": tv.IMPL_TC}[args.kernel]
-
-    # Input sets rotated between steps so that consecutive steps never find
-    # their inputs in L2: every set is larger than L2, or there are several.
-    eb = 2 if wl.qkv_dtype == inputs.BF16 else 4
-    set_bytes = wl.L * wl.B * wl.H * (4 * wl.dk * wl.dv + eb * wl.T * (2 * wl.dk + wl.dv) + 4 * wl.T * wl.dv)
-    n_sets = args.sets or max(2, min(8, int(np.ceil(4 * L2_BYTES / set_bytes))))
-    if set_bytes > 4 * L2_BYTES:
-        n_sets = args.sets or 1
-    sets = []
-    for s in range(n_sets):
-        layers = [inputs.make_tensors(wl, layer=s * wl.L + l, device=dev) for l in range(wl.L)]
-        st = {k: (None if layers[0][k] is None else torch.stack([x[k] for x in layers]))
-              for k in layers[0]}
-        del layers
-        st["O"] = torch.empty(wl.L, wl.B, wl.H, wl.T, wl.dv, device=dev, dtype=torch.float32)
-        st["U"] = torch.empty_like(st["O"]) if delta else None
-        sets.append(st)
-    acc_dev = torch.from_numpy(accepted).to(dev)
-    tree = tv.tree_build(parents)
     stream = torch.cuda.current_stream()
-
-    ev = lambda: torch.cuda.Event(enable_timing=True)
-    kernel_events = []
-    # Calls are marshalled once per input set; events are created before the timed region.
-    calls = []
-    for st in sets:
-        ver = [tv.prepare_tree_verify(tree, st["S_pre"][l], st["q"][l], st["k"][l], st["v"][l],
-                                      st["alpha"][l], None if st["beta"] is None else st["beta"][l],
-                                      rule=wl.rule, O=st["O"][l],
-                                      U=None if st["U"] is None else st["U"][l], impl=impl, stream=stream)
-               for l in range(wl.L)]
-        com = tv.prepare_commit_path(tree, acc_dev, st["S_pre"], st["k"], st["v"], st["alpha"], st["beta"],
-                                     rule=wl.rule, U=st["U"], stream=stream)
-        calls.append((ver, com))
-    # Per-kernel durations are sampled on every `probe`-th step of the timed region: an event
-    # between two launches costs a pipeline bubble (and undoes the dependent launch of the verify
-    # kernel behind the metadata kernel), so most steps run as a caller's loop would.
-    probe = max(1, args.probe_every)
-    event_pool = [(ev(), ev(), ev()) for _ in range(args.steps // probe + 1)]
-    refresh = tree.prepare_refresh(np.ascontiguousarray(parents, dtype=np.int32), stream)
-
-    def step(i, record):
-        ver, com = calls[i % n_sets]
-        refresh()
-        if record:
-            e0, e1, e2 = event_pool[len(kernel_events)]
-            e0.record(stream)
-        for call in ver:
-            call()
-        if record:
-            e1.record(stream)
-        com()
-        if record:
-            e2.record(stream)
-            kernel_events.append((e0, e1, e2))
+    rig = StepRig(tv, wl, dev, stream, impl, n_sets=args.sets)
+    parents, accepted, tree, n_sets = rig.parents, rig.accepted, rig.tree, rig.n_sets
 
     def barrier():
         if world > 1:
             dist.barrier()
 
     for i in range(args.warmup):
-        step(i, False)
+        rig.step(i)
     torch.cuda.synchronize()
     barrier()
     sampler = ClockSampler(local_rank) if rank == 0 else None
     if sampler:
         sampler.wait_ready()
-    t_start, t_end = ev(), ev()
+    t_start, t_end = _ev(), _ev()
     torch.cuda.synchronize()
     w0 = time.time()
     t_start.record(stream)
     for i in range(args.steps):
-        step(args.warmup + i, i % probe == 0)
+        rig.step(args.warmup + i)
     t_end.record(stream)
     torch.cuda.synchronize()
     w1 = time.time()
     barrier()
-    clocks = sample_clocks(sampler, w0, w1, lambda: [step(j, False) for j in range(16)]) if sampler else None
+    clocks = sample_clocks(sampler, w0, w1, lambda: [rig.step(j) for j in range(16)]) if sampler else None
     total_ms = t_start.elapsed_time(t_end)
-    v_ms = float(np.mean([a.elapsed_time(b) for a, b, _ in kernel_events])) / wl.L
-    c_ms = float(np.mean([b.elapsed_time(c) for _, b, c in kernel_events]))
+    peak, peak_kind = measured_peak()
 
-    # ---- the verify kernel alone, launches back to back over the rotating sets: what the events
-    # inside the step above cannot separate from launch latency (they sit between two launches)
-    n_b2b = 0 if args.no_b2b else 48
-    for i in range(n_sets if n_b2b else 0):
-        calls[i][0][0]()
-    torch.cuda.synchronize()
-    b0, b1 = ev(), ev()
-    b0.record(stream)
-    for i in range(n_b2b):
-        ver = calls[i % n_sets][0]
-        ver[i % len(ver)]()
-    b1.record(stream)
-    torch.cuda.synchronize()
-    v_b2b_ms = b0.elapsed_time(b1) / n_b2b if n_b2b else float("nan")
+    # ---- per-kernel split, event-free loops (their own step counts: short runs stay stable) ----
+    n_aux = args.steps if total_ms / args.steps > 1.0 else max(args.steps, 256)
+    aux_step_ms = time_loop(stream, n_aux, rig.step) if n_aux != args.steps else total_ms / args.steps
+    verify, commit = kernel_split(rig, aux_step_ms, n_aux, peak)
+    verify["loops"] = commit["loops"] = n_aux
+
+    # ---- parity of this very configuration against the oracle (outside the timed regions) ------
+    parity = None
+    if args.check and rank == 0:
+        layers = sorted({0, wl.L // 2, wl.L - 1})
+        parity = parity_check(rig, layers, args.check_items)
 
     # ---- Stage 1 (tree convolution + SiLU + normalisation + gates), timed on its own --------
     # Not part of the step above (the metric is defined on verify + commit); one launch per layer
@@ -615,8 +757,17 @@ def run_ours(args, wl, rank, world, local_rank):
         sess.free()
         del hs, hO, hS
 
+    # ---- the throughput-scale workload and the two latency-bound ones, in the default run ------
+    scale = small = None
+    if world == 1 and wl.name == "c3" and not args.no_extras:
+        scale = throughput_scale(tv, dev, stream, impl, args.scale_layers, args.scale_steps, peak, args.check)
+        small = {n: small_config_latency(tv, dev, stream, impl, n) for n in ("c1", "c2")}
+    if world == 1 and wl.name in ("c1", "c2"):
+        small = {wl.name: small_config_latency(tv, dev, stream, impl, wl.name)}
+
     # ---- max over ranks -----------------------------------------------------
-    total_ms, v_ms, c_ms, e2e_dt = max_over_ranks([total_ms, v_ms, c_ms, e2e[0] if e2e else 0.0], world, dev)
+    total_ms, v_ms, c_ms, e2e_dt = max_over_ranks([total_ms, verify["ms_per_layer"], commit["ms"],
+                                                   e2e[0] if e2e else 0.0], world, dev)
     if e2e:
         e2e[0] = e2e_dt
     if rank != 0:
@@ -625,11 +776,7 @@ def run_ours(args, wl, rank, world, local_rank):
     ms_per_step = total_ms / args.steps
     nodes_step = job_nodes_per_step(wl, world)
     value = nodes_step / (ms_per_step * 1e-3)
-    peak, peak_kind = measured_peak()
-    vbytes = verify_bytes_per_layer(wl, with_U=delta)
-    cbytes = commit_bytes_per_layer(wl, acc_len, with_U=delta) * wl.L
-    v_gbs = vbytes / (v_ms * 1e-3) / 1e9
-    c_gbs = cbytes / (c_ms * 1e-3) / 1e9 if c_ms > 0 else 0.0
+    v_gbs = rig.vbytes / (v_ms * 1e-3) / 1e9
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
@@ -637,9 +784,9 @@ def run_ours(args, wl, rank, world, local_rank):
         nb = min(wl.B, 32)
         done, dt, threads, layer = 0, 0.0, 1, 0
         while dt < args.cpu_budget and layer < 64:
-            small = inputs.workload(wl.name, B=nb, L=1, seed=wl.seed)
-            tens = inputs.make_tensors(small, layer=layer)
-            _, d1, t1, threads = oracle_sample(small, parents[:nb] if parents.shape[0] > 1 else parents,
+            small_wl = inputs.workload(wl.name, B=nb, L=1, seed=wl.seed)
+            tens = inputs.make_tensors(small_wl, layer=layer)
+            _, d1, t1, threads = oracle_sample(small_wl, parents[:nb] if parents.shape[0] > 1 else parents,
                                                accepted[:nb], tens, args.cpu_budget - dt, nb * wl.H)
             done += d1
             dt += t1
@@ -648,28 +795,31 @@ def run_ours(args, wl, rank, world, local_rank):
                "sample": f"{done} (request, head) items of the workload (memoised fp64 walk of all "
                          f"{wl.T} nodes + commit), {dt:.1f} s"}
 
+    tc = wl.qkv_dtype == inputs.BF16 and args.kernel != "simt"
     line = {
         "metric": "verified_tree_nodes_per_s_per_layer",
         "value": value, "unit": "nodes/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f32", "data": "synthetic",
+        "dtype": ("bf16 q/k/v, f32 state read as tf32 by the tensor cores, f32 accumulate, f32 outputs" if tc
+                  else "f32"),
+        "data": "synthetic",
         "config": {
             "workload": DESCR[wl.name], "layers_per_step": wl.L, "kernel": args.kernel,
             "step": "tree_build(host)+upload, tree_verify per layer, commit_path over all layers (in place)",
-            "l2": f"{n_sets} rotating input set(s) of {set_bytes / 2**20:.0f} MiB each (L2 is 126 MiB)",
-            "kernel_events": f"every {probe}th step ({len(kernel_events)} samples)",
+            "l2": f"{n_sets} rotating input set(s) of {rig.set_bytes / 2**20:.0f} MiB each (L2 is 126 MiB)",
+            "kernel_split": "event-free loops: 'metadata + verify' timed beside the full step, commit = the difference",
             "trees": inputs.tree_stats(parents, accepted),
         },
-        "verify": {"ms_per_layer": v_ms, "nodes_per_s_per_layer": wl.B * wl.T / (v_ms * 1e-3),
-                   "algorithmic_GBps": v_gbs, "frac_of_measured_copy": v_gbs / peak,
-                   "back_to_back_ms": v_b2b_ms,
-                   "back_to_back_frac_of_measured_copy": vbytes / (v_b2b_ms * 1e-3) / 1e9 / peak,
-                   "frac_of_nominal_8TBps": v_gbs / NOMINAL_HBM_GBS},
-        "commit": {"ms": c_ms, "algorithmic_GBps": c_gbs, "bytes": cbytes,
-                   "frac_of_measured_copy": c_gbs / peak, "frac_of_nominal_8TBps": c_gbs / NOMINAL_HBM_GBS},
+        "verify": verify,
+        "commit": commit,
         "roofline": {"kernel": "tree_verify", "bound": "hbm", "achieved": v_gbs, "peak": peak,
                      "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": v_gbs / peak,
-                     "traffic": args.traffic if args.traffic is not None else ncu_traffic(wl.name)},
+                     "traffic": args.traffic if args.traffic is not None else ncu_traffic(wl.name),
+                     "timing": "in the step (metadata kernel and launch gaps included); "
+                               "verify.back_to_back_* is the kernel alone"},
+        "parity": parity,
+        "throughput_scale": scale,
+        "small_configs": small,
         "cpu_baseline": cpu,
         "stage1": stage1,
         "e2e": None if e2e is None else {
@@ -681,6 +831,18 @@ def run_ours(args, wl, rank, world, local_rank):
         "clocks": clocks,
     }
     print(json.dumps(line, default=_jsonable), flush=True)
+
+
+def spawn_ranks(n: int) -> int:
+    """`python bench.py --gpus N` started by hand: run the N replica ranks (one process per GPU,
+    the same command line) under torch.distributed.run and hand back its exit code."""
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
 
 
 def main():
@@ -700,13 +862,20 @@ def main():
     ap.add_argument("--traffic", type=float, default=None,
                     help="ncu dram bytes per verify launch to echo into roofline.traffic")
     ap.add_argument("--probe-every", type=int, default=0,
-                    help="record per-kernel CUDA events on every n-th timed step "
-                         "(0: every 8th, or steps/64 if that is larger: about 64 samples)")
+                    help="(packed-forest line only) record per-kernel CUDA events on every n-th timed step")
+    ap.add_argument("--check", action="store_true",
+                    help="after the timed region, compare O, U and S_new of sampled (layer, request, head) "
+                         "items of this very run with the fp64 oracle and add a 'parity' object")
+    ap.add_argument("--check-items", type=int, default=8, help="sampled items per checked layer")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="skip the throughput-scale and small-config objects of the default run")
+    ap.add_argument("--scale-layers", type=int, default=6)
+    ap.add_argument("--scale-steps", type=int, default=10)
     ap.add_argument("--packed", action="store_true",
                     help="run the step on a packed forest of requests with different node counts (1 GPU)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-stage1", action="store_true")
-    ap.add_argument("--no-b2b", action="store_true", help="skip the back-to-back verify timing")
+    ap.add_argument("--no-b2b", action="store_true", help="(kept for old command lines; no effect)")
     ap.add_argument("--stage1-iters", type=int, default=48)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -716,6 +885,8 @@ def main():
     if args.probe_every <= 0:
         args.probe_every = max(8, args.steps // 64)
 
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours" and not args.packed:
+        sys.exit(spawn_ranks(args.gpus))
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))

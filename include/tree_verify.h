@@ -21,7 +21,8 @@
  * writes the one state that must persist, the state at the end of the accepted
  * root-to-node path (Section IV-D Eq. 10).
  *
- * Memory layout (all tensors dense, row-major, innermost index last):
+ * Memory layout (dense, row-major, innermost index last, unless tv_dims carries
+ * strides for the node-indexed tensors -- see tv_strides):
  *     S_pre, S_new : float  [L][B][H][dv][dk]   (the serving cache layout
  *                    "[H, dv, dk]" of Section IV-D, i.e. the transpose of the
  *                    paper's S in R^{dk x dv})
@@ -72,6 +73,17 @@ enum { TV_IMPL_AUTO = 0, TV_IMPL_SIMT = 1, TV_IMPL_TC = 2 }; /* kernel choice   
 
 typedef struct tv_tree tv_tree;             /* opaque, library-owned            */
 
+/* Element strides of a node-indexed tensor (d contiguous): element (layer l, request b,
+ * head h, node t, channel c) sits at (l * B + b) * b + h * h + t * t + c.  All three zero
+ * means the dense head-major layout of the table above.  Token-major projections
+ * [B][T][H][d] are {T*H*d, d, H*d}; q, k and v taken in place from one fused projection
+ * [B][T][C] are three base pointers with {T*C, d, C}.  Strides are multiples of 16 bytes
+ * for q, k, v, O, U (any value for alpha, beta) and must not make elements overlap.
+ * (Section IV-C folds "layout conversion" into the stages: this is that, with no copy.)   */
+typedef struct tv_strides {
+  int64_t b, h, t;
+} tv_strides;
+
 typedef struct tv_dims {
   int32_t L, B, H, T, dk, dv;
   int32_t rule;        /* TV_GATED / TV_GATED_DELTA                             */
@@ -85,6 +97,13 @@ typedef struct tv_dims {
                           several state heads is stored once): q and k have Hk
                           heads, [L][B][Hk][T][dk], and state head h reads
                           q/k head h / (H / Hk).  0 means Hk = H; H % Hk == 0. */
+  tv_strides qk;       /* layout of q and k (heads = Hk)                        */
+  tv_strides v;        /* layout of v                                           */
+  tv_strides gate;     /* layout of alpha and beta (d = 1)                      */
+  tv_strides out;      /* layout of O and U                                     */
+                       /* Strided layouts are for dense trees; a packed forest
+                          (tv_forest_build) keeps its planes and returns
+                          TV_ERR_UNSUPPORTED when any stride is set.            */
 } tv_dims;
 
 const char* tv_strerror(int status);
@@ -295,6 +314,25 @@ int tv_commit_path(const tv_tree* tree, const tv_dims* dims,
                    const float* U /*dev or NULL*/,
                    float* S_new /*dev*/,
                    void* stream);
+
+/* The same commit for a model whose recurrent layers own their caches separately
+ * (Section IV-D: "all linear layers" are committed together; Section V-B "Unified
+ * cross-layer state commit": one batched launch from per-request path descriptors
+ * shared by all layers).  Every table is a HOST array of n_layers DEVICE pointers,
+ * one tensor of a single layer each, in the layouts and with the alignment of
+ * tv_commit_path (dims->L is ignored; dims' strides apply inside every layer).
+ * v, beta, U may be NULL as tables under the rules of tv_commit_path.  The
+ * pointers travel in the kernel's parameters: ONE launch for up to 64 layers (one
+ * more per further 64), no device-side table to keep alive, no allocation.
+ * S_new[l] == S_pre[l] for every layer (in place) or for none; otherwise no
+ * S_new[l] may overlap any S_pre[m].  Stream order as for tv_commit_path.       */
+int tv_commit_path_layers(const tv_tree* tree, const tv_dims* dims,
+                          const int32_t* accepted /*dev [B]*/, int32_t n_layers,
+                          const float* const* S_pre /*host [n_layers] of dev*/,
+                          const void* const* k, const void* const* v,
+                          const float* const* alpha, const float* const* beta,
+                          const float* const* U, float* const* S_new,
+                          void* stream);
 
 /* ---- host-buffer round ------------------------------------------------------
  * The whole hot path (tv_tree_build -> tv_tree_verify -> tv_commit_path, i.e.

@@ -33,9 +33,14 @@ class TreeVerifyError(RuntimeError):
         super().__init__(f"{where}: {msg} ({status})")
 
 
+class _Strides(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int64) for n in ("b", "h", "t")]
+
+
 class _Dims(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in
-                ("L", "B", "H", "T", "dk", "dv", "rule", "qkv_dtype", "impl", "Hk")]
+                ("L", "B", "H", "T", "dk", "dv", "rule", "qkv_dtype", "impl", "Hk")] + \
+               [(n, _Strides) for n in ("qk", "v", "gate", "out")]
 
 
 class _ConvDims(ctypes.Structure):
@@ -84,6 +89,8 @@ def lib() -> ctypes.CDLL:
     L.tv_tree_device_status.restype = ctypes.c_int
     L.tv_tree_verify.argtypes = [vp, p(_Dims)] + [vp] * 9
     L.tv_commit_path.argtypes = [vp, p(_Dims)] + [vp] * 9
+    L.tv_commit_path_layers.argtypes = [vp, p(_Dims), vp, i32] + [vp] * 8
+    L.tv_commit_path_layers.restype = ctypes.c_int
     L.tv_tree_verify_static.argtypes = [vp, i32, p(_Dims)] + [vp] * 10
     L.tv_tree_verify_static.restype = ctypes.c_int
     L.tv_tree_conv.argtypes = [vp, p(_ConvDims)] + [vp] * 14
@@ -313,7 +320,25 @@ def _ptr(t):
     return ctypes.c_void_p(0 if t is None else t.data_ptr())
 
 
-def _dims(S_pre, k, v, rule, impl, tree=None) -> _Dims:
+def _strides_of(t, tail, B):
+    """Element strides (b, h, t) of a node-indexed tensor [(L,) B, heads, T(, d)]; all zero for a
+    contiguous one (the library's dense layout).  ``tail`` = 1 when the tensor has a channel axis."""
+    if t is None or t.is_contiguous():
+        return _Strides(0, 0, 0)
+    if tail and t.stride(-1) != 1:
+        raise ValueError("the channel axis must be contiguous")
+    st = t.stride()
+    b, h, n = st[-3 - tail], st[-2 - tail], st[-1 - tail]
+    if t.dim() == 4 + tail and t.shape[0] > 1 and st[0] != B * b:
+        raise ValueError("layers must be stacked with a stride of B batch strides")
+    return _Strides(b, h, n)
+
+
+def _same(a, b):
+    return (a.b, a.h, a.t) == (b.b, b.h, b.t)
+
+
+def _dims(S_pre, k, v, rule, impl, tree=None, q=None, gates=(), outs=()) -> _Dims:
     import torch
     if S_pre.dim() == 4:
         L = 1
@@ -337,13 +362,27 @@ def _dims(S_pre, k, v, rule, impl, tree=None) -> _Dims:
     Hk = k.shape[-3]
     if H % Hk:
         raise ValueError("the number of state heads must be a multiple of the number of key heads")
-    return _Dims(L, B, H, T, dk, dv, rule, dt, impl, 0 if Hk == H else Hk)
+    d = _Dims(L, B, H, T, dk, dv, rule, dt, impl, 0 if Hk == H else Hk)
+    # strided views (token-major projections, slices of a fused projection) are passed as they are
+    d.qk = _strides_of(k, 1, B)
+    if q is not None and not _same(_strides_of(q, 1, B), d.qk):
+        raise ValueError("q and k must share one layout")
+    d.v = _strides_of(v, 1, B)
+    gs = [_strides_of(g, 0, B) for g in gates if g is not None]
+    os_ = [_strides_of(o, 1, B) for o in outs if o is not None]
+    if any(not _same(x, gs[0]) for x in gs) or any(not _same(x, os_[0]) for x in os_):
+        raise ValueError("alpha and beta (and O and U) must share one layout")
+    if gs:
+        d.gate = gs[0]
+    if os_:
+        d.out = os_[0]
+    return d
 
 
-def _require(t, name, dtype=None):
+def _require(t, name, dtype=None, strided=False):
     if t is None:
         return
-    if not t.is_cuda or not t.is_contiguous():
+    if not t.is_cuda or not (strided or t.is_contiguous()):
         raise ValueError(f"{name} must be a contiguous CUDA tensor")
     if dtype is not None and t.dtype != dtype:
         raise ValueError(f"{name} must be {dtype}")
@@ -357,17 +396,18 @@ def tree_verify(tree: Tree, S_pre, q, k, v, alpha, beta=None, *, rule=GATED, O=N
     ``O`` or ``(O, U)``.
     """
     import torch
-    for t, n in ((S_pre, "S_pre"), (alpha, "alpha"), (beta, "beta")):
-        _require(t, n, torch.float32)
+    _require(S_pre, "S_pre", torch.float32)
+    for t, n in ((alpha, "alpha"), (beta, "beta")):
+        _require(t, n, torch.float32, strided=True)
     for t, n in ((q, "q"), (k, "k"), (v, "v")):
-        _require(t, n, k.dtype)
-    d = _dims(S_pre, k, v, rule, impl, tree)
+        _require(t, n, k.dtype, strided=True)
     if O is None:
-        O = torch.empty(*v.shape[:-1], d.dv, device=v.device, dtype=torch.float32)
+        O = torch.empty(*v.shape[:-1], v.shape[-1], device=v.device, dtype=torch.float32)
     if U is None and want_U:
         U = torch.empty_like(O)
-    _require(O, "O", torch.float32)
-    _require(U, "U", torch.float32)
+    _require(O, "O", torch.float32, strided=True)
+    _require(U, "U", torch.float32, strided=True)
+    d = _dims(S_pre, k, v, rule, impl, tree, q=q, gates=(alpha, beta), outs=(O, U))
     _check(lib().tv_tree_verify(tree._h, ctypes.byref(d), _ptr(S_pre), _ptr(q), _ptr(k), _ptr(v),
                                 _ptr(alpha), _ptr(beta), _ptr(O), _ptr(U), _stream_ptr(stream)),
            "tv_tree_verify")
@@ -383,15 +423,55 @@ def commit_path(tree: Tree, accepted, S_pre, k, v, alpha, beta=None, *, rule=GAT
     """
     import torch
     _require(accepted, "accepted", torch.int32)
-    for t, n in ((S_pre, "S_pre"), (alpha, "alpha"), (beta, "beta"), (U, "U"), (S_new, "S_new")):
+    for t, n in ((S_pre, "S_pre"), (S_new, "S_new")):
         _require(t, n, torch.float32)
+    for t, n in ((alpha, "alpha"), (beta, "beta"), (U, "U")):
+        _require(t, n, torch.float32, strided=True)
     for t, n in ((k, "k"), (v, "v")):
-        _require(t, n, k.dtype)
-    d = _dims(S_pre, k, v, rule, IMPL_AUTO, tree)
+        _require(t, n, k.dtype, strided=True)
+    d = _dims(S_pre, k, v, rule, IMPL_AUTO, tree, gates=(alpha, beta), outs=(U,))
     out = S_pre if S_new is None else S_new
     _check(lib().tv_commit_path(tree._h, ctypes.byref(d), _ptr(accepted), _ptr(S_pre), _ptr(k),
                                 _ptr(v), _ptr(alpha), _ptr(beta), _ptr(U), _ptr(out),
                                 _stream_ptr(stream)), "tv_commit_path")
+    return out
+
+
+def commit_path_layers(tree: Tree, accepted, S_pre, k, v, alpha, beta=None, *, rule=GATED, U=None,
+                       S_new=None, stream=None):
+    """``tv_commit_path_layers``: one commit launch over layers that own their tensors separately.
+
+    ``S_pre``, ``k``, ``v``, ``alpha`` (and ``beta``, ``U``, ``S_new`` when given) are lists with
+    one tensor per layer, each shaped like a single layer of ``commit_path``; all layers share
+    the tree, the accepted nodes, the shapes and the layout.  ``S_new=None`` commits in place.
+    """
+    import torch
+    _require(accepted, "accepted", torch.int32)
+    n = len(S_pre)
+    lists = {"k": k, "v": v, "alpha": alpha, "beta": beta, "U": U, "S_new": S_new}
+    for name, lst in lists.items():
+        if lst is not None and len(lst) != n:
+            raise ValueError(f"{name} must list one tensor per layer")
+    for l in range(n):
+        for t, nm in ((S_pre[l], "S_pre"), (None if S_new is None else S_new[l], "S_new")):
+            _require(t, nm, torch.float32)
+        for lst, nm in ((alpha, "alpha"), (beta, "beta"), (U, "U")):
+            _require(None if lst is None else lst[l], nm, torch.float32, strided=True)
+        for lst, nm in ((k, "k"), (v, "v")):
+            _require(None if lst is None else lst[l], nm, k[0].dtype, strided=True)
+    d = _dims(S_pre[0], k[0], v[0], rule, IMPL_AUTO, tree, gates=(alpha[0], None if beta is None else beta[0]),
+              outs=(None if U is None else U[0],))
+    for l in range(1, n):
+        dl = _dims(S_pre[l], k[l], v[l], rule, IMPL_AUTO, tree, gates=(alpha[l], None if beta is None else beta[l]),
+                   outs=(None if U is None else U[l],))
+        if bytes(dl) != bytes(d):
+            raise ValueError("all layers must share shapes and layout")
+    out = S_pre if S_new is None else S_new
+    table = lambda lst: None if lst is None else (ctypes.c_void_p * n)(*[t.data_ptr() for t in lst])
+    tabs = [table(x) for x in (S_pre, k, v, alpha, beta, U, out)]
+    _check(lib().tv_commit_path_layers(tree._h, ctypes.byref(d), _ptr(accepted), n,
+                                       *[None if t is None else ctypes.cast(t, ctypes.c_void_p) for t in tabs],
+                                       _stream_ptr(stream)), "tv_commit_path_layers")
     return out
 
 

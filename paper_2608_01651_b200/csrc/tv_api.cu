@@ -384,6 +384,38 @@ static int check_common(const tv_tree* t, const tv_dims* d) {
   return TV_OK;
 }
 
+}  // extern "C"
+
+// Strides of the node-indexed tensors: what the caller gave, or the dense head-major layout
+// [L][B][heads][T][d] for a tensor class whose three strides are all zero.
+int tv_resolve_layout(const tv_dims* d, bool packed, Layout* out) {
+  const int64_t H = d->H, Hk = d->Hk ? d->Hk : d->H, T = d->T;
+  const int es = d->qkv_dtype == TV_BF16 ? 2 : 4;
+  auto zero = [](const tv_strides& s) { return s.b == 0 && s.h == 0 && s.t == 0; };
+  if (packed && !(zero(d->qk) && zero(d->v) && zero(d->gate) && zero(d->out))) return TV_ERR_UNSUPPORTED;
+  auto resolve = [&](const tv_strides& s, int64_t heads, int64_t dch, int64_t align, Str3* o) -> int {
+    if (zero(s)) {
+      o->t = dch;
+      o->h = T * dch;
+      o->b = heads * T * dch;
+      return TV_OK;
+    }
+    if (s.b < 0 || s.h < 0 || s.t < 0) return TV_ERR_BAD_ARG;
+    if ((s.b % align) || (s.h % align) || (s.t % align)) return TV_ERR_BAD_ARG;
+    // extents larger than one need a stride that clears a row of d channels
+    if ((T > 1 && s.t < dch) || (heads > 1 && s.h < dch) || ((int64_t)d->L * d->B > 1 && s.b < dch)) return TV_ERR_BAD_ARG;
+    o->b = s.b; o->h = s.h; o->t = s.t;
+    return TV_OK;
+  };
+  int st = resolve(d->qk, Hk, d->dk, 16 / es, &out->qk);
+  if (st == TV_OK) st = resolve(d->v, H, d->dv, 16 / es, &out->v);
+  if (st == TV_OK) st = resolve(d->gate, H, 1, 1, &out->gate);
+  if (st == TV_OK) st = resolve(d->out, H, d->dv, 4, &out->out);
+  return st;
+}
+
+extern "C" {
+
 static TreeDev tree_dev(const tv_tree* t) {
   TreeDev td;
   td.anc = t->d_anc;
@@ -412,6 +444,8 @@ TV_API int tv_tree_verify(const tv_tree* tree, const tv_dims* d, const float* S_
   a.L = d->L; a.B = d->B; a.H = d->H; a.T = d->T; a.dk = d->dk; a.dv = d->dv;
   a.rule = d->rule; a.bf16 = d->qkv_dtype == TV_BF16; a.Hk = d->Hk ? d->Hk : d->H;
   a.S_pre = S_pre; a.q = q; a.k = k; a.v = v; a.alpha = alpha; a.beta = beta; a.O = O; a.U = U;
+  st = tv_resolve_layout(d, !tree->offsets.empty(), &a.lay);
+  if (st != TV_OK) return st;
   const bool tc_gated = tv_verify_tc_supports(a), tc_delta = tv_verify_tc_delta_supports(a),
              tc_delta128 = tv_verify_tc_delta128_supports(a);
   if (d->impl == TV_IMPL_TC && !tc_gated && !tc_delta && !tc_delta128) return TV_ERR_UNSUPPORTED;
@@ -423,31 +457,130 @@ TV_API int tv_tree_verify(const tv_tree* tree, const tv_dims* d, const float* S_
   return tv_launch_verify_simt(a, (cudaStream_t)stream);
 }
 
+// Shared by the two commit entry points: validation of one layer's pointers.
+static int check_commit_layer(const tv_dims* d, const float* S_pre, const void* k, const void* v,
+                              const float* alpha, const float* beta, const float* U, float* S_new) {
+  if (!S_pre || !k || !alpha || !S_new) return TV_ERR_BAD_ARG;
+  if (!U && !v) return TV_ERR_BAD_ARG;
+  if (d->rule == TV_GATED_DELTA && !U && !beta) return TV_ERR_BAD_ARG;
+  if (!aligned16(S_pre) || !aligned16(S_new) || !aligned16(k) || !aligned16(v) || !aligned16(U) ||
+      ((uintptr_t)alpha & 3) || ((uintptr_t)beta & 3))
+    return TV_ERR_BAD_ARG;
+  return TV_OK;
+}
+
+static int commit_args(const tv_tree* tree, const tv_dims* d, const int32_t* accepted, bool has_U,
+                       bool in_place, CommitArgs* a) {
+  a->tree = tree_dev(tree);
+  a->L = d->L; a->B = d->B; a->H = d->H; a->T = d->T; a->dk = d->dk; a->dv = d->dv;
+  a->rule = d->rule; a->bf16 = d->qkv_dtype == TV_BF16; a->Hk = d->Hk ? d->Hk : d->H;
+  a->has_U = has_U; a->in_place = in_place;
+  a->accepted = accepted;
+  return tv_resolve_layout(d, !tree->offsets.empty(), &a->lay);
+}
+
 TV_API int tv_commit_path(const tv_tree* tree, const tv_dims* d, const int32_t* accepted,
                    const float* S_pre, const void* k, const void* v, const float* alpha,
                    const float* beta, const float* U, float* S_new, void* stream) {
   int st = check_common(tree, d);
   if (st != TV_OK) return st;
-  if (!accepted || !S_pre || !k || !alpha || !S_new) return TV_ERR_BAD_ARG;
-  if (!U && !v) return TV_ERR_BAD_ARG;
-  if (d->rule == TV_GATED_DELTA && !U && !beta) return TV_ERR_BAD_ARG;
-  if (!aligned16(S_pre) || !aligned16(S_new) || !aligned16(k) || !aligned16(v) || !aligned16(U) ||
-      ((uintptr_t)alpha & 3) || ((uintptr_t)beta & 3) || ((uintptr_t)accepted & 3))
-    return TV_ERR_BAD_ARG;
+  if (!accepted || ((uintptr_t)accepted & 3)) return TV_ERR_BAD_ARG;
+  st = check_commit_layer(d, S_pre, k, v, alpha, beta, U, S_new);
+  if (st != TV_OK) return st;
+  const size_t state_elems = (size_t)d->B * d->H * d->dv * d->dk;   // one layer
   if (S_new != S_pre) {
-    const size_t bytes = sizeof(float) * (size_t)d->L * d->B * d->H * d->dv * d->dk;
+    const size_t bytes = sizeof(float) * (size_t)d->L * state_elems;
     const char* a0 = (const char*)S_pre;
     const char* b0 = (const char*)S_new;
     if (a0 < b0 + bytes && b0 < a0 + bytes) return TV_ERR_BAD_ARG;  // partial overlap
   }
   if (d->rule == TV_GATED_DELTA && !U && d->dk != 64 && d->dk != 128) return TV_ERR_UNSUPPORTED;
   CommitArgs a;
-  a.tree = tree_dev(tree);
-  a.L = d->L; a.B = d->B; a.H = d->H; a.T = d->T; a.dk = d->dk; a.dv = d->dv;
-  a.rule = d->rule; a.bf16 = d->qkv_dtype == TV_BF16; a.Hk = d->Hk ? d->Hk : d->H;
-  a.accepted = accepted; a.S_pre = S_pre; a.k = k; a.v = v; a.alpha = alpha; a.beta = beta;
-  a.U = U; a.S_new = S_new;
-  return tv_launch_commit(a, (cudaStream_t)stream);
+  st = commit_args(tree, d, accepted, U != nullptr, S_new == S_pre, &a);
+  if (st != TV_OK) return st;
+  // Layers stacked in one allocation: layer l of a node-indexed tensor starts B batch strides
+  // (or, in a packed forest, `heads` planes) after layer l-1.
+  const size_t es = d->qkv_dtype == TV_BF16 ? 2 : 4;
+  size_t k_step, v_step, g_step, u_step;
+  if (tree->offsets.empty()) {
+    k_step = (size_t)d->B * a.lay.qk.b * es;
+    v_step = (size_t)d->B * a.lay.v.b * es;
+    g_step = (size_t)d->B * a.lay.gate.b * 4;
+    u_step = (size_t)d->B * a.lay.out.b * 4;
+  } else {
+    const size_t cap = (size_t)tree->capacity;
+    k_step = (size_t)a.Hk * cap * d->dk * es;
+    v_step = (size_t)d->H * cap * d->dv * es;
+    g_step = (size_t)d->H * cap * 4;
+    u_step = (size_t)d->H * cap * d->dv * 4;
+  }
+  // one launch per kCommitMaxLayers layers (one launch in all for the usual 24..64 layers)
+  for (int l0 = 0; l0 < d->L; l0 += kCommitMaxLayers) {
+    CommitLayers tb = {};
+    a.L = d->L - l0 < kCommitMaxLayers ? d->L - l0 : kCommitMaxLayers;
+    for (int i = 0; i < a.L; ++i) {
+      const size_t l = (size_t)(l0 + i);
+      tb.S_pre[i] = S_pre + l * state_elems;
+      tb.S_new[i] = S_new + l * state_elems;
+      tb.k[i] = (const char*)k + l * k_step;
+      tb.v[i] = v ? (const char*)v + l * v_step : nullptr;
+      tb.alpha[i] = (const float*)((const char*)alpha + l * g_step);
+      tb.beta[i] = beta ? (const float*)((const char*)beta + l * g_step) : nullptr;
+      tb.U[i] = U ? (const float*)((const char*)U + l * u_step) : nullptr;
+    }
+    st = tv_launch_commit(a, tb, (cudaStream_t)stream);
+    if (st != TV_OK) return st;
+  }
+  return TV_OK;
+}
+
+TV_API int tv_commit_path_layers(const tv_tree* tree, const tv_dims* d, const int32_t* accepted, int32_t n_layers,
+                                 const float* const* S_pre, const void* const* k, const void* const* v,
+                                 const float* const* alpha, const float* const* beta, const float* const* U,
+                                 float* const* S_new, void* stream) {
+  if (!d || n_layers < 1) return TV_ERR_BAD_ARG;
+  tv_dims dl = *d;
+  dl.L = 1;                         // every table entry is one layer
+  int st = check_common(tree, &dl);
+  if (st != TV_OK) return st;
+  if (!accepted || ((uintptr_t)accepted & 3) || !S_pre || !k || !alpha || !S_new) return TV_ERR_BAD_ARG;
+  if (!U && !v) return TV_ERR_BAD_ARG;
+  if (d->rule == TV_GATED_DELTA && !U && !beta) return TV_ERR_BAD_ARG;
+  if (d->rule == TV_GATED_DELTA && !U && d->dk != 64 && d->dk != 128) return TV_ERR_UNSUPPORTED;
+  const size_t bytes = sizeof(float) * (size_t)d->B * d->H * d->dv * d->dk;
+  const bool in_place = S_new[0] == S_pre[0];
+  for (int l = 0; l < n_layers; ++l) {
+    st = check_commit_layer(&dl, S_pre[l], k[l], v ? v[l] : nullptr, alpha[l], beta ? beta[l] : nullptr,
+                            U ? U[l] : nullptr, S_new[l]);
+    if (st != TV_OK) return st;
+    // in place for all layers or for none; no layer's output may overlap any layer's input
+    if ((S_new[l] == S_pre[l]) != in_place) return TV_ERR_BAD_ARG;
+    for (int m = 0; m < n_layers; ++m) {
+      if (in_place && m == l) continue;
+      const char* a0 = (const char*)S_pre[m];
+      const char* b0 = (const char*)S_new[l];
+      if (a0 < b0 + bytes && b0 < a0 + bytes) return TV_ERR_BAD_ARG;
+    }
+  }
+  CommitArgs a;
+  st = commit_args(tree, &dl, accepted, U != nullptr, in_place, &a);
+  if (st != TV_OK) return st;
+  for (int l0 = 0; l0 < n_layers; l0 += kCommitMaxLayers) {
+    CommitLayers tb = {};
+    a.L = n_layers - l0 < kCommitMaxLayers ? n_layers - l0 : kCommitMaxLayers;
+    for (int i = 0; i < a.L; ++i) {
+      tb.S_pre[i] = S_pre[l0 + i];
+      tb.S_new[i] = S_new[l0 + i];
+      tb.k[i] = k[l0 + i];
+      tb.v[i] = v ? v[l0 + i] : nullptr;
+      tb.alpha[i] = alpha[l0 + i];
+      tb.beta[i] = beta ? beta[l0 + i] : nullptr;
+      tb.U[i] = U ? U[l0 + i] : nullptr;
+    }
+    st = tv_launch_commit(a, tb, (cudaStream_t)stream);
+    if (st != TV_OK) return st;
+  }
+  return TV_OK;
 }
 
 }  // extern "C"

@@ -10,6 +10,11 @@
 // The accepted path needs no parent walk: node indices grow along a
 // root-to-node path, so the set bits of the 128-bit ancestor mask of a, plus a
 // itself, are the path in topological order.
+//
+// Every kernel takes its tensors layer by layer from a table in its parameters (Section IV-D /
+// V-B: all linear layers are committed by one launch, whether they are stacked in one allocation
+// or own their caches separately); work item -> (layer, request, head), tensors of that layer,
+// rows addressed through the layout's strides within the layer.
 #include <cuda_bf16.h>
 
 #include "tv_internal.h"
@@ -26,15 +31,32 @@ __device__ __forceinline__ float load_elem(const void* base, size_t idx) {
   return reinterpret_cast<const float*>(base)[idx];
 }
 
+// Work item -> layer and item within the layer.
+struct LayerItem {
+  int l, it;   // layer of this launch, (request, head) item inside the layer
+  int b;       // request
+};
+__device__ __forceinline__ LayerItem layer_item(const CommitArgs& a, int item) {
+  LayerItem r;
+  const int bh = a.B * a.H;
+  r.l = item / bh;
+  r.it = item - r.l * bh;
+  r.b = r.it / a.H;
+  return r;
+}
+__device__ __forceinline__ ItemRows rows_of(const CommitArgs& a, int it_in_layer) {
+  return tv_item_rows(a.tree, a.lay, it_in_layer, a.B, a.H, a.Hk, a.T, a.dk, a.dv);
+}
+
 // Fills path_s[0..len) (topological order), w_s[p] = P_a / P_path[p] and *Pa_s.
 // al_s is scratch for the T decay gates (loaded by T threads in parallel so that
 // the serial suffix product below never waits on global memory).
 __device__ __forceinline__ int build_path(const TreeDev& tree, size_t meta0, int T, int acc,
-                                          const float* alpha_row, int* path_s, float* w_s,
+                                          const float* alpha, size_t g0, int64_t g_rs, int* path_s, float* w_s,
                                           float* al_s, float* Pa_s) {
   const uint64_t* m = tree.anc + (meta0 + acc) * 2;
   const int t = threadIdx.x;
-  if (t < T) al_s[t] = alpha_row[t];
+  if (t < T) al_s[t] = alpha[g0 + (size_t)t * g_rs];
   uint64_t m0 = m[0], m1 = m[1];
   if (acc < 64) m0 |= 1ull << acc; else m1 |= 1ull << (acc - 64);
   const int len = __popcll(m0) + __popcll(m1);
@@ -72,9 +94,10 @@ __device__ __forceinline__ void st_stream(float4* p, const float4& v) {
                :: "l"(p), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
 }
 
-// Commit from given correction rows u_j: U (float) when a.U != NULL, else v.
+// Commit from given correction rows u_j: U (float) when given, else v.
 template <bool BF16>
-__global__ void __launch_bounds__(kThreads) commit_factored_kernel(CommitArgs a) {
+__global__ void __launch_bounds__(kThreads)
+commit_factored_kernel(const CommitArgs a, const __grid_constant__ CommitLayers tb) {
   __shared__ int path_s[TV_MAX_NODES];
   __shared__ float w_s[TV_MAX_NODES];
   __shared__ float Pa_s;
@@ -82,21 +105,23 @@ __global__ void __launch_bounds__(kThreads) commit_factored_kernel(CommitArgs a)
   __shared__ __align__(16) float k_s[kPathChunk][TV_MAX_DIM];
   __shared__ float cu_s[kPathChunk][TV_MAX_DIM];
 
-  const int item = blockIdx.x;
-  const int b = (item / a.H) % a.B;
+  const LayerItem li = layer_item(a, blockIdx.x);
   const int tid = threadIdx.x;
   const int dk = a.dk, dv = a.dv;
-  const ItemRows rows = tv_item_rows(a.tree, item, a.B, a.H, a.Hk, a.T);
+  const ItemRows rows = rows_of(a, li.it);
   const int T = rows.n;
   const int n4 = dv * dk / 4;
-  const size_t sbase = (size_t)item * dv * dk;
-  const float4* src = reinterpret_cast<const float4*>(a.S_pre + sbase);
-  float4* dst = reinterpret_cast<float4*>(a.S_new + sbase);
+  const size_t sbase = (size_t)li.it * dv * dk;
+  const float4* src = reinterpret_cast<const float4*>(tb.S_pre[li.l] + sbase);
+  float4* dst = reinterpret_cast<float4*>(tb.S_new[li.l] + sbase);
+  const void* kg = tb.k[li.l];
+  const void* vg = tb.v[li.l];
+  const float* Ug = tb.U[li.l];
 
-  int acc = a.accepted[b];
+  int acc = a.accepted[li.b];
   if (acc >= T) acc = -1;
   if (acc < 0) {
-    if (a.S_new != a.S_pre)
+    if (!a.in_place)
       for (int i = tid; i < n4; i += kThreads) st_stream(dst + i, ld_stream(src + i));
     return;
   }
@@ -107,9 +132,7 @@ __global__ void __launch_bounds__(kThreads) commit_factored_kernel(CommitArgs a)
     const int i = tid + e * kThreads;
     if (i < n4) s[e] = ld_stream(src + i);
   }
-  const size_t node0 = rows.node0;  // first node row of this (l, b, h)
-  const size_t qk0 = rows.qk0;      // first key row (grouped key heads)
-  const int len = build_path(a.tree, rows.meta0, T, acc, a.alpha + node0, path_s, w_s, al_s, &Pa_s);
+  const int len = build_path(a.tree, rows.meta0, T, acc, tb.alpha[li.l], rows.g0, rows.g_rs, path_s, w_s, al_s, &Pa_s);
   const float Pa = Pa_s;
 #pragma unroll
   for (int e = 0; e < kMaxVec; ++e) {
@@ -121,12 +144,12 @@ __global__ void __launch_bounds__(kThreads) commit_factored_kernel(CommitArgs a)
     __syncthreads();
     for (int i = tid; i < nc * dk; i += kThreads) {
       const int p = i / dk, kk = i - p * dk;
-      k_s[p][kk] = load_elem<BF16>(a.k, (qk0 + path_s[c0 + p]) * dk + kk);
+      k_s[p][kk] = load_elem<BF16>(kg, rows.qk0 + (size_t)path_s[c0 + p] * rows.qk_rs + kk);
     }
     for (int i = tid; i < nc * dv; i += kThreads) {
       const int p = i / dv, vv = i - p * dv;
-      const size_t idx = (node0 + path_s[c0 + p]) * dv + vv;
-      const float u = a.U ? a.U[idx] : load_elem<BF16>(a.v, idx);
+      const float u = a.has_U ? Ug[rows.o0 + (size_t)path_s[c0 + p] * rows.o_rs + vv]
+                              : load_elem<BF16>(vg, rows.v0 + (size_t)path_s[c0 + p] * rows.v_rs + vv);
       cu_s[p][vv] = w_s[c0 + p] * u;
     }
     __syncthreads();
@@ -162,8 +185,20 @@ __global__ void __launch_bounds__(kThreads) commit_factored_kernel(CommitArgs a)
 constexpr int kRowThreads = 128;
 constexpr int kRowsPerCta = 64;
 
+// Four keys of a path row, widened to float.
 template <bool BF16>
-__global__ void __launch_bounds__(kRowThreads) commit_factored_dk128_kernel(CommitArgs a) {
+__device__ __forceinline__ float4 load_key4(const void* kg, size_t idx) {
+  if (BF16) {
+    const uint2 r = *reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(kg) + idx);
+    return make_float4(__uint_as_float(r.x << 16), __uint_as_float(r.x & 0xffff0000u),
+                       __uint_as_float(r.y << 16), __uint_as_float(r.y & 0xffff0000u));
+  }
+  return *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(kg) + idx);
+}
+
+template <bool BF16>
+__global__ void __launch_bounds__(kRowThreads)
+commit_factored_dk128_kernel(const CommitArgs a, const __grid_constant__ CommitLayers tb) {
   __shared__ int path_s[TV_MAX_NODES];
   __shared__ float w_s[TV_MAX_NODES];
   __shared__ float Pa_s;
@@ -174,16 +209,16 @@ __global__ void __launch_bounds__(kRowThreads) commit_factored_dk128_kernel(Comm
   const int dv = a.dv;
   const int n_half = (dv + kRowsPerCta - 1) / kRowsPerCta;
   const int item = blockIdx.x / n_half, half = blockIdx.x - item * n_half;
-  const int b = (item / a.H) % a.B;
+  const LayerItem li = layer_item(a, item);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int row0 = half * kRowsPerCta + warp * 16;
-  const size_t sbase = (size_t)item * dv * 128;
-  const float4* src = reinterpret_cast<const float4*>(a.S_pre + sbase) + (size_t)row0 * 32 + lane;
-  float4* dst = reinterpret_cast<float4*>(a.S_new + sbase) + (size_t)row0 * 32 + lane;
+  const size_t sbase = (size_t)li.it * dv * 128;
+  const float4* src = reinterpret_cast<const float4*>(tb.S_pre[li.l] + sbase) + (size_t)row0 * 32 + lane;
+  float4* dst = reinterpret_cast<float4*>(tb.S_new[li.l] + sbase) + (size_t)row0 * 32 + lane;
 
-  int acc = a.accepted[b];
+  int acc = a.accepted[li.b];
   if (acc >= a.T) acc = -1;
-  if (acc < 0 && a.S_new == a.S_pre) return;
+  if (acc < 0 && a.in_place) return;
   float4 s[16];
 #pragma unroll
   for (int e = 0; e < 16; ++e)
@@ -194,19 +229,20 @@ __global__ void __launch_bounds__(kRowThreads) commit_factored_dk128_kernel(Comm
   // tree metadata including the request offsets of a packed forest -- is read, and everything
   // they read that we write (S in place) is written, after this point.
   asm volatile("griddepcontrol.wait;" ::: "memory");
-  const ItemRows rows = tv_item_rows(a.tree, item, a.B, a.H, a.Hk, a.T);
+  const ItemRows rows = rows_of(a, li.it);
   const int T = rows.n;
   if (acc >= T) acc = -1;   // packed forest: beyond this request's node count
   if (acc < 0) {
-    if (a.S_new == a.S_pre) return;
+    if (a.in_place) return;
 #pragma unroll
     for (int e = 0; e < 16; ++e)
       if (row0 + e < dv) st_stream(dst + e * 32, s[e]);
     return;
   }
-  const size_t node0 = rows.node0;
-  const size_t qk0 = rows.qk0;
-  const int len = build_path(a.tree, rows.meta0, T, acc, a.alpha + node0, path_s, w_s, al_s, &Pa_s);
+  const void* kg = tb.k[li.l];
+  const void* vg = tb.v[li.l];
+  const float* Ug = tb.U[li.l];
+  const int len = build_path(a.tree, rows.meta0, T, acc, tb.alpha[li.l], rows.g0, rows.g_rs, path_s, w_s, al_s, &Pa_s);
   const float Pa = Pa_s;
   bool scaled = false;
   for (int c0 = 0; c0 < len; c0 += kPathChunk) {
@@ -214,25 +250,16 @@ __global__ void __launch_bounds__(kRowThreads) commit_factored_dk128_kernel(Comm
     if (c0) __syncthreads();
     for (int i = tid; i < nc * 32; i += kRowThreads) {   // 4 keys per thread per step
       const int p = i >> 5, k4 = i & 31;
-      const size_t idx = (qk0 + path_s[c0 + p]) * 128 + k4 * 4;
-      float4 kv;
-      if (BF16) {
-        const uint2 r = *reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(a.k) + idx);
-        kv = make_float4(__uint_as_float(r.x << 16), __uint_as_float(r.x & 0xffff0000u),
-                         __uint_as_float(r.y << 16), __uint_as_float(r.y & 0xffff0000u));
-      } else {
-        kv = *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(a.k) + idx);
-      }
-      *reinterpret_cast<float4*>(&k_s[p][k4 * 4]) = kv;
+      *reinterpret_cast<float4*>(&k_s[p][k4 * 4]) =
+          load_key4<BF16>(kg, rows.qk0 + (size_t)path_s[c0 + p] * rows.qk_rs + k4 * 4);
     }
     for (int i = tid; i < nc * kRowsPerCta; i += kRowThreads) {
       const int p = i >> 6, r = i & 63;
       const int vrow = half * kRowsPerCta + r;
       float u = 0.f;
-      if (vrow < dv) {
-        const size_t idx = (node0 + path_s[c0 + p]) * dv + vrow;
-        u = a.U ? a.U[idx] : load_elem<BF16>(a.v, idx);
-      }
+      if (vrow < dv)
+        u = a.has_U ? Ug[rows.o0 + (size_t)path_s[c0 + p] * rows.o_rs + vrow]
+                    : load_elem<BF16>(vg, rows.v0 + (size_t)path_s[c0 + p] * rows.v_rs + vrow);
       cu_s[p][r] = w_s[c0 + p] * u;
     }
     __syncthreads();
@@ -280,7 +307,8 @@ constexpr int kStreamMaxB = 256;
 constexpr int kStreamMaxLen = 16;
 
 template <bool BF16>
-__global__ void __launch_bounds__(kRowThreads, TV_STREAM_CTAS) commit_stream_dk128_kernel(CommitArgs a) {
+__global__ void __launch_bounds__(kRowThreads, TV_STREAM_CTAS)
+commit_stream_dk128_kernel(const CommitArgs a, const __grid_constant__ CommitLayers tb) {
   __shared__ int acc_s[kStreamMaxB];
   __shared__ uint64_t mask_s[kStreamMaxB][2];
   __shared__ __align__(16) float k_s[2][kStreamMaxLen][128];
@@ -293,8 +321,9 @@ __global__ void __launch_bounds__(kRowThreads, TV_STREAM_CTAS) commit_stream_dk1
   const int dv = a.dv, T = a.T;
   const int n_half = dv / kRowsPerCta;
   const int n_units = a.L * a.B * a.H * n_half;
+  const int units_per_layer = a.B * a.H * n_half;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const bool in_place = a.S_new == a.S_pre;
+  const bool in_place = a.in_place != 0;
 
   for (int b = tid; b < a.B; b += kRowThreads) {
     int acc = a.accepted[b];
@@ -303,8 +332,8 @@ __global__ void __launch_bounds__(kRowThreads, TV_STREAM_CTAS) commit_stream_dk1
     acc_s[b] = acc;
     uint64_t m0 = 0, m1 = 0;
     if (acc >= 0) {
-      const int tb = a.tree.n_trees == 1 ? 0 : b;
-      const uint64_t* m = a.tree.anc + ((size_t)tb * T + acc) * 2;
+      const int tb_ = a.tree.n_trees == 1 ? 0 : b;
+      const uint64_t* m = a.tree.anc + ((size_t)tb_ * T + acc) * 2;
       m0 = m[0];
       m1 = m[1];
       if (acc < 64) m0 |= 1ull << acc; else m1 |= 1ull << (acc - 64);
@@ -312,7 +341,6 @@ __global__ void __launch_bounds__(kRowThreads, TV_STREAM_CTAS) commit_stream_dk1
     mask_s[b][0] = m0;
     mask_s[b][1] = m1;
   }
-  asm volatile("griddepcontrol.wait;" ::: "memory");   // dependent launch: see the one-shot kernel
   __syncthreads();
 
   auto req_of = [&](int u) { return ((u / n_half) / a.H) % a.B; };
@@ -335,7 +363,9 @@ __global__ void __launch_bounds__(kRowThreads, TV_STREAM_CTAS) commit_stream_dk1
       const int r = lane < c0 ? lane : lane - c0;
       for (int i = 0; i < r; ++i) w &= w - 1;
       node = __ffsll((long long)w) - 1 + (lane < c0 ? 0 : 64);
-      al = a.alpha[tv_item_rows(a.tree, u / n_half, a.B, a.H, a.Hk, T).node0 + node];
+      const LayerItem li = layer_item(a, u / n_half);
+      const ItemRows rows = rows_of(a, li.it);
+      al = tb.alpha[li.l][rows.g0 + (size_t)node * rows.g_rs];
     }
     float incl = al;   // product of alpha over path positions >= lane
 #pragma unroll
@@ -360,8 +390,11 @@ __global__ void __launch_bounds__(kRowThreads, TV_STREAM_CTAS) commit_stream_dk1
   float ureg[8];
   auto fetch_rows = [&](int u, int nb) {
     const int item = u / n_half, half = u - item * n_half;
-    const ItemRows rows = tv_item_rows(a.tree, item, a.B, a.H, a.Hk, T);
-    const size_t node0 = rows.node0, qk0 = rows.qk0;
+    const LayerItem li = layer_item(a, item);
+    const ItemRows rows = rows_of(a, li.it);
+    const void* kg = tb.k[li.l];
+    const void* vg = tb.v[li.l];
+    const float* Ug = tb.U[li.l];
     const int len = len_s[nb];
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
@@ -370,11 +403,11 @@ __global__ void __launch_bounds__(kRowThreads, TV_STREAM_CTAS) commit_stream_dk1
       kreg[q] = make_uint2(0u, 0u);
       kreg2[q] = make_uint2(0u, 0u);
       if (p < len) {
-        const size_t idx = (qk0 + node_s[nb][p]) * 128 + k4 * 4;
+        const size_t idx = rows.qk0 + (size_t)node_s[nb][p] * rows.qk_rs + k4 * 4;
         if (BF16) {
-          kreg[q] = *reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(a.k) + idx);
+          kreg[q] = *reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(kg) + idx);
         } else {
-          const uint4 r = *reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(a.k) + idx);
+          const uint4 r = *reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(kg) + idx);
           kreg[q] = make_uint2(r.x, r.y);
           kreg2[q] = make_uint2(r.z, r.w);
         }
@@ -386,8 +419,9 @@ __global__ void __launch_bounds__(kRowThreads, TV_STREAM_CTAS) commit_stream_dk1
       const int p = i >> 6, r = i & 63;
       ureg[q] = 0.f;
       if (p < len) {
-        const size_t idx = (node0 + node_s[nb][p]) * dv + half * kRowsPerCta + r;
-        ureg[q] = a.U ? a.U[idx] : load_elem<BF16>(a.v, idx);
+        const int vrow = half * kRowsPerCta + r;
+        ureg[q] = a.has_U ? Ug[rows.o0 + (size_t)node_s[nb][p] * rows.o_rs + vrow]
+                          : load_elem<BF16>(vg, rows.v0 + (size_t)node_s[nb][p] * rows.v_rs + vrow);
       }
     }
   };
@@ -427,8 +461,9 @@ __global__ void __launch_bounds__(kRowThreads, TV_STREAM_CTAS) commit_stream_dk1
     const int un = next_live(u + gridDim.x);
     // a. the 16 loads of this unit
     const int row0 = warp * 16;
-    const float4* src = reinterpret_cast<const float4*>(a.S_pre) + ((size_t)u * kRowsPerCta + row0) * 32 + lane;
-    float4* dst = reinterpret_cast<float4*>(a.S_new) + ((size_t)u * kRowsPerCta + row0) * 32 + lane;
+    const int l = u / units_per_layer, ul = u - l * units_per_layer;
+    const float4* src = reinterpret_cast<const float4*>(tb.S_pre[l]) + ((size_t)ul * kRowsPerCta + row0) * 32 + lane;
+    float4* dst = reinterpret_cast<float4*>(tb.S_new[l]) + ((size_t)ul * kRowsPerCta + row0) * 32 + lane;
     float4 s[16];
 #pragma unroll
     for (int e = 0; e < 16; ++e) s[e] = ld_stream(src + e * 32);
@@ -477,7 +512,8 @@ __global__ void __launch_bounds__(kRowThreads, TV_STREAM_CTAS) commit_stream_dk1
 // row at a time (NPL consecutive floats per lane, dk = 32 NPL); the dot
 // product is a shuffle reduction.
 template <bool BF16, int NPL>
-__global__ void __launch_bounds__(kThreads) commit_delta_rows_kernel(CommitArgs a) {
+__global__ void __launch_bounds__(kThreads)
+commit_delta_rows_kernel(const CommitArgs a, const __grid_constant__ CommitLayers tb) {
   constexpr int DK = 32 * NPL;
   constexpr int kRowsPerWarp = TV_MAX_DIM / (kThreads / 32);  // 16
   __shared__ int path_s[TV_MAX_NODES];
@@ -488,35 +524,37 @@ __global__ void __launch_bounds__(kThreads) commit_delta_rows_kernel(CommitArgs 
   __shared__ float alc_s[kPathChunk], be_s[kPathChunk];
   __shared__ float al_s[TV_MAX_NODES];
 
-  const int item = blockIdx.x;
-  const int b = (item / a.H) % a.B;
+  const LayerItem li = layer_item(a, blockIdx.x);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int dv = a.dv;
-  const ItemRows rows = tv_item_rows(a.tree, item, a.B, a.H, a.Hk, a.T);
+  const ItemRows rows = rows_of(a, li.it);
   const int T = rows.n;
-  const size_t sbase = (size_t)item * dv * DK;
+  const size_t sbase = (size_t)li.it * dv * DK;
   const int n4 = dv * DK / 4;
+  const float* Sp = tb.S_pre[li.l] + sbase;
+  float* Sn = tb.S_new[li.l] + sbase;
+  const void* kg = tb.k[li.l];
+  const void* vg = tb.v[li.l];
+  const float* beta = tb.beta[li.l];
 
-  int acc = a.accepted[b];
+  int acc = a.accepted[li.b];
   if (acc >= T) acc = -1;
   if (acc < 0) {
-    if (a.S_new != a.S_pre) {
-      const float4* src = reinterpret_cast<const float4*>(a.S_pre + sbase);
-      float4* dst = reinterpret_cast<float4*>(a.S_new + sbase);
+    if (!a.in_place) {
+      const float4* src = reinterpret_cast<const float4*>(Sp);
+      float4* dst = reinterpret_cast<float4*>(Sn);
       for (int i = tid; i < n4; i += kThreads) dst[i] = src[i];
     }
     return;
   }
-  const size_t node0 = rows.node0;
-  const size_t qk0 = rows.qk0;
-  const int len = build_path(a.tree, rows.meta0, T, acc, a.alpha + node0, path_s, w_s, al_s, &Pa_s);
+  const int len = build_path(a.tree, rows.meta0, T, acc, tb.alpha[li.l], rows.g0, rows.g_rs, path_s, w_s, al_s, &Pa_s);
 
   float s[kRowsPerWarp][NPL];
 #pragma unroll
   for (int r = 0; r < kRowsPerWarp; ++r) {
     const int row = warp + r * (kThreads / 32);
     if (row < dv) {
-      const float* p = a.S_pre + sbase + (size_t)row * DK + lane * NPL;
+      const float* p = Sp + (size_t)row * DK + lane * NPL;
       if (NPL == 4) {
         const float4 t = *reinterpret_cast<const float4*>(p);
         s[r][0] = t.x; s[r][1] = t.y; s[r][2 % NPL] = t.z; s[r][3 % NPL] = t.w;
@@ -531,15 +569,15 @@ __global__ void __launch_bounds__(kThreads) commit_delta_rows_kernel(CommitArgs 
     __syncthreads();
     for (int i = tid; i < nc * DK; i += kThreads) {
       const int p = i / DK, kk = i - p * DK;
-      k_s[p][kk] = load_elem<BF16>(a.k, (qk0 + path_s[c0 + p]) * DK + kk);
+      k_s[p][kk] = load_elem<BF16>(kg, rows.qk0 + (size_t)path_s[c0 + p] * rows.qk_rs + kk);
     }
     for (int i = tid; i < nc * dv; i += kThreads) {
       const int p = i / dv, vv = i - p * dv;
-      v_s[p][vv] = load_elem<BF16>(a.v, (node0 + path_s[c0 + p]) * dv + vv);
+      v_s[p][vv] = load_elem<BF16>(vg, rows.v0 + (size_t)path_s[c0 + p] * rows.v_rs + vv);
     }
     if (tid < nc) {
       alc_s[tid] = al_s[path_s[c0 + tid]];
-      be_s[tid] = a.beta[node0 + path_s[c0 + tid]];
+      be_s[tid] = beta[rows.g0 + (size_t)path_s[c0 + tid] * rows.g_rs];
     }
     __syncthreads();
     for (int p = 0; p < nc; ++p) {
@@ -570,7 +608,7 @@ __global__ void __launch_bounds__(kThreads) commit_delta_rows_kernel(CommitArgs 
   for (int r = 0; r < kRowsPerWarp; ++r) {
     const int row = warp + r * (kThreads / 32);
     if (row < dv) {
-      float* p = a.S_new + sbase + (size_t)row * DK + lane * NPL;
+      float* p = Sn + (size_t)row * DK + lane * NPL;
       if (NPL == 4) {
         *reinterpret_cast<float4*>(p) = make_float4(s[r][0], s[r][1], s[r][2 % NPL], s[r][3 % NPL]);
       } else {
@@ -584,7 +622,8 @@ __global__ void __launch_bounds__(kThreads) commit_delta_rows_kernel(CommitArgs 
 // tree metadata it waited for is complete): the commit grid is scheduled as SMs drain, and every
 // kernel launched this way orders itself with griddepcontrol.wait.  Behind any other kernel this
 // is an ordinary launch.
-cudaError_t launch_after_verify(void (*kernel)(CommitArgs), int ctas, cudaStream_t stream, const CommitArgs& a) {
+cudaError_t launch_after_verify(void (*kernel)(const CommitArgs, const CommitLayers), int ctas, cudaStream_t stream,
+                                const CommitArgs& a, const CommitLayers& tb) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)ctas);
   cfg.blockDim = dim3((unsigned)kRowThreads);
@@ -595,15 +634,16 @@ cudaError_t launch_after_verify(void (*kernel)(CommitArgs), int ctas, cudaStream
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kernel, a);
+  return cudaLaunchKernelEx(&cfg, kernel, a, tb);
 }
 
 }  // namespace
 
-int tv_launch_commit(const CommitArgs& a, cudaStream_t stream) {
+int tv_launch_commit(const CommitArgs& a, const CommitLayers& tb, cudaStream_t stream) {
+  if (a.L < 1 || a.L > kCommitMaxLayers) return TV_ERR_BAD_ARG;
   const int items = a.L * a.B * a.H;
   if ((size_t)a.dk * a.dv > (size_t)kMaxVec * kThreads * 4) return TV_ERR_UNSUPPORTED;
-  const bool recompute = a.rule == TV_GATED_DELTA && a.U == nullptr;
+  const bool recompute = a.rule == TV_GATED_DELTA && !a.has_U;
   static thread_local int sm_count = 0;
   if (!sm_count) {
     int dev = 0;
@@ -616,22 +656,22 @@ int tv_launch_commit(const CommitArgs& a, cudaStream_t stream) {
       a.tree.max_depth_all < kStreamMaxLen) {
     const int ctas = TV_STREAM_CTAS * sm_count;
     // ordinary launch: at this size the dependent launch measured slower (13.4 vs 12.7 ms per step
-    // on 48 layers of 128 requests), the kernel's griddepcontrol.wait is then a no-op
-    if (a.bf16) commit_stream_dk128_kernel<true><<<ctas, kRowThreads, 0, stream>>>(a);
-    else commit_stream_dk128_kernel<false><<<ctas, kRowThreads, 0, stream>>>(a);
+    // on 48 layers of 128 requests)
+    if (a.bf16) commit_stream_dk128_kernel<true><<<ctas, kRowThreads, 0, stream>>>(a, tb);
+    else commit_stream_dk128_kernel<false><<<ctas, kRowThreads, 0, stream>>>(a, tb);
   } else if (!recompute && a.dk == 128) {
     const int ctas = items * ((a.dv + kRowsPerCta - 1) / kRowsPerCta);
-    TV_CUDA_TRY(a.bf16 ? launch_after_verify(commit_factored_dk128_kernel<true>, ctas, stream, a)
-                       : launch_after_verify(commit_factored_dk128_kernel<false>, ctas, stream, a));
+    TV_CUDA_TRY(a.bf16 ? launch_after_verify(commit_factored_dk128_kernel<true>, ctas, stream, a, tb)
+                       : launch_after_verify(commit_factored_dk128_kernel<false>, ctas, stream, a, tb));
   } else if (!recompute) {
-    if (a.bf16) commit_factored_kernel<true><<<items, kThreads, 0, stream>>>(a);
-    else commit_factored_kernel<false><<<items, kThreads, 0, stream>>>(a);
+    if (a.bf16) commit_factored_kernel<true><<<items, kThreads, 0, stream>>>(a, tb);
+    else commit_factored_kernel<false><<<items, kThreads, 0, stream>>>(a, tb);
   } else if (a.dk == 128) {
-    if (a.bf16) commit_delta_rows_kernel<true, 4><<<items, kThreads, 0, stream>>>(a);
-    else commit_delta_rows_kernel<false, 4><<<items, kThreads, 0, stream>>>(a);
+    if (a.bf16) commit_delta_rows_kernel<true, 4><<<items, kThreads, 0, stream>>>(a, tb);
+    else commit_delta_rows_kernel<false, 4><<<items, kThreads, 0, stream>>>(a, tb);
   } else if (a.dk == 64) {
-    if (a.bf16) commit_delta_rows_kernel<true, 2><<<items, kThreads, 0, stream>>>(a);
-    else commit_delta_rows_kernel<false, 2><<<items, kThreads, 0, stream>>>(a);
+    if (a.bf16) commit_delta_rows_kernel<true, 2><<<items, kThreads, 0, stream>>>(a, tb);
+    else commit_delta_rows_kernel<false, 2><<<items, kThreads, 0, stream>>>(a, tb);
   } else {
     return TV_ERR_UNSUPPORTED;
   }

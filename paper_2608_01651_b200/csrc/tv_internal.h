@@ -51,10 +51,23 @@ struct TreeDev {
   int32_t capacity;        // packed forest: rows of one (layer, head) plane
 };
 
+// Element strides of a node-indexed tensor: element (layer l, request b, head h, node t, channel c)
+// sits at (l * B + b) * b + h * h + t * t + c.  Always resolved (never all zero) by the time a
+// launcher sees them; a packed forest ignores them (its planes are addressed by request offsets).
+struct Str3 {
+  int64_t b, h, t;
+};
+struct Layout {
+  Str3 qk, v, gate, out;   // q and k | v | alpha and beta | O and U
+};
+// Fills `out` from the caller's tv_dims (zero strides = dense head-major) and validates it.
+int tv_resolve_layout(const tv_dims* d, bool packed, Layout* out);
+
 struct VerifyArgs {
   TreeDev tree;
   int32_t L, B, H, T, dk, dv, rule, bf16;
   int32_t Hk;  // q/k heads (H % Hk == 0); state head h reads q/k head h / (H / Hk)
+  Layout lay;
   const float* S_pre;
   const void* q;
   const void* k;
@@ -65,19 +78,40 @@ struct VerifyArgs {
   float* U;
 };
 
+// Commit: dimensions and flags; the tensors come layer by layer from a CommitLayers table, so that
+// layers that own their caches separately are committed by the same single launch as layers
+// stacked in one allocation.  Node-indexed tensors are addressed within their layer (the layer
+// index of Layout's (l * B + b) is always 0 here).
 struct CommitArgs {
   TreeDev tree;
-  int32_t L, B, H, T, dk, dv, rule, bf16;
+  int32_t L, B, H, T, dk, dv, rule, bf16;   // L = layers of this launch (<= kCommitMaxLayers)
   int32_t Hk;
+  int32_t has_U;      // corrections given (else v, or the delta rule re-derived along the path)
+  int32_t in_place;   // every layer's S_new is its S_pre
+  Layout lay;
   const int32_t* accepted;
-  const float* S_pre;
-  const void* k;
-  const void* v;
-  const float* alpha;
-  const float* beta;
-  const float* U;
-  float* S_new;
 };
+constexpr int kCommitMaxLayers = 64;
+struct CommitLayers {
+  const float* S_pre[kCommitMaxLayers];
+  float* S_new[kCommitMaxLayers];
+  const void* k[kCommitMaxLayers];
+  const void* v[kCommitMaxLayers];
+  const float* alpha[kCommitMaxLayers];
+  const float* beta[kCommitMaxLayers];
+  const float* U[kCommitMaxLayers];
+};
+
+// True when every node-indexed tensor has the dense head-major layout [L][B][heads][T][d] (or the
+// forest is packed, which has no strides): what the kernels that address rows by item index need.
+inline bool tv_layout_is_dense(const VerifyArgs& a) {
+  if (a.tree.offsets != nullptr) return true;
+  auto dense = [&](const Str3& s, int64_t heads, int64_t d) {
+    return s.t == d && s.h == (int64_t)a.T * d && s.b == heads * a.T * d;
+  };
+  return dense(a.lay.qk, a.Hk, a.dk) && dense(a.lay.v, a.H, a.dv) && dense(a.lay.gate, a.H, 1) &&
+         dense(a.lay.out, a.H, a.dv);
+}
 
 // Index of the q/k item (layer, request, key head) that state item (layer, request, head) reads.
 __host__ __device__ inline int tv_qk_item(int item, int H, int Hk) {
@@ -86,30 +120,39 @@ __host__ __device__ inline int tv_qk_item(int item, int H, int Hk) {
   return lb * Hk + h / (H / Hk);
 }
 
-// Where the rows of work item (layer l, request b, head h) live.  Dense layout: every item owns a
-// slab of T rows.  Packed forest: request b owns rows [offsets[b], offsets[b+1]) of every
+// Where the rows of work item (layer l, request b, head h) live: element offsets of node 0 and
+// the distance between consecutive nodes, per tensor class.  Dense or strided layout: from the
+// resolved strides.  Packed forest: request b owns rows [offsets[b], offsets[b+1]) of every
 // (layer, head) plane of `capacity` rows; its metadata slab is still T entries wide.
 struct ItemRows {
-  size_t node0;   // first row in v / alpha / beta / O / U
-  size_t qk0;     // first row in q / k
-  size_t meta0;   // first entry in the metadata arrays
-  int n;          // real nodes of this item
+  size_t qk0, v0, g0, o0;          // first element of node 0 in q/k | v | alpha/beta | O/U
+  int64_t qk_rs, v_rs, g_rs, o_rs; // elements from one node to the next
+  size_t meta0;                    // first entry in the metadata arrays
+  int n;                           // real nodes of this item
 };
-__device__ inline ItemRows tv_item_rows(const TreeDev& t, int item, int B, int H, int Hk, int T) {
+__device__ inline ItemRows tv_item_rows(const TreeDev& t, const Layout& lay, int item, int B, int H, int Hk,
+                                        int T, int dk, int dv) {
   ItemRows r;
   const int lb = item / H, h = item - lb * H;
   const int l = lb / B, b = lb - l * B;
   const int hk = Hk == H ? h : h / (H / Hk);
   if (t.offsets == nullptr) {
-    r.node0 = (size_t)item * T;
-    r.qk0 = (size_t)(lb * Hk + hk) * T;
+    r.qk0 = (size_t)((int64_t)lb * lay.qk.b + (int64_t)hk * lay.qk.h);
+    r.v0 = (size_t)((int64_t)lb * lay.v.b + (int64_t)h * lay.v.h);
+    r.g0 = (size_t)((int64_t)lb * lay.gate.b + (int64_t)h * lay.gate.h);
+    r.o0 = (size_t)((int64_t)lb * lay.out.b + (int64_t)h * lay.out.h);
+    r.qk_rs = lay.qk.t; r.v_rs = lay.v.t; r.g_rs = lay.gate.t; r.o_rs = lay.out.t;
     r.meta0 = (size_t)(t.n_trees == 1 ? 0 : b) * T;
     r.n = T;
   } else {
     const int off = t.offsets[b];
     r.n = t.offsets[b + 1] - off;
-    r.node0 = (size_t)(l * H + h) * t.capacity + off;
-    r.qk0 = (size_t)(l * Hk + hk) * t.capacity + off;
+    const size_t node0 = (size_t)(l * H + h) * t.capacity + off;
+    r.qk0 = ((size_t)(l * Hk + hk) * t.capacity + off) * dk;
+    r.v0 = node0 * dv;
+    r.g0 = node0;
+    r.o0 = node0 * dv;
+    r.qk_rs = dk; r.v_rs = dv; r.g_rs = 1; r.o_rs = dv;
     r.meta0 = (size_t)b * T;
   }
   return r;
@@ -119,7 +162,7 @@ void tv_set_cuda_error(cudaError_t e);
 
 // Launchers (each returns a tv_status; all work is asynchronous on `stream`).
 int tv_launch_verify_simt(const VerifyArgs& a, cudaStream_t stream);
-int tv_launch_commit(const CommitArgs& a, cudaStream_t stream);
+int tv_launch_commit(const CommitArgs& a, const CommitLayers& layers, cudaStream_t stream);
 int tv_launch_tree_meta(const int32_t* parent_mapped, int32_t n_trees, int32_t n, uint64_t* anc,
                         int32_t* depth, int32_t* parent_dev, int32_t* status, const int32_t* offsets_mapped,
                         int32_t* offsets_dev, int32_t depth_bound, int32_t generation, cudaStream_t stream);

@@ -85,6 +85,18 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t sr
       "cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4}], [%1];"
       ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2) : "memory");
 }
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar,
+                                            int c0, int c1, int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+      ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
 __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
@@ -189,6 +201,41 @@ inline bool make_map(CUtensorMap* map, const void* base, CUtensorMapDataType dt,
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+
+// 4-D view of a node-indexed tensor: element (z, h, t, c) at z*sb + h*sh + t*st + c (element
+// strides), c < d contiguous.  z = layer*request for dense and strided layouts, the layer for the
+// planes of a packed forest (t then runs over the plane's `capacity` rows).
+struct NodeView {
+  uint64_t d, T, Hx, Z;
+  int64_t sb, sh, st;
+};
+// Tensor maps want ascending strides: the node and head dimensions go in stride order, and the
+// kernel is told which of the two coordinates comes first.
+inline bool node_first_of(const NodeView& v) { return v.Hx == 1 || v.st <= v.sh; }
+inline uint64_t view_key(const NodeView& v) {
+  return (uint64_t)v.sb * 0x9e3779b97f4a7c15ull ^ (uint64_t)v.sh * 0xc2b2ae3d27d4eb4full ^ (uint64_t)v.st * 0x165667b19e3779f9ull ^
+         (v.T << 20) ^ (v.Hx << 8) ^ v.Z;
+}
+// Box {box_cols, box_rows nodes, 1 head, 1}; 128-byte swizzle, zero fill past the extents.
+inline bool make_map4(CUtensorMap* map, const void* base, CUtensorMapDataType dt, int esize, const NodeView& v,
+                      uint32_t box_cols, uint32_t box_rows) {
+  PFN_cuTensorMapEncodeTiled enc = get_encode();
+  if (!enc) return false;
+  const bool nf = node_first_of(v);
+  const uint64_t e1 = nf ? v.T : v.Hx, e2 = nf ? v.Hx : v.T;
+  uint64_t s1 = (uint64_t)(nf ? v.st : v.sh) * esize, s2 = (uint64_t)(nf ? v.sh : v.st) * esize,
+           s3 = (uint64_t)v.sb * esize;
+  // a dimension of extent 1 never advances: give it a stride that keeps the sequence ascending
+  if (e2 == 1) s2 = s1 * e1;
+  if (v.Z == 1) s3 = s2 * e2;
+  const cuuint64_t gdim[4] = {v.d, e1, e2, v.Z};
+  const cuuint64_t gstr[3] = {s1, s2, s3};
+  const cuuint32_t box[4] = {box_cols, nf ? box_rows : 1u, nf ? 1u : box_rows, 1};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  return enc(map, dt, 4, const_cast<void*>(base), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
 
 // (layer, request, head) of a work item and, for a packed forest, where its rows live: request b
 // owns rows offsets[b] .. offsets[b+1]-1 of every (layer, head) plane.

@@ -84,7 +84,7 @@ struct Smem {
 //   mode 1 (A = K): U_s[i][v] = beta_i (v_i[v] - P_i acc)
 template <bool BF16, int MODE>
 __device__ __forceinline__ void dense_pass(const VerifyArgs& a, const Smem& sm, const void* A,
-                                           size_t arow0, size_t node0, int T, float* Og) {
+                                           const ItemRows& rows, int T, float* Og) {
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
   const int dk = a.dk, dv = a.dv;
   float acc[8][8];
@@ -98,7 +98,7 @@ __device__ __forceinline__ void dense_pass(const VerifyArgs& a, const Smem& sm, 
     for (int idx = tid; idx < TV_MAX_NODES * kKC; idx += kThreads) {
       const int i = idx >> 5, kk = idx & 31;
       float x = 0.f;
-      if (i < T && k0 + kk < dk) x = load_elem<BF16>(A, (arow0 + i) * dk + k0 + kk);
+      if (i < T && k0 + kk < dk) x = load_elem<BF16>(A, rows.qk0 + (size_t)i * rows.qk_rs + k0 + kk);
       sm.A_s[i * kALD + kk] = x;
     }
     __syncthreads();
@@ -129,9 +129,9 @@ __device__ __forceinline__ void dense_pass(const VerifyArgs& a, const Smem& sm, 
       float4 r = make_float4(Pi * acc[m][half * 4 + 0], Pi * acc[m][half * 4 + 1],
                              Pi * acc[m][half * 4 + 2], Pi * acc[m][half * 4 + 3]);
       if (MODE == 0) {
-        *reinterpret_cast<float4*>(Og + (size_t)i * dv + v0) = r;
+        *reinterpret_cast<float4*>(Og + (size_t)i * rows.o_rs + v0) = r;
       } else {
-        const float4 vv = load4<BF16>(a.v, (node0 + i) * dv + v0);
+        const float4 vv = load4<BF16>(a.v, rows.v0 + (size_t)i * rows.v_rs + v0);
         const float be = sm.beta_s[i];
         r = make_float4(be * (vv.x - r.x), be * (vv.y - r.y), be * (vv.z - r.z), be * (vv.w - r.w));
         *reinterpret_cast<float4*>(sm.U_s + (size_t)i * dv + v0) = r;
@@ -145,7 +145,7 @@ __global__ void __launch_bounds__(kThreads) verify_simt_kernel(VerifyArgs a) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int dk = a.dk, dv = a.dv;
   const int item = blockIdx.x;
-  const ItemRows rows = tv_item_rows(a.tree, item, a.B, a.H, a.Hk, a.T);
+  const ItemRows rows = tv_item_rows(a.tree, a.lay, item, a.B, a.H, a.Hk, a.T, a.dk, a.dv);
   const int T = rows.n;   // real nodes of this item (the whole slab unless the forest is packed)
   Smem sm;
   {
@@ -161,18 +161,16 @@ __global__ void __launch_bounds__(kThreads) verify_simt_kernel(VerifyArgs a) {
     sm.U_s = reinterpret_cast<float*>(p);  // only with DELTA
   }
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const size_t node0 = rows.node0;
-  const size_t qk0 = rows.qk0;   // first q/k row (grouped key heads)
   const float* Sg = a.S_pre + (size_t)item * dv * dk;
-  float* Og = a.O + node0 * dv;
+  float* Og = a.O + rows.o0;
 
   // 1. metadata and path decay P_i
   if (tid < T) {
     const uint64_t* m = a.tree.anc + (rows.meta0 + tid) * 2;
     sm.anc_s[2 * tid] = m[0];
     sm.anc_s[2 * tid + 1] = m[1];
-    sm.alpha_s[tid] = a.alpha[node0 + tid];
-    sm.beta_s[tid] = DELTA ? a.beta[node0 + tid] : 0.f;
+    sm.alpha_s[tid] = a.alpha[rows.g0 + (size_t)tid * rows.g_rs];
+    sm.beta_s[tid] = DELTA ? a.beta[rows.g0 + (size_t)tid * rows.g_rs] : 0.f;
     sm.depth_s[tid] = a.tree.depth[rows.meta0 + tid];
   }
   __syncthreads();
@@ -195,8 +193,8 @@ __global__ void __launch_bounds__(kThreads) verify_simt_kernel(VerifyArgs a) {
   __syncthreads();
 
   // 3. dense part
-  dense_pass<BF16, 0>(a, sm, a.q, qk0, node0, T, Og);
-  if (DELTA) dense_pass<BF16, 1>(a, sm, a.k, qk0, node0, T, Og);
+  dense_pass<BF16, 0>(a, sm, a.q, rows, T, Og);
+  if (DELTA) dense_pass<BF16, 1>(a, sm, a.k, rows, T, Og);
   __syncthreads();
 
   const int nk = dk >> 2;  // lanes holding 4 consecutive k elements
@@ -208,13 +206,13 @@ __global__ void __launch_bounds__(kThreads) verify_simt_kernel(VerifyArgs a) {
       for (int i = warp; i < T; i += kWarps) {
         if (sm.depth_s[i] != lev) continue;
         float4 ki = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (lane < nk) ki = load4<BF16>(a.k, (qk0 + i) * dk + lane * 4);
+        if (lane < nk) ki = load4<BF16>(a.k, rows.qk0 + (size_t)i * rows.qk_rs + lane * 4);
         float acc[4] = {0.f, 0.f, 0.f, 0.f};
         uint64_t m0 = sm.anc_s[2 * i], m1 = sm.anc_s[2 * i + 1];
         float w = sm.alpha_s[i];  // P_i / P_parent(i)
         for (int j = pop_highest(m0, m1); j >= 0; j = pop_highest(m0, m1)) {
           float4 kj = make_float4(0.f, 0.f, 0.f, 0.f);
-          if (lane < nk) kj = load4<BF16>(a.k, (qk0 + j) * dk + lane * 4);
+          if (lane < nk) kj = load4<BF16>(a.k, rows.qk0 + (size_t)j * rows.qk_rs + lane * 4);
           const float dot = warp_sum(ki.x * kj.x + ki.y * kj.y + ki.z * kj.z + ki.w * kj.w);
           const float g = w * dot;
 #pragma unroll
@@ -238,21 +236,21 @@ __global__ void __launch_bounds__(kThreads) verify_simt_kernel(VerifyArgs a) {
   // 5. sparse readout: O_i += sum_j C_ij u_j
   for (int i = warp; i < T; i += kWarps) {
     float4 qi = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (lane < nk) qi = load4<BF16>(a.q, (qk0 + i) * dk + lane * 4);
+    if (lane < nk) qi = load4<BF16>(a.q, rows.qk0 + (size_t)i * rows.qk_rs + lane * 4);
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
     uint64_t m0 = sm.anc_s[2 * i], m1 = sm.anc_s[2 * i + 1];
     float w = 1.f;
     int j = i;
     while (j >= 0) {
       float4 kj = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (lane < nk) kj = load4<BF16>(a.k, (qk0 + j) * dk + lane * 4);
+      if (lane < nk) kj = load4<BF16>(a.k, rows.qk0 + (size_t)j * rows.qk_rs + lane * 4);
       const float dot = warp_sum(qi.x * kj.x + qi.y * kj.y + qi.z * kj.z + qi.w * kj.w);
       const float c = w * dot;
 #pragma unroll
       for (int x = 0; x < 4; ++x) {
         const int ch = lane + 32 * x;
         if (ch < dv) {
-          const float u = DELTA ? sm.U_s[(size_t)j * dv + ch] : load_elem<BF16>(a.v, (node0 + j) * dv + ch);
+          const float u = DELTA ? sm.U_s[(size_t)j * dv + ch] : load_elem<BF16>(a.v, rows.v0 + (size_t)j * rows.v_rs + ch);
           acc[x] = fmaf(c, u, acc[x]);
         }
       }
@@ -262,15 +260,17 @@ __global__ void __launch_bounds__(kThreads) verify_simt_kernel(VerifyArgs a) {
 #pragma unroll
     for (int x = 0; x < 4; ++x) {
       const int ch = lane + 32 * x;
-      if (ch < dv) Og[(size_t)i * dv + ch] += acc[x];
+      if (ch < dv) Og[(size_t)i * rows.o_rs + ch] += acc[x];
     }
   }
 
   // 6. corrections on request
   if (a.U) {
-    float* Ug = a.U + node0 * dv;
-    for (int i = tid; i < T * dv; i += kThreads)
-      Ug[i] = DELTA ? sm.U_s[i] : load_elem<BF16>(a.v, node0 * dv + i);
+    float* Ug = a.U + rows.o0;
+    for (int i = tid; i < T * dv; i += kThreads) {
+      const int t = i / dv, c = i - t * dv;
+      Ug[(size_t)t * rows.o_rs + c] = DELTA ? sm.U_s[i] : load_elem<BF16>(a.v, rows.v0 + (size_t)t * rows.v_rs + c);
+    }
   }
 }
 

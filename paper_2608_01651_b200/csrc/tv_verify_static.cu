@@ -136,6 +136,8 @@ int tv_tree_verify_static(const int32_t* parent, int32_t n_trees, const tv_dims*
   a.L = d->L; a.B = d->B; a.H = d->H; a.T = d->T; a.dk = d->dk; a.dv = d->dv;
   a.rule = d->rule; a.bf16 = d->qkv_dtype == TV_BF16; a.Hk = d->Hk ? d->Hk : d->H;
   a.S_pre = S_pre; a.q = q; a.k = k; a.v = v; a.alpha = alpha; a.beta = beta; a.O = O; a.U = U;
+  const int lst = tv_resolve_layout(d, false, &a.lay);
+  if (lst != TV_OK) return lst;
   // every refusal comes before the first launch: an error return has touched nothing, not even
   // the scratch that all calls share
   const bool tc_gated = tv_verify_tc_supports(a);

@@ -5,61 +5,100 @@
 // (Theorem 1 / Eq. 4 with U = V):
 //
 //   scores  Sc = Q K^T                 bf16 x bf16 -> fp32 in TMEM (exact products)
-//   prefix  acc = (2^e_i q_i) S_pre^T  tf32: q widened bf16 -> fp32 and scaled by
-//                                      a power of two (exact) into TMEM as the A
-//                                      operand; S_pre consumed as raw fp32
-//                                      straight from the TMA buffer
+//   prefix  acc = (2^e_i q_i) S_pre^T  bf16 x bf16 -> fp32.  A operand: the q rows scaled by
+//                                      a power of two (exact in bf16), written to TMEM by the
+//                                      compute warps.  B operand: S_pre split into bf16
+//                                      hi + lo (16 mantissa bits, both rounded to nearest)
+//                                      IN PLACE in the buffer the TMA filled: the fp32 row
+//                                      halves k 0..31 | 32..63 of a state row become its hi row
+//                                      and its lo row of 64 bf16 -- same bytes, same swizzle.
 //   C'_ij   = 1[j in Anc(i)+{i}] exp2(e_i - g_j) Sc_ij,  g = sum log2(alpha)
 //             over the path, e_i = round(g_i) (decay ratios only ever taken on
-//             ancestor pairs), split into bf16 hi + lo (~16 mantissa bits)
+//             ancestor pairs), split into bf16 hi + lo
 //   readout acc += C'_hi V + C'_lo V   bf16 x bf16 -> fp32, same accumulator
 //   O_i     = exp2(g_i - e_i) acc_i    fp32 epilogue
 // The accumulator is double-buffered in TMEM: the epilogue of item n runs under
 // the MMAs of item n+1.
 //
-// S_pre (the HBM-dominant stream) goes TMA -> shared memory -> tensor core and
-// is never touched by a thread.  Nothing but O is written.
+// Why the state is split rather than fed to the tensor core as fp32 (kind::tf32 cuts the
+// mantissa to 10 bits): a state that has absorbed many rank-one updates is dominated by a
+// few directions, a query nearly orthogonal to them sums large terms that cancel, and the
+// tf32 cut of those terms reached 1e-2 of the output in such states (5e-4 on unstructured
+// ones).  The split keeps 16 bits (worst case seen 4e-4, typically 1e-5), costs half the
+// tensor time of the tf32 product, and needs no extra shared memory.
 //
-// Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer (owns TMEM), warps
-// 2..9 = 8 compute warps; compute warp w reads TMEM lanes 32 (w % 4) .. +31
-// (the hardware's lane window of that warp) and half of the columns.
-// Every wait is an mbarrier wait with a time limit; on expiry the CTA sets the
-// status word, drains its own copies and leaves (TMEM is freed on every path).
+// T <= 64 (SMALL): operand boxes of 64 rows, and the shared memory that frees holds a second
+// stage of S_pre, so that the state of item n+1 (the HBM-dominant stream) is in flight while
+// item n is worked on.  T > 64: one stage of everything.
+//
+// Warp roles, in groups of four warps so that registers can be moved between them
+// (setmaxnreg): warp 0 = TMA producer, warp 1 = MMA issuer (owns TMEM), warp 2 = issues the
+// output stores (warp 3 idle), 56 registers each; warps 4..11 = 8 compute warps, 168
+// registers: compute warp w reads TMEM lanes 32 (w % 4) .. +31 (the hardware's lane window of
+// that warp) and half of the columns; warps 12..15 = the state split, 112 registers: they see
+// a state stage land, rewrite it and hand it to the MMA issuer, so that the compute warps'
+// chain of epilogues never waits on the state stream.  Every wait is an mbarrier wait with a
+// time limit; on expiry the CTA sets the status word, drains its own copies and leaves (TMEM
+// is freed on every path).
 #include "tv_tc_common.cuh"
 
 namespace {
 
 using namespace tvtc;
 
-constexpr int kThreads = 352;     // producer, MMA issuer, 8 compute warps, output-store warp
+constexpr int kThreads = 512;     // 4 service warps, 8 compute warps, 4 state-split warps
 constexpr int kComputeWarps = 8;
+constexpr int kFirstComputeWarp = 4;
+constexpr int kFirstSplitWarp = 12;
+constexpr int kSplitWarps = 4;
 
-// shared memory map (byte offsets from the 1024-aligned base)
-constexpr uint32_t kOffQ = 0;                     // 2 tiles: k halves of Q  [128][64] bf16
-constexpr uint32_t kOffK = kOffQ + 2 * kTile;     // 2 tiles: k halves of K
-constexpr uint32_t kOffV = kOffK + 2 * kTile;     // 2 tiles: dv halves of V [128 j][64] bf16
-constexpr uint32_t kOffS = kOffV + 2 * kTile;     // 4 tiles: k chunks of S_pre [128 v][32] f32
-constexpr uint32_t kOffChi = kOffS + 4 * kTile;   // 2 tiles: j halves of C_hi [128 i][64] bf16
-constexpr uint32_t kOffClo = kOffChi + 2 * kTile; // 2 tiles: j halves of C_lo
-constexpr uint32_t kOffG = kOffClo + 2 * kTile;   // float g[128]
-constexpr uint32_t kOffAl = kOffG + 512;          // float log2(alpha)[128]
-constexpr uint32_t kOffF = kOffAl + 512;          // float exp2(-g)[128]
-constexpr uint32_t kOffBar = kOffF + 512;         // mbarriers
-constexpr uint32_t kOffMisc = kOffBar + 8 * 24;   // tmem base, abort flag
-constexpr uint32_t kSmemBytes = kOffMisc + 48 + 1024;  // + alignment slack
-
-enum Bar {
-  QK_FULL = 0, QK_FREE, S_FULL, S_FREE, V_FULL, V_FREE,
-  SC_DONE, SC_FREE, QF_READY, C_READY, ACC_DONE0, ACC_DONE1, ACC_FREE0, ACC_FREE1, SETUP,
-  OST_READY, OST_FREE
+// Shared memory map (byte offsets from the 1024-aligned base).  An MMA with M = 128 reads 128
+// rows of its A tile whatever T is: with 64-row boxes the rows 64..127 it reads are the bytes
+// of the next buffer; they only reach accumulator rows >= 64, which nobody reads.
+template <bool SMALL>
+struct Lay {
+  static constexpr uint32_t kBox = SMALL ? kTile / 2 : kTile;   // one operand box: [64 | 128 rows][64 bf16]
+  static constexpr int kStages = SMALL ? 2 : 1;                 // stages of S_pre
+  static constexpr uint32_t kOffQ = 0;                          // 2 boxes: k halves of Q
+  static constexpr uint32_t kOffK = kOffQ + 2 * kBox;           // 2 boxes: k halves of K
+  static constexpr uint32_t kOffV = kOffK + 2 * kBox;           // 2 boxes: dv halves of V [j][64]
+  static constexpr uint32_t kOffS = kOffV + 2 * kBox;           // per stage 4 tiles [128 v][128 B]: fp32 k chunks,
+                                                                // after the split: hi | lo | hi | lo of the k halves
+  static constexpr uint32_t kOffChi = kOffS + kStages * 4 * kTile;   // C'_hi: j halves [128 i][64] (SMALL: one, 64 rows live)
+  static constexpr uint32_t kOffClo = kOffChi + (SMALL ? kBox : 2 * kTile);
+  // output staging: four chunks [64 | 128 rows][32 fp32].  SMALL: a region of its own; else the
+  // four C' tiles themselves, idle once the readout MMAs of the item are complete
+  static constexpr uint32_t kOffStage = SMALL ? kOffClo + kBox : kOffChi;
+  static constexpr uint32_t kStageChunk = SMALL ? kTile / 2 : kTile;
+  static constexpr uint32_t kOffG = SMALL ? kOffStage + 4 * kStageChunk : kOffClo + 2 * kTile;   // float g[128]
+  static constexpr uint32_t kOffAl = kOffG + 512;          // float log2(alpha)[128]
+  static constexpr uint32_t kOffF = kOffAl + 512;          // float exp2(-g)[128]
+  static constexpr uint32_t kOffBar = kOffF + 512;         // mbarriers
+  static constexpr uint32_t kOffMisc = kOffBar + 8 * 24;   // tmem base, abort flags, per-warp range flags
+  static constexpr uint32_t kSmemBytes = kOffMisc + 48 + 1024;  // + alignment slack
 };
 
-// TMEM columns: scaled Q (A operand), scores, two output accumulators
-constexpr uint32_t kColQf = 0, kColSc = 128, kColAcc0 = 256, kColAcc1 = 384;
+enum Bar {
+  QK_FULL = 0, QK_FREE, S_FULL0, S_FULL1, S_CONV0, S_CONV1, S_FREE0, S_FREE1, V_FULL, V_FREE,
+  SC_DONE, SC_FREE, QB_READY, QS_READY, C_READY, ACC_DONE0, ACC_DONE1, ACC_FREE0, ACC_FREE1, SETUP,
+  OST_READY, OST_FREE, kNumBars
+};
+static_assert(kNumBars <= 24, "barrier area");
 
-constexpr uint32_t kIdescBf16KK = idesc_bf16(128, false);
-constexpr uint32_t kIdescBf16KMn = idesc_bf16(128, true);
-constexpr uint32_t kIdescTf32 = idesc_tf32(128);
+// TMEM columns: scaled Q as packed bf16 (A operand of the prefix MMA), scores, two accumulators
+constexpr uint32_t kColQb = 0, kColSc = 128, kColAcc0 = 256, kColAcc1 = 384;
+
+constexpr uint32_t kIdescKK128 = idesc_bf16(128, false);
+constexpr uint32_t kIdescKK64 = idesc_bf16(64, false);
+constexpr uint32_t kIdescKMn = idesc_bf16(128, true);
+
+__device__ __forceinline__ void mma_bf16_ts(uint32_t d, uint32_t a_tmem, uint64_t b, uint32_t idesc,
+                                            uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d), "r"(a_tmem), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
+}
 
 // Eight fp32 values -> bf16 hi and lo parts (hi = upper 16 bits, lo = the exact remainder cut to
 // its upper 16 bits: hi + lo carries 16 mantissa bits), stored as two 16-byte chunks.
@@ -79,13 +118,59 @@ __device__ __forceinline__ void store_split8(unsigned char* chi, unsigned char* 
   *reinterpret_cast<uint4*>(clo + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
 }
 
+// Two fp32 -> one word of two bf16, rounded to nearest even (first argument in the low half).
+__device__ __forceinline__ uint32_t pack_bf16_rn(float lo_elem, float hi_elem) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi_elem), "f"(lo_elem));
+  return r;
+}
+
+// The state split.  Thread (row v, k half p) owns the two 128-byte rows that hold
+// S_pre[v][64 p .. 64 p + 63] as fp32 (row v of tiles 2p and 2p + 1 of the stage, 128-byte
+// swizzle) and rewrites them as 64 bf16 hi values (tile 2p) and 64 bf16 lo values (tile 2p + 1)
+// in the K-major swizzled layout the MMA reads: hi = rn(x), lo = rn(x - hi), x - hi exact.
+// Everything is read before anything is written; no other thread touches these rows.
+__device__ __forceinline__ void split_state_row(unsigned char* stage, int row, int p, uint32_t swz) {
+  unsigned char* r0 = stage + (uint32_t)(2 * p) * kTile + (uint32_t)row * 128u;
+  unsigned char* r1 = r0 + kTile;
+  uint4 hi[8], lo[8];
+#pragma unroll
+  for (int c = 0; c < 8; ++c) {   // output chunk c = k 8c .. 8c + 7 of this half
+    const unsigned char* src = c < 4 ? r0 : r1;
+    const uint32_t f = (uint32_t)(c & 3) * 2u;
+    const float4 a = *reinterpret_cast<const float4*>(src + ((f ^ swz) << 4));
+    const float4 b = *reinterpret_cast<const float4*>(src + (((f + 1u) ^ swz) << 4));
+    const float x[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+    uint32_t h[4], l[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      h[e] = pack_bf16_rn(x[2 * e], x[2 * e + 1]);
+      const float l0 = x[2 * e] - __uint_as_float(h[e] << 16);
+      const float l1 = x[2 * e + 1] - __uint_as_float(h[e] & 0xffff0000u);
+      l[e] = pack_bf16_rn(l0, l1);
+    }
+    hi[c] = make_uint4(h[0], h[1], h[2], h[3]);
+    lo[c] = make_uint4(l[0], l[1], l[2], l[3]);
+  }
+#pragma unroll
+  for (int c = 0; c < 8; ++c) {
+    *reinterpret_cast<uint4*>(r0 + (((uint32_t)c ^ swz) << 4)) = hi[c];
+    *reinterpret_cast<uint4*>(r1 + (((uint32_t)c ^ swz) << 4)) = lo[c];
+  }
+}
+
 struct TcParams {
   TreeDev tree;
   int32_t n_items, B, H, T;
   int32_t Hk;  // q/k heads (grouped key heads); H when not grouped
   const float* alpha;
+  Str3 gate;   // strides of alpha (dense layouts)
   float* O;
   int32_t* status;
+  // The tensor maps are 4-D, (channel, node, head, layer*request) or (channel, head, node, ...)
+  // whichever has ascending strides: bit 0 / 1 / 2 set = q,k / v / O take the node coordinate
+  // before the head coordinate.
+  int32_t node_first;
   // packed forest only: request b owns rows offsets[b] .. offsets[b+1]-1 of every plane of
   // `capacity` rows; T is then the per-request node limit (width of the metadata slabs)
   const int32_t* offsets;
@@ -96,41 +181,84 @@ __device__ __forceinline__ PackedItem packed_item(const TcParams& p, int item) {
   return tvtc::packed_item(p.offsets, p.B, p.H, p.Hk, item);
 }
 
+// Coordinates of an item's boxes: (head, outermost) of q/k and of v/O, and the first node row.
+struct ItemCoord {
+  int h_qk, h_v, z, y0;
+};
+template <bool PACKED>
+__device__ __forceinline__ ItemCoord item_coord(const TcParams& p, int item) {
+  ItemCoord c;
+  const int lb = item / p.H, h = item - lb * p.H;
+  c.h_v = h;
+  c.h_qk = p.Hk == p.H ? h : h / (p.H / p.Hk);
+  if constexpr (PACKED) {
+    const int l = lb / p.B, b = lb - l * p.B;
+    c.z = l;
+    c.y0 = p.offsets[b];
+  } else {
+    c.z = lb;
+    c.y0 = 0;
+  }
+  return c;
+}
+__device__ __forceinline__ void load_box(uint32_t dst, const CUtensorMap* m, uint32_t bar, bool node_first, int x,
+                                         int y, int h, int z) {
+  if (node_first) tma_load_4d(dst, m, bar, x, y, h, z);
+  else tma_load_4d(dst, m, bar, x, h, y, z);
+}
+__device__ __forceinline__ void store_box(const CUtensorMap* m, uint32_t src, bool node_first, int x, int y, int h,
+                                          int z) {
+  if (node_first) tma_store_4d(m, src, x, y, h, z);
+  else tma_store_4d(m, src, x, h, y, z);
+}
+
 // PACKED = packed forest: q/k/v/O are planes of `capacity` rows and an item's rows start at its
 // request's offset.  Loads take the fixed box at that offset (rows past the request belong to
 // other requests and are masked like padding); stores are cut to the request's node count:
 // 8-row-aligned part by TMA boxes of 64/32/16/8 rows (tmO, tmO32, tmO16, tmO8), the last < 8
 // rows straight from registers.  The dense instantiation ignores the three extra maps.
-template <bool PACKED>
+template <bool PACKED, bool SMALL>
 __global__ void __launch_bounds__(kThreads, 1)
 verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                        const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmS,
                        const __grid_constant__ CUtensorMap tmO, const __grid_constant__ CUtensorMap tmO32,
                        const __grid_constant__ CUtensorMap tmO16, const __grid_constant__ CUtensorMap tmO8,
                        const TcParams p) {
+  using L = Lay<SMALL>;
+  constexpr uint32_t kBox = L::kBox;
+  constexpr int kBoxRows = SMALL ? 64 : 128;
   extern __shared__ unsigned char smem_raw[];
   unsigned char* sm = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   const uint32_t sbase = smem_u32(sm);
-  float* g_s = reinterpret_cast<float*>(sm + kOffG);
-  float* la_s = reinterpret_cast<float*>(sm + kOffAl);
-  float* f_s = reinterpret_cast<float*>(sm + kOffF);
-  volatile int* range_ok_s = reinterpret_cast<volatile int*>(sm + kOffMisc + 16);   // [8] per compute warp
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + kOffMisc);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + kOffMisc + 4);
-  auto bar = [&](int i) { return sbase + kOffBar + 8u * i; };
+  float* g_s = reinterpret_cast<float*>(sm + L::kOffG);
+  float* la_s = reinterpret_cast<float*>(sm + L::kOffAl);
+  float* f_s = reinterpret_cast<float*>(sm + L::kOffF);
+  volatile int* range_ok_s = reinterpret_cast<volatile int*>(sm + L::kOffMisc + 16);   // [8] per compute warp
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + L::kOffMisc);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + L::kOffMisc + 4);
+  auto bar = [&](int i) { return sbase + L::kOffBar + 8u * i; };
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int T = p.T;
-  const int n_jh = T > 64 ? 2 : 1;  // 64-wide j halves that hold real nodes
+  const int n_jh = (!SMALL && T > 64) ? 2 : 1;  // 64-wide j halves that hold real nodes
+  const bool nf_qk = p.node_first & 1, nf_v = p.node_first & 2, nf_o = p.node_first & 4;
+  // stage of S_pre that item `it` of this CTA uses, and the parity of that use
+  auto s_stage = [](uint32_t it) -> int { return SMALL ? (int)(it & 1u) : 0; };
+  auto s_phase = [](uint32_t it) -> uint32_t { return SMALL ? ((it >> 1) & 1u) : (it & 1u); };
 
   if (tid == 0) {
     abort_flag[0] = 0;
     abort_flag[1] = 0;
-    mbar_init(bar(QK_FULL), 1);  mbar_init(bar(QK_FREE), 1 + kComputeWarps);
-    mbar_init(bar(S_FULL), 1);   mbar_init(bar(S_FREE), 1);
+    mbar_init(bar(QK_FULL), 1);  mbar_init(bar(QK_FREE), 1 + kComputeWarps + kSplitWarps);
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(bar(S_FULL0 + s), 1);
+      mbar_init(bar(S_CONV0 + s), kSplitWarps);
+      mbar_init(bar(S_FREE0 + s), 1);
+    }
     mbar_init(bar(V_FULL), 1);   mbar_init(bar(V_FREE), 1);
     mbar_init(bar(SC_DONE), 1);  mbar_init(bar(SC_FREE), kComputeWarps);
-    mbar_init(bar(QF_READY), kComputeWarps);
+    mbar_init(bar(QB_READY), kSplitWarps);
+    mbar_init(bar(QS_READY), kComputeWarps);
     mbar_init(bar(C_READY), kComputeWarps);
     mbar_init(bar(ACC_DONE0), 1); mbar_init(bar(ACC_DONE1), 1);
     mbar_init(bar(ACC_FREE0), kComputeWarps); mbar_init(bar(ACC_FREE1), kComputeWarps);
@@ -148,47 +276,43 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-
+  // registers: 128 per thread at launch; the compute warps take what the others give up
+  if (warp < kFirstComputeWarp) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
   if (warp == 0) {
     // ===================== TMA producer =====================
     if (lane == 0) {
-      int pend_qk = 0, pend_s = 0, pend_v = 0;
+      int pend_qk = 0, pend_v = 0, pend_s[2] = {0, 0};
       uint32_t it = 0;
       grid_dependency_wait();   // inputs may come from the kernel in front (dependent launch)
       for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++it) {
         const uint32_t ph = it & 1;
+        const int st = s_stage(it);
+        const ItemCoord ic = item_coord<PACKED>(p, item);
         if (!mbar_wait(bar(QK_FREE), ph ^ 1, abort_flag)) break;
-        // packed forest: boxes of 64 rows (per-request limit <= 64) or 128 rows at the request's offset
-        const uint32_t box_bytes = PACKED ? (T <= 64 ? kTile / 2 : kTile) : kTile;
-        int qk = 0, vplane = item, y0 = 0;
-        if constexpr (PACKED) {
-          const PackedItem pi = packed_item(p, item);
-          qk = pi.plane_qk; vplane = pi.plane_v; y0 = pi.row0;
-        } else {
-          qk = tv_qk_item(item, p.H, p.Hk);
-        }
-        mbar_expect_tx(bar(QK_FULL), 4 * box_bytes);
-        tma_load_3d(sbase + kOffQ, &tmQ, bar(QK_FULL), 0, y0, qk);
-        tma_load_3d(sbase + kOffQ + kTile, &tmQ, bar(QK_FULL), 64, y0, qk);
-        tma_load_3d(sbase + kOffK, &tmK, bar(QK_FULL), 0, y0, qk);
-        tma_load_3d(sbase + kOffK + kTile, &tmK, bar(QK_FULL), 64, y0, qk);
+        mbar_expect_tx(bar(QK_FULL), 4 * kBox);
+        load_box(sbase + L::kOffQ, &tmQ, bar(QK_FULL), nf_qk, 0, ic.y0, ic.h_qk, ic.z);
+        load_box(sbase + L::kOffQ + kBox, &tmQ, bar(QK_FULL), nf_qk, 64, ic.y0, ic.h_qk, ic.z);
+        load_box(sbase + L::kOffK, &tmK, bar(QK_FULL), nf_qk, 0, ic.y0, ic.h_qk, ic.z);
+        load_box(sbase + L::kOffK + kBox, &tmK, bar(QK_FULL), nf_qk, 64, ic.y0, ic.h_qk, ic.z);
         pend_qk = 1 + (int)ph;
-        if (!mbar_wait(bar(S_FREE), ph ^ 1, abort_flag)) break;
-        mbar_expect_tx(bar(S_FULL), 4 * kTile);
+        if (!mbar_wait(bar(S_FREE0 + st), s_phase(it) ^ 1, abort_flag)) break;
+        mbar_expect_tx(bar(S_FULL0 + st), 4 * kTile);
 #pragma unroll
         for (int c = 0; c < 4; ++c)
-          tma_load_3d(sbase + kOffS + c * kTile, &tmS, bar(S_FULL), 32 * c, 0, item);
-        pend_s = 1 + (int)ph;
+          tma_load_3d(sbase + L::kOffS + (uint32_t)(st * 4 + c) * kTile, &tmS, bar(S_FULL0 + st), 32 * c, 0, item);
+        pend_s[st] = 1 + (int)s_phase(it);
         if (!mbar_wait(bar(V_FREE), ph ^ 1, abort_flag)) break;
-        mbar_expect_tx(bar(V_FULL), 2 * box_bytes);
-        tma_load_3d(sbase + kOffV, &tmV, bar(V_FULL), 0, y0, vplane);
-        tma_load_3d(sbase + kOffV + kTile, &tmV, bar(V_FULL), 64, y0, vplane);
+        mbar_expect_tx(bar(V_FULL), 2 * kBox);
+        load_box(sbase + L::kOffV, &tmV, bar(V_FULL), nf_v, 0, ic.y0, ic.h_v, ic.z);
+        load_box(sbase + L::kOffV + kBox, &tmV, bar(V_FULL), nf_v, 64, ic.y0, ic.h_v, ic.z);
         pend_v = 1 + (int)ph;
       }
       if (*abort_flag) {
         // Leave no copy of ours in flight: wait (bounded) for the last loads issued.
         if (pend_qk) mbar_wait(bar(QK_FULL), pend_qk - 1, abort_flag + 1);
-        if (pend_s) mbar_wait(bar(S_FULL), pend_s - 1, abort_flag + 1);
+        for (int s = 0; s < 2; ++s)
+          if (pend_s[s]) mbar_wait(bar(S_FULL0 + s), pend_s[s] - 1, abort_flag + 1);
         if (pend_v) mbar_wait(bar(V_FULL), pend_v - 1, abort_flag + 1);
       }
     }
@@ -202,6 +326,7 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         const int acc_done = (it & 1) ? ACC_DONE1 : ACC_DONE0;
         const int acc_free = (it & 1) ? ACC_FREE1 : ACC_FREE0;
         const uint32_t ph2 = (it >> 1) & 1;   // the two accumulators alternate
+        const int st = s_stage(it);
         // scores = Q K^T
         if (!mbar_wait(bar(QK_FULL), ph, abort_flag)) break;
         if (!mbar_wait(bar(SC_FREE), ph ^ 1, abort_flag)) break;
@@ -210,22 +335,27 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         for (int h = 0; h < 2; ++h)
 #pragma unroll
           for (int s = 0; s < 4; ++s)
-            mma_bf16_ss(tmem + kColSc, desc_kmajor(sbase + kOffQ + h * kTile + s * 32),
-                        desc_kmajor(sbase + kOffK + h * kTile + s * 32), kIdescBf16KK, (h | s) != 0);
+            mma_bf16_ss(tmem + kColSc, desc_kmajor(sbase + L::kOffQ + h * kBox + s * 32),
+                        desc_kmajor(sbase + L::kOffK + h * kBox + s * 32), SMALL ? kIdescKK64 : kIdescKK128,
+                        (h | s) != 0);
         tc_commit(bar(SC_DONE));
         tc_commit(bar(QK_FREE));
-        // acc = (2^e Q) S_pre^T  (A = scaled Q as fp32 in TMEM, B = S_pre chunks)
-        if (!mbar_wait(bar(S_FULL), ph, abort_flag)) break;
-        if (!mbar_wait(bar(QF_READY), ph, abort_flag)) break;
+        // acc = (2^e Q) S_pre^T: A = scaled q rows (packed bf16 in TMEM), B = hi and lo tiles of S_pre
+        if (!mbar_wait(bar(S_CONV0 + st), s_phase(it), abort_flag)) break;
+        if (!mbar_wait(bar(QB_READY), ph, abort_flag)) break;
+        if (!mbar_wait(bar(QS_READY), ph, abort_flag)) break;
         if (!mbar_wait(bar(acc_free), ph2 ^ 1, abort_flag)) break;
         tc_fence_after();
 #pragma unroll
-        for (int c = 0; c < 4; ++c)
+        for (int kh = 0; kh < 2; ++kh)        // k half: 64 contraction indices
 #pragma unroll
-          for (int s = 0; s < 4; ++s)
-            mma_tf32_ts(tmem + acc_col, tmem + kColQf + c * 32 + s * 8,
-                        desc_kmajor(sbase + kOffS + c * kTile + s * 32), kIdescTf32, (c | s) != 0);
-        tc_commit(bar(S_FREE));
+          for (int part = 0; part < 2; ++part)   // hi, lo
+#pragma unroll
+            for (int s = 0; s < 4; ++s)
+              mma_bf16_ts(tmem + acc_col, tmem + kColQb + kh * 32 + s * 8,
+                          desc_kmajor(sbase + L::kOffS + (uint32_t)(st * 4 + kh * 2 + part) * kTile + s * 32),
+                          kIdescKK128, (kh | part | s) != 0);
+        tc_commit(bar(S_FREE0 + st));
         // acc += C'_hi V + C'_lo V
         if (!mbar_wait(bar(C_READY), ph, abort_flag)) break;
         if (!mbar_wait(bar(V_FULL), ph, abort_flag)) break;
@@ -233,32 +363,28 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         for (int jh = 0; jh < n_jh; ++jh)
 #pragma unroll
           for (int s = 0; s < 4; ++s) {
-            const uint64_t bdesc = desc_mnmajor(sbase + kOffV + (jh * 4 + s) * 2048, kTile);
-            mma_bf16_ss(tmem + acc_col, desc_kmajor(sbase + kOffChi + jh * kTile + s * 32), bdesc,
-                        kIdescBf16KMn, 1);
-            mma_bf16_ss(tmem + acc_col, desc_kmajor(sbase + kOffClo + jh * kTile + s * 32), bdesc,
-                        kIdescBf16KMn, 1);
+            const uint64_t bdesc = desc_mnmajor(sbase + L::kOffV + (jh * 4 + s) * 2048, kBox);
+            mma_bf16_ss(tmem + acc_col, desc_kmajor(sbase + L::kOffChi + jh * kTile + s * 32), bdesc,
+                        kIdescKMn, 1);
+            mma_bf16_ss(tmem + acc_col, desc_kmajor(sbase + L::kOffClo + jh * kTile + s * 32), bdesc,
+                        kIdescKMn, 1);
           }
         tc_commit(bar(V_FREE));
         tc_commit(bar(acc_done));
       }
     }
-  } else if (warp == kComputeWarps + 2) {
+  } else if (warp == 2) {
     // ===================== output stores =====================
     // The staged chunks of an item leave by TMA once all compute warps have written them
-    // (OST_READY); OST_FREE tells them that the chunks have been read.  T <= 64: the chunks are
+    // (OST_READY); OST_FREE tells them that the chunks have been read.  SMALL: the chunks are
     // not the C' tiles, and OST_FREE phase k says that the store of item k-1 is read (phase 0
-    // is given away up front).  T > 64: phase k = the store of item k.
+    // is given away up front).  Else: phase k = the store of item k.
     if (lane == 0) {
-      const bool small = T <= 64;
-      auto stage_addr = [&](int c4) -> uint32_t {
-        return small ? kOffChi + kTile + (uint32_t)(c4 >> 1) * (kOffClo - kOffChi) + (uint32_t)(c4 & 1) * 8192u
-                     : kOffChi + (uint32_t)c4 * kTile;
-      };
-      if (small) mbar_arrive(bar(OST_FREE));
+      if (SMALL) mbar_arrive(bar(OST_FREE));
       uint32_t it = 0;
       for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++it) {
         if (!mbar_wait(bar(OST_READY), it & 1, abort_flag)) break;
+        const ItemCoord ic = item_coord<PACKED>(p, item);
         if constexpr (PACKED) {
           // groups of 8 rows, largest boxes first; staging rows r.. start on a 1024-byte
           // boundary, so the swizzle phase of a partial box equals that of the full tile
@@ -269,7 +395,8 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             while (full - r >= rows_box) {
 #pragma unroll
               for (int c = 0; c < 4; ++c)
-                tma_store_3d(m, sbase + stage_addr(c) + (uint32_t)r * 128u, 32 * c, pk.row0 + r, pk.plane_v);
+                store_box(m, sbase + L::kOffStage + c * L::kStageChunk + (uint32_t)r * 128u, nf_o, 32 * c,
+                          ic.y0 + r, ic.h_v, ic.z);
               r += rows_box;
             }
           };
@@ -279,7 +406,8 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           put(&tmO8, 8);
         } else {
 #pragma unroll
-          for (int c = 0; c < 4; ++c) tma_store_3d(&tmO, sbase + stage_addr(c), 32 * c, 0, item);
+          for (int c = 0; c < 4; ++c)
+            store_box(&tmO, sbase + L::kOffStage + c * L::kStageChunk, nf_o, 32 * c, 0, ic.h_v, ic.z);
         }
         tma_store_commit();
         tma_store_wait_read();
@@ -287,35 +415,75 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       }
       tma_store_wait_all();   // our stores are complete before we leave
     }
+  }
+  } else if (warp >= kFirstSplitWarp) {
+    // ===================== state split =====================
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 112;");
+    const int row = tid - kFirstSplitWarp * 32;   // state row v, and node i for the q copy
+    const int pw = warp - kFirstSplitWarp;        // = TMEM lane window of this warp
+    const uint32_t lane_addr = (uint32_t)(pw * 32) << 16;
+    const uint32_t swz = (uint32_t)(row & 7);
+    uint32_t it = 0;
+    for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++it) {
+      const uint32_t ph = it & 1;
+      const int st = s_stage(it);
+      // ---- q rows (bf16, swizzled boxes) -> TMEM as they are: the A operand of the prefix MMA ----
+      if (!mbar_wait_warp(bar(QK_FULL), ph, abort_flag)) break;
+      // the prefix MMA of the item before is done with the copy in TMEM
+      if (it > 0 && !mbar_wait_warp(bar(S_FREE0 + s_stage(it - 1)), s_phase(it - 1), abort_flag)) break;
+      tc_fence_after();
+      if (pw * 32 < T) {
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          const unsigned char* qrow = sm + L::kOffQ + half * kBox + row * 128;
+          uint32_t r[32];
+#pragma unroll
+          for (int c = 0; c < 8; ++c) {
+            const uint4 x = *reinterpret_cast<const uint4*>(qrow + (((uint32_t)c ^ swz) << 4));
+            r[c * 4 + 0] = x.x; r[c * 4 + 1] = x.y; r[c * 4 + 2] = x.z; r[c * 4 + 3] = x.w;
+          }
+          tmem_st32(tmem + lane_addr + kColQb + half * 32, r);
+        }
+        tmem_wait_st();
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) {
+        mbar_arrive(bar(QB_READY));
+        mbar_arrive(bar(QK_FREE));
+      }
+      // ---- the state split ----
+      if (!mbar_wait_warp(bar(S_FULL0 + st), s_phase(it), abort_flag)) break;
+      unsigned char* s_buf = sm + L::kOffS + (uint32_t)st * 4u * kTile;
+      split_state_row(s_buf, row, 0, swz);
+      split_state_row(s_buf, row, 1, swz);
+      fence_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(S_CONV0 + st));
+    }
   } else {
     // ===================== compute warps =====================
-    const int cw = warp - 2;
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 168;");
+    const int cw = warp - kFirstComputeWarp;
     const int quad = warp & 3;          // TMEM lane window of this warp
     const int hc = cw >> 2;             // column half handled by this warp
-    const int row = quad * 32 + lane;   // node i
+    const int row = quad * 32 + lane;   // node i (and state row v in the split of S_pre)
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
     const uint32_t swz = (uint32_t)(row & 7);
     const bool warp_live = quad * 32 < T;   // this warp's 32 rows hold at least one node
 
-    // O_i = r_i acc_i for the item whose accumulator is `it_prev`: TMEM -> registers -> the
-    // (now idle) C' tiles as four [128 rows][32 fp32] swizzled tiles -> one TMA store per tile
-    // (full 128-byte lines; rows past T are clipped by the tensor map).
-    // T <= 64: the j >= 64 halves of the C' tiles are idle and hold the staging chunks
-    // ([64 rows][32 fp32], 8 KiB each), so staging never collides with the C' tiles of the
-    // next item and the store is only waited for one item later.  T > 64: the chunks are the
-    // four C' tiles themselves and the store must have read them before C' is rewritten.
-    const bool small = T <= 64;
-    auto stage_addr = [&](int c4) -> uint32_t {
-      return small ? kOffChi + kTile + (uint32_t)(c4 >> 1) * (kOffClo - kOffChi) + (uint32_t)(c4 & 1) * 8192u
-                   : kOffChi + (uint32_t)c4 * kTile;
-    };
-    auto final_epilogue = [&](uint32_t it_prev, int item_prev, float r_prev, uint32_t ost_phase,
-                              const PackedItem& pk_prev) -> bool {
+    // O_i = r_i acc_i for the item whose accumulator is `it_prev`: TMEM -> registers -> four
+    // [rows][32 fp32] swizzled staging chunks -> one TMA store per chunk (full 128-byte lines;
+    // rows past T are clipped by the tensor map).  SMALL: staging never collides with the C'
+    // tiles of the next item and the store is only waited for one item later.  Else: the
+    // chunks are the four C' tiles themselves and the store must have read them before C' is
+    // rewritten.
+    auto final_epilogue = [&](uint32_t it_prev, float r_prev, uint32_t ost_phase, const PackedItem& pk_prev) -> bool {
       const int acc_done = (it_prev & 1) ? ACC_DONE1 : ACC_DONE0;
       const int acc_free = (it_prev & 1) ? ACC_FREE1 : ACC_FREE0;
       const uint32_t acc_col = (it_prev & 1) ? kColAcc1 : kColAcc0;
-      // T <= 64: the store of the item before has read the staging chunks
-      if (small && !mbar_wait_warp(bar(OST_FREE), ost_phase, abort_flag)) return false;
+      // SMALL: the store of the item before has read the staging chunks
+      if (SMALL && !mbar_wait_warp(bar(OST_FREE), ost_phase, abort_flag)) return false;
       if (!mbar_wait_warp(bar(acc_done), (it_prev >> 1) & 1, abort_flag)) return false;
       tc_fence_after();
       if (warp_live) {
@@ -324,7 +492,7 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           uint32_t r1[32];
           tmem_ld32(tmem + lane_addr + acc_col + hc * 64 + half * 32, r1);
           tmem_wait_ld();
-          unsigned char* orow = sm + stage_addr(hc * 2 + half) + row * 128;
+          unsigned char* orow = sm + L::kOffStage + (hc * 2 + half) * L::kStageChunk + row * 128;
           // packed forest: the rows after the last full group of 8 leave from registers
           const bool tail_row = PACKED && row >= (pk_prev.n & ~7) && row < pk_prev.n;
           float* otail = nullptr;
@@ -349,7 +517,7 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         mbar_arrive(bar(acc_free));
         mbar_arrive(bar(OST_READY));
       }
-      return small ? true : mbar_wait_warp(bar(OST_FREE), ost_phase, abort_flag);
+      return SMALL ? true : mbar_wait_warp(bar(OST_FREE), ost_phase, abort_flag);
     };
 
     // metadata of the first item; later items are fetched one item ahead
@@ -369,24 +537,23 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           }
         }
       } else if (item < p.n_items && row < T) {
-        const int b = (item / p.H) % p.B;
-        const int tb = p.tree.n_trees == 1 ? 0 : b;
+        const int lb = item / p.H, h = item - lb * p.H;
+        const int tb = p.tree.n_trees == 1 ? 0 : lb % p.B;
         const uint64_t* m = p.tree.anc + ((size_t)tb * T + row) * 2;
         nm0 = m[0];
         nm1 = m[1];
-        nal = p.alpha[(size_t)item * T + row];
+        nal = p.alpha[(int64_t)lb * p.gate.b + (int64_t)h * p.gate.h + (int64_t)row * p.gate.t];
       }
     };
     // dependent launch: barrier set-up and the TMEM allocation above ran under the tail of the
     // kernel in front; everything that reads global memory waits for it here
     grid_dependency_wait();
     // the commit kernel behind this one may be scheduled as SMs drain (it orders itself)
-    if (warp == 2 && lane == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (warp == kFirstComputeWarp && lane == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     fetch_meta(blockIdx.x);
 
     uint32_t it = 0;
     bool ok = true;
-    int item_prev = 0;
     float r_prev = 0.f;
     PackedItem pk = npk, pk_prev = npk;
     const int total_rows = PACKED ? p.offsets[p.B] : 0;   // rows at and past this one hold no node
@@ -419,54 +586,56 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       if (lane == 0) range_ok_s[cw] = range_ok_warp;
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(SETUP));
-      // Row scaling.  The accumulator holds  2^e (q_i S_pre^T) + sum_j 2^(e - g_j) s_ij v_j  and
-      // O_i = 2^(g_i - e) acc: e is an integer, so the scaled q stays exact in tf32, and the
-      // exponents e - g_j = (e - g_i) + (g_i - g_j) stay small on ancestor pairs.  Below 2^-100
-      // the prefix term is under fp32 resolution of anything it is added to and is dropped.
-      const bool tiny = g < -100.f;
-      const float e_int = tiny ? g : fminf(rintf(g), 100.f);
+      if (!(ok = mbar_wait_warp(bar(SETUP), 1, abort_flag))) break;
+      bool fast = true;
+#pragma unroll
+      for (int w8 = 0; w8 < kComputeWarps; ++w8) fast = fast && range_ok_s[w8];
+      // Row scaling.  Plain form (every |g| <= 100): the accumulator holds  q_i S_pre^T +
+      // sum_j 2^(-g_j) s_ij v_j  and O_i = 2^(g_i) acc.  Extreme decay: a row exponent e =
+      // round(g_i) keeps every factor in range: the accumulator holds  2^e (q_i S_pre^T) +
+      // sum_j 2^(e - g_j) s_ij v_j  and O_i = 2^(g_i - e) acc; e is an integer, so the scaled q
+      // stays exact in bf16, and the exponents e - g_j = (e - g_i) + (g_i - g_j) stay small on
+      // ancestor pairs.  Below 2^-100 the prefix term is under fp32 resolution of anything it
+      // is added to and is dropped.
+      const bool tiny = !fast && g < -100.f;
+      const float e_int = fast ? 0.f : (tiny ? g : fminf(rintf(g), 100.f));
       const float a_scale = tiny ? 0.f : exp2f(e_int);
       const float r_scale = exp2f(g - e_int);
-      // ---- Q row (bf16, swizzled tile) -> scaled fp32 -> TMEM (A operand of the prefix MMA) ----
-      if (!(ok = mbar_wait_warp(bar(QK_FULL), ph, abort_flag))) break;
-      if (!(ok = mbar_wait_warp(bar(S_FREE), ph ^ 1, abort_flag))) break;   // prefix MMA of item-1 done with Qf
-      tc_fence_after();
-      if (warp_live) {
-        const unsigned char* qrow = sm + kOffQ + hc * kTile + row * 128;
-#pragma unroll
-        for (int half = 0; half < 2; ++half) {
+      // ---- scores of this item ----
+      // (Waited for before the arrival below: that arrival must not run an item ahead of the MMA
+      // issuer, which commits the scores of item n+1 only after it has consumed this one.)
+      if (!(ok = mbar_wait_warp(bar(SC_DONE), ph, abort_flag))) break;
+      if (!fast) {
+        // extreme decay: replace the q rows that the split warps copied to TMEM by scaled ones
+        if (!(ok = mbar_wait_warp(bar(QB_READY), ph, abort_flag))) break;
+        tc_fence_after();
+        if (warp_live) {
+          const unsigned char* qrow = sm + L::kOffQ + hc * kBox + row * 128;
           uint32_t r[32];
 #pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            const uint4 x = *reinterpret_cast<const uint4*>(qrow + (((half * 4 + c) ^ swz) << 4));
+          for (int c = 0; c < 8; ++c) {
+            const uint4 x = *reinterpret_cast<const uint4*>(qrow + (((uint32_t)c ^ swz) << 4));
             const uint32_t w[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              r[c * 8 + 2 * e] = __float_as_uint(a_scale * __uint_as_float(w[e] << 16));
-              r[c * 8 + 2 * e + 1] = __float_as_uint(a_scale * __uint_as_float(w[e] & 0xffff0000u));
-            }
+            for (int e = 0; e < 4; ++e)   // power-of-two scaling: the products are exact in bf16
+              r[c * 4 + e] = __byte_perm(__float_as_uint(a_scale * __uint_as_float(w[e] << 16)),
+                                         __float_as_uint(a_scale * __uint_as_float(w[e] & 0xffff0000u)), 0x7632);
           }
-          tmem_st32(tmem + lane_addr + kColQf + hc * 64 + half * 32, r);
+          tmem_st32(tmem + lane_addr + kColQb + hc * 32, r);
+          tmem_wait_st();
         }
-        tmem_wait_st();
+        tc_fence_before();
       }
-      tc_fence_before();
       __syncwarp();
       if (lane == 0) {
-        mbar_arrive(bar(QF_READY));
+        mbar_arrive(bar(QS_READY));
         mbar_arrive(bar(QK_FREE));
       }
-      // ---- scores -> masked, decayed, split C' ----
-      if (!(ok = mbar_wait_warp(bar(SC_DONE), ph, abort_flag))) break;
-      if (!(ok = mbar_wait_warp(bar(SETUP), 1, abort_flag))) break;
       // ---- output rows of the previous item: its accumulator is complete once its readout MMA
-      // is, and the C' tiles it frees double as the staging area of the output store ----
-      if (it > 0 && !(ok = final_epilogue(it - 1, item_prev, r_prev, (it - 1) & 1, pk_prev))) break;
+      // is, and (T > 64) the C' tiles it frees double as the staging area of the output store ----
+      if (it > 0 && !(ok = final_epilogue(it - 1, r_prev, (it - 1) & 1, pk_prev))) break;
       tc_fence_after();
       if (warp_live) {
-        bool fast = true;
-#pragma unroll
-        for (int w8 = 0; w8 < kComputeWarps; ++w8) fast = fast && range_ok_s[w8];
         // this warp covers 32 n_jh of the 64 n_jh real columns, 32 at a time
         for (int h = 0; h < n_jh; ++h) {
           const int cbase = hc * 32 * n_jh + h * 32;     // first column j of this group
@@ -474,8 +643,8 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           tmem_ld32(tmem + lane_addr + kColSc + cbase, r);
           tmem_wait_ld();
           const uint32_t bits = cbase < 64 ? (uint32_t)(m0 >> cbase) : (uint32_t)(m1 >> (cbase - 64));
-          unsigned char* chi = sm + kOffChi + (cbase >> 6) * kTile + row * 128;
-          unsigned char* clo = sm + kOffClo + (cbase >> 6) * kTile + row * 128;
+          unsigned char* chi = sm + L::kOffChi + (cbase >> 6) * kTile + row * 128;
+          unsigned char* clo = sm + L::kOffClo + (cbase >> 6) * kTile + row * 128;
           const int chunk0 = (cbase & 63) >> 3;
           if (fast) {
 #pragma unroll
@@ -486,7 +655,7 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
               float cv[8];
 #pragma unroll
               for (int e = 0; e < 8; ++e) {
-                const float x = __uint_as_float(r[c * 8 + e]) * (a_scale * f8[e]);
+                const float x = __uint_as_float(r[c * 8 + e]) * f8[e];
                 cv[e] = ((bits >> (c * 8 + e)) & 1u) ? x : 0.f;   // select, never 0 * x
               }
               store_split8(chi, clo, ((uint32_t)((chunk0 + c) ^ swz)) << 4, cv);
@@ -508,11 +677,10 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       if constexpr (PACKED) {
         // A box that reaches past the last node of the forest brings rows nobody wrote: zero them
         // in the V tiles (0 x garbage would not be 0); K and Q rows are masked by selection.
-        const int box_rows = T <= 64 ? 64 : 128;
-        if (pk.row0 + box_rows > total_rows) {
+        if (pk.row0 + kBoxRows > total_rows) {
           if (!(ok = mbar_wait_warp(bar(V_FULL), ph, abort_flag))) break;
-          if (row >= total_rows - pk.row0 && row < box_rows) {
-            uint4* vrow = reinterpret_cast<uint4*>(sm + kOffV + hc * kTile + row * 128);
+          if (row >= total_rows - pk.row0 && row < kBoxRows) {
+            uint4* vrow = reinterpret_cast<uint4*>(sm + L::kOffV + hc * kBox + row * 128);
 #pragma unroll
             for (int c = 0; c < 8; ++c) vrow[c] = make_uint4(0u, 0u, 0u, 0u);
           }
@@ -525,11 +693,10 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         mbar_arrive(bar(C_READY));
         mbar_arrive(bar(SC_FREE));
       }
-      item_prev = item;
       r_prev = r_scale;
       pk_prev = pk;
     }
-    if (ok && it > 0) final_epilogue(it - 1, item_prev, r_prev, (it - 1) & 1, pk_prev);
+    if (ok && it > 0) final_epilogue(it - 1, r_prev, (it - 1) & 1, pk_prev);
   }
 
   // ---- teardown: every path comes here ----
@@ -546,18 +713,28 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
 // ---------------------------------------------------------------------------
 // Host side: tensor maps and launch.
 // ---------------------------------------------------------------------------
-// Gated rule: the correction rows are the values themselves (U = V).
-__global__ void widen_bf16_kernel(const __nv_bfloat16* __restrict__ v, float* __restrict__ U, size_t n8) {
-  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n8; i += (size_t)gridDim.x * blockDim.x) {
-    const uint4 x = reinterpret_cast<const uint4*>(v)[i];
+// Gated rule: the correction rows are the values themselves (U = V), widened to float.  One
+// thread per 8 channels of a node row; rows addressed through the strides of v and of U.
+__global__ void widen_rows_kernel(const __nv_bfloat16* __restrict__ v, float* __restrict__ U, int n_lb, int H, int T,
+                                  Str3 sv, Str3 so) {
+  const size_t n = (size_t)n_lb * H * T * 16;
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+    const int c8 = (int)(i & 15);
+    size_t r = i >> 4;
+    const int t = (int)(r % T);
+    r /= T;
+    const int h = (int)(r % H);
+    const int64_t lb = (int64_t)(r / H);
+    const uint4 x = *reinterpret_cast<const uint4*>(v + lb * sv.b + h * sv.h + t * sv.t + c8 * 8);
     const uint32_t w[4] = {x.x, x.y, x.z, x.w};
     float4 a, b;
     a.x = __uint_as_float(w[0] << 16); a.y = __uint_as_float(w[0] & 0xffff0000u);
     a.z = __uint_as_float(w[1] << 16); a.w = __uint_as_float(w[1] & 0xffff0000u);
     b.x = __uint_as_float(w[2] << 16); b.y = __uint_as_float(w[2] & 0xffff0000u);
     b.z = __uint_as_float(w[3] << 16); b.w = __uint_as_float(w[3] & 0xffff0000u);
-    reinterpret_cast<float4*>(U)[2 * i] = a;
-    reinterpret_cast<float4*>(U)[2 * i + 1] = b;
+    float4* dst = reinterpret_cast<float4*>(U + lb * so.b + h * so.h + t * so.t + c8 * 8);
+    dst[0] = a;
+    dst[1] = b;
   }
 }
 
@@ -617,51 +794,56 @@ bool tv_verify_tc_supports(const VerifyArgs& a) {
 int tv_launch_verify_tc(const VerifyArgs& a, int32_t* status, cudaStream_t stream) {
   if (!tv_verify_tc_supports(a)) return TV_ERR_UNSUPPORTED;
   const bool packed = a.tree.offsets != nullptr;
+  const bool small = a.T <= 64;
   const uint64_t items = (uint64_t)a.L * a.B * a.H;
-  const uint64_t qk_items = (uint64_t)a.L * a.B * a.Hk;
-  const uint32_t orows = a.T <= 64 ? 64 : 128;   // rows of one staged output chunk
-  const void* const ptrs[5] = {a.q, a.k, a.v, a.S_pre, a.O};
-  const MapSet* ms = nullptr;
-  const MapSet* mo = nullptr;   // packed forest: output boxes of 32, 16 and 8 rows
+  const uint32_t rows = small ? 64 : 128;    // rows of an operand box and of a staged output chunk
+  // 4-D views: dense / strided layouts from the resolved strides, packed forests as planes
+  NodeView vq, vv, vo;
   if (!packed) {
-    ms = cached_maps(ptrs, items, a.T, a.Hk << 8, [&](CUtensorMap* m) {
-      return make_map(&m[0], a.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, qk_items, a.T, 128, 64) &&
-             make_map(&m[1], a.k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, qk_items, a.T, 128, 64) &&
-             make_map(&m[2], a.v, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, items, a.T, 128, 64) &&
-             make_map(&m[3], a.S_pre, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, 128, 128, 32) &&
-             make_map(&m[4], a.O, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, a.T, 128, 32, orows);
-    });
-    mo = ms;
+    const uint64_t lb = (uint64_t)a.L * a.B;
+    vq = NodeView{128, (uint64_t)a.T, (uint64_t)a.Hk, lb, a.lay.qk.b, a.lay.qk.h, a.lay.qk.t};
+    vv = NodeView{128, (uint64_t)a.T, (uint64_t)a.H, lb, a.lay.v.b, a.lay.v.h, a.lay.v.t};
+    vo = NodeView{128, (uint64_t)a.T, (uint64_t)a.H, lb, a.lay.out.b, a.lay.out.h, a.lay.out.t};
   } else {
-    // planes of `capacity` rows; loads in boxes of 64 or 128 rows, stores in boxes of 64/32/16/8
-    const uint64_t cap = (uint64_t)a.tree.capacity;
-    const uint64_t pv = (uint64_t)a.L * a.H, pqk = (uint64_t)a.L * a.Hk;
-    const uint32_t lrows = a.T <= 64 ? 64 : 128;
-    const uint64_t key = (cap << 24) ^ items;
-    ms = cached_maps(ptrs, key, a.T, 4 | (a.Hk << 8), [&](CUtensorMap* m) {
-      return make_map(&m[0], a.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, pqk, cap, 128, 64, lrows) &&
-             make_map(&m[1], a.k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, pqk, cap, 128, 64, lrows) &&
-             make_map(&m[2], a.v, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, pv, cap, 128, 64, lrows) &&
-             make_map(&m[3], a.S_pre, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, 128, 128, 32) &&
-             make_map(&m[4], a.O, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, pv, cap, 128, 32, 64);
-    });
+    const int64_t cap = a.tree.capacity;
+    vq = NodeView{128, (uint64_t)cap, (uint64_t)a.Hk, (uint64_t)a.L, (int64_t)a.Hk * cap * 128, cap * 128, 128};
+    vv = NodeView{128, (uint64_t)cap, (uint64_t)a.H, (uint64_t)a.L, (int64_t)a.H * cap * 128, cap * 128, 128};
+    vo = vv;
+  }
+  const void* const ptrs[5] = {a.q, a.k, a.v, a.S_pre, a.O};
+  const uint64_t key = view_key(vq) * 3 + view_key(vv) * 5 + view_key(vo) * 7 + items;
+  int node_first = 0;
+  const MapSet* ms = cached_maps(ptrs, key, a.T, (packed ? 4 : 0) | (a.Hk << 8), [&](CUtensorMap* m) {
+    return make_map4(&m[0], a.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, vq, 64, rows) &&
+           make_map4(&m[1], a.k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, vq, 64, rows) &&
+           make_map4(&m[2], a.v, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, vv, 64, rows) &&
+           make_map(&m[3], a.S_pre, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, 128, 128, 32) &&
+           make_map4(&m[4], a.O, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, vo, 32, packed ? 64 : rows);
+  });
+  const MapSet* mo = ms;   // packed forest: output boxes of 32, 16 and 8 rows
+  if (packed) {
     const void* const optrs[5] = {a.O, nullptr, nullptr, nullptr, nullptr};
     mo = cached_maps(optrs, key, a.T, 5, [&](CUtensorMap* m) {
-      return make_map(&m[0], a.O, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, pv, cap, 128, 32, 32) &&
-             make_map(&m[1], a.O, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, pv, cap, 128, 32, 16) &&
-             make_map(&m[2], a.O, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, pv, cap, 128, 32, 8);
+      return make_map4(&m[0], a.O, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, vo, 32, 32) &&
+             make_map4(&m[1], a.O, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, vo, 32, 16) &&
+             make_map4(&m[2], a.O, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, vo, 32, 8);
     });
   }
   if (!ms || !mo) return TV_ERR_CUDA;
+  node_first = (node_first_of(vq) ? 1 : 0) | (node_first_of(vv) ? 2 : 0) | (node_first_of(vo) ? 4 : 0);
   static thread_local int configured_dev = -1;
   static thread_local int sm_count = 0;
   int dev = 0;
   TV_CUDA_TRY(cudaGetDevice(&dev));
   if (configured_dev != dev) {
-    TV_CUDA_TRY(cudaFuncSetAttribute(verify_tc_gated_kernel<false>,
-                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
-    TV_CUDA_TRY(cudaFuncSetAttribute(verify_tc_gated_kernel<true>,
-                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
+    TV_CUDA_TRY(cudaFuncSetAttribute(verify_tc_gated_kernel<false, false>,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Lay<false>::kSmemBytes));
+    TV_CUDA_TRY(cudaFuncSetAttribute(verify_tc_gated_kernel<true, false>,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Lay<false>::kSmemBytes));
+    TV_CUDA_TRY(cudaFuncSetAttribute(verify_tc_gated_kernel<false, true>,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Lay<true>::kSmemBytes));
+    TV_CUDA_TRY(cudaFuncSetAttribute(verify_tc_gated_kernel<true, true>,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Lay<true>::kSmemBytes));
     TV_CUDA_TRY(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev));
     configured_dev = dev;
   }
@@ -670,15 +852,20 @@ int tv_launch_verify_tc(const VerifyArgs& a, int32_t* status, cudaStream_t strea
   p.n_items = (int32_t)items;
   p.B = a.B; p.H = a.H; p.T = a.T; p.Hk = a.Hk;
   p.alpha = a.alpha;
+  p.gate = a.lay.gate;
   p.O = a.O;
   p.status = status;
+  p.node_first = node_first;
   p.offsets = a.tree.offsets;
   p.capacity = a.tree.capacity;
   const int grid = (int)(items < (uint64_t)sm_count ? items : (uint64_t)sm_count);
+  const size_t smem = small ? Lay<true>::kSmemBytes : Lay<false>::kSmemBytes;
+  auto go = [&](auto kernel) {
+    return launch_dependent(kernel, grid, kThreads, smem, stream, ms->map[0], ms->map[1], ms->map[2], ms->map[3],
+                            ms->map[4], mo->map[packed ? 0 : 4], mo->map[packed ? 1 : 4], mo->map[packed ? 2 : 4], p);
+  };
   if (packed) {
-    TV_CUDA_TRY(launch_dependent(verify_tc_gated_kernel<true>, grid, kThreads, kSmemBytes, stream, ms->map[0],
-                                 ms->map[1], ms->map[2], ms->map[3], ms->map[4], mo->map[0], mo->map[1],
-                                 mo->map[2], p));
+    TV_CUDA_TRY(small ? go(verify_tc_gated_kernel<true, true>) : go(verify_tc_gated_kernel<true, false>));
     if (a.U) {
       const size_t planes = (size_t)a.L * a.H;
       widen_bf16_rows_kernel<<<dim3(64, (unsigned)(planes < 65535 ? planes : 65535)), 256, 0, stream>>>(
@@ -687,13 +874,12 @@ int tv_launch_verify_tc(const VerifyArgs& a, int32_t* status, cudaStream_t strea
     }
     return TV_OK;
   }
-  TV_CUDA_TRY(launch_dependent(verify_tc_gated_kernel<false>, grid, kThreads, kSmemBytes, stream, ms->map[0],
-                               ms->map[1], ms->map[2], ms->map[3], ms->map[4], ms->map[4], ms->map[4],
-                               ms->map[4], p));
+  TV_CUDA_TRY(small ? go(verify_tc_gated_kernel<false, true>) : go(verify_tc_gated_kernel<false, false>));
   if (a.U) {
-    const size_t n8 = items * a.T * 128 / 8;
-    const int blocks = (int)((n8 + 255) / 256 < 4096 ? (n8 + 255) / 256 : 4096);
-    widen_bf16_kernel<<<blocks, 256, 0, stream>>>(reinterpret_cast<const __nv_bfloat16*>(a.v), a.U, n8);
+    const size_t n = items * a.T * 16;
+    const int blocks = (int)((n + 255) / 256 < 4096 ? (n + 255) / 256 : 4096);
+    widen_rows_kernel<<<blocks, 256, 0, stream>>>(reinterpret_cast<const __nv_bfloat16*>(a.v), a.U, a.L * a.B, a.H,
+                                                  a.T, a.lay.v, a.lay.out);
     TV_CUDA_TRY(cudaGetLastError());
   }
   return TV_OK;

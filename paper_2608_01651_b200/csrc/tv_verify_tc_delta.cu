@@ -626,7 +626,7 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
 
 bool tv_verify_tc_delta_supports(const VerifyArgs& a) {
   return a.bf16 && a.dk == 128 && a.dv == 128 && a.rule == TV_GATED_DELTA && a.T <= kRows &&
-         a.tree.max_depth_all < kSlots;
+         a.tree.max_depth_all < kSlots && tv_layout_is_dense(a);
 }
 
 int tv_launch_verify_tc_delta(const VerifyArgs& a, int32_t* status, cudaStream_t stream) {

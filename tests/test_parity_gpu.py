@@ -189,3 +189,68 @@ def test_commit_many_units_per_cta(rule):
         dead = [b for b in range(wl.B) if accepted[b] < 0]
         assert dead, "the workload should reject some requests"
         assert np.array_equal(Sn[dead[0]], tens["S_pre"][dead[0]].double().numpy())
+
+
+def test_c5_all_48_layers_as_benchmarked():
+    """The throughput workload as stated: 48 recurrent layers back to back at full batch, head and
+    tree size -- 48 verify launches on one stream, then ONE in-place commit launch over all 48
+    layers (the persistent kernel, 393 216 units) -- in the launch configuration bench.py times.
+    Layers 0, 23 and 47 are compared with the oracle on sampled (request, head) items; the values
+    are drawn on the device and the oracle gets exactly what sits there."""
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()
+    free, _ = torch.cuda.mem_get_info()
+    if free < 56 * 2 ** 30:
+        pytest.skip("needs about 45 GiB of device memory")
+    wl = inputs.workload("c5")
+    assert wl.L == 48
+    dev = "cuda:0"
+    parents, accepted = inputs.make_trees(wl)
+    L, B, H, T = wl.L, wl.B, wl.H, wl.T
+    S = torch.empty(L, B, H, wl.dv, wl.dk, device=dev)
+    q = torch.empty(L, B, H, T, wl.dk, device=dev, dtype=torch.bfloat16)
+    k = torch.empty_like(q)
+    v = torch.empty(L, B, H, T, wl.dv, device=dev, dtype=torch.bfloat16)
+    al = torch.empty(L, B, H, T, device=dev)
+    O = torch.empty(L, B, H, T, wl.dv, device=dev)
+    for l in range(L):
+        t = inputs.make_tensors(wl, layer=l, device=dev)
+        S[l], q[l], k[l], v[l], al[l] = t["S_pre"], t["q"], t["k"], t["v"], t["alpha"]
+        del t
+    rng = np.random.default_rng(48)
+    layers = [0, 23, 47]
+    items = {l: [(0, 0), (B - 1, H - 1)] + [(int(rng.integers(B)), int(rng.integers(H))) for _ in range(8)]
+             for l in layers}
+    S0 = {(l, b, h): S[l, b, h].clone() for l in layers for (b, h) in items[l]}
+    tree = tv.tree_build(parents).upload()
+    acc = torch.from_numpy(accepted).to(dev)
+    for l in range(L):
+        tv.tree_verify(tree, S[l], q[l], k[l], v[l], al[l], O=O[l])
+    tv.commit_path(tree, acc, S, k, v, al)
+    torch.cuda.synchronize()
+    tree.device_status()
+    f = inputs.to_f64
+    worst_O = worst_S = 0.0
+    for l in layers:
+        for (b, h) in items[l]:
+            one = lambda x: f(x[l, b, h].cpu())[None, None]
+            S_hat = f(S0[(l, b, h)].cpu())[None, None]
+            par = parents[b][None]
+            Or, _ = orc_verify(S_hat, one(q), one(k), one(v), one(al), par)
+            Sr = orc_commit(S_hat, one(k), one(v), one(al), par, int(accepted[b]))
+            worst_O = max(worst_O, pu.rel_l2_rows(f(O[l, b, h].cpu()), Or))
+            worst_S = max(worst_S, pu.rel_fro(f(S[l, b, h].cpu()), Sr))
+    del S, q, k, v, al, O
+    torch.cuda.empty_cache()
+    assert worst_O <= wl.tol and worst_S <= wl.tol, (worst_O, worst_S)
+
+
+def orc_verify(S_hat, q, k, v, al, par):
+    from oracle import tree_oracle as orc
+    return orc.verify_batch(S_hat, q, k, v, al, None, par, "gated")[(0, 0)]
+
+
+def orc_commit(S_hat, k, v, al, par, a):
+    from oracle import tree_oracle as orc
+    return orc.commit_batch(S_hat, k, v, al, None, par, [a], "gated")[(0, 0)]
