@@ -611,8 +611,10 @@ def parity_check(rig, layers, n_items, seed=11):
             eU = max(eU, rel(f(st["U"][l, b, h].cpu()), Ur))
         Sn = f(st["S_pre"][l, b, h].cpu())
         eS = max(eS, float(np.linalg.norm(Sn - Sr) / max(np.linalg.norm(Sr), 1e-300)))
+    # O and S_new are what the bound is stated on; U is an internal factor whose rows shrink towards
+    # zero as the state converges (u = beta (v - S~^T k)), so its relative error is reported only
     return {"max_rel_l2_O": eO, "max_rel_l2_U": eU if st["U"] is not None else None, "max_rel_fro_S": eS,
-            "tol": wl.tol, "ok": bool(max(eO, eU, eS) <= wl.tol), "layers": list(layers), "items": len(items),
+            "tol": wl.tol, "ok": bool(max(eO, eS) <= wl.tol), "layers": list(layers), "items": len(items),
             "against": "fp64 oracle (per-node path walk) on the device-resident values, after the timed region"}
 
 

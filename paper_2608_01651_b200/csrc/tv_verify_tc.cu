@@ -5,26 +5,30 @@
 // (Theorem 1 / Eq. 4 with U = V):
 //
 //   scores  Sc = Q K^T                 bf16 x bf16 -> fp32 in TMEM (exact products)
-//   prefix  acc = (2^e_i q_i) S_pre^T  bf16 x bf16 -> fp32.  A operand: the q rows scaled by
-//                                      a power of two (exact in bf16), written to TMEM by the
-//                                      compute warps.  B operand: S_pre split into bf16
+//   prefix  acc = q_i S_pre^T          bf16 x bf16 -> fp32.  A operand: the q rows, copied to TMEM
+//                                      as packed bf16.  B operand: S_pre split into bf16
 //                                      hi + lo (16 mantissa bits, both rounded to nearest)
 //                                      IN PLACE in the buffer the TMA filled: the fp32 row
 //                                      halves k 0..31 | 32..63 of a state row become its hi row
 //                                      and its lo row of 64 bf16 -- same bytes, same swizzle.
-//   C'_ij   = 1[j in Anc(i)+{i}] exp2(e_i - g_j) Sc_ij,  g = sum log2(alpha)
-//             over the path, e_i = round(g_i) (decay ratios only ever taken on
-//             ancestor pairs), split into bf16 hi + lo
+//   C'_ij   = 1[j in Anc(i)+{i}] 2^(-g_j) Sc_ij,  g = sum log2(alpha) over the path (decay
+//             ratios only ever taken on ancestor pairs), split into bf16 hi + lo
 //   readout acc += C'_hi V + C'_lo V   bf16 x bf16 -> fp32, same accumulator
-//   O_i     = exp2(g_i - e_i) acc_i    fp32 epilogue
+//   O_i     = 2^(g_i) acc_i            fp32 epilogue
 // The accumulator is double-buffered in TMEM: the epilogue of item n runs under
 // the MMAs of item n+1.
+//
+// Extreme decay.  The plain form above is used as long as every |g| <= 100.  Otherwise a row
+// exponent e_i = round(g_i) keeps every factor in range: the compute warps replace the q rows
+// in TMEM by 2^e_i q_i (exact in bf16), C'_ij = 2^(e_i - g_j) Sc_ij, O_i = 2^(g_i - e_i) acc;
+// rows with g_i < -100 drop the prefix term, which is below fp32 resolution of anything it is
+// added to.
 //
 // Why the state is split rather than fed to the tensor core as fp32 (kind::tf32 cuts the
 // mantissa to 10 bits): a state that has absorbed many rank-one updates is dominated by a
 // few directions, a query nearly orthogonal to them sums large terms that cancel, and the
 // tf32 cut of those terms reached 1e-2 of the output in such states (5e-4 on unstructured
-// ones).  The split keeps 16 bits (worst case seen 4e-4, typically 1e-5), costs half the
+// ones).  The split keeps 16 bits (worst case seen 4e-4, typically 1e-5), costs the
 // tensor time of the tf32 product, and needs no extra shared memory.
 //
 // T <= 64 (SMALL): operand boxes of 64 rows, and the shared memory that frees holds a second
@@ -32,14 +36,17 @@
 // item n is worked on.  T > 64: one stage of everything.
 //
 // Warp roles, in groups of four warps so that registers can be moved between them
-// (setmaxnreg): warp 0 = TMA producer, warp 1 = MMA issuer (owns TMEM), warp 2 = issues the
-// output stores (warp 3 idle), 56 registers each; warps 4..11 = 8 compute warps, 168
-// registers: compute warp w reads TMEM lanes 32 (w % 4) .. +31 (the hardware's lane window of
-// that warp) and half of the columns; warps 12..15 = the state split, 112 registers: they see
-// a state stage land, rewrite it and hand it to the MMA issuer, so that the compute warps'
-// chain of epilogues never waits on the state stream.  Every wait is an mbarrier wait with a
-// time limit; on expiry the CTA sets the status word, drains its own copies and leaves (TMEM
-// is freed on every path).
+// (setmaxnreg).  The chain that paces an item is that of the compute warps; what depends on
+// loaded data only is taken off it.
+//   warps 0..3   service, 64 registers: 0 = TMA producer, 1 = MMA issuer (owns TMEM),
+//                2 = issues the output stores, 3 idle
+//   warps 4..11  compute, 168 registers: path decay, C' from the scores, O from the
+//                accumulator; warp w reads TMEM lanes 32 (w % 4) .. +31 (the hardware's lane
+//                window of that warp) and half of the columns
+//   warps 12..15 operands, 104 registers, thread r = node r = state row r: the q rows into TMEM,
+//                the split of S_pre
+// Every wait is an mbarrier wait with a time limit; on expiry the CTA sets the status word,
+// drains its own copies and leaves (TMEM is freed on every path).
 #include "tv_tc_common.cuh"
 
 namespace {
@@ -181,9 +188,20 @@ __device__ __forceinline__ PackedItem packed_item(const TcParams& p, int item) {
   return tvtc::packed_item(p.offsets, p.B, p.H, p.Hk, item);
 }
 
-// Coordinates of an item's boxes: (head, outermost) of q/k and of v/O, and the first node row.
+// Load boxes of q, k, v in three heights: the full box (64 or 128 rows), half and a quarter of it.
+// A packed forest takes, per request, the smallest that holds its nodes (Section V-B: only the
+// tiles inside a request are moved); dense trees always take the full one.
+struct LoadMaps {
+  CUtensorMap q[3], k[3], v[3];   // [0] quarter, [1] half, [2] full
+};
+__device__ __forceinline__ int box_class(int n, int full_rows) {
+  return n * 4 <= full_rows ? 0 : n * 2 <= full_rows ? 1 : 2;
+}
+
+// Coordinates of an item's boxes: (head, outermost) of q/k and of v/O, the first node row, and
+// (packed forest) the request's node count.
 struct ItemCoord {
-  int h_qk, h_v, z, y0;
+  int h_qk, h_v, z, y0, n;
 };
 template <bool PACKED>
 __device__ __forceinline__ ItemCoord item_coord(const TcParams& p, int item) {
@@ -195,9 +213,11 @@ __device__ __forceinline__ ItemCoord item_coord(const TcParams& p, int item) {
     const int l = lb / p.B, b = lb - l * p.B;
     c.z = l;
     c.y0 = p.offsets[b];
+    c.n = p.offsets[b + 1] - c.y0;
   } else {
     c.z = lb;
     c.y0 = 0;
+    c.n = p.T;
   }
   return c;
 }
@@ -219,8 +239,7 @@ __device__ __forceinline__ void store_box(const CUtensorMap* m, uint32_t src, bo
 // rows straight from registers.  The dense instantiation ignores the three extra maps.
 template <bool PACKED, bool SMALL>
 __global__ void __launch_bounds__(kThreads, 1)
-verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                       const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmS,
+verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constant__ CUtensorMap tmS,
                        const __grid_constant__ CUtensorMap tmO, const __grid_constant__ CUtensorMap tmO32,
                        const __grid_constant__ CUtensorMap tmO16, const __grid_constant__ CUtensorMap tmO8,
                        const TcParams p) {
@@ -272,13 +291,20 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                  ::"r"(smem_u32(tmem_slot)), "r"(512u) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
+  if constexpr (PACKED) {
+    // V rows below a request's box keep what earlier items left there and only ever meet zero
+    // coefficients; before the first item they must not hold NaN patterns (0 x NaN is not 0)
+    for (uint32_t o = (uint32_t)tid * 16u; o < 2 * kBox; o += kThreads * 16u)
+      *reinterpret_cast<uint4*>(sm + L::kOffV + o) = make_uint4(0u, 0u, 0u, 0u);
+    fence_async_smem();
+  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
   // registers: 128 per thread at launch; the compute warps take what the others give up
   if (warp < kFirstComputeWarp) {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");
   if (warp == 0) {
     // ===================== TMA producer =====================
     if (lane == 0) {
@@ -290,11 +316,14 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         const int st = s_stage(it);
         const ItemCoord ic = item_coord<PACKED>(p, item);
         if (!mbar_wait(bar(QK_FREE), ph ^ 1, abort_flag)) break;
-        mbar_expect_tx(bar(QK_FULL), 4 * kBox);
-        load_box(sbase + L::kOffQ, &tmQ, bar(QK_FULL), nf_qk, 0, ic.y0, ic.h_qk, ic.z);
-        load_box(sbase + L::kOffQ + kBox, &tmQ, bar(QK_FULL), nf_qk, 64, ic.y0, ic.h_qk, ic.z);
-        load_box(sbase + L::kOffK, &tmK, bar(QK_FULL), nf_qk, 0, ic.y0, ic.h_qk, ic.z);
-        load_box(sbase + L::kOffK + kBox, &tmK, bar(QK_FULL), nf_qk, 64, ic.y0, ic.h_qk, ic.z);
+        // rows of the boxes of this item (the tile layout in shared memory does not depend on it)
+        const int bc = PACKED ? box_class(ic.n, kBoxRows) : 2;
+        const uint32_t box_bytes = kBox >> (2 - bc);
+        mbar_expect_tx(bar(QK_FULL), 4 * box_bytes);
+        load_box(sbase + L::kOffQ, &lm.q[bc], bar(QK_FULL), nf_qk, 0, ic.y0, ic.h_qk, ic.z);
+        load_box(sbase + L::kOffQ + kBox, &lm.q[bc], bar(QK_FULL), nf_qk, 64, ic.y0, ic.h_qk, ic.z);
+        load_box(sbase + L::kOffK, &lm.k[bc], bar(QK_FULL), nf_qk, 0, ic.y0, ic.h_qk, ic.z);
+        load_box(sbase + L::kOffK + kBox, &lm.k[bc], bar(QK_FULL), nf_qk, 64, ic.y0, ic.h_qk, ic.z);
         pend_qk = 1 + (int)ph;
         if (!mbar_wait(bar(S_FREE0 + st), s_phase(it) ^ 1, abort_flag)) break;
         mbar_expect_tx(bar(S_FULL0 + st), 4 * kTile);
@@ -303,9 +332,9 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           tma_load_3d(sbase + L::kOffS + (uint32_t)(st * 4 + c) * kTile, &tmS, bar(S_FULL0 + st), 32 * c, 0, item);
         pend_s[st] = 1 + (int)s_phase(it);
         if (!mbar_wait(bar(V_FREE), ph ^ 1, abort_flag)) break;
-        mbar_expect_tx(bar(V_FULL), 2 * kBox);
-        load_box(sbase + L::kOffV, &tmV, bar(V_FULL), nf_v, 0, ic.y0, ic.h_v, ic.z);
-        load_box(sbase + L::kOffV + kBox, &tmV, bar(V_FULL), nf_v, 64, ic.y0, ic.h_v, ic.z);
+        mbar_expect_tx(bar(V_FULL), 2 * box_bytes);
+        load_box(sbase + L::kOffV, &lm.v[bc], bar(V_FULL), nf_v, 0, ic.y0, ic.h_v, ic.z);
+        load_box(sbase + L::kOffV + kBox, &lm.v[bc], bar(V_FULL), nf_v, 64, ic.y0, ic.h_v, ic.z);
         pend_v = 1 + (int)ph;
       }
       if (*abort_flag) {
@@ -418,7 +447,7 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   }
   } else if (warp >= kFirstSplitWarp) {
     // ===================== state split =====================
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 112;");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 104;");
     const int row = tid - kFirstSplitWarp * 32;   // state row v, and node i for the q copy
     const int pw = warp - kFirstSplitWarp;        // = TMEM lane window of this warp
     const uint32_t lane_addr = (uint32_t)(pw * 32) << 16;
@@ -677,9 +706,10 @@ verify_tc_gated_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       if constexpr (PACKED) {
         // A box that reaches past the last node of the forest brings rows nobody wrote: zero them
         // in the V tiles (0 x garbage would not be 0); K and Q rows are masked by selection.
-        if (pk.row0 + kBoxRows > total_rows) {
+        const int rows_loaded = kBoxRows >> (2 - box_class(pk.n, kBoxRows));
+        if (pk.row0 + rows_loaded > total_rows) {
           if (!(ok = mbar_wait_warp(bar(V_FULL), ph, abort_flag))) break;
-          if (row >= total_rows - pk.row0 && row < kBoxRows) {
+          if (row >= total_rows - pk.row0 && row < rows_loaded) {
             uint4* vrow = reinterpret_cast<uint4*>(sm + L::kOffV + hc * kBox + row * 128);
 #pragma unroll
             for (int c = 0; c < 8; ++c) vrow[c] = make_uint4(0u, 0u, 0u, 0u);
@@ -829,7 +859,27 @@ int tv_launch_verify_tc(const VerifyArgs& a, int32_t* status, cudaStream_t strea
              make_map4(&m[2], a.O, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, vo, 32, 8);
     });
   }
-  if (!ms || !mo) return TV_ERR_CUDA;
+  // packed forest: q, k, v boxes of half and a quarter of the full height
+  const MapSet* mh[2] = {ms, ms};
+  if (packed) {
+    for (int c = 0; c < 2; ++c) {
+      const uint32_t r = rows >> (2 - c);
+      const void* const lptrs[5] = {a.q, a.k, a.v, nullptr, nullptr};
+      mh[c] = cached_maps(lptrs, key, a.T, 6 + c, [&](CUtensorMap* m) {
+        return make_map4(&m[0], a.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, vq, 64, r) &&
+               make_map4(&m[1], a.k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, vq, 64, r) &&
+               make_map4(&m[2], a.v, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, vv, 64, r);
+      });
+    }
+  }
+  if (!ms || !mo || !mh[0] || !mh[1]) return TV_ERR_CUDA;
+  LoadMaps lm;
+  for (int c = 0; c < 3; ++c) {
+    const MapSet* src = c == 2 ? ms : mh[c];
+    lm.q[c] = src->map[0];
+    lm.k[c] = src->map[1];
+    lm.v[c] = src->map[2];
+  }
   node_first = (node_first_of(vq) ? 1 : 0) | (node_first_of(vv) ? 2 : 0) | (node_first_of(vo) ? 4 : 0);
   static thread_local int configured_dev = -1;
   static thread_local int sm_count = 0;
@@ -861,8 +911,7 @@ int tv_launch_verify_tc(const VerifyArgs& a, int32_t* status, cudaStream_t strea
   const int grid = (int)(items < (uint64_t)sm_count ? items : (uint64_t)sm_count);
   const size_t smem = small ? Lay<true>::kSmemBytes : Lay<false>::kSmemBytes;
   auto go = [&](auto kernel) {
-    return launch_dependent(kernel, grid, kThreads, smem, stream, ms->map[0], ms->map[1], ms->map[2], ms->map[3],
-                            ms->map[4], mo->map[packed ? 0 : 4], mo->map[packed ? 1 : 4], mo->map[packed ? 2 : 4], p);
+    return launch_dependent(kernel, grid, kThreads, smem, stream, lm, ms->map[3], ms->map[4], mo->map[packed ? 0 : 4], mo->map[packed ? 1 : 4], mo->map[packed ? 2 : 4], p);
   };
   if (packed) {
     TV_CUDA_TRY(small ? go(verify_tc_gated_kernel<true, true>) : go(verify_tc_gated_kernel<true, false>));
