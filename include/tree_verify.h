@@ -158,7 +158,9 @@ int tv_tree_meta_device(tv_tree* tree, uint64_t* anc, int32_t* depth, void* stre
  * core completion that never came): TV_OK or TV_ERR_DEVICE_TIMEOUT.  After a
  * timeout the outputs of that launch are undefined; the context stays usable.
  * TV_ERR_UNSUPPORTED: the trees of the last tv_forest_upload_device were deeper
- * than the bound that call was given.                                         */
+ * than the bound that call was given.  TV_ERR_CUDA: a tensor-core kernel found
+ * its shared-memory window off the 1024-byte boundary its tiles need and left
+ * without computing (outputs undefined, as after a timeout).                  */
 int tv_tree_device_status(tv_tree* tree, void* stream);
 /* Self-test of that mechanism: launches one CTA that waits, with a limit of a
  * few milliseconds, on a barrier nothing ever signals, and writes what the

@@ -347,6 +347,7 @@ TV_API int tv_tree_device_status(tv_tree* t, void* stream) {
   int32_t st[2] = {0, 0};
   TV_CUDA_TRY(cudaMemcpyAsync(st, t->d_status, sizeof(st), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
   TV_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+  if (st[0] == TV_ERR_CUDA) return TV_ERR_CUDA;   // a kernel refused its shared-memory window
   if (st[0] != 0) return TV_ERR_DEVICE_TIMEOUT;
   if (st[1] != 0 && st[1] == t->upload_gen) return TV_ERR_UNSUPPORTED;   // trees deeper than the stated bound
   return TV_OK;

@@ -46,21 +46,26 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-// Bounded wait.  Returns false when the limit ran out or another role gave up.
+// Bounded wait.  Returns false when the limit ran out or another role gave up.  Kept short (32-bit
+// clock, one exit for both reasons): a kernel has dozens of these, all inlined, and their code
+// competes with the working loops for the instruction cache.  The clock is first read after
+// 1024 failed tries and then every 1024; `limit` is cut to 2^31 cycles.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                           long long limit = kWaitLimitCycles) {
-  if (mbar_try(bar, parity)) return true;
-  const long long t0 = clock64();
-  for (uint32_t spin = 1;; ++spin) {
-    if (mbar_try(bar, parity)) return true;
-    if ((spin & 1023u) == 0) {
-      if (*abort_flag) return false;
-      if (clock64() - t0 > limit) {
+  const uint32_t limit32 = limit > (long long)0x7fffffff ? 0x7fffffffu : (uint32_t)limit;
+  uint32_t spin = 0, t0 = 0;
+  while (!mbar_try(bar, parity)) {
+    if ((++spin & 1023u) == 0) {
+      const uint32_t now = (uint32_t)clock();
+      if (spin == 1024u) {
+        t0 = now;
+      } else if (*abort_flag || now - t0 > limit32) {
         *abort_flag = 1;
         return false;
       }
     }
   }
+  return true;
 }
 
 // Same for a whole warp: every lane gets the same answer, so that the warp never
@@ -239,6 +244,23 @@ inline bool make_map4(CUtensorMap* map, const void* base, CUtensorMapDataType dt
 
 // (layer, request, head) of a work item and, for a packed forest, where its rows live: request b
 // owns rows offsets[b] .. offsets[b+1]-1 of every (layer, head) plane.
+// Division by a launch constant: quotient = (mulhi(n, mul) + n) >> sh for every n < 2^31
+// (round-up method; sh = ceil(log2 d)).  The persistent kernels turn item numbers into
+// (layer, request, head) in several roles; the generic 32-bit division is some twenty
+// instructions at every one of those places.
+struct FastDiv {
+  uint32_t d, mul, sh;
+};
+inline FastDiv make_fastdiv(uint32_t d) {
+  FastDiv f;
+  f.d = d;
+  f.sh = 0;
+  while ((1ull << f.sh) < d) ++f.sh;
+  f.mul = (uint32_t)((((1ull << f.sh) - d) << 32) / d + 1);
+  return f;
+}
+__device__ __forceinline__ uint32_t fdiv(uint32_t n, const FastDiv& f) { return (__umulhi(n, f.mul) + n) >> f.sh; }
+
 struct PackedItem {
   int b, plane_v, plane_qk, row0, n;
 };

@@ -77,22 +77,29 @@ struct Lay {
   // four C' tiles themselves, idle once the readout MMAs of the item are complete
   static constexpr uint32_t kOffStage = SMALL ? kOffClo + kBox : kOffChi;
   static constexpr uint32_t kStageChunk = SMALL ? kTile / 2 : kTile;
-  static constexpr uint32_t kOffG = SMALL ? kOffStage + 4 * kStageChunk : kOffClo + 2 * kTile;   // float g[128]
-  static constexpr uint32_t kOffAl = kOffG + 512;          // float log2(alpha)[128]
-  static constexpr uint32_t kOffF = kOffAl + 512;          // float exp2(-g)[128]
-  static constexpr uint32_t kOffBar = kOffF + 512;         // mbarriers
-  static constexpr uint32_t kOffMisc = kOffBar + 8 * 24;   // tmem base, abort flags, per-warp range flags
-  static constexpr uint32_t kSmemBytes = kOffMisc + 48 + 1024;  // + alignment slack
+  // path decay of two items in flight: g[2][kNodes], exp2(-g)[2][kNodes]; log2(alpha)[kNodes] is
+  // the decay warp's own scratch
+  static constexpr uint32_t kNodes = SMALL ? 64 : 128;
+  static constexpr uint32_t kOffG = SMALL ? kOffStage + 4 * kStageChunk : kOffClo + 2 * kTile;
+  static constexpr uint32_t kOffF = kOffG + 2 * kNodes * 4;
+  static constexpr uint32_t kOffAl = kOffF + 2 * kNodes * 4;
+  static constexpr uint32_t kOffBar = kOffAl + kNodes * 4;   // mbarriers
+  static constexpr uint32_t kOffMisc = kOffBar + 8 * 32;     // tmem base, abort flags, range flags of two items
+  // The dynamic shared memory of a CTA starts on a 1024-byte boundary (asked for in the
+  // declaration and checked at entry), so there is no alignment slack in this figure.
+  static constexpr uint32_t kSmemBytes = kOffMisc + 32;
+  static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
 };
 
 enum Bar {
   QK_FULL = 0, QK_FREE, S_FULL0, S_FULL1, S_CONV0, S_CONV1, S_FREE0, S_FREE1, V_FULL, V_FREE,
-  SC_DONE, SC_FREE, QB_READY, QS_READY, C_READY, ACC_DONE0, ACC_DONE1, ACC_FREE0, ACC_FREE1, SETUP,
-  OST_READY, OST_FREE, kNumBars
+  SC_DONE, SC_FREE, QB_READY0, QB_READY1, QS_READY0, QS_READY1, C_READY, ACC_DONE0, ACC_DONE1, ACC_FREE0, ACC_FREE1,
+  META_READY0, META_READY1, META_FREE0, META_FREE1, OST_READY, OST_FREE, kNumBars
 };
-static_assert(kNumBars <= 24, "barrier area");
+static_assert(kNumBars <= 32, "barrier area");
 
-// TMEM columns: scaled Q as packed bf16 (A operand of the prefix MMA), scores, two accumulators
+// TMEM columns: Q as packed bf16 (A operand of the prefix MMA; two copies of 64 columns, items
+// alternate), scores, two accumulators
 constexpr uint32_t kColQb = 0, kColSc = 128, kColAcc0 = 256, kColAcc1 = 384;
 
 constexpr uint32_t kIdescKK128 = idesc_bf16(128, false);
@@ -182,10 +189,19 @@ struct TcParams {
   // `capacity` rows; T is then the per-request node limit (width of the metadata slabs)
   const int32_t* offsets;
   int32_t capacity;
+  FastDiv dH, dB, dG;   // division by H, by B, by the q/k group size H / Hk
 };
 
 __device__ __forceinline__ PackedItem packed_item(const TcParams& p, int item) {
-  return tvtc::packed_item(p.offsets, p.B, p.H, p.Hk, item);
+  PackedItem r;
+  const int lb = (int)fdiv((uint32_t)item, p.dH), h = item - lb * p.H;
+  const int l = (int)fdiv((uint32_t)lb, p.dB);
+  r.b = lb - l * p.B;
+  r.plane_v = l * p.H + h;
+  r.plane_qk = l * p.Hk + (int)fdiv((uint32_t)h, p.dG);
+  r.row0 = p.offsets[r.b];
+  r.n = p.offsets[r.b + 1] - r.row0;
+  return r;
 }
 
 // Load boxes of q, k, v in three heights: the full box (64 or 128 rows), half and a quarter of it.
@@ -206,11 +222,11 @@ struct ItemCoord {
 template <bool PACKED>
 __device__ __forceinline__ ItemCoord item_coord(const TcParams& p, int item) {
   ItemCoord c;
-  const int lb = item / p.H, h = item - lb * p.H;
+  const int lb = (int)fdiv((uint32_t)item, p.dH), h = item - lb * p.H;
   c.h_v = h;
-  c.h_qk = p.Hk == p.H ? h : h / (p.H / p.Hk);
+  c.h_qk = (int)fdiv((uint32_t)h, p.dG);
   if constexpr (PACKED) {
-    const int l = lb / p.B, b = lb - l * p.B;
+    const int l = (int)fdiv((uint32_t)lb, p.dB), b = lb - l * p.B;
     c.z = l;
     c.y0 = p.offsets[b];
     c.n = p.offsets[b + 1] - c.y0;
@@ -246,13 +262,18 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
   using L = Lay<SMALL>;
   constexpr uint32_t kBox = L::kBox;
   constexpr int kBoxRows = SMALL ? 64 : 128;
-  extern __shared__ unsigned char smem_raw[];
-  unsigned char* sm = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  unsigned char* sm = smem_raw;
   const uint32_t sbase = smem_u32(sm);
-  float* g_s = reinterpret_cast<float*>(sm + L::kOffG);
-  float* la_s = reinterpret_cast<float*>(sm + L::kOffAl);
-  float* f_s = reinterpret_cast<float*>(sm + L::kOffF);
-  volatile int* range_ok_s = reinterpret_cast<volatile int*>(sm + L::kOffMisc + 16);   // [8] per compute warp
+  if (sbase & 1023u) {   // the swizzled tiles need this alignment; refuse rather than compute garbage
+    if (threadIdx.x == 0 && p.status) atomicExch(p.status, (int)TV_ERR_CUDA);
+    return;
+  }
+  constexpr int kNodes = (int)L::kNodes;
+  float* g_s = reinterpret_cast<float*>(sm + L::kOffG);     // [2][kNodes]
+  float* f_s = reinterpret_cast<float*>(sm + L::kOffF);     // [2][kNodes]
+  float* la_s = reinterpret_cast<float*>(sm + L::kOffAl);   // [kNodes], decay warp only
+  volatile int* fast_s = reinterpret_cast<volatile int*>(sm + L::kOffMisc + 16);   // [2]: every |g| <= 100
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + L::kOffMisc);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + L::kOffMisc + 4);
   auto bar = [&](int i) { return sbase + L::kOffBar + 8u * i; };
@@ -268,7 +289,7 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
   if (tid == 0) {
     abort_flag[0] = 0;
     abort_flag[1] = 0;
-    mbar_init(bar(QK_FULL), 1);  mbar_init(bar(QK_FREE), 1 + kComputeWarps + kSplitWarps);
+    mbar_init(bar(QK_FULL), 1);  mbar_init(bar(QK_FREE), 1 + kSplitWarps);
     for (int s = 0; s < 2; ++s) {
       mbar_init(bar(S_FULL0 + s), 1);
       mbar_init(bar(S_CONV0 + s), kSplitWarps);
@@ -276,12 +297,17 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
     }
     mbar_init(bar(V_FULL), 1);   mbar_init(bar(V_FREE), 1);
     mbar_init(bar(SC_DONE), 1);  mbar_init(bar(SC_FREE), kComputeWarps);
-    mbar_init(bar(QB_READY), kSplitWarps);
-    mbar_init(bar(QS_READY), kComputeWarps);
+    mbar_init(bar(QB_READY0), kSplitWarps);
+    mbar_init(bar(QB_READY1), kSplitWarps);
+    mbar_init(bar(QS_READY0), kComputeWarps);
+    mbar_init(bar(QS_READY1), kComputeWarps);
     mbar_init(bar(C_READY), kComputeWarps);
     mbar_init(bar(ACC_DONE0), 1); mbar_init(bar(ACC_DONE1), 1);
     mbar_init(bar(ACC_FREE0), kComputeWarps); mbar_init(bar(ACC_FREE1), kComputeWarps);
-    mbar_init(bar(SETUP), kComputeWarps);
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(bar(META_READY0 + s), 1);
+      mbar_init(bar(META_FREE0 + s), kComputeWarps + 1);   // + the MMA issuer
+    }
     mbar_init(bar(OST_READY), kComputeWarps);
     mbar_init(bar(OST_FREE), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -307,99 +333,135 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
     asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");
   if (warp == 0) {
     // ===================== TMA producer =====================
+    // Three independent load streams (q+k, v, S_pre), each in item order and each gated by the
+    // barrier that says its buffer is free.  One thread polls the three gates and issues
+    // whatever is ready, so that no stream waits for another one's buffer.
     if (lane == 0) {
       int pend_qk = 0, pend_v = 0, pend_s[2] = {0, 0};
-      uint32_t it = 0;
+      const uint32_t n_it = blockIdx.x < (uint32_t)p.n_items
+                                ? ((uint32_t)p.n_items - blockIdx.x + gridDim.x - 1) / gridDim.x : 0u;
+      uint32_t i_qk = 0, i_v = 0, i_s = 0;
       grid_dependency_wait();   // inputs may come from the kernel in front (dependent launch)
-      for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++it) {
-        const uint32_t ph = it & 1;
-        const int st = s_stage(it);
-        const ItemCoord ic = item_coord<PACKED>(p, item);
-        if (!mbar_wait(bar(QK_FREE), ph ^ 1, abort_flag)) break;
-        // rows of the boxes of this item (the tile layout in shared memory does not depend on it)
-        const int bc = PACKED ? box_class(ic.n, kBoxRows) : 2;
-        const uint32_t box_bytes = kBox >> (2 - bc);
-        mbar_expect_tx(bar(QK_FULL), 4 * box_bytes);
-        load_box(sbase + L::kOffQ, &lm.q[bc], bar(QK_FULL), nf_qk, 0, ic.y0, ic.h_qk, ic.z);
-        load_box(sbase + L::kOffQ + kBox, &lm.q[bc], bar(QK_FULL), nf_qk, 64, ic.y0, ic.h_qk, ic.z);
-        load_box(sbase + L::kOffK, &lm.k[bc], bar(QK_FULL), nf_qk, 0, ic.y0, ic.h_qk, ic.z);
-        load_box(sbase + L::kOffK + kBox, &lm.k[bc], bar(QK_FULL), nf_qk, 64, ic.y0, ic.h_qk, ic.z);
-        pend_qk = 1 + (int)ph;
-        if (!mbar_wait(bar(S_FREE0 + st), s_phase(it) ^ 1, abort_flag)) break;
-        mbar_expect_tx(bar(S_FULL0 + st), 4 * kTile);
-#pragma unroll
-        for (int c = 0; c < 4; ++c)
-          tma_load_3d(sbase + L::kOffS + (uint32_t)(st * 4 + c) * kTile, &tmS, bar(S_FULL0 + st), 32 * c, 0, item);
-        pend_s[st] = 1 + (int)s_phase(it);
-        if (!mbar_wait(bar(V_FREE), ph ^ 1, abort_flag)) break;
-        mbar_expect_tx(bar(V_FULL), 2 * box_bytes);
-        load_box(sbase + L::kOffV, &lm.v[bc], bar(V_FULL), nf_v, 0, ic.y0, ic.h_v, ic.z);
-        load_box(sbase + L::kOffV + kBox, &lm.v[bc], bar(V_FULL), nf_v, 64, ic.y0, ic.h_v, ic.z);
-        pend_v = 1 + (int)ph;
+      long long t_idle = clock64();
+      uint32_t spin = 0;
+      while (i_qk < n_it || i_v < n_it || i_s < n_it) {
+        bool progress = false;
+        if (i_s < n_it && mbar_try(bar(S_FREE0 + s_stage(i_s)), s_phase(i_s) ^ 1)) {
+          const int sj = s_stage(i_s);
+          const int item = (int)(blockIdx.x + i_s * gridDim.x);
+          mbar_expect_tx(bar(S_FULL0 + sj), 4 * kTile);
+#pragma unroll 1
+          for (int c = 0; c < 4; ++c)
+            tma_load_3d(sbase + L::kOffS + (uint32_t)(sj * 4 + c) * kTile, &tmS, bar(S_FULL0 + sj), 32 * c, 0, item);
+          pend_s[sj] = 1 + (int)s_phase(i_s);
+          ++i_s;
+          progress = true;
+        }
+        if (i_qk < n_it && mbar_try(bar(QK_FREE), (i_qk & 1) ^ 1)) {
+          const ItemCoord ic = item_coord<PACKED>(p, (int)(blockIdx.x + i_qk * gridDim.x));
+          // rows of the boxes of this item (the tile layout in shared memory does not depend on it)
+          const int bc = PACKED ? box_class(ic.n, kBoxRows) : 2;
+          const uint32_t box_bytes = kBox >> (2 - bc);
+          mbar_expect_tx(bar(QK_FULL), 4 * box_bytes);
+#pragma unroll 1
+          for (uint32_t i = 0; i < 4; ++i)   // q: k halves 0, 1; k: k halves 0, 1 (consecutive boxes)
+            load_box(sbase + L::kOffQ + i * kBox, i < 2 ? &lm.q[bc] : &lm.k[bc], bar(QK_FULL), nf_qk,
+                     (int)(i & 1u) * 64, ic.y0, ic.h_qk, ic.z);
+          pend_qk = 1 + (int)(i_qk & 1);
+          ++i_qk;
+          progress = true;
+        }
+        if (i_v < n_it && mbar_try(bar(V_FREE), (i_v & 1) ^ 1)) {
+          const ItemCoord ic = item_coord<PACKED>(p, (int)(blockIdx.x + i_v * gridDim.x));
+          const int bc = PACKED ? box_class(ic.n, kBoxRows) : 2;
+          const uint32_t box_bytes = kBox >> (2 - bc);
+          mbar_expect_tx(bar(V_FULL), 2 * box_bytes);
+#pragma unroll 1
+          for (uint32_t i = 0; i < 2; ++i)
+            load_box(sbase + L::kOffV + i * kBox, &lm.v[bc], bar(V_FULL), nf_v, (int)i * 64, ic.y0, ic.h_v, ic.z);
+          pend_v = 1 + (int)(i_v & 1);
+          ++i_v;
+          progress = true;
+        }
+        if (progress) {
+          t_idle = clock64();
+          spin = 0;
+        } else if ((++spin & 255u) == 0) {   // the same limit as every other wait of the kernel
+          if (*abort_flag) break;
+          if (clock64() - t_idle > kWaitLimitCycles) {
+            *abort_flag = 1;
+            break;
+          }
+        }
       }
       if (*abort_flag) {
         // Leave no copy of ours in flight: wait (bounded) for the last loads issued.
         if (pend_qk) mbar_wait(bar(QK_FULL), pend_qk - 1, abort_flag + 1);
-        for (int s = 0; s < 2; ++s)
-          if (pend_s[s]) mbar_wait(bar(S_FULL0 + s), pend_s[s] - 1, abort_flag + 1);
+        for (int s2 = 0; s2 < 2; ++s2)
+          if (pend_s[s2]) mbar_wait(bar(S_FULL0 + s2), pend_s[s2] - 1, abort_flag + 1);
         if (pend_v) mbar_wait(bar(V_FULL), pend_v - 1, abort_flag + 1);
       }
     }
   } else if (warp == 1) {
     // ===================== MMA issuer =====================
+    // The loops over the MMAs of a product are kept rolled (descriptor = base + step): the
+    // issue rate does not need more, and the roles of a CTA share one instruction cache.
     if (lane == 0) {
+      const uint64_t dQ = desc_kmajor(sbase + L::kOffQ), dK = desc_kmajor(sbase + L::kOffK);
+      const uint64_t dS = desc_kmajor(sbase + L::kOffS), dV = desc_mnmajor(sbase + L::kOffV, kBox);
+      const uint64_t dChi = desc_kmajor(sbase + L::kOffChi), dClo = desc_kmajor(sbase + L::kOffClo);
+      // a list of up to ten waits, 6 bits each: barrier index * 2 + parity, first wait in the low bits
+      auto wait_list = [&](uint64_t w, int n) -> bool {
+#pragma unroll 1
+        for (; n > 0; --n, w >>= 6)
+          if (!mbar_wait(bar((int)((w >> 1) & 31u)), (uint32_t)(w & 1u), abort_flag)) return false;
+        return true;
+      };
+      auto W = [](int b, uint32_t parity) -> uint64_t { return (uint64_t)(b * 2) | parity; };
       uint32_t it = 0;
+#pragma unroll 1
       for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++it) {
         const uint32_t ph = it & 1;
-        const uint32_t acc_col = (it & 1) ? kColAcc1 : kColAcc0;
-        const int acc_done = (it & 1) ? ACC_DONE1 : ACC_DONE0;
-        const int acc_free = (it & 1) ? ACC_FREE1 : ACC_FREE0;
+        const uint32_t acc_col = ph ? kColAcc1 : kColAcc0;
         const uint32_t ph2 = (it >> 1) & 1;   // the two accumulators alternate
         const int st = s_stage(it);
         // scores = Q K^T
-        if (!mbar_wait(bar(QK_FULL), ph, abort_flag)) break;
-        if (!mbar_wait(bar(SC_FREE), ph ^ 1, abort_flag)) break;
+        if (!wait_list(W(QK_FULL, ph) | W(SC_FREE, ph ^ 1) << 6, 2)) break;
         tc_fence_after();
-#pragma unroll
-        for (int h = 0; h < 2; ++h)
-#pragma unroll
-          for (int s = 0; s < 4; ++s)
-            mma_bf16_ss(tmem + kColSc, desc_kmajor(sbase + L::kOffQ + h * kBox + s * 32),
-                        desc_kmajor(sbase + L::kOffK + h * kBox + s * 32), SMALL ? kIdescKK64 : kIdescKK128,
-                        (h | s) != 0);
+#pragma unroll 1
+        for (uint32_t i = 0; i < 8; ++i) {   // k half i >> 2, 16 contraction indices (32 bytes) per step
+          const uint32_t off = ((i >> 2) * kBox + (i & 3u) * 32u) >> 4;
+          mma_bf16_ss(tmem + kColSc, dQ + off, dK + off, SMALL ? kIdescKK64 : kIdescKK128, i);
+        }
         tc_commit(bar(SC_DONE));
         tc_commit(bar(QK_FREE));
-        // acc = (2^e Q) S_pre^T: A = scaled q rows (packed bf16 in TMEM), B = hi and lo tiles of S_pre
-        if (!mbar_wait(bar(S_CONV0 + st), s_phase(it), abort_flag)) break;
-        if (!mbar_wait(bar(QB_READY), ph, abort_flag)) break;
-        if (!mbar_wait(bar(QS_READY), ph, abort_flag)) break;
-        if (!mbar_wait(bar(acc_free), ph2 ^ 1, abort_flag)) break;
+        // acc = Q S_pre^T: A = the q rows (packed bf16 in TMEM), B = hi and lo tiles of S_pre
+        if (!wait_list(W(S_CONV0 + st, s_phase(it)) | W(QB_READY0 + (int)ph, ph2) << 6 |
+                           W(META_READY0 + (int)ph, ph2) << 12, 3)) break;
+        // extreme decay only: the compute warps have replaced the q rows by scaled ones
+        const bool rescaled = fast_s[ph] == 0;
+        mbar_arrive(bar(META_FREE0 + (int)ph));
+        if (!wait_list(W(ACC_FREE0 + (int)ph, ph2 ^ 1) | W(QS_READY0 + (int)ph, ph2) << 6, rescaled ? 2 : 1)) break;
         tc_fence_after();
-#pragma unroll
-        for (int kh = 0; kh < 2; ++kh)        // k half: 64 contraction indices
-#pragma unroll
-          for (int part = 0; part < 2; ++part)   // hi, lo
-#pragma unroll
-            for (int s = 0; s < 4; ++s)
-              mma_bf16_ts(tmem + acc_col, tmem + kColQb + kh * 32 + s * 8,
-                          desc_kmajor(sbase + L::kOffS + (uint32_t)(st * 4 + kh * 2 + part) * kTile + s * 32),
-                          kIdescKK128, (kh | part | s) != 0);
+#pragma unroll 1
+        for (uint32_t i = 0; i < 16; ++i) {   // tile i >> 2 of the stage = (k half, hi | lo)
+          const uint32_t off = (((uint32_t)st * 4u + (i >> 2)) * kTile + (i & 3u) * 32u) >> 4;
+          mma_bf16_ts(tmem + acc_col, tmem + kColQb + ph * 64 + (i >> 3) * 32 + (i & 3u) * 8, dS + off,
+                      kIdescKK128, i);
+        }
         tc_commit(bar(S_FREE0 + st));
         // acc += C'_hi V + C'_lo V
-        if (!mbar_wait(bar(C_READY), ph, abort_flag)) break;
-        if (!mbar_wait(bar(V_FULL), ph, abort_flag)) break;
+        if (!wait_list(W(C_READY, ph) | W(V_FULL, ph) << 6, 2)) break;
         tc_fence_after();
-        for (int jh = 0; jh < n_jh; ++jh)
-#pragma unroll
-          for (int s = 0; s < 4; ++s) {
-            const uint64_t bdesc = desc_mnmajor(sbase + L::kOffV + (jh * 4 + s) * 2048, kBox);
-            mma_bf16_ss(tmem + acc_col, desc_kmajor(sbase + L::kOffChi + jh * kTile + s * 32), bdesc,
-                        kIdescKMn, 1);
-            mma_bf16_ss(tmem + acc_col, desc_kmajor(sbase + L::kOffClo + jh * kTile + s * 32), bdesc,
-                        kIdescKMn, 1);
-          }
+#pragma unroll 1
+        for (uint32_t i = 0; i < 4u * (uint32_t)n_jh; ++i) {   // j half i >> 2
+          const uint64_t bdesc = dV + ((i * 2048u) >> 4);
+          const uint32_t off = ((i >> 2) * kTile + (i & 3u) * 32u) >> 4;
+          mma_bf16_ss(tmem + acc_col, dChi + off, bdesc, kIdescKMn, 1);
+          mma_bf16_ss(tmem + acc_col, dClo + off, bdesc, kIdescKMn, 1);
+        }
         tc_commit(bar(V_FREE));
-        tc_commit(bar(acc_done));
+        tc_commit(bar(ACC_DONE0 + (int)ph));
       }
     }
   } else if (warp == 2) {
@@ -444,9 +506,106 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
       }
       tma_store_wait_all();   // our stores are complete before we leave
     }
+  } else {
+    // ===================== path decay, ahead of the compute warps =====================
+    // g_i = sum of log2(alpha_j) over j in Anc(i) + {i}, for every node of the item: lane l takes
+    // nodes l, l + 32, ...; the sum runs over the mask bits against log2(alpha) in shared memory.
+    // Results of item n go to copy n & 1 of g / exp2(-g) / the range flag.
+    grid_dependency_wait();
+    uint32_t it = 0;
+    for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++it) {
+      const int par = (int)(it & 1);
+      const uint64_t* mrow;
+      const float* arow;
+      int64_t astep;
+      int Tb;
+      if constexpr (PACKED) {
+        const PackedItem pk = packed_item(p, item);
+        mrow = p.tree.anc + (size_t)pk.b * T * 2;
+        arow = p.alpha + (size_t)pk.plane_v * p.capacity + pk.row0;
+        astep = 1;
+        Tb = pk.n;
+      } else {
+        const int lb = (int)fdiv((uint32_t)item, p.dH), h = item - lb * p.H;
+        const int tb = p.tree.n_trees == 1 ? 0 : lb - (int)fdiv((uint32_t)lb, p.dB) * p.B;
+        mrow = p.tree.anc + (size_t)tb * T * 2;
+        arow = p.alpha + (int64_t)lb * p.gate.b + (int64_t)h * p.gate.h;
+        astep = p.gate.t;
+        Tb = T;
+      }
+      constexpr int kRows = kNodes / 32;   // nodes per lane
+      constexpr int kNone = 255;
+      float sum[kRows];   // log2(alpha) summed over the path from the node up to, not including, `up`
+      int up[kRows];      // how far that path reaches: an ancestor, or kNone once it is past the root
+#pragma unroll
+      for (int k = 0; k < kRows; ++k) {
+        const int r = k * 32 + lane;
+        sum[k] = 1.f;   // the gate for now; rows past the item: log2 = 0
+        up[k] = kNone;
+        if (r < Tb) {
+          sum[k] = arow[(int64_t)r * astep];
+          // parents precede their children, so the parent is the highest ancestor
+          const uint64_t m0 = mrow[2 * r], m1 = mrow[2 * r + 1];
+          if (m1) up[k] = 127 - __clzll((long long)m1);
+          else if (m0) up[k] = 63 - __clzll((long long)m0);
+        }
+      }
+      // the compute warps are done with this copy (item it - 2)
+      if (!mbar_wait_warp(bar(META_FREE0 + par), ((it >> 1) & 1) ^ 1, abort_flag)) break;
+      float* gw = g_s + par * kNodes;
+      int* up_s = reinterpret_cast<int*>(la_s);
+#pragma unroll
+      for (int k = 0; k < kRows; ++k) {
+        sum[k] = log2f(sum[k]);
+        gw[k * 32 + lane] = sum[k];
+        up_s[k * 32 + lane] = up[k];
+      }
+      __syncwarp();
+      // pointer jumping: every round doubles the length of the summed path; ceil(log2(depth + 1))
+      // rounds, whatever the shape of the tree
+      while (true) {
+        bool open = false;
+#pragma unroll
+        for (int k = 0; k < kRows; ++k) open = open || up[k] != kNone;
+        if (!__any_sync(0xffffffffu, open)) break;
+        float add[kRows];
+        int nup[kRows];
+#pragma unroll
+        for (int k = 0; k < kRows; ++k) {
+          add[k] = 0.f;
+          nup[k] = kNone;
+          if (up[k] != kNone) {
+            add[k] = gw[up[k]];
+            nup[k] = up_s[up[k]];
+          }
+        }
+        __syncwarp();
+#pragma unroll
+        for (int k = 0; k < kRows; ++k) {
+          if (up[k] != kNone) {
+            sum[k] += add[k];
+            up[k] = nup[k];
+            gw[k * 32 + lane] = sum[k];
+            up_s[k * 32 + lane] = nup[k];
+          }
+        }
+        __syncwarp();
+      }
+      bool in_range = true;
+#pragma unroll
+      for (int k = 0; k < kRows; ++k) {
+        f_s[par * kNodes + k * 32 + lane] = exp2f(-sum[k]);
+        in_range = in_range && fabsf(sum[k]) <= 100.f;
+      }
+      // exp2(e_i - g_j) = 2^e_i * 2^-g_j is safe when every |g| <= 100; otherwise exp2 is taken per pair
+      const bool fast = __all_sync(0xffffffffu, in_range);
+      if (lane == 0) fast_s[par] = fast;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(META_READY0 + par));
+    }
   }
   } else if (warp >= kFirstSplitWarp) {
-    // ===================== state split =====================
+    // ===================== operand warps: q rows into TMEM, state split =====================
     asm volatile("setmaxnreg.dec.sync.aligned.u32 104;");
     const int row = tid - kFirstSplitWarp * 32;   // state row v, and node i for the q copy
     const int pw = warp - kFirstSplitWarp;        // = TMEM lane window of this warp
@@ -456,10 +615,12 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
     for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++it) {
       const uint32_t ph = it & 1;
       const int st = s_stage(it);
-      // ---- q rows (bf16, swizzled boxes) -> TMEM as they are: the A operand of the prefix MMA ----
+      // ---- q rows (bf16, swizzled boxes) -> TMEM as they are: the A operand of the prefix MMA.
+      // Copy it & 1, last read by the prefix MMA of item it - 2.  Two stages: that MMA freed the
+      // stage this item now uses.  One stage: the state of item it - 1, already seen here, was
+      // only loaded after that MMA had freed the stage.
+      if (SMALL && it >= 2 && !mbar_wait_warp(bar(S_FREE0 + st), s_phase(it - 2), abort_flag)) break;
       if (!mbar_wait_warp(bar(QK_FULL), ph, abort_flag)) break;
-      // the prefix MMA of the item before is done with the copy in TMEM
-      if (it > 0 && !mbar_wait_warp(bar(S_FREE0 + s_stage(it - 1)), s_phase(it - 1), abort_flag)) break;
       tc_fence_after();
       if (pw * 32 < T) {
 #pragma unroll
@@ -471,21 +632,21 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
             const uint4 x = *reinterpret_cast<const uint4*>(qrow + (((uint32_t)c ^ swz) << 4));
             r[c * 4 + 0] = x.x; r[c * 4 + 1] = x.y; r[c * 4 + 2] = x.z; r[c * 4 + 3] = x.w;
           }
-          tmem_st32(tmem + lane_addr + kColQb + half * 32, r);
+          tmem_st32(tmem + lane_addr + kColQb + ph * 64 + half * 32, r);
         }
         tmem_wait_st();
       }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) {
-        mbar_arrive(bar(QB_READY));
+        mbar_arrive(bar(QB_READY0 + (int)ph));
         mbar_arrive(bar(QK_FREE));
       }
       // ---- the state split ----
       if (!mbar_wait_warp(bar(S_FULL0 + st), s_phase(it), abort_flag)) break;
       unsigned char* s_buf = sm + L::kOffS + (uint32_t)st * 4u * kTile;
-      split_state_row(s_buf, row, 0, swz);
-      split_state_row(s_buf, row, 1, swz);
+#pragma unroll 1
+      for (int half = 0; half < 2; ++half) split_state_row(s_buf, row, half, swz);   // one copy of the code
       fence_async_smem();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(S_CONV0 + st));
@@ -551,10 +712,9 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
 
     // metadata of the first item; later items are fetched one item ahead
     uint64_t nm0 = 0, nm1 = 0;
-    float nal = 1.f;   // raw decay gate of the next item (log2 taken when it is used)
     PackedItem npk = {0, 0, 0, 0, T};   // packed forest: rows of the next item
     auto fetch_meta = [&](int item) {
-      nm0 = 0; nm1 = 0; nal = 1.f;
+      nm0 = 0; nm1 = 0;
       if constexpr (PACKED) {
         if (item < p.n_items) {
           npk = packed_item(p, item);
@@ -562,16 +722,14 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
             const uint64_t* m = p.tree.anc + ((size_t)npk.b * T + row) * 2;
             nm0 = m[0];
             nm1 = m[1];
-            nal = p.alpha[(size_t)npk.plane_v * p.capacity + npk.row0 + row];
           }
         }
       } else if (item < p.n_items && row < T) {
-        const int lb = item / p.H, h = item - lb * p.H;
-        const int tb = p.tree.n_trees == 1 ? 0 : lb % p.B;
+        const int lb = (int)fdiv((uint32_t)item, p.dH);
+        const int tb = p.tree.n_trees == 1 ? 0 : lb - (int)fdiv((uint32_t)lb, p.dB) * p.B;
         const uint64_t* m = p.tree.anc + ((size_t)tb * T + row) * 2;
         nm0 = m[0];
         nm1 = m[1];
-        nal = p.alpha[(int64_t)lb * p.gate.b + (int64_t)h * p.gate.h + (int64_t)row * p.gate.t];
       }
     };
     // dependent launch: barrier set-up and the TMEM allocation above ran under the tail of the
@@ -586,39 +744,29 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
     float r_prev = 0.f;
     PackedItem pk = npk, pk_prev = npk;
     const int total_rows = PACKED ? p.offsets[p.B] : 0;   // rows at and past this one hold no node
-    for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++it) {
+    // One pass more than the CTA has items: the last one only writes out the last item (the
+    // output code exists once).
+#pragma unroll 1
+    for (int item = blockIdx.x;; item += gridDim.x, ++it) {
+      const bool live = item < p.n_items;
       const uint32_t ph = it & 1;
+      const int par = (int)ph;
       uint64_t m0 = nm0, m1 = nm1;
       pk = npk;
       const int Tb = PACKED ? pk.n : T;   // real nodes of this item
-      // ---- path decay: g_i = sum of log2(alpha) over Anc(i) + {i} ----
-      const float la_own = log2f(nal);
-      if (hc == 0 && row < Tb) la_s[row] = la_own;
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(SETUP));
-      fetch_meta(item + (int)gridDim.x);   // next item's metadata rides under this item's work
-      if (!(ok = mbar_wait_warp(bar(SETUP), 0, abort_flag))) break;   // SETUP: two phases per item
-      float g = 0.f;
+      const float* gs = g_s + par * kNodes;
+      const float* fs = f_s + par * kNodes;
+      bool fast = true;
+      float e_int = 0.f, r_scale = 0.f;
+      if (live) {
+      fetch_meta(item + (int)gridDim.x);   // next item's masks ride under this item's work
       if (row < Tb) {
-        g = la_own;
-        uint64_t a0 = m0, a1 = m1;
-        while (a0) { const int j = __ffsll((long long)a0) - 1; a0 &= a0 - 1; g += la_s[j]; }
-        while (a1) { const int j = __ffsll((long long)a1) - 1; a1 &= a1 - 1; g += la_s[64 + j]; }
         if (row < 64) m0 |= 1ull << row; else m1 |= 1ull << (row - 64);   // M+ = M- + I
       }
-      if (hc == 0 && row < Tb) {
-        g_s[row] = g;
-        f_s[row] = exp2f(-g);
-      }
-      // exp2(e_i - g_j) = 2^e_i * 2^-g_j is safe when every |g| <= 100; otherwise take exp2 per pair
-      const bool range_ok_warp = __all_sync(0xffffffffu, row >= Tb || fabsf(g) <= 100.f);
-      if (lane == 0) range_ok_s[cw] = range_ok_warp;
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(SETUP));
-      if (!(ok = mbar_wait_warp(bar(SETUP), 1, abort_flag))) break;
-      bool fast = true;
-#pragma unroll
-      for (int w8 = 0; w8 < kComputeWarps; ++w8) fast = fast && range_ok_s[w8];
+      // ---- path decay g, exp2(-g) and the range flag of this item: written by the decay warp ----
+      if (!(ok = mbar_wait_warp(bar(META_READY0 + par), (it >> 1) & 1, abort_flag))) break;
+      const float g = row < Tb ? gs[row] : 0.f;
+      fast = fast_s[par] != 0;
       // Row scaling.  Plain form (every |g| <= 100): the accumulator holds  q_i S_pre^T +
       // sum_j 2^(-g_j) s_ij v_j  and O_i = 2^(g_i) acc.  Extreme decay: a row exponent e =
       // round(g_i) keeps every factor in range: the accumulator holds  2^e (q_i S_pre^T) +
@@ -627,42 +775,38 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
       // ancestor pairs.  Below 2^-100 the prefix term is under fp32 resolution of anything it
       // is added to and is dropped.
       const bool tiny = !fast && g < -100.f;
-      const float e_int = fast ? 0.f : (tiny ? g : fminf(rintf(g), 100.f));
+      e_int = fast ? 0.f : (tiny ? g : fminf(rintf(g), 100.f));
       const float a_scale = tiny ? 0.f : exp2f(e_int);
-      const float r_scale = exp2f(g - e_int);
-      // ---- scores of this item ----
-      // (Waited for before the arrival below: that arrival must not run an item ahead of the MMA
-      // issuer, which commits the scores of item n+1 only after it has consumed this one.)
-      if (!(ok = mbar_wait_warp(bar(SC_DONE), ph, abort_flag))) break;
+      r_scale = exp2f(g - e_int);
       if (!fast) {
-        // extreme decay: replace the q rows that the split warps copied to TMEM by scaled ones
-        if (!(ok = mbar_wait_warp(bar(QB_READY), ph, abort_flag))) break;
+        // extreme decay: replace the q rows that the operand warps copied to TMEM by scaled ones
+        if (!(ok = mbar_wait_warp(bar(QB_READY0 + (int)ph), (it >> 1) & 1, abort_flag))) break;
         tc_fence_after();
         if (warp_live) {
-          const unsigned char* qrow = sm + L::kOffQ + hc * kBox + row * 128;
           uint32_t r[32];
+          tmem_ld32(tmem + lane_addr + kColQb + ph * 64 + hc * 32, r);
+          tmem_wait_ld();
 #pragma unroll
-          for (int c = 0; c < 8; ++c) {
-            const uint4 x = *reinterpret_cast<const uint4*>(qrow + (((uint32_t)c ^ swz) << 4));
-            const uint32_t w[4] = {x.x, x.y, x.z, x.w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e)   // power-of-two scaling: the products are exact in bf16
-              r[c * 4 + e] = __byte_perm(__float_as_uint(a_scale * __uint_as_float(w[e] << 16)),
-                                         __float_as_uint(a_scale * __uint_as_float(w[e] & 0xffff0000u)), 0x7632);
-          }
-          tmem_st32(tmem + lane_addr + kColQb + hc * 32, r);
+          for (int e = 0; e < 32; ++e)   // power-of-two scaling: the products are exact in bf16
+            r[e] = __byte_perm(__float_as_uint(a_scale * __uint_as_float(r[e] << 16)),
+                               __float_as_uint(a_scale * __uint_as_float(r[e] & 0xffff0000u)), 0x7632);
+          tmem_st32(tmem + lane_addr + kColQb + ph * 64 + hc * 32, r);
           tmem_wait_st();
         }
         tc_fence_before();
       }
       __syncwarp();
-      if (lane == 0) {
-        mbar_arrive(bar(QS_READY));
-        mbar_arrive(bar(QK_FREE));
+      // (one barrier per copy of q: an arrival for item n + 2 comes after the scores of item
+      // n + 1, which the MMA issuer commits after it is through with this one)
+      if (lane == 0) mbar_arrive(bar(QS_READY0 + (int)ph));
       }
       // ---- output rows of the previous item: its accumulator is complete once its readout MMA
-      // is, and (T > 64) the C' tiles it frees double as the staging area of the output store ----
+      // is, and (T > 64) the C' tiles it frees double as the staging area of the output store.
+      // Taken before the scores of this item are waited for: they are computed meanwhile. ----
       if (it > 0 && !(ok = final_epilogue(it - 1, r_prev, (it - 1) & 1, pk_prev))) break;
+      if (!live) break;
+      // ---- scores of this item ----
+      if (!(ok = mbar_wait_warp(bar(SC_DONE), ph, abort_flag))) break;
       tc_fence_after();
       if (warp_live) {
         // this warp covers 32 n_jh of the 64 n_jh real columns, 32 at a time
@@ -678,8 +822,8 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
           if (fast) {
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
-              const float4 fa = *reinterpret_cast<const float4*>(f_s + cbase + c * 8);
-              const float4 fb = *reinterpret_cast<const float4*>(f_s + cbase + c * 8 + 4);
+              const float4 fa = *reinterpret_cast<const float4*>(fs + cbase + c * 8);
+              const float4 fb = *reinterpret_cast<const float4*>(fs + cbase + c * 8 + 4);
               const float f8[8] = {fa.x, fa.y, fa.z, fa.w, fb.x, fb.y, fb.z, fb.w};
               float cv[8];
 #pragma unroll
@@ -695,7 +839,7 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
               float cv[8];
 #pragma unroll
               for (int e = 0; e < 8; ++e) {
-                const float x = __uint_as_float(r[c * 8 + e]) * exp2f(e_int - g_s[cbase + c * 8 + e]);
+                const float x = __uint_as_float(r[c * 8 + e]) * exp2f(e_int - gs[cbase + c * 8 + e]);
                 cv[e] = ((bits >> (c * 8 + e)) & 1u) ? x : 0.f;
               }
               store_split8(chi, clo, ((uint32_t)((chunk0 + c) ^ swz)) << 4, cv);
@@ -722,11 +866,11 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
       if (lane == 0) {
         mbar_arrive(bar(C_READY));
         mbar_arrive(bar(SC_FREE));
+        mbar_arrive(bar(META_FREE0 + par));   // this copy of g may take item it + 2
       }
       r_prev = r_scale;
       pk_prev = pk;
     }
-    if (ok && it > 0) final_epilogue(it - 1, r_prev, (it - 1) & 1, pk_prev);
   }
 
   // ---- teardown: every path comes here ----
@@ -908,6 +1052,9 @@ int tv_launch_verify_tc(const VerifyArgs& a, int32_t* status, cudaStream_t strea
   p.node_first = node_first;
   p.offsets = a.tree.offsets;
   p.capacity = a.tree.capacity;
+  p.dH = make_fastdiv((uint32_t)a.H);
+  p.dB = make_fastdiv((uint32_t)a.B);
+  p.dG = make_fastdiv((uint32_t)(a.H / a.Hk));
   const int grid = (int)(items < (uint64_t)sm_count ? items : (uint64_t)sm_count);
   const size_t smem = small ? Lay<true>::kSmemBytes : Lay<false>::kSmemBytes;
   auto go = [&](auto kernel) {
