@@ -276,6 +276,39 @@ __device__ __forceinline__ PackedItem packed_item(const int32_t* offsets, int B,
   return r;
 }
 
+// The same with the divisions by H, B and the q/k group size H / Hk done as multiply-shift.
+struct ItemDiv {
+  FastDiv dH, dB, dG;
+};
+inline ItemDiv make_item_div(int B, int H, int Hk) {
+  ItemDiv d;
+  d.dH = make_fastdiv((uint32_t)H);
+  d.dB = make_fastdiv((uint32_t)B);
+  d.dG = make_fastdiv((uint32_t)(H / Hk));
+  return d;
+}
+__device__ __forceinline__ PackedItem packed_item(const int32_t* offsets, int B, int H, int Hk, int item,
+                                                  const ItemDiv& d) {
+  PackedItem r;
+  const int lb = (int)fdiv((uint32_t)item, d.dH), h = item - lb * H;
+  const int l = (int)fdiv((uint32_t)lb, d.dB);
+  r.b = lb - l * B;
+  r.plane_v = l * H + h;
+  r.plane_qk = l * Hk + (int)fdiv((uint32_t)h, d.dG);
+  r.row0 = offsets[r.b];
+  r.n = offsets[r.b + 1] - r.row0;
+  return r;
+}
+// dense layout: the q/k item of state item `item`, and the tree of its request
+__device__ __forceinline__ int qk_item(int item, int H, int Hk, const ItemDiv& d) {
+  const int lb = (int)fdiv((uint32_t)item, d.dH), h = item - lb * H;
+  return lb * Hk + (int)fdiv((uint32_t)h, d.dG);
+}
+__device__ __forceinline__ int request_of(int item, int B, const ItemDiv& d) {
+  const int lb = (int)fdiv((uint32_t)item, d.dH);
+  return lb - (int)fdiv((uint32_t)lb, d.dB) * B;
+}
+
 // Programmatic dependent launch: the kernel may start while the kernel in front of it on the
 // stream is still running, provided that kernel released its dependents early; whatever reads
 // that kernel's output first passes grid_dependency_wait().

@@ -404,8 +404,10 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
     }
   } else if (warp == 1) {
     // ===================== MMA issuer =====================
-    // The loops over the MMAs of a product are kept rolled (descriptor = base + step): the
-    // issue rate does not need more, and the roles of a CTA share one instruction cache.
+    // The loops over the MMAs of a product: unrolled for T <= 64 (rolled, the address arithmetic
+    // between two MMAs slowed their issue enough to cost 1.6 us of a 32 us launch), rolled for
+    // T > 64, where the items are twice as long and the smaller code measured 4 % faster (the
+    // roles of a CTA share one instruction cache).
     if (lane == 0) {
       const uint64_t dQ = desc_kmajor(sbase + L::kOffQ), dK = desc_kmajor(sbase + L::kOffK);
       const uint64_t dS = desc_kmajor(sbase + L::kOffS), dV = desc_mnmajor(sbase + L::kOffV, kBox);
@@ -428,7 +430,7 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
         // scores = Q K^T
         if (!wait_list(W(QK_FULL, ph) | W(SC_FREE, ph ^ 1) << 6, 2)) break;
         tc_fence_after();
-#pragma unroll 1
+#pragma unroll(SMALL ? 8 : 1)
         for (uint32_t i = 0; i < 8; ++i) {   // k half i >> 2, 16 contraction indices (32 bytes) per step
           const uint32_t off = ((i >> 2) * kBox + (i & 3u) * 32u) >> 4;
           mma_bf16_ss(tmem + kColSc, dQ + off, dK + off, SMALL ? kIdescKK64 : kIdescKK128, i);
@@ -443,7 +445,7 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
         mbar_arrive(bar(META_FREE0 + (int)ph));
         if (!wait_list(W(ACC_FREE0 + (int)ph, ph2 ^ 1) | W(QS_READY0 + (int)ph, ph2) << 6, rescaled ? 2 : 1)) break;
         tc_fence_after();
-#pragma unroll 1
+#pragma unroll(SMALL ? 16 : 1)
         for (uint32_t i = 0; i < 16; ++i) {   // tile i >> 2 of the stage = (k half, hi | lo)
           const uint32_t off = (((uint32_t)st * 4u + (i >> 2)) * kTile + (i & 3u) * 32u) >> 4;
           mma_bf16_ts(tmem + acc_col, tmem + kColQb + ph * 64 + (i >> 3) * 32 + (i & 3u) * 8, dS + off,
@@ -454,12 +456,14 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
         if (!wait_list(W(C_READY, ph) | W(V_FULL, ph) << 6, 2)) break;
         tc_fence_after();
 #pragma unroll 1
-        for (uint32_t i = 0; i < 4u * (uint32_t)n_jh; ++i) {   // j half i >> 2
-          const uint64_t bdesc = dV + ((i * 2048u) >> 4);
-          const uint32_t off = ((i >> 2) * kTile + (i & 3u) * 32u) >> 4;
-          mma_bf16_ss(tmem + acc_col, dChi + off, bdesc, kIdescKMn, 1);
-          mma_bf16_ss(tmem + acc_col, dClo + off, bdesc, kIdescKMn, 1);
-        }
+        for (uint32_t jh = 0; jh < (uint32_t)n_jh; ++jh)   // j half
+#pragma unroll(SMALL ? 4 : 1)
+          for (uint32_t i = 0; i < 4; ++i) {
+            const uint64_t bdesc = dV + (((jh * 4u + i) * 2048u) >> 4);
+            const uint32_t off = (jh * kTile + i * 32u) >> 4;
+            mma_bf16_ss(tmem + acc_col, dChi + off, bdesc, kIdescKMn, 1);
+            mma_bf16_ss(tmem + acc_col, dClo + off, bdesc, kIdescKMn, 1);
+          }
         tc_commit(bar(V_FREE));
         tc_commit(bar(ACC_DONE0 + (int)ph));
       }

@@ -85,6 +85,7 @@ struct DeltaParams {
   // outputs as plain pointers for the rows that leave from registers
   const int32_t* offsets;
   int32_t capacity;
+  ItemDiv div;   // divisions by H, B, H / Hk as multiply-shift
   float* O;
   float* U;
 };
@@ -176,10 +177,10 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         mbar_expect_tx(bar(qfull), 4 * 8192);
         int qk = 0, vplane = item, y0 = 0;
         if constexpr (PACKED) {
-          const PackedItem pi = packed_item(p.offsets, p.B, p.H, p.Hk, item);
+          const PackedItem pi = packed_item(p.offsets, p.B, p.H, p.Hk, item, p.div);
           qk = pi.plane_qk; vplane = pi.plane_v; y0 = pi.row0;
         } else {
-          qk = tv_qk_item(item, p.H, p.Hk);
+          qk = qk_item(item, p.H, p.Hk, p.div);
         }
         tma_load_3d(sbase + qk_base, &tmQ, bar(qfull), 0, y0, qk);
         tma_load_3d(sbase + qk_base + kTile, &tmQ, bar(qfull), 64, y0, qk);
@@ -220,12 +221,14 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         if (!mbar_wait(bar((j & 1) ? QK_FULL1 : QK_FULL), (j >> 1) & 1, abort_flag)) return false;
         if (!mbar_wait(bar(G_FREE), (j & 1) ^ 1, abort_flag)) return false;   // score columns read by E1 of j-1
         tc_fence_after();
+        // (the MMA loops are kept rolled, descriptor = base + step: the roles of a CTA share one
+        // instruction cache)
+        const uint64_t dA = desc_kmajor(sbase + qk_base), dB = desc_kmajor(sbase + qk_base + 8192);
 #pragma unroll
-        for (int h = 0; h < 2; ++h)
-#pragma unroll
-          for (int s = 0; s < 4; ++s)
-            mma_bf16_ss(tmem + kColSc, desc_kmajor(sbase + qk_base + h * kTile + s * 32),
-                        desc_kmajor(sbase + qk_base + h * kTile + 8192 + s * 32), kIdGram, (h | s) != 0);
+        for (uint32_t i = 0; i < 8; ++i) {   // k half i >> 2, 32 bytes of k per step
+          const uint32_t off = ((i >> 2) * kTile + (i & 3u) * 32u) >> 4;
+          mma_bf16_ss(tmem + kColSc, dA + off, dB + off, kIdGram, i);
+        }
         tc_commit(bar(G_DONE));
         return true;
       };
@@ -237,12 +240,13 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         // Qf += -(W D_P) K  (rows 64..127: -(A D_P) K); the compute warps initialised Qf with D_P Q
         if (!mbar_wait(bar(W_READY), ph, abort_flag)) break;
         tc_fence_after();
+        {
+          const uint64_t dAk = desc_kmajor(sbase + kOffAk), dKr = desc_mnmajor(sbase + qk_base + 4 * 2048, kTile);
 #pragma unroll
-        for (int part = 0; part < 2; ++part)      // hi, lo
-#pragma unroll
-          for (int j = 4; j < 8; ++j)             // the K rows of the stacked tile
-            mma_bf16_ss(tmem + kColQf, desc_kmajor(sbase + kOffAk + part * kTile + (j & 3) * 32),
-                        desc_mnmajor(sbase + qk_base + j * 2048, kTile), kIdMn, 1);
+          for (uint32_t i = 0; i < 8; ++i)   // part i >> 2 (hi, lo), K rows 16 (i & 3) .. of the stacked tile
+            mma_bf16_ss(tmem + kColQf, dAk + (((i >> 2) * kTile + (i & 3u) * 32u) >> 4),
+                        dKr + (((i & 3u) * 2048u) >> 4), kIdMn, 1);
+        }
         tc_commit(bar(D1_DONE));
         tc_commit(bar((it & 1) ? QK_FREE1 : QK_FREE));
         // acc = Qf S_pre^T: Qf must be complete in TMEM before it is read as the A operand
@@ -250,21 +254,23 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         if (!mbar_wait(bar(S_FULL), ph, abort_flag)) break;
         if (!mbar_wait(bar(ACC_FREE), ph ^ 1, abort_flag)) break;
         tc_fence_after();
+        {
+          const uint64_t dS = desc_kmajor(sbase + kOffS);
 #pragma unroll
-        for (int c = 0; c < 4; ++c)
-#pragma unroll
-          for (int s = 0; s < 4; ++s)
-            mma_tf32_ts(tmem + kColAcc, tmem + kColQf + c * 32 + s * 8,
-                        desc_kmajor(sbase + kOffS + c * kTile + s * 32), kIdTf32, (c | s) != 0);
+          for (uint32_t i = 0; i < 16; ++i)   // k chunk i >> 2 of the state, 8 values of k per step
+            mma_tf32_ts(tmem + kColAcc, tmem + kColQf + i * 8, dS + (((i >> 2) * kTile + (i & 3u) * 32u) >> 4),
+                        kIdTf32, i);
+        }
         tc_commit(bar(S_FREE));
         // acc += [W ; A] V
         if (!mbar_wait(bar(V_FULL), ph, abort_flag)) break;
         tc_fence_after();
+        {
+          const uint64_t dW = desc_kmajor(sbase + kOffW), dVr = desc_mnmajor(sbase + kOffV, kTile);
 #pragma unroll
-        for (int s = 0; s < 4; ++s) {
-          const uint64_t bdesc = desc_mnmajor(sbase + kOffV + s * 2048, kTile);
-          mma_bf16_ss(tmem + kColAcc, desc_kmajor(sbase + kOffW + s * 32), bdesc, kIdMn, 1);
-          mma_bf16_ss(tmem + kColAcc, desc_kmajor(sbase + kOffW + kTile + s * 32), bdesc, kIdMn, 1);
+          for (uint32_t i = 0; i < 8; ++i)   // 16 nodes j per step; hi then lo tile of [W ; A]
+            mma_bf16_ss(tmem + kColAcc, dW + (((i & 1u) * kTile + (i >> 1) * 32u) >> 4),
+                        dVr + (((i >> 1) * 2048u) >> 4), kIdMn, 1);
         }
         tc_commit(bar(V_FREE));
         tc_commit(bar(ACC_DONE));
@@ -280,7 +286,7 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         if (!mbar_wait(bar(OST_READY), it & 1, abort_flag)) break;
         if constexpr (PACKED) {
           // groups of 8 rows, largest boxes first (staging rows start on 1024-byte boundaries)
-          const PackedItem pi = packed_item(p.offsets, p.B, p.H, p.Hk, item);
+          const PackedItem pi = packed_item(p.offsets, p.B, p.H, p.Hk, item, p.div);
           const int full = pi.n & ~7;
           for (int part = 0; part < (want_U ? 2 : 1); ++part) {
             const OutMaps& mm = part == 0 ? mapsO : mapsU;
@@ -325,12 +331,12 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       int n = T, tb = 0;
       size_t g0 = (size_t)item * T;                     // first gate of the item
       if constexpr (PACKED) {
-        const PackedItem pi = packed_item(p.offsets, p.B, p.H, p.Hk, item);
+        const PackedItem pi = packed_item(p.offsets, p.B, p.H, p.Hk, item, p.div);
         n = pi.n;
         tb = pi.b;
         g0 = (size_t)pi.plane_v * p.capacity + pi.row0;
       } else {
-        tb = p.tree.n_trees == 1 ? 0 : (item / p.H) % p.B;
+        tb = p.tree.n_trees == 1 ? 0 : request_of(item, p.B, p.div);
       }
       float* tab = tab_s + buf * (2 * kRows);
       // all six loads first: one trip to memory, not one per table
@@ -383,7 +389,7 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     PackedItem npk = {0, 0, 0, 0, T};   // packed forest: rows of the next item
     auto next_rows = [&](int item) {
       if constexpr (PACKED) {
-        if (item < p.n_items) npk = packed_item(p.offsets, p.B, p.H, p.Hk, item);
+        if (item < p.n_items) npk = packed_item(p.offsets, p.B, p.H, p.Hk, item, p.div);
       }
     };
     grid_dependency_wait();   // tree metadata comes from the kernel in front (dependent launch)
@@ -431,11 +437,21 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     bool ok = true;
     PackedItem pk = npk, pk_prev = npk;
     const int total_rows = PACKED ? p.offsets[p.B] : 0;   // rows at and past this one hold no node
-    for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++it) {
+    // One pass more than the CTA has items: the last one only writes out the last item (the
+    // output code exists once).
+#pragma unroll 1
+    for (int item = blockIdx.x;; item += gridDim.x, ++it) {
+      const bool item_live = item < p.n_items;
       const uint32_t ph = it & 1;
       pk = npk;
       const int Tb = PACKED ? pk.n : T;                       // real nodes of this item
-      const bool live_i = live && node < Tb;
+      const bool live_i = live && node < Tb && item_live;
+      constexpr int NS = DMAX + 1;                            // path slots in use
+      int path[NS];
+      float al[NS], bt[NS], pre[NS], vec[NS];
+      float Pi = 1.f;                                         // P_i: product of alpha along the path
+      int depth = 0;
+      if (item_live) {
       // Every warp has finished the row solve of the previous item (it read the slot tables and
       // the per-node tables that this item is about to overwrite; with the Gram product issued one
       // item ahead, nothing else would hold a fast warp back).
@@ -446,7 +462,7 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       const float* al_s = tab_s + ph * (2 * kRows);
       const float* be_s = al_s + kRows;
       next_rows(item + (int)gridDim.x);
-      const int depth = __popcll(m);
+      depth = __popcll(m);
 
       // ---- E1: raw path-sparse rows: part 0 <- Q K^T (path incl. the node), part 1 <- K K^T ----
       if (!(ok = mbar_wait_warp(bar(G_DONE), ph, abort_flag))) break;
@@ -479,10 +495,6 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       if (!(ok = mbar_wait_warp(bar(E1_SYNC), ph, abort_flag))) break;
 
       // ---- E2: decay factors, one back-substitution per row, operand tiles ----
-      constexpr int NS = DMAX + 1;                            // path slots in use
-      int path[NS];
-      float al[NS], bt[NS], pre[NS], vec[NS];
-      float Pi = 1.f;                                         // P_i: product of alpha along the path
       if (live_i) {
         const uint32_t* pw = reinterpret_cast<const uint32_t*>(Ps_all + (ph * kRows + node) * kLdP);
         const uint32_t pword[4] = {pw[0], pw[1], pw[2], pw[3]};
@@ -500,7 +512,9 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       // ---- output of the previous item: its MMAs ran under E1 and the gather above, so the
       // accumulator is complete by now; the TMA stores that take the staged chunks away read them
       // under the back-substitution and the Qf initialisation below ----
+      }
       if (it > 0 && !(ok = final_epilogue(it - 1, pk_prev))) break;
+      if (!item_live) break;
       if (live_i) {
         // C_{i,p_s} = (q_i . k_{p_s}) P_i / P_{p_s}: the ratio is the product of alpha over the
         // slots after s, built up from the node's own slot backwards
@@ -609,7 +623,6 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       }
       pk_prev = pk;
     }
-    if (ok && it > 0) final_epilogue(it - 1, pk_prev);
   }
 
   tc_fence_before();
@@ -713,6 +726,7 @@ int tv_launch_verify_tc_delta(const VerifyArgs& a, int32_t* status, cudaStream_t
   p.status = status;
   p.offsets = a.tree.offsets;
   p.capacity = a.tree.capacity;
+  p.div = make_item_div(a.B, a.H, a.Hk);
   p.O = a.O;
   p.U = Uout;
   const int grid = (int)(items < (uint64_t)sm_count ? items : (uint64_t)sm_count);

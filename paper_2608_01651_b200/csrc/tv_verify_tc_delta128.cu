@@ -77,6 +77,7 @@ struct Delta128Params {
   // packed forest only: row offsets of the requests and rows per (layer, head) plane
   const int32_t* offsets;
   int32_t capacity;
+  ItemDiv div;   // divisions by H, B, H / Hk as multiply-shift
 };
 
 // bf16 hi/lo parts of x (hi = upper 16 bits, lo = upper 16 bits of the exact remainder)
@@ -153,10 +154,10 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
         const uint32_t ph = it & 1;
         int qk = 0, vplane = item, y0 = 0;
         if constexpr (PACKED) {
-          const PackedItem pi = packed_item(p.offsets, p.B, p.H, p.Hk, item);
+          const PackedItem pi = packed_item(p.offsets, p.B, p.H, p.Hk, item, p.div);
           qk = pi.plane_qk; vplane = pi.plane_v; y0 = pi.row0;
         } else {
-          qk = tv_qk_item(item, p.H, p.Hk);
+          qk = qk_item(item, p.H, p.Hk, p.div);
         }
         if (!mbar_wait(bar(QK_FREE), ph ^ 1, abort_flag)) break;
         mbar_expect_tx(bar(QK_FULL), 8 * 8192);
@@ -287,12 +288,12 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
       int n = T, tb = 0;
       size_t g0 = (size_t)item * T;   // first gate (and first output row) of the item
       if constexpr (PACKED) {
-        const PackedItem pi = packed_item(p.offsets, p.B, p.H, p.Hk, item);
+        const PackedItem pi = packed_item(p.offsets, p.B, p.H, p.Hk, item, p.div);
         n = pi.n;
         tb = pi.b;
         g0 = (size_t)pi.plane_v * p.capacity + pi.row0;
       } else {
-        tb = p.tree.n_trees == 1 ? 0 : (item / p.H) % p.B;
+        tb = p.tree.n_trees == 1 ? 0 : request_of(item, p.B, p.div);
       }
       float* tab = tab_s + buf * (2 * kNodes);
       // all loads first: one trip to memory, not one per table
@@ -721,6 +722,7 @@ int tv_launch_verify_tc_delta128(const VerifyArgs& a, int32_t* status, cudaStrea
   const int grid = (int)(items < (uint64_t)sm_count ? items : (uint64_t)sm_count);
   p.offsets = a.tree.offsets;
   p.capacity = a.tree.capacity;
+  p.div = make_item_div(a.B, a.H, a.Hk);
   const bool shallow = a.tree.max_depth_all <= 8;
   auto launch = [&](auto kernel) {
     // packed forests store from registers only: the output maps are placeholders there
