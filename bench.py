@@ -472,7 +472,7 @@ class StepRig:
     marshalled once per set, and the step itself."""
 
     def __init__(self, tv, wl, dev, stream, impl, n_sets=0):
-        self.tv, self.wl, self.stream = tv, wl, stream
+        self.tv, self.wl, self.stream, self.dev = tv, wl, stream, dev
         self.parents, self.accepted = inputs.make_trees(wl)
         self.acc_len = accepted_lengths(self.parents, self.accepted)
         delta = wl.rule == inputs.DELTA
@@ -546,6 +546,22 @@ def time_loop(stream, n, body, warm=3):
     return e0.elapsed_time(e1) / n
 
 
+def copy_yardstick(dev, stream, nbytes, n=48):
+    """A plain device copy that moves the same number of bytes as a kernel launch (half read,
+    half written), launched back to back over rotating buffers larger than L2: what a launch of
+    that SIZE can reach on this GPU, next to the copy peak measured on gigabytes.  torch's
+    copy kernel, a yardstick only."""
+    half = max(min(int(nbytes), 2**30) // 2 // 16 * 16, 16)   # launches beyond 1 GiB: 1 GiB says it all
+    sets = min(max(2, int(4 * 126 * 2**20 // (2 * half)) + 1), 64)
+    src = [torch.empty(half, dtype=torch.uint8, device=dev) for _ in range(sets)]
+    dst = [torch.empty(half, dtype=torch.uint8, device=dev) for _ in range(sets)]
+    for t in src:
+        t.zero_()
+    ms = time_loop(stream, n, lambda i: dst[i % sets].copy_(src[i % sets]), warm=sets)
+    return {"bytes": 2 * half, "ms": ms, "GBps": 2 * half / (ms * 1e-3) / 1e9,
+            "what": "torch copy_ of bytes/2, back to back, L2-cold"}
+
+
 def kernel_split(rig, step_ms, n, peak):
     """Per-kernel times WITHOUT events between launches (an event between two launches costs a
     bubble and undoes the dependent launches): the loop 'metadata + verify' is timed next to the
@@ -575,6 +591,11 @@ def kernel_split(rig, step_ms, n, peak):
               "back_to_back_ms": c_b2b,
               "back_to_back_frac_of_measured_copy": gbs(rig.cbytes, c_b2b) / peak,
               "back_to_back_frac_of_nominal_8TBps": gbs(rig.cbytes, c_b2b) / NOMINAL_HBM_GBS}
+    for obj, nbytes in ((verify, rig.vbytes), (commit, rig.cbytes)):
+        y = copy_yardstick(rig.dev, stream, nbytes)
+        y["frac_of_measured_copy"] = y["GBps"] / peak
+        y["kernel_back_to_back_vs_this_copy"] = y["ms"] / obj["back_to_back_ms"]
+        obj["copy_of_same_bytes"] = y
     return verify, commit
 
 
