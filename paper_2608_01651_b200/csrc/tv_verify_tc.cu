@@ -346,7 +346,10 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
       uint32_t spin = 0;
       while (i_qk < n_it || i_v < n_it || i_s < n_it) {
         bool progress = false;
-        if (i_s < n_it && mbar_try(bar(S_FREE0 + s_stage(i_s)), s_phase(i_s) ^ 1)) {
+        // (two stages: the second item's state is not asked for before the first item's operands
+        // have landed -- at the start of a launch every CTA's first loads share the memory system)
+        if (i_s < n_it && (!SMALL || i_s != 1 || (mbar_try(bar(S_FULL0), 0) && mbar_try(bar(QK_FULL), 0))) &&
+            mbar_try(bar(S_FREE0 + s_stage(i_s)), s_phase(i_s) ^ 1)) {
           const int sj = s_stage(i_s);
           const int item = (int)(blockIdx.x + i_s * gridDim.x);
           mbar_expect_tx(bar(S_FULL0 + sj), 4 * kTile);
