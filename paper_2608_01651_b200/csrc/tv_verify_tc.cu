@@ -1,6 +1,7 @@
 // Tree verification on the 5th-generation tensor cores (tcgen05 + TMEM + TMA).
 //
-// Shapes: bf16 q/k/v, fp32 state, dk = dv = 128, T <= 128, gated rule.
+// Shapes: bf16 q/k/v, fp32 state, dk = dv = 128 (or 64, dense layouts), T <= 128, gated rule.
+// The text below is written for 128.
 // One persistent CTA per SM walks (layer, request, head) items.  Per item
 // (Theorem 1 / Eq. 4 with U = V):
 //
@@ -253,7 +254,9 @@ __device__ __forceinline__ void store_box(const CUtensorMap* m, uint32_t src, bo
 // other requests and are masked like padding); stores are cut to the request's node count:
 // 8-row-aligned part by TMA boxes of 64/32/16/8 rows (tmO, tmO32, tmO16, tmO8), the last < 8
 // rows straight from registers.  The dense instantiation ignores the three extra maps.
-template <bool PACKED, bool SMALL>
+// D = dk = dv, 128 or 64.  D = 64 keeps the shared-memory map of D = 128 and uses the first k half,
+// the first dv half and the first 64 rows of the state tiles.
+template <bool PACKED, bool SMALL, int D>
 __global__ void __launch_bounds__(kThreads, 1)
 verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constant__ CUtensorMap tmS,
                        const __grid_constant__ CUtensorMap tmO, const __grid_constant__ CUtensorMap tmO32,
@@ -262,6 +265,9 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
   using L = Lay<SMALL>;
   constexpr uint32_t kBox = L::kBox;
   constexpr int kBoxRows = SMALL ? 64 : 128;
+  constexpr int NH = D / 64;    // 64-wide halves of a q / k / v row
+  constexpr int NC = D / 32;    // 32-float chunks of a state row and of an output row
+  constexpr uint32_t kIdescPrefix = idesc_bf16(D, false), kIdescReadout = idesc_bf16(D, true);
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   unsigned char* sm = smem_raw;
   const uint32_t sbase = smem_u32(sm);
@@ -352,9 +358,9 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
             mbar_try(bar(S_FREE0 + s_stage(i_s)), s_phase(i_s) ^ 1)) {
           const int sj = s_stage(i_s);
           const int item = (int)(blockIdx.x + i_s * gridDim.x);
-          mbar_expect_tx(bar(S_FULL0 + sj), 4 * kTile);
+          mbar_expect_tx(bar(S_FULL0 + sj), NC * D * 128);
 #pragma unroll 1
-          for (int c = 0; c < 4; ++c)
+          for (int c = 0; c < NC; ++c)
             tma_load_3d(sbase + L::kOffS + (uint32_t)(sj * 4 + c) * kTile, &tmS, bar(S_FULL0 + sj), 32 * c, 0, item);
           pend_s[sj] = 1 + (int)s_phase(i_s);
           ++i_s;
@@ -365,11 +371,12 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
           // rows of the boxes of this item (the tile layout in shared memory does not depend on it)
           const int bc = PACKED ? box_class(ic.n, kBoxRows) : 2;
           const uint32_t box_bytes = kBox >> (2 - bc);
-          mbar_expect_tx(bar(QK_FULL), 4 * box_bytes);
+          mbar_expect_tx(bar(QK_FULL), 2 * NH * box_bytes);
 #pragma unroll 1
           for (uint32_t i = 0; i < 4; ++i)   // q: k halves 0, 1; k: k halves 0, 1 (consecutive boxes)
-            load_box(sbase + L::kOffQ + i * kBox, i < 2 ? &lm.q[bc] : &lm.k[bc], bar(QK_FULL), nf_qk,
-                     (int)(i & 1u) * 64, ic.y0, ic.h_qk, ic.z);
+            if ((int)(i & 1u) < NH)
+              load_box(sbase + L::kOffQ + i * kBox, i < 2 ? &lm.q[bc] : &lm.k[bc], bar(QK_FULL), nf_qk,
+                       (int)(i & 1u) * 64, ic.y0, ic.h_qk, ic.z);
           pend_qk = 1 + (int)(i_qk & 1);
           ++i_qk;
           progress = true;
@@ -378,9 +385,9 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
           const ItemCoord ic = item_coord<PACKED>(p, (int)(blockIdx.x + i_v * gridDim.x));
           const int bc = PACKED ? box_class(ic.n, kBoxRows) : 2;
           const uint32_t box_bytes = kBox >> (2 - bc);
-          mbar_expect_tx(bar(V_FULL), 2 * box_bytes);
+          mbar_expect_tx(bar(V_FULL), NH * box_bytes);
 #pragma unroll 1
-          for (uint32_t i = 0; i < 2; ++i)
+          for (uint32_t i = 0; i < NH; ++i)
             load_box(sbase + L::kOffV + i * kBox, &lm.v[bc], bar(V_FULL), nf_v, (int)i * 64, ic.y0, ic.h_v, ic.z);
           pend_v = 1 + (int)(i_v & 1);
           ++i_v;
@@ -433,8 +440,8 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
         // scores = Q K^T
         if (!wait_list(W(QK_FULL, ph) | W(SC_FREE, ph ^ 1) << 6, 2)) break;
         tc_fence_after();
-#pragma unroll(SMALL ? 8 : 1)
-        for (uint32_t i = 0; i < 8; ++i) {   // k half i >> 2, 16 contraction indices (32 bytes) per step
+#pragma unroll(SMALL ? 4 * NH : 1)
+        for (uint32_t i = 0; i < 4 * NH; ++i) {   // k half i >> 2, 16 contraction indices (32 bytes) per step
           const uint32_t off = ((i >> 2) * kBox + (i & 3u) * 32u) >> 4;
           mma_bf16_ss(tmem + kColSc, dQ + off, dK + off, SMALL ? kIdescKK64 : kIdescKK128, i);
         }
@@ -448,11 +455,11 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
         mbar_arrive(bar(META_FREE0 + (int)ph));
         if (!wait_list(W(ACC_FREE0 + (int)ph, ph2 ^ 1) | W(QS_READY0 + (int)ph, ph2) << 6, rescaled ? 2 : 1)) break;
         tc_fence_after();
-#pragma unroll(SMALL ? 16 : 1)
-        for (uint32_t i = 0; i < 16; ++i) {   // tile i >> 2 of the stage = (k half, hi | lo)
+#pragma unroll(SMALL ? 8 * NH : 1)
+        for (uint32_t i = 0; i < 8 * NH; ++i) {   // tile i >> 2 of the stage = (k half, hi | lo)
           const uint32_t off = (((uint32_t)st * 4u + (i >> 2)) * kTile + (i & 3u) * 32u) >> 4;
           mma_bf16_ts(tmem + acc_col, tmem + kColQb + ph * 64 + (i >> 3) * 32 + (i & 3u) * 8, dS + off,
-                      kIdescKK128, i);
+                      kIdescPrefix, i);
         }
         tc_commit(bar(S_FREE0 + st));
         // acc += C'_hi V + C'_lo V
@@ -464,8 +471,8 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
           for (uint32_t i = 0; i < 4; ++i) {
             const uint64_t bdesc = dV + (((jh * 4u + i) * 2048u) >> 4);
             const uint32_t off = (jh * kTile + i * 32u) >> 4;
-            mma_bf16_ss(tmem + acc_col, dChi + off, bdesc, kIdescKMn, 1);
-            mma_bf16_ss(tmem + acc_col, dClo + off, bdesc, kIdescKMn, 1);
+            mma_bf16_ss(tmem + acc_col, dChi + off, bdesc, kIdescReadout, 1);
+            mma_bf16_ss(tmem + acc_col, dClo + off, bdesc, kIdescReadout, 1);
           }
         tc_commit(bar(V_FREE));
         tc_commit(bar(ACC_DONE0 + (int)ph));
@@ -492,7 +499,7 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
           auto put = [&](const CUtensorMap* m, int rows_box) {
             while (full - r >= rows_box) {
 #pragma unroll
-              for (int c = 0; c < 4; ++c)
+              for (int c = 0; c < NC; ++c)
                 store_box(m, sbase + L::kOffStage + c * L::kStageChunk + (uint32_t)r * 128u, nf_o, 32 * c,
                           ic.y0 + r, ic.h_v, ic.z);
               r += rows_box;
@@ -504,7 +511,7 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
           put(&tmO8, 8);
         } else {
 #pragma unroll
-          for (int c = 0; c < 4; ++c)
+          for (int c = 0; c < NC; ++c)
             store_box(&tmO, sbase + L::kOffStage + c * L::kStageChunk, nf_o, 32 * c, 0, ic.h_v, ic.z);
         }
         tma_store_commit();
@@ -631,7 +638,7 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
       tc_fence_after();
       if (pw * 32 < T) {
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
+        for (int half = 0; half < NH; ++half) {
           const unsigned char* qrow = sm + L::kOffQ + half * kBox + row * 128;
           uint32_t r[32];
 #pragma unroll
@@ -652,8 +659,10 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
       // ---- the state split ----
       if (!mbar_wait_warp(bar(S_FULL0 + st), s_phase(it), abort_flag)) break;
       unsigned char* s_buf = sm + L::kOffS + (uint32_t)st * 4u * kTile;
+      if (row < D) {   // state rows v < dv
 #pragma unroll 1
-      for (int half = 0; half < 2; ++half) split_state_row(s_buf, row, half, swz);   // one copy of the code
+        for (int half = 0; half < NH; ++half) split_state_row(s_buf, row, half, swz);   // one copy of the code
+      }
       fence_async_smem();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(S_CONV0 + st));
@@ -685,16 +694,16 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
       tc_fence_after();
       if (warp_live) {
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
+        for (int half = 0; half < NH; ++half) {   // this warp's D / 2 columns, 32 at a time
           uint32_t r1[32];
-          tmem_ld32(tmem + lane_addr + acc_col + hc * 64 + half * 32, r1);
+          tmem_ld32(tmem + lane_addr + acc_col + hc * (D / 2) + half * 32, r1);
           tmem_wait_ld();
-          unsigned char* orow = sm + L::kOffStage + (hc * 2 + half) * L::kStageChunk + row * 128;
+          unsigned char* orow = sm + L::kOffStage + (hc * NH + half) * L::kStageChunk + row * 128;
           // packed forest: the rows after the last full group of 8 leave from registers
           const bool tail_row = PACKED && row >= (pk_prev.n & ~7) && row < pk_prev.n;
           float* otail = nullptr;
           if constexpr (PACKED)
-            otail = p.O + ((size_t)pk_prev.plane_v * p.capacity + pk_prev.row0 + row) * 128 + hc * 64 + half * 32;
+            otail = p.O + ((size_t)pk_prev.plane_v * p.capacity + pk_prev.row0 + row) * D + hc * (D / 2) + half * 32;
 #pragma unroll
           for (int c = 0; c < 8; ++c) {
             float4 o;
@@ -789,7 +798,7 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
         // extreme decay: replace the q rows that the operand warps copied to TMEM by scaled ones
         if (!(ok = mbar_wait_warp(bar(QB_READY0 + (int)ph), (it >> 1) & 1, abort_flag))) break;
         tc_fence_after();
-        if (warp_live) {
+        if (warp_live && hc < NH) {
           uint32_t r[32];
           tmem_ld32(tmem + lane_addr + kColQb + ph * 64 + hc * 32, r);
           tmem_wait_ld();
@@ -860,7 +869,7 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
         const int rows_loaded = kBoxRows >> (2 - box_class(pk.n, kBoxRows));
         if (pk.row0 + rows_loaded > total_rows) {
           if (!(ok = mbar_wait_warp(bar(V_FULL), ph, abort_flag))) break;
-          if (row >= total_rows - pk.row0 && row < rows_loaded) {
+          if (row >= total_rows - pk.row0 && row < rows_loaded && hc < NH) {
             uint4* vrow = reinterpret_cast<uint4*>(sm + L::kOffV + hc * kBox + row * 128);
 #pragma unroll
             for (int c = 0; c < 8; ++c) vrow[c] = make_uint4(0u, 0u, 0u, 0u);
@@ -897,11 +906,11 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
 // Gated rule: the correction rows are the values themselves (U = V), widened to float.  One
 // thread per 8 channels of a node row; rows addressed through the strides of v and of U.
 __global__ void widen_rows_kernel(const __nv_bfloat16* __restrict__ v, float* __restrict__ U, int n_lb, int H, int T,
-                                  Str3 sv, Str3 so) {
-  const size_t n = (size_t)n_lb * H * T * 16;
+                                  int groups, Str3 sv, Str3 so) {   // groups = dv / 8
+  const size_t n = (size_t)n_lb * H * T * groups;
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
-    const int c8 = (int)(i & 15);
-    size_t r = i >> 4;
+    const int c8 = (int)(i % groups);
+    size_t r = i / groups;
     const int t = (int)(r % T);
     r /= T;
     const int h = (int)(r % H);
@@ -969,7 +978,9 @@ extern "C" __attribute__((visibility("default"))) int tv_selftest_wait_timeout(i
 }
 
 bool tv_verify_tc_supports(const VerifyArgs& a) {
-  return a.bf16 && a.dk == 128 && a.dv == 128 && a.rule == TV_GATED && a.T <= 128;
+  const bool d128 = a.dk == 128 && a.dv == 128;
+  const bool d64 = a.dk == 64 && a.dv == 64 && a.tree.offsets == nullptr;   // dense layouts only
+  return a.bf16 && (d128 || d64) && a.rule == TV_GATED && a.T <= 128;
 }
 
 int tv_launch_verify_tc(const VerifyArgs& a, int32_t* status, cudaStream_t stream) {
@@ -978,13 +989,14 @@ int tv_launch_verify_tc(const VerifyArgs& a, int32_t* status, cudaStream_t strea
   const bool small = a.T <= 64;
   const uint64_t items = (uint64_t)a.L * a.B * a.H;
   const uint32_t rows = small ? 64 : 128;    // rows of an operand box and of a staged output chunk
+  const uint32_t D = (uint32_t)a.dk;         // = dv
   // 4-D views: dense / strided layouts from the resolved strides, packed forests as planes
   NodeView vq, vv, vo;
   if (!packed) {
     const uint64_t lb = (uint64_t)a.L * a.B;
-    vq = NodeView{128, (uint64_t)a.T, (uint64_t)a.Hk, lb, a.lay.qk.b, a.lay.qk.h, a.lay.qk.t};
-    vv = NodeView{128, (uint64_t)a.T, (uint64_t)a.H, lb, a.lay.v.b, a.lay.v.h, a.lay.v.t};
-    vo = NodeView{128, (uint64_t)a.T, (uint64_t)a.H, lb, a.lay.out.b, a.lay.out.h, a.lay.out.t};
+    vq = NodeView{D, (uint64_t)a.T, (uint64_t)a.Hk, lb, a.lay.qk.b, a.lay.qk.h, a.lay.qk.t};
+    vv = NodeView{D, (uint64_t)a.T, (uint64_t)a.H, lb, a.lay.v.b, a.lay.v.h, a.lay.v.t};
+    vo = NodeView{D, (uint64_t)a.T, (uint64_t)a.H, lb, a.lay.out.b, a.lay.out.h, a.lay.out.t};
   } else {
     const int64_t cap = a.tree.capacity;
     vq = NodeView{128, (uint64_t)cap, (uint64_t)a.Hk, (uint64_t)a.L, (int64_t)a.Hk * cap * 128, cap * 128, 128};
@@ -998,7 +1010,7 @@ int tv_launch_verify_tc(const VerifyArgs& a, int32_t* status, cudaStream_t strea
     return make_map4(&m[0], a.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, vq, 64, rows) &&
            make_map4(&m[1], a.k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, vq, 64, rows) &&
            make_map4(&m[2], a.v, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, vv, 64, rows) &&
-           make_map(&m[3], a.S_pre, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, 128, 128, 32) &&
+           make_map(&m[3], a.S_pre, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, D, D, 32, D) &&
            make_map4(&m[4], a.O, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, vo, 32, packed ? 64 : rows);
   });
   const MapSet* mo = ms;   // packed forest: output boxes of 32, 16 and 8 rows
@@ -1037,13 +1049,17 @@ int tv_launch_verify_tc(const VerifyArgs& a, int32_t* status, cudaStream_t strea
   int dev = 0;
   TV_CUDA_TRY(cudaGetDevice(&dev));
   if (configured_dev != dev) {
-    TV_CUDA_TRY(cudaFuncSetAttribute(verify_tc_gated_kernel<false, false>,
+    TV_CUDA_TRY(cudaFuncSetAttribute(verify_tc_gated_kernel<false, false, 128>,
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Lay<false>::kSmemBytes));
-    TV_CUDA_TRY(cudaFuncSetAttribute(verify_tc_gated_kernel<true, false>,
+    TV_CUDA_TRY(cudaFuncSetAttribute(verify_tc_gated_kernel<true, false, 128>,
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Lay<false>::kSmemBytes));
-    TV_CUDA_TRY(cudaFuncSetAttribute(verify_tc_gated_kernel<false, true>,
+    TV_CUDA_TRY(cudaFuncSetAttribute(verify_tc_gated_kernel<false, true, 128>,
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Lay<true>::kSmemBytes));
-    TV_CUDA_TRY(cudaFuncSetAttribute(verify_tc_gated_kernel<true, true>,
+    TV_CUDA_TRY(cudaFuncSetAttribute(verify_tc_gated_kernel<true, true, 128>,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Lay<true>::kSmemBytes));
+    TV_CUDA_TRY(cudaFuncSetAttribute(verify_tc_gated_kernel<false, false, 64>,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Lay<false>::kSmemBytes));
+    TV_CUDA_TRY(cudaFuncSetAttribute(verify_tc_gated_kernel<false, true, 64>,
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Lay<true>::kSmemBytes));
     TV_CUDA_TRY(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev));
     configured_dev = dev;
@@ -1068,7 +1084,7 @@ int tv_launch_verify_tc(const VerifyArgs& a, int32_t* status, cudaStream_t strea
     return launch_dependent(kernel, grid, kThreads, smem, stream, lm, ms->map[3], ms->map[4], mo->map[packed ? 0 : 4], mo->map[packed ? 1 : 4], mo->map[packed ? 2 : 4], p);
   };
   if (packed) {
-    TV_CUDA_TRY(small ? go(verify_tc_gated_kernel<true, true>) : go(verify_tc_gated_kernel<true, false>));
+    TV_CUDA_TRY(small ? go(verify_tc_gated_kernel<true, true, 128>) : go(verify_tc_gated_kernel<true, false, 128>));
     if (a.U) {
       const size_t planes = (size_t)a.L * a.H;
       widen_bf16_rows_kernel<<<dim3(64, (unsigned)(planes < 65535 ? planes : 65535)), 256, 0, stream>>>(
@@ -1077,12 +1093,15 @@ int tv_launch_verify_tc(const VerifyArgs& a, int32_t* status, cudaStream_t strea
     }
     return TV_OK;
   }
-  TV_CUDA_TRY(small ? go(verify_tc_gated_kernel<false, true>) : go(verify_tc_gated_kernel<false, false>));
+  if (D == 64)
+    TV_CUDA_TRY(small ? go(verify_tc_gated_kernel<false, true, 64>) : go(verify_tc_gated_kernel<false, false, 64>));
+  else
+    TV_CUDA_TRY(small ? go(verify_tc_gated_kernel<false, true, 128>) : go(verify_tc_gated_kernel<false, false, 128>));
   if (a.U) {
-    const size_t n = items * a.T * 16;
+    const size_t n = items * a.T * (D / 8);
     const int blocks = (int)((n + 255) / 256 < 4096 ? (n + 255) / 256 : 4096);
     widen_rows_kernel<<<blocks, 256, 0, stream>>>(reinterpret_cast<const __nv_bfloat16*>(a.v), a.U, a.L * a.B, a.H,
-                                                  a.T, a.lay.v, a.lay.out);
+                                                  a.T, (int)(D / 8), a.lay.v, a.lay.out);
     TV_CUDA_TRY(cudaGetLastError());
   }
   return TV_OK;

@@ -20,17 +20,19 @@ IMPLS = [tv.IMPL_SIMT, tv.IMPL_TC]
 
 
 def _tc_ok(wl, parents=None):
-    if not (wl.qkv_dtype == inputs.BF16 and wl.dk == 128 and wl.dv == 128):
+    if wl.qkv_dtype != inputs.BF16 or wl.dk != wl.dv:
         return False
     if wl.rule == inputs.GATED:
-        return True
+        return wl.dk in (64, 128)
+    if wl.dk != 128:
+        return False
     depth = max(int(inputs.node_depths(p).max()) for p in parents) if parents is not None else 0
     return depth <= 15
 
 
 def _skip_unless_supported(wl, impl, parents=None):
     if impl == tv.IMPL_TC and not _tc_ok(wl, parents):
-        pytest.skip("tensor-core kernels cover bf16, dk = dv = 128 (delta rule: tree depth <= 15)")
+        pytest.skip("tensor-core kernels cover bf16, dk = dv = 128 (gated rule also 64; delta rule: tree depth <= 15)")
 
 
 def _run(wl, parents, accepted, tens, tol, items=None, **kw):
@@ -108,6 +110,10 @@ EDGE = [
     (40, 64, 128, 2, 2, "frontier", False),    # dk != dv
     (40, 128, 64, 2, 2, "frontier", False),
     (33, 32, 96, 1, 2, "frontier", True),
+    (63, 64, 64, 2, 3, "frontier", False),     # 64-wide heads on the tensor cores (gated rule)
+    (64, 64, 64, 3, 2, "binary", True),
+    (100, 64, 64, 2, 2, "spine", False),
+    (128, 64, 64, 1, 3, "frontier", False),
 ]
 
 
