@@ -23,6 +23,12 @@ the channel order is [q heads | k heads | v heads]; the normalisation that the
 paper folds into its stages without a formula is read as an optional L2
 normalisation of each q and k head vector after SiLU, x / sqrt(sum x^2 + eps);
 the gate formulas are not given by the paper either (see gate_prep below).
+
+Pins.  tree_conv and conv_commit are pinned by what the definition fixes (hand
+example, numpy.convolve on chains, path locality, ...).  gate_prep and the
+normalisation are readings: their tests fix the reading against library
+softplus / sigmoid and closed forms, but nothing in the paper fixes the formula
+itself -- parity of gate_prep is UNPINNED BY THE PAPER.
 """
 from __future__ import annotations
 
