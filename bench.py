@@ -594,7 +594,7 @@ def kernel_split(rig, step_ms, n, peak):
     for obj, nbytes in ((verify, rig.vbytes), (commit, rig.cbytes)):
         y = copy_yardstick(rig.dev, stream, nbytes)
         y["frac_of_measured_copy"] = y["GBps"] / peak
-        y["kernel_back_to_back_vs_this_copy"] = y["ms"] / obj["back_to_back_ms"]
+        y["kernel_back_to_back_vs_this_copy"] = (nbytes / (obj["back_to_back_ms"] * 1e-3) / 1e9) / y["GBps"]   # rates
         obj["copy_of_same_bytes"] = y
     return verify, commit
 
