@@ -90,10 +90,10 @@ typedef struct tv_dims {
   int32_t qkv_dtype;   /* TV_F32 / TV_BF16                                      */
   int32_t impl;        /* TV_IMPL_AUTO picks a tensor-core kernel when the
                           shape allows it (bf16, dk = dv = 128; gated rule
-                          also dk = dv = 64 in dense layouts; delta rule only
-                          dense layouts and tree depth <= 15) and the SIMT fp32
-                          kernel otherwise; TV_IMPL_TC returns
-                          TV_ERR_UNSUPPORTED instead of falling back            */
+                          also dk = dv = 64 in dense layouts; delta rule: tree
+                          depth <= 15) and the SIMT fp32 kernel otherwise;
+                          TV_IMPL_TC returns TV_ERR_UNSUPPORTED instead of
+                          falling back                                          */
   int32_t Hk;          /* grouped key heads (Section IV-D: a K factor shared by
                           several state heads is stored once): q and k have Hk
                           heads, [L][B][Hk][T][dk], and state head h reads

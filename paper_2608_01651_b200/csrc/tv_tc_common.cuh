@@ -102,6 +102,19 @@ __device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, uint32_t sr
       "cp.async.bulk.tensor.4d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
       ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
 }
+// A box of a 4-D map (channel, node | head, head | node, outermost): the two middle coordinates
+// are ordered by stride when the map is built (make_map4), `node_first` says which way.
+__device__ __forceinline__ void load_box(uint32_t dst, const CUtensorMap* m, uint32_t bar, bool node_first, int x,
+                                         int y, int h, int z) {
+  if (node_first) tma_load_4d(dst, m, bar, x, y, h, z);
+  else tma_load_4d(dst, m, bar, x, h, y, z);
+}
+__device__ __forceinline__ void store_box(const CUtensorMap* m, uint32_t src, bool node_first, int x, int y, int h,
+                                          int z) {
+  if (node_first) tma_store_4d(m, src, x, y, h, z);
+  else tma_store_4d(m, src, x, h, y, z);
+}
+
 __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
@@ -299,11 +312,7 @@ __device__ __forceinline__ PackedItem packed_item(const int32_t* offsets, int B,
   r.n = offsets[r.b + 1] - r.row0;
   return r;
 }
-// dense layout: the q/k item of state item `item`, and the tree of its request
-__device__ __forceinline__ int qk_item(int item, int H, int Hk, const ItemDiv& d) {
-  const int lb = (int)fdiv((uint32_t)item, d.dH), h = item - lb * H;
-  return lb * Hk + (int)fdiv((uint32_t)h, d.dG);
-}
+// dense layout: the tree of the request that item `item` belongs to
 __device__ __forceinline__ int request_of(int item, int B, const ItemDiv& d) {
   const int lb = (int)fdiv((uint32_t)item, d.dH);
   return lb - (int)fdiv((uint32_t)lb, d.dB) * B;

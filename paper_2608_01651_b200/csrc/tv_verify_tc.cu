@@ -238,17 +238,6 @@ __device__ __forceinline__ ItemCoord item_coord(const TcParams& p, int item) {
   }
   return c;
 }
-__device__ __forceinline__ void load_box(uint32_t dst, const CUtensorMap* m, uint32_t bar, bool node_first, int x,
-                                         int y, int h, int z) {
-  if (node_first) tma_load_4d(dst, m, bar, x, y, h, z);
-  else tma_load_4d(dst, m, bar, x, h, y, z);
-}
-__device__ __forceinline__ void store_box(const CUtensorMap* m, uint32_t src, bool node_first, int x, int y, int h,
-                                          int z) {
-  if (node_first) tma_store_4d(m, src, x, y, h, z);
-  else tma_store_4d(m, src, x, h, y, z);
-}
-
 // PACKED = packed forest: q/k/v/O are planes of `capacity` rows and an item's rows start at its
 // request's offset.  Loads take the fixed box at that offset (rows past the request belong to
 // other requests and are masked like padding); stores are cut to the request's node count:

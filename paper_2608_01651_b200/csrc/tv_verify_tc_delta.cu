@@ -86,6 +86,10 @@ struct DeltaParams {
   const int32_t* offsets;
   int32_t capacity;
   ItemDiv div;   // divisions by H, B, H / Hk as multiply-shift
+  Str3 gate;     // strides of alpha and beta (dense layouts)
+  // The q, k, v, O, U maps are 4-D, (channel, node, head, layer*request) or (channel, head, node, ...)
+  // whichever has ascending strides: bit 0 / 1 / 2 set = q,k / v / O,U take the node coordinate first.
+  int32_t node_first;
   float* O;
   float* U;
 };
@@ -130,6 +134,26 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int T = p.T;
   const bool want_U = p.want_U != 0;
+  const bool nf_qk = p.node_first & 1, nf_v = p.node_first & 2, nf_o = p.node_first & 4;
+  // box coordinates of an item: q/k head, v/O/U head, outermost index (layer*request, or the layer
+  // of a packed forest) and the first node row
+  struct Coord {
+    int hq, h, z, y0;
+  };
+  auto coord_of = [&](int item) -> Coord {
+    Coord c;
+    const int lb = (int)fdiv((uint32_t)item, p.div.dH);
+    c.h = item - lb * p.H;
+    c.hq = (int)fdiv((uint32_t)c.h, p.div.dG);
+    c.z = lb;
+    c.y0 = 0;
+    if constexpr (PACKED) {
+      const int l = (int)fdiv((uint32_t)lb, p.div.dB);
+      c.z = l;
+      c.y0 = p.offsets[lb - l * p.B];
+    }
+    return c;
+  };
 
   if (tid == 0) {
     abort_flag[0] = 0;
@@ -175,17 +199,11 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         const int qfull = qb ? QK_FULL1 : QK_FULL, qfree = qb ? QK_FREE1 : QK_FREE;
         if (!mbar_wait(bar(qfree), qph ^ 1, abort_flag)) break;
         mbar_expect_tx(bar(qfull), 4 * 8192);
-        int qk = 0, vplane = item, y0 = 0;
-        if constexpr (PACKED) {
-          const PackedItem pi = packed_item(p.offsets, p.B, p.H, p.Hk, item, p.div);
-          qk = pi.plane_qk; vplane = pi.plane_v; y0 = pi.row0;
-        } else {
-          qk = qk_item(item, p.H, p.Hk, p.div);
-        }
-        tma_load_3d(sbase + qk_base, &tmQ, bar(qfull), 0, y0, qk);
-        tma_load_3d(sbase + qk_base + kTile, &tmQ, bar(qfull), 64, y0, qk);
-        tma_load_3d(sbase + qk_base + 8192, &tmK, bar(qfull), 0, y0, qk);
-        tma_load_3d(sbase + qk_base + kTile + 8192, &tmK, bar(qfull), 64, y0, qk);
+        const Coord co = coord_of(item);
+        load_box(sbase + qk_base, &tmQ, bar(qfull), nf_qk, 0, co.y0, co.hq, co.z);
+        load_box(sbase + qk_base + kTile, &tmQ, bar(qfull), nf_qk, 64, co.y0, co.hq, co.z);
+        load_box(sbase + qk_base + 8192, &tmK, bar(qfull), nf_qk, 0, co.y0, co.hq, co.z);
+        load_box(sbase + qk_base + kTile + 8192, &tmK, bar(qfull), nf_qk, 64, co.y0, co.hq, co.z);
         pend_qk_bar = qfull;
         pend_qk = 1 + (int)qph;
         if (!mbar_wait(bar(S_FREE), ph ^ 1, abort_flag)) break;
@@ -196,8 +214,8 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         pend_s = 1 + (int)ph;
         if (!mbar_wait(bar(V_FREE), ph ^ 1, abort_flag)) break;
         mbar_expect_tx(bar(V_FULL), 2 * 8192);
-        tma_load_3d(sbase + kOffV, &tmV, bar(V_FULL), 0, y0, vplane);
-        tma_load_3d(sbase + kOffV + kTile, &tmV, bar(V_FULL), 64, y0, vplane);
+        load_box(sbase + kOffV, &tmV, bar(V_FULL), nf_v, 0, co.y0, co.h, co.z);
+        load_box(sbase + kOffV + kTile, &tmV, bar(V_FULL), nf_v, 64, co.y0, co.h, co.z);
         pend_v = 1 + (int)ph;
       }
       if (*abort_flag) {
@@ -284,6 +302,7 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       uint32_t it = 0;
       for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++it) {
         if (!mbar_wait(bar(OST_READY), it & 1, abort_flag)) break;
+        const Coord co = coord_of(item);
         if constexpr (PACKED) {
           // groups of 8 rows, largest boxes first (staging rows start on 1024-byte boundaries)
           const PackedItem pi = packed_item(p.offsets, p.B, p.H, p.Hk, item, p.div);
@@ -295,8 +314,8 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
               while (full - r >= rows_box) {
 #pragma unroll
                 for (int c = 0; c < 4; ++c)
-                  tma_store_3d(m, sbase + kOffStage + (part * 4 + c) * 8192 + (uint32_t)r * 128u, 32 * c,
-                               pi.row0 + r, pi.plane_v);
+                  store_box(m, sbase + kOffStage + (part * 4 + c) * 8192 + (uint32_t)r * 128u, nf_o, 32 * c,
+                            co.y0 + r, co.h, co.z);
                 r += rows_box;
               }
             };
@@ -307,10 +326,10 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           }
         } else {
 #pragma unroll
-          for (int c = 0; c < 4; ++c) tma_store_3d(&tmO, sbase + kOffStage + c * 8192, 32 * c, 0, item);
+          for (int c = 0; c < 4; ++c) store_box(&tmO, sbase + kOffStage + c * 8192, nf_o, 32 * c, 0, co.h, co.z);
           if (want_U) {
 #pragma unroll
-            for (int c = 0; c < 4; ++c) tma_store_3d(&tmU, sbase + kOffStage + (4 + c) * 8192, 32 * c, 0, item);
+            for (int c = 0; c < 4; ++c) store_box(&tmU, sbase + kOffStage + (4 + c) * 8192, nf_o, 32 * c, 0, co.h, co.z);
           }
         }
         tma_store_commit();
@@ -329,14 +348,17 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       const uint32_t buf = j & 1, use = j >> 1;
       if (use > 0 && !mbar_wait_warp(bar(buf ? META_FREE1 : META_FREE), (use - 1) & 1, abort_flag)) break;
       int n = T, tb = 0;
-      size_t g0 = (size_t)item * T;                     // first gate of the item
+      int64_t g0, gstep = 1;                            // first gate of the item, step between nodes
       if constexpr (PACKED) {
         const PackedItem pi = packed_item(p.offsets, p.B, p.H, p.Hk, item, p.div);
         n = pi.n;
         tb = pi.b;
-        g0 = (size_t)pi.plane_v * p.capacity + pi.row0;
+        g0 = (int64_t)pi.plane_v * p.capacity + pi.row0;
       } else {
+        const int lb = (int)fdiv((uint32_t)item, p.div.dH);
         tb = p.tree.n_trees == 1 ? 0 : request_of(item, p.B, p.div);
+        g0 = (int64_t)lb * p.gate.b + (int64_t)(item - lb * p.H) * p.gate.h;
+        gstep = p.gate.t;
       }
       float* tab = tab_s + buf * (2 * kRows);
       // all six loads first: one trip to memory, not one per table
@@ -347,8 +369,8 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         const int nd = lane + 32 * h;
         if (nd < n) {
           mk[h] = __ldg(reinterpret_cast<const unsigned long long*>(p.tree.anc) + ((size_t)tb * T + nd) * 2);
-          al[h] = __ldg(p.alpha + g0 + nd);
-          be[h] = __ldg(p.beta + g0 + nd);
+          al[h] = __ldg(p.alpha + g0 + nd * gstep);
+          be[h] = __ldg(p.beta + g0 + nd * gstep);
         }
       }
 #pragma unroll
@@ -639,7 +661,7 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
 
 bool tv_verify_tc_delta_supports(const VerifyArgs& a) {
   return a.bf16 && a.dk == 128 && a.dv == 128 && a.rule == TV_GATED_DELTA && a.T <= kRows &&
-         a.tree.max_depth_all < kSlots && tv_layout_is_dense(a);
+         a.tree.max_depth_all < kSlots;
 }
 
 int tv_launch_verify_tc_delta(const VerifyArgs& a, int32_t* status, cudaStream_t stream) {
@@ -650,39 +672,42 @@ int tv_launch_verify_tc_delta(const VerifyArgs& a, int32_t* status, cudaStream_t
   float* Uout = a.U ? a.U : a.O;
   const void* const ptrs[5] = {a.q, a.k, a.v, a.S_pre, a.O};
   const void* const uptrs[5] = {Uout, nullptr, nullptr, nullptr, nullptr};
-  const uint64_t qk_items = (uint64_t)a.L * a.B * a.Hk;
+  // 4-D views: dense / strided layouts from the resolved strides, packed forests as planes
+  NodeView vq, vv, vo;
+  if (!packed) {
+    const uint64_t lb = (uint64_t)a.L * a.B;
+    vq = NodeView{128, (uint64_t)a.T, (uint64_t)a.Hk, lb, a.lay.qk.b, a.lay.qk.h, a.lay.qk.t};
+    vv = NodeView{128, (uint64_t)a.T, (uint64_t)a.H, lb, a.lay.v.b, a.lay.v.h, a.lay.v.t};
+    vo = NodeView{128, (uint64_t)a.T, (uint64_t)a.H, lb, a.lay.out.b, a.lay.out.h, a.lay.out.t};
+  } else {
+    const int64_t cap = a.tree.capacity;
+    vq = NodeView{128, (uint64_t)cap, (uint64_t)a.Hk, (uint64_t)a.L, (int64_t)a.Hk * cap * 128, cap * 128, 128};
+    vv = NodeView{128, (uint64_t)cap, (uint64_t)a.H, (uint64_t)a.L, (int64_t)a.H * cap * 128, cap * 128, 128};
+    vo = vv;
+  }
+  const uint64_t key = view_key(vq) * 3 + view_key(vv) * 5 + view_key(vo) * 7 + items;
   const MapSet* ms = nullptr;   // q, k, v, S, O (64-row boxes)
   const MapSet* mu = nullptr;   // U (64-row boxes)
   const MapSet* mo2 = nullptr;  // packed forest: O boxes of 32, 16, 8 rows
   const MapSet* mu2 = nullptr;  // packed forest: U boxes of 32, 16, 8 rows
+  ms = cached_maps(ptrs, key, a.T, (packed ? 6 : 1) | (a.Hk << 8), [&](CUtensorMap* m) {
+    return make_map4(&m[0], a.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, vq, 64, 64) &&
+           make_map4(&m[1], a.k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, vq, 64, 64) &&
+           make_map4(&m[2], a.v, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, vv, 64, 64) &&
+           make_map(&m[3], a.S_pre, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, 128, 128, 32, 128) &&
+           make_map4(&m[4], a.O, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, vo, 32, 64);
+  });
   if (!packed) {
-    ms = cached_maps(ptrs, items, a.T, 1 | (a.Hk << 8), [&](CUtensorMap* m) {
-      return make_map(&m[0], a.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, qk_items, a.T, 128, 64, 64) &&
-             make_map(&m[1], a.k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, qk_items, a.T, 128, 64, 64) &&
-             make_map(&m[2], a.v, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, items, a.T, 128, 64, 64) &&
-             make_map(&m[3], a.S_pre, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, 128, 128, 32, 128) &&
-             make_map(&m[4], a.O, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, a.T, 128, 32, 64);
-    });
-    mu = cached_maps(uptrs, items, a.T, 2, [&](CUtensorMap* m) {
-      return make_map(&m[0], Uout, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, a.T, 128, 32, 64);
+    mu = cached_maps(uptrs, key, a.T, 2, [&](CUtensorMap* m) {
+      return make_map4(&m[0], Uout, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, vo, 32, 64);
     });
   } else {
-    const uint64_t cap = (uint64_t)a.tree.capacity;
-    const uint64_t pv = (uint64_t)a.L * a.H, pqk = (uint64_t)a.L * a.Hk;
-    const uint64_t key = (cap << 24) ^ items;
-    ms = cached_maps(ptrs, key, a.T, 6 | (a.Hk << 8), [&](CUtensorMap* m) {
-      return make_map(&m[0], a.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, pqk, cap, 128, 64, 64) &&
-             make_map(&m[1], a.k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, pqk, cap, 128, 64, 64) &&
-             make_map(&m[2], a.v, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, pv, cap, 128, 64, 64) &&
-             make_map(&m[3], a.S_pre, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, 128, 128, 32, 128) &&
-             make_map(&m[4], a.O, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, pv, cap, 128, 32, 64);
-    });
     auto small_boxes = [&](float* base) {
       return [=](CUtensorMap* m) {
-        return make_map(&m[0], base, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, pv, cap, 128, 32, 32) &&
-               make_map(&m[1], base, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, pv, cap, 128, 32, 16) &&
-               make_map(&m[2], base, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, pv, cap, 128, 32, 8) &&
-               make_map(&m[3], base, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, pv, cap, 128, 32, 64);
+        return make_map4(&m[0], base, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, vo, 32, 32) &&
+               make_map4(&m[1], base, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, vo, 32, 16) &&
+               make_map4(&m[2], base, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, vo, 32, 8) &&
+               make_map4(&m[3], base, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, vo, 32, 64);
       };
     };
     const void* const optrs[5] = {a.O, nullptr, nullptr, nullptr, (const void*)1};
@@ -727,6 +752,8 @@ int tv_launch_verify_tc_delta(const VerifyArgs& a, int32_t* status, cudaStream_t
   p.offsets = a.tree.offsets;
   p.capacity = a.tree.capacity;
   p.div = make_item_div(a.B, a.H, a.Hk);
+  p.gate = a.lay.gate;
+  p.node_first = (node_first_of(vq) ? 1 : 0) | (node_first_of(vv) ? 2 : 0) | (node_first_of(vo) ? 4 : 0);
   p.O = a.O;
   p.U = Uout;
   const int grid = (int)(items < (uint64_t)sm_count ? items : (uint64_t)sm_count);

@@ -78,6 +78,10 @@ struct Delta128Params {
   const int32_t* offsets;
   int32_t capacity;
   ItemDiv div;   // divisions by H, B, H / Hk as multiply-shift
+  Str3 gate, out;   // strides of alpha / beta and of O / U (dense layouts)
+  // The q, k, v, O, U maps are 4-D, (channel, node, head, layer*request) or (channel, head, node, ...)
+  // whichever has ascending strides: bit 0 / 1 / 2 set = q,k / v / O,U take the node coordinate first.
+  int32_t node_first;
 };
 
 // bf16 hi/lo parts of x (hi = upper 16 bits, lo = upper 16 bits of the exact remainder)
@@ -116,6 +120,26 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int T = p.T;
   const bool want_U = p.want_U != 0;
+  const bool nf_qk = p.node_first & 1, nf_v = p.node_first & 2, nf_o = p.node_first & 4;
+  // box coordinates of an item: q/k head, v/O/U head, outermost index (layer*request, or the layer
+  // of a packed forest) and the first node row
+  struct Coord {
+    int hq, h, z, y0;
+  };
+  auto coord_of = [&](int item) -> Coord {
+    Coord c;
+    const int lb = (int)fdiv((uint32_t)item, p.div.dH);
+    c.h = item - lb * p.H;
+    c.hq = (int)fdiv((uint32_t)c.h, p.div.dG);
+    c.z = lb;
+    c.y0 = 0;
+    if constexpr (PACKED) {
+      const int l = (int)fdiv((uint32_t)lb, p.div.dB);
+      c.z = l;
+      c.y0 = p.offsets[lb - l * p.B];
+    }
+    return c;
+  };
 
   if (tid == 0) {
     abort_flag[0] = 0;
@@ -152,13 +176,7 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
       grid_dependency_wait();   // inputs may come from the kernel in front (dependent launch)
       for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++it) {
         const uint32_t ph = it & 1;
-        int qk = 0, vplane = item, y0 = 0;
-        if constexpr (PACKED) {
-          const PackedItem pi = packed_item(p.offsets, p.B, p.H, p.Hk, item, p.div);
-          qk = pi.plane_qk; vplane = pi.plane_v; y0 = pi.row0;
-        } else {
-          qk = qk_item(item, p.H, p.Hk, p.div);
-        }
+        const Coord co = coord_of(item);
         if (!mbar_wait(bar(QK_FREE), ph ^ 1, abort_flag)) break;
         mbar_expect_tx(bar(QK_FULL), 8 * 8192);
 #pragma unroll
@@ -166,8 +184,8 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
 #pragma unroll
           for (int d = 0; d < 2; ++d) {    // dk half
             const uint32_t dst = sbase + (h ? kOffQK1 : kOffQK0) + d * kTile;
-            tma_load_3d(dst, &tmQ, bar(QK_FULL), 64 * d, y0 + 64 * h, qk);
-            tma_load_3d(dst + 8192, &tmK, bar(QK_FULL), 64 * d, y0 + 64 * h, qk);
+            load_box(dst, &tmQ, bar(QK_FULL), nf_qk, 64 * d, co.y0 + 64 * h, co.hq, co.z);
+            load_box(dst + 8192, &tmK, bar(QK_FULL), nf_qk, 64 * d, co.y0 + 64 * h, co.hq, co.z);
           }
         pend_qk = 1 + (int)ph;
         if (!mbar_wait(bar(S_FREE), ph ^ 1, abort_flag)) break;
@@ -182,7 +200,7 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
         for (int h = 0; h < 2; ++h)
 #pragma unroll
           for (int d = 0; d < 2; ++d)
-            tma_load_3d(sbase + kOffV + d * kTile + h * 8192, &tmV, bar(V_FULL), 64 * d, y0 + 64 * h, vplane);
+            load_box(sbase + kOffV + d * kTile + h * 8192, &tmV, bar(V_FULL), nf_v, 64 * d, co.y0 + 64 * h, co.h, co.z);
         pend_v = 1 + (int)ph;
       }
       if (*abort_flag) {
@@ -286,14 +304,20 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
       const uint32_t buf = j & 1, use = j >> 1;
       if (use > 0 && !mbar_wait_warp(bar(buf ? META_FREE1 : META_FREE), (use - 1) & 1, abort_flag)) break;
       int n = T, tb = 0;
-      size_t g0 = (size_t)item * T;   // first gate (and first output row) of the item
+      int64_t g0, gstep = 1;   // first gate of the item, step between nodes
+      size_t o0;               // element offset of the item's first output row
       if constexpr (PACKED) {
         const PackedItem pi = packed_item(p.offsets, p.B, p.H, p.Hk, item, p.div);
         n = pi.n;
         tb = pi.b;
-        g0 = (size_t)pi.plane_v * p.capacity + pi.row0;
+        g0 = (int64_t)pi.plane_v * p.capacity + pi.row0;
+        o0 = (size_t)g0 * 128;
       } else {
+        const int lb = (int)fdiv((uint32_t)item, p.div.dH), h = item - lb * p.H;
         tb = p.tree.n_trees == 1 ? 0 : request_of(item, p.B, p.div);
+        g0 = (int64_t)lb * p.gate.b + (int64_t)h * p.gate.h;
+        gstep = p.gate.t;
+        o0 = (size_t)((int64_t)lb * p.out.b + (int64_t)h * p.out.h);
       }
       float* tab = tab_s + buf * (2 * kNodes);
       // all loads first: one trip to memory, not one per table
@@ -307,8 +331,8 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
         be[h] = 0.f;
         if (nd < n) {
           mk[h] = __ldg(reinterpret_cast<const ulonglong2*>(p.tree.anc) + (size_t)tb * T + nd);
-          al[h] = __ldg(p.alpha + g0 + nd);
-          be[h] = __ldg(p.beta + g0 + nd);
+          al[h] = __ldg(p.alpha + g0 + nd * gstep);
+          be[h] = __ldg(p.beta + g0 + nd * gstep);
         }
       }
 #pragma unroll
@@ -337,8 +361,8 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
       }
       if (lane == 0) {
         item_s[buf * 4 + 0] = n;
-        item_s[buf * 4 + 1] = (int32_t)(g0 & 0xffffffffu);
-        item_s[buf * 4 + 2] = (int32_t)(g0 >> 32);
+        item_s[buf * 4 + 1] = (int32_t)(o0 & 0xffffffffu);
+        item_s[buf * 4 + 2] = (int32_t)(o0 >> 32);
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(buf ? META_FULL1 : META_FULL));
@@ -354,12 +378,13 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
         uint32_t r = 0;
         bool ok = true;
         for (int item = blockIdx.x; ok && item < p.n_items; item += gridDim.x) {
+          const Coord co = coord_of(item);
           for (int b = 0; b < 2; ++b, ++r) {
             if (!(ok = mbar_wait(bar(OST_READY), r & 1, abort_flag))) break;
 #pragma unroll
             for (int hc2 = 0; hc2 < 2; ++hc2) {
-              tma_store_3d(&tmO, sbase + kOffCoef + hc2 * 8192, 64 * hc2, kBlk * b, item);
-              if (want_U) tma_store_3d(&tmU, sbase + kOffCoef + (2 + hc2) * 8192, 64 * hc2, kBlk * b, item);
+              store_box(&tmO, sbase + kOffCoef + hc2 * 8192, nf_o, 64 * hc2, kBlk * b, co.h, co.z);
+              if (want_U) store_box(&tmU, sbase + kOffCoef + (2 + hc2) * 8192, nf_o, 64 * hc2, kBlk * b, co.h, co.z);
             }
             tma_store_commit();
             tma_store_wait_read();
@@ -386,7 +411,7 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
     if (warp == 2 && lane == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     // acc rows 0..63 -> O rows, rows 64..127 -> U rows of block pb of an item with pn nodes whose
-    // output rows start at row prow0.  Each thread owns 64 consecutive floats of one row.  Dense
+    // output rows start at element prow0.  Each thread owns 64 consecutive floats of one row.  Dense
     // layout: the first 32 go to a swizzled staging chunk in the (idle) coefficient tiles and leave
     // by TMA, the other 32 leave from registers in 32-byte stores (whole sectors); a warp-wide
     // register store touches 32 different lines and keeps the load/store unit busy for as many
@@ -409,7 +434,7 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
               *reinterpret_cast<uint4*>(orow + (((uint32_t)c ^ nswz) << 4)) =
                   make_uint4(r1[4 * c], r1[4 * c + 1], r1[4 * c + 2], r1[4 * c + 3]);
           } else if (nd < pn) {
-            float* o = (part == 0 ? p.O : p.U) + (prow0 + nd) * 128 + hc * 64 + half * 32;
+            float* o = (part == 0 ? p.O : p.U) + prow0 + (size_t)nd * (size_t)(PACKED ? 128 : p.out.t) + hc * 64 + half * 32;
 #pragma unroll
             for (int c = 0; c < 4; ++c)
               asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(o + 8 * c), "r"(r1[8 * c]),
@@ -434,9 +459,9 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
     bool ok = true;
     uint32_t n_read = 0;      // read-outs done so far (one per block, from the second block on)
     int pn = -1, pb = 0;      // block whose output is still in TMEM: nodes of its item, block,
-    size_t prow0 = 0;         // first output row of its item
+    size_t prow0 = 0;         // element offset of the first output row of its item
     int Tn = T;               // nodes of the current item
-    size_t row0 = 0;          // its first gate / output row
+    size_t row0 = 0;          // element offset of its first output row (packed forest: 128 x the row)
     for (int item = blockIdx.x; ok && item < p.n_items; item += gridDim.x, ++it) {
       const uint32_t ph = it & 1;
       const float* al_s = tab_s + ph * (2 * kNodes);
@@ -498,7 +523,7 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
           // A box that reaches past the last node of the forest brings rows nobody wrote.  They only
           // ever meet zero coefficients, but 0 x garbage need not be 0: zero the K and V rows (the B
           // operands of the coefficient MMAs) once both Gram products have read K.
-          const int lim = total_rows - (int)(row0 % (size_t)p.capacity);   // rows of the box that exist
+          const int lim = total_rows - (int)((row0 / 128) % (size_t)p.capacity);   // rows of the box that exist
           if (b == 0 && lim < kNodes) {
             if (!(ok = mbar_wait_warp(bar(GD1), ph, abort_flag))) break;
             if (!(ok = mbar_wait_warp(bar(V_FULL), ph, abort_flag))) break;
@@ -655,42 +680,46 @@ verify_tc_delta128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
 
 bool tv_verify_tc_delta128_supports(const VerifyArgs& a) {
   return a.bf16 && a.dk == 128 && a.dv == 128 && a.rule == TV_GATED_DELTA && a.T > kBlk && a.T <= kNodes &&
-         a.tree.max_depth_all < kSlots && tv_layout_is_dense(a);
+         a.tree.max_depth_all < kSlots;
 }
 
 int tv_launch_verify_tc_delta128(const VerifyArgs& a, int32_t* status, cudaStream_t stream) {
   if (!tv_verify_tc_delta128_supports(a)) return TV_ERR_UNSUPPORTED;
   const uint64_t items = (uint64_t)a.L * a.B * a.H;
-  const uint64_t qk_items = (uint64_t)a.L * a.B * a.Hk;
   const bool packed = a.tree.offsets != nullptr;
   float* Uout = a.U ? a.U : a.O;   // never written when U is not requested
   const void* const ptrs[5] = {a.q, a.k, a.v, a.S_pre, a.O};
   const void* const uptrs[5] = {Uout, nullptr, nullptr, nullptr, (const void*)3};
-  const MapSet* mu = nullptr;   // dense layout: U in boxes of 64 rows x 32 columns
-  // q, k, v in boxes of 64 rows x 64 columns (rows past the tensor read as zero), S_pre in 4 chunks
-  // of 32 columns; a packed forest addresses (layer, head) planes of `capacity` rows
-  const MapSet* ms = nullptr;
+  // 4-D views: dense / strided layouts from the resolved strides, packed forests as planes
+  NodeView vq, vv, vo;
   if (!packed) {
-    ms = cached_maps(ptrs, items, a.T, 9 | (a.Hk << 8), [&](CUtensorMap* m) {
-      return make_map(&m[0], a.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, qk_items, a.T, 128, 64, 64) &&
-             make_map(&m[1], a.k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, qk_items, a.T, 128, 64, 64) &&
-             make_map(&m[2], a.v, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, items, a.T, 128, 64, 64) &&
-             make_map(&m[3], a.S_pre, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, 128, 128, 32, 128) &&
-             make_map(&m[4], a.O, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, a.T, 128, 32, 64);
-    });
-    mu = cached_maps(uptrs, items, a.T, 11, [&](CUtensorMap* m) {
-      return make_map(&m[0], Uout, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, a.T, 128, 32, 64);
+    const uint64_t lb = (uint64_t)a.L * a.B;
+    vq = NodeView{128, (uint64_t)a.T, (uint64_t)a.Hk, lb, a.lay.qk.b, a.lay.qk.h, a.lay.qk.t};
+    vv = NodeView{128, (uint64_t)a.T, (uint64_t)a.H, lb, a.lay.v.b, a.lay.v.h, a.lay.v.t};
+    vo = NodeView{128, (uint64_t)a.T, (uint64_t)a.H, lb, a.lay.out.b, a.lay.out.h, a.lay.out.t};
+  } else {
+    const int64_t cap = a.tree.capacity;
+    vq = NodeView{128, (uint64_t)cap, (uint64_t)a.Hk, (uint64_t)a.L, (int64_t)a.Hk * cap * 128, cap * 128, 128};
+    vv = NodeView{128, (uint64_t)cap, (uint64_t)a.H, (uint64_t)a.L, (int64_t)a.H * cap * 128, cap * 128, 128};
+    vo = vv;
+  }
+  const uint64_t key = view_key(vq) * 3 + view_key(vv) * 5 + view_key(vo) * 7 + items;
+  // q, k, v in boxes of 64 rows x 64 columns (rows past the tensor read as zero), S_pre in 4 chunks
+  // of 32 columns; dense layouts: O and U in boxes of 64 rows x 32 columns (a packed forest stores
+  // from registers only)
+  const MapSet* mu = nullptr;
+  const MapSet* ms = cached_maps(ptrs, key, a.T, (packed ? 10 : 9) | (a.Hk << 8), [&](CUtensorMap* m) {
+    return make_map4(&m[0], a.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, vq, 64, 64) &&
+           make_map4(&m[1], a.k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, vq, 64, 64) &&
+           make_map4(&m[2], a.v, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, vv, 64, 64) &&
+           make_map(&m[3], a.S_pre, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, 128, 128, 32, 128) &&
+           (packed || make_map4(&m[4], a.O, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, vo, 32, 64));
+  });
+  if (!packed) {
+    mu = cached_maps(uptrs, key, a.T, 11, [&](CUtensorMap* m) {
+      return make_map4(&m[0], Uout, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, vo, 32, 64);
     });
     if (!mu) return TV_ERR_CUDA;
-  } else {
-    const uint64_t cap = (uint64_t)a.tree.capacity;
-    const uint64_t pv = (uint64_t)a.L * a.H, pqk = (uint64_t)a.L * a.Hk;
-    ms = cached_maps(ptrs, (cap << 24) ^ items, a.T, 10 | (a.Hk << 8), [&](CUtensorMap* m) {
-      return make_map(&m[0], a.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, pqk, cap, 128, 64, 64) &&
-             make_map(&m[1], a.k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, pqk, cap, 128, 64, 64) &&
-             make_map(&m[2], a.v, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, pv, cap, 128, 64, 64) &&
-             make_map(&m[3], a.S_pre, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, items, 128, 128, 32, 128);
-    });
   }
   if (!ms) return TV_ERR_CUDA;
   static thread_local int configured_dev = -1;
@@ -723,6 +752,9 @@ int tv_launch_verify_tc_delta128(const VerifyArgs& a, int32_t* status, cudaStrea
   p.offsets = a.tree.offsets;
   p.capacity = a.tree.capacity;
   p.div = make_item_div(a.B, a.H, a.Hk);
+  p.gate = a.lay.gate;
+  p.out = a.lay.out;
+  p.node_first = (node_first_of(vq) ? 1 : 0) | (node_first_of(vv) ? 2 : 0) | (node_first_of(vo) ? 4 : 0);
   const bool shallow = a.tree.max_depth_all <= 8;
   auto launch = [&](auto kernel) {
     // packed forests store from registers only: the output maps are placeholders there

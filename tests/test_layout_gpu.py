@@ -38,6 +38,10 @@ CASES = [  # name, B, H, T, rule, dtype, impl
     ("c5", 2, 3, 100, inputs.GATED, inputs.BF16, tv.IMPL_TC),
     ("c3", 3, 4, 37, inputs.GATED, inputs.BF16, tv.IMPL_SIMT),
     ("c4", 3, 4, 64, inputs.DELTA, inputs.BF16, tv.IMPL_AUTO),
+    ("c4", 3, 4, 64, inputs.DELTA, inputs.BF16, tv.IMPL_TC),
+    ("c4", 2, 3, 33, inputs.DELTA, inputs.BF16, tv.IMPL_TC),
+    ("c4", 2, 2, 100, inputs.DELTA, inputs.BF16, tv.IMPL_TC),       # the kernel for 65..128 nodes
+    ("c4", 2, 3, 128, inputs.DELTA, inputs.BF16, tv.IMPL_TC),
     ("c1", 2, 4, 15, inputs.GATED, inputs.F32, tv.IMPL_AUTO),
     ("c4", 2, 2, 40, inputs.DELTA, inputs.F32, tv.IMPL_AUTO),
 ]
@@ -67,10 +71,8 @@ def test_token_major_inputs_and_outputs(name, B, H, T, rule, dtype, impl):
     torch.cuda.synchronize()
     tree.device_status()
     assert torch.isfinite(O_buf).all() and torch.isfinite(U_buf).all()
-    if not (rule == inputs.DELTA and dtype == inputs.BF16):
-        # same kernel on both layouts (the delta tensor-core kernels take dense tensors only, the
-        # strided call runs the general kernel): identical bits
-        assert torch.equal(O, O_d) and torch.equal(U, U_d) and torch.equal(Sn, S_d)
+    # the same kernel runs on both layouts: identical bits
+    assert torch.equal(O, O_d) and torch.equal(U, U_d) and torch.equal(Sn, S_d)
     ver, com = pu.oracle_round(wl, parents, accepted, tens)
     eO, eU, eS = pu.compare(wl, O.cpu().double().numpy(), U.cpu().double().numpy(), Sn.cpu().double().numpy(),
                             ver, com)
