@@ -888,9 +888,10 @@ def main():
                     help="ncu dram bytes per verify launch to echo into roofline.traffic")
     ap.add_argument("--probe-every", type=int, default=0,
                     help="(packed-forest line only) record per-kernel CUDA events on every n-th timed step")
-    ap.add_argument("--check", action="store_true",
+    ap.add_argument("--check", action=argparse.BooleanOptionalAction, default=True,
                     help="after the timed region, compare O, U and S_new of sampled (layer, request, head) "
-                         "items of this very run with the fp64 oracle and add a 'parity' object")
+                         "items of this very run with the fp64 oracle and add a 'parity' object "
+                         "(on by default, a few seconds outside every timed region; --no-check drops it)")
     ap.add_argument("--check-items", type=int, default=8, help="sampled items per checked layer")
     ap.add_argument("--no-extras", action="store_true",
                     help="skip the throughput-scale and small-config objects of the default run")
