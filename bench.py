@@ -825,7 +825,8 @@ def run_ours(args, wl, rank, world, local_rank):
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": (("bf16 q/k/v, f32 state read by the tensor cores as a bf16 hi+lo pair (16 mantissa bits), "
                    "f32 accumulate, f32 outputs" if wl.rule_name == "gated" else
-                   "bf16 q/k/v, f32 state read as tf32 by the tensor cores, f32 accumulate, f32 outputs") if tc
+                   "bf16 q/k/v, f32 state read as tf32 by the tensor cores (mean of the cut compensated), "
+                   "f32 accumulate, f32 outputs") if tc
                   else "f32"),
         "data": "synthetic",
         "config": {
