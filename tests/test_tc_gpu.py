@@ -54,6 +54,32 @@ def test_extreme_decay(tree, mu, impl):
     assert eO <= wl.tol and eS <= wl.tol
 
 
+@pytest.mark.parametrize("T", [64, 100])
+def test_ordinary_and_extreme_decay_items_alternate_on_one_cta(T):
+    """More items than SMs, and the decay of an item depends on the pass in which a CTA meets it:
+    ordinary gates in the first pass, path products far below fp32 range in the second, ordinary
+    again in the third.  The two forms of the kernel (plain, and row exponents with a rescaled q
+    copy) then follow each other item by item on every CTA."""
+    n_sm = torch.cuda.get_device_properties(0).multi_processor_count
+    B, H = 8, 40
+    wl = inputs.workload("c5", B=B, H=H, T=T, L=1, tree="frontier", seed=91)
+    parents, accepted = inputs.make_trees(wl)
+    tens = inputs.make_tensors(wl)
+    item = torch.arange(B * H).view(B, H)
+    second_pass = ((item // n_sm) % 2 == 1)
+    g = torch.Generator().manual_seed(5)
+    harsh = torch.sigmoid(torch.randn(B, H, T, generator=g) - 14.0).clamp_min(1e-9)   # alpha ~ 1e-6: |g| > 100 from depth 5 on
+    tens["alpha"] = torch.where(second_pass[:, :, None], harsh, tens["alpha"])
+    O, U, Sn, _ = pu.gpu_round(wl, parents, accepted, tens, impl=tv.IMPL_TC, want_U=False)
+    assert np.isfinite(O).all() and np.isfinite(Sn).all()
+    picks = [(b, h) for b in range(B) for h in range(H) if (b * H + h) % 23 == 0]
+    picks += [(int(i) // H, int(i) % H) for i in (n_sm - 1, n_sm, n_sm + 1, 2 * n_sm - 1, 2 * n_sm, B * H - 1)
+              if i < B * H]
+    ver, com = pu.oracle_round(wl, parents, accepted, tens, items=sorted(set(picks)))
+    eO, _, eS = pu.compare(wl, O, None, Sn, ver, com)
+    assert eO <= wl.tol and eS <= wl.tol, (eO, eS)
+
+
 @pytest.mark.parametrize("B,H,T,tree", [(1, 1, 64, "frontier"), (1, 2, 37, "frontier"), (2, 3, 1, "chain"),
                                          (3, 4, 16, "chain"), (16, 32, 64, "frontier"), (5, 7, 50, "levels")])
 def test_tc_delta(B, H, T, tree):
