@@ -164,6 +164,28 @@ def test_tc_delta_run_to_run_identical(T):
             assert np.array_equal(U, outs[0][1])
 
 
+@pytest.mark.parametrize("T,B,H", [(64, 32, 32), (128, 20, 32), (40, 24, 20)])
+def test_tc_gated_run_to_run_identical(T, B, H):
+    """Several items per CTA, many launches back to back on the same inputs: O identical bit for
+    bit every time (the roles of the kernel hand buffers to each other through barriers only; a
+    buffer reused one hand-over too early shows up as a run that differs)."""
+    wl = inputs.workload("c5" if T > 64 else "c3", B=B, H=H, T=T, L=1, tree="frontier", seed=31 + T)
+    parents, accepted = inputs.make_trees(wl)
+    t = {k: (None if v is None else v.cuda()) for k, v in inputs.make_tensors(wl).items()}
+    tree = tv.tree_build(parents).upload()
+    first = None
+    for i in range(24):
+        O = torch.full((B, H, T, wl.dv), float("nan"), device="cuda")
+        tv.tree_verify(tree, t["S_pre"], t["q"], t["k"], t["v"], t["alpha"], O=O, impl=tv.IMPL_TC)
+        if first is None:
+            first = O
+        else:
+            assert torch.equal(O, first), f"launch {i} differs"
+    torch.cuda.synchronize()
+    tree.device_status()
+    assert torch.isfinite(first).all()
+
+
 def test_tc_delta_falls_back_on_deep_trees():
     wl = inputs.workload("c4", B=1, H=2, T=40, tree="chain", seed=5)   # depth 39 > 15
     parents, accepted = inputs.make_trees(wl)
