@@ -37,15 +37,19 @@
 // item n is worked on.  T > 64: one stage of everything.
 //
 // Warp roles, in groups of four warps so that registers can be moved between them
-// (setmaxnreg).  The chain that paces an item is that of the compute warps; what depends on
-// loaded data only is taken off it.
-//   warps 0..3   service, 64 registers: 0 = TMA producer, 1 = MMA issuer (owns TMEM),
-//                2 = issues the output stores, 3 idle
-//   warps 4..11  compute, 168 registers: path decay, C' from the scores, O from the
-//                accumulator; warp w reads TMEM lanes 32 (w % 4) .. +31 (the hardware's lane
+// (setmaxnreg).  Whatever depends on loaded data only is taken off the compute warps' chain.
+//   warps 0..3   service, 64 registers: 0 = TMA producer (one thread polls the gates of three
+//                independent load streams: q+k, v, S_pre), 1 = MMA issuer (owns TMEM), 2 = issues
+//                the output stores, 3 = path decay: g, 2^-g and the range flag of item n+1 and
+//                n+2 by pointer jumping over the tree, into one of two shared-memory copies
+//   warps 4..11  compute, 168 registers: O of item n-1 from the accumulator, then C' of item n
+//                from the scores; warp w reads TMEM lanes 32 (w % 4) .. +31 (the hardware's lane
 //                window of that warp) and half of the columns
-//   warps 12..15 operands, 104 registers, thread r = node r = state row r: the q rows into TMEM,
-//                the split of S_pre
+//   warps 12..15 operands, 104 registers, thread r = node r = state row r: the q rows into TMEM
+//                (two copies, items alternate), the split of S_pre
+// The code is kept small where that is free (one output site, a short bounded wait, division
+// by launch constants as multiply-shift): the five roles share one instruction cache, and at
+// 79 KB of code it hit in 59 % of its requests.
 // Every wait is an mbarrier wait with a time limit; on expiry the CTA sets the status word,
 // drains its own copies and leaves (TMEM is freed on every path).
 #include "tv_tc_common.cuh"
@@ -54,7 +58,7 @@ namespace {
 
 using namespace tvtc;
 
-constexpr int kThreads = 512;     // 4 service warps, 8 compute warps, 4 state-split warps
+constexpr int kThreads = 512;     // 4 service warps, 8 compute warps, 4 operand warps
 constexpr int kComputeWarps = 8;
 constexpr int kFirstComputeWarp = 4;
 constexpr int kFirstSplitWarp = 12;
