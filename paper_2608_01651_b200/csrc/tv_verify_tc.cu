@@ -261,6 +261,15 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
   constexpr int NH = D / 64;    // 64-wide halves of a q / k / v row
   constexpr int NC = D / 32;    // 32-float chunks of a state row and of an output row
   constexpr uint32_t kIdescPrefix = idesc_bf16(D, false), kIdescReadout = idesc_bf16(D, true);
+  // STACK (T <= 64, D = 128): the hi and lo tiles of a k half lie one behind the other, so one
+  // MMA with N = 256 multiplies q by both -- half as many prefix MMAs, each twice as large (an MMA
+  // costs about as much to issue whatever its N).  Its 256 columns are one accumulator,
+  // q S_hi^T in the first 128 (the readout adds C' V there) and q S_lo^T in the second; the output
+  // epilogue adds the two.  TMEM then holds one accumulator, not two: the prefix MMA of item
+  // n+1 waits for the output of item n to be read, which it can (it runs under the C' epilogue).
+  constexpr bool STACK = SMALL && D == 128;
+  constexpr uint32_t kColAccS = 192;   // columns 192..447
+  constexpr uint32_t kIdescStack = idesc_bf16(256, false);
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   unsigned char* sm = smem_raw;
   const uint32_t sbase = smem_u32(sm);
@@ -427,7 +436,7 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
 #pragma unroll 1
       for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++it) {
         const uint32_t ph = it & 1;
-        const uint32_t acc_col = ph ? kColAcc1 : kColAcc0;
+        const uint32_t acc_col = STACK ? kColAccS : ph ? kColAcc1 : kColAcc0;
         const uint32_t ph2 = (it >> 1) & 1;   // the two accumulators alternate
         const int st = s_stage(it);
         // scores = Q K^T
@@ -446,13 +455,23 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
         // extreme decay only: the compute warps have replaced the q rows by scaled ones
         const bool rescaled = fast_s[ph] == 0;
         mbar_arrive(bar(META_FREE0 + (int)ph));
-        if (!wait_list(W(ACC_FREE0 + (int)ph, ph2 ^ 1) | W(QS_READY0 + (int)ph, ph2) << 6, rescaled ? 2 : 1)) break;
+        if (!wait_list((STACK ? W(ACC_FREE0, ph ^ 1) : W(ACC_FREE0 + (int)ph, ph2 ^ 1)) | W(QS_READY0 + (int)ph, ph2) << 6,
+                       rescaled ? 2 : 1)) break;
         tc_fence_after();
+        if constexpr (STACK) {
+#pragma unroll
+          for (uint32_t i = 0; i < 8; ++i) {   // k half i >> 2: its hi tile and, right behind it, its lo tile
+            const uint32_t off = (((uint32_t)st * 4u + (i >> 2) * 2u) * kTile + (i & 3u) * 32u) >> 4;
+            mma_bf16_ts(tmem + acc_col, tmem + kColQb + ph * 64 + (i >> 2) * 32 + (i & 3u) * 8, dS + off,
+                        kIdescStack, i);
+          }
+        } else {
 #pragma unroll(SMALL ? 8 * NH : 1)
-        for (uint32_t i = 0; i < 8 * NH; ++i) {   // tile i >> 2 of the stage = (k half, hi | lo)
-          const uint32_t off = (((uint32_t)st * 4u + (i >> 2)) * kTile + (i & 3u) * 32u) >> 4;
-          mma_bf16_ts(tmem + acc_col, tmem + kColQb + ph * 64 + (i >> 3) * 32 + (i & 3u) * 8, dS + off,
-                      kIdescPrefix, i);
+          for (uint32_t i = 0; i < 8 * NH; ++i) {   // tile i >> 2 of the stage = (k half, hi | lo)
+            const uint32_t off = (((uint32_t)st * 4u + (i >> 2)) * kTile + (i & 3u) * 32u) >> 4;
+            mma_bf16_ts(tmem + acc_col, tmem + kColQb + ph * 64 + (i >> 3) * 32 + (i & 3u) * 8, dS + off,
+                        kIdescPrefix, i);
+          }
         }
         tc_commit(bar(S_FREE0 + st));
         // acc += C'_hi V + C'_lo V
@@ -468,7 +487,7 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
             mma_bf16_ss(tmem + acc_col, dClo + off, bdesc, kIdescReadout, 1);
           }
         tc_commit(bar(V_FREE));
-        tc_commit(bar(ACC_DONE0 + (int)ph));
+        tc_commit(bar(STACK ? ACC_DONE0 : ACC_DONE0 + (int)ph));
       }
     }
   } else if (warp == 2) {
@@ -678,18 +697,25 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
     // chunks are the four C' tiles themselves and the store must have read them before C' is
     // rewritten.
     auto final_epilogue = [&](uint32_t it_prev, float r_prev, uint32_t ost_phase, const PackedItem& pk_prev) -> bool {
-      const int acc_done = (it_prev & 1) ? ACC_DONE1 : ACC_DONE0;
-      const int acc_free = (it_prev & 1) ? ACC_FREE1 : ACC_FREE0;
-      const uint32_t acc_col = (it_prev & 1) ? kColAcc1 : kColAcc0;
+      const int acc_done = STACK ? ACC_DONE0 : (it_prev & 1) ? ACC_DONE1 : ACC_DONE0;
+      const int acc_free = STACK ? ACC_FREE0 : (it_prev & 1) ? ACC_FREE1 : ACC_FREE0;
+      const uint32_t acc_col = STACK ? kColAccS : (it_prev & 1) ? kColAcc1 : kColAcc0;
       // SMALL: the store of the item before has read the staging chunks
       if (SMALL && !mbar_wait_warp(bar(OST_FREE), ost_phase, abort_flag)) return false;
-      if (!mbar_wait_warp(bar(acc_done), (it_prev >> 1) & 1, abort_flag)) return false;
+      if (!mbar_wait_warp(bar(acc_done), STACK ? (it_prev & 1) : (it_prev >> 1) & 1, abort_flag)) return false;
       tc_fence_after();
       if (warp_live) {
 #pragma unroll
         for (int half = 0; half < NH; ++half) {   // this warp's D / 2 columns, 32 at a time
           uint32_t r1[32];
           tmem_ld32(tmem + lane_addr + acc_col + hc * (D / 2) + half * 32, r1);
+          if constexpr (STACK) {   // + q S_lo^T from the second half of the accumulator
+            uint32_t r2[32];
+            tmem_ld32(tmem + lane_addr + acc_col + 128 + hc * 64 + half * 32, r2);
+            tmem_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 32; ++e) r1[e] = __float_as_uint(__uint_as_float(r1[e]) + __uint_as_float(r2[e]));
+          }
           tmem_wait_ld();
           unsigned char* orow = sm + L::kOffStage + (hc * NH + half) * L::kStageChunk + row * 128;
           // packed forest: the rows after the last full group of 8 leave from registers
