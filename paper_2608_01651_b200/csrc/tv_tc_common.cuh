@@ -46,6 +46,17 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
+// Non-blocking look at a barrier (try_wait may park the thread for a while when the phase is
+// not complete; a loop that polls several barriers must not be parked at one of them).
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
 // Bounded wait.  Returns false when the limit ran out or another role gave up.  Kept short (32-bit
 // clock, one exit for both reasons): a kernel has dozens of these, all inlined, and their code
 // competes with the working loops for the instruction cache.  The clock is first read after
