@@ -348,17 +348,20 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
       int pend_qk = 0, pend_v = 0, pend_s[2] = {0, 0};
       const uint32_t n_it = blockIdx.x < (uint32_t)p.n_items
                                 ? ((uint32_t)p.n_items - blockIdx.x + gridDim.x - 1) / gridDim.x : 0u;
-      uint32_t i_qk = 0, i_v = 0, i_s = 0, i_sc = 0;
+      uint32_t i_qk = 0, i_v = 0, i_s = 0, i_sc = SMALL ? 0u : 0xffffffffu;   // T > 64: the MMA issuer keeps the scores
+      // T <= 64 polls without parking (test_wait); T > 64, with items twice as long, measured 1 % faster
+      // parked in try_wait
+      auto poll = [](uint32_t b, uint32_t parity) { return SMALL ? mbar_test(b, parity) : mbar_try(b, parity); };
       const uint64_t dQ = desc_kmajor(sbase + L::kOffQ), dK = desc_kmajor(sbase + L::kOffK);
       grid_dependency_wait();   // inputs may come from the kernel in front (dependent launch)
       long long t_idle = clock64();
       uint32_t spin = 0;
-      while (i_qk < n_it || i_v < n_it || i_s < n_it || i_sc < n_it) {
+      while (i_qk < n_it || i_v < n_it || i_s < n_it || (SMALL && i_sc < n_it)) {
         bool progress = false;
         // A fourth stream, not a load: the score MMAs Sc = Q K^T of item i_sc, issued from here the
         // moment q and k have landed and the score columns are free -- the MMA issuer's thread
         // is the busiest of the CTA, and these eight instructions depend on nothing it does.
-        if (i_sc < n_it && mbar_test(bar(QK_FULL), i_sc & 1) && mbar_test(bar(SC_FREE), (i_sc & 1) ^ 1)) {
+        if (SMALL && i_sc < n_it && poll(bar(QK_FULL), i_sc & 1) && poll(bar(SC_FREE), (i_sc & 1) ^ 1)) {
           tc_fence_after();
 #pragma unroll(SMALL ? 4 : 1)
           for (uint32_t i = 0; i < 4 * NH; ++i) {   // k half i >> 2, 16 contraction indices (32 bytes) per step
@@ -372,8 +375,8 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
         }
         // (two stages: the second item's state is not asked for before the first item's operands
         // have landed -- at the start of a launch every CTA's first loads share the memory system)
-        if (i_s < n_it && (!SMALL || i_s != 1 || (mbar_test(bar(S_FULL0), 0) && mbar_test(bar(QK_FULL), 0))) &&
-            mbar_test(bar(S_FREE0 + s_stage(i_s)), s_phase(i_s) ^ 1)) {
+        if (i_s < n_it && (!SMALL || i_s != 1 || (poll(bar(S_FULL0), 0) && poll(bar(QK_FULL), 0))) &&
+            poll(bar(S_FREE0 + s_stage(i_s)), s_phase(i_s) ^ 1)) {
           const int sj = s_stage(i_s);
           const int item = (int)(blockIdx.x + i_s * gridDim.x);
           mbar_expect_tx(bar(S_FULL0 + sj), NC * D * 128);
@@ -384,7 +387,7 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
           ++i_s;
           progress = true;
         }
-        if (i_qk < n_it && mbar_test(bar(QK_FREE), (i_qk & 1) ^ 1)) {
+        if (i_qk < n_it && poll(bar(QK_FREE), (i_qk & 1) ^ 1)) {
           const ItemCoord ic = item_coord<PACKED>(p, (int)(blockIdx.x + i_qk * gridDim.x));
           // rows of the boxes of this item (the tile layout in shared memory does not depend on it)
           const int bc = PACKED ? box_class(ic.n, kBoxRows) : 2;
@@ -399,7 +402,7 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
           ++i_qk;
           progress = true;
         }
-        if (i_v < n_it && mbar_test(bar(V_FREE), (i_v & 1) ^ 1)) {
+        if (i_v < n_it && poll(bar(V_FREE), (i_v & 1) ^ 1)) {
           const ItemCoord ic = item_coord<PACKED>(p, (int)(blockIdx.x + i_v * gridDim.x));
           const int bc = PACKED ? box_class(ic.n, kBoxRows) : 2;
           const uint32_t box_bytes = kBox >> (2 - bc);
@@ -454,7 +457,19 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
         const uint32_t acc_col = STACK ? kColAccS : ph ? kColAcc1 : kColAcc0;
         const uint32_t ph2 = (it >> 1) & 1;   // the two accumulators alternate
         const int st = s_stage(it);
-        // (the score MMAs of the item are issued by the producer thread)
+        // scores = Q K^T (T <= 64: issued by the producer thread)
+        if constexpr (!SMALL) {
+          if (!wait_list(W(QK_FULL, ph) | W(SC_FREE, ph ^ 1) << 6, 2)) break;
+          tc_fence_after();
+          const uint64_t dQ = desc_kmajor(sbase + L::kOffQ), dK = desc_kmajor(sbase + L::kOffK);
+#pragma unroll 1
+          for (uint32_t i = 0; i < 4 * NH; ++i) {   // k half i >> 2, 16 contraction indices (32 bytes) per step
+            const uint32_t off = ((i >> 2) * kBox + (i & 3u) * 32u) >> 4;
+            mma_bf16_ss(tmem + kColSc, dQ + off, dK + off, kIdescKK128, i);
+          }
+          tc_commit(bar(SC_DONE));
+          tc_commit(bar(QK_FREE));
+        }
         // acc = Q S_pre^T: A = the q rows (packed bf16 in TMEM), B = hi and lo tiles of S_pre
         if (!wait_list(W(S_CONV0 + st, s_phase(it)) | W(QB_READY0 + (int)ph, ph2) << 6 |
                            W(META_READY0 + (int)ph, ph2) << 12, 3)) break;

@@ -68,9 +68,8 @@ constexpr uint32_t kSmemBytes = kOffMisc + 64 + 1024;
 enum Bar {
   QK_FULL = 0, QK_FREE, S_FULL, S_FREE, V_FULL, V_FREE,
   G_DONE, G_FREE, W_READY, D1_DONE, ACC_DONE, ACC_FREE, E1_SYNC,
-  OST_READY, OST_FREE, QK_FULL1, QK_FREE1, META_FULL, META_FULL1, META_FREE, META_FREE1, WV_DONE, kNumBars
+  OST_READY, OST_FREE, QK_FULL1, QK_FREE1, META_FULL, META_FULL1, META_FREE, META_FREE1
 };
-static_assert(kNumBars <= 24, "barrier area");
 
 constexpr uint32_t kColSc = 0, kColQf = 128, kColAcc = 256;
 // The tensor core cuts a tf32 operand to 10 explicit mantissa bits by dropping the rest (towards
@@ -175,7 +174,6 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     mbar_init(bar(G_DONE), 1);   mbar_init(bar(G_FREE), kComputeWarps);
     mbar_init(bar(W_READY), kComputeWarps);
     mbar_init(bar(D1_DONE), 1);
-    mbar_init(bar(WV_DONE), 1);
     mbar_init(bar(ACC_DONE), 1); mbar_init(bar(ACC_FREE), kComputeWarps);
     mbar_init(bar(META_FULL), 1);  mbar_init(bar(META_FULL1), 1);
     mbar_init(bar(META_FREE), kComputeWarps); mbar_init(bar(META_FREE1), kComputeWarps);
@@ -196,100 +194,41 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
 
   if (warp == 0) {
     if (lane == 0) {
-      // ===================== TMA producer, and the MMAs that depend on loads only =====================
-      // One thread polls the gates of five independent streams and serves whichever is ready:
-      // the loads of [Q ; K] (two buffers), S_pre and V, the Gram product [Q ; K] K^T of an item
-      // (needs its q and k and the score columns) and the readout product [W ; A] V (needs the
-      // coefficient tiles, V and the accumulator).  The MMA issuer's thread keeps the chain key
-      // product -> state product, which these two would otherwise sit in front of.
-      constexpr uint32_t kIdGram = idesc_bf16(64, false);
-      constexpr uint32_t kIdMn = idesc_bf16(128, true);
-      int pend_qk[2] = {0, 0}, pend_s = 0, pend_v = 0;
-      const uint32_t n_it = blockIdx.x < (uint32_t)p.n_items
-                                ? ((uint32_t)p.n_items - blockIdx.x + gridDim.x - 1) / gridDim.x : 0u;
-      uint32_t i_qk = 0, i_s = 0, i_v = 0, i_g = 0, i_w = 0;
+      // ===================== TMA producer =====================
+      int pend_qk = 0, pend_qk_bar = QK_FULL, pend_s = 0, pend_v = 0;
+      uint32_t it = 0;
       grid_dependency_wait();   // inputs may come from the kernel in front (dependent launch)
-      long long t_idle = clock64();
-      uint32_t spin = 0;
-      while (i_qk < n_it || i_s < n_it || i_v < n_it || i_g < n_it || i_w < n_it) {
-        bool progress = false;
-        if (i_w < n_it && mbar_test(bar(W_READY), i_w & 1) && mbar_test(bar(V_FULL), i_w & 1) &&
-            mbar_test(bar(ACC_FREE), (i_w & 1) ^ 1)) {
-          // acc = [W ; A] V: the first product into the accumulator of the item
-          tc_fence_after();
-          const uint64_t dW = desc_kmajor(sbase + kOffW), dVr = desc_mnmajor(sbase + kOffV, kTile);
+      for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, ++it) {
+        const uint32_t ph = it & 1;
+        // [Q ; K] is double-buffered: item it uses buffer it & 1, each buffer's barriers flip
+        // every second item
+        const int qb = (int)(it & 1);
+        const uint32_t qph = (it >> 1) & 1;
+        const uint32_t qk_base = qb ? kOffQK1 : kOffQK;
+        const int qfull = qb ? QK_FULL1 : QK_FULL, qfree = qb ? QK_FREE1 : QK_FREE;
+        if (!mbar_wait(bar(qfree), qph ^ 1, abort_flag)) break;
+        mbar_expect_tx(bar(qfull), 4 * 8192);
+        const Coord co = coord_of(item);
+        load_box(sbase + qk_base, &tmQ, bar(qfull), nf_qk, 0, co.y0, co.hq, co.z);
+        load_box(sbase + qk_base + kTile, &tmQ, bar(qfull), nf_qk, 64, co.y0, co.hq, co.z);
+        load_box(sbase + qk_base + 8192, &tmK, bar(qfull), nf_qk, 0, co.y0, co.hq, co.z);
+        load_box(sbase + qk_base + kTile + 8192, &tmK, bar(qfull), nf_qk, 64, co.y0, co.hq, co.z);
+        pend_qk_bar = qfull;
+        pend_qk = 1 + (int)qph;
+        if (!mbar_wait(bar(S_FREE), ph ^ 1, abort_flag)) break;
+        mbar_expect_tx(bar(S_FULL), 4 * kTile);
 #pragma unroll
-          for (uint32_t i = 0; i < 8; ++i)   // 16 nodes j per step; hi then lo tile of [W ; A]
-            mma_bf16_ss(tmem + kColAcc, dW + (((i & 1u) * kTile + (i >> 1) * 32u) >> 4),
-                        dVr + (((i >> 1) * 2048u) >> 4), kIdMn, i);
-          tc_commit(bar(WV_DONE));
-          tc_commit(bar(V_FREE));
-          ++i_w;
-          progress = true;
-        }
-        if (i_g < n_it && mbar_test(bar((i_g & 1) ? QK_FULL1 : QK_FULL), (i_g >> 1) & 1) &&
-            mbar_test(bar(G_FREE), (i_g & 1) ^ 1)) {   // score columns read by E1 of the item before
-          // Sc = [Q ; K] K^T, as early as its operands allow: it runs under the row solve of the item before
-          tc_fence_after();
-          const uint32_t qk_base = (i_g & 1) ? kOffQK1 : kOffQK;
-          const uint64_t dA = desc_kmajor(sbase + qk_base), dB = desc_kmajor(sbase + qk_base + 8192);
-#pragma unroll
-          for (uint32_t i = 0; i < 8; ++i) {   // k half i >> 2, 32 bytes of k per step
-            const uint32_t off = ((i >> 2) * kTile + (i & 3u) * 32u) >> 4;
-            mma_bf16_ss(tmem + kColSc, dA + off, dB + off, kIdGram, i);
-          }
-          tc_commit(bar(G_DONE));
-          ++i_g;
-          progress = true;
-        }
-        if (i_qk < n_it && mbar_test(bar((i_qk & 1) ? QK_FREE1 : QK_FREE), ((i_qk >> 1) & 1) ^ 1)) {
-          // [Q ; K] is double-buffered: item it uses buffer it & 1, each buffer's barriers flip
-          // every second item
-          const int qb = (int)(i_qk & 1);
-          const uint32_t qk_base = qb ? kOffQK1 : kOffQK;
-          const int qfull = qb ? QK_FULL1 : QK_FULL;
-          const Coord co = coord_of((int)(blockIdx.x + i_qk * gridDim.x));
-          mbar_expect_tx(bar(qfull), 4 * 8192);
-          load_box(sbase + qk_base, &tmQ, bar(qfull), nf_qk, 0, co.y0, co.hq, co.z);
-          load_box(sbase + qk_base + kTile, &tmQ, bar(qfull), nf_qk, 64, co.y0, co.hq, co.z);
-          load_box(sbase + qk_base + 8192, &tmK, bar(qfull), nf_qk, 0, co.y0, co.hq, co.z);
-          load_box(sbase + qk_base + kTile + 8192, &tmK, bar(qfull), nf_qk, 64, co.y0, co.hq, co.z);
-          pend_qk[qb] = 1 + (int)((i_qk >> 1) & 1);
-          ++i_qk;
-          progress = true;
-        }
-        if (i_s < n_it && mbar_test(bar(S_FREE), (i_s & 1) ^ 1)) {
-          mbar_expect_tx(bar(S_FULL), 4 * kTile);
-#pragma unroll 1
-          for (int c = 0; c < 4; ++c)
-            tma_load_3d(sbase + kOffS + c * kTile, &tmS, bar(S_FULL), 32 * c, 0, (int)(blockIdx.x + i_s * gridDim.x));
-          pend_s = 1 + (int)(i_s & 1);
-          ++i_s;
-          progress = true;
-        }
-        if (i_v < n_it && mbar_test(bar(V_FREE), (i_v & 1) ^ 1)) {
-          const Coord co = coord_of((int)(blockIdx.x + i_v * gridDim.x));
-          mbar_expect_tx(bar(V_FULL), 2 * 8192);
-          load_box(sbase + kOffV, &tmV, bar(V_FULL), nf_v, 0, co.y0, co.h, co.z);
-          load_box(sbase + kOffV + kTile, &tmV, bar(V_FULL), nf_v, 64, co.y0, co.h, co.z);
-          pend_v = 1 + (int)(i_v & 1);
-          ++i_v;
-          progress = true;
-        }
-        if (progress) {
-          t_idle = clock64();
-          spin = 0;
-        } else if ((++spin & 255u) == 0) {   // the same limit as every other wait of the kernel
-          if (*abort_flag) break;
-          if (clock64() - t_idle > kWaitLimitCycles) {
-            *abort_flag = 1;
-            break;
-          }
-        }
+        for (int c = 0; c < 4; ++c)
+          tma_load_3d(sbase + kOffS + c * kTile, &tmS, bar(S_FULL), 32 * c, 0, item);
+        pend_s = 1 + (int)ph;
+        if (!mbar_wait(bar(V_FREE), ph ^ 1, abort_flag)) break;
+        mbar_expect_tx(bar(V_FULL), 2 * 8192);
+        load_box(sbase + kOffV, &tmV, bar(V_FULL), nf_v, 0, co.y0, co.h, co.z);
+        load_box(sbase + kOffV + kTile, &tmV, bar(V_FULL), nf_v, 64, co.y0, co.h, co.z);
+        pend_v = 1 + (int)ph;
       }
       if (*abort_flag) {
-        for (int q2 = 0; q2 < 2; ++q2)
-          if (pend_qk[q2]) mbar_wait(bar(q2 ? QK_FULL1 : QK_FULL), pend_qk[q2] - 1, abort_flag + 1);
+        if (pend_qk) mbar_wait(bar(pend_qk_bar), pend_qk - 1, abort_flag + 1);
         if (pend_s) mbar_wait(bar(S_FULL), pend_s - 1, abort_flag + 1);
         if (pend_v) mbar_wait(bar(V_FULL), pend_v - 1, abort_flag + 1);
       }
@@ -297,19 +236,38 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   } else if (warp == 1) {
     // ===================== MMA issuer =====================
     if (lane == 0) {
+      constexpr uint32_t kIdGram = idesc_bf16(64, false);
       constexpr uint32_t kIdMn = idesc_bf16(128, true);
       constexpr uint32_t kIdTf32 = idesc_tf32(128);
+      // Sc = [Q ; K] K^T of local item j, issued one item ahead of the rest of the chain so that
+      // it runs under the row solve of the item before
       const uint32_t n_local = p.n_items > (int)blockIdx.x
                                    ? (uint32_t)((p.n_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x) : 0u;
-      for (uint32_t it = 0; it < n_local; ++it) {
+      auto gram = [&](uint32_t j) -> bool {
+        const uint32_t qk_base = (j & 1) ? kOffQK1 : kOffQK;
+        if (!mbar_wait(bar((j & 1) ? QK_FULL1 : QK_FULL), (j >> 1) & 1, abort_flag)) return false;
+        if (!mbar_wait(bar(G_FREE), (j & 1) ^ 1, abort_flag)) return false;   // score columns read by E1 of j-1
+        tc_fence_after();
+        // (the MMA loops are kept rolled, descriptor = base + step: the roles of a CTA share one
+        // instruction cache)
+        const uint64_t dA = desc_kmajor(sbase + qk_base), dB = desc_kmajor(sbase + qk_base + 8192);
+#pragma unroll
+        for (uint32_t i = 0; i < 8; ++i) {   // k half i >> 2, 32 bytes of k per step
+          const uint32_t off = ((i >> 2) * kTile + (i & 3u) * 32u) >> 4;
+          mma_bf16_ss(tmem + kColSc, dA + off, dB + off, kIdGram, i);
+        }
+        tc_commit(bar(G_DONE));
+        return true;
+      };
+      bool mma_ok = n_local == 0 || gram(0);
+      for (uint32_t it = 0; mma_ok && it < n_local; ++it) {
         const uint32_t ph = it & 1;
         const uint32_t qk_base = (it & 1) ? kOffQK1 : kOffQK;
+        if (it + 1 < n_local && !gram(it + 1)) break;
         // Qf += -(W D_P) K  (rows 64..127: -(A D_P) K); the compute warps initialised Qf with D_P Q
         if (!mbar_wait(bar(W_READY), ph, abort_flag)) break;
         tc_fence_after();
         {
-          // (descriptor = base + step; the loops are unrolled: rolled, the arithmetic between two
-          // MMAs slowed their issue by 3 us per 64-node launch)
           const uint64_t dAk = desc_kmajor(sbase + kOffAk), dKr = desc_mnmajor(sbase + qk_base + 4 * 2048, kTile);
 #pragma unroll
           for (uint32_t i = 0; i < 8; ++i)   // part i >> 2 (hi, lo), K rows 16 (i & 3) .. of the stacked tile
@@ -318,20 +276,30 @@ verify_tc_delta_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         }
         tc_commit(bar(D1_DONE));
         tc_commit(bar((it & 1) ? QK_FREE1 : QK_FREE));
-        // acc += Qf S_pre^T: Qf must be complete in TMEM before it is read as the A operand, and
-        // the readout product (issued by the producer thread) must have initialised the accumulator
+        // acc = Qf S_pre^T: Qf must be complete in TMEM before it is read as the A operand
         if (!mbar_wait(bar(D1_DONE), ph, abort_flag)) break;
         if (!mbar_wait(bar(S_FULL), ph, abort_flag)) break;
-        if (!mbar_wait(bar(WV_DONE), ph, abort_flag)) break;
+        if (!mbar_wait(bar(ACC_FREE), ph ^ 1, abort_flag)) break;
         tc_fence_after();
         {
           const uint64_t dS = desc_kmajor(sbase + kOffS);
 #pragma unroll
           for (uint32_t i = 0; i < 16; ++i)   // k chunk i >> 2 of the state, 8 values of k per step
             mma_tf32_ts(tmem + kColAcc, tmem + kColQf + i * 8, dS + (((i >> 2) * kTile + (i & 3u) * 32u) >> 4),
-                        kIdTf32, 1);
+                        kIdTf32, i);
         }
         tc_commit(bar(S_FREE));
+        // acc += [W ; A] V
+        if (!mbar_wait(bar(V_FULL), ph, abort_flag)) break;
+        tc_fence_after();
+        {
+          const uint64_t dW = desc_kmajor(sbase + kOffW), dVr = desc_mnmajor(sbase + kOffV, kTile);
+#pragma unroll
+          for (uint32_t i = 0; i < 8; ++i)   // 16 nodes j per step; hi then lo tile of [W ; A]
+            mma_bf16_ss(tmem + kColAcc, dW + (((i & 1u) * kTile + (i >> 1) * 32u) >> 4),
+                        dVr + (((i >> 1) * 2048u) >> 4), kIdMn, 1);
+        }
+        tc_commit(bar(V_FREE));
         tc_commit(bar(ACC_DONE));
       }
     }
