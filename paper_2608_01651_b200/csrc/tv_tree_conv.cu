@@ -134,8 +134,23 @@ __device__ __forceinline__ float rsqrt_fast(float x) {
   return r;
 }
 
+// Gate arithmetic on the special-function unit (ex2 / lg2 / rcp: relative error about 2^-22 each).
+// softplus(z) = max(z, 0) + log(1 + e^-|z|): the rounding of 1 + e^-|z| leaves an absolute error of
+// 6e-8, which the gate exp(-c * softplus) turns into a relative error of c * 6e-8.
+__device__ __forceinline__ float exp_fast(float x) {
+  float r;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x * 1.4426950408889634f));
+  return r;
+}
 __device__ __forceinline__ float softplus(float z) {
-  return fmaxf(z, 0.0f) + log1pf(expf(-fabsf(z)));
+  float l;
+  asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(l) : "f"(1.0f + exp_fast(-fabsf(z))));
+  return fmaf(l, 0.6931471805599453f, fmaxf(z, 0.0f));
+}
+__device__ __forceinline__ float sigmoid_fast(float z) {
+  float r;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(1.0f + exp_fast(-z)));
+  return r;
 }
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
@@ -152,9 +167,12 @@ __device__ __forceinline__ void cp_async_wait_all() {
 // channels; a CTA walks a contiguous range of them, so its filter registers are reloaded only
 // when the slice changes.  Shared memory, every block on a 16-byte boundary:
 //   2 x [T+W-1][d] staged rows (context rows first, oldest first, then the nodes),
-//   2 x [T] parents, 2 x [T][WP] byte offsets of each node's tap rows (WP = 4 or 8).
-// While item n is computed, the rows of item n+1 and the parents of item n+2 are in flight
-// (cp.async) and the tap table of item n+1 is derived: one __syncthreads per item.
+//   2 x [T] parents, 2 x [T][WP] byte offsets of each node's tap rows (WP = 4 or 8),
+//   2 x ([128 NJ][W] filter taps + [128 NJ] bias) of a slice; every group of 8 channels is shifted
+//   by two words, so that the 16 lanes of a row, which own 8 channels each, read 16 banks.
+// While item n is computed, the rows of item n+1 (with the filter of its slice, when that is a
+// new one) and the parents of item n+2 are in flight (cp.async) and the tap table of item n+1
+// is derived: one __syncthreads per item, and no load whose latency is exposed after the first.
 struct ConvItem {
   int slice, b, kind, h, d, c0;
   int n;          // node rows of this request
@@ -179,7 +197,10 @@ tree_conv_kernel(const ConvArgs a) {
   const uint32_t xs_u32 = smem_u32(smem_raw);
   int32_t* par_s = reinterpret_cast<int32_t*>(smem_raw + (single ? 1 : 2) * (size_t)buf_bytes);  // [2][Tp]
   uint32_t* taps_s = reinterpret_cast<uint32_t*>(par_s + 2 * Tp);                                // [2][T][WP]
-  const uint32_t par_u32 = smem_u32(par_s), taps_u32 = smem_u32(taps_s);
+  constexpr int kBiasAt = 128 * NJ * W + 32 * NJ;         // words; kFiltAt(c, t) below
+  constexpr int kFiltFloats = kBiasAt + 128 * NJ + 32 * NJ;
+  float* filt_s = reinterpret_cast<float*>(taps_s + 2 * T * WP);                                 // [2][kFiltFloats]
+  const uint32_t par_u32 = smem_u32(par_s), taps_u32 = smem_u32(taps_s), filt_u32 = smem_u32(filt_s);
 
   const long long n_items = 3LL * H * B;
   const int first = (int)(n_items * blockIdx.x / gridDim.x);
@@ -260,6 +281,17 @@ tree_conv_kernel(const ConvArgs a) {
       if (cv >= vpr) { cv -= vpr; ++row; }
     }
   };
+  // the slice's d x W filter taps and d bias values, contiguous in global memory
+  auto fetch_filter = [&](const ConvItem& it, int slot) {
+    const uint32_t dst = filt_u32 + (uint32_t)(slot * kFiltFloats) * 4;
+    const float* wsrc = a.weight + (size_t)it.c0 * W;
+    for (int c = tid; c < it.d; c += kConvThreads) {
+      const uint32_t shift = 2 * (c >> 3);
+#pragma unroll
+      for (int t = 0; t < W; ++t) cp_async4(dst + (c * W + t + shift) * 4, wsrc + c * W + t);
+      if (a.bias != nullptr) cp_async4(dst + (kBiasAt + c + shift) * 4, a.bias + it.c0 + c);
+    }
+  };
   // (the last warps do this, the first ones prepare the gates: neither is late at the barrier)
   auto build_taps = [&](const ConvItem& it, int slot) {
     const int node = kConvThreads - 1 - tid;
@@ -285,6 +317,7 @@ tree_conv_kernel(const ConvArgs a) {
   fetch_parents(cur.b, 0);
   if (first + 1 < last) fetch_parents(nxt.b, 1);
   if (!single) fetch_rows(cur, 0);
+  fetch_filter(cur, 0);
   cp_async_wait_all();
   __syncthreads();
   build_taps(cur, 0);
@@ -294,7 +327,15 @@ tree_conv_kernel(const ConvArgs a) {
   float wreg[NJ][W][8], breg[NJ][8];
   bool live0[NJ], live1[NJ];
   uint32_t off0[NJ], off1[NJ];
-  int loaded_slice = -1;
+  // this thread's gate input of an item (alpha with the q slice, beta with the k slice), loaded
+  // one item ahead
+  auto fetch_gate = [&](const ConvItem& it) -> IO {
+    const void* src = it.kind == 0 ? a.gate_a : it.kind == 1 ? a.gate_b : nullptr;
+    if (src == nullptr || tid >= it.n) return IO(0.0f);
+    return reinterpret_cast<const IO*>(src)[((size_t)it.row0 + tid) * H + it.h];
+  };
+  IO gate_next = fetch_gate(cur);
+  int loaded_slice = -1, fslot = 0;   // fslot: the buffer that holds the filter of cur's slice
   const float eps = a.eps;
   const bool want_norm = a.normalize != 0;
 
@@ -311,6 +352,7 @@ tree_conv_kernel(const ConvArgs a) {
     if (item + 1 < last) {
       if (!single) fetch_rows(nxt, s ^ 1);
       if (item + 2 < last) fetch_parents(b2, s);
+      if (nxt.slice != cur.slice) fetch_filter(nxt, fslot ^ 1);
       build_taps(nxt, s ^ 1);
     }
     const int d = cur.d, c0 = cur.c0;
@@ -318,6 +360,8 @@ tree_conv_kernel(const ConvArgs a) {
     // ---- this lane's filter taps and bias, when the slice changes
     if (cur.slice != loaded_slice) {
       loaded_slice = cur.slice;
+      const float* wf = filt_s + fslot * kFiltFloats;
+      const float* bf = wf + kBiasAt;
 #pragma unroll
       for (int j = 0; j < NJ; ++j) {
         const int g0 = 128 * j + Geo<IO>::g0(l16), g1 = 128 * j + Geo<IO>::g1(l16);
@@ -329,22 +373,23 @@ tree_conv_kernel(const ConvArgs a) {
         for (int e = 0; e < 8; ++e) {
           const int c = e < 4 ? g0 + e : g1 + e - 4;
           const bool live = e < 4 ? live0[j] : live1[j];
-          breg[j][e] = live && a.bias ? __ldg(a.bias + c0 + c) : 0.0f;
+          const int shift = 2 * (c >> 3);
+          breg[j][e] = live && a.bias ? bf[c + shift] : 0.0f;
 #pragma unroll
-          for (int r = 0; r < W; ++r)
-            wreg[j][r][e] = live ? __ldg(a.weight + (size_t)(c0 + c) * W + (W - 1 - r)) : 0.0f;
+          for (int r = 0; r < W; ++r) wreg[j][r][e] = live ? wf[c * W + (W - 1 - r) + shift] : 0.0f;
         }
       }
     }
 
-    // ---- gate preparation for this (request, head), done with the q slice: the inputs are
-    // requested here and used after the row loop, so nobody waits for them at the next barrier
-    const bool do_gates = cur.kind == 0 && a.gate_a != nullptr && tid < cur.n;
-    float gate_in_a = 0.f, gate_in_b = 0.f, gate_A = 0.f, gate_dt = 0.f;
-    if (do_gates) {
-      const size_t gi = ((size_t)cur.row0 + tid) * H + cur.h;
-      gate_in_a = to_f32(reinterpret_cast<const IO*>(a.gate_a)[gi]);
-      if (a.gate_b != nullptr) gate_in_b = to_f32(reinterpret_cast<const IO*>(a.gate_b)[gi]);
+    // ---- gate preparation for this (request, head): alpha with the q slice, beta with the k
+    // slice (the work is spread over the CTAs of two thirds of the slices); the input was
+    // requested one item ago.
+    const bool do_alpha = cur.kind == 0 && a.gate_a != nullptr && tid < cur.n;
+    const bool do_beta = cur.kind == 1 && a.gate_b != nullptr && tid < cur.n;
+    const IO gate_raw = gate_next;
+    if (item + 1 < last) gate_next = fetch_gate(nxt);
+    float gate_A = 0.f, gate_dt = 0.f;
+    if (do_alpha) {
       gate_A = __ldg(a.A_log + cur.h);
       gate_dt = __ldg(a.dt_bias + cur.h);
     }
@@ -403,11 +448,9 @@ tree_conv_kernel(const ConvArgs a) {
                row_live && live1[j], y[j]);
       }
     }
-    if (do_gates) {
-      const size_t go = cur.orow0 + tid;
-      a.alpha[go] = expf(-expf(gate_A) * softplus(gate_in_a + gate_dt));
-      if (a.gate_b != nullptr) a.beta[go] = 1.0f / (1.0f + expf(-gate_in_b));
-    }
+    if (do_alpha) a.alpha[cur.orow0 + tid] = exp_fast(-exp_fast(gate_A) * softplus(to_f32(gate_raw) + gate_dt));
+    if (do_beta) a.beta[cur.orow0 + tid] = sigmoid_fast(to_f32(gate_raw));
+    if (nxt.slice != cur.slice) fslot ^= 1;
     cur = nxt;
     advance(nxt);
     b2 = b2 + 1 == B ? 0 : b2 + 1;
@@ -474,7 +517,8 @@ int launch_conv(const ConvArgs& a_in, cudaStream_t stream) {
   ConvArgs a = a_in;
   const int dmax = a.dk > a.dv ? a.dk : a.dv;
   const size_t buf = (size_t)(a.T + W - 1) * dmax * sizeof(IO);
-  const size_t tables = 2 * ((size_t)((a.T + 3) & ~3) * 4 + (size_t)a.T * (W <= 4 ? 4 : 8) * 4);
+  const size_t tables = 2 * ((size_t)((a.T + 3) & ~3) * 4 + (size_t)a.T * (W <= 4 ? 4 : 8) * 4) +
+                        2 * (size_t)(dmax <= 128 ? 1 : 2) * (128 * (W + 1) + 64) * 4;
   a.single = 2 * buf + tables > 200 * 1024;
   const size_t smem = (a.single ? 1 : 2) * buf + tables;
   int dev = 0, sms = 0;
