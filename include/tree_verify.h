@@ -159,9 +159,10 @@ int tv_tree_meta_device(tv_tree* tree, uint64_t* anc, int32_t* depth, void* stre
  * core completion that never came): TV_OK or TV_ERR_DEVICE_TIMEOUT.  After a
  * timeout the outputs of that launch are undefined; the context stays usable.
  * TV_ERR_UNSUPPORTED: the trees of the last tv_forest_upload_device were deeper
- * than the bound that call was given.  TV_ERR_CUDA: a tensor-core kernel found
- * its shared-memory window off the 1024-byte boundary its tiles need and left
- * without computing (outputs undefined, as after a timeout).                  */
+ * than the bound that call was given.  TV_ERR_CUDA: a tensor-core kernel (or
+ * tv_tree_conv, whose row boxes arrive by TMA) found its shared-memory window
+ * off the boundary its tiles need and left without computing (outputs
+ * undefined, as after a timeout).                                             */
 int tv_tree_device_status(tv_tree* tree, void* stream);
 /* Self-test of that mechanism: launches one CTA that waits, with a limit of a
  * few milliseconds, on a barrier nothing ever signals, and writes what the
@@ -395,7 +396,9 @@ int tv_session_free(tv_session* s);
  * (row offsets[r] + i = node i of request r), q, k, v [H][capacity][d],
  * alpha, beta [H][capacity]; ctx keeps [B][W-1][C].  Outputs must not alias
  * inputs.  Asynchronous on `stream`; returns a tv_status, launches nothing on
- * an error. */
+ * an error.  The kernel's waits (row boxes arriving by TMA) are bounded like
+ * those of the tensor-core kernels: tv_tree_device_status(tree) reports one
+ * that ran out. */
 #define TV_CONV_MAX_TAPS 8
 typedef struct tv_conv_dims {
   int32_t B, H, T, dk, dv;

@@ -6,14 +6,16 @@
 // operator needs W unpack+multiply-add pairs, a SiLU (two special-function operations) and its
 // share of the row normalisation: about 20 instructions per 4 bytes moved, so on this GPU the
 // kernel is bound by instruction issue before it is bound by HBM.  The design therefore spends
-// its effort on instructions per element: persistent CTAs walk (request, head, q|k|v) slices so
-// that the filter stays in registers, rows arrive by cp.async one item ahead, each node's W tap
-// rows are derived from the parent array once per item into a table of shared-memory offsets,
-// and a half-warp owns a node row (8 channels per lane), so a row's sum of squares is a 4-step
-// shuffle reduction and the row leaves as contiguous 16-byte stores.
+// its effort on instructions per element and on keeping the warps busy: persistent CTAs walk
+// (request, head, q|k|v) slices so that the filter stays in registers; the rows of an item arrive
+// as one TMA box two items ahead and are handed over through mbarriers, so the eight warps of a
+// CTA never meet at a CTA-wide barrier; each half-warp derives the W tap rows of its own node rows
+// from the parent array; and a half-warp owns a node row (8 channels per lane), so a row's sum of
+// squares is a 4-step shuffle reduction and the row leaves as contiguous 16-byte stores.
 #include <cuda_bf16.h>
 
 #include "tv_internal.h"
+#include "tv_tc_common.cuh"
 
 namespace {
 
@@ -31,7 +33,8 @@ struct ConvArgs {
   int32_t capacity;       // packed forest: rows of one output plane
   int32_t n_trees;
   int32_t B, H, T, dk, dv, W, normalize;
-  int32_t single;  // one row buffer only (two do not fit): no prefetch of the next item's rows
+  int32_t slots;   // row buffers of a CTA (1..3): items requested slots - 1 ahead
+  int32_t* status; // device status word of the tree (a wait that ran out is reported there)
   float eps;
   const void* x;      // [B][T][C]
   const void* ctx;    // [B][W-1][C]
@@ -76,10 +79,9 @@ template <> struct Geo<float> {
   static __device__ __forceinline__ int g1(int l16) { return 64 + 4 * l16; }
 };
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ uint4 lds16(uint32_t addr) {
   uint4 r;
-  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "r"(addr));
+  asm("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "r"(addr));
   return r;
 }
 
@@ -159,53 +161,77 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
 __device__ __forceinline__ void cp_async4(uint32_t dst, const void* src) {
   asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
 }
-__device__ __forceinline__ void cp_async_wait_all() {
-  asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
-}
 
 // Work items are (slice, request) pairs, slice-major, where a slice is one head's q, k or v
 // channels; a CTA walks a contiguous range of them, so its filter registers are reloaded only
-// when the slice changes.  Shared memory, every block on a 16-byte boundary:
-//   2 x [T+W-1][d] staged rows (context rows first, oldest first, then the nodes),
-//   2 x [T] parents, 2 x [T][WP] byte offsets of each node's tap rows (WP = 4 or 8),
-//   2 x ([128 NJ][W] filter taps + [128 NJ] bias) of a slice; every group of 8 channels is shifted
-//   by two words, so that the 16 lanes of a row, which own 8 channels each, read 16 banks.
-// While item n is computed, the rows of item n+1 (with the filter of its slice, when that is a
-// new one) and the parents of item n+2 are in flight (cp.async) and the tap table of item n+1
-// is derived: one __syncthreads per item, and no load whose latency is exposed after the first.
+// when the slice changes.  Shared memory:
+//   NS x slot: [T][d] node rows (one TMA box of x) then [W-1][d] context rows, oldest first,
+//   NS x [T] parents,
+//   4 x ([128 NJ][W] filter taps + [128 NJ] bias) of a slice; every group of 8 channels is shifted
+//   by two words, so that the 16 lanes of a row, which own 8 channels each, read 16 banks,
+//   NS x (full, empty) mbarriers.
+// The eight warps run from item to item without a CTA-wide barrier.  Item n lives in slot n % NS.
+// One warp (n % 8) requests item n + NS - 1 when it has finished item n (NS >= 3; with fewer slots,
+// before it starts item n): the row box by TMA, parents, context rows and -- when the slice
+// changes -- the filter by cp.async, all arriving on the slot's `full` barrier; before that it
+// waits on the slot's `empty` barrier, on which every warp arrives when it has read the item that
+// lived there.  Each half-warp derives the tap rows of the node rows it owns itself (lane k walks
+// the parents of the half-warp's k-th row once per item; the row loop fetches them by shuffle),
+// so nothing a warp needs is produced by another warp.
 struct ConvItem {
   int slice, b, kind, h, d, c0;
   int n;          // node rows of this request
   int row0;       // first row of the request in x and in the gate inputs
   size_t orow0;   // first row of this (request, head) in q/k/v and in the gate outputs
+  int fc;         // slice changes since the CTA's first item: filter buffer fc % 4
 };
+
+constexpr long long kConvDrainCycles = 1ll << 21;   // ~1 ms: copies still in flight after a timeout
 
 template <typename IO, int W, int NJ>
 __global__ void __launch_bounds__(kConvThreads, (NJ == 1 && W <= 4) ? kConvMinBlocks : 1)
-tree_conv_kernel(const ConvArgs a) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
+tree_conv_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+                 const ConvArgs a) {
+  using namespace tvtc;
+  extern __shared__ __align__(128) unsigned char smem_raw[];
   constexpr int VEC = 16 / (int)sizeof(IO);
-  constexpr int WP = W <= 4 ? 4 : 8;
   const int T = a.T, H = a.H, B = a.B, dk = a.dk, dv = a.dv;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, l16 = lane & 15, half = lane >> 4;
   const int C = H * (2 * dk + dv);
   const int dmax = dk > dv ? dk : dv;
   const int Tp = (T + 3) & ~3;
-  const bool single = a.single != 0;
+  const int NS = a.slots, PD = NS - 1;
+  const bool issue_first = NS < 3;
 
-  const uint32_t buf_bytes = (uint32_t)(T + W - 1) * dmax * sizeof(IO);
-  const uint32_t xs_u32 = smem_u32(smem_raw);
-  int32_t* par_s = reinterpret_cast<int32_t*>(smem_raw + (single ? 1 : 2) * (size_t)buf_bytes);  // [2][Tp]
-  uint32_t* taps_s = reinterpret_cast<uint32_t*>(par_s + 2 * Tp);                                // [2][T][WP]
-  constexpr int kBiasAt = 128 * NJ * W + 32 * NJ;         // words; kFiltAt(c, t) below
+  constexpr int kBiasAt = 128 * NJ * W + 32 * NJ;         // words
   constexpr int kFiltFloats = kBiasAt + 128 * NJ + 32 * NJ;
-  float* filt_s = reinterpret_cast<float*>(taps_s + 2 * T * WP);                                 // [2][kFiltFloats]
-  const uint32_t par_u32 = smem_u32(par_s), taps_u32 = smem_u32(taps_s), filt_u32 = smem_u32(filt_s);
+  const uint32_t slot_bytes = ((uint32_t)(T + W - 1) * dmax * sizeof(IO) + 127u) & ~127u;
+  const uint32_t xs_u32 = smem_u32(smem_raw);
+  const int32_t* par_s = reinterpret_cast<const int32_t*>(smem_raw + (size_t)NS * slot_bytes);   // [NS][Tp]
+  const float* filt_s = reinterpret_cast<const float*>(par_s + NS * Tp);                          // [4][kFiltFloats]
+  const uint32_t par_u32 = smem_u32(par_s), filt_u32 = smem_u32(filt_s);
+  const uint32_t bar_u32 = filt_u32 + 4 * kFiltFloats * 4;   // full[NS], empty[NS] (8 bytes each)
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_raw + (bar_u32 - xs_u32) + 16 * NS);
+  auto full_bar = [&](int s) { return bar_u32 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_u32 + 8u * (NS + s); };
 
+  if ((xs_u32 & 127u) != 0) {   // TMA wants its destination on a 128-byte boundary
+    if (tid == 0 && a.status) atomicExch(a.status, (int)TV_ERR_CUDA);
+    return;
+  }
   const long long n_items = 3LL * H * B;
   const int first = (int)(n_items * blockIdx.x / gridDim.x);
-  const int last = (int)(n_items * (blockIdx.x + 1) / gridDim.x);
-  if (first >= last) return;
+  const int count = (int)(n_items * (blockIdx.x + 1) / gridDim.x) - first;
+  if (count <= 0) return;
+  if (tid == 0) {
+    for (int s = 0; s < NS; ++s) {
+      mbar_init(full_bar(s), 33);            // the issuing warp: expect_tx by lane 0, cp.async arrivals of 32 lanes
+      mbar_init(empty_bar(s), kConvWarps);
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
 
   // item cursors advance without divisions
   auto set_slice = [&](ConvItem& it) {
@@ -231,6 +257,7 @@ tree_conv_kernel(const ConvArgs a) {
     if (++it.b == B) {
       it.b = 0;
       ++it.slice;
+      ++it.fc;
       set_slice(it);
     }
     set_request(it);
@@ -238,95 +265,55 @@ tree_conv_kernel(const ConvArgs a) {
   ConvItem cur;
   cur.slice = first / B;
   cur.b = first - cur.slice * B;
+  cur.fc = 0;
   set_slice(cur);
   set_request(cur);
-  ConvItem nxt = cur;
-  advance(nxt);
-  int b2 = nxt.b + 1 == B ? 0 : nxt.b + 1;  // request of the item after next
+  ConvItem pre = cur;   // the item PD ahead of cur (meaningful while it exists)
+  int pre_fc_prev = -1; // filter buffer generation of the item in front of `pre`
 
-  // This thread's share of a row block: 16-byte vector tid, tid + 256, ... of [rows][d/VEC];
-  // 256 consecutive vectors advance (rstep rows, cstep vectors).  Recomputed when d changes.
-  int g_d = -1, vpr = 1, rstep = 0, cstep = 0, row0 = 0, cv0 = 0;
-  auto set_geometry = [&](int d) {
-    g_d = d;
-    vpr = d / VEC;
-    rstep = kConvThreads / vpr;
-    cstep = kConvThreads - rstep * vpr;
-    row0 = tid / vpr;
-    cv0 = tid - row0 * vpr;
-  };
-  auto fetch_parents = [&](int b, int slot) {
-    if (tid < T)
-      cp_async4(par_u32 + (uint32_t)(slot * Tp + tid) * 4, a.parent + (size_t)(a.n_trees == 1 ? 0 : b) * T + tid);
-  };
-  auto fetch_rows = [&](const ConvItem& it, int slot) {
-    if (it.d != g_d) set_geometry(it.d);
-    const IO* xb = reinterpret_cast<const IO*>(a.x) + (size_t)it.row0 * C + it.c0;
-    const IO* cb = reinterpret_cast<const IO*>(a.ctx) + (size_t)it.b * (W - 1) * C + it.c0;
-    const uint32_t dctx = xs_u32 + (uint32_t)slot * buf_bytes;
-    const uint32_t dx = dctx + (uint32_t)((W - 1) * it.d * sizeof(IO));
-    int row = row0, cv = cv0;
-    while (row < W - 1) {  // context rows
-      cp_async16(dctx + (uint32_t)((row * it.d + cv * VEC) * sizeof(IO)), cb + (row * C + cv * VEC));
-      row += rstep;
-      cv += cstep;
-      if (cv >= vpr) { cv -= vpr; ++row; }
+  // The whole warp requests item m (descriptor `it`, slot m % NS).  False: a wait ran out.
+  auto issue = [&](int m, int slot, const ConvItem& it, bool new_filter) -> bool {
+    if (m >= NS && !mbar_wait_warp(empty_bar(slot), (uint32_t)((m / NS - 1) & 1), abort_flag)) return false;
+    const uint32_t dst = xs_u32 + (uint32_t)slot * slot_bytes;
+    const uint32_t row_bytes = (uint32_t)it.d * sizeof(IO);
+    if (lane == 0) {
+      mbar_expect_tx(full_bar(slot), (uint32_t)T * row_bytes);
+      tma_load_2d(dst, it.kind == 2 ? &map_v : &map_k, full_bar(slot), it.c0, it.row0);
     }
-    row = row0;
-    cv = cv0;
-    while (row < it.n) {  // node rows
-      cp_async16(dx + (uint32_t)((row * it.d + cv * VEC) * sizeof(IO)), xb + (row * C + cv * VEC));
-      row += rstep;
-      cv += cstep;
-      if (cv >= vpr) { cv -= vpr; ++row; }
-    }
-  };
-  // the slice's d x W filter taps and d bias values, contiguous in global memory
-  auto fetch_filter = [&](const ConvItem& it, int slot) {
-    const uint32_t dst = filt_u32 + (uint32_t)(slot * kFiltFloats) * 4;
-    const float* wsrc = a.weight + (size_t)it.c0 * W;
-    for (int c = tid; c < it.d; c += kConvThreads) {
-      const uint32_t shift = 2 * (c >> 3);
+    const int32_t* psrc = a.parent + (size_t)(a.n_trees == 1 ? 0 : it.b) * T;
+    for (int i = lane; i < T; i += 32) cp_async4(par_u32 + (uint32_t)(slot * Tp + i) * 4, psrc + i);
+    if (W > 1) {
+      const IO* cb = reinterpret_cast<const IO*>(a.ctx) + (size_t)it.b * (W - 1) * C + it.c0;
+      const int vpr = it.d / VEC;
 #pragma unroll
-      for (int t = 0; t < W; ++t) cp_async4(dst + (c * W + t + shift) * 4, wsrc + c * W + t);
-      if (a.bias != nullptr) cp_async4(dst + (kBiasAt + c + shift) * 4, a.bias + it.c0 + c);
+      for (int r = 0; r < W - 1; ++r)
+        for (int cv = lane; cv < vpr; cv += 32)
+          cp_async16(dst + (uint32_t)(T + r) * row_bytes + cv * 16, cb + (size_t)r * C + cv * VEC);
     }
-  };
-  // (the last warps do this, the first ones prepare the gates: neither is late at the barrier)
-  auto build_taps = [&](const ConvItem& it, int slot) {
-    const int node = kConvThreads - 1 - tid;
-    if (node < it.n) {
-      const uint32_t row_bytes = (uint32_t)it.d * sizeof(IO);
-      const int32_t* par = par_s + slot * Tp;
-      int j = node, ctx_row = W - 2;
+    if (new_filter) {
+      const uint32_t fdst = filt_u32 + (uint32_t)((it.fc & 3) * kFiltFloats) * 4;
+      const float* wsrc = a.weight + (size_t)it.c0 * W;
+      for (int c = lane; c < it.d; c += 32) {
+        const uint32_t shift = 2 * (c >> 3);
 #pragma unroll
-      for (int r = 0; r < W; ++r) {
-        int row;
-        if (j >= 0) {
-          row = W - 1 + j;
-          j = par[j];
-        } else {
-          row = ctx_row--;
-        }
-        taps_s[(slot * T + node) * WP + r] = (uint32_t)row * row_bytes;
+        for (int t = 0; t < W; ++t) cp_async4(fdst + (c * W + t + shift) * 4, wsrc + c * W + t);
+        if (a.bias != nullptr) cp_async4(fdst + (kBiasAt + c + shift) * 4, a.bias + it.c0 + c);
       }
     }
+    cp_async_arrive(full_bar(slot));
+    return true;
   };
 
-  // ---- prologue: parents of the first two items, rows of the first, taps of the first
-  fetch_parents(cur.b, 0);
-  if (first + 1 < last) fetch_parents(nxt.b, 1);
-  if (!single) fetch_rows(cur, 0);
-  fetch_filter(cur, 0);
-  cp_async_wait_all();
-  __syncthreads();
-  build_taps(cur, 0);
+  // ---- prologue: the first PD items (the first one when there is a single slot)
+  {
+    const int ahead = PD > 0 ? PD : 0;
+    for (int m = 0; m < ahead && m < count; ++m) {
+      if (warp == (m & (kConvWarps - 1))) issue(m, m, pre, pre.fc != pre_fc_prev);
+      pre_fc_prev = pre.fc;
+      advance(pre);
+    }
+  }
 
-  // Dead channel groups (past the slice's width) keep zero weights and read the row's first
-  // bytes, so the row loop is straight-line code; only their store is predicated off.
-  float wreg[NJ][W][8], breg[NJ][8];
-  bool live0[NJ], live1[NJ];
-  uint32_t off0[NJ], off1[NJ];
   // this thread's gate input of an item (alpha with the q slice, beta with the k slice), loaded
   // one item ahead
   auto fetch_gate = [&](const ConvItem& it) -> IO {
@@ -335,32 +322,31 @@ tree_conv_kernel(const ConvArgs a) {
     return reinterpret_cast<const IO*>(src)[((size_t)it.row0 + tid) * H + it.h];
   };
   IO gate_next = fetch_gate(cur);
-  int loaded_slice = -1, fslot = 0;   // fslot: the buffer that holds the filter of cur's slice
+
+  // Dead channel groups (past the slice's width) keep zero weights and read the row's first
+  // bytes, so the row loop is straight-line code; only their store is predicated off.
+  float wreg[NJ][W][8], breg[NJ][8];
+  bool live0[NJ], live1[NJ];
+  uint32_t off0[NJ], off1[NJ];
+  int loaded_slice = -1;
   const float eps = a.eps;
   const bool want_norm = a.normalize != 0;
+  bool ok = true;
+  int slot = 0, pre_slot = PD % NS, n = 0;
+  uint32_t phase = 0;   // parity of the slot's `full` barrier for item n
 
-  for (int item = first; item < last; ++item) {
-    const int s = (item - first) & 1, xs_slot = single ? 0 : s;
-    // rows of this item and parents of the next have landed; everyone is done with the last item
-    cp_async_wait_all();
-    __syncthreads();
-    if (single) {
-      fetch_rows(cur, 0);
-      cp_async_wait_all();
-      __syncthreads();
+  for (; n < count; ++n) {
+    if (issue_first && n + PD < count) {
+      if (warp == ((n + PD) & (kConvWarps - 1)) && !issue(n + PD, pre_slot, pre, pre.fc != pre_fc_prev)) { ok = false; break; }
     }
-    if (item + 1 < last) {
-      if (!single) fetch_rows(nxt, s ^ 1);
-      if (item + 2 < last) fetch_parents(b2, s);
-      if (nxt.slice != cur.slice) fetch_filter(nxt, fslot ^ 1);
-      build_taps(nxt, s ^ 1);
-    }
-    const int d = cur.d, c0 = cur.c0;
+    if (!mbar_wait_warp(full_bar(slot), phase, abort_flag)) { ok = false; break; }
+    const int d = cur.d;
+    const uint32_t row_bytes = (uint32_t)d * sizeof(IO);
 
     // ---- this lane's filter taps and bias, when the slice changes
     if (cur.slice != loaded_slice) {
       loaded_slice = cur.slice;
-      const float* wf = filt_s + fslot * kFiltFloats;
+      const float* wf = filt_s + (cur.fc & 3) * kFiltFloats;
       const float* bf = wf + kBiasAt;
 #pragma unroll
       for (int j = 0; j < NJ; ++j) {
@@ -387,39 +373,50 @@ tree_conv_kernel(const ConvArgs a) {
     const bool do_alpha = cur.kind == 0 && a.gate_a != nullptr && tid < cur.n;
     const bool do_beta = cur.kind == 1 && a.gate_b != nullptr && tid < cur.n;
     const IO gate_raw = gate_next;
-    if (item + 1 < last) gate_next = fetch_gate(nxt);
     float gate_A = 0.f, gate_dt = 0.f;
     if (do_alpha) {
       gate_A = __ldg(a.A_log + cur.h);
       gate_dt = __ldg(a.dt_bias + cur.h);
     }
 
-    // ---- each half-warp takes one node row at a time (the last row is repeated, unstored,
-    // when T is odd)
-    IO* out = reinterpret_cast<IO*>(cur.kind == 0 ? a.q : cur.kind == 1 ? a.k : a.v) + cur.orow0 * d;
+    // ---- tap rows: lane k of a half-warp walks the parents of the half-warp's k-th row
     const int Tn = cur.n;
+    const uint32_t xs_item = xs_u32 + (uint32_t)slot * slot_bytes;
+    uint32_t mytap[W];
+    {
+      const int32_t* par = par_s + slot * Tp;
+      int j = 2 * warp + half + 2 * kConvWarps * l16, ctx_row = W - 2;
+      if (j >= Tn) j = Tn - 1;   // rows past the end repeat the last one (computed, not stored)
+#pragma unroll
+      for (int r = 0; r < W; ++r) {
+        int row;
+        if (j >= 0) {
+          row = j;
+          j = par[j];
+        } else {
+          row = T + ctx_row--;
+        }
+        mytap[r] = (uint32_t)row * row_bytes;
+      }
+    }
+
+    // ---- each half-warp takes one node row at a time
+    IO* out = reinterpret_cast<IO*>(cur.kind == 0 ? a.q : cur.kind == 1 ? a.k : a.v) + cur.orow0 * d;
     const bool norm = want_norm && cur.kind < 2;
-    const uint32_t xs_item = xs_u32 + (uint32_t)xs_slot * buf_bytes;
-    const uint32_t taps_item = taps_u32 + (uint32_t)(s * T) * (WP * 4);
     uint32_t base0[NJ], base1[NJ];
 #pragma unroll
     for (int j = 0; j < NJ; ++j) {
       base0[j] = xs_item + off0[j];
       base1[j] = xs_item + off1[j];
     }
+    int src_lane = lane & 16;
 #pragma unroll kConvUnroll
-    for (int i0 = 2 * warp; i0 < Tn; i0 += 2 * kConvWarps) {
+    for (int i0 = 2 * warp; i0 < Tn; i0 += 2 * kConvWarps, ++src_lane) {
       const bool row_live = i0 + half < Tn;
       const int i = row_live ? i0 + half : Tn - 1;
-      uint32_t tap[WP];
-      {
-        const uint4 t0 = lds16(taps_item + (uint32_t)i * (WP * 4));
-        tap[0] = t0.x; tap[1] = t0.y; tap[2] = t0.z; tap[3] = t0.w;
-        if constexpr (WP == 8) {
-          const uint4 t1 = lds16(taps_item + (uint32_t)i * (WP * 4) + 16);
-          tap[4] = t1.x; tap[5] = t1.y; tap[6] = t1.z; tap[7] = t1.w;
-        }
-      }
+      uint32_t tap[W];
+#pragma unroll
+      for (int r = 0; r < W; ++r) tap[r] = __shfl_sync(0xffffffffu, mytap[r], src_lane);
       float y[NJ][8];
       float ss = 0.0f;
 #pragma unroll
@@ -448,12 +445,37 @@ tree_conv_kernel(const ConvArgs a) {
                row_live && live1[j], y[j]);
       }
     }
+    // this warp has read the slot
+    __syncwarp();
+    if (lane == 0) mbar_arrive(empty_bar(slot));
+
     if (do_alpha) a.alpha[cur.orow0 + tid] = exp_fast(-exp_fast(gate_A) * softplus(to_f32(gate_raw) + gate_dt));
     if (do_beta) a.beta[cur.orow0 + tid] = sigmoid_fast(to_f32(gate_raw));
-    if (nxt.slice != cur.slice) fslot ^= 1;
-    cur = nxt;
-    advance(nxt);
-    b2 = b2 + 1 == B ? 0 : b2 + 1;
+
+    if (!issue_first && n + PD < count) {
+      if (warp == ((n + PD) & (kConvWarps - 1)) && !issue(n + PD, pre_slot, pre, pre.fc != pre_fc_prev)) { ok = false; break; }
+    }
+    if (n + PD < count) {
+      pre_fc_prev = pre.fc;
+      advance(pre);
+      pre_slot = pre_slot + 1 == NS ? 0 : pre_slot + 1;
+    }
+    advance(cur);
+    if (n + 1 < count) gate_next = fetch_gate(cur);
+    if (++slot == NS) {
+      slot = 0;
+      phase ^= 1;
+    }
+  }
+
+  if (!ok) {
+    // A wait ran out (or another warp's did).  Copies requested for the items this warp has not
+    // consumed may still be in flight: give them a moment before the CTA's memory is released.
+    int dummy = 0;
+    for (int m = n; m <= n + PD && m < count; ++m)
+      mbar_wait(full_bar(m % NS), (uint32_t)((m / NS) & 1), &dummy, kConvDrainCycles);
+    asm volatile("cp.async.wait_all;" ::: "memory");
+    if (lane == 0 && a.status) atomicExch(a.status, (int)TV_ERR_DEVICE_TIMEOUT);
   }
 }
 
@@ -515,12 +537,29 @@ int check_conv(const tv_tree* t, const tv_conv_dims* d) {
 template <typename IO, int W>
 int launch_conv(const ConvArgs& a_in, cudaStream_t stream) {
   ConvArgs a = a_in;
+  constexpr bool kTwoPerSm = W <= 4;   // and d <= 128: the kernel's launch bounds
   const int dmax = a.dk > a.dv ? a.dk : a.dv;
-  const size_t buf = (size_t)(a.T + W - 1) * dmax * sizeof(IO);
-  const size_t tables = 2 * ((size_t)((a.T + 3) & ~3) * 4 + (size_t)a.T * (W <= 4 ? 4 : 8) * 4) +
-                        2 * (size_t)(dmax <= 128 ? 1 : 2) * (128 * (W + 1) + 64) * 4;
-  a.single = 2 * buf + tables > 200 * 1024;
-  const size_t smem = (a.single ? 1 : 2) * buf + tables;
+  const int NJ = dmax <= 128 ? 1 : 2;
+  const size_t slot = ((size_t)(a.T + W - 1) * dmax * sizeof(IO) + 127) & ~(size_t)127;
+  auto smem_for = [&](int ns) {
+    return ns * slot + (size_t)ns * ((a.T + 3) & ~3) * 4 + 4 * (size_t)NJ * (128 * (W + 1) + 64) * 4 + 16 * ns + 16;
+  };
+  // three slots with two CTAs per SM if that fits (a fourth measured slower: 41.4 against 39.4 us
+  // on B = 32, T = 64), else as many slots, up to three, as fit a CTA that has the SM's shared
+  // memory to itself
+  const size_t half_sm = 112 * 1024, whole_sm = 226 * 1024;
+  if (kTwoPerSm && NJ == 1 && smem_for(3) <= half_sm) a.slots = 3;
+  else a.slots = smem_for(3) <= whole_sm ? 3 : smem_for(2) <= whole_sm ? 2 : 1;
+  const size_t smem = smem_for(a.slots);
+  if (smem > whole_sm) return TV_ERR_UNSUPPORTED;
+  // x as a [rows][C] tensor; one box = the T node rows of a request x the d channels of a slice
+  const int C = a.H * (2 * a.dk + a.dv);
+  const uint64_t rows = a.offsets ? (uint64_t)a.capacity : (uint64_t)a.B * a.T;
+  const CUtensorMapDataType dt = sizeof(IO) == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
+  alignas(64) CUtensorMap map_k, map_v;
+  if (!tvtc::make_map2_plain(&map_k, a.x, dt, sizeof(IO), rows, C, a.dk, a.T) ||
+      !tvtc::make_map2_plain(&map_v, a.x, dt, sizeof(IO), rows, C, a.dv, a.T))
+    return TV_ERR_CUDA;
   int dev = 0, sms = 0;
   TV_CUDA_TRY(cudaGetDevice(&dev));
   TV_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
@@ -532,11 +571,11 @@ int launch_conv(const ConvArgs& a_in, cudaStream_t stream) {
     if (per_sm < 1) return TV_ERR_UNSUPPORTED;
     const long long items = 3LL * a.H * a.B, slots = (long long)sms * per_sm;
     const unsigned grid = (unsigned)(items < slots ? items : slots);
-    kernel<<<grid, kConvThreads, smem, stream>>>(a);
+    kernel<<<grid, kConvThreads, smem, stream>>>(map_k, map_v, a);
     TV_CUDA_TRY(cudaGetLastError());
     return TV_OK;
   };
-  return dmax <= 128 ? go(tree_conv_kernel<IO, W, 1>) : go(tree_conv_kernel<IO, W, 2>);
+  return NJ == 1 ? go(tree_conv_kernel<IO, W, 1>) : go(tree_conv_kernel<IO, W, 2>);
 }
 
 template <typename IO>
@@ -608,7 +647,7 @@ TV_API int tv_tree_conv(const tv_tree* tree, const tv_conv_dims* d, const void* 
   a.parent = tree->d_parent; a.n_trees = tree->n_trees;
   a.offsets = tree->d_offsets; a.capacity = tree->capacity;
   a.B = d->B; a.H = d->H; a.T = d->T; a.dk = d->dk; a.dv = d->dv; a.W = d->W;
-  a.normalize = d->normalize_qk != 0; a.eps = d->eps;
+  a.normalize = d->normalize_qk != 0; a.eps = d->eps; a.slots = 0; a.status = tree->d_status;
   a.x = x; a.ctx = ctx; a.weight = weight; a.bias = bias; a.gate_a = gate_a; a.gate_b = gate_b;
   a.A_log = A_log; a.dt_bias = dt_bias; a.q = q; a.k = k; a.v = v; a.alpha = alpha; a.beta = beta;
   return d->io_dtype == TV_BF16 ? launch_conv_w<__nv_bfloat16>(a, (cudaStream_t)stream)
