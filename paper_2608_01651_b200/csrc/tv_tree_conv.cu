@@ -35,6 +35,7 @@ struct ConvArgs {
   int32_t B, H, T, dk, dv, W, normalize;
   int32_t slots;   // row buffers of a CTA (1..3): items requested slots - 1 ahead
   int32_t* status; // device status word of the tree (a wait that ran out is reported there)
+  tvtc::FastDiv dB, dH;   // item -> (slice, request), slice -> (q|k|v, head)
   float eps;
   const void* x;      // [B][T][C]
   const void* ctx;    // [B][W-1][C]
@@ -182,8 +183,7 @@ struct ConvItem {
   int slice, b, kind, h, d, c0;
   int n;          // node rows of this request
   int row0;       // first row of the request in x and in the gate inputs
-  size_t orow0;   // first row of this (request, head) in q/k/v and in the gate outputs
-  int fc;         // slice changes since the CTA's first item: filter buffer fc % 4
+  uint32_t orow;  // first row of this (request, head) in q/k/v and in the gate outputs
 };
 
 constexpr long long kConvDrainCycles = 1ll << 21;   // ~1 ms: copies still in flight after a timeout
@@ -233,9 +233,10 @@ tree_conv_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
   }
   __syncthreads();
 
-  // item cursors advance without divisions
+  // An item's coordinates.  The cursor of the item being computed advances without divisions;
+  // the warp that requests an item derives that item's coordinates from its number.
   auto set_slice = [&](ConvItem& it) {
-    it.kind = it.slice / H;
+    it.kind = (int)tvtc::fdiv((uint32_t)it.slice, a.dH);
     it.h = it.slice - it.kind * H;
     it.d = it.kind == 2 ? dv : dk;
     it.c0 = it.kind == 0 ? it.h * dk : it.kind == 1 ? (H + it.h) * dk : 2 * H * dk + it.h * dv;
@@ -246,34 +247,31 @@ tree_conv_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
     if (a.offsets == nullptr) {
       it.n = T;
       it.row0 = it.b * T;
-      it.orow0 = ((size_t)it.b * H + it.h) * T;
-    } else if (it.slice < 3 * H) {
+      it.orow = (uint32_t)(it.b * H + it.h) * (uint32_t)T;
+    } else {
       it.row0 = a.offsets[it.b];
       it.n = a.offsets[it.b + 1] - it.row0;
-      it.orow0 = (size_t)it.h * a.capacity + it.row0;
+      it.orow = (uint32_t)it.h * (uint32_t)a.capacity + (uint32_t)it.row0;
     }
   };
-  auto advance = [&](ConvItem& it) {
-    if (++it.b == B) {
-      it.b = 0;
-      ++it.slice;
-      ++it.fc;
-      set_slice(it);
-    }
+  auto describe = [&](int item) {
+    ConvItem it;
+    it.slice = (int)tvtc::fdiv((uint32_t)item, a.dB);
+    it.b = item - it.slice * B;
+    set_slice(it);
     set_request(it);
+    return it;
   };
-  ConvItem cur;
-  cur.slice = first / B;
-  cur.b = first - cur.slice * B;
-  cur.fc = 0;
-  set_slice(cur);
-  set_request(cur);
-  ConvItem pre = cur;   // the item PD ahead of cur (meaningful while it exists)
-  int pre_fc_prev = -1; // filter buffer generation of the item in front of `pre`
+  const int slice_first = (int)tvtc::fdiv((uint32_t)first, a.dB);
+  ConvItem cur = describe(first);
 
   // The whole warp requests item m (descriptor `it`, slot m % NS).  False: a wait ran out.
-  auto issue = [&](int m, int slot, const ConvItem& it, bool new_filter) -> bool {
-    if (m >= NS && !mbar_wait_warp(empty_bar(slot), (uint32_t)((m / NS - 1) & 1), abort_flag)) return false;
+  // `use` = m / NS, how often the slot has been filled before.
+  auto issue = [&](int m, int slot, int use) -> bool {
+    if (use > 0 && !mbar_wait_warp(empty_bar(slot), (uint32_t)((use - 1) & 1), abort_flag)) return false;
+    const ConvItem it = describe(first + m);
+    const int fc = it.slice - slice_first;   // slice changes since the CTA's first item: filter buffer fc % 4
+    const bool new_filter = m == 0 || it.b == 0;
     const uint32_t dst = xs_u32 + (uint32_t)slot * slot_bytes;
     const uint32_t row_bytes = (uint32_t)it.d * sizeof(IO);
     if (lane == 0) {
@@ -291,7 +289,7 @@ tree_conv_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
           cp_async16(dst + (uint32_t)(T + r) * row_bytes + cv * 16, cb + (size_t)r * C + cv * VEC);
     }
     if (new_filter) {
-      const uint32_t fdst = filt_u32 + (uint32_t)((it.fc & 3) * kFiltFloats) * 4;
+      const uint32_t fdst = filt_u32 + (uint32_t)((fc & 3) * kFiltFloats) * 4;
       const float* wsrc = a.weight + (size_t)it.c0 * W;
       for (int c = lane; c < it.d; c += 32) {
         const uint32_t shift = 2 * (c >> 3);
@@ -307,11 +305,8 @@ tree_conv_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
   // ---- prologue: the first PD items (the first one when there is a single slot)
   {
     const int ahead = PD > 0 ? PD : 0;
-    for (int m = 0; m < ahead && m < count; ++m) {
-      if (warp == (m & (kConvWarps - 1))) issue(m, m, pre, pre.fc != pre_fc_prev);
-      pre_fc_prev = pre.fc;
-      advance(pre);
-    }
+    for (int m = 0; m < ahead && m < count; ++m)
+      if (warp == (m & (kConvWarps - 1))) issue(m, m, 0);
   }
 
   // this thread's gate input of an item (alpha with the q slice, beta with the k slice), loaded
@@ -319,7 +314,7 @@ tree_conv_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
   auto fetch_gate = [&](const ConvItem& it) -> IO {
     const void* src = it.kind == 0 ? a.gate_a : it.kind == 1 ? a.gate_b : nullptr;
     if (src == nullptr || tid >= it.n) return IO(0.0f);
-    return reinterpret_cast<const IO*>(src)[((size_t)it.row0 + tid) * H + it.h];
+    return reinterpret_cast<const IO*>(src)[(uint32_t)(it.row0 + tid) * (uint32_t)H + (uint32_t)it.h];
   };
   IO gate_next = fetch_gate(cur);
 
@@ -332,12 +327,13 @@ tree_conv_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
   const float eps = a.eps;
   const bool want_norm = a.normalize != 0;
   bool ok = true;
-  int slot = 0, pre_slot = PD % NS, n = 0;
-  uint32_t phase = 0;   // parity of the slot's `full` barrier for item n
+  int slot = 0, n = 0;
+  int pre_slot = PD, pre_use = 0;   // slot of item n + PD and how often it has been filled
+  uint32_t phase = 0;               // parity of the slot's `full` barrier for item n
 
   for (; n < count; ++n) {
     if (issue_first && n + PD < count) {
-      if (warp == ((n + PD) & (kConvWarps - 1)) && !issue(n + PD, pre_slot, pre, pre.fc != pre_fc_prev)) { ok = false; break; }
+      if (warp == ((n + PD) & (kConvWarps - 1)) && !issue(n + PD, pre_slot, pre_use)) { ok = false; break; }
     }
     if (!mbar_wait_warp(full_bar(slot), phase, abort_flag)) { ok = false; break; }
     const int d = cur.d;
@@ -346,7 +342,7 @@ tree_conv_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
     // ---- this lane's filter taps and bias, when the slice changes
     if (cur.slice != loaded_slice) {
       loaded_slice = cur.slice;
-      const float* wf = filt_s + (cur.fc & 3) * kFiltFloats;
+      const float* wf = filt_s + ((cur.slice - slice_first) & 3) * kFiltFloats;
       const float* bf = wf + kBiasAt;
 #pragma unroll
       for (int j = 0; j < NJ; ++j) {
@@ -401,7 +397,7 @@ tree_conv_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
     }
 
     // ---- each half-warp takes one node row at a time
-    IO* out = reinterpret_cast<IO*>(cur.kind == 0 ? a.q : cur.kind == 1 ? a.k : a.v) + cur.orow0 * d;
+    IO* out = reinterpret_cast<IO*>(cur.kind == 0 ? a.q : cur.kind == 1 ? a.k : a.v) + (size_t)cur.orow * d;
     const bool norm = want_norm && cur.kind < 2;
     uint32_t base0[NJ], base1[NJ];
 #pragma unroll
@@ -449,19 +445,25 @@ tree_conv_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
     __syncwarp();
     if (lane == 0) mbar_arrive(empty_bar(slot));
 
-    if (do_alpha) a.alpha[cur.orow0 + tid] = exp_fast(-exp_fast(gate_A) * softplus(to_f32(gate_raw) + gate_dt));
-    if (do_beta) a.beta[cur.orow0 + tid] = sigmoid_fast(to_f32(gate_raw));
+    if (do_alpha) a.alpha[cur.orow + tid] = exp_fast(-exp_fast(gate_A) * softplus(to_f32(gate_raw) + gate_dt));
+    if (do_beta) a.beta[cur.orow + tid] = sigmoid_fast(to_f32(gate_raw));
 
     if (!issue_first && n + PD < count) {
-      if (warp == ((n + PD) & (kConvWarps - 1)) && !issue(n + PD, pre_slot, pre, pre.fc != pre_fc_prev)) { ok = false; break; }
+      if (warp == ((n + PD) & (kConvWarps - 1)) && !issue(n + PD, pre_slot, pre_use)) { ok = false; break; }
     }
-    if (n + PD < count) {
-      pre_fc_prev = pre.fc;
-      advance(pre);
-      pre_slot = pre_slot + 1 == NS ? 0 : pre_slot + 1;
+    if (++pre_slot == NS) {
+      pre_slot = 0;
+      ++pre_use;
     }
-    advance(cur);
-    if (n + 1 < count) gate_next = fetch_gate(cur);
+    if (n + 1 < count) {
+      if (++cur.b == B) {
+        cur.b = 0;
+        ++cur.slice;
+        set_slice(cur);
+      }
+      set_request(cur);
+      gate_next = fetch_gate(cur);
+    }
     if (++slot == NS) {
       slot = 0;
       phase ^= 1;
@@ -530,6 +532,9 @@ int check_conv(const tv_tree* t, const tv_conv_dims* d) {
   if (t->n_trees != 1 && t->n_trees != d->B) return TV_ERR_BAD_ARG;
   if (!t->offsets.empty() && t->n_trees != d->B) return TV_ERR_BAD_ARG;
   if ((int64_t)d->B * d->H * 3 > 0x7fffffffLL || d->B > 65535) return TV_ERR_UNSUPPORTED;
+  // rows of an output plane and gate elements are indexed in 32 bits
+  const int64_t out_rows = t->offsets.empty() ? (int64_t)d->B * d->H * d->T : (int64_t)d->H * t->capacity;
+  if (out_rows > 0x7fffffffLL) return TV_ERR_UNSUPPORTED;
   if (!t->uploaded) return TV_ERR_NOT_UPLOADED;
   return TV_OK;
 }
@@ -648,6 +653,7 @@ TV_API int tv_tree_conv(const tv_tree* tree, const tv_conv_dims* d, const void* 
   a.offsets = tree->d_offsets; a.capacity = tree->capacity;
   a.B = d->B; a.H = d->H; a.T = d->T; a.dk = d->dk; a.dv = d->dv; a.W = d->W;
   a.normalize = d->normalize_qk != 0; a.eps = d->eps; a.slots = 0; a.status = tree->d_status;
+  a.dB = tvtc::make_fastdiv((uint32_t)d->B); a.dH = tvtc::make_fastdiv((uint32_t)d->H);
   a.x = x; a.ctx = ctx; a.weight = weight; a.bias = bias; a.gate_a = gate_a; a.gate_b = gate_b;
   a.A_log = A_log; a.dt_bias = dt_bias; a.q = q; a.k = k; a.v = v; a.alpha = alpha; a.beta = beta;
   return d->io_dtype == TV_BF16 ? launch_conv_w<__nv_bfloat16>(a, (cudaStream_t)stream)
