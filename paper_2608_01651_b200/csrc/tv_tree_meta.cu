@@ -3,6 +3,7 @@
 // and writes the strict-ancestor masks, depths and a device copy of the parents.  Nodes are
 // indexed parent before child, so walking parent links from node i visits exactly Anc(i).
 #include "tv_internal.h"
+#include "tv_tc_common.cuh"
 
 namespace {
 
@@ -16,21 +17,25 @@ tree_meta_kernel(const int32_t* __restrict__ parent, int32_t n, uint64_t* __rest
   // a verify kernel launched behind this one may be scheduled now and set itself up; it waits
   // for this grid to finish before it reads global memory
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // This kernel is itself launched as a dependent of the kernels in front of it.  The parents and
+  // offsets may be their output (a forest built on the device), and they may still be reading the
+  // metadata of the previous upload: nothing is read or written before they have finished.
+  tvtc::grid_dependency_wait();
   if (i < n) {
     // host-built trees are validated there; device-built ones (tv_forest_upload_device) are not:
     // an out-of-range parent is treated as a child of the virtual root so the walk stays in bounds
     const int p = parent[(size_t)t * n + i];
     par_s[i] = (p < -1 || p >= i) ? -1 : p;
   }
-  if (t == 0 && i == 0) *status = 0;
   // packed forest: the row offsets travel with the parents (tree t copies entry t, the last
   // tree also the end marker)
-  if (offsets != nullptr && i == 0) {
-    offsets_dev[t] = offsets[t];
-    if (t == (int)gridDim.x - 1) offsets_dev[t + 1] = offsets[t + 1];
+  int32_t off0 = 0, off1 = 0;
+  const bool copy_offsets = offsets != nullptr && i == 0, last_tree = t == (int)gridDim.x - 1;
+  if (copy_offsets) {
+    off0 = offsets[t];
+    if (last_tree) off1 = offsets[t + 1];
   }
   __syncthreads();
-  if (i >= n) return;
   uint64_t w0 = 0, w1 = 0;
   int d = 0;
   // -1 <= parent[j] < j holds by now, so the walk ends within n steps.  The caller's depth bound
@@ -38,11 +43,17 @@ tree_meta_kernel(const int32_t* __restrict__ parent, int32_t n, uint64_t* __rest
   // depth_bound ancestors only (every mask then fits those kernels' tables) and the upload is
   // marked as failed -- status[1] receives the generation of this upload (all CTAs write the same value),
   // which needs no clearing and so no ordering between the CTAs of this grid.
-  int p = par_s[i];
+  int p = i < n ? par_s[i] : -1;
   for (; p >= 0 && d < depth_bound; p = par_s[p]) {
     if (p < 64) w0 |= 1ull << p; else w1 |= 1ull << (p - 64);
     ++d;
   }
+  if (t == 0 && i == 0) *status = 0;
+  if (copy_offsets) {
+    offsets_dev[t] = off0;
+    if (last_tree) offsets_dev[t + 1] = off1;
+  }
+  if (i >= n) return;
   if (p >= 0) atomicExch(status + 1, generation);
   const size_t o = (size_t)t * n + i;
   anc[2 * o] = w0;
@@ -71,19 +82,23 @@ tree_meta_param_kernel(const __grid_constant__ ParentBytes<NB> pb, const __grid_
   const int t = blockIdx.x, i = threadIdx.x;
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // as in the kernel above
   if (i < n) par_s[i] = pb.p[t * n + i];
+  __syncthreads();
+  uint64_t w0 = 0, w1 = 0;
+  int d = 0;
+  for (int p = i < n ? par_s[i] : -1; p >= 0 && d < n; p = par_s[p]) {
+    if (p < 64) w0 |= 1ull << p; else w1 |= 1ull << (p - 64);
+    ++d;
+  }
+  // Everything above read the kernel's parameters only.  The kernels in front on the stream may
+  // still be reading the metadata of the previous upload (this kernel is launched as their
+  // dependent): nothing is written before they have finished.
+  tvtc::grid_dependency_wait();
   if (t == 0 && i == 0) *status = 0;
   if (has_offsets && i == 0) {
     offsets_dev[t] = off.o[t];
     if (t == (int)gridDim.x - 1) offsets_dev[t + 1] = off.o[t + 1];
   }
-  __syncthreads();
   if (i >= n) return;
-  uint64_t w0 = 0, w1 = 0;
-  int d = 0;
-  for (int p = par_s[i]; p >= 0 && d < n; p = par_s[p]) {
-    if (p < 64) w0 |= 1ull << p; else w1 |= 1ull << (p - 64);
-    ++d;
-  }
   const size_t o = (size_t)t * n + i;
   anc[2 * o] = w0;
   anc[2 * o + 1] = w1;
@@ -101,9 +116,9 @@ int launch_param(const int32_t* parent_host, int32_t n_trees, int32_t n, uint64_
   OffsetWords off;
   if (offsets_host)
     for (int i = 0; i <= n_trees; ++i) off.o[i] = offsets_host[i];
-  tree_meta_param_kernel<NB><<<n_trees, TV_MAX_NODES, 0, stream>>>(pb, off, offsets_host != nullptr, n, anc, depth,
-                                                                  parent_dev, status, offsets_dev);
-  TV_CUDA_TRY(cudaGetLastError());
+  TV_CUDA_TRY(tvtc::launch_dependent(tree_meta_param_kernel<NB>, n_trees, TV_MAX_NODES, 0, stream, pb, off,
+                                     (int32_t)(offsets_host != nullptr), n, anc, depth, parent_dev, status,
+                                     offsets_dev));
   return TV_OK;
 }
 
@@ -127,8 +142,7 @@ int tv_launch_tree_meta_params(const int32_t* parent_host, int32_t n_trees, int3
 int tv_launch_tree_meta(const int32_t* parent_mapped, int32_t n_trees, int32_t n, uint64_t* anc,
                         int32_t* depth, int32_t* parent_dev, int32_t* status, const int32_t* offsets_mapped,
                         int32_t* offsets_dev, int32_t depth_bound, int32_t generation, cudaStream_t stream) {
-  tree_meta_kernel<<<n_trees, TV_MAX_NODES, 0, stream>>>(parent_mapped, n, anc, depth, parent_dev, status,
-                                                        offsets_mapped, offsets_dev, depth_bound, generation);
-  TV_CUDA_TRY(cudaGetLastError());
+  TV_CUDA_TRY(tvtc::launch_dependent(tree_meta_kernel, n_trees, TV_MAX_NODES, 0, stream, parent_mapped, n, anc, depth,
+                                     parent_dev, status, offsets_mapped, offsets_dev, depth_bound, generation));
   return TV_OK;
 }
