@@ -231,7 +231,12 @@ tree_conv_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  // Dependent launches on both sides: the kernel behind this one may set itself up now (the
+  // library's kernels read nothing this one writes before their own wait), and this one has
+  // come this far under the tail of the kernel in front, whose output x may be.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   __syncthreads();
+  grid_dependency_wait();
 
   // An item's coordinates.  The cursor of the item being computed advances without divisions;
   // the warp that requests an item derives that item's coordinates from its number.
@@ -576,8 +581,7 @@ int launch_conv(const ConvArgs& a_in, cudaStream_t stream) {
     if (per_sm < 1) return TV_ERR_UNSUPPORTED;
     const long long items = 3LL * a.H * a.B, slots = (long long)sms * per_sm;
     const unsigned grid = (unsigned)(items < slots ? items : slots);
-    kernel<<<grid, kConvThreads, smem, stream>>>(map_k, map_v, a);
-    TV_CUDA_TRY(cudaGetLastError());
+    TV_CUDA_TRY(tvtc::launch_dependent(kernel, (int)grid, kConvThreads, smem, stream, map_k, map_v, a));
     return TV_OK;
   };
   return NJ == 1 ? go(tree_conv_kernel<IO, W, 1>) : go(tree_conv_kernel<IO, W, 2>);
