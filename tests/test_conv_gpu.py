@@ -138,6 +138,15 @@ def test_shapes(shape, dtype, W):
     run_case(wl, parents, W=W, normalize=bool(W & 2), gates=True, gate_b=bool(W & 4), bias=W != 2)
 
 
+@pytest.mark.parametrize("B,H", [(1, 160), (2, 100), (3, 70)])
+def test_many_slices_per_cta(B, H):
+    """More (slice, request) items than CTAs with one to three requests per slice: every CTA walks
+    several items whose filter changes with (almost) every item, through all of its slots."""
+    wl = dataclasses.replace(inputs.workload("c2"), B=B, H=H, T=12, dk=16, dv=8, seed=4000 + B)
+    parents, _ = inputs.make_trees(wl)
+    run_case(wl, parents, W=4, normalize=True, gates=True, gate_b=True)
+
+
 @pytest.mark.parametrize("kind", ["chain", "star", "shared"])
 def test_tree_kinds(kind):
     wl = dataclasses.replace(inputs.workload("c2"), B=3, H=2, T=40)
