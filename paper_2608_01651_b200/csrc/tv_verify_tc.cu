@@ -109,7 +109,6 @@ constexpr uint32_t kColQb = 0, kColSc = 128, kColAcc0 = 256, kColAcc1 = 384;
 
 constexpr uint32_t kIdescKK128 = idesc_bf16(128, false);
 constexpr uint32_t kIdescKK64 = idesc_bf16(64, false);
-constexpr uint32_t kIdescKMn = idesc_bf16(128, true);
 
 __device__ __forceinline__ void mma_bf16_ts(uint32_t d, uint32_t a_tmem, uint64_t b, uint32_t idesc,
                                             uint32_t accumulate) {
