@@ -98,6 +98,7 @@ __device__ __forceinline__ void st_stream(float4* p, const float4& v) {
 template <bool BF16>
 __global__ void __launch_bounds__(kThreads)
 commit_factored_kernel(const CommitArgs a, const __grid_constant__ CommitLayers tb) {
+  asm volatile("griddepcontrol.wait;" ::: "memory");   // dependent launch: nothing is read before the kernel in front is done
   __shared__ int path_s[TV_MAX_NODES];
   __shared__ float w_s[TV_MAX_NODES];
   __shared__ float Pa_s;
@@ -514,6 +515,7 @@ commit_stream_dk128_kernel(const CommitArgs a, const __grid_constant__ CommitLay
 template <bool BF16, int NPL>
 __global__ void __launch_bounds__(kThreads)
 commit_delta_rows_kernel(const CommitArgs a, const __grid_constant__ CommitLayers tb) {
+  asm volatile("griddepcontrol.wait;" ::: "memory");   // dependent launch: nothing is read before the kernel in front is done
   constexpr int DK = 32 * NPL;
   constexpr int kRowsPerWarp = TV_MAX_DIM / (kThreads / 32);  // 16
   __shared__ int path_s[TV_MAX_NODES];
@@ -623,10 +625,10 @@ commit_delta_rows_kernel(const CommitArgs a, const __grid_constant__ CommitLayer
 // kernel launched this way orders itself with griddepcontrol.wait.  Behind any other kernel this
 // is an ordinary launch.
 cudaError_t launch_after_verify(void (*kernel)(const CommitArgs, const CommitLayers), int ctas, cudaStream_t stream,
-                                const CommitArgs& a, const CommitLayers& tb) {
+                                const CommitArgs& a, const CommitLayers& tb, int threads = kRowThreads) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)ctas);
-  cfg.blockDim = dim3((unsigned)kRowThreads);
+  cfg.blockDim = dim3((unsigned)threads);
   cfg.dynamicSmemBytes = 0;
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
@@ -664,14 +666,14 @@ int tv_launch_commit(const CommitArgs& a, const CommitLayers& tb, cudaStream_t s
     TV_CUDA_TRY(a.bf16 ? launch_after_verify(commit_factored_dk128_kernel<true>, ctas, stream, a, tb)
                        : launch_after_verify(commit_factored_dk128_kernel<false>, ctas, stream, a, tb));
   } else if (!recompute) {
-    if (a.bf16) commit_factored_kernel<true><<<items, kThreads, 0, stream>>>(a, tb);
-    else commit_factored_kernel<false><<<items, kThreads, 0, stream>>>(a, tb);
+    TV_CUDA_TRY(a.bf16 ? launch_after_verify(commit_factored_kernel<true>, items, stream, a, tb, kThreads)
+                       : launch_after_verify(commit_factored_kernel<false>, items, stream, a, tb, kThreads));
   } else if (a.dk == 128) {
-    if (a.bf16) commit_delta_rows_kernel<true, 4><<<items, kThreads, 0, stream>>>(a, tb);
-    else commit_delta_rows_kernel<false, 4><<<items, kThreads, 0, stream>>>(a, tb);
+    TV_CUDA_TRY(a.bf16 ? launch_after_verify(commit_delta_rows_kernel<true, 4>, items, stream, a, tb, kThreads)
+                       : launch_after_verify(commit_delta_rows_kernel<false, 4>, items, stream, a, tb, kThreads));
   } else if (a.dk == 64) {
-    if (a.bf16) commit_delta_rows_kernel<true, 2><<<items, kThreads, 0, stream>>>(a, tb);
-    else commit_delta_rows_kernel<false, 2><<<items, kThreads, 0, stream>>>(a, tb);
+    TV_CUDA_TRY(a.bf16 ? launch_after_verify(commit_delta_rows_kernel<true, 2>, items, stream, a, tb, kThreads)
+                       : launch_after_verify(commit_delta_rows_kernel<false, 2>, items, stream, a, tb, kThreads));
   } else {
     return TV_ERR_UNSUPPORTED;
   }

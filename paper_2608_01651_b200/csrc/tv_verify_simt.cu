@@ -19,6 +19,7 @@
 #include <cuda_bf16.h>
 
 #include "tv_internal.h"
+#include "tv_tc_common.cuh"
 
 namespace {
 
@@ -143,6 +144,11 @@ __device__ __forceinline__ void dense_pass(const VerifyArgs& a, const Smem& sm, 
 template <bool BF16, bool DELTA>
 __global__ void __launch_bounds__(kThreads) verify_simt_kernel(VerifyArgs a) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
+  // Dependent launch on both sides: the kernel behind this one may set itself up now (the
+  // library's kernels read nothing this one writes before their own wait); this one reads
+  // nothing -- the tree metadata may come from the kernel in front -- before that kernel is done.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  tvtc::grid_dependency_wait();
   const int dk = a.dk, dv = a.dv;
   const int item = blockIdx.x;
   const ItemRows rows = tv_item_rows(a.tree, a.lay, item, a.B, a.H, a.Hk, a.T, a.dk, a.dv);
@@ -293,8 +299,7 @@ int launch(const VerifyArgs& a, cudaStream_t stream) {
     TV_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     slot = dev;
   }
-  kern<<<a.L * a.B * a.H, kThreads, smem, stream>>>(a);
-  TV_CUDA_TRY(cudaGetLastError());
+  TV_CUDA_TRY(tvtc::launch_dependent(kern, a.L * a.B * a.H, kThreads, smem, stream, a));
   return TV_OK;
 }
 
