@@ -34,7 +34,7 @@
 // stores and the per-item tables (masks, gates) each have a warp of their own.
 // S_pre goes TMA -> shared memory -> tensor core untouched; O and U leave
 // through swizzled staging chunks and TMA stores.  Every wait is a bounded
-// mbarrier wait (status word on expiry); no TMA multicast.
+// mbarrier wait (status word on expiry); every TMA load is a plain per-CTA copy.
 #include "tv_tc_common.cuh"
 
 namespace {

@@ -25,7 +25,7 @@
 // block is read out after the row solve of the next block (of the next item for block 1), when
 // its MMAs are long complete.  Twelve warps: TMA producer, MMA issuer, eight compute warps, one
 // warp that stages the next item's ancestor masks, gates and path tables, one that issues the
-// output stores.  Every wait is a bounded mbarrier wait; no TMA multicast.
+// output stores.  Every wait is a bounded mbarrier wait; every TMA load is a plain per-CTA copy.
 #include "tv_tc_common.cuh"
 
 namespace {
