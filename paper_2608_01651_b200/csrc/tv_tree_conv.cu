@@ -231,12 +231,13 @@ tree_conv_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  // Dependent launches on both sides: the kernel behind this one may set itself up now (the
-  // library's kernels read nothing this one writes before their own wait), and this one has
-  // come this far under the tail of the kernel in front, whose output x may be.
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // Dependent launches on both sides: this kernel has come this far under the tail of the kernel
+  // in front, whose output x may be; the kernel behind it may set itself up from here on (the
+  // library's kernels read nothing this one writes before their own wait).  Dependents are
+  // released after the wait, so that they never run beside anything older than this grid.
   __syncthreads();
   grid_dependency_wait();
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   // An item's coordinates.  The cursor of the item being computed advances without divisions;
   // the warp that requests an item derives that item's coordinates from its number.

@@ -14,13 +14,15 @@ tree_meta_kernel(const int32_t* __restrict__ parent, int32_t n, uint64_t* __rest
                  int32_t depth_bound, int32_t generation) {
   __shared__ int32_t par_s[TV_MAX_NODES];
   const int t = blockIdx.x, i = threadIdx.x;
-  // a verify kernel launched behind this one may be scheduled now and set itself up; it waits
-  // for this grid to finish before it reads global memory
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   // This kernel is itself launched as a dependent of the kernels in front of it.  The parents and
   // offsets may be their output (a forest built on the device), and they may still be reading the
   // metadata of the previous upload: nothing is read or written before they have finished.
   tvtc::grid_dependency_wait();
+  // A kernel launched behind this one may be scheduled now and set itself up; it waits for this
+  // grid to finish before it reads the metadata.  Released only after the wait above, so that a
+  // dependent never runs beside anything older than this grid (the library's kernels read data
+  // that an older kernel may write -- the state -- before their own wait).
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (i < n) {
     // host-built trees are validated there; device-built ones (tv_forest_upload_device) are not:
     // an out-of-range parent is treated as a child of the virtual root so the walk stays in bounds
@@ -80,7 +82,6 @@ tree_meta_param_kernel(const __grid_constant__ ParentBytes<NB> pb, const __grid_
                        int32_t* __restrict__ parent_dev, int32_t* status, int32_t* __restrict__ offsets_dev) {
   __shared__ int32_t par_s[TV_MAX_NODES];
   const int t = blockIdx.x, i = threadIdx.x;
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // as in the kernel above
   if (i < n) par_s[i] = pb.p[t * n + i];
   __syncthreads();
   uint64_t w0 = 0, w1 = 0;
@@ -93,6 +94,7 @@ tree_meta_param_kernel(const __grid_constant__ ParentBytes<NB> pb, const __grid_
   // still be reading the metadata of the previous upload (this kernel is launched as their
   // dependent): nothing is written before they have finished.
   tvtc::grid_dependency_wait();
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // after the wait, as in the kernel above
   if (t == 0 && i == 0) *status = 0;
   if (has_offsets && i == 0) {
     offsets_dev[t] = off.o[t];

@@ -144,11 +144,12 @@ __device__ __forceinline__ void dense_pass(const VerifyArgs& a, const Smem& sm, 
 template <bool BF16, bool DELTA>
 __global__ void __launch_bounds__(kThreads) verify_simt_kernel(VerifyArgs a) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  // Dependent launch on both sides: the kernel behind this one may set itself up now (the
-  // library's kernels read nothing this one writes before their own wait); this one reads
-  // nothing -- the tree metadata may come from the kernel in front -- before that kernel is done.
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // Dependent launch on both sides: this kernel reads nothing -- the tree metadata may come from
+  // the kernel in front -- before that kernel is done; the kernel behind it may set itself up from
+  // then on (the library's kernels read nothing this one writes before their own wait, and a
+  // dependent released after the wait never runs beside anything older than this grid).
   tvtc::grid_dependency_wait();
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int dk = a.dk, dv = a.dv;
   const int item = blockIdx.x;
   const ItemRows rows = tv_item_rows(a.tree, a.lay, item, a.B, a.H, a.Hk, a.T, a.dk, a.dv);

@@ -186,6 +186,38 @@ def test_tc_gated_run_to_run_identical(T, B, H):
     assert torch.isfinite(first).all()
 
 
+def test_in_place_commits_with_only_an_upload_between():
+    """commit (in place) -> tree upload -> commit (in place) on one stream, nothing else and no
+    synchronisation in between.  Every kernel in that chain is a dependent launch, and the commit
+    kernel fetches its state rows before its own wait: the second commit must not be scheduled
+    while the first one still writes those rows (a kernel releases its dependents only after its
+    own wait, so a dependent never runs beside anything older than the kernel in front of it)."""
+    from oracle import tree_oracle as orc
+    wl = inputs.workload("c3", B=32, H=32, T=64, L=1, seed=91)
+    parents, accepted = inputs.make_trees(wl)
+    tens = inputs.make_tensors(wl)
+    t = {k: (None if v is None else v.cuda()) for k, v in tens.items()}
+    acc = torch.from_numpy(np.asarray(accepted, dtype=np.int32)).cuda()
+    tree = tv.tree_build(parents).upload()
+    items = [(0, 0), (7, 31), (19, 5), (31, 31)]
+    f = {k: inputs.to_f64(v) for k, v in tens.items()}
+    once = orc.commit_batch(f["S_pre"], f["k"], f["v"], f["alpha"], None, parents, accepted, wl.rule_name, items=items)
+    S1 = np.array(f["S_pre"], dtype=np.float64, copy=True)
+    for (b, h), Sn in once.items():
+        S1[b, h] = Sn
+    twice = orc.commit_batch(S1, f["k"], f["v"], f["alpha"], None, parents, accepted, wl.rule_name, items=items)
+    for rep in range(6):
+        S = t["S_pre"].clone()
+        torch.cuda.synchronize()
+        tv.commit_path(tree, acc, S, t["k"], t["v"], t["alpha"])
+        tree.upload()
+        tv.commit_path(tree, acc, S, t["k"], t["v"], t["alpha"])
+        torch.cuda.synchronize()
+        Sh = S.cpu().double().numpy()
+        for (b, h), Sr in twice.items():
+            assert pu.rel_fro(Sh[b, h], Sr) <= 1e-5, (rep, b, h)
+
+
 def test_tc_delta_falls_back_on_deep_trees():
     wl = inputs.workload("c4", B=1, H=2, T=40, tree="chain", seed=5)   # depth 39 > 15
     parents, accepted = inputs.make_trees(wl)
