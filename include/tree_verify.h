@@ -303,13 +303,15 @@ int tv_tree_verify_static(const int32_t* parent /*dev*/, int32_t n_trees, const 
  * tv_tree_verify, or NULL -- then TV_GATED uses u_j = v_j and TV_GATED_DELTA
  * re-derives u_j along the accepted path from S_pre (needs dk in {64,128}).
  * S_new may alias S_pre exactly (in place) or not overlap it at all.
- * Stream order: when the call directly follows tv_tree_verify, tv_tree_upload
- * or tv_forest_upload_device on the same stream, the commit grid may be
- * scheduled while that kernel drains and read S_pre and accepted early; it
- * reads the tree metadata and U, and writes S_new, only after that kernel has
- * completed.  (Behind any other work it starts after that work, as usual.)  So
- * accepted and S_pre must not be outputs of the library call in front of it --
- * U and the tree metadata are the only ones that may be.                      */
+ * Stream order: when the call directly follows tv_tree_verify, tv_tree_upload,
+ * tv_forest_upload_device or tv_tree_conv on the same stream, the commit grid
+ * may be scheduled while that kernel drains and read S_pre and accepted early;
+ * it reads the tree metadata and U, and writes S_new, only after that kernel
+ * has completed -- and that kernel lets it start only once everything in front
+ * of itself has completed.  (Behind any other work it starts after that work,
+ * as usual.)  So accepted and S_pre must not be outputs of the library call
+ * directly in front of it -- U and the tree metadata are the only ones that
+ * may be.                                                                     */
 int tv_commit_path(const tv_tree* tree, const tv_dims* dims,
                    const int32_t* accepted /*dev [B]*/,
                    const float* S_pre /*dev*/,
