@@ -1,6 +1,7 @@
-// Device and host helpers shared by the tensor-core verify kernels: mbarrier, TMA,
-// tcgen05 / TMEM wrappers (inline PTX for sm_100a), shared-memory matrix descriptors and
-// tensor-map construction.
+// Device and host helpers shared by the kernels: mbarrier, TMA, tcgen05 / TMEM wrappers (inline
+// PTX for sm_100a), shared-memory matrix descriptors, tensor-map construction, division by launch
+// constants and dependent launches.  The tensor-core verify kernels use all of it; the Stage 1
+// kernel the mbarrier / TMA part; the metadata, SIMT and commit kernels the dependent launch.
 #pragma once
 #include <cuda.h>
 #include <cudaTypedefs.h>
