@@ -248,7 +248,15 @@ int tv_forest_upload_device(tv_tree* forest, const int32_t* parent_padded /*dev*
  * uploaded.  S_pre is read only.  beta may be NULL for TV_GATED.  U may be
  * NULL; when given it receives the correction rows u_i (for TV_GATED a copy of
  * v widened to float).  One asynchronous launch sequence on `stream`; no
- * allocation, no host synchronisation.                                        */
+ * allocation, no host synchronisation.  Stream order: the kernel may be
+ * scheduled while the library kernel directly in front of it on the stream
+ * drains (a tree upload, another tv_tree_verify, tv_tree_conv), and asks for
+ * its first S_pre tile then; everything else it reads after that kernel has
+ * completed.  None of those kernels writes a state, and behind any other work
+ * (tv_commit_path included) the kernel starts after that work, as usual -- a
+ * caller's own kernel that writes S_pre and releases its dependents early
+ * (programmatic dependent launch) is the one thing that must not sit directly
+ * in front of this call.                                                      */
 int tv_tree_verify(const tv_tree* tree, const tv_dims* dims,
                    const float* S_pre /*dev*/,
                    const void* q /*dev*/, const void* k /*dev*/, const void* v /*dev*/,

@@ -352,6 +352,19 @@ verify_tc_gated_kernel(const __grid_constant__ LoadMaps lm, const __grid_constan
       // parked in try_wait
       auto poll = [](uint32_t b, uint32_t parity) { return SMALL ? mbar_test(b, parity) : mbar_try(b, parity); };
       const uint64_t dQ = desc_kmajor(sbase + L::kOffQ), dK = desc_kmajor(sbase + L::kOffK);
+      // The first state tile is requested before the wait: the state is written by commit kernels
+      // and by the caller's own work only, neither of which releases a dependent before it ends, and
+      // the library's kernels that do (metadata, verify, Stage 1) release theirs only after their
+      // own wait -- so whenever this kernel runs, S_pre is complete.  q, k, v and the gates may be
+      // the output of the kernel directly in front (Stage 1) and wait.
+      if (n_it > 0) {
+        mbar_expect_tx(bar(S_FULL0), NC * D * 128);
+#pragma unroll 1
+        for (int c = 0; c < NC; ++c)
+          tma_load_3d(sbase + L::kOffS + (uint32_t)c * kTile, &tmS, bar(S_FULL0), 32 * c, 0, (int)blockIdx.x);
+        pend_s[0] = 1;
+        i_s = 1;
+      }
       grid_dependency_wait();   // inputs may come from the kernel in front (dependent launch)
       long long t_idle = clock64();
       uint32_t spin = 0;
