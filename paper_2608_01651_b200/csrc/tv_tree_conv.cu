@@ -496,6 +496,7 @@ conv_commit_kernel(const int32_t* __restrict__ parent, int32_t n_trees, const in
                    const int32_t* __restrict__ accepted, int32_t T, int32_t C, const IO* x, const IO* ctx,
                    IO* ctx_new) {
   constexpr int VEC = 16 / (int)sizeof(IO);
+  tvtc::grid_dependency_wait();   // dependent launch: nothing is read before the kernel in front is done
   const int b = blockIdx.y;
   const int col = (blockIdx.x * kConvThreads + threadIdx.x) * VEC;
   if (col >= C) return;
@@ -609,9 +610,18 @@ int launch_conv_commit(const tv_tree* t, const tv_conv_dims* d, const int32_t* a
   constexpr int VEC = 16 / (int)sizeof(IO);
   const int C = d->H * (2 * d->dk + d->dv);
   dim3 grid((unsigned)((C / VEC + kConvThreads - 1) / kConvThreads), (unsigned)d->B);
-  conv_commit_kernel<IO, W><<<grid, kConvThreads, 0, s>>>(t->d_parent, t->n_trees, t->d_offsets, accepted, d->T, C,
-                                                         (const IO*)x, (const IO*)ctx, (IO*)ctx_new);
-  TV_CUDA_TRY(cudaGetLastError());
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(kConvThreads);
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  TV_CUDA_TRY(cudaLaunchKernelEx(&cfg, conv_commit_kernel<IO, W>, (const int32_t*)t->d_parent, (int32_t)t->n_trees,
+                                 (const int32_t*)t->d_offsets, accepted, (int32_t)d->T, (int32_t)C, (const IO*)x,
+                                 (const IO*)ctx, (IO*)ctx_new));
   return TV_OK;
 }
 
