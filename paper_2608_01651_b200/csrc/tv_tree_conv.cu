@@ -568,18 +568,42 @@ int launch_conv(const ConvArgs& a_in, cudaStream_t stream) {
   const int C = a.H * (2 * a.dk + a.dv);
   const uint64_t rows = a.offsets ? (uint64_t)a.capacity : (uint64_t)a.B * a.T;
   const CUtensorMapDataType dt = sizeof(IO) == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
-  alignas(64) CUtensorMap map_k, map_v;
-  if (!tvtc::make_map2_plain(&map_k, a.x, dt, sizeof(IO), rows, C, a.dk, a.T) ||
-      !tvtc::make_map2_plain(&map_v, a.x, dt, sizeof(IO), rows, C, a.dv, a.T))
-    return TV_ERR_CUDA;
-  int dev = 0, sms = 0;
+  // A serving loop calls with the same buffers and shapes round after round: the two tensor maps
+  // and what the runtime says about the kernel (SM count, CTAs per SM at this shared-memory size)
+  // are kept per thread for the last call's arguments.
+  struct MapCache {
+    const void* x = nullptr;
+    uint64_t rows = 0;
+    int C = 0, dk = 0, dv = 0, T = 0;
+    alignas(64) CUtensorMap map_k, map_v;
+  };
+  struct LaunchCache {
+    const void* kernel = nullptr;
+    size_t smem = 0;
+    int dev = -1, sms = 0, per_sm = 0;
+  };
+  static thread_local MapCache mc;
+  static thread_local LaunchCache lc;
+  if (mc.x != a.x || mc.rows != rows || mc.C != C || mc.dk != a.dk || mc.dv != a.dv || mc.T != a.T) {
+    mc.x = nullptr;
+    if (!tvtc::make_map2_plain(&mc.map_k, a.x, dt, sizeof(IO), rows, C, a.dk, a.T) ||
+        !tvtc::make_map2_plain(&mc.map_v, a.x, dt, sizeof(IO), rows, C, a.dv, a.T))
+      return TV_ERR_CUDA;
+    mc.x = a.x; mc.rows = rows; mc.C = C; mc.dk = a.dk; mc.dv = a.dv; mc.T = a.T;
+  }
+  const CUtensorMap &map_k = mc.map_k, &map_v = mc.map_v;
+  int dev = 0;
   TV_CUDA_TRY(cudaGetDevice(&dev));
-  TV_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
   auto go = [&](auto kernel) -> int {
-    if (smem > 48 * 1024)
-      TV_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    int per_sm = 0;
-    TV_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kConvThreads, smem));
+    if (lc.kernel != (const void*)kernel || lc.smem != smem || lc.dev != dev) {
+      lc.kernel = nullptr;
+      TV_CUDA_TRY(cudaDeviceGetAttribute(&lc.sms, cudaDevAttrMultiProcessorCount, dev));
+      if (smem > 48 * 1024)
+        TV_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+      TV_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&lc.per_sm, kernel, kConvThreads, smem));
+      lc.kernel = (const void*)kernel; lc.smem = smem; lc.dev = dev;
+    }
+    const int sms = lc.sms, per_sm = lc.per_sm;
     if (per_sm < 1) return TV_ERR_UNSUPPORTED;
     const long long items = 3LL * a.H * a.B, slots = (long long)sms * per_sm;
     const unsigned grid = (unsigned)(items < slots ? items : slots);
