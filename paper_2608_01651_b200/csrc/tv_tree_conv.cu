@@ -8,7 +8,7 @@
 // kernel is bound by instruction issue before it is bound by HBM.  The design therefore spends
 // its effort on instructions per element and on keeping the warps busy: persistent CTAs walk
 // (request, head, q|k|v) slices so that the filter stays in registers; the rows of an item arrive
-// as one TMA box two items ahead and are handed over through mbarriers, so the eight warps of a
+// as one TMA box one or two items ahead and are handed over through mbarriers, so the warps of a
 // CTA never meet at a CTA-wide barrier; each half-warp derives the W tap rows of its own node rows
 // from the parent array; and a half-warp owns a node row (8 channels per lane), so a row's sum of
 // squares is a 4-step shuffle reduction and the row leaves as contiguous 16-byte stores.
@@ -19,12 +19,12 @@
 
 namespace {
 
-// Two CTAs per SM (up to 128 registers, no spills) with the row loop unrolled twice measured
-// faster than three CTAs at 80 registers: the kernel is bound by instruction issue, not by occupancy.
+// Sixteen warps per SM (up to 128 registers, no spills: two CTAs of eight warps, or four of four
+// for trees of up to 64 nodes) with the row loop unrolled twice measured faster than 24 warps at
+// 80 registers.
 constexpr int kConvMinBlocks = 2;
 constexpr int kConvUnroll = 2;
 constexpr int kConvThreads = 256;
-constexpr int kConvWarps = kConvThreads / 32;
 constexpr int kMaxConvDim = 256;
 
 struct ConvArgs {
@@ -171,8 +171,9 @@ __device__ __forceinline__ void cp_async4(uint32_t dst, const void* src) {
 //   4 x ([128 NJ][W] filter taps + [128 NJ] bias) of a slice; every group of 8 channels is shifted
 //   by two words, so that the 16 lanes of a row, which own 8 channels each, read 16 banks,
 //   NS x (full, empty) mbarriers.
-// The eight warps run from item to item without a CTA-wide barrier.  Item n lives in slot n % NS.
-// One warp (n % 8) requests item n + NS - 1 when it has finished item n (NS >= 3; with fewer slots,
+// The NW warps (eight, or four for trees of up to 64 nodes) run from item to item without a
+// CTA-wide barrier.  Item n lives in slot n % NS.
+// One warp (n % NW) requests item n + NS - 1 when it has finished item n (NS >= 3; with fewer slots,
 // before it starts item n): the row box by TMA, parents, context rows and -- when the slice
 // changes -- the filter by cp.async, all arriving on the slot's `full` barrier; before that it
 // waits on the slot's `empty` barrier, on which every warp arrives when it has read the item that
@@ -188,8 +189,8 @@ struct ConvItem {
 
 constexpr long long kConvDrainCycles = 1ll << 21;   // ~1 ms: copies still in flight after a timeout
 
-template <typename IO, int W, int NJ>
-__global__ void __launch_bounds__(kConvThreads, (NJ == 1 && W <= 4) ? kConvMinBlocks : 1)
+template <typename IO, int W, int NJ, int NW>
+__global__ void __launch_bounds__(NW * 32, (NJ == 1 && W <= 4) ? (NW == 4 ? 4 : kConvMinBlocks) : 1)
 tree_conv_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                  const ConvArgs a) {
   using namespace tvtc;
@@ -226,7 +227,7 @@ tree_conv_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
   if (tid == 0) {
     for (int s = 0; s < NS; ++s) {
       mbar_init(full_bar(s), 33);            // the issuing warp: expect_tx by lane 0, cp.async arrivals of 32 lanes
-      mbar_init(empty_bar(s), kConvWarps);
+      mbar_init(empty_bar(s), NW);
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -312,7 +313,7 @@ tree_conv_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
   {
     const int ahead = PD > 0 ? PD : 0;
     for (int m = 0; m < ahead && m < count; ++m)
-      if (warp == (m & (kConvWarps - 1))) issue(m, m, 0);
+      if (warp == (m & (NW - 1))) issue(m, m, 0);
   }
 
   // this thread's gate input of an item (alpha with the q slice, beta with the k slice), loaded
@@ -339,7 +340,7 @@ tree_conv_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
 
   for (; n < count; ++n) {
     if (issue_first && n + PD < count) {
-      if (warp == ((n + PD) & (kConvWarps - 1)) && !issue(n + PD, pre_slot, pre_use)) { ok = false; break; }
+      if (warp == ((n + PD) & (NW - 1)) && !issue(n + PD, pre_slot, pre_use)) { ok = false; break; }
     }
     if (!mbar_wait_warp(full_bar(slot), phase, abort_flag)) { ok = false; break; }
     const int d = cur.d;
@@ -387,7 +388,7 @@ tree_conv_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
     uint32_t mytap[W];
     {
       const int32_t* par = par_s + slot * Tp;
-      int j = 2 * warp + half + 2 * kConvWarps * l16, ctx_row = W - 2;
+      int j = 2 * warp + half + 2 * NW * l16, ctx_row = W - 2;
       if (j >= Tn) j = Tn - 1;   // rows past the end repeat the last one (computed, not stored)
 #pragma unroll
       for (int r = 0; r < W; ++r) {
@@ -413,7 +414,7 @@ tree_conv_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
     }
     int src_lane = lane & 16;
 #pragma unroll kConvUnroll
-    for (int i0 = 2 * warp; i0 < Tn; i0 += 2 * kConvWarps, ++src_lane) {
+    for (int i0 = 2 * warp; i0 < Tn; i0 += 2 * NW, ++src_lane) {
       const bool row_live = i0 + half < Tn;
       const int i = row_live ? i0 + half : Tn - 1;
       uint32_t tap[W];
@@ -455,7 +456,7 @@ tree_conv_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
     if (do_beta) a.beta[cur.orow + tid] = sigmoid_fast(to_f32(gate_raw));
 
     if (!issue_first && n + PD < count) {
-      if (warp == ((n + PD) & (kConvWarps - 1)) && !issue(n + PD, pre_slot, pre_use)) { ok = false; break; }
+      if (warp == ((n + PD) & (NW - 1)) && !issue(n + PD, pre_slot, pre_use)) { ok = false; break; }
     }
     if (++pre_slot == NS) {
       pre_slot = 0;
@@ -562,6 +563,12 @@ int launch_conv(const ConvArgs& a_in, cudaStream_t stream) {
   const size_t half_sm = 112 * 1024, whole_sm = 226 * 1024;
   if (kTwoPerSm && NJ == 1 && smem_for(3) <= half_sm) a.slots = 3;
   else a.slots = smem_for(3) <= whole_sm ? 3 : smem_for(2) <= whole_sm ? 2 : 1;
+  // Up to 64 nodes: CTAs of four warps, four per SM, two slots each.  A warp then takes twice as
+  // many rows of an item, which halves the per-item part of its work (a third of an item at 64
+  // nodes with eight warps): 39.4 -> 37.4 us on B = 32, T = 64 and 84.3 -> 66.1 us on B = 128,
+  // T = 32.  At 128 nodes the four CTAs' slots do not fit.
+  const bool small = kTwoPerSm && NJ == 1 && a.T <= 64 && smem_for(2) <= 55 * 1024;
+  if (small) a.slots = 2;
   const size_t smem = smem_for(a.slots);
   if (smem > whole_sm) return TV_ERR_UNSUPPORTED;
   // x as a [rows][C] tensor; one box = the T node rows of a request x the d channels of a slice
@@ -594,23 +601,24 @@ int launch_conv(const ConvArgs& a_in, cudaStream_t stream) {
   const CUtensorMap &map_k = mc.map_k, &map_v = mc.map_v;
   int dev = 0;
   TV_CUDA_TRY(cudaGetDevice(&dev));
-  auto go = [&](auto kernel) -> int {
+  auto go = [&](auto kernel, int threads) -> int {
     if (lc.kernel != (const void*)kernel || lc.smem != smem || lc.dev != dev) {
       lc.kernel = nullptr;
       TV_CUDA_TRY(cudaDeviceGetAttribute(&lc.sms, cudaDevAttrMultiProcessorCount, dev));
       if (smem > 48 * 1024)
         TV_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-      TV_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&lc.per_sm, kernel, kConvThreads, smem));
+      TV_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&lc.per_sm, kernel, threads, smem));
       lc.kernel = (const void*)kernel; lc.smem = smem; lc.dev = dev;
     }
     const int sms = lc.sms, per_sm = lc.per_sm;
     if (per_sm < 1) return TV_ERR_UNSUPPORTED;
     const long long items = 3LL * a.H * a.B, slots = (long long)sms * per_sm;
     const unsigned grid = (unsigned)(items < slots ? items : slots);
-    TV_CUDA_TRY(tvtc::launch_dependent(kernel, (int)grid, kConvThreads, smem, stream, map_k, map_v, a));
+    TV_CUDA_TRY(tvtc::launch_dependent(kernel, (int)grid, threads, smem, stream, map_k, map_v, a));
     return TV_OK;
   };
-  return NJ == 1 ? go(tree_conv_kernel<IO, W, 1>) : go(tree_conv_kernel<IO, W, 2>);
+  if (small) return go(tree_conv_kernel<IO, W, 1, 4>, 128);
+  return NJ == 1 ? go(tree_conv_kernel<IO, W, 1, 8>, 256) : go(tree_conv_kernel<IO, W, 2, 8>, 256);
 }
 
 template <typename IO>
