@@ -19,10 +19,9 @@
 
 namespace {
 
-// Sixteen warps per SM (up to 128 registers, no spills: two CTAs of eight warps, or four of four
-// for trees of up to 64 nodes) with the row loop unrolled twice measured faster than 24 warps at
-// 80 registers.
-constexpr int kConvMinBlocks = 2;
+// Sixteen warps per SM (up to 128 registers, no spills: two CTAs of eight warps, four of four for
+// trees of up to 64 nodes, eight of two up to 32) with the row loop unrolled twice measured faster
+// than 24 warps at 80 registers.
 constexpr int kConvUnroll = 2;
 constexpr int kConvThreads = 256;
 constexpr int kMaxConvDim = 256;
@@ -168,7 +167,7 @@ __device__ __forceinline__ void cp_async4(uint32_t dst, const void* src) {
 // when the slice changes.  Shared memory:
 //   NS x slot: [T][d] node rows (one TMA box of x) then [W-1][d] context rows, oldest first,
 //   NS x [T] parents,
-//   4 x ([128 NJ][W] filter taps + [128 NJ] bias) of a slice; every group of 8 channels is shifted
+//   4 x ([128 NJ][W] filter taps + [128 NJ] bias) of a slice (3 x in the two-warp CTAs); every group of 8 channels is shifted
 //   by two words, so that the 16 lanes of a row, which own 8 channels each, read 16 banks,
 //   NS x (full, empty) mbarriers.
 // The NW warps (eight, or four for trees of up to 64 nodes) run from item to item without a
@@ -190,7 +189,7 @@ struct ConvItem {
 constexpr long long kConvDrainCycles = 1ll << 21;   // ~1 ms: copies still in flight after a timeout
 
 template <typename IO, int W, int NJ, int NW>
-__global__ void __launch_bounds__(NW * 32, (NJ == 1 && W <= 4) ? (NW == 4 ? 4 : kConvMinBlocks) : 1)
+__global__ void __launch_bounds__(NW * 32, (NJ == 1 && W <= 4) ? 16 / NW : 1)
 tree_conv_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                  const ConvArgs a) {
   using namespace tvtc;
@@ -209,9 +208,11 @@ tree_conv_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
   const uint32_t slot_bytes = ((uint32_t)(T + W - 1) * dmax * sizeof(IO) + 127u) & ~127u;
   const uint32_t xs_u32 = smem_u32(smem_raw);
   const int32_t* par_s = reinterpret_cast<const int32_t*>(smem_raw + (size_t)NS * slot_bytes);   // [NS][Tp]
-  const float* filt_s = reinterpret_cast<const float*>(par_s + NS * Tp);                          // [4][kFiltFloats]
+  // filter buffers: the items in flight (NS <= 3; two with two-warp CTAs) belong to NS slices at most
+  constexpr int NF = NW == 2 ? 3 : 4;
+  const float* filt_s = reinterpret_cast<const float*>(par_s + NS * Tp);                          // [NF][kFiltFloats]
   const uint32_t par_u32 = smem_u32(par_s), filt_u32 = smem_u32(filt_s);
-  const uint32_t bar_u32 = filt_u32 + 4 * kFiltFloats * 4;   // full[NS], empty[NS] (8 bytes each)
+  const uint32_t bar_u32 = filt_u32 + (uint32_t)NF * kFiltFloats * 4;   // full[NS], empty[NS] (8 bytes each)
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_raw + (bar_u32 - xs_u32) + 16 * NS);
   auto full_bar = [&](int s) { return bar_u32 + 8u * s; };
   auto empty_bar = [&](int s) { return bar_u32 + 8u * (NS + s); };
@@ -277,7 +278,7 @@ tree_conv_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
   auto issue = [&](int m, int slot, int use) -> bool {
     if (use > 0 && !mbar_wait_warp(empty_bar(slot), (uint32_t)((use - 1) & 1), abort_flag)) return false;
     const ConvItem it = describe(first + m);
-    const int fc = it.slice - slice_first;   // slice changes since the CTA's first item: filter buffer fc % 4
+    const int fc = it.slice - slice_first;   // slice changes since the CTA's first item: filter buffer fc % NF
     const bool new_filter = m == 0 || it.b == 0;
     const uint32_t dst = xs_u32 + (uint32_t)slot * slot_bytes;
     const uint32_t row_bytes = (uint32_t)it.d * sizeof(IO);
@@ -296,7 +297,7 @@ tree_conv_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
           cp_async16(dst + (uint32_t)(T + r) * row_bytes + cv * 16, cb + (size_t)r * C + cv * VEC);
     }
     if (new_filter) {
-      const uint32_t fdst = filt_u32 + (uint32_t)((fc & 3) * kFiltFloats) * 4;
+      const uint32_t fdst = filt_u32 + (uint32_t)((fc % NF) * kFiltFloats) * 4;
       const float* wsrc = a.weight + (size_t)it.c0 * W;
       for (int c = lane; c < it.d; c += 32) {
         const uint32_t shift = 2 * (c >> 3);
@@ -349,7 +350,7 @@ tree_conv_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
     // ---- this lane's filter taps and bias, when the slice changes
     if (cur.slice != loaded_slice) {
       loaded_slice = cur.slice;
-      const float* wf = filt_s + ((cur.slice - slice_first) & 3) * kFiltFloats;
+      const float* wf = filt_s + ((cur.slice - slice_first) % NF) * kFiltFloats;
       const float* bf = wf + kBiasAt;
 #pragma unroll
       for (int j = 0; j < NJ; ++j) {
@@ -568,8 +569,12 @@ int launch_conv(const ConvArgs& a_in, cudaStream_t stream) {
   // nodes with eight warps): 39.4 -> 37.4 us on B = 32, T = 64 and 84.3 -> 66.1 us on B = 128,
   // T = 32.  At 128 nodes the four CTAs' slots do not fit.
   const bool small = kTwoPerSm && NJ == 1 && a.T <= 64 && smem_for(2) <= 55 * 1024;
+  // up to 32 nodes: CTAs of two warps, eight per SM, by the same argument
+  // (three filter buffers instead of four there: one fewer than smem_for() counts)
+  const size_t filt_bytes = (size_t)(128 * (W + 1) + 64) * 4;
+  const bool tiny = small && a.T <= 32 && smem_for(2) - filt_bytes <= 27 * 1024;
   if (small) a.slots = 2;
-  const size_t smem = smem_for(a.slots);
+  const size_t smem = smem_for(a.slots) - (tiny ? filt_bytes : 0);
   if (smem > whole_sm) return TV_ERR_UNSUPPORTED;
   // x as a [rows][C] tensor; one box = the T node rows of a request x the d channels of a slice
   const int C = a.H * (2 * a.dk + a.dv);
@@ -617,6 +622,7 @@ int launch_conv(const ConvArgs& a_in, cudaStream_t stream) {
     TV_CUDA_TRY(tvtc::launch_dependent(kernel, (int)grid, threads, smem, stream, map_k, map_v, a));
     return TV_OK;
   };
+  if (tiny) return go(tree_conv_kernel<IO, W, 1, 2>, 64);
   if (small) return go(tree_conv_kernel<IO, W, 1, 4>, 128);
   return NJ == 1 ? go(tree_conv_kernel<IO, W, 1, 8>, 256) : go(tree_conv_kernel<IO, W, 2, 8>, 256);
 }
