@@ -103,6 +103,12 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       " [%0], [%1, {%3, %4}], [%2];"
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
 }
+// Untiled bulk copy global -> shared (16-byte aligned on both sides, a multiple of 16 bytes),
+// completing on `bar` like a TMA box.
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
 // The calling thread's earlier cp.async copies arrive on `bar` when they have landed (the arrival
 // is one of the barrier's expected count).
 __device__ __forceinline__ void cp_async_arrive(uint32_t bar) {

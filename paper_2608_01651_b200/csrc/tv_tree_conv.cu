@@ -33,6 +33,7 @@ struct ConvArgs {
   int32_t n_trees;
   int32_t B, H, T, dk, dv, W, normalize;
   int32_t slots;   // row buffers of a CTA (1..3): items requested slots - 1 ahead
+  int32_t par_bulk; // the parents of a tree start on a 16-byte boundary and fill whole 16-byte units
   int32_t* status; // device status word of the tree (a wait that ran out is reported there)
   tvtc::FastDiv dB, dH;   // item -> (slice, request), slice -> (q|k|v, head)
   float eps;
@@ -282,20 +283,23 @@ tree_conv_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
     const bool new_filter = m == 0 || it.b == 0;
     const uint32_t dst = xs_u32 + (uint32_t)slot * slot_bytes;
     const uint32_t row_bytes = (uint32_t)it.d * sizeof(IO);
-    if (lane == 0) {
-      mbar_expect_tx(full_bar(slot), (uint32_t)T * row_bytes);
-      tma_load_2d(dst, it.kind == 2 ? &map_v : &map_k, full_bar(slot), it.c0, it.row0);
-    }
+    // one thread: the row box (TMA), the W - 1 context rows and -- when its rows start on 16-byte
+    // boundaries -- the parents as untiled bulk copies, all counted in bytes on the barrier
     const int32_t* psrc = a.parent + (size_t)(a.n_trees == 1 ? 0 : it.b) * T;
-    for (int i = lane; i < T; i += 32) cp_async4(par_u32 + (uint32_t)(slot * Tp + i) * 4, psrc + i);
-    if (W > 1) {
-      const IO* cb = reinterpret_cast<const IO*>(a.ctx) + (size_t)it.b * (W - 1) * C + it.c0;
-      const int vpr = it.d / VEC;
+    const bool par_bulk = a.par_bulk != 0;
+    if (lane == 0) {
+      mbar_expect_tx(full_bar(slot), (uint32_t)(T + W - 1) * row_bytes + (par_bulk ? (uint32_t)T * 4u : 0u));
+      tma_load_2d(dst, it.kind == 2 ? &map_v : &map_k, full_bar(slot), it.c0, it.row0);
+      if (W > 1) {
+        const IO* cb = reinterpret_cast<const IO*>(a.ctx) + (size_t)it.b * (W - 1) * C + it.c0;
 #pragma unroll
-      for (int r = 0; r < W - 1; ++r)
-        for (int cv = lane; cv < vpr; cv += 32)
-          cp_async16(dst + (uint32_t)(T + r) * row_bytes + cv * 16, cb + (size_t)r * C + cv * VEC);
+        for (int r = 0; r < W - 1; ++r)
+          bulk_load(dst + (uint32_t)(T + r) * row_bytes, cb + (size_t)r * C, row_bytes, full_bar(slot));
+      }
+      if (par_bulk) bulk_load(par_u32 + (uint32_t)(slot * Tp) * 4, psrc, (uint32_t)T * 4u, full_bar(slot));
     }
+    if (!par_bulk)
+      for (int i = lane; i < T; i += 32) cp_async4(par_u32 + (uint32_t)(slot * Tp + i) * 4, psrc + i);
     if (new_filter) {
       const uint32_t fdst = filt_u32 + (uint32_t)((fc % NF) * kFiltFloats) * 4;
       const float* wsrc = a.weight + (size_t)it.c0 * W;
@@ -706,6 +710,7 @@ TV_API int tv_tree_conv(const tv_tree* tree, const tv_conv_dims* d, const void* 
   a.offsets = tree->d_offsets; a.capacity = tree->capacity;
   a.B = d->B; a.H = d->H; a.T = d->T; a.dk = d->dk; a.dv = d->dv; a.W = d->W;
   a.normalize = d->normalize_qk != 0; a.eps = d->eps; a.slots = 0; a.status = tree->d_status;
+  a.par_bulk = (d->T % 4 == 0) && aligned16(tree->d_parent);
   a.dB = tvtc::make_fastdiv((uint32_t)d->B); a.dH = tvtc::make_fastdiv((uint32_t)d->H);
   a.x = x; a.ctx = ctx; a.weight = weight; a.bias = bias; a.gate_a = gate_a; a.gate_b = gate_b;
   a.A_log = A_log; a.dt_bias = dt_bias; a.q = q; a.k = k; a.v = v; a.alpha = alpha; a.beta = beta;
