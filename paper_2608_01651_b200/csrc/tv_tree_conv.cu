@@ -174,8 +174,9 @@ __device__ __forceinline__ void cp_async4(uint32_t dst, const void* src) {
 // The NW warps (eight, or four for trees of up to 64 nodes) run from item to item without a
 // CTA-wide barrier.  Item n lives in slot n % NS.
 // One warp (n % NW) requests item n + NS - 1 when it has finished item n (NS >= 3; with fewer slots,
-// before it starts item n): the row box by TMA, parents, context rows and -- when the slice
-// changes -- the filter by cp.async, all arriving on the slot's `full` barrier; before that it
+// before it starts item n): the row box by TMA, the context rows and the parents by untiled bulk
+// copies (unaligned parents and, when the slice changes, the filter by cp.async), all arriving on
+// the slot's `full` barrier; before that it
 // waits on the slot's `empty` barrier, on which every warp arrives when it has read the item that
 // lived there.  Each half-warp derives the tap rows of the node rows it owns itself (lane k walks
 // the parents of the half-warp's k-th row once per item; the row loop fetches them by shuffle),
